@@ -1,0 +1,277 @@
+"""Float64 CPU oracle for the Trainable Weight Averaging (TWA) subspace path.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain statement of what the
+method computes.  It shares no code with the CUDA library, is never imported by
+it, and must only be used by the tests, by the smoke check and by the CPU
+baseline timing of the benchmark.  Nothing here is tuned.
+
+Conventions
+-----------
+* A matrix of n vectors in R^D is a 2-D numpy array of shape (D, n): column j is
+  vector j, as in the paper's P = [e_1, ..., e_n] (Section 4.2).  Any strides
+  are accepted; passing ``arr.T`` of an (n, D) C-ordered array makes every
+  column contiguous.
+* Inputs carry the bytes the GPU sees (float32 candidates, float32 or widened
+  bfloat16 gradients, int8 code values, float32 scales); all arithmetic widens
+  them to float64 first.
+* The paper writes beta for the coefficients on the basis vectors; the code
+  calls them ``alpha`` like the library's interface does.
+
+Every function is pinned by tests/test_oracle_*.py against closed forms,
+library factorizations, brute force and the invariants the method fixes; no
+function here is "parity unpinned".
+"""
+
+from __future__ import annotations
+
+import numpy as np
+
+QMAX = {8: 127, 4: 7}
+
+
+# --------------------------------------------------------------------------- #
+# Subspace construction
+# --------------------------------------------------------------------------- #
+def mean(W):
+    """Centre point of the candidates, w_bar = (1/n) sum_i w_i.
+
+    Section 4.1, the subspace-construction equation; Algorithm 1; Section 4.3
+    uses it as the initial point w^(0).
+    Summation runs over i in index order in float64.
+    """
+    W = np.asarray(W)
+    D, n = W.shape
+    acc = np.zeros(D, dtype=np.float64)
+    for i in range(n):
+        acc += W[:, i].astype(np.float64)
+    return acc / float(n)
+
+
+def cgs2(A, rel_tol=1e-10):
+    """Schmidt orthogonalisation of the raw candidates, one vector after the
+    other (Section 4.1, the paragraph on orthogonalising {w_i}), in the
+    classical Gram-Schmidt form with one re-orthogonalisation ("CGS2").
+
+    For j = 0..n-1:  v <- a_j;  exactly twice:  c_k = <q_k, v> for every k < j
+    computed from the SAME v (classical, not modified), then
+    v <- v - sum_k c_k q_k;  r_jj = ||v||_2;  q_j = v / r_jj.
+
+    Returns (Q, R, deficient): Q is (D, n) float64 with orthonormal columns,
+    R is the (n, n) upper-triangular factor with positive diagonal (A = Q R),
+    deficient is None, or the index of the first column whose remainder
+    satisfies r_jj <= rel_tol * ||a_j||_2 (columns from there on are left 0).
+    """
+    A = np.asarray(A)
+    D, n = A.shape
+    Q = np.zeros((D, n), dtype=np.float64, order="F")
+    R = np.zeros((n, n), dtype=np.float64)
+    for j in range(n):
+        a = A[:, j].astype(np.float64)
+        a_norm = float(np.sqrt(np.dot(a, a)))
+        v = a.copy()
+        for _pass in range(2):
+            if j > 0:
+                c = Q[:, :j].T @ v          # all coefficients from the same v
+                v = v - Q[:, :j] @ c
+                R[:j, j] += c
+        r_jj = float(np.sqrt(np.dot(v, v)))
+        if not (r_jj > rel_tol * a_norm):
+            return Q, R, j
+        R[j, j] = r_jj
+        Q[:, j] = v / r_jj
+    return Q, R, None
+
+
+# --------------------------------------------------------------------------- #
+# Low-bit storage of the projection matrix: per-column absmax, symmetric
+# --------------------------------------------------------------------------- #
+def absmax_scales(P32, bits):
+    """Per-column scale s_j = fl32(max_r |P[r, j]| / qmax), qmax = 2^(bits-1)-1.
+
+    This is the symmetric, per-column variant of the uniform quantiser of
+    Section 4.6 (one factor per column instead of the paper's two per layer).
+    Returns (scales float32 (n,), absmax float32 (n,)).
+    """
+    qmax = QMAX[bits]
+    P32 = np.asarray(P32)
+    assert P32.dtype == np.float32
+    n = P32.shape[1]
+    m = np.zeros(n, dtype=np.float32)
+    for j in range(n):
+        col = P32[:, j]
+        m[j] = np.max(np.abs(col)) if col.size else np.float32(0)
+    s = (m.astype(np.float64) / float(qmax)).astype(np.float32)
+    return s, m
+
+
+def encode(P32, scales, bits):
+    """Codes for given scales: code = clamp(round_half_even(fl32(p / s_j)),
+    -qmax, +qmax); a column with s_j == 0 is all zeros.
+
+    The quotient is formed in float64 from the float32 operands and rounded
+    once to float32, which equals the IEEE float32 division; rounding to the
+    integer is ties-to-even (Section 4.6 leaves the rounding mode open).
+    Returns an int8 array of shape (D, n) holding the code VALUES (also for
+    bits == 4; packing is a separate step).
+    """
+    qmax = QMAX[bits]
+    P32 = np.asarray(P32)
+    assert P32.dtype == np.float32
+    D, n = P32.shape
+    codes = np.zeros((D, n), dtype=np.int8, order="F")
+    for j in range(n):
+        s = np.float32(scales[j])
+        if s == 0:
+            continue
+        t = (P32[:, j].astype(np.float64) / np.float64(s)).astype(np.float32)
+        q = np.rint(t)                      # numpy rint: ties to even
+        q = np.clip(q, -qmax, qmax)
+        codes[:, j] = q.astype(np.int8)
+    return codes
+
+
+def quantize(P32, bits):
+    """Whole quantiser: scales from the column absmax, then codes."""
+    s, _ = absmax_scales(P32, bits)
+    return encode(P32, s, bits), s
+
+
+def pack_codes(codes, bits):
+    """Canonical byte image of the codes, one row of bytes per column.
+
+    bits == 8: byte r of column j is code[r, j] (two's complement).
+    bits == 4: byte k of column j holds row 2k in its low nibble and row 2k+1
+    in its high nibble, both as two's-complement nibbles; an odd D leaves the
+    last high nibble 0.  Returns uint8 of shape (n, ceil(D*bits/8)).
+    """
+    codes = np.asarray(codes)
+    D, n = codes.shape
+    if bits == 8:
+        return np.ascontiguousarray(codes.T).view(np.uint8).copy()
+    assert bits == 4
+    nb = (D + 1) // 2
+    out = np.zeros((n, nb), dtype=np.uint8)
+    for j in range(n):
+        col = codes[:, j].astype(np.int16)
+        nib = (col & 0xF).astype(np.uint8)
+        lo = nib[0::2]
+        hi = nib[1::2]
+        out[j, : lo.size] = lo
+        out[j, : hi.size] |= (hi << 4).astype(np.uint8)
+    return out
+
+
+def unpack_codes(packed, D, bits):
+    """Inverse of pack_codes: (n, bytes) uint8 -> int8 code values (D, n)."""
+    packed = np.asarray(packed, dtype=np.uint8)
+    n = packed.shape[0]
+    if bits == 8:
+        return np.asfortranarray(packed.view(np.int8)[:, :D].T)
+    assert bits == 4
+    codes = np.zeros((D, n), dtype=np.int8, order="F")
+    for j in range(n):
+        b = packed[j].astype(np.int16)
+        lo = b & 0xF
+        hi = (b >> 4) & 0xF
+        lo = np.where(lo >= 8, lo - 16, lo)
+        hi = np.where(hi >= 8, hi - 16, hi)
+        inter = np.empty(2 * b.size, dtype=np.int16)
+        inter[0::2] = lo
+        inter[1::2] = hi
+        codes[:, j] = inter[:D].astype(np.int8)
+    return codes
+
+
+def storage_bytes(D, n, bits):
+    """Bytes of the stored projection matrix in this per-column format:
+    n columns of ceil(D*bits/8) code bytes plus one float32 scale per column
+    (bits == 32: plain float32, 4nD).  Mirrors the accounting of the table
+    "memory_projection" (Section 4.6): 4nD against nBD/8 plus the factors."""
+    if bits == 32:
+        return 4 * n * D
+    return n * ((D * bits + 7) // 8) + 4 * n
+
+
+def paper_storage_bytes(D, n, bits, L=1, k=1):
+    """The table "memory_projection" of Section 4.6 as printed: 4*ceil(n/k)*D
+    bytes at 32 bits, ceil(n/k)*B*D/8 + 8L bytes at B bits."""
+    cols = -(-n // k)
+    if bits == 32:
+        return 4 * cols * D
+    return cols * bits * D / 8 + 8 * L
+
+
+# --------------------------------------------------------------------------- #
+# Subspace step
+# --------------------------------------------------------------------------- #
+def project(codes, scales, g):
+    """Coefficient gradient c = P~^T g with P~[r, j] = s_j * code[r, j]
+    (Section 4.2, the chain-rule equation; Algorithm 1, the update of the
+    variables).  c_j = s_j * sum_r code[r, j] * g[r], all in float64."""
+    codes = np.asarray(codes)
+    g64 = np.asarray(g).astype(np.float64)
+    n = codes.shape[1]
+    c = np.zeros(n, dtype=np.float64)
+    for j in range(n):
+        c[j] = np.float64(scales[j]) * np.dot(codes[:, j].astype(np.float64), g64)
+    return c
+
+
+def project_f32(P32, g):
+    """c = P^T g for an unquantised float32 basis, in float64."""
+    P32 = np.asarray(P32)
+    g64 = np.asarray(g).astype(np.float64)
+    n = P32.shape[1]
+    c = np.zeros(n, dtype=np.float64)
+    for j in range(n):
+        c[j] = np.dot(P32[:, j].astype(np.float64), g64)
+    return c
+
+
+def sgd_update(alpha, c, lr, lam=0.0):
+    """alpha <- (1 - lr*lam) * alpha - lr * c  (the gradient-descent update rule
+    of Section 4.2; Algorithm 1 writes it with the factor (1 - eta*lambda))."""
+    alpha = np.asarray(alpha, dtype=np.float64)
+    c = np.asarray(c, dtype=np.float64)
+    return (1.0 - float(lr) * float(lam)) * alpha - float(lr) * c
+
+
+def lift(codes, scales, alpha, base=None):
+    """w = base + P~ alpha (Section 4.3: w_twa = w_bar + P beta; Algorithm 1,
+    the update of the weights).  base None means 0.
+    w[r] = base[r] + sum_j (s_j * alpha_j) * code[r, j], in float64."""
+    codes = np.asarray(codes)
+    D, n = codes.shape
+    w = np.zeros(D, dtype=np.float64) if base is None else np.asarray(base).astype(np.float64).copy()
+    for j in range(n):
+        a = np.float64(scales[j]) * np.float64(alpha[j])
+        w += a * codes[:, j].astype(np.float64)
+    return w
+
+
+def lift_f32(P32, alpha, base=None):
+    """w = base + P alpha for an unquantised float32 basis, in float64."""
+    P32 = np.asarray(P32)
+    D, n = P32.shape
+    w = np.zeros(D, dtype=np.float64) if base is None else np.asarray(base).astype(np.float64).copy()
+    for j in range(n):
+        w += np.float64(alpha[j]) * P32[:, j].astype(np.float64)
+    return w
+
+
+def step(codes, scales, g, alpha, wbar, lr, lam=0.0):
+    """One iteration of the loop body of Algorithm 1: project the gradient,
+    update the coefficients, rebuild the weights from w_bar.
+    Returns (alpha_new, w_new, c)."""
+    c = project(codes, scales, g)
+    alpha_new = sgd_update(alpha, c, lr, lam)
+    w_new = lift(codes, scales, alpha_new, wbar)
+    return alpha_new, w_new, c
+
+
+def step_f32(P32, g, alpha, wbar, lr, lam=0.0):
+    """Same iteration with an unquantised float32 basis."""
+    c = project_f32(P32, g)
+    alpha_new = sgd_update(alpha, c, lr, lam)
+    w_new = lift_f32(P32, alpha_new, wbar)
+    return alpha_new, w_new, c
