@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the TWA subspace step on B200.
+
+One "step" is one fused subspace iteration (project the gradient, update the
+coefficients, lift the weights) through the C-ABI call twa_step on a basis built and
+quantised by the library from synthetic correlated candidates; the basis build and the
+quantisation are timed once and reported beside the step throughput.
+
+    python bench.py --gpus N --steps K --warmup W [--workload vitb16] [--bits 8]
+    python bench.py --impl reference ...     # the float64 CPU oracle on a bounded sample
+
+Prints one JSON line (rank 0).  With N > 1 every rank runs an independent replica of the
+workload on its own GPU (the path has no exchange step); value is the sum over ranks.
+"""
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "twa_fused_step_GBps_int8"
+UNIT = "GB/s"
+
+
+def step_bytes(D, n, bits, g_bytes):
+    """Algorithmic bytes of one fused step: P~ read by the projection and again by the lift,
+    g read once, w_bar read once, w written once."""
+    p = n * ((D * bits + 7) // 8)
+    return 2 * p + D * g_bytes + 4 * D + 4 * D
+
+
+def kernel_bytes(D, n, bits, g_bytes):
+    p = n * ((D * bits + 7) // 8)
+    return {"project": p + D * g_bytes, "lift": p + 8 * D}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi samples of one GPU's clocks and throttle reasons while a region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 8:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[4:8]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def oracle_sample_run(wl, bits, sample_rows, steps, warmup):
+    """The float64 oracle's fused step on the first `sample_rows` rows of the workload
+    (candidates -> float32 basis by the oracle's CGS2 is NOT timed; only the step is)."""
+    import numpy as np
+    import torch
+    from oracle import twa_oracle as orc
+    from paper_2205_13104_b200 import inputs
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        cores = 1
+    D, n = sample_rows, wl.n
+    rng = np.random.default_rng(0)
+    # a random orthonormal-scale basis is enough for timing: the oracle's cost does not depend on values
+    P32 = (rng.standard_normal((n, D)) / np.sqrt(D)).astype(np.float32).T
+    codes, s = orc.quantize(P32, bits)
+    wbar = rng.standard_normal(D).astype(np.float32)
+    alpha = np.zeros(n)
+    gdt = torch.bfloat16 if wl.g_dtype == "bf16" else torch.float32
+    times = []
+    for t in range(warmup + steps):
+        g = inputs.gradient(D, wl.g_std, wl.seed, t, gdt, "cpu").float().numpy()
+        t0 = time.perf_counter()
+        alpha, w, c = orc.step(codes, s, g, alpha, wbar, 0.1, 0.0)
+        dt = time.perf_counter() - t0
+        if t >= warmup:
+            times.append(dt)
+    g_bytes = 2 if wl.g_dtype == "bf16" else 4
+    gbps = step_bytes(D, n, bits, g_bytes) / (sum(times) / len(times)) / 1e9
+    return gbps, cores, sum(times) / len(times)
+
+
+def run_reference(args):
+    from paper_2205_13104_b200 import inputs
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = inputs.WORKLOADS[args.workload]
+    sample_rows = min(wl.D, args.reference_rows)
+    gbps, cores, sec = oracle_sample_run(wl, args.bits, sample_rows, args.steps, args.warmup)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbps, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3 * wl.D / sample_rows,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": f"{wl.name}: D={wl.D} n={wl.n} int{args.bits} P, {wl.g_dtype} g",
+                   "sample": f"first {sample_rows} rows of D; ms_per_step scaled to full D"},
+        "cpu_baseline": {"value": gbps, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"fused step on the first {sample_rows} of {wl.D} rows, all {wl.n} columns"},
+        "e2e": {"value": gbps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2205_13104_b200 import inputs, twa
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    twa.load()
+    wl = inputs.WORKLOADS[args.workload]
+    D, n, bits = wl.D, wl.n, args.bits
+    gdt = torch.bfloat16 if wl.g_dtype == "bf16" else torch.float32
+    g_bytes = 2 if wl.g_dtype == "bf16" else 4
+    ctx = twa.twa_create(local)
+    ws = twa.new_workspace(dev)
+
+    # ---- basis build and quantisation, timed once each -------------------------------
+    W = wl.candidates(dev, ld=inputs.padded_ld(D, 128))
+    wbar = torch.empty(D, dtype=torch.float32, device=dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    torch.cuda.synchronize()
+    ev[0].record()
+    P32 = twa.twa_build_basis(ctx, W, D, wbar, ws)
+    ev[1].record()
+    Pq = twa.twa_quantize_basis(ctx, P32, bits, ws) if bits != 32 else P32
+    ev[2].record()
+    torch.cuda.synchronize()
+    build_ms, quant_ms = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
+    code, detail = twa.twa_get_status(ctx)
+    if code != 0:
+        raise RuntimeError(f"basis build failed: {twa.twa_strerror(code)} column {detail}")
+    if bits != 32:
+        del W, P32
+        torch.cuda.empty_cache()
+
+    # ---- per-step inputs: a pool of distinct gradients, cycled ------------------------
+    pool = [wl.gradient(t, dev) for t in range(args.g_pool)]
+    alpha = torch.zeros(n, dtype=torch.float32, device=dev)
+    w = torch.empty(D, dtype=torch.float32, device=dev)
+    lr, lam = 0.1, 0.0
+
+    def step(t):
+        twa.twa_step(ctx, Pq, pool[t % len(pool)], lr, lam, alpha, wbar, w, ws)
+
+    for t in range(args.warmup):
+        step(t)
+    barrier()
+    twa.twa_profile_enable(ctx, args.steps)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for t in range(args.steps):
+        step(args.warmup + t)
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = e0.elapsed_time(e1)
+    proj_ms, lift_ms, rec = twa.twa_profile_read(ctx)
+    twa.twa_profile_enable(ctx, 0)
+    code, detail = twa.twa_get_status(ctx)
+    if code != 0:
+        raise RuntimeError(f"step failed: {twa.twa_strerror(code)}")
+
+    # ---- end to end: gradient from pinned host memory, weights back to the host --------
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    g_host = [p.cpu().pin_memory() for p in pool[:2]]
+    w_host = torch.empty(D, dtype=torch.float32).pin_memory()
+    g_stage = torch.empty(D, dtype=gdt, device=dev)
+    alpha2 = torch.zeros(n, dtype=torch.float32, device=dev)
+    for t in range(2):
+        twa.twa_step_host(ctx, Pq, g_host[t % 2], lr, lam, alpha2, wbar, w, w_host, g_stage, ws)
+    barrier()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for t in range(e2e_steps):
+        twa.twa_step_host(ctx, Pq, g_host[t % 2], lr, lam, alpha2, wbar, w, w_host, g_stage, ws)
+    t1.record()
+    barrier()
+    e2e_ms = t0.elapsed_time(t1) / e2e_steps
+
+    # ---- max over ranks ------------------------------------------------------------------
+    stats = torch.tensor([total_ms, e2e_ms, proj_ms, lift_ms, build_ms, quant_ms],
+                         dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms, proj_ms, lift_ms, build_ms, quant_ms = stats.tolist()
+
+    if rank == 0:
+        peak, peak_kind = load_peaks()
+        sb = step_bytes(D, n, bits, g_bytes)
+        kb = kernel_bytes(D, n, bits, g_bytes)
+        ms_per_step = total_ms / args.steps
+        value = world * sb / (ms_per_step * 1e-3) / 1e9
+        dom = "project" if proj_ms >= lift_ms else "lift"
+        dom_ms = (proj_ms if dom == "project" else lift_ms) / max(rec, 1)
+        achieved = kb[dom] / (dom_ms * 1e-3) / 1e9
+        other = "lift" if dom == "project" else "project"
+        other_ms = (lift_ms if dom == "project" else proj_ms) / max(rec, 1)
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "traffic.json")
+        if os.path.exists(tpath):
+            with open(tpath) as f:
+                tj = json.load(f)
+            key = f"{wl.name}_int{bits}_{dom}"
+            traffic = tj.get(key)
+        # CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            rows = min(D, args.reference_rows)
+            gbps, cores, sec = oracle_sample_run(wl, bits if bits != 32 else 8, rows, 2, 1)
+            cpu = {"value": gbps, "unit": UNIT, "cores": cores, "kind": "oracle",
+                   "sample": f"fused step on the first {rows} of {D} rows, all {n} columns, 2 timed steps"}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{wl.name}: D={D} n={n} int{bits} P, {wl.g_dtype} g, lr={lr} lambda={lam}",
+                       "l2": f"inputs larger than L2: P~ is {n * ((D * bits + 7) // 8) / 1e6:.0f} MB per pass",
+                       "gradients": f"{len(pool)} distinct gradients generated before the timed region, cycled",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "bytes_per_step": sb,
+            "frac_of_hbm_peak": value / world / peak,
+            "frac_of_8TBps": value / world / 8000.0,
+            "basis_build_ms": build_ms, "quantize_ms": quant_ms,
+            "roofline": {"bound": "hbm", "kernel": f"twa_{dom}_kernel", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                         "traffic": traffic, "bytes_per_launch": kb[dom], "ms_per_launch": dom_ms,
+                         "other_kernel": {"kernel": f"twa_{other}_kernel", "ms_per_launch": other_ms,
+                                          "achieved": kb[other] / (other_ms * 1e-3) / 1e9,
+                                          "bytes_per_launch": kb[other]}},
+            "cpu_baseline": cpu,
+            "e2e": {"value": world * sb / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+                    "ms_per_step": e2e_ms, "steps": e2e_steps,
+                    "h2d_bytes_per_step": D * g_bytes, "d2h_bytes_per_step": 4 * D},
+            "gpu_launches": 2 * args.steps,
+            "clocks": clocks,
+        }
+        print(json.dumps(line))
+    twa.twa_destroy(ctx)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="vitb16")
+    ap.add_argument("--bits", type=int, default=8, choices=[32, 8, 4])
+    ap.add_argument("--g-pool", type=int, default=8)
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--reference-rows", type=int, default=1 << 21)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

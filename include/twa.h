@@ -1,0 +1,203 @@
+/*
+ * twa.h -- C ABI of the B200 (sm_100a) library for the subspace step of
+ * Trainable Weight Averaging (TWA, arXiv 2205.13104).
+ *
+ * What the library computes (paper's notation, with the coefficients on the
+ * basis vectors called alpha here instead of beta):
+ *
+ *   build      w_bar = (1/n) sum_i w_i                       Section 4.1, Algorithm 1
+ *              P = [e_1 .. e_n], orthonormal, span P = span{w_i}
+ *                                                            Section 4.1 (Schmidt
+ *                                                            orthogonalisation of {w_i})
+ *   quantise   P~ = low-bit codes of P plus scale factors    Section 4.6
+ *   project    c = P~^T g                                    Section 4.2 (chain rule)
+ *   update     alpha <- (1 - eta*lambda) alpha - eta c       Section 4.2, Algorithm 1
+ *   lift       w = w_bar + P~ alpha                          Section 4.3, Algorithm 1
+ *
+ * General rules
+ *  - Every pointer is a DEVICE pointer on the context's device unless its
+ *    comment says "host".  The caller owns every buffer; the library
+ *    allocates a few hundred bytes per context and nothing else.
+ *  - Matrices are column-major: column j of a D x n matrix starts at
+ *    data + j * col_stride (bytes).  Vectors are contiguous.
+ *  - Alignment: data pointers of matrices, g, base, w and workspaces must be
+ *    16-byte aligned; col_stride must be a multiple of 16 bytes.
+ *  - Limits: 1 <= n <= TWA_MAX_N, 1 <= D < 2^31.
+ *  - Calls enqueue work on the context's stream and return without waiting
+ *    for it.  Return value 0 = enqueued; a negative TWA_ERR_* = rejected on
+ *    the host, nothing enqueued.  Errors found on the device (non-finite
+ *    input, rank deficiency, a wait that ran out) are recorded in the
+ *    context's status word and read with twa_get_status(), which
+ *    synchronises the stream.  After a device-side error the outputs of that
+ *    call are unspecified.
+ *  - One context per stream; calls on one context must not overlap in time
+ *    from several host threads.
+ *  - Results are run-to-run bit-identical for fixed arguments on one device
+ *    model: every reduction is combined in a fixed order, no floating-point
+ *    atomics are used.
+ */
+#ifndef TWA_H_
+#define TWA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TWA_MAX_N 128
+
+enum {
+  TWA_OK = 0,
+  TWA_ERR_INVALID_ARG = -1,    /* null pointer, size out of range                        */
+  TWA_ERR_MISALIGNED = -2,     /* pointer or stride not 16-byte aligned                  */
+  TWA_ERR_UNSUPPORTED = -3,    /* bits not in {32, 8, 4}, n > TWA_MAX_N, wrong device    */
+  TWA_ERR_RANK_DEFICIENT = -4, /* device: candidate `detail` lies in the span of earlier */
+  TWA_ERR_NONFINITE = -5,      /* device: NaN/Inf met in column `detail`                 */
+  TWA_ERR_TIMEOUT = -6,        /* device: a bounded wait inside a kernel ran out         */
+  TWA_ERR_CUDA = -7,           /* a CUDA runtime/driver call failed (twa_last_error)     */
+  TWA_ERR_WORKSPACE = -8       /* workspace missing or smaller than twa_workspace_bytes  */
+};
+
+typedef enum { TWA_F32 = 0, TWA_BF16 = 1 } twa_dtype;
+
+typedef struct twa_ctx twa_ctx;
+
+/* Descriptor of a projection matrix P (D x n), held by the caller.
+ *  bits == 32: data holds float32 values.
+ *  bits == 8 : one byte per element, value = code + 128 (offset binary), code in [-127,127].
+ *  bits == 4 : two elements per byte, row 2k in the low nibble and row 2k+1 in the high
+ *              nibble, nibble = code + 8, code in [-7,7].
+ *  The represented value is scales[j] * code (Section 4.6, with one symmetric factor per
+ *  column instead of two per layer).  The storage of codes is internal to the library;
+ *  twa_basis_export / twa_basis_import convert to and from the canonical two's-complement
+ *  image.  Bytes of a column beyond ceil(D*bits/8) up to col_stride are padding. */
+typedef struct {
+  void* data;         /* device, 16-byte aligned, n * col_stride bytes                 */
+  float* scales;      /* device, n floats; ignored when bits == 32                     */
+  int64_t D;          /* rows                                                          */
+  int64_t col_stride; /* bytes between consecutive columns, multiple of 16             */
+  int32_t n;          /* columns                                                       */
+  int32_t bits;       /* 32, 8 or 4                                                    */
+} twa_basis;
+
+/* ---- context ------------------------------------------------------------------------ */
+
+/* Creates a context bound to CUDA device `device` and to `cuda_stream` (a cudaStream_t
+ * passed as void*, NULL = the legacy default stream).  Allocates the device status word.
+ * Must not be called while the stream is being captured. */
+int twa_create(twa_ctx** out, int device, void* cuda_stream);
+void twa_destroy(twa_ctx* ctx);
+
+/* Reads and keeps the first device-side error since the last twa_clear_status.  Waits for
+ * the stream.  *code is TWA_OK or a TWA_ERR_*, *detail the offending column or -1. */
+int twa_get_status(twa_ctx* ctx, int* code, int* detail);
+int twa_clear_status(twa_ctx* ctx);
+const char* twa_strerror(int code);
+/* Host string describing the last failed CUDA call of this context ("" if none). */
+const char* twa_last_error(const twa_ctx* ctx);
+
+/* Tuning knobs for measurements; value 0 restores the built-in choice.
+ *  TWA_TUNE_PROJECT_WARPS / TWA_TUNE_LIFT_WARPS: consumer warps per block (8..20; lift: even, >= 16)
+ *  TWA_TUNE_STAGES: depth of the shared-memory ring (2..16)
+ *  TWA_TUNE_WAIT_LIMIT_MS: bound of every in-kernel wait (default 2000 ms)             */
+enum { TWA_TUNE_PROJECT_WARPS = 1, TWA_TUNE_LIFT_WARPS = 2, TWA_TUNE_STAGES = 3,
+       TWA_TUNE_WAIT_LIMIT_MS = 4 };
+int twa_set_tuning(twa_ctx* ctx, int key, int value);
+
+/* Per-kernel timing of twa_step for measurements.  twa_profile_enable(ctx, max_steps > 0)
+ * creates CUDA events; from then on each twa_step records three of them (before the
+ * projection kernel, between the two kernels, after the lift kernel) until max_steps steps
+ * were recorded.  twa_profile_read waits for the stream, returns the summed durations in
+ * milliseconds and the number of steps they cover, and starts a new series.
+ * twa_profile_enable(ctx, 0) destroys the events. */
+int twa_profile_enable(twa_ctx* ctx, int max_steps);
+int twa_profile_read(twa_ctx* ctx, double* project_ms, double* lift_ms, int* steps);
+
+/* ---- sizes -------------------------------------------------------------------------- */
+
+/* Bytes between columns the library uses for a D-row basis of the given width
+ * (ceil(D*bits/8) rounded up to 128). */
+int64_t twa_basis_col_stride(int64_t D, int bits);
+/* n * twa_basis_col_stride: size of the `data` buffer the caller must provide. */
+size_t twa_basis_bytes(int64_t D, int n, int bits);
+/* Size of the scratch buffer `ws` every call below takes (device, 16-byte aligned).  Its
+ * contents need no initialisation and carry nothing between calls. */
+size_t twa_workspace_bytes(int64_t D, int n, int bits);
+
+/* ---- subspace construction (Section 4.1; Algorithm 1) ------------------------------- */
+
+/* w_bar and the orthonormal basis of the n candidates.
+ *  W        in/out: D x n float32 candidates, column i = w_i, column stride ldw ELEMENTS
+ *           (ldw >= D, ldw % 4 == 0).  Overwritten by the basis: on return column j holds
+ *           e_j, obtained by classical Gram-Schmidt with one re-orthogonalisation, column
+ *           after column in the given order, each normalised to unit length.
+ *  wbar_out out: D floats, the mean of the candidates (written before W is overwritten).
+ *  P32_out  out (host struct): filled with {W, NULL, D, 4*ldw, n, 32}.
+ * Device-side errors: TWA_ERR_NONFINITE, TWA_ERR_RANK_DEFICIENT (a column whose remainder
+ * is below 1e-5 of its length; that column is set to zero). */
+int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float* wbar_out,
+                    twa_basis* P32_out, void* ws, size_t ws_bytes);
+
+/* Mean only: wbar_out[r] = (1/n) sum_i W[r, i]. */
+int twa_mean(twa_ctx* ctx, const float* W, int64_t D, int n, int64_t ldw, float* wbar_out);
+
+/* ---- low-bit storage (Section 4.6, per-column symmetric variant) -------------------- */
+
+/* Quantises a float32 basis.  For every column: s_j = absmax_j / qmax (IEEE float32
+ * division), qmax = 127 (bits 8) or 7 (bits 4); code = clamp(rint(P[r,j] / s_j), -qmax,
+ * qmax) with round-half-to-even; an all-zero column gets s_j = 0 and codes 0.
+ *  P32  in: descriptor with bits == 32.
+ *  Pq   in/out (host struct): the caller sets Pq->data (twa_basis_bytes(D, n, bits) bytes)
+ *       and Pq->scales (n floats); the call fills D, col_stride, n, bits and the buffers.
+ * Device-side error: TWA_ERR_NONFINITE. */
+int twa_quantize_basis(twa_ctx* ctx, const twa_basis* P32, int bits, twa_basis* Pq, void* ws,
+                       size_t ws_bytes);
+
+/* Canonical image of a quantised basis, for parity checks and checkpoints:
+ *  codes_out  device, n * ceil(D*bits/8) bytes, column after column without padding;
+ *             bits 8: two's-complement int8; bits 4: row 2k low nibble, row 2k+1 high
+ *             nibble, two's-complement nibbles, last high nibble 0 when D is odd.
+ *  scales_out device, n floats. */
+int twa_basis_export(twa_ctx* ctx, const twa_basis* Pq, void* codes_out, float* scales_out);
+/* Inverse of twa_basis_export; Pq->data / Pq->scales set by the caller as for quantise. */
+int twa_basis_import(twa_ctx* ctx, const void* codes, const float* scales, int64_t D, int n,
+                     int bits, twa_basis* Pq);
+
+/* ---- subspace step (Sections 4.2-4.3; loop body of Algorithm 1) --------------------- */
+
+/* c_out[j] = s_j * sum_r code[r,j] * g[r]  (bits 32: sum_r P[r,j] g[r]).
+ *  g      in: D elements of g_dtype (bfloat16 is widened exactly inside the kernel).
+ *  c_out  out: n floats.
+ * Products and partial sums are float32, the final combine over blocks is float64 in block
+ * order. */
+int twa_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
+                float* c_out, void* ws, size_t ws_bytes);
+
+/* w_out[r] = base[r] + sum_j (s_j * alpha[j]) * code[r,j].
+ *  alpha  in: n floats.   base  in: D floats, or NULL for 0.
+ *  w_out  out: D floats; may be the same buffer as base, must not overlap P. */
+int twa_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, const float* base,
+             float* w_out, void* ws, size_t ws_bytes);
+
+/* One training iteration of the subspace: c = P~^T g; alpha <- (1 - lr*lambda) alpha - lr c;
+ * w = wbar + P~ alpha.  alpha (n floats) is updated in place; w (D floats) is overwritten and
+ * may be the same buffer as wbar only if the caller wants wbar replaced.  c_out (n floats)
+ * receives c and may be NULL. */
+int twa_step(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype, float lr,
+             float lambda, float* alpha, const float* wbar, float* w, float* c_out, void* ws,
+             size_t ws_bytes);
+
+/* The same iteration for a caller whose gradient and weights live in HOST memory (pinned
+ * memory makes the copies asynchronous): copies g_host (D elements) into the device
+ * staging buffer g_stage, runs twa_step into the device buffer w, and copies w back to
+ * w_host (D floats).  All three operations are enqueued on the context's stream. */
+int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host /* host */,
+                  twa_dtype g_dtype, float lr, float lambda, float* alpha, const float* wbar,
+                  float* w, float* w_host /* host */, void* g_stage, void* ws, size_t ws_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TWA_H_ */

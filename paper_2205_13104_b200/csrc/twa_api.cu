@@ -1,0 +1,238 @@
+// C entry points: context, status, and the per-step calls (project, lift, step).
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "twa_common.cuh"
+
+namespace {
+
+int check_ws(const void* ws, size_t ws_bytes) {
+  if (!ws || ws_bytes < TWA_WS_BYTES) return TWA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(ws) & 15) return TWA_ERR_MISALIGNED;
+  return TWA_OK;
+}
+
+bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
+
+}  // namespace
+
+extern "C" {
+
+int twa_create(twa_ctx** out, int device, void* cuda_stream) {
+  if (!out) return TWA_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count)
+    return TWA_ERR_INVALID_ARG;
+  twa_ctx* ctx = static_cast<twa_ctx*>(calloc(1, sizeof(twa_ctx)));
+  if (!ctx) return TWA_ERR_INVALID_ARG;
+  ctx->device = device;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  ctx->wait_limit_ns = 2000ull * 1000ull * 1000ull;
+  int rc = [&]() -> int {
+    TWA_CUDA_OK(ctx, cudaSetDevice(device));
+    cudaDeviceProp prop;
+    TWA_CUDA_OK(ctx, cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) {
+      snprintf(ctx->last_error, sizeof(ctx->last_error),
+               "device %d is compute capability %d.%d; this library is built for sm_100a only",
+               device, prop.major, prop.minor);
+      return TWA_ERR_UNSUPPORTED;
+    }
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    TWA_CUDA_OK(ctx, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) {
+      snprintf(ctx->last_error, sizeof(ctx->last_error), "cuTensorMapEncodeTiled not found in the driver");
+      return TWA_ERR_CUDA;
+    }
+    ctx->encode_tiled = reinterpret_cast<twa_encode_tiled_fn>(fn);
+    void* d = nullptr;
+    TWA_CUDA_OK(ctx, cudaMalloc(&d, 256));
+    TWA_CUDA_OK(ctx, cudaMemset(d, 0, 256));
+    ctx->d_status = static_cast<int*>(d);
+    ctx->d_ticket = reinterpret_cast<unsigned*>(static_cast<char*>(d) + 128);
+    return TWA_OK;
+  }();
+  if (rc != TWA_OK) {
+    fprintf(stderr, "twa_create: %s\n", ctx->last_error);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    free(ctx);
+    return rc;
+  }
+  *out = ctx;
+  return TWA_OK;
+}
+
+void twa_destroy(twa_ctx* ctx) {
+  if (!ctx) return;
+  cudaSetDevice(ctx->device);
+  cudaStreamSynchronize(ctx->stream);
+  if (ctx->prof_events) {
+    for (int i = 0; i < 3 * ctx->prof_cap; ++i) cudaEventDestroy(ctx->prof_events[i]);
+    free(ctx->prof_events);
+  }
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  free(ctx);
+}
+
+int twa_get_status(twa_ctx* ctx, int* code, int* detail) {
+  if (!ctx || !code) return TWA_ERR_INVALID_ARG;
+  int h[2] = {0, -1};
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  TWA_CUDA_OK(ctx, cudaMemcpyAsync(h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost, ctx->stream));
+  TWA_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));
+  *code = h[0];
+  if (detail) *detail = h[0] ? h[1] : -1;
+  return TWA_OK;
+}
+
+int twa_clear_status(twa_ctx* ctx) {
+  if (!ctx) return TWA_ERR_INVALID_ARG;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  TWA_CUDA_OK(ctx, cudaMemsetAsync(ctx->d_status, 0, 256, ctx->stream));
+  return TWA_OK;
+}
+
+const char* twa_strerror(int code) {
+  switch (code) {
+    case TWA_OK: return "ok";
+    case TWA_ERR_INVALID_ARG: return "invalid argument";
+    case TWA_ERR_MISALIGNED: return "pointer or stride not 16-byte aligned";
+    case TWA_ERR_UNSUPPORTED: return "unsupported size, width or device";
+    case TWA_ERR_RANK_DEFICIENT: return "candidates are linearly dependent";
+    case TWA_ERR_NONFINITE: return "non-finite value in the input";
+    case TWA_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case TWA_ERR_CUDA: return "CUDA call failed";
+    case TWA_ERR_WORKSPACE: return "workspace missing or too small";
+    default: return "unknown error";
+  }
+}
+
+const char* twa_last_error(const twa_ctx* ctx) { return ctx ? ctx->last_error : ""; }
+
+int twa_set_tuning(twa_ctx* ctx, int key, int value) {
+  if (!ctx || value < 0) return TWA_ERR_INVALID_ARG;
+  switch (key) {
+    case TWA_TUNE_PROJECT_WARPS: ctx->tune_project_warps = value; return TWA_OK;
+    case TWA_TUNE_LIFT_WARPS: ctx->tune_lift_warps = value; return TWA_OK;
+    case TWA_TUNE_STAGES: ctx->tune_stages = value; return TWA_OK;
+    case TWA_TUNE_WAIT_LIMIT_MS:
+      ctx->wait_limit_ns = (value ? static_cast<unsigned long long>(value) : 2000ull) * 1000000ull;
+      return TWA_OK;
+    default: return TWA_ERR_INVALID_ARG;
+  }
+}
+
+int twa_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype, float* c_out,
+                void* ws, size_t ws_bytes) {
+  if (!ctx || !g || !c_out) return TWA_ERR_INVALID_ARG;
+  if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
+  int rc = twa_check_basis(P);
+  if (rc) return rc;
+  rc = check_ws(ws, ws_bytes);
+  if (rc) return rc;
+  if (misaligned16(g)) return TWA_ERR_MISALIGNED;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  twa_project_epilogue epi = {c_out, nullptr, 0.0f, 0.0f, -1};
+  return twa_launch_project(ctx, P, g, g_dtype, epi, ws);
+}
+
+int twa_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, const float* base, float* w_out,
+             void* ws, size_t ws_bytes) {
+  if (!ctx || !alpha || !w_out) return TWA_ERR_INVALID_ARG;
+  int rc = twa_check_basis(P);
+  if (rc) return rc;
+  rc = check_ws(ws, ws_bytes);
+  if (rc) return rc;
+  if (misaligned16(w_out) || (base && misaligned16(base))) return TWA_ERR_MISALIGNED;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  return twa_launch_lift(ctx, P, alpha, 1.0f, base, w_out, false);
+}
+
+int twa_step(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype, float lr, float lambda,
+             float* alpha, const float* wbar, float* w, float* c_out, void* ws, size_t ws_bytes) {
+  if (!ctx || !g || !alpha || !wbar || !w) return TWA_ERR_INVALID_ARG;
+  if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
+  int rc = twa_check_basis(P);
+  if (rc) return rc;
+  rc = check_ws(ws, ws_bytes);
+  if (rc) return rc;
+  if (misaligned16(g) || misaligned16(w) || misaligned16(wbar)) return TWA_ERR_MISALIGNED;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  twa_project_epilogue epi = {c_out, alpha, lr, lambda, -1};
+  cudaEvent_t* ev = nullptr;
+  if (ctx->prof_events && ctx->prof_count < ctx->prof_cap) ev = ctx->prof_events + 3 * ctx->prof_count;
+  if (ev) TWA_CUDA_OK(ctx, cudaEventRecord(ev[0], ctx->stream));
+  rc = twa_launch_project(ctx, P, g, g_dtype, epi, ws);
+  if (rc) return rc;
+  if (ev) TWA_CUDA_OK(ctx, cudaEventRecord(ev[1], ctx->stream));
+  // The lift walks the tiles backwards: the part of P~ the projection read last is the part
+  // most likely still in L2.
+  rc = twa_launch_lift(ctx, P, alpha, 1.0f, wbar, w, true);
+  if (rc) return rc;
+  if (ev) {
+    TWA_CUDA_OK(ctx, cudaEventRecord(ev[2], ctx->stream));
+    ctx->prof_count++;
+  }
+  return TWA_OK;
+}
+
+int twa_profile_enable(twa_ctx* ctx, int max_steps) {
+  if (!ctx || max_steps < 0 || max_steps > 65536) return TWA_ERR_INVALID_ARG;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  if (ctx->prof_events) {
+    TWA_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));
+    for (int i = 0; i < 3 * ctx->prof_cap; ++i) cudaEventDestroy(ctx->prof_events[i]);
+    free(ctx->prof_events);
+    ctx->prof_events = nullptr;
+    ctx->prof_cap = ctx->prof_count = 0;
+  }
+  if (max_steps == 0) return TWA_OK;
+  ctx->prof_events = static_cast<cudaEvent_t*>(calloc(3 * static_cast<size_t>(max_steps), sizeof(cudaEvent_t)));
+  if (!ctx->prof_events) return TWA_ERR_INVALID_ARG;
+  for (int i = 0; i < 3 * max_steps; ++i) TWA_CUDA_OK(ctx, cudaEventCreate(&ctx->prof_events[i]));
+  ctx->prof_cap = max_steps;
+  ctx->prof_count = 0;
+  return TWA_OK;
+}
+
+int twa_profile_read(twa_ctx* ctx, double* project_ms, double* lift_ms, int* steps) {
+  if (!ctx || !project_ms || !lift_ms || !steps) return TWA_ERR_INVALID_ARG;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  TWA_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));
+  double p = 0, l = 0;
+  for (int i = 0; i < ctx->prof_count; ++i) {
+    float a = 0, b = 0;
+    TWA_CUDA_OK(ctx, cudaEventElapsedTime(&a, ctx->prof_events[3 * i], ctx->prof_events[3 * i + 1]));
+    TWA_CUDA_OK(ctx, cudaEventElapsedTime(&b, ctx->prof_events[3 * i + 1], ctx->prof_events[3 * i + 2]));
+    p += a;
+    l += b;
+  }
+  *project_ms = p;
+  *lift_ms = l;
+  *steps = ctx->prof_count;
+  ctx->prof_count = 0;
+  return TWA_OK;
+}
+
+int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host, twa_dtype g_dtype, float lr,
+                  float lambda, float* alpha, const float* wbar, float* w, float* w_host, void* g_stage,
+                  void* ws, size_t ws_bytes) {
+  if (!ctx || !g_host || !w_host || !g_stage || !P) return TWA_ERR_INVALID_ARG;
+  if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
+  if (P->D < 1) return TWA_ERR_INVALID_ARG;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  const size_t gbytes = static_cast<size_t>(P->D) * (g_dtype == TWA_BF16 ? 2 : 4);
+  TWA_CUDA_OK(ctx, cudaMemcpyAsync(g_stage, g_host, gbytes, cudaMemcpyHostToDevice, ctx->stream));
+  int rc = twa_step(ctx, P, g_stage, g_dtype, lr, lambda, alpha, wbar, w, nullptr, ws, ws_bytes);
+  if (rc) return rc;
+  TWA_CUDA_OK(ctx, cudaMemcpyAsync(w_host, w, static_cast<size_t>(P->D) * 4, cudaMemcpyDeviceToHost,
+                                   ctx->stream));
+  return TWA_OK;
+}
+
+}  // extern "C"

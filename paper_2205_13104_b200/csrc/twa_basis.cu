@@ -1,0 +1,392 @@
+// Subspace construction and low-bit storage: mean of the candidates, classical Gram-Schmidt
+// with re-orthogonalisation (Section 4.1 of the paper), per-column absmax quantisation
+// (the symmetric per-column variant of Section 4.6) and the canonical export / import.
+#include <math.h>
+#include <stdio.h>
+
+#include "twa_common.cuh"
+
+namespace {
+
+constexpr int BLOCK = 256;
+
+// ---- mean ---------------------------------------------------------------------------------
+// One thread owns four consecutive rows and walks the n columns in index order.
+__global__ void __launch_bounds__(BLOCK) mean_kernel(const float* __restrict__ W, long long D, int n,
+                                                     long long ldw, float* __restrict__ out) {
+  const long long nvec = D >> 2;
+  const double dn = static_cast<double>(n);
+  for (long long v = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; v < nvec;
+       v += static_cast<long long>(gridDim.x) * BLOCK) {
+    double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+    for (int i = 0; i < n; ++i) {
+      const float4 x = __ldcs(reinterpret_cast<const float4*>(W + i * ldw) + v);
+      s0 += x.x; s1 += x.y; s2 += x.z; s3 += x.w;
+    }
+    out[4 * v + 0] = static_cast<float>(s0 / dn);
+    out[4 * v + 1] = static_cast<float>(s1 / dn);
+    out[4 * v + 2] = static_cast<float>(s2 / dn);
+    out[4 * v + 3] = static_cast<float>(s3 / dn);
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (D & 3)) {
+    const long long r = (nvec << 2) + threadIdx.x;
+    double s = 0;
+    for (int i = 0; i < n; ++i) s += W[i * ldw + r];
+    out[r] = static_cast<float>(s / dn);
+  }
+}
+
+// ---- squared norm of a column ----------------------------------------------------------------
+__device__ __forceinline__ double block_sum(double v, double* sh) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) sh[warp] = v;
+  __syncthreads();
+  double t = 0;
+  if (threadIdx.x == 0)
+    for (int w = 0; w < BLOCK / 32; ++w) t += sh[w];
+  return t;   // valid in thread 0
+}
+
+__global__ void __launch_bounds__(BLOCK) sumsq_kernel(const float* __restrict__ v, long long D,
+                                                      double* __restrict__ dpart,
+                                                      double* __restrict__ result,
+                                                      unsigned* __restrict__ ticket) {
+  __shared__ double sh[BLOCK / 32];
+  __shared__ int last;
+  const long long nvec = D >> 2;
+  double s = 0;
+  for (long long i = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; i < nvec;
+       i += static_cast<long long>(gridDim.x) * BLOCK) {
+    const float4 x = reinterpret_cast<const float4*>(v)[i];
+    s += static_cast<double>(x.x) * x.x + static_cast<double>(x.y) * x.y +
+         static_cast<double>(x.z) * x.z + static_cast<double>(x.w) * x.w;
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (D & 3)) {
+    const double x = v[(nvec << 2) + threadIdx.x];
+    s += x * x;
+  }
+  const double bs = block_sum(s, sh);
+  if (threadIdx.x == 0) {
+    dpart[blockIdx.x] = bs;
+    __threadfence();
+    last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (last && threadIdx.x == 0) {
+    __threadfence();
+    double t = 0;
+    for (unsigned b = 0; b < gridDim.x; ++b) t += __ldcg(&dpart[b]);
+    *result = t;
+    *ticket = 0u;
+  }
+}
+
+// ---- normalise a column: v <- v / |v|, with the rank and finiteness checks -------------------
+__global__ void __launch_bounds__(BLOCK) normalise_kernel(float* __restrict__ v, long long D,
+                                                          const double* __restrict__ norms, int column,
+                                                          int* status) {
+  const double na = norms[0], nv = norms[1];
+  double f;
+  if (!isfinite(na) || !isfinite(nv)) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) twa_set_status(status, TWA_ERR_NONFINITE, column);
+    f = 0.0;
+  } else if (!(sqrt(nv) > 1e-5 * sqrt(na))) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) twa_set_status(status, TWA_ERR_RANK_DEFICIENT, column);
+    f = 0.0;
+  } else {
+    f = 1.0 / sqrt(nv);
+  }
+  const long long nvec = D >> 2;
+  for (long long i = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; i < nvec;
+       i += static_cast<long long>(gridDim.x) * BLOCK) {
+    float4 x = reinterpret_cast<float4*>(v)[i];
+    x.x = static_cast<float>(x.x * f); x.y = static_cast<float>(x.y * f);
+    x.z = static_cast<float>(x.z * f); x.w = static_cast<float>(x.w * f);
+    reinterpret_cast<float4*>(v)[i] = x;
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (D & 3)) {
+    const long long r = (nvec << 2) + threadIdx.x;
+    v[r] = static_cast<float>(v[r] * f);
+  }
+}
+
+// ---- quantiser -------------------------------------------------------------------------------
+// Bit pattern of |x|: ordering as unsigned integers equals ordering of the magnitudes, and
+// every NaN or Inf compares above every finite value, so non-finite input surfaces in the max.
+__global__ void __launch_bounds__(BLOCK) absmax_kernel(const float* __restrict__ P, long long D,
+                                                       long long ld, unsigned* __restrict__ absmax) {
+  __shared__ unsigned sh[BLOCK / 32];
+  const float* col = P + blockIdx.y * ld;
+  const long long nvec = D >> 2;
+  unsigned m = 0;
+  for (long long i = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; i < nvec;
+       i += static_cast<long long>(gridDim.x) * BLOCK) {
+    const uint4 x = reinterpret_cast<const uint4*>(col)[i];
+    m = max(m, x.x & 0x7FFFFFFFu); m = max(m, x.y & 0x7FFFFFFFu);
+    m = max(m, x.z & 0x7FFFFFFFu); m = max(m, x.w & 0x7FFFFFFFu);
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (D & 3))
+    m = max(m, __float_as_uint(col[(nvec << 2) + threadIdx.x]) & 0x7FFFFFFFu);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < BLOCK / 32; ++w) m = max(m, sh[w]);
+    atomicMax(&absmax[blockIdx.y], m);
+  }
+}
+
+__global__ void scales_kernel(const unsigned* __restrict__ absmax, int n, float qmax,
+                              float* __restrict__ scales, int* status) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= n) return;
+  const unsigned b = absmax[j];
+  if (b >= 0x7F800000u) {
+    twa_set_status(status, TWA_ERR_NONFINITE, j);
+    scales[j] = 0.0f;
+  } else {
+    scales[j] = __fdiv_rn(__uint_as_float(b), qmax);
+  }
+}
+
+__device__ __forceinline__ int encode_one(float p, float s, float qmax) {
+  if (s == 0.0f) return 0;
+  float q = rintf(__fdiv_rn(p, s));                   // round half to even
+  q = fminf(fmaxf(q, -qmax), qmax);
+  return static_cast<int>(q);
+}
+
+// One thread produces 16 bytes of a column (16 rows at 8 bits, 32 rows at 4 bits), including
+// the padding up to the column stride, which is filled with the code 0.
+template <int BITS>
+__global__ void __launch_bounds__(BLOCK) encode_kernel(const float* __restrict__ P, long long D,
+                                                       long long ld, const float* __restrict__ scales,
+                                                       unsigned char* __restrict__ out,
+                                                       long long out_stride) {
+  constexpr int RPT = 128 / BITS;                     // rows per thread-iteration
+  constexpr float QMAX = BITS == 8 ? 127.0f : 7.0f;
+  constexpr int BIAS = BITS == 8 ? 128 : 8;
+  const int j = blockIdx.y;
+  const float* col = P + j * ld;
+  const float s = scales[j];
+  uint4* dst = reinterpret_cast<uint4*>(out + j * out_stride);
+  const long long chunks = out_stride / 16;
+  for (long long q = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; q < chunks;
+       q += static_cast<long long>(gridDim.x) * BLOCK) {
+    const long long r0 = q * RPT;
+    float p[RPT];
+    if (r0 + RPT <= D) {
+#pragma unroll
+      for (int k = 0; k < RPT / 4; ++k) {
+        const float4 x = __ldcs(reinterpret_cast<const float4*>(col + r0) + k);
+        p[4 * k] = x.x; p[4 * k + 1] = x.y; p[4 * k + 2] = x.z; p[4 * k + 3] = x.w;
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < RPT; ++k) p[k] = (r0 + k < D) ? col[r0 + k] : 0.0f;
+    }
+    uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int k = 0; k < RPT; ++k) {
+      const uint32_t u = static_cast<uint32_t>(encode_one(p[k], s, QMAX) + BIAS);
+      if (BITS == 8) w[k >> 2] |= u << (8 * (k & 3));
+      else w[k >> 3] |= u << (4 * (k & 7));
+    }
+    dst[q] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+// internal (offset binary, padded) <-> canonical (two's complement, tight)
+__global__ void __launch_bounds__(BLOCK) recode_kernel(const unsigned char* __restrict__ in,
+                                                       long long in_stride,
+                                                       unsigned char* __restrict__ out,
+                                                       long long out_stride, long long row_bytes,
+                                                       long long fill_to, unsigned char mask) {
+  const unsigned char* src = in + blockIdx.y * in_stride;
+  unsigned char* dst = out + blockIdx.y * out_stride;
+  for (long long b = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; b < fill_to;
+       b += static_cast<long long>(gridDim.x) * BLOCK)
+    dst[b] = (b < row_bytes) ? static_cast<unsigned char>(src[b] ^ mask) : mask;
+}
+
+int grid_for(const twa_ctx* ctx, long long items, int per_block, int blocks_per_sm) {
+  long long g = (items + per_block - 1) / per_block;
+  const long long cap = static_cast<long long>(ctx->sm_count) * blocks_per_sm;
+  if (g > cap) g = cap;
+  if (g > TWA_MAX_GRID) g = TWA_MAX_GRID;
+  if (g < 1) g = 1;
+  return static_cast<int>(g);
+}
+
+int launch_sumsq(twa_ctx* ctx, const float* v, long long D, void* ws, int slot) {
+  char* w = static_cast<char*>(ws);
+  const int grid = grid_for(ctx, D, BLOCK * 16, 4);
+  sumsq_kernel<<<grid, BLOCK, 0, ctx->stream>>>(v, D, reinterpret_cast<double*>(w + TWA_WS_DPART),
+                                                reinterpret_cast<double*>(w + TWA_WS_NORMS) + slot,
+                                                ctx->d_ticket);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t twa_basis_col_stride(int64_t D, int bits) {
+  if (D < 1 || (bits != 32 && bits != 8 && bits != 4)) return 0;
+  const int64_t row_bytes = (D * bits + 7) / 8;
+  return (row_bytes + 127) / 128 * 128;
+}
+
+size_t twa_basis_bytes(int64_t D, int n, int bits) {
+  if (n < 1) return 0;
+  return static_cast<size_t>(twa_basis_col_stride(D, bits)) * static_cast<size_t>(n);
+}
+
+size_t twa_workspace_bytes(int64_t, int, int) { return TWA_WS_BYTES; }
+
+int twa_mean(twa_ctx* ctx, const float* W, int64_t D, int n, int64_t ldw, float* wbar_out) {
+  if (!ctx || !W || !wbar_out || D < 1 || n < 1 || ldw < D) return TWA_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(W) & 15) || (ldw & 3) || (reinterpret_cast<uintptr_t>(wbar_out) & 15))
+    return TWA_ERR_MISALIGNED;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  const int grid = grid_for(ctx, D, BLOCK * 4, 8);
+  mean_kernel<<<grid, BLOCK, 0, ctx->stream>>>(W, D, n, ldw, wbar_out);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float* wbar_out,
+                    twa_basis* P32_out, void* ws, size_t ws_bytes) {
+  if (!ctx || !W || !wbar_out || !P32_out) return TWA_ERR_INVALID_ARG;
+  if (D < 1 || D >= (1LL << 31) || n < 1 || ldw < D) return TWA_ERR_INVALID_ARG;
+  if (n > TWA_MAX_N) return TWA_ERR_UNSUPPORTED;
+  if (!ws || ws_bytes < TWA_WS_BYTES) return TWA_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(W) & 15) || (ldw & 3) || (reinterpret_cast<uintptr_t>(ws) & 15) ||
+      (reinterpret_cast<uintptr_t>(wbar_out) & 15))
+    return TWA_ERR_MISALIGNED;
+  int rc = twa_mean(ctx, W, D, n, ldw, wbar_out);
+  if (rc) return rc;
+
+  char* w = static_cast<char*>(ws);
+  float* coef = reinterpret_cast<float*>(w + TWA_WS_COEF);
+  const double* norms = reinterpret_cast<const double*>(w + TWA_WS_NORMS);
+  const int egrid = grid_for(ctx, D, BLOCK * 16, 4);
+  for (int j = 0; j < n; ++j) {
+    float* col = W + j * ldw;
+    rc = launch_sumsq(ctx, col, D, ws, 0);                       // |a_j|^2
+    if (rc) return rc;
+    if (j > 0) {
+      twa_basis Q = {W, nullptr, D, 4 * ldw, j, 32};
+      twa_project_epilogue epi = {coef, nullptr, 0.0f, 0.0f, j};
+      for (int pass = 0; pass < 2; ++pass) {
+        rc = twa_launch_project(ctx, &Q, col, TWA_F32, epi, ws);  // c = Q^T v, all from the same v
+        if (rc) return rc;
+        rc = twa_launch_lift(ctx, &Q, coef, -1.0f, col, col, false);   // v <- v - Q c
+        if (rc) return rc;
+      }
+    }
+    rc = launch_sumsq(ctx, col, D, ws, 1);                       // |v|^2
+    if (rc) return rc;
+    normalise_kernel<<<egrid, BLOCK, 0, ctx->stream>>>(col, D, norms, j, ctx->d_status);
+    TWA_CUDA_OK(ctx, cudaGetLastError());
+  }
+  P32_out->data = W;
+  P32_out->scales = nullptr;
+  P32_out->D = D;
+  P32_out->col_stride = 4 * ldw;
+  P32_out->n = n;
+  P32_out->bits = 32;
+  return TWA_OK;
+}
+
+int twa_quantize_basis(twa_ctx* ctx, const twa_basis* P32, int bits, twa_basis* Pq, void* ws,
+                       size_t ws_bytes) {
+  if (!ctx || !P32 || !Pq) return TWA_ERR_INVALID_ARG;
+  if (bits != 8 && bits != 4) return TWA_ERR_UNSUPPORTED;
+  if (!Pq->data || !Pq->scales) return TWA_ERR_INVALID_ARG;
+  int rc = twa_check_basis(P32);
+  if (rc) return rc;
+  if (P32->bits != 32) return TWA_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < TWA_WS_BYTES) return TWA_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(Pq->data) & 15) || (reinterpret_cast<uintptr_t>(ws) & 15))
+    return TWA_ERR_MISALIGNED;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  const long long D = P32->D;
+  const int n = P32->n;
+  const long long ld = P32->col_stride / 4;
+  const float* P = static_cast<const float*>(P32->data);
+  unsigned* absmax = reinterpret_cast<unsigned*>(static_cast<char*>(ws) + TWA_WS_ABSMAX);
+  TWA_CUDA_OK(ctx, cudaMemsetAsync(absmax, 0, sizeof(unsigned) * n, ctx->stream));
+  int per_col = grid_for(ctx, D, BLOCK * 16, 8) / n;
+  if (per_col < 1) per_col = 1;
+  absmax_kernel<<<dim3(per_col, n), BLOCK, 0, ctx->stream>>>(P, D, ld, absmax);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  scales_kernel<<<1, 128, 0, ctx->stream>>>(absmax, n, bits == 8 ? 127.0f : 7.0f, Pq->scales,
+                                            ctx->d_status);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  const long long stride = twa_basis_col_stride(D, bits);
+  int eper = grid_for(ctx, stride / 16, BLOCK, 8) / n;
+  if (eper < 1) eper = 1;
+  if (bits == 8)
+    encode_kernel<8><<<dim3(eper, n), BLOCK, 0, ctx->stream>>>(
+        P, D, ld, Pq->scales, static_cast<unsigned char*>(Pq->data), stride);
+  else
+    encode_kernel<4><<<dim3(eper, n), BLOCK, 0, ctx->stream>>>(
+        P, D, ld, Pq->scales, static_cast<unsigned char*>(Pq->data), stride);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  Pq->D = D;
+  Pq->col_stride = stride;
+  Pq->n = n;
+  Pq->bits = bits;
+  return TWA_OK;
+}
+
+int twa_basis_export(twa_ctx* ctx, const twa_basis* Pq, void* codes_out, float* scales_out) {
+  if (!ctx || !codes_out || !scales_out) return TWA_ERR_INVALID_ARG;
+  int rc = twa_check_basis(Pq);
+  if (rc) return rc;
+  if (Pq->bits == 32) return TWA_ERR_UNSUPPORTED;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  const long long row_bytes = (Pq->D * Pq->bits + 7) / 8;
+  int per = grid_for(ctx, row_bytes, BLOCK * 8, 8) / Pq->n;
+  if (per < 1) per = 1;
+  recode_kernel<<<dim3(per, Pq->n), BLOCK, 0, ctx->stream>>>(
+      static_cast<const unsigned char*>(Pq->data), Pq->col_stride,
+      static_cast<unsigned char*>(codes_out), row_bytes, row_bytes, row_bytes,
+      Pq->bits == 8 ? 0x80 : 0x88);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  TWA_CUDA_OK(ctx, cudaMemcpyAsync(scales_out, Pq->scales, sizeof(float) * Pq->n,
+                                   cudaMemcpyDeviceToDevice, ctx->stream));
+  return TWA_OK;
+}
+
+int twa_basis_import(twa_ctx* ctx, const void* codes, const float* scales, int64_t D, int n, int bits,
+                     twa_basis* Pq) {
+  if (!ctx || !codes || !scales || !Pq || !Pq->data || !Pq->scales) return TWA_ERR_INVALID_ARG;
+  if (bits != 8 && bits != 4) return TWA_ERR_UNSUPPORTED;
+  if (D < 1 || D >= (1LL << 31) || n < 1) return TWA_ERR_INVALID_ARG;
+  if (n > TWA_MAX_N) return TWA_ERR_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(Pq->data) & 15) return TWA_ERR_MISALIGNED;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  const long long row_bytes = (D * bits + 7) / 8;
+  const long long stride = twa_basis_col_stride(D, bits);
+  int per = grid_for(ctx, stride, BLOCK * 8, 8) / n;
+  if (per < 1) per = 1;
+  recode_kernel<<<dim3(per, n), BLOCK, 0, ctx->stream>>>(
+      static_cast<const unsigned char*>(codes), row_bytes, static_cast<unsigned char*>(Pq->data),
+      stride, row_bytes, stride, bits == 8 ? 0x80 : 0x88);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  TWA_CUDA_OK(ctx, cudaMemcpyAsync(Pq->scales, scales, sizeof(float) * n, cudaMemcpyDeviceToDevice,
+                                   ctx->stream));
+  Pq->D = D;
+  Pq->col_stride = stride;
+  Pq->n = n;
+  Pq->bits = bits;
+  return TWA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,195 @@
+// Shared declarations of the TWA CUDA library: context, workspace layout, device-side
+// status reporting, and thin wrappers over the mbarrier / bulk-tensor-copy PTX used by the
+// streaming kernels.  sm_100a only.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "twa.h"
+
+// ------------------------------------------------------------------------------------------
+// Host-side context
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*twa_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                        const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                        const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                        CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct twa_ctx {
+  int device;
+  cudaStream_t stream;
+  int sm_count;
+  int smem_optin;             // largest dynamic shared memory a block may request
+  int* d_status;              // [0] first error code, [1] its detail
+  unsigned int* d_ticket;     // block-completion counters, zero between kernels
+  twa_encode_tiled_fn encode_tiled;
+  unsigned long long wait_limit_ns;
+  int tune_project_warps, tune_lift_warps, tune_stages;
+  cudaEvent_t* prof_events;   // 3 per recorded step, or null
+  int prof_cap, prof_count;   // steps
+  char last_error[256];
+};
+
+#define TWA_CUDA_OK(ctx, expr)                                                              \
+  do {                                                                                      \
+    cudaError_t e__ = (expr);                                                               \
+    if (e__ != cudaSuccess) {                                                               \
+      snprintf((ctx)->last_error, sizeof((ctx)->last_error), "%s: %s", #expr,               \
+               cudaGetErrorString(e__));                                                    \
+      return TWA_ERR_CUDA;                                                                  \
+    }                                                                                       \
+  } while (0)
+
+// ------------------------------------------------------------------------------------------
+// Workspace layout (bytes from the start of `ws`)
+// ------------------------------------------------------------------------------------------
+constexpr int TWA_MAX_GRID = 1024;                       // upper bound on blocks of a reduction
+constexpr size_t TWA_WS_PARTIALS = 0;                    // float [TWA_MAX_GRID][TWA_MAX_N]
+constexpr size_t TWA_WS_COEF = TWA_WS_PARTIALS + sizeof(float) * TWA_MAX_GRID * TWA_MAX_N;
+                                                         // float [TWA_MAX_N]  projection coefficients
+constexpr size_t TWA_WS_NORMS = TWA_WS_COEF + sizeof(float) * TWA_MAX_N;
+                                                         // double[4]: 0 = |a_j|^2, 1 = |v|^2
+constexpr size_t TWA_WS_DPART = TWA_WS_NORMS + 64;       // double [TWA_MAX_GRID] partial sums
+constexpr size_t TWA_WS_ABSMAX = TWA_WS_DPART + sizeof(double) * TWA_MAX_GRID;
+                                                         // uint  [TWA_MAX_N]  bit patterns of column absmax
+constexpr size_t TWA_WS_BYTES = TWA_WS_ABSMAX + sizeof(unsigned) * TWA_MAX_N;
+
+// ------------------------------------------------------------------------------------------
+// Streaming-kernel geometry
+// ------------------------------------------------------------------------------------------
+constexpr int TWA_TILE_COL_BYTES = 512;                  // bytes of one column inside one tile
+constexpr int TWA_TILE_COL_WORDS = TWA_TILE_COL_BYTES / 4;
+constexpr int TWA_MAX_STAGES = 16;
+constexpr int TWA_MAX_CONSUMER_WARPS = 20;
+constexpr int TWA_MAX_THREADS = (TWA_MAX_CONSUMER_WARPS + 1) * 32;
+constexpr int TWA_PROJECT_CPW = 8;                       // columns one warp owns at most (project)
+constexpr int TWA_LIFT_CPW = 16;                         // columns one warp owns at most (lift)
+constexpr int TWA_SMEM_HEADER = 2048;                    // barriers + small arrays before the ring
+
+// rows covered by one tile for a storage width
+__host__ __device__ constexpr int twa_tile_rows(int bits) { return TWA_TILE_COL_BYTES * 8 / bits; }
+
+// ------------------------------------------------------------------------------------------
+// Device helpers
+// ------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ void twa_set_status(int* status, int code, int detail) {
+  if (atomicCAS(&status[0], 0, code) == 0) status[1] = detail;
+}
+
+__device__ __forceinline__ uint32_t twa_smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ unsigned long long twa_globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void twa_mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void twa_fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+__device__ __forceinline__ void twa_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+
+__device__ __forceinline__ void twa_mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ uint32_t twa_mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+
+// Waits for the phase `parity` of an mbarrier, for at most `limit_ns`.  Returns false when
+// the wait ran out or another thread of the block already gave up (*abort_flag != 0); the
+// caller then leaves its loop.  The first thread to give up raises the flag.
+__device__ __forceinline__ bool twa_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                              unsigned long long limit_ns) {
+  for (int i = 0; i < 64; ++i)
+    if (twa_mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = twa_globaltimer();
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (twa_mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (twa_globaltimer() - t0 > limit_ns) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
+
+// Bulk tensor copies global -> this block's shared memory, completion counted on an mbarrier.
+__device__ __forceinline__ void twa_tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                                uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void twa_tma_load_1d(uint32_t dst, const CUtensorMap* map, int x,
+                                                uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.1d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2}], [%3];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void twa_prefetch_tensormap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void twa_named_barrier(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// ---- code -> float ------------------------------------------------------------------------
+// A byte u in [0,255] placed in the low mantissa bits of 2^23 gives the float 2^23 + u
+// exactly; subtracting 2^23 + bias leaves the signed code as a float.
+__device__ __forceinline__ float twa_byte_to_float(uint32_t word, int byte, float magic) {
+  const uint32_t sel = 0x7440u + static_cast<uint32_t>(byte);
+  return __uint_as_float(__byte_perm(word, 0x4B000000u, sel)) - magic;
+}
+constexpr float TWA_MAGIC_I8 = 8388608.0f + 128.0f;
+constexpr float TWA_MAGIC_I4 = 8388608.0f + 8.0f;
+
+__device__ __forceinline__ float twa_bf16_lo(uint32_t pair) { return __uint_as_float(pair << 16); }
+__device__ __forceinline__ float twa_bf16_hi(uint32_t pair) { return __uint_as_float(pair & 0xFFFF0000u); }
+
+#endif  // __CUDACC__
+
+// ------------------------------------------------------------------------------------------
+// Internal launchers (defined in the .cu files)
+// ------------------------------------------------------------------------------------------
+struct twa_project_epilogue {
+  float* c_out;        // n floats or null
+  float* alpha;        // when non-null: alpha <- (1 - lr*lambda) alpha - lr c
+  float lr, lambda;
+  int nonfinite_detail; // detail reported with TWA_ERR_NONFINITE; -1 = index of the coefficient
+};
+
+int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
+                       const twa_project_epilogue& epi, void* ws);
+int twa_launch_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
+                    const float* base, float* out, bool reverse_tiles);
+int twa_check_basis(const twa_basis* P);

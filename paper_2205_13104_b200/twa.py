@@ -1,0 +1,330 @@
+"""ctypes binding of libtwa.so: one Python function per C entry point of include/twa.h,
+with the same name.  The functions only marshal arguments (torch tensors -> device
+pointers); every step of the computation runs in the CUDA library.  There is no CPU
+fallback: if the library has not been built, loading it raises.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_ROOT = os.path.dirname(_HERE)
+LIB_PATH = os.path.join(_HERE, "libtwa.so")
+CSRC = os.path.join(_HERE, "csrc")
+SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_stream.cu"]
+
+TWA_MAX_N = 128
+TWA_OK = 0
+TWA_ERR_INVALID_ARG = -1
+TWA_ERR_MISALIGNED = -2
+TWA_ERR_UNSUPPORTED = -3
+TWA_ERR_RANK_DEFICIENT = -4
+TWA_ERR_NONFINITE = -5
+TWA_ERR_TIMEOUT = -6
+TWA_ERR_CUDA = -7
+TWA_ERR_WORKSPACE = -8
+TWA_F32 = 0
+TWA_BF16 = 1
+TWA_TUNE_PROJECT_WARPS = 1
+TWA_TUNE_LIFT_WARPS = 2
+TWA_TUNE_STAGES = 3
+TWA_TUNE_WAIT_LIMIT_MS = 4
+
+EXPORTS = [
+    "twa_create", "twa_destroy", "twa_get_status", "twa_clear_status", "twa_strerror",
+    "twa_last_error", "twa_set_tuning", "twa_profile_enable", "twa_profile_read",
+    "twa_basis_col_stride", "twa_basis_bytes",
+    "twa_workspace_bytes", "twa_build_basis", "twa_mean", "twa_quantize_basis",
+    "twa_basis_export", "twa_basis_import", "twa_project", "twa_lift", "twa_step",
+    "twa_step_host",
+]
+
+
+class twa_basis(ctypes.Structure):
+    """Mirror of the C struct twa_basis."""
+    _fields_ = [("data", ctypes.c_void_p), ("scales", ctypes.c_void_p),
+                ("D", ctypes.c_int64), ("col_stride", ctypes.c_int64),
+                ("n", ctypes.c_int32), ("bits", ctypes.c_int32)]
+
+
+class TwaError(RuntimeError):
+    def __init__(self, code, where, extra=""):
+        self.code = code
+        msg = f"{where}: {twa_strerror(code)} ({code})"
+        if extra:
+            msg += f" -- {extra}"
+        super().__init__(msg)
+
+
+def build_command(out=LIB_PATH):
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    return [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(_ROOT, "include"),
+            "-o", out] + [os.path.join(CSRC, s) for s in SOURCES]
+
+
+def build_library(force=False, verbose=False):
+    """Compiles the CUDA library for sm_100a next to this file (nvcc cross-compiles without
+    a GPU).  Skipped when the library is newer than every source."""
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(_ROOT, "include", "twa.h")]
+    if not force and os.path.exists(LIB_PATH) and \
+            all(os.path.getmtime(LIB_PATH) >= os.path.getmtime(d) for d in deps):
+        return LIB_PATH
+    cmd = build_command()
+    if verbose:
+        print(" ".join(cmd))
+    subprocess.run(cmd, check=True)
+    return LIB_PATH
+
+
+_lib = None
+
+
+def load():
+    """Loads libtwa.so (once) and declares the argument types of every entry point."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                           "`python -c 'import __graft_entry__ as g; g.build()'`; there is no fallback path")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float
+    szt = ctypes.c_size_t
+    bp = ctypes.POINTER(twa_basis)
+    sig = {
+        "twa_create": (i32, [ctypes.POINTER(vp), i32, vp]),
+        "twa_destroy": (None, [vp]),
+        "twa_get_status": (i32, [vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]),
+        "twa_clear_status": (i32, [vp]),
+        "twa_strerror": (ctypes.c_char_p, [i32]),
+        "twa_last_error": (ctypes.c_char_p, [vp]),
+        "twa_set_tuning": (i32, [vp, i32, i32]),
+        "twa_profile_enable": (i32, [vp, i32]),
+        "twa_profile_read": (i32, [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
+                                   ctypes.POINTER(i32)]),
+        "twa_basis_col_stride": (i64, [i64, i32]),
+        "twa_basis_bytes": (szt, [i64, i32, i32]),
+        "twa_workspace_bytes": (szt, [i64, i32, i32]),
+        "twa_build_basis": (i32, [vp, vp, i64, i32, i64, vp, bp, vp, szt]),
+        "twa_mean": (i32, [vp, vp, i64, i32, i64, vp]),
+        "twa_quantize_basis": (i32, [vp, bp, i32, bp, vp, szt]),
+        "twa_basis_export": (i32, [vp, bp, vp, vp]),
+        "twa_basis_import": (i32, [vp, vp, vp, i64, i32, i32, bp]),
+        "twa_project": (i32, [vp, bp, vp, i32, vp, vp, szt]),
+        "twa_lift": (i32, [vp, bp, vp, vp, vp, vp, szt]),
+        "twa_step": (i32, [vp, bp, vp, i32, f32, f32, vp, vp, vp, vp, vp, szt]),
+        "twa_step_host": (i32, [vp, bp, vp, i32, f32, f32, vp, vp, vp, vp, vp, vp, szt]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+# --------------------------------------------------------------------------------------
+# helpers
+# --------------------------------------------------------------------------------------
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _dtype_code(t):
+    if t.dtype == torch.float32:
+        return TWA_F32
+    if t.dtype == torch.bfloat16:
+        return TWA_BF16
+    raise TypeError(f"gradient dtype {t.dtype} not supported (float32 or bfloat16)")
+
+
+def _check(rc, where, ctx=None):
+    if rc != TWA_OK:
+        extra = ""
+        if rc == TWA_ERR_CUDA and ctx is not None:
+            extra = twa_last_error(ctx)
+        raise TwaError(rc, where, extra)
+
+
+class Basis:
+    """A twa_basis descriptor together with the tensors that own its memory."""
+
+    def __init__(self, desc, data, scales):
+        self.desc = desc
+        self.data = data          # keeps the device buffers alive
+        self.scales = scales
+
+    D = property(lambda self: self.desc.D)
+    n = property(lambda self: self.desc.n)
+    bits = property(lambda self: self.desc.bits)
+    col_stride = property(lambda self: self.desc.col_stride)
+
+
+# --------------------------------------------------------------------------------------
+# entry points (same names as in include/twa.h)
+# --------------------------------------------------------------------------------------
+def twa_strerror(code):
+    return load().twa_strerror(int(code)).decode()
+
+
+def twa_last_error(ctx):
+    return load().twa_last_error(ctx).decode()
+
+
+def twa_create(device=0, stream=None):
+    """Context on `device` bound to `stream` (a torch.cuda.Stream; None = the current one)."""
+    lib = load()
+    if stream is None:
+        stream = torch.cuda.current_stream(device)
+    handle = ctypes.c_void_p()
+    rc = lib.twa_create(ctypes.byref(handle), int(device), ctypes.c_void_p(stream.cuda_stream))
+    _check(rc, "twa_create")
+    return handle
+
+
+def twa_destroy(ctx):
+    load().twa_destroy(ctx)
+
+
+def twa_get_status(ctx):
+    code, detail = ctypes.c_int(0), ctypes.c_int(-1)
+    _check(load().twa_get_status(ctx, ctypes.byref(code), ctypes.byref(detail)), "twa_get_status", ctx)
+    return code.value, detail.value
+
+
+def twa_clear_status(ctx):
+    _check(load().twa_clear_status(ctx), "twa_clear_status", ctx)
+
+
+def twa_set_tuning(ctx, key, value):
+    _check(load().twa_set_tuning(ctx, int(key), int(value)), "twa_set_tuning", ctx)
+
+
+def twa_profile_enable(ctx, max_steps):
+    _check(load().twa_profile_enable(ctx, int(max_steps)), "twa_profile_enable", ctx)
+
+
+def twa_profile_read(ctx):
+    """(project_ms, lift_ms, steps) summed over the steps recorded since the last read."""
+    p, l, k = ctypes.c_double(0), ctypes.c_double(0), ctypes.c_int(0)
+    _check(load().twa_profile_read(ctx, ctypes.byref(p), ctypes.byref(l), ctypes.byref(k)),
+           "twa_profile_read", ctx)
+    return p.value, l.value, k.value
+
+
+def twa_basis_col_stride(D, bits):
+    return int(load().twa_basis_col_stride(int(D), int(bits)))
+
+
+def twa_basis_bytes(D, n, bits):
+    return int(load().twa_basis_bytes(int(D), int(n), int(bits)))
+
+
+def twa_workspace_bytes(D, n, bits):
+    return int(load().twa_workspace_bytes(int(D), int(n), int(bits)))
+
+
+def new_workspace(device, D=1, n=1, bits=8):
+    return torch.empty(twa_workspace_bytes(D, n, bits), dtype=torch.uint8, device=device)
+
+
+def twa_mean(ctx, W, D, wbar_out):
+    n, ldw = W.shape
+    _check(load().twa_mean(ctx, _ptr(W), int(D), int(n), int(ldw), _ptr(wbar_out)), "twa_mean", ctx)
+    return wbar_out
+
+
+def twa_build_basis(ctx, W, D, wbar_out, ws):
+    """W: float32 CUDA tensor (n, ldw), row i = candidate w_i; overwritten by the basis."""
+    assert W.dtype == torch.float32 and W.is_contiguous()
+    n, ldw = W.shape
+    desc = twa_basis()
+    rc = load().twa_build_basis(ctx, _ptr(W), int(D), int(n), int(ldw), _ptr(wbar_out),
+                                ctypes.byref(desc), _ptr(ws), ws.numel())
+    _check(rc, "twa_build_basis", ctx)
+    return Basis(desc, W, None)
+
+
+def basis_from_tensor(P32, D):
+    """Descriptor for a float32 CUDA tensor (n, ld) holding a basis column per row."""
+    assert P32.dtype == torch.float32 and P32.is_contiguous()
+    n, ld = P32.shape
+    desc = twa_basis(P32.data_ptr(), None, int(D), 4 * int(ld), int(n), 32)
+    return Basis(desc, P32, None)
+
+
+def _new_quantised(D, n, bits, device):
+    data = torch.empty(twa_basis_bytes(D, n, bits), dtype=torch.uint8, device=device)
+    scales = torch.empty(n, dtype=torch.float32, device=device)
+    desc = twa_basis(data.data_ptr(), scales.data_ptr(), 0, 0, 0, 0)
+    return desc, data, scales
+
+
+def twa_quantize_basis(ctx, P32, bits, ws):
+    desc, data, scales = _new_quantised(P32.D, P32.n, bits, P32.data.device)
+    rc = load().twa_quantize_basis(ctx, ctypes.byref(P32.desc), int(bits), ctypes.byref(desc),
+                                   _ptr(ws), ws.numel())
+    _check(rc, "twa_quantize_basis", ctx)
+    return Basis(desc, data, scales)
+
+
+def twa_basis_export(ctx, Pq):
+    """Canonical codes (n, ceil(D*bits/8)) uint8 and scales (n,) float32, on the device."""
+    row_bytes = (Pq.D * Pq.bits + 7) // 8
+    codes = torch.empty((Pq.n, row_bytes), dtype=torch.uint8, device=Pq.data.device)
+    scales = torch.empty(Pq.n, dtype=torch.float32, device=Pq.data.device)
+    rc = load().twa_basis_export(ctx, ctypes.byref(Pq.desc), _ptr(codes), _ptr(scales))
+    _check(rc, "twa_basis_export", ctx)
+    return codes, scales
+
+
+def twa_basis_import(ctx, codes, scales, D, bits):
+    n = codes.shape[0]
+    assert codes.dtype == torch.uint8 and codes.is_contiguous()
+    assert codes.shape[1] == (D * bits + 7) // 8
+    desc, data, sc = _new_quantised(D, n, bits, codes.device)
+    rc = load().twa_basis_import(ctx, _ptr(codes), _ptr(scales), int(D), int(n), int(bits),
+                                 ctypes.byref(desc))
+    _check(rc, "twa_basis_import", ctx)
+    return Basis(desc, data, sc)
+
+
+def twa_project(ctx, P, g, c_out, ws):
+    rc = load().twa_project(ctx, ctypes.byref(P.desc), _ptr(g), _dtype_code(g), _ptr(c_out),
+                            _ptr(ws), ws.numel())
+    _check(rc, "twa_project", ctx)
+    return c_out
+
+
+def twa_lift(ctx, P, alpha, base, w_out, ws):
+    rc = load().twa_lift(ctx, ctypes.byref(P.desc), _ptr(alpha), _ptr(base), _ptr(w_out),
+                         _ptr(ws), ws.numel())
+    _check(rc, "twa_lift", ctx)
+    return w_out
+
+
+def twa_step(ctx, P, g, lr, lam, alpha, wbar, w, ws, c_out=None):
+    rc = load().twa_step(ctx, ctypes.byref(P.desc), _ptr(g), _dtype_code(g), float(lr), float(lam),
+                         _ptr(alpha), _ptr(wbar), _ptr(w), _ptr(c_out), _ptr(ws), ws.numel())
+    _check(rc, "twa_step", ctx)
+    return w
+
+
+def twa_step_host(ctx, P, g_host, lr, lam, alpha, wbar, w, w_host, g_stage, ws):
+    """g_host / w_host: CPU tensors (pinned for asynchronous copies)."""
+    assert not g_host.is_cuda and not w_host.is_cuda
+    rc = load().twa_step_host(ctx, ctypes.byref(P.desc), _ptr(g_host), _dtype_code(g_host),
+                              float(lr), float(lam), _ptr(alpha), _ptr(wbar), _ptr(w),
+                              _ptr(w_host), _ptr(g_stage), _ptr(ws), ws.numel())
+    _check(rc, "twa_step_host", ctx)
+    return w_host

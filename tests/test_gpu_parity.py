@@ -1,0 +1,350 @@
+"""GPU parity: every C-ABI call against the float64 CPU oracle on the same seeded bytes.
+
+Sizes span several tiles (a tile is 512 rows at 8 bits, 1024 at 4 bits, 128 at 32 bits),
+ragged tails (D not a multiple of 2, 4, 16, 128) and the column counts 1, 2, 3, 33, 100, 128.
+Bounds: codes and scales bit-exact; projection, lift and step within 1e-5 relative L2;
+basis orthonormal to 1e-5.
+"""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import twa_oracle as orc
+from paper_2205_13104_b200 import inputs, twa
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def env():
+    torch.cuda.set_device(0)
+    ctx = twa.twa_create(0)
+    ws = twa.new_workspace(DEV)
+    yield ctx, ws
+    torch.cuda.synchronize()
+    twa.twa_destroy(ctx)
+
+
+def rel(x, y):
+    x = np.asarray(x, dtype=np.float64)
+    y = np.asarray(y, dtype=np.float64)
+    d = np.linalg.norm(y)
+    return np.linalg.norm(x - y) / d if d > 0 else np.linalg.norm(x)
+
+
+def status_ok(ctx):
+    code, detail = twa.twa_get_status(ctx)
+    assert code == 0, (twa.twa_strerror(code), detail)
+
+
+def random_basis(D, n, seed, scale=1.0):
+    """float32 matrix (n, ld) on the GPU with unit-ish columns of different magnitude."""
+    ld = inputs.padded_ld(D, 4)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(seed)
+    P = torch.zeros((n, ld), dtype=torch.float32, device=DEV)
+    P[:, :D] = torch.randn((n, D), generator=g, device=DEV) * scale / np.sqrt(D)
+    P[:, :D] *= (1.0 + torch.arange(n, device=DEV, dtype=torch.float32))[:, None] * 0.37
+    return P
+
+
+def host_cols(P, D):
+    return P[:, :D].cpu().numpy().T          # (D, n) view with contiguous columns
+
+
+SHAPES = [(1, 1), (5, 2), (127, 3), (513, 1), (1024, 2), (4099, 33), (70001, 100), (33333, 128),
+          (300007, 20)]
+
+
+# ------------------------------------------------------------------ mean
+@pytest.mark.parametrize("D,n", [(1, 1), (6, 3), (1023, 7), (40002, 33)])
+def test_mean(env, D, n):
+    ctx, _ = env
+    W = inputs.trajectory_candidates(D, n, 0.01, 0.002, 3, DEV, ld=inputs.padded_ld(D, 4))
+    wbar = torch.full((D + 8,), 7.0, dtype=torch.float32, device=DEV)
+    twa.twa_mean(ctx, W, D, wbar)
+    status_ok(ctx)
+    ref = orc.mean(host_cols(W, D)).astype(np.float32)
+    np.testing.assert_array_equal(wbar[:D].cpu().numpy(), ref)
+    assert torch.all(wbar[D:] == 7.0)            # nothing written past D
+
+
+# ------------------------------------------------------------------ quantiser
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("D,n", SHAPES)
+def test_quantize_bit_exact(env, D, n, bits):
+    ctx, ws = env
+    P = random_basis(D, n, 11 + D)
+    if n >= 3:
+        P[1].zero_()                              # an all-zero column
+        P[2, :D] = -P[2, :D].abs()                # absmax element negative
+    P32 = twa.basis_from_tensor(P, D)
+    Pq = twa.twa_quantize_basis(ctx, P32, bits, ws)
+    status_ok(ctx)
+    codes_g, s_g = twa.twa_basis_export(ctx, Pq)
+    codes_o, s_o = orc.quantize(np.asfortranarray(host_cols(P, D)), bits)
+    np.testing.assert_array_equal(s_g.cpu().numpy(), s_o)
+    np.testing.assert_array_equal(codes_g.cpu().numpy(), orc.pack_codes(codes_o, bits))
+    assert Pq.data.numel() == twa.twa_basis_bytes(D, n, bits)
+    assert codes_g.numel() + 4 * n == orc.storage_bytes(D, n, bits)
+
+
+def test_quantize_ties_round_to_even(env):
+    ctx, ws = env
+    vals = [127.0, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 3.5, -126.5, 64.5]
+    P = torch.zeros((2, 12), dtype=torch.float32, device=DEV)
+    P[0, :10] = torch.tensor(vals, device=DEV)
+    P[1, :10] = torch.tensor([7.0, 0.5, 1.5, 2.5, -3.5, -6.5, 6.5, -7.0, 4.5, 5.5], device=DEV)
+    P32 = twa.basis_from_tensor(P, 10)
+    for bits, row, want in ((8, 0, [127, 0, 2, 2, 0, -2, -2, 4, -126, 64]),
+                            (4, 1, [7, 0, 2, 2, -4, -6, 6, -7, 4, 6])):
+        Pq = twa.twa_quantize_basis(ctx, P32, bits, ws)
+        codes, s = twa.twa_basis_export(ctx, Pq)
+        got = orc.unpack_codes(codes.cpu().numpy(), 10, bits)
+        assert s[row].item() == 1.0
+        np.testing.assert_array_equal(got[:, row], want)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_export_import_roundtrip(env, bits):
+    ctx, ws = env
+    D, n = 7001, 5
+    P = random_basis(D, n, 5)
+    Pq = twa.twa_quantize_basis(ctx, twa.basis_from_tensor(P, D), bits, ws)
+    codes, s = twa.twa_basis_export(ctx, Pq)
+    Pq2 = twa.twa_basis_import(ctx, codes, s, D, bits)
+    codes2, s2 = twa.twa_basis_export(ctx, Pq2)
+    status_ok(ctx)
+    assert torch.equal(codes, codes2) and torch.equal(s, s2)
+    g = torch.randn(D, device=DEV)
+    c1 = torch.empty(n, device=DEV)
+    c2 = torch.empty(n, device=DEV)
+    twa.twa_project(ctx, Pq, g, c1, ws)
+    twa.twa_project(ctx, Pq2, g, c2, ws)
+    assert torch.equal(c1, c2)
+
+
+# ------------------------------------------------------------------ project / lift
+@pytest.mark.parametrize("gdt", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("bits", [32, 8, 4])
+@pytest.mark.parametrize("D,n", SHAPES)
+def test_project_and_lift(env, D, n, bits, gdt):
+    ctx, ws = env
+    P = random_basis(D, n, 100 + D + n)
+    P32 = twa.basis_from_tensor(P, D)
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(D * 7 + n)
+    g = (torch.randn(D + 16, generator=gen, device=DEV) * 1e-3).to(gdt)
+    g[D:] = float("nan")                           # must never be read
+    alpha = torch.randn(n, generator=gen, device=DEV)
+    base = torch.randn(D, generator=gen, device=DEV)
+    if bits == 32:
+        B = P32
+        Ph = host_cols(P, D)
+        proj = lambda gg: orc.project_f32(Ph, gg)
+        lift = lambda a, b: orc.lift_f32(Ph, a, b)
+    else:
+        B = twa.twa_quantize_basis(ctx, P32, bits, ws)
+        codes, s = twa.twa_basis_export(ctx, B)
+        co = orc.unpack_codes(codes.cpu().numpy(), D, bits)
+        so = s.cpu().numpy()
+        proj = lambda gg: orc.project(co, so, gg)
+        lift = lambda a, b: orc.lift(co, so, a, b)
+    c = torch.full((n + 4,), 3.0, device=DEV)
+    twa.twa_project(ctx, B, g[:D], c, ws)
+    status_ok(ctx)
+    c_ref = proj(g[:D].float().cpu().numpy())
+    assert rel(c[:n].cpu().numpy(), c_ref) <= TOL
+    assert torch.all(c[n:] == 3.0)
+
+    w = torch.full((D + 8,), 5.0, device=DEV)
+    twa.twa_lift(ctx, B, alpha, None, w, ws)       # P alpha alone: the meaningful bound
+    status_ok(ctx)
+    assert rel(w[:D].cpu().numpy(), lift(alpha.cpu().numpy(), None)) <= TOL
+    assert torch.all(w[D:] == 5.0)
+    twa.twa_lift(ctx, B, alpha, base, w, ws)
+    w_ref = lift(alpha.cpu().numpy(), base.cpu().numpy())
+    assert rel(w[:D].cpu().numpy(), w_ref) <= TOL
+    assert np.max(np.abs(w[:D].cpu().numpy() - w_ref.astype(np.float32))) <= 4 * np.spacing(
+        np.float32(np.max(np.abs(w_ref))))
+    # in place: base and output the same buffer
+    w2 = base.clone()
+    twa.twa_lift(ctx, B, alpha, w2, w2, ws)
+    assert torch.equal(w2, w[:D])
+
+
+@pytest.mark.parametrize("bits", [32, 8, 4])
+def test_step_sequence_and_determinism(env, bits):
+    ctx, ws = env
+    D, n, lr, lam = 50021, 24, 0.1, 0.05
+    W = inputs.trajectory_candidates(D, n, 0.005, 0.001, 9, DEV, ld=inputs.padded_ld(D, 4))
+    wbar = torch.empty(D, device=DEV)
+    P32 = twa.twa_build_basis(ctx, W, D, wbar, ws)
+    B = P32 if bits == 32 else twa.twa_quantize_basis(ctx, P32, bits, ws)
+    if bits == 32:
+        Ph = host_cols(W, D)
+        ostep = lambda g, a: orc.step_f32(Ph, g, a, wbar.cpu().numpy(), lr, lam)
+    else:
+        codes, s = twa.twa_basis_export(ctx, B)
+        co, so = orc.unpack_codes(codes.cpu().numpy(), D, bits), s.cpu().numpy()
+        ostep = lambda g, a: orc.step(co, so, g, a, wbar.cpu().numpy(), lr, lam)
+    runs = []
+    for rep in range(2):
+        alpha = torch.zeros(n, device=DEV)
+        w = torch.empty(D, device=DEV)
+        c = torch.empty(n, device=DEV)
+        a_o = np.zeros(n)
+        outs = []
+        for t in range(4):
+            g = inputs.gradient(D, 1e-3, 9, t, torch.float32, DEV)
+            twa.twa_step(ctx, B, g, lr, lam, alpha, wbar, w, ws, c_out=c)
+            status_ok(ctx)
+            if rep == 0:
+                a_o, w_o, c_o = ostep(g.cpu().numpy(), a_o)
+                assert rel(c.cpu().numpy(), c_o) <= TOL
+                assert rel(alpha.cpu().numpy(), a_o) <= TOL
+                assert rel(w.cpu().numpy(), w_o) <= TOL
+                assert rel(w.cpu().numpy().astype(np.float64) - wbar.cpu().numpy(),
+                           w_o - wbar.cpu().numpy()) <= 1e-3   # increment, carried by a float32 w
+            outs.append((alpha.clone(), w.clone(), c.clone()))
+        runs.append(outs)
+    for (a1, w1, c1), (a2, w2, c2) in zip(*runs):
+        assert torch.equal(a1, a2) and torch.equal(w1, w2) and torch.equal(c1, c2)
+
+
+def test_step_host_matches_device_step(env):
+    ctx, ws = env
+    D, n = 30011, 10
+    P = random_basis(D, n, 77)
+    B = twa.twa_quantize_basis(ctx, twa.basis_from_tensor(P, D), 8, ws)
+    wbar = torch.randn(D, device=DEV)
+    g = (torch.randn(D, device=DEV) * 1e-3).bfloat16()
+    a1 = torch.zeros(n, device=DEV)
+    a2 = torch.zeros(n, device=DEV)
+    w1 = torch.empty(D, device=DEV)
+    w2 = torch.empty(D, device=DEV)
+    twa.twa_step(ctx, B, g, 0.1, 0.0, a1, wbar, w1, ws)
+    g_host = g.cpu().pin_memory()
+    w_host = torch.empty(D, dtype=torch.float32).pin_memory()
+    g_stage = torch.empty(D, dtype=torch.bfloat16, device=DEV)
+    twa.twa_step_host(ctx, B, g_host, 0.1, 0.0, a2, wbar, w2, w_host, g_stage, ws)
+    status_ok(ctx)
+    assert torch.equal(a1, a2) and torch.equal(w1, w2) and torch.equal(w_host, w1.cpu())
+
+
+# ------------------------------------------------------------------ basis
+@pytest.mark.parametrize("D,n", [(1, 1), (130, 2), (5003, 3), (70001, 33), (200004, 100), (40001, 128)])
+def test_build_basis(env, D, n):
+    ctx, ws = env
+    if n > D:
+        pytest.skip("n <= D required")
+    W = inputs.trajectory_candidates(D, n, 0.005, 0.001, 21, DEV, ld=inputs.padded_ld(D, 4))
+    A = host_cols(W, D).copy()
+    wbar = torch.empty(D, device=DEV)
+    P32 = twa.twa_build_basis(ctx, W, D, wbar, ws)
+    status_ok(ctx)
+    assert (P32.D, P32.n, P32.bits, P32.col_stride) == (D, n, 32, 4 * W.shape[1])
+    np.testing.assert_array_equal(wbar.cpu().numpy(), orc.mean(A).astype(np.float32))
+    Pg = host_cols(W, D).astype(np.float64)
+    assert np.max(np.abs(Pg.T @ Pg - np.eye(n))) <= 1e-5
+    Q, R, bad = orc.cgs2(A)
+    assert bad is None
+    # same factorisation: P^T A upper triangular with positive diagonal, A = P (P^T A)
+    T = Pg.T @ A.astype(np.float64)
+    assert np.all(np.diag(T) > 0)
+    assert np.max(np.abs(np.tril(T, -1))) <= 2e-5 * np.max(np.abs(T))
+    assert np.linalg.norm(A - Pg @ T) <= 1e-5 * np.linalg.norm(A)
+    kappa = np.linalg.cond(A.astype(np.float64))
+    assert np.max(np.linalg.norm(Pg - Q, axis=0)) <= 10 * kappa * np.finfo(np.float32).eps
+    # pad columns untouched
+    assert torch.all(W[:, D:] == 0)
+
+
+def test_basis_invariants_recover_candidates_and_reject_orthogonal(env):
+    ctx, ws = env
+    D, n = 60013, 10
+    W = inputs.trajectory_candidates(D, n, 0.01, 0.002, 0, DEV, ld=inputs.padded_ld(D, 4))
+    A = W[:, :D].clone()
+    wbar = torch.empty(D, device=DEV)
+    P32 = twa.twa_build_basis(ctx, W, D, wbar, ws)
+    c = torch.empty(n, device=DEV)
+    w = torch.empty(D, device=DEV)
+    for i in range(n):
+        twa.twa_project(ctx, P32, A[i].clone(), c, ws)
+        twa.twa_lift(ctx, P32, c, None, w, ws)
+        assert rel(w.cpu().numpy(), A[i].cpu().numpy()) <= 1e-5          # lift(project(w_i)) = w_i
+        twa.twa_project(ctx, P32, A[i] - wbar, c, ws)
+        twa.twa_lift(ctx, P32, c, wbar, w, ws)
+        assert rel(w.cpu().numpy(), A[i].cpu().numpy()) <= 1e-5
+    # alpha = 0 lifts to w_bar exactly
+    twa.twa_lift(ctx, P32, torch.zeros(n, device=DEV), wbar, w, ws)
+    assert torch.equal(w, wbar)
+    # a vector orthogonal to the span (made so on the CPU in float64) projects to ~0
+    A64 = A.cpu().numpy().T.astype(np.float64)
+    x = np.random.default_rng(0).standard_normal(D)
+    x -= A64 @ np.linalg.lstsq(A64, x, rcond=None)[0]
+    xg = torch.tensor(x, dtype=torch.float32, device=DEV)
+    twa.twa_project(ctx, P32, xg, c, ws)
+    assert np.max(np.abs(c.cpu().numpy())) <= 1e-5 * np.linalg.norm(x)
+    status_ok(ctx)
+
+
+def test_rank_deficient_and_nonfinite_are_reported(env):
+    ctx, ws = env
+    D, n = 9001, 4
+    W = inputs.trajectory_candidates(D, n, 0.01, 0.002, 1, DEV, ld=inputs.padded_ld(D, 4))
+    W[2] = W[0] * -2.0
+    wbar = torch.empty(D, device=DEV)
+    twa.twa_build_basis(ctx, W, D, wbar, ws)
+    code, detail = twa.twa_get_status(ctx)
+    assert (code, detail) == (twa.TWA_ERR_RANK_DEFICIENT, 2)
+    twa.twa_clear_status(ctx)
+    status_ok(ctx)
+    W = inputs.trajectory_candidates(D, n, 0.01, 0.002, 1, DEV, ld=inputs.padded_ld(D, 4))
+    W[1, 17] = float("inf")
+    twa.twa_build_basis(ctx, W, D, wbar, ws)
+    code, detail = twa.twa_get_status(ctx)
+    assert (code, detail) == (twa.TWA_ERR_NONFINITE, 1)
+    twa.twa_clear_status(ctx)
+    P = random_basis(D, n, 3)
+    P[3, 5] = float("nan")
+    twa.twa_quantize_basis(ctx, twa.basis_from_tensor(P, D), 8, ws)
+    code, detail = twa.twa_get_status(ctx)
+    assert (code, detail) == (twa.TWA_ERR_NONFINITE, 3)
+    twa.twa_clear_status(ctx)
+    status_ok(ctx)
+
+
+def test_host_side_argument_errors(env):
+    ctx, ws = env
+    D, n = 1000, 4
+    P = random_basis(D, n, 1)
+    P32 = twa.basis_from_tensor(P, D)
+    g = torch.zeros(D + 4, device=DEV)
+    c = torch.zeros(n, device=DEV)
+
+    def code_of(fn):
+        with pytest.raises(twa.TwaError) as e:
+            fn()
+        return e.value.code
+
+    assert code_of(lambda: twa.twa_project(ctx, P32, g[1:D + 1], c, ws)) == twa.TWA_ERR_MISALIGNED
+    assert code_of(lambda: twa.twa_project(ctx, P32, g[:D], c, ws[:16])) == twa.TWA_ERR_WORKSPACE
+    assert code_of(lambda: twa.twa_quantize_basis(ctx, P32, 5, ws)) == twa.TWA_ERR_UNSUPPORTED
+    bad = twa.basis_from_tensor(P, D)
+    bad.desc.n = 0
+    assert code_of(lambda: twa.twa_project(ctx, bad, g[:D], c, ws)) == twa.TWA_ERR_INVALID_ARG
+    bad.desc.n = twa.TWA_MAX_N + 1
+    assert code_of(lambda: twa.twa_project(ctx, bad, g[:D], c, ws)) == twa.TWA_ERR_UNSUPPORTED
+    bad.desc.n = n
+    bad.desc.col_stride = 4 * D - 8
+    assert code_of(lambda: twa.twa_project(ctx, bad, g[:D], c, ws)) in (
+        twa.TWA_ERR_MISALIGNED, twa.TWA_ERR_INVALID_ARG)
+    wide = torch.zeros((twa.TWA_MAX_N + 1, 16), device=DEV)
+    assert code_of(lambda: twa.twa_build_basis(ctx, wide, 16, torch.zeros(16, device=DEV), ws)) == \
+        twa.TWA_ERR_UNSUPPORTED
+    status_ok(ctx)
