@@ -197,6 +197,37 @@ int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host /* host *
                   twa_dtype g_dtype, float lr, float lambda, float* alpha, const float* wbar,
                   float* w, float* w_host /* host */, void* g_stage, void* ws, size_t ws_bytes);
 
+/* ---- projection without any allocation ----------------------------------------------- */
+
+/* (No counterpart in the paper: this entry point exists for the way some programs manage
+ * GPU memory, not for the method.)
+ *
+ * c_out[j] = s_j * sum_r code[r,j] * g[r], exactly as twa_project, for callers that cannot
+ * allocate device memory at the point of the call: a program whose caching allocator owns
+ * the whole device, a loop that may not make calls which can synchronise the device, a
+ * plug-in that is handed its input and output buffers and nothing else.  It takes no
+ * context (twa_create allocates) and no workspace: the per-block partial sums, the
+ * completion counter and the status word live in one fixed array of
+ * twa_noalloc_scratch_bytes() = 131,328 bytes inside the library's device image, which every
+ * GPU that loads the library holds until the process exits.  The call itself makes no
+ * cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ *  device, cuda_stream  where to run (cudaStream_t as void*, NULL = legacy default stream).
+ *  P, g, g_dtype, c_out as for twa_project; the caller still owns inputs and outputs.
+ *  status_out           device, 2 ints, or NULL: receives {TWA_OK or the device-side error,
+ *                       detail} when the kernel has run.
+ * Limits: n <= TWA_MAX_N (128) columns and at most 256 blocks of partial sums; a larger n is
+ * rejected with TWA_ERR_UNSUPPORTED and a message in twa_noalloc_last_error().
+ * The first call on a device looks up the device address of the array and the driver entry
+ * point it needs; make that first call before any stream capture begins.
+ * All calls on one device share the array: the call clears the counter and the status on the
+ * stream before the kernel, and calls that overlap on the GPU (different streams, or
+ * different host threads without ordering) race on it -- serialise them. */
+int twa_project_noalloc(int device, void* cuda_stream, const twa_basis* P, const void* g,
+                        twa_dtype g_dtype, float* c_out, int* status_out);
+const char* twa_noalloc_last_error(void);
+size_t twa_noalloc_scratch_bytes(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libtwa.so")
 CSRC = os.path.join(_HERE, "csrc")
-SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_stream.cu"]
+SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_stream.cu", "twa_noalloc.cu"]
 
 TWA_MAX_N = 128
 TWA_OK = 0
@@ -41,7 +41,7 @@ EXPORTS = [
     "twa_basis_col_stride", "twa_basis_bytes",
     "twa_workspace_bytes", "twa_build_basis", "twa_mean", "twa_quantize_basis",
     "twa_basis_export", "twa_basis_import", "twa_project", "twa_lift", "twa_step",
-    "twa_step_host",
+    "twa_step_host", "twa_project_noalloc", "twa_noalloc_last_error", "twa_noalloc_scratch_bytes",
 ]
 
 
@@ -120,6 +120,9 @@ def load():
         "twa_lift": (i32, [vp, bp, vp, vp, vp, vp, szt]),
         "twa_step": (i32, [vp, bp, vp, i32, f32, f32, vp, vp, vp, vp, vp, szt]),
         "twa_step_host": (i32, [vp, bp, vp, i32, f32, f32, vp, vp, vp, vp, vp, vp, szt]),
+        "twa_project_noalloc": (i32, [i32, vp, bp, vp, i32, vp, vp]),
+        "twa_noalloc_last_error": (ctypes.c_char_p, []),
+        "twa_noalloc_scratch_bytes": (szt, []),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -328,3 +331,25 @@ def twa_step_host(ctx, P, g_host, lr, lam, alpha, wbar, w, w_host, g_stage, ws):
                               _ptr(w_host), _ptr(g_stage), _ptr(ws), ws.numel())
     _check(rc, "twa_step_host", ctx)
     return w_host
+
+
+def twa_noalloc_last_error():
+    return load().twa_noalloc_last_error().decode()
+
+
+def twa_noalloc_scratch_bytes():
+    return int(load().twa_noalloc_scratch_bytes())
+
+
+def twa_project_noalloc(device, stream, P, g, c_out, status_out=None):
+    """Projection that needs neither a context nor a workspace: for callers that cannot
+    allocate device memory when they call (see include/twa.h).  `stream` is a
+    torch.cuda.Stream or None for the current one; status_out an int32 CUDA tensor of 2."""
+    if stream is None:
+        stream = torch.cuda.current_stream(device)
+    rc = load().twa_project_noalloc(int(device), ctypes.c_void_p(stream.cuda_stream),
+                                    ctypes.byref(P.desc), _ptr(g), _dtype_code(g), _ptr(c_out),
+                                    _ptr(status_out))
+    if rc != TWA_OK:
+        raise TwaError(rc, "twa_project_noalloc", twa_noalloc_last_error())
+    return c_out
