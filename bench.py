@@ -67,7 +67,7 @@ class ClockSampler:
             self.out = open(self.path, "w")
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=self.out, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -181,19 +181,31 @@ def run_ours(args):
 
     twa.load()
     wl = inputs.WORKLOADS[args.workload]
+    if args.rows:
+        import dataclasses
+        wl = dataclasses.replace(wl, name=f"{wl.name}[rows={args.rows}]", D=args.rows)
     D, n, bits = wl.D, wl.n, args.bits
     gdt = torch.bfloat16 if wl.g_dtype == "bf16" else torch.float32
     g_bytes = 2 if wl.g_dtype == "bf16" else 4
     ctx = twa.twa_create(local)
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_DEQUANT_PATH, args.dequant_path)
     ws = twa.new_workspace(dev)
 
     # ---- basis build and quantisation, timed once each -------------------------------
-    W = wl.candidates(dev, ld=inputs.padded_ld(D, 128))
     wbar = torch.empty(D, dtype=torch.float32, device=dev)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-    torch.cuda.synchronize()
-    ev[0].record()
-    P32 = twa.twa_build_basis(ctx, W, D, wbar, ws)
+    if args.random_basis:
+        # profiling aid: skip the Gram-Schmidt launches; the step kernels do the same work on any values
+        W = torch.randn((n, inputs.padded_ld(D, 128)), device=dev) / (D ** 0.5)
+        twa.twa_mean(ctx, W, D, wbar)
+        torch.cuda.synchronize()
+        ev[0].record()
+        P32 = twa.basis_from_tensor(W, D)
+    else:
+        W = wl.candidates(dev, ld=inputs.padded_ld(D, 128))
+        torch.cuda.synchronize()
+        ev[0].record()
+        P32 = twa.twa_build_basis(ctx, W, D, wbar, ws)
     ev[1].record()
     Pq = twa.twa_quantize_basis(ctx, P32, bits, ws) if bits != 32 else P32
     ev[2].record()
@@ -268,6 +280,7 @@ def run_ours(args):
         kb = kernel_bytes(D, n, bits, g_bytes)
         ms_per_step = total_ms / args.steps
         value = world * sb / (ms_per_step * 1e-3) / 1e9
+        suffix = "_mma" if args.dequant_path == 0 and bits != 32 else ""
         dom = "project" if proj_ms >= lift_ms else "lift"
         dom_ms = (proj_ms if dom == "project" else lift_ms) / max(rec, 1)
         achieved = kb[dom] / (dom_ms * 1e-3) / 1e9
@@ -294,15 +307,16 @@ def run_ours(args):
             "config": {"workload": f"{wl.name}: D={D} n={n} int{bits} P, {wl.g_dtype} g, lr={lr} lambda={lam}",
                        "l2": f"inputs larger than L2: P~ is {n * ((D * bits + 7) // 8) / 1e6:.0f} MB per pass",
                        "gradients": f"{len(pool)} distinct gradients generated before the timed region, cycled",
+                       "dequant_path": "tensor-pipe integer dot products" if args.dequant_path == 0 else "float32 FMA",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "bytes_per_step": sb,
             "frac_of_hbm_peak": value / world / peak,
             "frac_of_8TBps": value / world / 8000.0,
-            "basis_build_ms": build_ms, "quantize_ms": quant_ms,
-            "roofline": {"bound": "hbm", "kernel": f"twa_{dom}_kernel", "achieved": achieved, "peak": peak,
+            "basis_build_ms": None if args.random_basis else build_ms, "quantize_ms": quant_ms,
+            "roofline": {"bound": "hbm", "kernel": f"twa_{dom}{suffix}_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "traffic": traffic, "bytes_per_launch": kb[dom], "ms_per_launch": dom_ms,
-                         "other_kernel": {"kernel": f"twa_{other}_kernel", "ms_per_launch": other_ms,
+                         "other_kernel": {"kernel": f"twa_{other}{suffix}_kernel", "ms_per_launch": other_ms,
                                           "achieved": kb[other] / (other_ms * 1e-3) / 1e9,
                                           "bytes_per_launch": kb[other]}},
             "cpu_baseline": cpu,
@@ -321,7 +335,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vitb16")
@@ -330,6 +344,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--reference-rows", type=int, default=1 << 21)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dequant-path", type=int, default=0, choices=[0, 1],
+                    help="0: integer dot products on the tensor pipe (default); 1: float32 FMA path")
+    ap.add_argument("--rows", type=int, default=0, help="override D (smaller cases for profiler captures)")
+    ap.add_argument("--random-basis", action="store_true",
+                    help="profiling aid: quantise a random matrix instead of building the basis")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -70,9 +70,12 @@ typedef struct twa_ctx twa_ctx;
  *  bits == 4 : two elements per byte, row 2k in the low nibble and row 2k+1 in the high
  *              nibble, nibble = code + 8, code in [-7,7].
  *  The represented value is scales[j] * code (Section 4.6, with one symmetric factor per
- *  column instead of two per layer).  The storage of codes is internal to the library;
- *  twa_basis_export / twa_basis_import convert to and from the canonical two's-complement
- *  image.  Bytes of a column beyond ceil(D*bits/8) up to col_stride are padding. */
+ *  column instead of two per layer).  The storage of codes is internal to the library: inside
+ *  every aligned 512-byte segment of a column the 16-byte chunks are stored in a
+ *  column-dependent order (conflict-free shared-memory reads), so only the library should
+ *  produce or read `data` for bits 8 and 4; twa_basis_export / twa_basis_import convert to
+ *  and from the canonical two's-complement image.  Bytes of a column beyond ceil(D*bits/8)
+ *  up to col_stride are padding. */
 typedef struct {
   void* data;         /* device, 16-byte aligned, n * col_stride bytes                 */
   float* scales;      /* device, n floats; ignored when bits == 32                     */
@@ -101,9 +104,13 @@ const char* twa_last_error(const twa_ctx* ctx);
 /* Tuning knobs for measurements; value 0 restores the built-in choice.
  *  TWA_TUNE_PROJECT_WARPS / TWA_TUNE_LIFT_WARPS: consumer warps per block (8..20; lift: even, >= 16)
  *  TWA_TUNE_STAGES: depth of the shared-memory ring (2..16)
- *  TWA_TUNE_WAIT_LIMIT_MS: bound of every in-kernel wait (default 2000 ms)             */
+ *  TWA_TUNE_WAIT_LIMIT_MS: bound of every in-kernel wait (default 2000 ms)
+ *  TWA_TUNE_DEQUANT_PATH: how 8/4-bit codes meet g and alpha: 0 = exact integer dot products
+ *      on the tensor pipe against block-fixed-point digits of g / alpha (default),
+ *      1 = code -> float32 conversion and float32 FMA.  The warp and stage knobs act on the
+ *      float path and on 32-bit bases only.                                             */
 enum { TWA_TUNE_PROJECT_WARPS = 1, TWA_TUNE_LIFT_WARPS = 2, TWA_TUNE_STAGES = 3,
-       TWA_TUNE_WAIT_LIMIT_MS = 4 };
+       TWA_TUNE_WAIT_LIMIT_MS = 4, TWA_TUNE_DEQUANT_PATH = 5 };
 int twa_set_tuning(twa_ctx* ctx, int key, int value);
 
 /* Per-kernel timing of twa_step for measurements.  twa_profile_enable(ctx, max_steps > 0)
@@ -117,8 +124,8 @@ int twa_profile_read(twa_ctx* ctx, double* project_ms, double* lift_ms, int* ste
 
 /* ---- sizes -------------------------------------------------------------------------- */
 
-/* Bytes between columns the library uses for a D-row basis of the given width
- * (ceil(D*bits/8) rounded up to 128). */
+/* Bytes between columns the library uses for a D-row basis of the given width:
+ * ceil(D*bits/8) rounded up to 512 for bits 8 and 4, to 128 for bits 32. */
 int64_t twa_basis_col_stride(int64_t D, int bits);
 /* n * twa_basis_col_stride: size of the `data` buffer the caller must provide. */
 size_t twa_basis_bytes(int64_t D, int n, int bits);

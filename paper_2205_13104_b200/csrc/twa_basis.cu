@@ -195,21 +195,40 @@ __global__ void __launch_bounds__(BLOCK) encode_kernel(const float* __restrict__
       if (BITS == 8) w[k >> 2] |= u << (8 * (k & 3));
       else w[k >> 3] |= u << (4 * (k & 7));
     }
-    dst[q] = make_uint4(w[0], w[1], w[2], w[3]);
+    dst[(q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j)] = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
 
-// internal (offset binary, padded) <-> canonical (two's complement, tight)
-__global__ void __launch_bounds__(BLOCK) recode_kernel(const unsigned char* __restrict__ in,
+// Position of logical byte b of column j in the internal (chunk-permuted) order.
+__device__ __forceinline__ long long internal_pos(long long b, int j) {
+  const long long q = b >> 4;
+  return (((q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j)) << 4) | (b & 15);
+}
+
+// internal (offset binary, chunk-permuted, padded) -> canonical (two's complement, tight)
+__global__ void __launch_bounds__(BLOCK) export_kernel(const unsigned char* __restrict__ in,
                                                        long long in_stride,
                                                        unsigned char* __restrict__ out,
-                                                       long long out_stride, long long row_bytes,
-                                                       long long fill_to, unsigned char mask) {
-  const unsigned char* src = in + blockIdx.y * in_stride;
-  unsigned char* dst = out + blockIdx.y * out_stride;
-  for (long long b = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; b < fill_to;
+                                                       long long row_bytes, unsigned char mask) {
+  const int j = blockIdx.y;
+  const unsigned char* src = in + j * in_stride;
+  unsigned char* dst = out + j * row_bytes;
+  for (long long b = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; b < row_bytes;
        b += static_cast<long long>(gridDim.x) * BLOCK)
-    dst[b] = (b < row_bytes) ? static_cast<unsigned char>(src[b] ^ mask) : mask;
+    dst[b] = static_cast<unsigned char>(src[internal_pos(b, j)] ^ mask);
+}
+
+// canonical -> internal; bytes between the end of the column and the stride get the code 0
+__global__ void __launch_bounds__(BLOCK) import_kernel(const unsigned char* __restrict__ in,
+                                                       long long row_bytes,
+                                                       unsigned char* __restrict__ out,
+                                                       long long out_stride, unsigned char mask) {
+  const int j = blockIdx.y;
+  const unsigned char* src = in + j * row_bytes;
+  unsigned char* dst = out + j * out_stride;
+  for (long long b = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; b < out_stride;
+       b += static_cast<long long>(gridDim.x) * BLOCK)
+    dst[internal_pos(b, j)] = (b < row_bytes) ? static_cast<unsigned char>(src[b] ^ mask) : mask;
 }
 
 int grid_for(const twa_ctx* ctx, long long items, int per_block, int blocks_per_sm) {
@@ -238,7 +257,8 @@ extern "C" {
 int64_t twa_basis_col_stride(int64_t D, int bits) {
   if (D < 1 || (bits != 32 && bits != 8 && bits != 4)) return 0;
   const int64_t row_bytes = (D * bits + 7) / 8;
-  return (row_bytes + 127) / 128 * 128;
+  if (bits == 32) return (row_bytes + 127) / 128 * 128;
+  return (row_bytes + 511) / 512 * 512;      // whole 512-byte segments: see twa_chunk_slot
 }
 
 size_t twa_basis_bytes(int64_t D, int n, int bits) {
@@ -354,10 +374,9 @@ int twa_basis_export(twa_ctx* ctx, const twa_basis* Pq, void* codes_out, float* 
   const long long row_bytes = (Pq->D * Pq->bits + 7) / 8;
   int per = grid_for(ctx, row_bytes, BLOCK * 8, 8) / Pq->n;
   if (per < 1) per = 1;
-  recode_kernel<<<dim3(per, Pq->n), BLOCK, 0, ctx->stream>>>(
+  export_kernel<<<dim3(per, Pq->n), BLOCK, 0, ctx->stream>>>(
       static_cast<const unsigned char*>(Pq->data), Pq->col_stride,
-      static_cast<unsigned char*>(codes_out), row_bytes, row_bytes, row_bytes,
-      Pq->bits == 8 ? 0x80 : 0x88);
+      static_cast<unsigned char*>(codes_out), row_bytes, Pq->bits == 8 ? 0x80 : 0x88);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   TWA_CUDA_OK(ctx, cudaMemcpyAsync(scales_out, Pq->scales, sizeof(float) * Pq->n,
                                    cudaMemcpyDeviceToDevice, ctx->stream));
@@ -376,9 +395,9 @@ int twa_basis_import(twa_ctx* ctx, const void* codes, const float* scales, int64
   const long long stride = twa_basis_col_stride(D, bits);
   int per = grid_for(ctx, stride, BLOCK * 8, 8) / n;
   if (per < 1) per = 1;
-  recode_kernel<<<dim3(per, n), BLOCK, 0, ctx->stream>>>(
+  import_kernel<<<dim3(per, n), BLOCK, 0, ctx->stream>>>(
       static_cast<const unsigned char*>(codes), row_bytes, static_cast<unsigned char*>(Pq->data),
-      stride, row_bytes, stride, bits == 8 ? 0x80 : 0x88);
+      stride, bits == 8 ? 0x80 : 0x88);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   TWA_CUDA_OK(ctx, cudaMemcpyAsync(Pq->scales, scales, sizeof(float) * n, cudaMemcpyDeviceToDevice,
                                    ctx->stream));

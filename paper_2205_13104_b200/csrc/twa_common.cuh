@@ -27,6 +27,7 @@ struct twa_ctx {
   twa_encode_tiled_fn encode_tiled;
   unsigned long long wait_limit_ns;
   int tune_project_warps, tune_lift_warps, tune_stages;
+  int tune_dequant_path;      // 0 = integer tensor-pipe dot products, 1 = float FMA
   cudaEvent_t* prof_events;   // 3 per recorded step, or null
   int prof_cap, prof_count;   // steps
   char last_error[256];
@@ -70,6 +71,28 @@ constexpr int TWA_SMEM_HEADER = 2048;                    // barriers + small arr
 
 // rows covered by one tile for a storage width
 __host__ __device__ constexpr int twa_tile_rows(int bits) { return TWA_TILE_COL_BYTES * 8 / bits; }
+
+// Storage order of 8- and 4-bit codes inside a column.  Every aligned 512-byte segment of a
+// column holds its 32 chunks of 16 bytes permuted: logical chunk c sits in slot
+// (c & 24) | ((c ^ j) & 7), j the column index.  In shared memory, where a tile is
+// [n columns][512 bytes], the same chunk of eight neighbouring columns then falls into eight
+// different bank groups, so 8 x 16-byte matrix loads across columns are conflict-free, while
+// global memory and the TMA copies keep 512 contiguous bytes per column and tile.
+__host__ __device__ __forceinline__ int twa_chunk_slot(int c, int j) { return (c & 24) | ((c ^ j) & 7); }
+
+// First bytes of every streaming kernel's shared memory.
+struct twa_smem_header {
+  unsigned long long full[TWA_MAX_STAGES];    // stage filled by the producer's copies
+  unsigned long long empty[TWA_MAX_STAGES];   // stage released by every consumer warp
+  int abort_flag;                             // a bounded wait ran out somewhere in the block
+  int last_flag;                              // this block finished last (project)
+  int bad_flag;                               // non-finite input met
+  unsigned amax_bits;                         // lift: bit pattern of max |coefficient|
+  float digit_scale[4];                       // lift: weight of each coefficient digit
+  int pad[54];
+  float c_part[TWA_MAX_N];                    // project: this block's column sums
+};
+static_assert(sizeof(twa_smem_header) <= TWA_SMEM_HEADER, "header too large");
 
 // ------------------------------------------------------------------------------------------
 // Device helpers
@@ -193,3 +216,11 @@ int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtyp
 int twa_launch_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
                     const float* base, float* out, bool reverse_tiles);
 int twa_check_basis(const twa_basis* P);
+// Variants of the two launchers for 8- and 4-bit storage that compute the integer dot
+// products on the tensor pipe (twa_stream_mma.cu).
+int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
+                           const twa_project_epilogue& epi, void* ws);
+int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
+                        const float* base, float* out, bool reverse_tiles);
+// Sets the dynamic shared memory limit of a kernel only when it has to grow.
+int twa_ensure_smem(twa_ctx* ctx, const void* kernel, int* current, int wanted);

@@ -41,15 +41,7 @@ struct LiftArgs {
   unsigned long long wait_limit_ns;
 };
 
-struct SmemHeader {
-  unsigned long long full[TWA_MAX_STAGES];
-  unsigned long long empty[TWA_MAX_STAGES];
-  int abort_flag;
-  int last_flag;
-  int pad[62];
-  float c_part[TWA_MAX_N];
-};
-static_assert(sizeof(SmemHeader) <= TWA_SMEM_HEADER, "header too large");
+using SmemHeader = twa_smem_header;
 
 // Producer loop shared by both kernels.  G_BOXES 1-D boxes of the gradient follow the tile
 // of P~ in the same stage (project only).
@@ -222,7 +214,8 @@ twa_project_kernel(const __grid_constant__ CUtensorMap map_p,
       for (int k = 0; k < TWA_PROJECT_CPW; ++k) {
         if (k < cpw) {
           const int j = warp + k * W;
-          acc[k] += lane_dot<BITS>(st + j * TWA_TILE_COL_BYTES + lane * 16, g);
+          const int slot = BITS == 32 ? lane : twa_chunk_slot(lane, j);
+          acc[k] += lane_dot<BITS>(st + j * TWA_TILE_COL_BYTES + slot * 16, g);
         }
       }
       __syncwarp();
@@ -370,10 +363,14 @@ twa_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LiftArgs a) {
     for (int i = 0; i < LR; ++i) acc[i] = 0.0f;
     const bool ok = twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns);
     if (ok) {
-      const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes + byte_off;
+      const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
 #pragma unroll
       for (int k = 0; k < TWA_LIFT_CPW; ++k) {
-        if (k < cpw) lane_axpy<BITS, LR>(st + (cg + k * CG) * TWA_TILE_COL_BYTES, coef[k], acc);
+        if (k < cpw) {
+          const int j = cg + k * CG;
+          const int off = BITS == 32 ? byte_off : (twa_chunk_slot(byte_off >> 4, j) << 4) | (byte_off & 15);
+          lane_axpy<BITS, LR>(st + j * TWA_TILE_COL_BYTES + off, coef[k], acc);
+        }
       }
       __syncwarp();
       if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
@@ -405,7 +402,9 @@ twa_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LiftArgs a) {
 int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
 int encode_basis_map(twa_ctx* ctx, const twa_basis* P, CUtensorMap* map) {
-  const long long row_bytes = (P->D * P->bits + 7) / 8;
+  long long row_bytes = (P->D * P->bits + 7) / 8;
+  // quantised columns are stored in whole, internally permuted 512-byte segments
+  if (P->bits != 32) row_bytes = (row_bytes + 511) / 512 * 512;
   cuuint64_t dims[2] = {static_cast<cuuint64_t>((row_bytes + 3) / 4), static_cast<cuuint64_t>(P->n)};
   cuuint64_t strides[1] = {static_cast<cuuint64_t>(P->col_stride)};
   cuuint32_t box[2] = {TWA_TILE_COL_WORDS, static_cast<cuuint32_t>(P->n)};
@@ -491,7 +490,9 @@ template <int BITS, bool GBF16>
 int launch_project_t(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg, const ProjectArgs& a,
                      int grid, int smem) {
   auto kern = twa_project_kernel<BITS, GBF16>;
-  TWA_CUDA_OK(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  static int smem_limit[64] = {0};   // per device
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[ctx->device & 63], smem);
+  if (rc) return rc;
   kern<<<grid, (a.warps + 1) * 32, smem, ctx->stream>>>(mp, mg, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
@@ -500,13 +501,23 @@ int launch_project_t(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg,
 template <int BITS>
 int launch_lift_t(twa_ctx* ctx, const CUtensorMap& mp, const LiftArgs& a, int grid, int smem) {
   auto kern = twa_lift_kernel<BITS>;
-  TWA_CUDA_OK(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  static int smem_limit[64] = {0};   // per device
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[ctx->device & 63], smem);
+  if (rc) return rc;
   kern<<<grid, (a.warps + 1) * 32, smem, ctx->stream>>>(mp, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
 }
 
 }  // namespace
+
+int twa_ensure_smem(twa_ctx* ctx, const void* kernel, int* current, int wanted) {
+  if (wanted > *current) {
+    TWA_CUDA_OK(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, wanted));
+    *current = wanted;
+  }
+  return TWA_OK;
+}
 
 int twa_check_basis(const twa_basis* P) {
   if (!P || !P->data) return TWA_ERR_INVALID_ARG;
@@ -516,11 +527,14 @@ int twa_check_basis(const twa_basis* P) {
   if (P->bits != 32 && !P->scales) return TWA_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(P->data) & 15) || (P->col_stride & 15)) return TWA_ERR_MISALIGNED;
   if (P->col_stride < (P->D * P->bits + 7) / 8) return TWA_ERR_INVALID_ARG;
+  if (P->bits != 32 && (P->col_stride & 511)) return TWA_ERR_MISALIGNED;   // whole 512-byte segments
   return TWA_OK;
 }
 
 int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
                        const twa_project_epilogue& epi, void* ws) {
+  if (P->bits != 32 && ctx->tune_dequant_path == 0)
+    return twa_launch_project_mma(ctx, P, g, g_dtype, epi, ws);
   const bool bf16 = g_dtype == TWA_BF16;
   const int rows = twa_tile_rows(P->bits);
   const int gsz = bf16 ? 2 : 4;
@@ -569,6 +583,8 @@ int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtyp
 
 int twa_launch_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
                     const float* base, float* out, bool reverse_tiles) {
+  if (P->bits != 32 && ctx->tune_dequant_path == 0)
+    return twa_launch_lift_mma(ctx, P, alpha, alpha_mult, base, out, reverse_tiles);
   const int rows = twa_tile_rows(P->bits);
   CUtensorMap mp;
   int rc = encode_basis_map(ctx, P, &mp);

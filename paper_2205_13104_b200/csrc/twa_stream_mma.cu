@@ -1,0 +1,695 @@
+// Projection and lift for 8- and 4-bit bases with the code x value products done as exact
+// integer dot products on the tensor pipe (Section 4.2 / 4.3 of the paper; loop body of
+// Algorithm 1; storage of Section 4.6).
+//
+// Why: the streams are HBM-bound only if the SM keeps up.  Turning every code into a float
+// costs three issue slots per code (byte permute, subtract, FMA) plus the compiler's register
+// traffic, which measured 5.7 instructions per code and 80 % issue utilisation at 60 % of DRAM
+// throughput.  Here the codes go from shared memory to the tensor pipe as they are:
+//
+//   project:  g is cut, per 32 (8-bit) or 64 (4-bit) rows, into four signed base-128 digits of a
+//             common power-of-two scale (block fixed point, 2^-29 of the block maximum, finer
+//             than float32 relative to the block), and  sum_r code[r,j] * digit_k[r]  is one
+//             integer MMA per 16 columns; the four digit sums are recombined in float32.
+//   lift:     the n coefficients s_j * alpha_j are cut into digits once per kernel, and
+//             sum_j code[r,j] * digit_k[j]  is an integer MMA per 16 rows and 32 columns.
+//
+// Integer sums are exact, so the results do not depend on the order of accumulation; the only
+// roundings are the digit cut (absolute, 2^-29 of the block maximum), the float32 recombination
+// and the float32 accumulation across tiles, which runs in a fixed order.
+//
+// Data movement is the same as in the float path (twa_stream.cu): persistent blocks, one
+// producer lane issuing TMA copies into a ring of stages, full/empty mbarriers with bounded
+// waits.  A tile is [n columns][512 bytes] in shared memory, one TMA box per stage; the 16-byte
+// chunks of a column are stored permuted (twa_chunk_slot) so that ldmatrix reads of eight
+// neighbouring columns hit eight different bank groups.
+// Warp w of the 16 consumer warps owns bytes [32w, 32w+32) of every column of a tile; warps
+// never wait for one another inside the tile loop.
+#include <stdio.h>
+
+#include "twa_common.cuh"
+
+namespace {
+
+constexpr int MMA_WARPS = 16;
+constexpr int MMA_THREADS = (MMA_WARPS + 1) * 32;
+constexpr int DIGIT_SCRATCH = 256;             // bytes of digit scratch per warp
+constexpr float RND = 12582912.0f;             // 2^23 + 2^22: x + RND rounds x to an integer (ties to even)
+
+struct ProjectMmaArgs {
+  long long D;
+  int n, stages, tiles;
+  unsigned stage_bytes, g_off, tx_bytes, scratch_off;
+  const float* scales;
+  float* partials;
+  unsigned* ticket;
+  int* status;
+  float* c_out;
+  float* alpha;
+  float lr, lambda;
+  int nonfinite_detail;
+  unsigned long long wait_limit_ns;
+};
+
+struct LiftMmaArgs {
+  long long D;
+  int n, stages, tiles;
+  unsigned stage_bytes, tx_bytes, table_off;
+  const float* scales;
+  const float* alpha;
+  float alpha_mult;
+  const float* base;
+  float* out;
+  int reverse;
+  int* status;
+  unsigned long long wait_limit_ns;
+};
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+
+// d += a (16 x 32, s8) * b (32 x 8, s8), int32 accumulation
+__device__ __forceinline__ void mma_s8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// |v| < 2^22 -> float, exactly, without the conversion unit
+__device__ __forceinline__ float small_int_to_float(int v) {
+  return __int_as_float(0x4B400000 + v) - RND;
+}
+
+// Four signed base-128 digits of t (|t| <= 64): t = d0 + d1/128 + d2/128^2 + d3/128^3 + eps,
+// |eps| <= 2^-22, every digit in [-64, 64].  Returned packed, digit k in byte k.
+__device__ __forceinline__ uint32_t cut_digits(float t) {
+  const float m0 = t + RND;
+  t = (t - (m0 - RND)) * 128.0f;
+  const float m1 = t + RND;
+  t = (t - (m1 - RND)) * 128.0f;
+  const float m2 = t + RND;
+  t = (t - (m2 - RND)) * 128.0f;
+  const float m3 = t + RND;
+  const uint32_t lo = __byte_perm(__float_as_uint(m0), __float_as_uint(m1), 0x0040);  // bytes m0.b0, m1.b0
+  const uint32_t hi = __byte_perm(__float_as_uint(m2), __float_as_uint(m3), 0x0040);
+  return __byte_perm(lo, hi, 0x5410);
+}
+
+// Shared address of logical 16-byte chunk `chunk` (0..31) of column j of a tile.
+__device__ __forceinline__ uint32_t chunk_addr(uint32_t tile_base, int j, int chunk) {
+  return tile_base + static_cast<uint32_t>(j) * TWA_TILE_COL_BYTES +
+         (static_cast<uint32_t>(twa_chunk_slot(chunk, j)) << 4);
+}
+
+template <int G_BOXES, int G_BOX_ELEMS, int G_ELEM_BYTES, int ROWS>
+__device__ __forceinline__ void producer_loop_mma(twa_smem_header* hdr, unsigned char* ring,
+                                                  const CUtensorMap* map_p, const CUtensorMap* map_g,
+                                                  int tiles, int stages, unsigned stage_bytes,
+                                                  unsigned g_off, unsigned tx_bytes,
+                                                  bool reverse, int* status, unsigned long long limit) {
+  twa_prefetch_tensormap(map_p);
+  if (G_BOXES > 0) twa_prefetch_tensormap(map_g);
+  volatile int* abort_flag = &hdr->abort_flag;
+  int s = 0, issued = 0;
+  unsigned phase = 0;
+  bool ok = true;
+  for (int t = blockIdx.x; t < tiles; t += gridDim.x) {
+    if (issued >= stages) {
+      if (!twa_mbar_wait(twa_smem_u32(&hdr->empty[s]), phase, abort_flag, limit)) {
+        ok = false;
+        break;
+      }
+    }
+    const int tile = reverse ? (tiles - 1 - t) : t;
+    const uint32_t fb = twa_smem_u32(&hdr->full[s]);
+    const uint32_t dst = twa_smem_u32(ring + static_cast<size_t>(s) * stage_bytes);
+    twa_mbar_expect_tx(fb, tx_bytes);
+    twa_tma_load_2d(dst, map_p, tile * TWA_TILE_COL_WORDS, 0, fb);
+#pragma unroll
+    for (int b = 0; b < G_BOXES; ++b)
+      twa_tma_load_1d(dst + g_off + b * G_BOX_ELEMS * G_ELEM_BYTES, map_g, tile * ROWS + b * G_BOX_ELEMS, fb);
+    ++issued;
+    if (++s == stages) {
+      s = 0;
+      if (issued > stages) phase ^= 1u;
+    }
+  }
+  if (!ok) {
+    twa_set_status(status, TWA_ERR_TIMEOUT, -1);
+    const int live = issued < stages ? issued : stages;
+    for (int q = 0; q < live; ++q) {      // let the copies already issued land
+      const int last = ((issued - 1 - q) / stages) * stages + q;
+      const unsigned par = static_cast<unsigned>(last / stages) & 1u;
+      const unsigned long long t0 = twa_globaltimer();
+      while (!twa_mbar_try_wait(twa_smem_u32(&hdr->full[q]), par)) {
+        if (twa_globaltimer() - t0 > limit) break;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void init_barriers(twa_smem_header* hdr, int stages) {
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      twa_mbar_init(twa_smem_u32(&hdr->full[s]), 1);
+      twa_mbar_init(twa_smem_u32(&hdr->empty[s]), MMA_WARPS);
+    }
+    hdr->abort_flag = 0;
+    hdr->last_flag = 0;
+    hdr->bad_flag = 0;
+    hdr->amax_bits = 0;
+    twa_fence_barrier_init();
+  }
+}
+
+// =================================================================================================
+// project
+// =================================================================================================
+template <int BITS, bool GBF16>
+__global__ void __launch_bounds__(MMA_THREADS, 1)
+twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
+                       const __grid_constant__ CUtensorMap map_g, const ProjectMmaArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  // stages start on 1024-byte boundaries (TMA destinations need 128)
+  unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
+  constexpr int ROWS = twa_tile_rows(BITS);            // 512 or 1024 rows per tile
+  constexpr int WROWS = ROWS / MMA_WARPS;              // 32 or 64 rows per warp
+  constexpr int GSZ = GBF16 ? 2 : 4;
+  constexpr int GBOX = 256;
+  twa_smem_header* hdr = reinterpret_cast<twa_smem_header*>(smem);
+  unsigned char* ring = smem + TWA_SMEM_HEADER;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gid = lane >> 2, tig = lane & 3;
+
+  init_barriers(hdr, a.stages);
+  if (threadIdx.x < TWA_MAX_N) hdr->c_part[threadIdx.x] = 0.0f;
+  __syncthreads();
+
+  const int MT = (a.n + 15) >> 4;                      // 16-column groups
+  float facc[8][2];
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) facc[mt][0] = facc[mt][1] = 0.0f;
+
+  if (warp == MMA_WARPS) {
+    if (lane == 0)
+      producer_loop_mma<ROWS / GBOX, GBOX, GSZ, ROWS>(hdr, ring, &map_p, &map_g, a.tiles, a.stages,
+                                                      a.stage_bytes, a.g_off, a.tx_bytes,
+                                                      false, a.status, a.wait_limit_ns);
+  } else {
+    unsigned char* digw = smem + a.scratch_off + warp * DIGIT_SCRATCH;   // this warp's digit bytes
+    const int c0 = warp * 2;                            // this warp's two 16-byte chunks of every column
+    const int lm = lane >> 3, lr = lane & 7;            // ldmatrix: matrix and row this lane addresses
+    const int jmax = a.n - 1;                           // last column that exists in shared memory
+    volatile int* abort_flag = &hdr->abort_flag;
+    int s = 0;
+    unsigned phase = 0;
+    bool bad = false;
+    for (int t = blockIdx.x; t < a.tiles; t += gridDim.x) {
+      if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
+        twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+        break;
+      }
+      const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
+      // ---- this warp's rows of g: 1 (8-bit) or 2 (4-bit) per lane ------------------------
+      float g0, g1 = 0.0f;
+      if (BITS == 8) {
+        if (GBF16) g0 = __uint_as_float(static_cast<uint32_t>(
+                        reinterpret_cast<const unsigned short*>(st + a.g_off)[warp * WROWS + lane]) << 16);
+        else g0 = reinterpret_cast<const float*>(st + a.g_off)[warp * WROWS + lane];
+      } else {
+        if (GBF16) {
+          const uint32_t pr = reinterpret_cast<const uint32_t*>(st + a.g_off)[warp * 32 + lane];
+          g0 = twa_bf16_lo(pr);
+          g1 = twa_bf16_hi(pr);
+        } else {
+          const float2 pr = reinterpret_cast<const float2*>(st + a.g_off)[warp * 32 + lane];
+          g0 = pr.x;
+          g1 = pr.y;
+        }
+      }
+      unsigned mb = __float_as_uint(g0) & 0x7FFFFFFFu;
+      if (BITS == 4) mb = max(mb, __float_as_uint(g1) & 0x7FFFFFFFu);
+      mb = __reduce_max_sync(0xFFFFFFFFu, mb);
+      const unsigned ebits = mb >> 23;
+      if (ebits >= 255u) bad = true;                    // NaN or Inf in g
+      // Blocks whose largest |g| is below 2^-122 contribute nothing representable: skipped.
+      if (ebits >= 5u && ebits < 255u) {
+        // |g| < 2^(ebits-126) in the block; t = g * 2^(132-ebits) lies in (-64, 64)
+        const float up = __uint_as_float((259u - ebits) << 23);
+        const uint32_t d0 = cut_digits(g0 * up);
+        // weight of digit k: 2^(ebits-132) / 128^k
+        const float w0 = (ebits >= 6u) ? __uint_as_float((ebits - 5u) << 23) : 5.877471754e-39f;
+        const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
+        float wa = tig == 0 ? w0 : (tig == 1 ? w2 : 0.0f);        // digits 2*tig, 2*tig+1 sit in this lane's
+        float wb = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);        // accumulator columns
+        if (BITS == 4) { wa *= 0.0625f; wb *= 0.0625f; }          // 4-bit codes enter the MMA times 16
+        uint32_t b0, b1, b2 = 0, b3 = 0;
+        if (BITS == 8) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) digw[k * 32 + lane] = static_cast<unsigned char>(d0 >> (8 * k));
+          __syncwarp();
+          b0 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 4 * tig) : 0u;
+          b1 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 16 + 4 * tig) : 0u;
+        } else {
+          const uint32_t d1 = cut_digits(g1 * up);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            digw[k * 32 + lane] = static_cast<unsigned char>(d0 >> (8 * k));          // even rows
+            digw[128 + k * 32 + lane] = static_cast<unsigned char>(d1 >> (8 * k));    // odd rows
+          }
+          __syncwarp();
+          b0 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 4 * tig) : 0u;
+          b1 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 16 + 4 * tig) : 0u;
+          b2 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 4 * tig) : 0u;
+          b3 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 16 + 4 * tig) : 0u;
+        }
+        const uint32_t tile_base = twa_smem_u32(st);
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          if (mt < MT) {
+            int j = mt * 16 + lr + 8 * (lm & 1);
+            j = j < jmax ? j : jmax;
+            uint32_t r[4];
+            ldmatrix_x4(chunk_addr(tile_base, j, c0 + (lm >> 1)), r);
+            int c[4] = {0, 0, 0, 0};
+            if (BITS == 8) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) r[i] ^= 0x80808080u;             // code + 128 -> code
+              mma_s8(c, r, b0, b1);
+            } else {
+              uint32_t e[4], o[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                e[i] = ((r[i] << 4) & 0xF0F0F0F0u) ^ 0x80808080u;          // even rows: 16 * code
+                o[i] = (r[i] & 0xF0F0F0F0u) ^ 0x80808080u;                 // odd rows:  16 * code
+              }
+              mma_s8(c, e, b0, b1);
+              mma_s8(c, o, b2, b3);
+            }
+            facc[mt][0] = fmaf(small_int_to_float(c[0]), wa, facc[mt][0]);
+            facc[mt][0] = fmaf(small_int_to_float(c[1]), wb, facc[mt][0]);
+            facc[mt][1] = fmaf(small_int_to_float(c[2]), wa, facc[mt][1]);
+            facc[mt][1] = fmaf(small_int_to_float(c[3]), wb, facc[mt][1]);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
+      if (++s == a.stages) {
+        s = 0;
+        phase ^= 1u;
+      }
+    }
+    if (bad) hdr->bad_flag = 1;
+  }
+  __syncthreads();                                       // every stage consumed; the ring is free
+
+  // ---- column sums of the block: lanes -> warps -> block, in a fixed order ------------------
+  float* part = reinterpret_cast<float*>(ring);         // [MMA_WARPS][TWA_MAX_N]
+  if (warp < MMA_WARPS) {
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt) {
+      float v0 = facc[mt][0], v1 = facc[mt][1];
+      v0 += __shfl_xor_sync(0xFFFFFFFFu, v0, 1);
+      v1 += __shfl_xor_sync(0xFFFFFFFFu, v1, 1);
+      v0 += __shfl_xor_sync(0xFFFFFFFFu, v0, 2);
+      v1 += __shfl_xor_sync(0xFFFFFFFFu, v1, 2);
+      if (tig == 0) {
+        part[warp * TWA_MAX_N + mt * 16 + gid] = v0;
+        part[warp * TWA_MAX_N + mt * 16 + gid + 8] = v1;
+      }
+    }
+  }
+  __syncthreads();
+  const int tid = threadIdx.x;
+  if (tid < a.n) {
+    float sum = 0.0f;
+#pragma unroll
+    for (int w = 0; w < MMA_WARPS; ++w) sum += part[w * TWA_MAX_N + tid];
+    if (hdr->bad_flag) sum = __int_as_float(0x7FC00000);
+    a.partials[static_cast<size_t>(blockIdx.x) * a.n + tid] = sum;
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned ticket = atomicAdd(a.ticket, 1u);
+    hdr->last_flag = (ticket == gridDim.x - 1) ? 1 : 0;
+  }
+  __syncthreads();
+  if (hdr->last_flag) {
+    __threadfence();
+    if (tid < a.n) {
+      double sum = 0.0;
+      for (unsigned b = 0; b < gridDim.x; ++b)
+        sum += static_cast<double>(__ldcg(&a.partials[static_cast<size_t>(b) * a.n + tid]));
+      const double c = sum * static_cast<double>(a.scales[tid]);
+      if (!isfinite(c))
+        twa_set_status(a.status, TWA_ERR_NONFINITE, a.nonfinite_detail >= 0 ? a.nonfinite_detail : tid);
+      if (a.c_out) a.c_out[tid] = static_cast<float>(c);
+      if (a.alpha) {
+        const double decay = 1.0 - static_cast<double>(a.lr) * static_cast<double>(a.lambda);
+        a.alpha[tid] = static_cast<float>(decay * static_cast<double>(a.alpha[tid]) -
+                                          static_cast<double>(a.lr) * c);
+      }
+    }
+    if (tid == 0) *a.ticket = 0u;
+  }
+}
+
+// =================================================================================================
+// lift
+// =================================================================================================
+template <int BITS>
+__global__ void __launch_bounds__(MMA_THREADS, 1)
+twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
+  constexpr int ROWS = twa_tile_rows(BITS);
+  constexpr int LROWS = BITS == 8 ? 2 : 4;             // rows one lane finishes per chunk
+  twa_smem_header* hdr = reinterpret_cast<twa_smem_header*>(smem);
+  unsigned char* ring = smem + TWA_SMEM_HEADER;
+  unsigned char* table = smem + a.table_off;           // digit k of coefficient j at table[k*128 + j]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gid = lane >> 2, tig = lane & 3;
+  const int tid = threadIdx.x;
+
+  init_barriers(hdr, a.stages);
+  __syncthreads();
+
+  // ---- digits of the coefficients a_j = s_j * alpha_j * mult, common scale over all j --------
+  float coef = 0.0f;
+  if (tid < TWA_MAX_N) {
+    if (tid < a.n) coef = a.alpha[tid] * a.alpha_mult * a.scales[tid];
+    atomicMax(&hdr->amax_bits, __float_as_uint(coef) & 0x7FFFFFFFu);
+  }
+  __syncthreads();
+  const unsigned ebits = hdr->amax_bits >> 23;
+  const bool bad = ebits >= 255u;                       // NaN or Inf among the coefficients
+  const bool live = ebits >= 5u && !bad;                // all-zero (or vanishing) coefficients: w = base
+  if (tid < TWA_MAX_N) {
+    uint32_t d = 0;
+    if (live) d = cut_digits(coef * __uint_as_float((259u - ebits) << 23));
+#pragma unroll
+    for (int k = 0; k < 4; ++k) table[k * TWA_MAX_N + tid] = static_cast<unsigned char>(d >> (8 * k));
+  }
+  __syncthreads();
+
+  if (warp == MMA_WARPS) {
+    if (lane == 0)
+      producer_loop_mma<0, 1, 1, ROWS>(hdr, ring, &map_p, nullptr, a.tiles, a.stages, a.stage_bytes,
+                                       0, a.tx_bytes, a.reverse != 0, a.status,
+                                       a.wait_limit_ns);
+    return;
+  }
+  if (bad && tid == 0) twa_set_status(a.status, TWA_ERR_NONFINITE, -1);
+
+  const float w0 = !live ? 0.0f : (ebits >= 6u ? __uint_as_float((ebits - 5u) << 23) : 5.877471754e-39f);
+  const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
+  float wa = tig == 0 ? w0 : (tig == 1 ? w2 : 0.0f);
+  float wb = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);
+  if (BITS == 4) { wa *= 0.0625f; wb *= 0.0625f; }
+  const float poison = bad ? __int_as_float(0x7FC00000) : 0.0f;
+
+  // B fragments: k-slot 4*tig+i of a 32-column step holds column j0 + {2tig, 2tig+1, 8+2tig, 9+2tig}[i]
+  // (and the same + 16 for the second register), the order the transposing loads deliver.
+  const int KS = (a.n + 31) >> 5;
+  uint32_t bfrag[4][2];
+#pragma unroll
+  for (int ks = 0; ks < 4; ++ks) {
+    bfrag[ks][0] = bfrag[ks][1] = 0u;
+    if (ks < KS && gid < 4) {
+      const unsigned char* tk = table + gid * TWA_MAX_N + ks * 32 + 2 * tig;
+      bfrag[ks][0] = static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(tk)) |
+                     (static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(tk + 8)) << 16);
+      bfrag[ks][1] = static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(tk + 16)) |
+                     (static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(tk + 24)) << 16);
+    }
+  }
+
+  const int c0 = warp * 2;
+  const int lm = lane >> 3, lr = lane & 7;
+  const int jmax = a.n - 1;
+  // Rows this lane finishes (tig < 2 only): chunk c0 + tig, LROWS rows starting at LROWS * gid.
+  const int lane_row = (warp * 32 + 16 * tig) * (8 / BITS) + LROWS * gid;
+  volatile int* abort_flag = &hdr->abort_flag;
+  int s = 0;
+  unsigned phase = 0;
+  for (int t = blockIdx.x; t < a.tiles; t += gridDim.x) {
+    const int tile = a.reverse ? (a.tiles - 1 - t) : t;
+    const long long row = static_cast<long long>(tile) * ROWS + lane_row;
+    float bv[LROWS];
+#pragma unroll
+    for (int i = 0; i < LROWS; ++i) bv[i] = 0.0f;
+    if (a.base && tig < 2) {
+      if (row + LROWS <= a.D) {
+        if (LROWS == 2) {
+          const float2 x = *reinterpret_cast<const float2*>(a.base + row);
+          bv[0] = x.x; bv[1] = x.y;
+        } else {
+          const float4 x = *reinterpret_cast<const float4*>(a.base + row);
+          bv[0] = x.x; bv[1] = x.y; bv[2] = x.z; bv[3] = x.w;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < LROWS; ++i)
+          if (row + i < a.D) bv[i] = a.base[row + i];
+      }
+    }
+    if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
+      twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+      break;
+    }
+    const uint32_t tile_base = twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes);
+    float keep[LROWS];
+#pragma unroll
+    for (int i = 0; i < LROWS; ++i) keep[i] = 0.0f;
+#pragma unroll
+    for (int ch = 0; ch < 2; ++ch) {
+      int acc0[4] = {0, 0, 0, 0};                       // 8-bit: rows 2gid, 2gid+1; 4-bit: rows 4gid, 4gid+2
+      int acc1[4] = {0, 0, 0, 0};                       // 4-bit only: rows 4gid+1, 4gid+3
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks) {
+        if (ks < KS) {
+          int j = ks * 32 + lm * 8 + lr;
+          j = j < jmax ? j : jmax;
+          uint32_t r[4];
+          ldmatrix_x4_trans(chunk_addr(tile_base, j, c0 + ch), r);
+          if (BITS == 8) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) r[i] ^= 0x80808080u;
+            const uint32_t af[4] = {__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[0], r[1], 0x7531),
+                                    __byte_perm(r[2], r[3], 0x6420), __byte_perm(r[2], r[3], 0x7531)};
+            mma_s8(acc0, af, bfrag[ks][0], bfrag[ks][1]);
+          } else {
+            uint32_t e[4], o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              e[i] = ((r[i] << 4) & 0xF0F0F0F0u) ^ 0x80808080u;
+              o[i] = (r[i] & 0xF0F0F0F0u) ^ 0x80808080u;
+            }
+            const uint32_t ae[4] = {__byte_perm(e[0], e[1], 0x6420), __byte_perm(e[0], e[1], 0x7531),
+                                    __byte_perm(e[2], e[3], 0x6420), __byte_perm(e[2], e[3], 0x7531)};
+            const uint32_t ao[4] = {__byte_perm(o[0], o[1], 0x6420), __byte_perm(o[0], o[1], 0x7531),
+                                    __byte_perm(o[2], o[3], 0x6420), __byte_perm(o[2], o[3], 0x7531)};
+            mma_s8(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
+            mma_s8(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
+          }
+        }
+      }
+      // digit sums -> float; the four digits of a row sit in lanes tig = 0, 1 of its quad
+      float v[LROWS];
+      if (BITS == 8) {
+        v[0] = fmaf(small_int_to_float(acc0[1]), wb, small_int_to_float(acc0[0]) * wa);
+        v[1] = fmaf(small_int_to_float(acc0[3]), wb, small_int_to_float(acc0[2]) * wa);
+      } else {
+        v[0] = fmaf(small_int_to_float(acc0[1]), wb, small_int_to_float(acc0[0]) * wa);
+        v[2] = fmaf(small_int_to_float(acc0[3]), wb, small_int_to_float(acc0[2]) * wa);
+        v[1] = fmaf(small_int_to_float(acc1[1]), wb, small_int_to_float(acc1[0]) * wa);
+        v[3] = fmaf(small_int_to_float(acc1[3]), wb, small_int_to_float(acc1[2]) * wa);
+      }
+#pragma unroll
+      for (int i = 0; i < LROWS; ++i) {
+        v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 1);
+        v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 2);
+        if (tig == ch) keep[i] = v[i];
+      }
+    }
+    __syncwarp();
+    if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
+    if (tig < 2) {
+      if (row + LROWS <= a.D) {
+        if (LROWS == 2) {
+          *reinterpret_cast<float2*>(a.out + row) = make_float2(bv[0] + keep[0] + poison, bv[1] + keep[1] + poison);
+        } else {
+          *reinterpret_cast<float4*>(a.out + row) =
+              make_float4(bv[0] + keep[0] + poison, bv[1] + keep[1] + poison, bv[2] + keep[2] + poison,
+                          bv[3] + keep[3] + poison);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < LROWS; ++i)
+          if (row + i < a.D) a.out[row + i] = bv[i] + keep[i] + poison;
+      }
+    }
+    if (++s == a.stages) {
+      s = 0;
+      phase ^= 1u;
+    }
+  }
+}
+
+// =================================================================================================
+// host side
+// =================================================================================================
+int encode_tile_map(twa_ctx* ctx, const twa_basis* P, CUtensorMap* map) {
+  long long row_bytes = (P->D * P->bits + 7) / 8;
+  // quantised columns are stored in whole, internally permuted 512-byte segments
+  if (P->bits != 32) row_bytes = (row_bytes + 511) / 512 * 512;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>((row_bytes + 3) / 4), static_cast<cuuint64_t>(P->n)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(P->col_stride)};
+  cuuint32_t box[2] = {TWA_TILE_COL_WORDS, static_cast<cuuint32_t>(P->n)};
+  cuuint32_t es[2] = {1, 1};
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, P->data, dims, strides, box, es,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(ctx->last_error, sizeof(ctx->last_error), "cuTensorMapEncodeTiled(P) failed: %d",
+             static_cast<int>(r));
+    return TWA_ERR_CUDA;
+  }
+  return TWA_OK;
+}
+
+int encode_g_map(twa_ctx* ctx, const void* g, long long D, bool bf16, CUtensorMap* map) {
+  cuuint64_t dims[1] = {static_cast<cuuint64_t>(D)};
+  cuuint64_t strides[1] = {0};
+  cuuint32_t box[1] = {256};
+  cuuint32_t es[1] = {1};
+  CUresult r = ctx->encode_tiled(
+      map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 1,
+      const_cast<void*>(g), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+      CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(ctx->last_error, sizeof(ctx->last_error), "cuTensorMapEncodeTiled(g) failed: %d",
+             static_cast<int>(r));
+    return TWA_ERR_CUDA;
+  }
+  return TWA_OK;
+}
+
+int round_up_i(int x, int m) { return (x + m - 1) / m * m; }
+
+template <int BITS, bool GBF16>
+int launch_project_mma_t(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg,
+                         const ProjectMmaArgs& a, int grid, int smem) {
+  auto kern = twa_project_mma_kernel<BITS, GBF16>;
+  static int smem_limit[64] = {0};   // per device
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[ctx->device & 63], smem);
+  if (rc) return rc;
+  kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, mg, a);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+template <int BITS>
+int launch_lift_mma_t(twa_ctx* ctx, const CUtensorMap& mp, const LiftMmaArgs& a, int grid, int smem) {
+  auto kern = twa_lift_mma_kernel<BITS>;
+  static int smem_limit[64] = {0};   // per device
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[ctx->device & 63], smem);
+  if (rc) return rc;
+  kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, a);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+}  // namespace
+
+int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
+                           const twa_project_epilogue& epi, void* ws) {
+  const bool bf16 = g_dtype == TWA_BF16;
+  const int rows = twa_tile_rows(P->bits);
+  const int gsz = bf16 ? 2 : 4;
+  CUtensorMap mp, mg;
+  int rc = encode_tile_map(ctx, P, &mp);
+  if (rc) return rc;
+  rc = encode_g_map(ctx, g, P->D, bf16, &mg);
+  if (rc) return rc;
+
+  ProjectMmaArgs a;
+  a.D = P->D;
+  a.n = P->n;
+  a.tiles = static_cast<int>((P->D + rows - 1) / rows);
+  a.g_off = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES;
+  a.tx_bytes = a.g_off + static_cast<unsigned>(rows * gsz);
+  a.stage_bytes = static_cast<unsigned>(round_up_i(static_cast<int>(a.tx_bytes), 1024));
+  const int fixed = TWA_SMEM_HEADER + MMA_WARPS * DIGIT_SCRATCH + 1024;   // 1024: alignment slack
+  int stages = (ctx->smem_optin - fixed) / static_cast<int>(a.stage_bytes);
+  if (stages > TWA_MAX_STAGES) stages = TWA_MAX_STAGES;
+  if (ctx->tune_stages >= 2 && ctx->tune_stages < stages) stages = ctx->tune_stages;
+  if (stages < 2) return TWA_ERR_UNSUPPORTED;
+  // the ring is reused for the block's [16][128] float partials after the tile loop
+  while (stages * static_cast<int>(a.stage_bytes) < MMA_WARPS * TWA_MAX_N * 4) ++stages;
+  a.stages = stages;
+  a.scratch_off = TWA_SMEM_HEADER + static_cast<unsigned>(stages) * a.stage_bytes;
+  a.scales = P->scales;
+  a.partials = reinterpret_cast<float*>(static_cast<char*>(ws) + TWA_WS_PARTIALS);
+  a.ticket = ctx->d_ticket;
+  a.status = ctx->d_status;
+  a.c_out = epi.c_out;
+  a.alpha = epi.alpha;
+  a.lr = epi.lr;
+  a.lambda = epi.lambda;
+  a.nonfinite_detail = epi.nonfinite_detail;
+  a.wait_limit_ns = ctx->wait_limit_ns;
+  int grid = ctx->sm_count < a.tiles ? ctx->sm_count : a.tiles;
+  if (grid > TWA_MAX_GRID) grid = TWA_MAX_GRID;
+  const int smem = static_cast<int>(a.scratch_off) + MMA_WARPS * DIGIT_SCRATCH + 1024;
+  if (P->bits == 8)
+    return bf16 ? launch_project_mma_t<8, true>(ctx, mp, mg, a, grid, smem)
+                : launch_project_mma_t<8, false>(ctx, mp, mg, a, grid, smem);
+  return bf16 ? launch_project_mma_t<4, true>(ctx, mp, mg, a, grid, smem)
+              : launch_project_mma_t<4, false>(ctx, mp, mg, a, grid, smem);
+}
+
+int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
+                        const float* base, float* out, bool reverse_tiles) {
+  const int rows = twa_tile_rows(P->bits);
+  CUtensorMap mp;
+  int rc = encode_tile_map(ctx, P, &mp);
+  if (rc) return rc;
+  LiftMmaArgs a;
+  a.D = P->D;
+  a.n = P->n;
+  a.tiles = static_cast<int>((P->D + rows - 1) / rows);
+  a.tx_bytes = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES;
+  a.stage_bytes = static_cast<unsigned>(round_up_i(static_cast<int>(a.tx_bytes), 1024));
+  const int fixed = TWA_SMEM_HEADER + 4 * TWA_MAX_N + 1024;               // 1024: alignment slack
+  int stages = (ctx->smem_optin - fixed) / static_cast<int>(a.stage_bytes);
+  if (stages > TWA_MAX_STAGES) stages = TWA_MAX_STAGES;
+  if (ctx->tune_stages >= 2 && ctx->tune_stages < stages) stages = ctx->tune_stages;
+  if (stages < 2) return TWA_ERR_UNSUPPORTED;
+  a.stages = stages;
+  a.table_off = TWA_SMEM_HEADER + static_cast<unsigned>(stages) * a.stage_bytes;
+  a.scales = P->scales;
+  a.alpha = alpha;
+  a.alpha_mult = alpha_mult;
+  a.base = base;
+  a.out = out;
+  a.reverse = reverse_tiles ? 1 : 0;
+  a.status = ctx->d_status;
+  a.wait_limit_ns = ctx->wait_limit_ns;
+  const int grid = ctx->sm_count < a.tiles ? ctx->sm_count : a.tiles;
+  const int smem = static_cast<int>(a.table_off) + 4 * TWA_MAX_N + 1024;
+  return P->bits == 8 ? launch_lift_mma_t<8>(ctx, mp, a, grid, smem)
+                      : launch_lift_mma_t<4>(ctx, mp, a, grid, smem);
+}

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libtwa.so")
 CSRC = os.path.join(_HERE, "csrc")
-SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_stream.cu", "twa_noalloc.cu"]
+SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_stream.cu", "twa_stream_mma.cu", "twa_noalloc.cu"]
 
 TWA_MAX_N = 128
 TWA_OK = 0
@@ -34,6 +34,7 @@ TWA_TUNE_PROJECT_WARPS = 1
 TWA_TUNE_LIFT_WARPS = 2
 TWA_TUNE_STAGES = 3
 TWA_TUNE_WAIT_LIMIT_MS = 4
+TWA_TUNE_DEQUANT_PATH = 5
 
 EXPORTS = [
     "twa_create", "twa_destroy", "twa_get_status", "twa_clear_status", "twa_strerror",

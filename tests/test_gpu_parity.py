@@ -129,11 +129,22 @@ def test_export_import_roundtrip(env, bits):
 
 
 # ------------------------------------------------------------------ project / lift
+@pytest.fixture(params=[0, 1], ids=["tensor-pipe", "float-fma"])
+def dequant_path(request, env):
+    """Both ways the library turns 8/4-bit codes into products (TWA_TUNE_DEQUANT_PATH)."""
+    ctx, _ = env
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_DEQUANT_PATH, request.param)
+    yield request.param
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_DEQUANT_PATH, 0)
+
+
 @pytest.mark.parametrize("gdt", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("bits", [32, 8, 4])
 @pytest.mark.parametrize("D,n", SHAPES)
-def test_project_and_lift(env, D, n, bits, gdt):
+def test_project_and_lift(env, dequant_path, D, n, bits, gdt):
     ctx, ws = env
+    if bits == 32 and dequant_path == 1:
+        pytest.skip("the path choice only exists for 8/4-bit storage")
     P = random_basis(D, n, 100 + D + n)
     P32 = twa.basis_from_tensor(P, D)
     gen = torch.Generator(device=DEV)
@@ -178,8 +189,10 @@ def test_project_and_lift(env, D, n, bits, gdt):
 
 
 @pytest.mark.parametrize("bits", [32, 8, 4])
-def test_step_sequence_and_determinism(env, bits):
+def test_step_sequence_and_determinism(env, dequant_path, bits):
     ctx, ws = env
+    if bits == 32 and dequant_path == 1:
+        pytest.skip("the path choice only exists for 8/4-bit storage")
     D, n, lr, lam = 50021, 24, 0.1, 0.05
     W = inputs.trajectory_candidates(D, n, 0.005, 0.001, 9, DEV, ld=inputs.padded_ld(D, 4))
     wbar = torch.empty(D, device=DEV)
