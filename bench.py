@@ -49,6 +49,27 @@ def load_peaks():
     return 6650.0, "fallback"
 
 
+def read_traffic(key):
+    """DRAM bytes per launch from profiles/traffic.md, or None when there is no entry or the
+    kernel sources changed since the counters were taken."""
+    import hashlib
+    import re
+    path = os.path.join(ROOT, "profiles", "traffic.md")
+    if not os.path.exists(path):
+        return None
+    h = hashlib.sha256()
+    for name in ("twa_stream_mma.cu", "twa_common.cuh"):
+        with open(os.path.join(ROOT, "paper_2205_13104_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    digest = h.hexdigest()[:16]
+    with open(path) as f:
+        for line in f:
+            m = re.match(r"^(\S+) = (\d+) \| ([0-9a-f]{16})\s*$", line)
+            if m and m.group(1) == key:
+                return int(m.group(2)) if m.group(3) == digest else None
+    return None
+
+
 class ClockSampler:
     """nvidia-smi samples of one GPU's clocks and throttle reasons while a region runs."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -286,13 +307,7 @@ def run_ours(args):
         achieved = kb[dom] / (dom_ms * 1e-3) / 1e9
         other = "lift" if dom == "project" else "project"
         other_ms = (lift_ms if dom == "project" else proj_ms) / max(rec, 1)
-        traffic = None
-        tpath = os.path.join(ROOT, "profiles", "traffic.json")
-        if os.path.exists(tpath):
-            with open(tpath) as f:
-                tj = json.load(f)
-            key = f"{wl.name}_int{bits}_{dom}"
-            traffic = tj.get(key)
+        traffic = read_traffic(f"{wl.name}_int{bits}_{dom}") if args.dequant_path == 0 else None
         # CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
