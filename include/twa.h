@@ -147,6 +147,40 @@ size_t twa_workspace_bytes(int64_t D, int n, int bits);
 int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float* wbar_out,
                     twa_basis* P32_out, void* ws, size_t ws_bytes);
 
+/* The same basis for candidate sets too large to be resident (e.g. 1.3 G rows x 32 columns =
+ * 168 GB of float32): the caller feeds row chunks of the candidates, once per pass, and never
+ * holds more than one chunk.  The orthonormal basis with span{e_1..e_j} = span{w_1..w_j} and
+ * positive diagonal is unique, so it is computed in Gram form with every n x n quantity in
+ * float64: G1 = A^T A, R1 = chol(G1); G2 = (A R1^-1)^T (A R1^-1), R2 = chol(G2);
+ * Q = A (R1^-1 R2^-1) -- orthogonalise, then re-orthogonalise.  n <= 64.
+ *
+ *   twa_build_begin(ctx, D, n, wbar_out, bws, bws_bytes)
+ *   pass 0: twa_build_feed(ctx, 0, chunk, ...) for every chunk   -> mean rows into wbar_out, G1
+ *           twa_build_end_pass(ctx, 0, 0, NULL)
+ *   pass 1: feed every chunk again                                -> G2
+ *           twa_build_end_pass(ctx, 1, 0, NULL)
+ *   pass 2: feed again (q32_out optional)                         -> column absmax of Q
+ *           twa_build_end_pass(ctx, 2, bits, Pq)                  -> scales; fills *Pq
+ *   pass 3: feed again with Pq                                    -> codes of Q (bits 8 / 4)
+ *           twa_build_end_pass(ctx, 3, 0, NULL)
+ *
+ *  chunk   rows x n float32, column-major with column stride ldc elements: rows
+ *          [row0, row0+rows) of the candidates.  row0 must be a multiple of 1024, rows a
+ *          multiple of 1024 except for the chunk that ends at D.  Any order, each row range
+ *          exactly once per pass, the same partition in every pass.
+ *  q32_out passes 2 and 3, optional: D x n float32 destination (column stride ldq elements)
+ *          that receives the float32 basis rows of the chunk.  With bits == 32 this is the
+ *          only output and pass 3 is not run.
+ *  Pq      the caller sets data (twa_basis_bytes) and scales before twa_build_end_pass(2).
+ *  bws     device scratch of twa_build_workspace_bytes(n) bytes, alive until the last call.
+ * Device-side errors: TWA_ERR_RANK_DEFICIENT (same 1e-5 rule as twa_build_basis),
+ * TWA_ERR_NONFINITE.  Codes are exactly the quantiser applied to the float32 rows of pass 2. */
+size_t twa_build_workspace_bytes(int n);
+int twa_build_begin(twa_ctx* ctx, int64_t D, int n, float* wbar_out, void* bws, size_t bws_bytes);
+int twa_build_feed(twa_ctx* ctx, int pass, const float* chunk, int64_t ldc, int64_t row0,
+                   int64_t rows, const twa_basis* Pq, float* q32_out, int64_t ldq);
+int twa_build_end_pass(twa_ctx* ctx, int pass, int bits, twa_basis* Pq);
+
 /* Mean only: wbar_out[r] = (1/n) sum_i W[r, i]. */
 int twa_mean(twa_ctx* ctx, const float* W, int64_t D, int n, int64_t ldw, float* wbar_out);
 

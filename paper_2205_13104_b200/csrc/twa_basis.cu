@@ -152,13 +152,6 @@ __global__ void scales_kernel(const unsigned* __restrict__ absmax, int n, float 
   }
 }
 
-__device__ __forceinline__ int encode_one(float p, float s, float qmax) {
-  if (s == 0.0f) return 0;
-  float q = rintf(__fdiv_rn(p, s));                   // round half to even
-  q = fminf(fmaxf(q, -qmax), qmax);
-  return static_cast<int>(q);
-}
-
 // One thread produces 16 bytes of a column (16 rows at 8 bits, 32 rows at 4 bits), including
 // the padding up to the column stride, which is filled with the code 0.
 template <int BITS>
@@ -191,7 +184,7 @@ __global__ void __launch_bounds__(BLOCK) encode_kernel(const float* __restrict__
     uint32_t w[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int k = 0; k < RPT; ++k) {
-      const uint32_t u = static_cast<uint32_t>(encode_one(p[k], s, QMAX) + BIAS);
+      const uint32_t u = static_cast<uint32_t>(twa_encode_one(p[k], s, QMAX) + BIAS);
       if (BITS == 8) w[k >> 2] |= u << (8 * (k & 3));
       else w[k >> 3] |= u << (4 * (k & 7));
     }
@@ -251,6 +244,12 @@ int launch_sumsq(twa_ctx* ctx, const float* v, long long D, void* ws, int slot) 
 }
 
 }  // namespace
+
+int twa_launch_scales(twa_ctx* ctx, const unsigned* absmax, int n, int bits, float* scales) {
+  scales_kernel<<<1, 128, 0, ctx->stream>>>(absmax, n, bits == 8 ? 127.0f : 7.0f, scales, ctx->d_status);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
 
 extern "C" {
 
@@ -345,9 +344,8 @@ int twa_quantize_basis(twa_ctx* ctx, const twa_basis* P32, int bits, twa_basis* 
   if (per_col < 1) per_col = 1;
   absmax_kernel<<<dim3(per_col, n), BLOCK, 0, ctx->stream>>>(P, D, ld, absmax);
   TWA_CUDA_OK(ctx, cudaGetLastError());
-  scales_kernel<<<1, 128, 0, ctx->stream>>>(absmax, n, bits == 8 ? 127.0f : 7.0f, Pq->scales,
-                                            ctx->d_status);
-  TWA_CUDA_OK(ctx, cudaGetLastError());
+  rc = twa_launch_scales(ctx, absmax, n, bits, Pq->scales);
+  if (rc) return rc;
   const long long stride = twa_basis_col_stride(D, bits);
   int eper = grid_for(ctx, stride / 16, BLOCK, 8) / n;
   if (eper < 1) eper = 1;

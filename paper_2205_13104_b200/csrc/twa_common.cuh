@@ -30,6 +30,11 @@ struct twa_ctx {
   int tune_dequant_path;      // 0 = integer tensor-pipe dot products, 1 = float FMA
   cudaEvent_t* prof_events;   // 3 per recorded step, or null
   int prof_cap, prof_count;   // steps
+  // state of a row-chunked basis build (twa_build_begin .. twa_build_end_pass)
+  long long build_D;
+  int build_n;
+  float* build_wbar;
+  char* build_ws;
   char last_error[256];
 };
 
@@ -196,6 +201,14 @@ __device__ __forceinline__ float twa_byte_to_float(uint32_t word, int byte, floa
 constexpr float TWA_MAGIC_I8 = 8388608.0f + 128.0f;
 constexpr float TWA_MAGIC_I4 = 8388608.0f + 8.0f;
 
+// One element of the quantiser: IEEE float32 quotient, round half to even, clamp to +-qmax.
+__device__ __forceinline__ int twa_encode_one(float p, float s, float qmax) {
+  if (s == 0.0f) return 0;
+  float q = rintf(__fdiv_rn(p, s));
+  q = fminf(fmaxf(q, -qmax), qmax);
+  return static_cast<int>(q);
+}
+
 __device__ __forceinline__ float twa_bf16_lo(uint32_t pair) { return __uint_as_float(pair << 16); }
 __device__ __forceinline__ float twa_bf16_hi(uint32_t pair) { return __uint_as_float(pair & 0xFFFF0000u); }
 
@@ -216,6 +229,8 @@ int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtyp
 int twa_launch_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
                     const float* base, float* out, bool reverse_tiles);
 int twa_check_basis(const twa_basis* P);
+// scales[j] = absmax_j / qmax from the bit patterns of the column maxima; flags NaN/Inf
+int twa_launch_scales(twa_ctx* ctx, const unsigned* absmax, int n, int bits, float* scales);
 // Variants of the two launchers for 8- and 4-bit storage that compute the integer dot
 // products on the tensor pipe (twa_stream_mma.cu).
 int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,

@@ -16,7 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libtwa.so")
 CSRC = os.path.join(_HERE, "csrc")
-SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_stream.cu", "twa_stream_mma.cu", "twa_noalloc.cu"]
+SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_chunked.cu", "twa_stream.cu", "twa_stream_mma.cu",
+           "twa_noalloc.cu"]
 
 TWA_MAX_N = 128
 TWA_OK = 0
@@ -40,7 +41,8 @@ EXPORTS = [
     "twa_create", "twa_destroy", "twa_get_status", "twa_clear_status", "twa_strerror",
     "twa_last_error", "twa_set_tuning", "twa_profile_enable", "twa_profile_read",
     "twa_basis_col_stride", "twa_basis_bytes",
-    "twa_workspace_bytes", "twa_build_basis", "twa_mean", "twa_quantize_basis",
+    "twa_workspace_bytes", "twa_build_basis", "twa_build_workspace_bytes", "twa_build_begin",
+    "twa_build_feed", "twa_build_end_pass", "twa_mean", "twa_quantize_basis",
     "twa_basis_export", "twa_basis_import", "twa_project", "twa_lift", "twa_step",
     "twa_step_host", "twa_project_noalloc", "twa_noalloc_last_error", "twa_noalloc_scratch_bytes",
 ]
@@ -113,6 +115,10 @@ def load():
         "twa_basis_bytes": (szt, [i64, i32, i32]),
         "twa_workspace_bytes": (szt, [i64, i32, i32]),
         "twa_build_basis": (i32, [vp, vp, i64, i32, i64, vp, bp, vp, szt]),
+        "twa_build_workspace_bytes": (szt, [i32]),
+        "twa_build_begin": (i32, [vp, i64, i32, vp, vp, szt]),
+        "twa_build_feed": (i32, [vp, i32, vp, i64, i64, i64, bp, vp, i64]),
+        "twa_build_end_pass": (i32, [vp, i32, i32, bp]),
         "twa_mean": (i32, [vp, vp, i64, i32, i64, vp]),
         "twa_quantize_basis": (i32, [vp, bp, i32, bp, vp, szt]),
         "twa_basis_export": (i32, [vp, bp, vp, vp]),
@@ -257,6 +263,37 @@ def twa_build_basis(ctx, W, D, wbar_out, ws):
                                 ctypes.byref(desc), _ptr(ws), ws.numel())
     _check(rc, "twa_build_basis", ctx)
     return Basis(desc, W, None)
+
+
+def twa_build_workspace_bytes(n):
+    return int(load().twa_build_workspace_bytes(int(n)))
+
+
+def twa_build_begin(ctx, D, n, wbar_out, bws):
+    _check(load().twa_build_begin(ctx, int(D), int(n), _ptr(wbar_out), _ptr(bws), bws.numel()),
+           "twa_build_begin", ctx)
+
+
+def twa_build_feed(ctx, pass_index, chunk, row0, rows, Pq=None, q32_out=None):
+    """chunk: float32 CUDA tensor view (n, >= rows) whose row i holds rows [row0, row0+rows) of
+    candidate i (stride(0) = column stride); q32_out: float32 (n, ldq) tensor or None."""
+    assert chunk.dtype == torch.float32 and chunk.stride(1) == 1
+    rc = load().twa_build_feed(ctx, int(pass_index), _ptr(chunk), int(chunk.stride(0)), int(row0),
+                               int(rows), ctypes.byref(Pq.desc) if Pq is not None else None,
+                               _ptr(q32_out), int(q32_out.stride(0)) if q32_out is not None else 0)
+    _check(rc, "twa_build_feed", ctx)
+
+
+def twa_build_end_pass(ctx, pass_index, bits=0, Pq=None):
+    rc = load().twa_build_end_pass(ctx, int(pass_index), int(bits),
+                                   ctypes.byref(Pq.desc) if Pq is not None else None)
+    _check(rc, "twa_build_end_pass", ctx)
+
+
+def new_quantised_basis(D, n, bits, device):
+    """Empty Basis with library-sized buffers, for twa_build_end_pass(2) to fill."""
+    desc, data, scales = _new_quantised(D, n, bits, device)
+    return Basis(desc, data, scales)
 
 
 def basis_from_tensor(P32, D):

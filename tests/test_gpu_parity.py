@@ -361,3 +361,82 @@ def test_host_side_argument_errors(env):
     assert code_of(lambda: twa.twa_build_basis(ctx, wide, 16, torch.zeros(16, device=DEV), ws)) == \
         twa.TWA_ERR_UNSUPPORTED
     status_ok(ctx)
+
+
+# ------------------------------------------------------------------ row-chunked build
+def _chunked_build(ctx, W, D, bits, chunk_rows, want_q32=True):
+    n = W.shape[0]
+    bws = torch.empty(twa.twa_build_workspace_bytes(n), dtype=torch.uint8, device=DEV)
+    wbar = torch.full((D + 4,), 9.0, device=DEV)
+    q32 = torch.zeros((n, inputs.padded_ld(D, 4)), device=DEV) if want_q32 else None
+    Pq = twa.new_quantised_basis(D, n, bits, DEV) if bits != 32 else None
+    starts = list(range(0, D, chunk_rows))
+    twa.twa_build_begin(ctx, D, n, wbar, bws)
+    for p in range(4 if bits != 32 else 3):
+        order = starts if p % 2 == 0 else starts[::-1]          # any order within a pass
+        for r0 in order:
+            rows = min(chunk_rows, D - r0)
+            twa.twa_build_feed(ctx, p, W[:, r0:], r0, rows, Pq=Pq if p == 3 else None,
+                               q32_out=q32 if p >= 2 else None)
+        twa.twa_build_end_pass(ctx, p, bits if p == 2 else 0, Pq if p == 2 else None)
+    return wbar, q32, Pq
+
+
+@pytest.mark.parametrize("D,n,chunk_rows", [(300007, 20, 131072), (70001, 33, 8192), (5000, 3, 1024),
+                                           (260000, 64, 65536)])
+def test_chunked_build_matches_oracle_and_resident_build(env, D, n, chunk_rows):
+    ctx, ws = env
+    W = inputs.trajectory_candidates(D, n, 0.005, 0.001, 31, DEV, ld=inputs.padded_ld(D, 4))
+    A = host_cols(W, D).copy()
+    wbar, q32, _ = _chunked_build(ctx, W, D, 32, chunk_rows)
+    status_ok(ctx)
+    np.testing.assert_array_equal(wbar[:D].cpu().numpy(), orc.mean(A).astype(np.float32))
+    assert torch.all(wbar[D:] == 9.0)
+    Qg = host_cols(q32, D).astype(np.float64)
+    assert np.max(np.abs(Qg.T @ Qg - np.eye(n))) <= 1e-5
+    Q, _, bad = orc.cgs2(A)
+    assert bad is None
+    kappa = np.linalg.cond(A.astype(np.float64))
+    assert np.max(np.linalg.norm(Qg - Q, axis=0)) <= 1e-6 + 100 * kappa * np.finfo(np.float64).eps
+    assert torch.all(q32[:, D:] == 0)
+    # the resident float32 Gram-Schmidt build gives the same basis up to its float32 rounding
+    W2 = W.clone()
+    wbar2 = torch.empty(D, device=DEV)
+    twa.twa_build_basis(ctx, W2, D, wbar2, ws)
+    status_ok(ctx)
+    assert torch.equal(wbar2, wbar[:D])
+    assert np.max(np.linalg.norm(host_cols(W2, D) - Qg, axis=0)) <= 10 * kappa * np.finfo(np.float32).eps
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_chunked_build_codes_are_the_quantiser_of_its_float32_rows(env, bits):
+    ctx, ws = env
+    D, n, chunk_rows = 150001, 12, 32768
+    W = inputs.trajectory_candidates(D, n, 0.005, 0.001, 32, DEV, ld=inputs.padded_ld(D, 4))
+    wbar, q32, Pq = _chunked_build(ctx, W, D, bits, chunk_rows)
+    status_ok(ctx)
+    codes_g, s_g = twa.twa_basis_export(ctx, Pq)
+    codes_o, s_o = orc.quantize(np.asfortranarray(host_cols(q32, D)), bits)
+    np.testing.assert_array_equal(s_g.cpu().numpy(), s_o)
+    np.testing.assert_array_equal(codes_g.cpu().numpy(), orc.pack_codes(codes_o, bits))
+    # identical to quantising the float32 rows with the resident quantiser, padding included
+    Pq2 = twa.twa_quantize_basis(ctx, twa.basis_from_tensor(q32, D), bits, ws)
+    assert torch.equal(Pq.data, Pq2.data) and torch.equal(Pq.scales, Pq2.scales)
+    # and usable by the step kernels
+    g = inputs.gradient(D, 1e-3, 5, 0, torch.float32, DEV)
+    c = torch.empty(n, device=DEV)
+    twa.twa_project(ctx, Pq, g, c, ws)
+    c_ref = orc.project(codes_o, s_o, g.cpu().numpy())
+    assert rel(c.cpu().numpy(), c_ref) <= TOL
+    status_ok(ctx)
+
+
+def test_chunked_build_reports_rank_deficiency(env):
+    ctx, ws = env
+    D, n = 20000, 5
+    W = inputs.trajectory_candidates(D, n, 0.01, 0.002, 33, DEV, ld=inputs.padded_ld(D, 4))
+    W[3] = W[1] * 0.5
+    _chunked_build(ctx, W, D, 32, 4096)
+    code, detail = twa.twa_get_status(ctx)
+    assert (code, detail) == (twa.TWA_ERR_RANK_DEFICIENT, 3)
+    twa.twa_clear_status(ctx)
