@@ -202,8 +202,8 @@ def run_ours(args):
 
     twa.load()
     wl = inputs.WORKLOADS[args.workload]
+    import dataclasses
     if args.rows:
-        import dataclasses
         wl = dataclasses.replace(wl, name=f"{wl.name}[rows={args.rows}]", D=args.rows)
     D, n, bits = wl.D, wl.n, args.bits
     gdt = torch.bfloat16 if wl.g_dtype == "bf16" else torch.float32
@@ -216,22 +216,51 @@ def run_ours(args):
     wbar = torch.empty(D, dtype=torch.float32, device=dev)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
     if args.random_basis:
+        wl = dataclasses.replace(wl, chunked_build=False)
         # profiling aid: skip the Gram-Schmidt launches; the step kernels do the same work on any values
         W = torch.randn((n, inputs.padded_ld(D, 128)), device=dev) / (D ** 0.5)
         twa.twa_mean(ctx, W, D, wbar)
         torch.cuda.synchronize()
         ev[0].record()
         P32 = twa.basis_from_tensor(W, D)
+    elif wl.chunked_build:
+        # The candidates (4*n*D bytes) do not fit beside P~: every row chunk is regenerated from
+        # its seed once per pass and fed to the chunked build.  Library time = CUDA events around
+        # the feed calls only; generating the chunks is not counted.
+        if bits == 32:
+            raise SystemExit("the chunked workload has no resident float32 basis; use --bits 8 or 4")
+        bws = torch.empty(twa.twa_build_workspace_bytes(n), dtype=torch.uint8, device=dev)
+        Pq = twa.new_quantised_basis(D, n, bits, dev)
+        buf = torch.empty((n, inputs.CHUNK_ROWS), dtype=torch.float32, device=dev)
+        pairs = []
+        twa.twa_build_begin(ctx, D, n, wbar, bws)
+        for p in range(4):
+            for r0 in range(0, D, inputs.CHUNK_ROWS):
+                rows = min(inputs.CHUNK_ROWS, D - r0)
+                inputs.trajectory_rows(D, n, wl.step, wl.drift, wl.seed, dev, row0=r0, rows=rows,
+                                       out=buf[:, :rows])
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                twa.twa_build_feed(ctx, p, buf, r0, rows, Pq=Pq if p == 3 else None)
+                if r0 + rows == D:
+                    twa.twa_build_end_pass(ctx, p, bits if p == 2 else 0, Pq if p == 2 else None)
+                b.record()
+                pairs.append((a, b))
+        torch.cuda.synchronize()
+        build_ms, quant_ms = sum(a.elapsed_time(b) for a, b in pairs), 0.0
+        del buf, bws, pairs
+        W = P32 = None
     else:
         W = wl.candidates(dev, ld=inputs.padded_ld(D, 128))
         torch.cuda.synchronize()
         ev[0].record()
         P32 = twa.twa_build_basis(ctx, W, D, wbar, ws)
-    ev[1].record()
-    Pq = twa.twa_quantize_basis(ctx, P32, bits, ws) if bits != 32 else P32
-    ev[2].record()
-    torch.cuda.synchronize()
-    build_ms, quant_ms = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
+    if not wl.chunked_build or args.random_basis:
+        ev[1].record()
+        Pq = twa.twa_quantize_basis(ctx, P32, bits, ws) if bits != 32 else P32
+        ev[2].record()
+        torch.cuda.synchronize()
+        build_ms, quant_ms = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
     code, detail = twa.twa_get_status(ctx)
     if code != 0:
         raise RuntimeError(f"basis build failed: {twa.twa_strerror(code)} column {detail}")
@@ -240,7 +269,8 @@ def run_ours(args):
         torch.cuda.empty_cache()
 
     # ---- per-step inputs: a pool of distinct gradients, cycled ------------------------
-    pool = [wl.gradient(t, dev) for t in range(args.g_pool)]
+    g_pool = args.g_pool if D * g_bytes * args.g_pool <= 8e9 else max(2, int(8e9 // (D * g_bytes)))
+    pool = [wl.gradient(t, dev) for t in range(g_pool)]
     alpha = torch.zeros(n, dtype=torch.float32, device=dev)
     w = torch.empty(D, dtype=torch.float32, device=dev)
     lr, lam = 0.1, 0.0
@@ -327,7 +357,10 @@ def run_ours(args):
             "bytes_per_step": sb,
             "frac_of_hbm_peak": value / world / peak,
             "frac_of_8TBps": value / world / 8000.0,
-            "basis_build_ms": None if args.random_basis else build_ms, "quantize_ms": quant_ms,
+            "basis_build_ms": None if args.random_basis else build_ms,
+            "quantize_ms": None if wl.chunked_build else quant_ms,
+            "basis_build": ("row-chunked Gram-form build incl. quantisation, 4 passes, chunk generation not counted"
+                            if wl.chunked_build else "resident classical Gram-Schmidt with re-orthogonalisation"),
             "roofline": {"bound": "hbm", "kernel": f"twa_{dom}{suffix}_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "traffic": traffic, "bytes_per_launch": kb[dom], "ms_per_launch": dom_ms,

@@ -108,9 +108,11 @@ const char* twa_last_error(const twa_ctx* ctx);
  *  TWA_TUNE_DEQUANT_PATH: how 8/4-bit codes meet g and alpha: 0 = exact integer dot products
  *      on the tensor pipe against block-fixed-point digits of g / alpha (default),
  *      1 = code -> float32 conversion and float32 FMA.  The warp and stage knobs act on the
- *      float path and on 32-bit bases only.                                             */
+ *      float path and on 32-bit bases only.
+ *  TWA_TUNE_TILE_SEGMENTS: tensor-pipe path, 512-byte segments of a column per tile: 1 or 2
+ *      (default: 2 for n <= 64, else 1).                                                */
 enum { TWA_TUNE_PROJECT_WARPS = 1, TWA_TUNE_LIFT_WARPS = 2, TWA_TUNE_STAGES = 3,
-       TWA_TUNE_WAIT_LIMIT_MS = 4, TWA_TUNE_DEQUANT_PATH = 5 };
+       TWA_TUNE_WAIT_LIMIT_MS = 4, TWA_TUNE_DEQUANT_PATH = 5, TWA_TUNE_TILE_SEGMENTS = 6 };
 int twa_set_tuning(twa_ctx* ctx, int key, int value);
 
 /* Per-kernel timing of twa_step for measurements.  twa_profile_enable(ctx, max_steps > 0)

@@ -28,6 +28,7 @@ struct twa_ctx {
   unsigned long long wait_limit_ns;
   int tune_project_warps, tune_lift_warps, tune_stages;
   int tune_dequant_path;      // 0 = integer tensor-pipe dot products, 1 = float FMA
+  int tune_tile_segments;     // tensor-pipe path: 512-byte segments per tile column (0 = choose)
   cudaEvent_t* prof_events;   // 3 per recorded step, or null
   int prof_cap, prof_count;   // steps
   // state of a row-chunked basis build (twa_build_begin .. twa_build_end_pass)

@@ -39,6 +39,7 @@ constexpr float RND = 12582912.0f;             // 2^23 + 2^22: x + RND rounds x 
 struct ProjectMmaArgs {
   long long D;
   int n, stages, tiles;
+  int kt;                      // 512-byte segments of a column per tile (1 or 2)
   unsigned stage_bytes, g_off, tx_bytes, scratch_off;
   const float* scales;
   float* partials;
@@ -54,6 +55,7 @@ struct ProjectMmaArgs {
 struct LiftMmaArgs {
   long long D;
   int n, stages, tiles;
+  int kt;                      // 512-byte segments of a column per tile (1 or 2)
   unsigned stage_bytes, tx_bytes, table_off;
   const float* scales;
   const float* alpha;
@@ -105,20 +107,22 @@ __device__ __forceinline__ uint32_t cut_digits(float t) {
   return __byte_perm(lo, hi, 0x5410);
 }
 
-// Shared address of logical 16-byte chunk `chunk` (0..31) of column j of a tile.
-__device__ __forceinline__ uint32_t chunk_addr(uint32_t tile_base, int j, int chunk) {
-  return tile_base + static_cast<uint32_t>(j) * TWA_TILE_COL_BYTES +
-         (static_cast<uint32_t>(twa_chunk_slot(chunk, j)) << 4);
+// Shared address of logical 16-byte chunk `chunk` (0 .. 32*kt-1) of column j of a tile whose
+// columns are col_bytes = 512*kt long.
+__device__ __forceinline__ uint32_t chunk_addr(uint32_t tile_base, int col_bytes, int j, int chunk) {
+  return tile_base + static_cast<uint32_t>(j * col_bytes + ((chunk >> 5) << 9)) +
+         (static_cast<uint32_t>(twa_chunk_slot(chunk & 31, j)) << 4);
 }
 
-template <int G_BOXES, int G_BOX_ELEMS, int G_ELEM_BYTES, int ROWS>
+// g_boxes 1-D boxes of 256 gradient elements follow the tile of P~ in a stage (project only).
 __device__ __forceinline__ void producer_loop_mma(twa_smem_header* hdr, unsigned char* ring,
                                                   const CUtensorMap* map_p, const CUtensorMap* map_g,
-                                                  int tiles, int stages, unsigned stage_bytes,
+                                                  int tiles, int stages, unsigned stage_bytes, int kt,
+                                                  int g_boxes, int g_elem_bytes, int tile_rows,
                                                   unsigned g_off, unsigned tx_bytes,
                                                   bool reverse, int* status, unsigned long long limit) {
   twa_prefetch_tensormap(map_p);
-  if (G_BOXES > 0) twa_prefetch_tensormap(map_g);
+  if (g_boxes > 0) twa_prefetch_tensormap(map_g);
   volatile int* abort_flag = &hdr->abort_flag;
   int s = 0, issued = 0;
   unsigned phase = 0;
@@ -134,10 +138,9 @@ __device__ __forceinline__ void producer_loop_mma(twa_smem_header* hdr, unsigned
     const uint32_t fb = twa_smem_u32(&hdr->full[s]);
     const uint32_t dst = twa_smem_u32(ring + static_cast<size_t>(s) * stage_bytes);
     twa_mbar_expect_tx(fb, tx_bytes);
-    twa_tma_load_2d(dst, map_p, tile * TWA_TILE_COL_WORDS, 0, fb);
-#pragma unroll
-    for (int b = 0; b < G_BOXES; ++b)
-      twa_tma_load_1d(dst + g_off + b * G_BOX_ELEMS * G_ELEM_BYTES, map_g, tile * ROWS + b * G_BOX_ELEMS, fb);
+    twa_tma_load_2d(dst, map_p, tile * TWA_TILE_COL_WORDS * kt, 0, fb);
+    for (int b = 0; b < g_boxes; ++b)
+      twa_tma_load_1d(dst + g_off + b * 256 * g_elem_bytes, map_g, tile * tile_rows + b * 256, fb);
     ++issued;
     if (++s == stages) {
       s = 0;
@@ -182,10 +185,9 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   // stages start on 1024-byte boundaries (TMA destinations need 128)
   unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
-  constexpr int ROWS = twa_tile_rows(BITS);            // 512 or 1024 rows per tile
-  constexpr int WROWS = ROWS / MMA_WARPS;              // 32 or 64 rows per warp
+  constexpr int SROWS = twa_tile_rows(BITS);           // rows behind one 512-byte segment: 512 or 1024
+  constexpr int WROWS = SROWS / MMA_WARPS;             // rows behind 32 bytes: 32 or 64
   constexpr int GSZ = GBF16 ? 2 : 4;
-  constexpr int GBOX = 256;
   twa_smem_header* hdr = reinterpret_cast<twa_smem_header*>(smem);
   unsigned char* ring = smem + TWA_SMEM_HEADER;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -202,14 +204,14 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
 
   if (warp == MMA_WARPS) {
     if (lane == 0)
-      producer_loop_mma<ROWS / GBOX, GBOX, GSZ, ROWS>(hdr, ring, &map_p, &map_g, a.tiles, a.stages,
-                                                      a.stage_bytes, a.g_off, a.tx_bytes,
-                                                      false, a.status, a.wait_limit_ns);
+      producer_loop_mma(hdr, ring, &map_p, &map_g, a.tiles, a.stages, a.stage_bytes, a.kt,
+                        SROWS * a.kt / 256, GSZ, SROWS * a.kt, a.g_off, a.tx_bytes, false, a.status,
+                        a.wait_limit_ns);
   } else {
     unsigned char* digw = smem + a.scratch_off + warp * DIGIT_SCRATCH;   // this warp's digit bytes
-    const int c0 = warp * 2;                            // this warp's two 16-byte chunks of every column
     const int lm = lane >> 3, lr = lane & 7;            // ldmatrix: matrix and row this lane addresses
     const int jmax = a.n - 1;                           // last column that exists in shared memory
+    const int col_bytes = TWA_TILE_COL_BYTES * a.kt;
     volatile int* abort_flag = &hdr->abort_flag;
     int s = 0;
     unsigned phase = 0;
@@ -220,19 +222,24 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
         break;
       }
       const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
-      // ---- this warp's rows of g: 1 (8-bit) or 2 (4-bit) per lane ------------------------
+      // The warp owns bytes [32*kt*warp, 32*kt*(warp+1)) of every column: kt blocks of 32 bytes,
+      // each with its own digit scale.
+      for (int u = 0; u < a.kt; ++u) {
+      const int vw = warp * a.kt + u;                   // index of the 32-byte block in the column
+      const int c0 = vw * 2;                            // its two 16-byte chunks
+      // ---- the block's rows of g: 1 (8-bit) or 2 (4-bit) per lane ------------------------
       float g0, g1 = 0.0f;
       if (BITS == 8) {
         if (GBF16) g0 = __uint_as_float(static_cast<uint32_t>(
-                        reinterpret_cast<const unsigned short*>(st + a.g_off)[warp * WROWS + lane]) << 16);
-        else g0 = reinterpret_cast<const float*>(st + a.g_off)[warp * WROWS + lane];
+                        reinterpret_cast<const unsigned short*>(st + a.g_off)[vw * WROWS + lane]) << 16);
+        else g0 = reinterpret_cast<const float*>(st + a.g_off)[vw * WROWS + lane];
       } else {
         if (GBF16) {
-          const uint32_t pr = reinterpret_cast<const uint32_t*>(st + a.g_off)[warp * 32 + lane];
+          const uint32_t pr = reinterpret_cast<const uint32_t*>(st + a.g_off)[vw * 32 + lane];
           g0 = twa_bf16_lo(pr);
           g1 = twa_bf16_hi(pr);
         } else {
-          const float2 pr = reinterpret_cast<const float2*>(st + a.g_off)[warp * 32 + lane];
+          const float2 pr = reinterpret_cast<const float2*>(st + a.g_off)[vw * 32 + lane];
           g0 = pr.x;
           g1 = pr.y;
         }
@@ -280,7 +287,7 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
             int j = mt * 16 + lr + 8 * (lm & 1);
             j = j < jmax ? j : jmax;
             uint32_t r[4];
-            ldmatrix_x4(chunk_addr(tile_base, j, c0 + (lm >> 1)), r);
+            ldmatrix_x4(chunk_addr(tile_base, col_bytes, j, c0 + (lm >> 1)), r);
             int c[4] = {0, 0, 0, 0};
             if (BITS == 8) {
 #pragma unroll
@@ -303,7 +310,8 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
           }
         }
       }
-      __syncwarp();
+      __syncwarp();                                      // digit scratch is reused by the next block
+      }  // blocks of the warp
       if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
       if (++s == a.stages) {
         s = 0;
@@ -406,9 +414,8 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
 
   if (warp == MMA_WARPS) {
     if (lane == 0)
-      producer_loop_mma<0, 1, 1, ROWS>(hdr, ring, &map_p, nullptr, a.tiles, a.stages, a.stage_bytes,
-                                       0, a.tx_bytes, a.reverse != 0, a.status,
-                                       a.wait_limit_ns);
+      producer_loop_mma(hdr, ring, &map_p, nullptr, a.tiles, a.stages, a.stage_bytes, a.kt, 0, 0, 0, 0,
+                        a.tx_bytes, a.reverse != 0, a.status, a.wait_limit_ns);
     return;
   }
   if (bad && tid == 0) twa_set_status(a.status, TWA_ERR_NONFINITE, -1);
@@ -436,33 +443,38 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
     }
   }
 
-  const int c0 = warp * 2;
   const int lm = lane >> 3, lr = lane & 7;
   const int jmax = a.n - 1;
-  // Rows this lane finishes (tig < 2 only): chunk c0 + tig, LROWS rows starting at LROWS * gid.
-  const int lane_row = (warp * 32 + 16 * tig) * (8 / BITS) + LROWS * gid;
+  const int col_bytes = TWA_TILE_COL_BYTES * a.kt;
+  // The warp owns bytes [32*kt*warp, 32*kt*(warp+1)) of every column: kt blocks of two 16-byte
+  // chunks.  Lanes with tig < 2 finish chunk tig of a block: LROWS rows starting at LROWS * gid.
   volatile int* abort_flag = &hdr->abort_flag;
   int s = 0;
   unsigned phase = 0;
   for (int t = blockIdx.x; t < a.tiles; t += gridDim.x) {
     const int tile = a.reverse ? (a.tiles - 1 - t) : t;
-    const long long row = static_cast<long long>(tile) * ROWS + lane_row;
-    float bv[LROWS];
+    const long long tile_row0 = static_cast<long long>(tile) * ROWS * a.kt;
+    long long row[2];
+    float bv[2][LROWS];
 #pragma unroll
-    for (int i = 0; i < LROWS; ++i) bv[i] = 0.0f;
-    if (a.base && tig < 2) {
-      if (row + LROWS <= a.D) {
-        if (LROWS == 2) {
-          const float2 x = *reinterpret_cast<const float2*>(a.base + row);
-          bv[0] = x.x; bv[1] = x.y;
+    for (int u = 0; u < 2; ++u) {
+      row[u] = tile_row0 + ((warp * a.kt + u) * 32 + 16 * tig) * (8 / BITS) + LROWS * gid;
+#pragma unroll
+      for (int i = 0; i < LROWS; ++i) bv[u][i] = 0.0f;
+      if (u < a.kt && a.base && tig < 2) {
+        if (row[u] + LROWS <= a.D) {
+          if (LROWS == 2) {
+            const float2 x = *reinterpret_cast<const float2*>(a.base + row[u]);
+            bv[u][0] = x.x; bv[u][1] = x.y;
+          } else {
+            const float4 x = *reinterpret_cast<const float4*>(a.base + row[u]);
+            bv[u][0] = x.x; bv[u][1] = x.y; bv[u][2] = x.z; bv[u][3] = x.w;
+          }
         } else {
-          const float4 x = *reinterpret_cast<const float4*>(a.base + row);
-          bv[0] = x.x; bv[1] = x.y; bv[2] = x.z; bv[3] = x.w;
-        }
-      } else {
 #pragma unroll
-        for (int i = 0; i < LROWS; ++i)
-          if (row + i < a.D) bv[i] = a.base[row + i];
+          for (int i = 0; i < LROWS; ++i)
+            if (row[u] + i < a.D) bv[u][i] = a.base[row[u] + i];
+        }
       }
     }
     if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
@@ -470,75 +482,85 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
       break;
     }
     const uint32_t tile_base = twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes);
-    float keep[LROWS];
+    float keep[2][LROWS];
 #pragma unroll
-    for (int i = 0; i < LROWS; ++i) keep[i] = 0.0f;
+    for (int u = 0; u < 2; ++u) {
 #pragma unroll
-    for (int ch = 0; ch < 2; ++ch) {
-      int acc0[4] = {0, 0, 0, 0};                       // 8-bit: rows 2gid, 2gid+1; 4-bit: rows 4gid, 4gid+2
-      int acc1[4] = {0, 0, 0, 0};                       // 4-bit only: rows 4gid+1, 4gid+3
+      for (int i = 0; i < LROWS; ++i) keep[u][i] = 0.0f;
+      if (u < a.kt) {
+        const int c0 = (warp * a.kt + u) * 2;
 #pragma unroll
-      for (int ks = 0; ks < 4; ++ks) {
-        if (ks < KS) {
-          int j = ks * 32 + lm * 8 + lr;
-          j = j < jmax ? j : jmax;
-          uint32_t r[4];
-          ldmatrix_x4_trans(chunk_addr(tile_base, j, c0 + ch), r);
-          if (BITS == 8) {
+        for (int ch = 0; ch < 2; ++ch) {
+          int acc0[4] = {0, 0, 0, 0};                   // 8-bit: rows 2gid, 2gid+1; 4-bit: rows 4gid, 4gid+2
+          int acc1[4] = {0, 0, 0, 0};                   // 4-bit only: rows 4gid+1, 4gid+3
 #pragma unroll
-            for (int i = 0; i < 4; ++i) r[i] ^= 0x80808080u;
-            const uint32_t af[4] = {__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[0], r[1], 0x7531),
-                                    __byte_perm(r[2], r[3], 0x6420), __byte_perm(r[2], r[3], 0x7531)};
-            mma_s8(acc0, af, bfrag[ks][0], bfrag[ks][1]);
-          } else {
-            uint32_t e[4], o[4];
+          for (int ks = 0; ks < 4; ++ks) {
+            if (ks < KS) {
+              int j = ks * 32 + lm * 8 + lr;
+              j = j < jmax ? j : jmax;
+              uint32_t r[4];
+              ldmatrix_x4_trans(chunk_addr(tile_base, col_bytes, j, c0 + ch), r);
+              if (BITS == 8) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              e[i] = ((r[i] << 4) & 0xF0F0F0F0u) ^ 0x80808080u;
-              o[i] = (r[i] & 0xF0F0F0F0u) ^ 0x80808080u;
+                for (int i = 0; i < 4; ++i) r[i] ^= 0x80808080u;
+                const uint32_t af[4] = {__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[0], r[1], 0x7531),
+                                        __byte_perm(r[2], r[3], 0x6420), __byte_perm(r[2], r[3], 0x7531)};
+                mma_s8(acc0, af, bfrag[ks][0], bfrag[ks][1]);
+              } else {
+                uint32_t e[4], o[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  e[i] = ((r[i] << 4) & 0xF0F0F0F0u) ^ 0x80808080u;
+                  o[i] = (r[i] & 0xF0F0F0F0u) ^ 0x80808080u;
+                }
+                const uint32_t ae[4] = {__byte_perm(e[0], e[1], 0x6420), __byte_perm(e[0], e[1], 0x7531),
+                                        __byte_perm(e[2], e[3], 0x6420), __byte_perm(e[2], e[3], 0x7531)};
+                const uint32_t ao[4] = {__byte_perm(o[0], o[1], 0x6420), __byte_perm(o[0], o[1], 0x7531),
+                                        __byte_perm(o[2], o[3], 0x6420), __byte_perm(o[2], o[3], 0x7531)};
+                mma_s8(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
+                mma_s8(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
+              }
             }
-            const uint32_t ae[4] = {__byte_perm(e[0], e[1], 0x6420), __byte_perm(e[0], e[1], 0x7531),
-                                    __byte_perm(e[2], e[3], 0x6420), __byte_perm(e[2], e[3], 0x7531)};
-            const uint32_t ao[4] = {__byte_perm(o[0], o[1], 0x6420), __byte_perm(o[0], o[1], 0x7531),
-                                    __byte_perm(o[2], o[3], 0x6420), __byte_perm(o[2], o[3], 0x7531)};
-            mma_s8(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
-            mma_s8(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
+          }
+          // digit sums -> float; the four digits of a row sit in lanes tig = 0, 1 of its quad
+          float v[LROWS];
+          if (BITS == 8) {
+            v[0] = fmaf(small_int_to_float(acc0[1]), wb, small_int_to_float(acc0[0]) * wa);
+            v[1] = fmaf(small_int_to_float(acc0[3]), wb, small_int_to_float(acc0[2]) * wa);
+          } else {
+            v[0] = fmaf(small_int_to_float(acc0[1]), wb, small_int_to_float(acc0[0]) * wa);
+            v[2] = fmaf(small_int_to_float(acc0[3]), wb, small_int_to_float(acc0[2]) * wa);
+            v[1] = fmaf(small_int_to_float(acc1[1]), wb, small_int_to_float(acc1[0]) * wa);
+            v[3] = fmaf(small_int_to_float(acc1[3]), wb, small_int_to_float(acc1[2]) * wa);
+          }
+#pragma unroll
+          for (int i = 0; i < LROWS; ++i) {
+            v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 1);
+            v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 2);
+            if (tig == ch) keep[u][i] = v[i];
           }
         }
-      }
-      // digit sums -> float; the four digits of a row sit in lanes tig = 0, 1 of its quad
-      float v[LROWS];
-      if (BITS == 8) {
-        v[0] = fmaf(small_int_to_float(acc0[1]), wb, small_int_to_float(acc0[0]) * wa);
-        v[1] = fmaf(small_int_to_float(acc0[3]), wb, small_int_to_float(acc0[2]) * wa);
-      } else {
-        v[0] = fmaf(small_int_to_float(acc0[1]), wb, small_int_to_float(acc0[0]) * wa);
-        v[2] = fmaf(small_int_to_float(acc0[3]), wb, small_int_to_float(acc0[2]) * wa);
-        v[1] = fmaf(small_int_to_float(acc1[1]), wb, small_int_to_float(acc1[0]) * wa);
-        v[3] = fmaf(small_int_to_float(acc1[3]), wb, small_int_to_float(acc1[2]) * wa);
-      }
-#pragma unroll
-      for (int i = 0; i < LROWS; ++i) {
-        v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 1);
-        v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 2);
-        if (tig == ch) keep[i] = v[i];
       }
     }
     __syncwarp();
     if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
-    if (tig < 2) {
-      if (row + LROWS <= a.D) {
-        if (LROWS == 2) {
-          *reinterpret_cast<float2*>(a.out + row) = make_float2(bv[0] + keep[0] + poison, bv[1] + keep[1] + poison);
-        } else {
-          *reinterpret_cast<float4*>(a.out + row) =
-              make_float4(bv[0] + keep[0] + poison, bv[1] + keep[1] + poison, bv[2] + keep[2] + poison,
-                          bv[3] + keep[3] + poison);
-        }
-      } else {
 #pragma unroll
-        for (int i = 0; i < LROWS; ++i)
-          if (row + i < a.D) a.out[row + i] = bv[i] + keep[i] + poison;
+    for (int u = 0; u < 2; ++u) {
+      if (u < a.kt && tig < 2) {
+        if (row[u] + LROWS <= a.D) {
+          if (LROWS == 2) {
+            *reinterpret_cast<float2*>(a.out + row[u]) =
+                make_float2(bv[u][0] + keep[u][0] + poison, bv[u][1] + keep[u][1] + poison);
+          } else {
+            *reinterpret_cast<float4*>(a.out + row[u]) =
+                make_float4(bv[u][0] + keep[u][0] + poison, bv[u][1] + keep[u][1] + poison,
+                            bv[u][2] + keep[u][2] + poison, bv[u][3] + keep[u][3] + poison);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < LROWS; ++i)
+            if (row[u] + i < a.D) a.out[row[u] + i] = bv[u][i] + keep[u][i] + poison;
+        }
       }
     }
     if (++s == a.stages) {
@@ -551,13 +573,19 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
 // =================================================================================================
 // host side
 // =================================================================================================
-int encode_tile_map(twa_ctx* ctx, const twa_basis* P, CUtensorMap* map) {
+// segments per tile column: two for narrow bases, so that a tile stays worth a handshake
+int choose_kt(const twa_ctx* ctx, int n) {
+  if (ctx->tune_tile_segments == 1 || ctx->tune_tile_segments == 2) return ctx->tune_tile_segments;
+  return n <= 64 ? 2 : 1;
+}
+
+int encode_tile_map(twa_ctx* ctx, const twa_basis* P, int kt, CUtensorMap* map) {
   long long row_bytes = (P->D * P->bits + 7) / 8;
   // quantised columns are stored in whole, internally permuted 512-byte segments
   if (P->bits != 32) row_bytes = (row_bytes + 511) / 512 * 512;
   cuuint64_t dims[2] = {static_cast<cuuint64_t>((row_bytes + 3) / 4), static_cast<cuuint64_t>(P->n)};
   cuuint64_t strides[1] = {static_cast<cuuint64_t>(P->col_stride)};
-  cuuint32_t box[2] = {TWA_TILE_COL_WORDS, static_cast<cuuint32_t>(P->n)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(TWA_TILE_COL_WORDS * kt), static_cast<cuuint32_t>(P->n)};
   cuuint32_t es[2] = {1, 1};
   CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, P->data, dims, strides, box, es,
                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
@@ -617,10 +645,11 @@ int launch_lift_mma_t(twa_ctx* ctx, const CUtensorMap& mp, const LiftMmaArgs& a,
 int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
                            const twa_project_epilogue& epi, void* ws) {
   const bool bf16 = g_dtype == TWA_BF16;
-  const int rows = twa_tile_rows(P->bits);
+  const int kt = choose_kt(ctx, P->n);
+  const int rows = twa_tile_rows(P->bits) * kt;
   const int gsz = bf16 ? 2 : 4;
   CUtensorMap mp, mg;
-  int rc = encode_tile_map(ctx, P, &mp);
+  int rc = encode_tile_map(ctx, P, kt, &mp);
   if (rc) return rc;
   rc = encode_g_map(ctx, g, P->D, bf16, &mg);
   if (rc) return rc;
@@ -629,7 +658,8 @@ int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_
   a.D = P->D;
   a.n = P->n;
   a.tiles = static_cast<int>((P->D + rows - 1) / rows);
-  a.g_off = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES;
+  a.kt = kt;
+  a.g_off = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt;
   a.tx_bytes = a.g_off + static_cast<unsigned>(rows * gsz);
   a.stage_bytes = static_cast<unsigned>(round_up_i(static_cast<int>(a.tx_bytes), 1024));
   const int fixed = TWA_SMEM_HEADER + MMA_WARPS * DIGIT_SCRATCH + 1024;   // 1024: alignment slack
@@ -663,15 +693,17 @@ int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_
 
 int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
                         const float* base, float* out, bool reverse_tiles) {
-  const int rows = twa_tile_rows(P->bits);
+  const int kt = choose_kt(ctx, P->n);
+  const int rows = twa_tile_rows(P->bits) * kt;
   CUtensorMap mp;
-  int rc = encode_tile_map(ctx, P, &mp);
+  int rc = encode_tile_map(ctx, P, kt, &mp);
   if (rc) return rc;
   LiftMmaArgs a;
   a.D = P->D;
   a.n = P->n;
   a.tiles = static_cast<int>((P->D + rows - 1) / rows);
-  a.tx_bytes = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES;
+  a.kt = kt;
+  a.tx_bytes = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt;
   a.stage_bytes = static_cast<unsigned>(round_up_i(static_cast<int>(a.tx_bytes), 1024));
   const int fixed = TWA_SMEM_HEADER + 4 * TWA_MAX_N + 1024;               // 1024: alignment slack
   int stages = (ctx->smem_optin - fixed) / static_cast<int>(a.stage_bytes);

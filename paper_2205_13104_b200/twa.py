@@ -36,6 +36,7 @@ TWA_TUNE_LIFT_WARPS = 2
 TWA_TUNE_STAGES = 3
 TWA_TUNE_WAIT_LIMIT_MS = 4
 TWA_TUNE_DEQUANT_PATH = 5
+TWA_TUNE_TILE_SEGMENTS = 6
 
 EXPORTS = [
     "twa_create", "twa_destroy", "twa_get_status", "twa_clear_status", "twa_strerror",

@@ -440,3 +440,35 @@ def test_chunked_build_reports_rank_deficiency(env):
     code, detail = twa.twa_get_status(ctx)
     assert (code, detail) == (twa.TWA_ERR_RANK_DEFICIENT, 3)
     twa.twa_clear_status(ctx)
+
+
+@pytest.mark.parametrize("segments", [1, 2])
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("D,n", [(4099, 33), (70001, 100), (131072, 8)])
+def test_tile_segments_knob(env, D, n, bits, segments):
+    """Both tile heights of the tensor-pipe kernels, whatever the built-in choice for this n."""
+    ctx, ws = env
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_TILE_SEGMENTS, segments)
+    try:
+        P = random_basis(D, n, 900 + D + n)
+        B = twa.twa_quantize_basis(ctx, twa.basis_from_tensor(P, D), bits, ws)
+        codes, s = twa.twa_basis_export(ctx, B)
+        co, so = orc.unpack_codes(codes.cpu().numpy(), D, bits), s.cpu().numpy()
+        gen = torch.Generator(device=DEV)
+        gen.manual_seed(D + n + bits)
+        g = (torch.randn(D, generator=gen, device=DEV) * 1e-4).bfloat16()
+        alpha = torch.randn(n, generator=gen, device=DEV)
+        base = torch.randn(D, generator=gen, device=DEV)
+        c = torch.empty(n, device=DEV)
+        w = torch.full((D + 8,), 5.0, device=DEV)
+        twa.twa_project(ctx, B, g, c, ws)
+        twa.twa_lift(ctx, B, alpha, base, w, ws)
+        status_ok(ctx)
+        assert rel(c.cpu().numpy(), orc.project(co, so, g.float().cpu().numpy())) <= TOL
+        w_ref = orc.lift(co, so, alpha.cpu().numpy(), base.cpu().numpy())
+        assert rel(w[:D].cpu().numpy(), w_ref) <= TOL
+        assert rel(w[:D].cpu().numpy().astype(np.float64) - base.cpu().numpy(),
+                   w_ref - base.cpu().numpy()) <= 1e-4          # P alpha carried by a float32 w
+        assert torch.all(w[D:] == 5.0)
+    finally:
+        twa.twa_set_tuning(ctx, twa.TWA_TUNE_TILE_SEGMENTS, 0)
