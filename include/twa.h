@@ -170,9 +170,10 @@ int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float
  *          [row0, row0+rows) of the candidates.  row0 must be a multiple of 1024, rows a
  *          multiple of 1024 except for the chunk that ends at D.  Any order, each row range
  *          exactly once per pass, the same partition in every pass.
- *  q32_out passes 2 and 3, optional: D x n float32 destination (column stride ldq elements)
- *          that receives the float32 basis rows of the chunk.  With bits == 32 this is the
- *          only output and pass 3 is not run.
+ *  q32_out passes 2 and 3, optional: rows x n float32 destination for the float32 basis rows
+ *          of this chunk, column-major with column stride ldq >= rows elements (to assemble
+ *          the whole basis pass base + row0 and the full column stride).  With bits == 32
+ *          this is the only output and pass 3 is not run.
  *  Pq      the caller sets data (twa_basis_bytes) and scales before twa_build_end_pass(2).
  *  bws     device scratch of twa_build_workspace_bytes(n) bytes, alive until the last call.
  * Device-side errors: TWA_ERR_RANK_DEFICIENT (same 1e-5 rule as twa_build_basis),

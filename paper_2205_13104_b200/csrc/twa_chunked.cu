@@ -32,7 +32,7 @@ struct ChunkArgs {
   double* partials;         // [grid][NP*NP]  (modes 0, 1)
   float* wbar;              // mode 0
   unsigned* absmax;         // mode 2
-  float* q32;               // modes 2, 3, optional: q32[j * ldq + global row]
+  float* q32;               // modes 2, 3, optional: q32[j * ldq + row inside the chunk]
   long long ldq;
   unsigned char* codes;     // mode 3
   long long code_stride;
@@ -136,11 +136,10 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
             for (int v = 0; v < JB; ++v) acc[u][v] = fma(x[u], y[v], acc[u][v]);
         }
       } else {
-        const long long grow = a.row0 + r;
 #pragma unroll
         for (int j = 0; j < NP; ++j) {
           const float qf = static_cast<float>(q[j]);
-          if (a.q32 && valid && j < a.n) a.q32[j * a.ldq + grow] = qf;
+          if (a.q32 && valid && j < a.n) a.q32[j * a.ldq + r] = qf;
           if (MODE == 2) {
             const unsigned m = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(qf) & 0x7FFFFFFFu);
             if ((tid & 31) == 0 && j < a.n) atomicMax(&smax[j], m);
@@ -318,7 +317,7 @@ int twa_build_feed(twa_ctx* ctx, int pass, const float* chunk, int64_t ldc, int6
   if (rows < 1 || row0 < 0 || row0 + rows > D || ldc < rows) return TWA_ERR_INVALID_ARG;
   // chunks start and (except the last) end on whole code segments
   if (row0 % 1024 != 0 || (row0 + rows != D && rows % 1024 != 0)) return TWA_ERR_MISALIGNED;
-  if (q32_out && ldq < D) return TWA_ERR_INVALID_ARG;
+  if (q32_out && ldq < rows) return TWA_ERR_INVALID_ARG;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
   const BuildLayout l = layout_for(np);
   char* ws = ctx->build_ws;

@@ -277,7 +277,8 @@ def twa_build_begin(ctx, D, n, wbar_out, bws):
 
 def twa_build_feed(ctx, pass_index, chunk, row0, rows, Pq=None, q32_out=None):
     """chunk: float32 CUDA tensor view (n, >= rows) whose row i holds rows [row0, row0+rows) of
-    candidate i (stride(0) = column stride); q32_out: float32 (n, ldq) tensor or None."""
+    candidate i (stride(0) = column stride); q32_out: None or a float32 view (n, >= rows) laid out
+    the same way that receives the float32 basis rows of this chunk."""
     assert chunk.dtype == torch.float32 and chunk.stride(1) == 1
     rc = load().twa_build_feed(ctx, int(pass_index), _ptr(chunk), int(chunk.stride(0)), int(row0),
                                int(rows), ctypes.byref(Pq.desc) if Pq is not None else None,
@@ -289,6 +290,23 @@ def twa_build_end_pass(ctx, pass_index, bits=0, Pq=None):
     rc = load().twa_build_end_pass(ctx, int(pass_index), int(bits),
                                    ctypes.byref(Pq.desc) if Pq is not None else None)
     _check(rc, "twa_build_end_pass", ctx)
+
+
+def basis_view(P, row0=0, rows=None, col0=0, cols=None):
+    """Descriptor of a block of rows and columns of a basis, sharing its memory.  For 8/4-bit
+    storage the block must respect the internal chunk order: col0 a multiple of 8 and row0 a
+    multiple of one 512-byte segment (512 rows at 8 bits, 1024 at 4 bits)."""
+    rows = P.D - row0 if rows is None else rows
+    cols = P.n - col0 if cols is None else cols
+    assert 0 <= row0 and row0 + rows <= P.D and 0 <= col0 and col0 + cols <= P.n
+    if P.bits != 32:
+        assert col0 % 8 == 0 and (row0 * P.bits // 8) % 512 == 0
+    else:
+        assert row0 % 4 == 0
+    off = col0 * P.col_stride + row0 * P.bits // 8
+    desc = twa_basis(P.desc.data + off, (P.desc.scales + 4 * col0) if P.desc.scales else None,
+                     int(rows), P.col_stride, int(cols), P.bits)
+    return Basis(desc, P.data, P.scales)
 
 
 def new_quantised_basis(D, n, bits, device):

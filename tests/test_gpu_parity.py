@@ -377,7 +377,7 @@ def _chunked_build(ctx, W, D, bits, chunk_rows, want_q32=True):
         for r0 in order:
             rows = min(chunk_rows, D - r0)
             twa.twa_build_feed(ctx, p, W[:, r0:], r0, rows, Pq=Pq if p == 3 else None,
-                               q32_out=q32 if p >= 2 else None)
+                               q32_out=q32[:, r0:] if p >= 2 else None)
         twa.twa_build_end_pass(ctx, p, bits if p == 2 else 0, Pq if p == 2 else None)
     return wbar, q32, Pq
 
