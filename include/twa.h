@@ -66,9 +66,9 @@ typedef struct twa_ctx twa_ctx;
 
 /* Descriptor of a projection matrix P (D x n), held by the caller.
  *  bits == 32: data holds float32 values.
- *  bits == 8 : one byte per element, value = code + 128 (offset binary), code in [-127,127].
+ *  bits == 8 : one two's-complement byte per element, code in [-127,127].
  *  bits == 4 : two elements per byte, row 2k in the low nibble and row 2k+1 in the high
- *              nibble, nibble = code + 8, code in [-7,7].
+ *              nibble, two's-complement nibbles, code in [-7,7].
  *  The represented value is scales[j] * code (Section 4.6, with one symmetric factor per
  *  column instead of two per layer).  The storage of codes is internal to the library: inside
  *  every aligned 512-byte segment of a column the 16-byte chunks are stored in a

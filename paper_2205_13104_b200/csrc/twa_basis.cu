@@ -161,7 +161,7 @@ __global__ void __launch_bounds__(BLOCK) encode_kernel(const float* __restrict__
                                                        long long out_stride) {
   constexpr int RPT = 128 / BITS;                     // rows per thread-iteration
   constexpr float QMAX = BITS == 8 ? 127.0f : 7.0f;
-  constexpr int BIAS = BITS == 8 ? 128 : 8;
+  constexpr uint32_t MASK = BITS == 8 ? 0xFFu : 0xFu;    // two's-complement byte or nibble
   const int j = blockIdx.y;
   const float* col = P + j * ld;
   const float s = scales[j];
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(BLOCK) encode_kernel(const float* __restrict__
     uint32_t w[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int k = 0; k < RPT; ++k) {
-      const uint32_t u = static_cast<uint32_t>(twa_encode_one(p[k], s, QMAX) + BIAS);
+      const uint32_t u = static_cast<uint32_t>(twa_encode_one(p[k], s, QMAX)) & MASK;
       if (BITS == 8) w[k >> 2] |= u << (8 * (k & 3));
       else w[k >> 3] |= u << (4 * (k & 7));
     }
@@ -198,7 +198,8 @@ __device__ __forceinline__ long long internal_pos(long long b, int j) {
   return (((q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j)) << 4) | (b & 15);
 }
 
-// internal (offset binary, chunk-permuted, padded) -> canonical (two's complement, tight)
+// internal (chunk-permuted, padded) -> canonical (tight); `mask` is XORed into every byte (0 today:
+// both images hold two's-complement codes)
 __global__ void __launch_bounds__(BLOCK) export_kernel(const unsigned char* __restrict__ in,
                                                        long long in_stride,
                                                        unsigned char* __restrict__ out,
@@ -374,7 +375,7 @@ int twa_basis_export(twa_ctx* ctx, const twa_basis* Pq, void* codes_out, float* 
   if (per < 1) per = 1;
   export_kernel<<<dim3(per, Pq->n), BLOCK, 0, ctx->stream>>>(
       static_cast<const unsigned char*>(Pq->data), Pq->col_stride,
-      static_cast<unsigned char*>(codes_out), row_bytes, Pq->bits == 8 ? 0x80 : 0x88);
+      static_cast<unsigned char*>(codes_out), row_bytes, 0);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   TWA_CUDA_OK(ctx, cudaMemcpyAsync(scales_out, Pq->scales, sizeof(float) * Pq->n,
                                    cudaMemcpyDeviceToDevice, ctx->stream));
@@ -395,7 +396,7 @@ int twa_basis_import(twa_ctx* ctx, const void* codes, const float* scales, int64
   if (per < 1) per = 1;
   import_kernel<<<dim3(per, n), BLOCK, 0, ctx->stream>>>(
       static_cast<const unsigned char*>(codes), row_bytes, static_cast<unsigned char*>(Pq->data),
-      stride, bits == 8 ? 0x80 : 0x88);
+      stride, 0);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   TWA_CUDA_OK(ctx, cudaMemcpyAsync(Pq->scales, scales, sizeof(float) * n, cudaMemcpyDeviceToDevice,
                                    ctx->stream));

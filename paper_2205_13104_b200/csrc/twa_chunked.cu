@@ -161,11 +161,11 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
             if (a.bits == 8) {
 #pragma unroll
               for (int k = 0; k < 16; ++k)
-                w[k >> 2] |= static_cast<uint32_t>(twa_encode_one(src[k], s, qmax) + 128) << (8 * (k & 3));
+                w[k >> 2] |= (static_cast<uint32_t>(twa_encode_one(src[k], s, qmax)) & 0xFFu) << (8 * (k & 3));
             } else {
 #pragma unroll
               for (int k = 0; k < 32; ++k)
-                w[k >> 3] |= static_cast<uint32_t>(twa_encode_one(src[k], s, qmax) + 8) << (4 * (k & 7));
+                w[k >> 3] |= (static_cast<uint32_t>(twa_encode_one(src[k], s, qmax)) & 0xFu) << (4 * (k & 7));
             }
             const long long qidx = (a.row0 + tile * RT) / rows_per_chunk + c;   // logical 16-byte chunk of the column
             const long long slot = (qidx & ~31LL) | twa_chunk_slot(static_cast<int>(qidx & 31), j);

@@ -193,8 +193,9 @@ __device__ __forceinline__ void twa_named_barrier(int id, int threads) {
 }
 
 // ---- code -> float ------------------------------------------------------------------------
-// A byte u in [0,255] placed in the low mantissa bits of 2^23 gives the float 2^23 + u
-// exactly; subtracting 2^23 + bias leaves the signed code as a float.
+// Float path: a two's-complement byte (nibble) becomes offset binary by flipping its top bit;
+// a byte u in [0,255] placed in the low mantissa bits of 2^23 gives the float 2^23 + u exactly;
+// subtracting 2^23 + bias leaves the signed code as a float.
 __device__ __forceinline__ float twa_byte_to_float(uint32_t word, int byte, float magic) {
   const uint32_t sel = 0x7440u + static_cast<uint32_t>(byte);
   return __uint_as_float(__byte_perm(word, 0x4B000000u, sel)) - magic;

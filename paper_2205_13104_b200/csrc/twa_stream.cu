@@ -100,7 +100,8 @@ __device__ __forceinline__ void producer_loop(SmemHeader* hdr, unsigned char* ri
 template <int BITS>
 __device__ __forceinline__ float lane_dot(const unsigned char* col16, const float* g) {
   const uint4 c = *reinterpret_cast<const uint4*>(col16);
-  const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+  const uint32_t flip = BITS == 8 ? 0x80808080u : (BITS == 4 ? 0x88888888u : 0u);   // code -> offset binary
+  const uint32_t w[4] = {c.x ^ flip, c.y ^ flip, c.z ^ flip, c.w ^ flip};
   float t;
   if (BITS == 32) {
     t = __uint_as_float(w[0]) * g[0];
@@ -271,7 +272,9 @@ twa_project_kernel(const __grid_constant__ CUtensorMap map_p,
 // acc[i] += coef * code for the lane's 8 bytes of one column.
 template <int BITS, int LR>
 __device__ __forceinline__ void lane_axpy(const unsigned char* col8, float coef, float* acc) {
-  const uint2 c = *reinterpret_cast<const uint2*>(col8);
+  uint2 c = *reinterpret_cast<const uint2*>(col8);
+  if (BITS == 8) { c.x ^= 0x80808080u; c.y ^= 0x80808080u; }      // code -> offset binary
+  if (BITS == 4) { c.x ^= 0x88888888u; c.y ^= 0x88888888u; }
   if (BITS == 32) {
     acc[0] = fmaf(__uint_as_float(c.x), coef, acc[0]);
     acc[1] = fmaf(__uint_as_float(c.y), coef, acc[1]);

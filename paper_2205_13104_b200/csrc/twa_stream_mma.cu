@@ -7,9 +7,9 @@
 // traffic, which measured 5.7 instructions per code and 80 % issue utilisation at 60 % of DRAM
 // throughput.  Here the codes go from shared memory to the tensor pipe as they are:
 //
-//   project:  g is cut, per 32 (8-bit) or 64 (4-bit) rows, into four signed base-128 digits of a
-//             common power-of-two scale (block fixed point, 2^-29 of the block maximum, finer
-//             than float32 relative to the block), and  sum_r code[r,j] * digit_k[r]  is one
+//   project:  g is cut, per 32 or 64 bytes of a column (32 to 128 rows), into four signed base-128
+//             digits of a common power-of-two scale (block fixed point, 2^-29 of the block
+//             maximum, finer than float32 relative to the block), and  sum_r code[r,j] * digit_k[r]  is one
 //             integer MMA per 16 columns; the four digit sums are recombined in float32.
 //   lift:     the n coefficients s_j * alpha_j are cut into digits once per kernel, and
 //             sum_j code[r,j] * digit_k[j]  is an integer MMA per 16 rows and 32 columns.
@@ -105,13 +105,6 @@ __device__ __forceinline__ uint32_t cut_digits(float t) {
   const uint32_t lo = __byte_perm(__float_as_uint(m0), __float_as_uint(m1), 0x0040);  // bytes m0.b0, m1.b0
   const uint32_t hi = __byte_perm(__float_as_uint(m2), __float_as_uint(m3), 0x0040);
   return __byte_perm(lo, hi, 0x5410);
-}
-
-// Shared address of logical 16-byte chunk `chunk` (0 .. 32*kt-1) of column j of a tile whose
-// columns are col_bytes = 512*kt long.
-__device__ __forceinline__ uint32_t chunk_addr(uint32_t tile_base, int col_bytes, int j, int chunk) {
-  return tile_base + static_cast<uint32_t>(j * col_bytes + ((chunk >> 5) << 9)) +
-         (static_cast<uint32_t>(twa_chunk_slot(chunk & 31, j)) << 4);
 }
 
 // g_boxes 1-D boxes of 256 gradient elements follow the tile of P~ in a stage (project only).
@@ -212,6 +205,20 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
     const int lm = lane >> 3, lr = lane & 7;            // ldmatrix: matrix and row this lane addresses
     const int jmax = a.n - 1;                           // last column that exists in shared memory
     const int col_bytes = TWA_TILE_COL_BYTES * a.kt;
+    // The warp owns bytes [32*kt*warp, 32*kt*(warp+1)) of every column: kt blocks of 32 bytes.
+    // Offsets, inside a tile, of the 16-byte chunk this lane hands to ldmatrix for block u and
+    // column group mt (they do not change from tile to tile).
+    uint32_t aoff[2][8];
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt) {
+        int j = mt * 16 + lr + 8 * (lm & 1);
+        j = j < jmax ? j : jmax;
+        const int chunk = (warp * a.kt + (u < a.kt ? u : 0)) * 2 + (lm >> 1);
+        aoff[u][mt] = static_cast<uint32_t>(j * col_bytes + ((chunk >> 5) << 9) +
+                                            (twa_chunk_slot(chunk & 31, j) << 4));
+      }
     volatile int* abort_flag = &hdr->abort_flag;
     int s = 0;
     unsigned phase = 0;
@@ -222,96 +229,101 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
         break;
       }
       const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
-      // The warp owns bytes [32*kt*warp, 32*kt*(warp+1)) of every column: kt blocks of 32 bytes,
-      // each with its own digit scale.
-      for (int u = 0; u < a.kt; ++u) {
-      const int vw = warp * a.kt + u;                   // index of the 32-byte block in the column
-      const int c0 = vw * 2;                            // its two 16-byte chunks
-      // ---- the block's rows of g: 1 (8-bit) or 2 (4-bit) per lane ------------------------
-      float g0, g1 = 0.0f;
-      if (BITS == 8) {
-        if (GBF16) g0 = __uint_as_float(static_cast<uint32_t>(
-                        reinterpret_cast<const unsigned short*>(st + a.g_off)[vw * WROWS + lane]) << 16);
-        else g0 = reinterpret_cast<const float*>(st + a.g_off)[vw * WROWS + lane];
-      } else {
-        if (GBF16) {
-          const uint32_t pr = reinterpret_cast<const uint32_t*>(st + a.g_off)[vw * 32 + lane];
-          g0 = twa_bf16_lo(pr);
-          g1 = twa_bf16_hi(pr);
-        } else {
-          const float2 pr = reinterpret_cast<const float2*>(st + a.g_off)[vw * 32 + lane];
-          g0 = pr.x;
-          g1 = pr.y;
+      const uint32_t tile_base = twa_smem_u32(st);
+      // ---- the warp's rows of g: per block 1 (8-bit) or 2 (4-bit) per lane -------------------
+      float g0[2] = {0.0f, 0.0f}, g1[2] = {0.0f, 0.0f};
+      unsigned mb = 0u;
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        if (u < a.kt) {
+          const int vw = warp * a.kt + u;               // index of the 32-byte block in the column
+          if (BITS == 8) {
+            if (GBF16) g0[u] = __uint_as_float(static_cast<uint32_t>(
+                           reinterpret_cast<const unsigned short*>(st + a.g_off)[vw * WROWS + lane]) << 16);
+            else g0[u] = reinterpret_cast<const float*>(st + a.g_off)[vw * WROWS + lane];
+          } else {
+            if (GBF16) {
+              const uint32_t pr = reinterpret_cast<const uint32_t*>(st + a.g_off)[vw * 32 + lane];
+              g0[u] = twa_bf16_lo(pr);
+              g1[u] = twa_bf16_hi(pr);
+            } else {
+              const float2 pr = reinterpret_cast<const float2*>(st + a.g_off)[vw * 32 + lane];
+              g0[u] = pr.x;
+              g1[u] = pr.y;
+            }
+            mb = max(mb, __float_as_uint(g1[u]) & 0x7FFFFFFFu);
+          }
+          mb = max(mb, __float_as_uint(g0[u]) & 0x7FFFFFFFu);
         }
       }
-      unsigned mb = __float_as_uint(g0) & 0x7FFFFFFFu;
-      if (BITS == 4) mb = max(mb, __float_as_uint(g1) & 0x7FFFFFFFu);
-      mb = __reduce_max_sync(0xFFFFFFFFu, mb);
+      mb = __reduce_max_sync(0xFFFFFFFFu, mb);          // one digit scale for the warp's rows of the tile
       const unsigned ebits = mb >> 23;
       if (ebits >= 255u) bad = true;                    // NaN or Inf in g
-      // Blocks whose largest |g| is below 2^-122 contribute nothing representable: skipped.
+      // Rows whose largest |g| is below 2^-122 contribute nothing representable: skipped.
       if (ebits >= 5u && ebits < 255u) {
-        // |g| < 2^(ebits-126) in the block; t = g * 2^(132-ebits) lies in (-64, 64)
+        // |g| < 2^(ebits-126) here; t = g * 2^(132-ebits) lies in (-64, 64)
         const float up = __uint_as_float((259u - ebits) << 23);
-        const uint32_t d0 = cut_digits(g0 * up);
         // weight of digit k: 2^(ebits-132) / 128^k
         const float w0 = (ebits >= 6u) ? __uint_as_float((ebits - 5u) << 23) : 5.877471754e-39f;
         const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
         float wa = tig == 0 ? w0 : (tig == 1 ? w2 : 0.0f);        // digits 2*tig, 2*tig+1 sit in this lane's
         float wb = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);        // accumulator columns
         if (BITS == 4) { wa *= 0.0625f; wb *= 0.0625f; }          // 4-bit codes enter the MMA times 16
-        uint32_t b0, b1, b2 = 0, b3 = 0;
-        if (BITS == 8) {
+        int c[8][4];
 #pragma unroll
-          for (int k = 0; k < 4; ++k) digw[k * 32 + lane] = static_cast<unsigned char>(d0 >> (8 * k));
-          __syncwarp();
-          b0 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 4 * tig) : 0u;
-          b1 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 16 + 4 * tig) : 0u;
-        } else {
-          const uint32_t d1 = cut_digits(g1 * up);
+        for (int mt = 0; mt < 8; ++mt) c[mt][0] = c[mt][1] = c[mt][2] = c[mt][3] = 0;
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            digw[k * 32 + lane] = static_cast<unsigned char>(d0 >> (8 * k));          // even rows
-            digw[128 + k * 32 + lane] = static_cast<unsigned char>(d1 >> (8 * k));    // odd rows
+        for (int u = 0; u < 2; ++u) {
+          if (u < a.kt) {
+            const uint32_t d0 = cut_digits(g0[u] * up);
+            uint32_t b0, b1, b2 = 0, b3 = 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) digw[k * 32 + lane] = static_cast<unsigned char>(d0 >> (8 * k));
+            if (BITS == 4) {
+              const uint32_t d1 = cut_digits(g1[u] * up);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) digw[128 + k * 32 + lane] = static_cast<unsigned char>(d1 >> (8 * k));
+            }
+            __syncwarp();
+            b0 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 4 * tig) : 0u;
+            b1 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 16 + 4 * tig) : 0u;
+            if (BITS == 4) {                              // second scratch half: the odd rows
+              b2 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 4 * tig) : 0u;
+              b3 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 16 + 4 * tig) : 0u;
+            }
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+              if (mt < MT) {
+                uint32_t r[4];
+                ldmatrix_x4(tile_base + aoff[u][mt], r);
+                if (BITS == 8) {
+                  mma_s8(c[mt], r, b0, b1);
+                } else {
+                  uint32_t e[4], o[4];
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    e[i] = (r[i] << 4) & 0xF0F0F0F0u;     // even rows: 16 * code
+                    o[i] = r[i] & 0xF0F0F0F0u;            // odd rows:  16 * code
+                  }
+                  mma_s8(c[mt], e, b0, b1);
+                  mma_s8(c[mt], o, b2, b3);
+                }
+              }
+            }
+            __syncwarp();                                // the digit scratch is rewritten by the next block
           }
-          __syncwarp();
-          b0 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 4 * tig) : 0u;
-          b1 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 16 + 4 * tig) : 0u;
-          b2 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 4 * tig) : 0u;
-          b3 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 16 + 4 * tig) : 0u;
         }
-        const uint32_t tile_base = twa_smem_u32(st);
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt) {
           if (mt < MT) {
-            int j = mt * 16 + lr + 8 * (lm & 1);
-            j = j < jmax ? j : jmax;
-            uint32_t r[4];
-            ldmatrix_x4(chunk_addr(tile_base, col_bytes, j, c0 + (lm >> 1)), r);
-            int c[4] = {0, 0, 0, 0};
-            if (BITS == 8) {
-#pragma unroll
-              for (int i = 0; i < 4; ++i) r[i] ^= 0x80808080u;             // code + 128 -> code
-              mma_s8(c, r, b0, b1);
-            } else {
-              uint32_t e[4], o[4];
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                e[i] = ((r[i] << 4) & 0xF0F0F0F0u) ^ 0x80808080u;          // even rows: 16 * code
-                o[i] = (r[i] & 0xF0F0F0F0u) ^ 0x80808080u;                 // odd rows:  16 * code
-              }
-              mma_s8(c, e, b0, b1);
-              mma_s8(c, o, b2, b3);
-            }
-            facc[mt][0] = fmaf(small_int_to_float(c[0]), wa, facc[mt][0]);
-            facc[mt][0] = fmaf(small_int_to_float(c[1]), wb, facc[mt][0]);
-            facc[mt][1] = fmaf(small_int_to_float(c[2]), wa, facc[mt][1]);
-            facc[mt][1] = fmaf(small_int_to_float(c[3]), wb, facc[mt][1]);
+            facc[mt][0] = fmaf(small_int_to_float(c[mt][0]), wa, facc[mt][0]);
+            facc[mt][0] = fmaf(small_int_to_float(c[mt][1]), wb, facc[mt][0]);
+            facc[mt][1] = fmaf(small_int_to_float(c[mt][2]), wa, facc[mt][1]);
+            facc[mt][1] = fmaf(small_int_to_float(c[mt][3]), wb, facc[mt][1]);
           }
         }
       }
-      __syncwarp();                                      // digit scratch is reused by the next block
-      }  // blocks of the warp
+      __syncwarp();
       if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
       if (++s == a.stages) {
         s = 0;
@@ -448,32 +460,52 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
   const int col_bytes = TWA_TILE_COL_BYTES * a.kt;
   // The warp owns bytes [32*kt*warp, 32*kt*(warp+1)) of every column: kt blocks of two 16-byte
   // chunks.  Lanes with tig < 2 finish chunk tig of a block: LROWS rows starting at LROWS * gid.
+  // Offsets, inside a tile, of the chunk this lane hands to ldmatrix for block u, chunk ch and
+  // 32-column step ks (they do not change from tile to tile).
+  uint32_t loff[2][2][4];
+#pragma unroll
+  for (int u = 0; u < 2; ++u)
+#pragma unroll
+    for (int ch = 0; ch < 2; ++ch)
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks) {
+        int j = ks * 32 + lm * 8 + lr;
+        j = j < jmax ? j : jmax;
+        const int chunk = (warp * a.kt + (u < a.kt ? u : 0)) * 2 + ch;
+        loff[u][ch][ks] = static_cast<uint32_t>(j * col_bytes + ((chunk >> 5) << 9) +
+                                                (twa_chunk_slot(chunk & 31, j) << 4));
+      }
+  int lane_row[2];
+#pragma unroll
+  for (int u = 0; u < 2; ++u)
+    lane_row[u] = ((warp * a.kt + u) * 32 + 16 * tig) * (8 / BITS) + LROWS * gid;
+  const int tile_rows = ROWS * a.kt;
   volatile int* abort_flag = &hdr->abort_flag;
   int s = 0;
   unsigned phase = 0;
   for (int t = blockIdx.x; t < a.tiles; t += gridDim.x) {
     const int tile = a.reverse ? (a.tiles - 1 - t) : t;
-    const long long tile_row0 = static_cast<long long>(tile) * ROWS * a.kt;
-    long long row[2];
+    const long long tile_row0 = static_cast<long long>(tile) * tile_rows;
+    const bool whole = tile_row0 + tile_rows <= a.D;     // no row of the tile lies past D
     float bv[2][LROWS];
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
-      row[u] = tile_row0 + ((warp * a.kt + u) * 32 + 16 * tig) * (8 / BITS) + LROWS * gid;
 #pragma unroll
       for (int i = 0; i < LROWS; ++i) bv[u][i] = 0.0f;
       if (u < a.kt && a.base && tig < 2) {
-        if (row[u] + LROWS <= a.D) {
+        const long long row = tile_row0 + lane_row[u];
+        if (whole || row + LROWS <= a.D) {
           if (LROWS == 2) {
-            const float2 x = *reinterpret_cast<const float2*>(a.base + row[u]);
+            const float2 x = *reinterpret_cast<const float2*>(a.base + row);
             bv[u][0] = x.x; bv[u][1] = x.y;
           } else {
-            const float4 x = *reinterpret_cast<const float4*>(a.base + row[u]);
+            const float4 x = *reinterpret_cast<const float4*>(a.base + row);
             bv[u][0] = x.x; bv[u][1] = x.y; bv[u][2] = x.z; bv[u][3] = x.w;
           }
         } else {
 #pragma unroll
           for (int i = 0; i < LROWS; ++i)
-            if (row[u] + i < a.D) bv[u][i] = a.base[row[u] + i];
+            if (row + i < a.D) bv[u][i] = a.base[row + i];
         }
       }
     }
@@ -488,7 +520,6 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
 #pragma unroll
       for (int i = 0; i < LROWS; ++i) keep[u][i] = 0.0f;
       if (u < a.kt) {
-        const int c0 = (warp * a.kt + u) * 2;
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
           int acc0[4] = {0, 0, 0, 0};                   // 8-bit: rows 2gid, 2gid+1; 4-bit: rows 4gid, 4gid+2
@@ -496,13 +527,9 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
             if (ks < KS) {
-              int j = ks * 32 + lm * 8 + lr;
-              j = j < jmax ? j : jmax;
               uint32_t r[4];
-              ldmatrix_x4_trans(chunk_addr(tile_base, col_bytes, j, c0 + ch), r);
+              ldmatrix_x4_trans(tile_base + loff[u][ch][ks], r);
               if (BITS == 8) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) r[i] ^= 0x80808080u;
                 const uint32_t af[4] = {__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[0], r[1], 0x7531),
                                         __byte_perm(r[2], r[3], 0x6420), __byte_perm(r[2], r[3], 0x7531)};
                 mma_s8(acc0, af, bfrag[ks][0], bfrag[ks][1]);
@@ -510,8 +537,8 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
                 uint32_t e[4], o[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                  e[i] = ((r[i] << 4) & 0xF0F0F0F0u) ^ 0x80808080u;
-                  o[i] = (r[i] & 0xF0F0F0F0u) ^ 0x80808080u;
+                  e[i] = (r[i] << 4) & 0xF0F0F0F0u;
+                  o[i] = r[i] & 0xF0F0F0F0u;
                 }
                 const uint32_t ae[4] = {__byte_perm(e[0], e[1], 0x6420), __byte_perm(e[0], e[1], 0x7531),
                                         __byte_perm(e[2], e[3], 0x6420), __byte_perm(e[2], e[3], 0x7531)};
@@ -522,7 +549,8 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
               }
             }
           }
-          // digit sums -> float; the four digits of a row sit in lanes tig = 0, 1 of its quad
+          // digit sums -> float; the four digits of a row sit in lanes tig = 0 and 1 of its quad,
+          // and only those two lanes need the total
           float v[LROWS];
           if (BITS == 8) {
             v[0] = fmaf(small_int_to_float(acc0[1]), wb, small_int_to_float(acc0[0]) * wa);
@@ -536,7 +564,6 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
 #pragma unroll
           for (int i = 0; i < LROWS; ++i) {
             v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 1);
-            v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 2);
             if (tig == ch) keep[u][i] = v[i];
           }
         }
@@ -547,19 +574,20 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
       if (u < a.kt && tig < 2) {
-        if (row[u] + LROWS <= a.D) {
+        const long long row = tile_row0 + lane_row[u];
+        if (whole || row + LROWS <= a.D) {
           if (LROWS == 2) {
-            *reinterpret_cast<float2*>(a.out + row[u]) =
+            *reinterpret_cast<float2*>(a.out + row) =
                 make_float2(bv[u][0] + keep[u][0] + poison, bv[u][1] + keep[u][1] + poison);
           } else {
-            *reinterpret_cast<float4*>(a.out + row[u]) =
+            *reinterpret_cast<float4*>(a.out + row) =
                 make_float4(bv[u][0] + keep[u][0] + poison, bv[u][1] + keep[u][1] + poison,
                             bv[u][2] + keep[u][2] + poison, bv[u][3] + keep[u][3] + poison);
           }
         } else {
 #pragma unroll
           for (int i = 0; i < LROWS; ++i)
-            if (row[u] + i < a.D) a.out[row[u] + i] = bv[u][i] + keep[u][i] + poison;
+            if (row + i < a.D) a.out[row + i] = bv[u][i] + keep[u][i] + poison;
         }
       }
     }
