@@ -171,7 +171,9 @@ __device__ __forceinline__ void init_barriers(twa_smem_header* hdr, int stages) 
 // =================================================================================================
 // project
 // =================================================================================================
-template <int BITS, bool GBF16>
+// MT = number of 16-column groups, ceil(n / 16): a compile-time constant so that the MMA loops
+// carry no guards and only the accumulators that exist are kept.
+template <int BITS, bool GBF16, int MT>
 __global__ void __launch_bounds__(MMA_THREADS, 1)
 twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
                        const __grid_constant__ CUtensorMap map_g, const ProjectMmaArgs a) {
@@ -190,10 +192,9 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
   if (threadIdx.x < TWA_MAX_N) hdr->c_part[threadIdx.x] = 0.0f;
   __syncthreads();
 
-  const int MT = (a.n + 15) >> 4;                      // 16-column groups
-  float facc[8][2];
+  float facc[MT][2];
 #pragma unroll
-  for (int mt = 0; mt < 8; ++mt) facc[mt][0] = facc[mt][1] = 0.0f;
+  for (int mt = 0; mt < MT; ++mt) facc[mt][0] = facc[mt][1] = 0.0f;
 
   if (warp == MMA_WARPS) {
     if (lane == 0)
@@ -208,11 +209,11 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
     // The warp owns bytes [32*kt*warp, 32*kt*(warp+1)) of every column: kt blocks of 32 bytes.
     // Offsets, inside a tile, of the 16-byte chunk this lane hands to ldmatrix for block u and
     // column group mt (they do not change from tile to tile).
-    uint32_t aoff[2][8];
+    uint32_t aoff[2][MT];
 #pragma unroll
     for (int u = 0; u < 2; ++u)
 #pragma unroll
-      for (int mt = 0; mt < 8; ++mt) {
+      for (int mt = 0; mt < MT; ++mt) {
         int j = mt * 16 + lr + 8 * (lm & 1);
         j = j < jmax ? j : jmax;
         const int chunk = (warp * a.kt + (u < a.kt ? u : 0)) * 2 + (lm >> 1);
@@ -269,9 +270,9 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
         float wa = tig == 0 ? w0 : (tig == 1 ? w2 : 0.0f);        // digits 2*tig, 2*tig+1 sit in this lane's
         float wb = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);        // accumulator columns
         if (BITS == 4) { wa *= 0.0625f; wb *= 0.0625f; }          // 4-bit codes enter the MMA times 16
-        int c[8][4];
+        int c[MT][4];
 #pragma unroll
-        for (int mt = 0; mt < 8; ++mt) c[mt][0] = c[mt][1] = c[mt][2] = c[mt][3] = 0;
+        for (int mt = 0; mt < MT; ++mt) c[mt][0] = c[mt][1] = c[mt][2] = c[mt][3] = 0;
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
           if (u < a.kt) {
@@ -292,35 +293,31 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
               b3 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 16 + 4 * tig) : 0u;
             }
 #pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-              if (mt < MT) {
-                uint32_t r[4];
-                ldmatrix_x4(tile_base + aoff[u][mt], r);
-                if (BITS == 8) {
-                  mma_s8(c[mt], r, b0, b1);
-                } else {
-                  uint32_t e[4], o[4];
+            for (int mt = 0; mt < MT; ++mt) {
+              uint32_t r[4];
+              ldmatrix_x4(tile_base + aoff[u][mt], r);
+              if (BITS == 8) {
+                mma_s8(c[mt], r, b0, b1);
+              } else {
+                uint32_t e[4], o[4];
 #pragma unroll
-                  for (int i = 0; i < 4; ++i) {
-                    e[i] = (r[i] << 4) & 0xF0F0F0F0u;     // even rows: 16 * code
-                    o[i] = r[i] & 0xF0F0F0F0u;            // odd rows:  16 * code
-                  }
-                  mma_s8(c[mt], e, b0, b1);
-                  mma_s8(c[mt], o, b2, b3);
+                for (int i = 0; i < 4; ++i) {
+                  e[i] = (r[i] << 4) & 0xF0F0F0F0u;       // even rows: 16 * code
+                  o[i] = r[i] & 0xF0F0F0F0u;              // odd rows:  16 * code
                 }
+                mma_s8(c[mt], e, b0, b1);
+                mma_s8(c[mt], o, b2, b3);
               }
             }
             __syncwarp();                                // the digit scratch is rewritten by the next block
           }
         }
 #pragma unroll
-        for (int mt = 0; mt < 8; ++mt) {
-          if (mt < MT) {
-            facc[mt][0] = fmaf(small_int_to_float(c[mt][0]), wa, facc[mt][0]);
-            facc[mt][0] = fmaf(small_int_to_float(c[mt][1]), wb, facc[mt][0]);
-            facc[mt][1] = fmaf(small_int_to_float(c[mt][2]), wa, facc[mt][1]);
-            facc[mt][1] = fmaf(small_int_to_float(c[mt][3]), wb, facc[mt][1]);
-          }
+        for (int mt = 0; mt < MT; ++mt) {
+          facc[mt][0] = fmaf(small_int_to_float(c[mt][0]), wa, facc[mt][0]);
+          facc[mt][0] = fmaf(small_int_to_float(c[mt][1]), wb, facc[mt][0]);
+          facc[mt][1] = fmaf(small_int_to_float(c[mt][2]), wa, facc[mt][1]);
+          facc[mt][1] = fmaf(small_int_to_float(c[mt][3]), wb, facc[mt][1]);
         }
       }
       __syncwarp();
@@ -338,7 +335,7 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
   float* part = reinterpret_cast<float*>(ring);         // [MMA_WARPS][TWA_MAX_N]
   if (warp < MMA_WARPS) {
 #pragma unroll
-    for (int mt = 0; mt < 8; ++mt) {
+    for (int mt = 0; mt < MT; ++mt) {
       float v0 = facc[mt][0], v1 = facc[mt][1];
       v0 += __shfl_xor_sync(0xFFFFFFFFu, v0, 1);
       v1 += __shfl_xor_sync(0xFFFFFFFFu, v1, 1);
@@ -389,7 +386,8 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
 // =================================================================================================
 // lift
 // =================================================================================================
-template <int BITS>
+// KS = number of 32-column steps, ceil(n / 32), a compile-time constant.
+template <int BITS, int KS>
 __global__ void __launch_bounds__(MMA_THREADS, 1)
 twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -441,12 +439,11 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
 
   // B fragments: k-slot 4*tig+i of a 32-column step holds column j0 + {2tig, 2tig+1, 8+2tig, 9+2tig}[i]
   // (and the same + 16 for the second register), the order the transposing loads deliver.
-  const int KS = (a.n + 31) >> 5;
-  uint32_t bfrag[4][2];
+  uint32_t bfrag[KS][2];
 #pragma unroll
-  for (int ks = 0; ks < 4; ++ks) {
+  for (int ks = 0; ks < KS; ++ks) {
     bfrag[ks][0] = bfrag[ks][1] = 0u;
-    if (ks < KS && gid < 4) {
+    if (gid < 4) {
       const unsigned char* tk = table + gid * TWA_MAX_N + ks * 32 + 2 * tig;
       bfrag[ks][0] = static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(tk)) |
                      (static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(tk + 8)) << 16);
@@ -462,13 +459,13 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
   // chunks.  Lanes with tig < 2 finish chunk tig of a block: LROWS rows starting at LROWS * gid.
   // Offsets, inside a tile, of the chunk this lane hands to ldmatrix for block u, chunk ch and
   // 32-column step ks (they do not change from tile to tile).
-  uint32_t loff[2][2][4];
+  uint32_t loff[2][2][KS];
 #pragma unroll
   for (int u = 0; u < 2; ++u)
 #pragma unroll
     for (int ch = 0; ch < 2; ++ch)
 #pragma unroll
-      for (int ks = 0; ks < 4; ++ks) {
+      for (int ks = 0; ks < KS; ++ks) {
         int j = ks * 32 + lm * 8 + lr;
         j = j < jmax ? j : jmax;
         const int chunk = (warp * a.kt + (u < a.kt ? u : 0)) * 2 + ch;
@@ -525,8 +522,8 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
           int acc0[4] = {0, 0, 0, 0};                   // 8-bit: rows 2gid, 2gid+1; 4-bit: rows 4gid, 4gid+2
           int acc1[4] = {0, 0, 0, 0};                   // 4-bit only: rows 4gid+1, 4gid+3
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
-            if (ks < KS) {
+          for (int ks = 0; ks < KS; ++ks) {
+            {
               uint32_t r[4];
               ldmatrix_x4_trans(tile_base + loff[u][ch][ks], r);
               if (BITS == 8) {
@@ -645,10 +642,10 @@ int encode_g_map(twa_ctx* ctx, const void* g, long long D, bool bf16, CUtensorMa
 
 int round_up_i(int x, int m) { return (x + m - 1) / m * m; }
 
-template <int BITS, bool GBF16>
+template <int BITS, bool GBF16, int MT>
 int launch_project_mma_t(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg,
                          const ProjectMmaArgs& a, int grid, int smem) {
-  auto kern = twa_project_mma_kernel<BITS, GBF16>;
+  auto kern = twa_project_mma_kernel<BITS, GBF16, MT>;
   static int smem_limit[64] = {0};   // per device
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[ctx->device & 63], smem);
   if (rc) return rc;
@@ -657,15 +654,44 @@ int launch_project_mma_t(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap&
   return TWA_OK;
 }
 
-template <int BITS>
+template <int BITS, bool GBF16>
+int launch_project_mma_mt(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg,
+                          const ProjectMmaArgs& a, int grid, int smem);
+
+template <int BITS, int KS>
 int launch_lift_mma_t(twa_ctx* ctx, const CUtensorMap& mp, const LiftMmaArgs& a, int grid, int smem) {
-  auto kern = twa_lift_mma_kernel<BITS>;
+  auto kern = twa_lift_mma_kernel<BITS, KS>;
   static int smem_limit[64] = {0};   // per device
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[ctx->device & 63], smem);
   if (rc) return rc;
   kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
+}
+
+template <int BITS, bool GBF16>
+int launch_project_mma_mt(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg,
+                          const ProjectMmaArgs& a, int grid, int smem) {
+  switch ((a.n + 15) >> 4) {
+    case 1: return launch_project_mma_t<BITS, GBF16, 1>(ctx, mp, mg, a, grid, smem);
+    case 2: return launch_project_mma_t<BITS, GBF16, 2>(ctx, mp, mg, a, grid, smem);
+    case 3: return launch_project_mma_t<BITS, GBF16, 3>(ctx, mp, mg, a, grid, smem);
+    case 4: return launch_project_mma_t<BITS, GBF16, 4>(ctx, mp, mg, a, grid, smem);
+    case 5: return launch_project_mma_t<BITS, GBF16, 5>(ctx, mp, mg, a, grid, smem);
+    case 6: return launch_project_mma_t<BITS, GBF16, 6>(ctx, mp, mg, a, grid, smem);
+    case 7: return launch_project_mma_t<BITS, GBF16, 7>(ctx, mp, mg, a, grid, smem);
+    default: return launch_project_mma_t<BITS, GBF16, 8>(ctx, mp, mg, a, grid, smem);
+  }
+}
+
+template <int BITS>
+int launch_lift_mma_ks(twa_ctx* ctx, const CUtensorMap& mp, const LiftMmaArgs& a, int grid, int smem) {
+  switch ((a.n + 31) >> 5) {
+    case 1: return launch_lift_mma_t<BITS, 1>(ctx, mp, a, grid, smem);
+    case 2: return launch_lift_mma_t<BITS, 2>(ctx, mp, a, grid, smem);
+    case 3: return launch_lift_mma_t<BITS, 3>(ctx, mp, a, grid, smem);
+    default: return launch_lift_mma_t<BITS, 4>(ctx, mp, a, grid, smem);
+  }
 }
 
 }  // namespace
@@ -713,10 +739,10 @@ int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_
   if (grid > TWA_MAX_GRID) grid = TWA_MAX_GRID;
   const int smem = static_cast<int>(a.scratch_off) + MMA_WARPS * DIGIT_SCRATCH + 1024;
   if (P->bits == 8)
-    return bf16 ? launch_project_mma_t<8, true>(ctx, mp, mg, a, grid, smem)
-                : launch_project_mma_t<8, false>(ctx, mp, mg, a, grid, smem);
-  return bf16 ? launch_project_mma_t<4, true>(ctx, mp, mg, a, grid, smem)
-              : launch_project_mma_t<4, false>(ctx, mp, mg, a, grid, smem);
+    return bf16 ? launch_project_mma_mt<8, true>(ctx, mp, mg, a, grid, smem)
+                : launch_project_mma_mt<8, false>(ctx, mp, mg, a, grid, smem);
+  return bf16 ? launch_project_mma_mt<4, true>(ctx, mp, mg, a, grid, smem)
+              : launch_project_mma_mt<4, false>(ctx, mp, mg, a, grid, smem);
 }
 
 int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
@@ -750,6 +776,6 @@ int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, fl
   a.wait_limit_ns = ctx->wait_limit_ns;
   const int grid = ctx->sm_count < a.tiles ? ctx->sm_count : a.tiles;
   const int smem = static_cast<int>(a.table_off) + 4 * TWA_MAX_N + 1024;
-  return P->bits == 8 ? launch_lift_mma_t<8>(ctx, mp, a, grid, smem)
-                      : launch_lift_mma_t<4>(ctx, mp, a, grid, smem);
+  return P->bits == 8 ? launch_lift_mma_ks<8>(ctx, mp, a, grid, smem)
+                      : launch_lift_mma_ks<4>(ctx, mp, a, grid, smem);
 }
