@@ -173,7 +173,7 @@ __device__ __forceinline__ void init_barriers(twa_smem_header* hdr, int stages) 
 // =================================================================================================
 // MT = number of 16-column groups, ceil(n / 16): a compile-time constant so that the MMA loops
 // carry no guards and only the accumulators that exist are kept.
-template <int BITS, bool GBF16, int MT>
+template <int BITS, bool GBF16, int MT, int KT>
 __global__ void __launch_bounds__(MMA_THREADS, 1)
 twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
                        const __grid_constant__ CUtensorMap map_g, const ProjectMmaArgs a) {
@@ -198,25 +198,25 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
 
   if (warp == MMA_WARPS) {
     if (lane == 0)
-      producer_loop_mma(hdr, ring, &map_p, &map_g, a.tiles, a.stages, a.stage_bytes, a.kt,
-                        SROWS * a.kt / 256, GSZ, SROWS * a.kt, a.g_off, a.tx_bytes, false, a.status,
+      producer_loop_mma(hdr, ring, &map_p, &map_g, a.tiles, a.stages, a.stage_bytes, KT,
+                        SROWS * KT / 256, GSZ, SROWS * KT, a.g_off, a.tx_bytes, false, a.status,
                         a.wait_limit_ns);
   } else {
     unsigned char* digw = smem + a.scratch_off + warp * DIGIT_SCRATCH;   // this warp's digit bytes
     const int lm = lane >> 3, lr = lane & 7;            // ldmatrix: matrix and row this lane addresses
     const int jmax = a.n - 1;                           // last column that exists in shared memory
-    const int col_bytes = TWA_TILE_COL_BYTES * a.kt;
-    // The warp owns bytes [32*kt*warp, 32*kt*(warp+1)) of every column: kt blocks of 32 bytes.
+    constexpr int col_bytes = TWA_TILE_COL_BYTES * KT;
+    // The warp owns bytes [32*KT*warp, 32*KT*(warp+1)) of every column: KT blocks of 32 bytes.
     // Offsets, inside a tile, of the 16-byte chunk this lane hands to ldmatrix for block u and
     // column group mt (they do not change from tile to tile).
-    uint32_t aoff[2][MT];
+    uint32_t aoff[KT][MT];
 #pragma unroll
-    for (int u = 0; u < 2; ++u)
+    for (int u = 0; u < KT; ++u)
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
         int j = mt * 16 + lr + 8 * (lm & 1);
         j = j < jmax ? j : jmax;
-        const int chunk = (warp * a.kt + (u < a.kt ? u : 0)) * 2 + (lm >> 1);
+        const int chunk = (warp * KT + u) * 2 + (lm >> 1);
         aoff[u][mt] = static_cast<uint32_t>(j * col_bytes + ((chunk >> 5) << 9) +
                                             (twa_chunk_slot(chunk & 31, j) << 4));
       }
@@ -232,12 +232,13 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
       const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
       const uint32_t tile_base = twa_smem_u32(st);
       // ---- the warp's rows of g: per block 1 (8-bit) or 2 (4-bit) per lane -------------------
-      float g0[2] = {0.0f, 0.0f}, g1[2] = {0.0f, 0.0f};
+      float g0[KT], g1[KT];
       unsigned mb = 0u;
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        if (u < a.kt) {
-          const int vw = warp * a.kt + u;               // index of the 32-byte block in the column
+      for (int u = 0; u < KT; ++u) {
+        {
+          g1[u] = 0.0f;
+          const int vw = warp * KT + u;                 // index of the 32-byte block in the column
           if (BITS == 8) {
             if (GBF16) g0[u] = __uint_as_float(static_cast<uint32_t>(
                            reinterpret_cast<const unsigned short*>(st + a.g_off)[vw * WROWS + lane]) << 16);
@@ -274,8 +275,8 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) c[mt][0] = c[mt][1] = c[mt][2] = c[mt][3] = 0;
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          if (u < a.kt) {
+        for (int u = 0; u < KT; ++u) {
+          {
             const uint32_t d0 = cut_digits(g0[u] * up);
             uint32_t b0, b1, b2 = 0, b3 = 0;
 #pragma unroll
@@ -387,7 +388,7 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
 // lift
 // =================================================================================================
 // KS = number of 32-column steps, ceil(n / 32), a compile-time constant.
-template <int BITS, int KS>
+template <int BITS, int KS, int KT>
 __global__ void __launch_bounds__(MMA_THREADS, 1)
 twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -424,7 +425,7 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
 
   if (warp == MMA_WARPS) {
     if (lane == 0)
-      producer_loop_mma(hdr, ring, &map_p, nullptr, a.tiles, a.stages, a.stage_bytes, a.kt, 0, 0, 0, 0,
+      producer_loop_mma(hdr, ring, &map_p, nullptr, a.tiles, a.stages, a.stage_bytes, KT, 0, 0, 0, 0,
                         a.tx_bytes, a.reverse != 0, a.status, a.wait_limit_ns);
     return;
   }
@@ -454,44 +455,45 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
 
   const int lm = lane >> 3, lr = lane & 7;
   const int jmax = a.n - 1;
-  const int col_bytes = TWA_TILE_COL_BYTES * a.kt;
-  // The warp owns bytes [32*kt*warp, 32*kt*(warp+1)) of every column: kt blocks of two 16-byte
+  constexpr int col_bytes = TWA_TILE_COL_BYTES * KT;
+  // The warp owns bytes [32*KT*warp, 32*KT*(warp+1)) of every column: KT blocks of two 16-byte
   // chunks.  Lanes with tig < 2 finish chunk tig of a block: LROWS rows starting at LROWS * gid.
   // Offsets, inside a tile, of the chunk this lane hands to ldmatrix for block u, chunk ch and
   // 32-column step ks (they do not change from tile to tile).
-  uint32_t loff[2][2][KS];
+  uint32_t loff[KT][2][KS];
 #pragma unroll
-  for (int u = 0; u < 2; ++u)
+  for (int u = 0; u < KT; ++u)
 #pragma unroll
     for (int ch = 0; ch < 2; ++ch)
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
         int j = ks * 32 + lm * 8 + lr;
         j = j < jmax ? j : jmax;
-        const int chunk = (warp * a.kt + (u < a.kt ? u : 0)) * 2 + ch;
+        const int chunk = (warp * KT + u) * 2 + ch;
         loff[u][ch][ks] = static_cast<uint32_t>(j * col_bytes + ((chunk >> 5) << 9) +
                                                 (twa_chunk_slot(chunk & 31, j) << 4));
       }
-  int lane_row[2];
+  int lane_row[KT];
 #pragma unroll
-  for (int u = 0; u < 2; ++u)
-    lane_row[u] = ((warp * a.kt + u) * 32 + 16 * tig) * (8 / BITS) + LROWS * gid;
-  const int tile_rows = ROWS * a.kt;
+  for (int u = 0; u < KT; ++u)
+    lane_row[u] = ((warp * KT + u) * 32 + 16 * tig) * (8 / BITS) + LROWS * gid;
+  constexpr int tile_rows = ROWS * KT;
+  const int D = static_cast<int>(a.D);                   // D < 2^31
   volatile int* abort_flag = &hdr->abort_flag;
   int s = 0;
   unsigned phase = 0;
   for (int t = blockIdx.x; t < a.tiles; t += gridDim.x) {
     const int tile = a.reverse ? (a.tiles - 1 - t) : t;
-    const long long tile_row0 = static_cast<long long>(tile) * tile_rows;
-    const bool whole = tile_row0 + tile_rows <= a.D;     // no row of the tile lies past D
-    float bv[2][LROWS];
+    const int tile_row0 = tile * tile_rows;               // < D < 2^31
+    const bool whole = tile_row0 <= D - tile_rows;        // no row of the tile lies past D
+    float bv[KT][LROWS];
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < KT; ++u) {
 #pragma unroll
       for (int i = 0; i < LROWS; ++i) bv[u][i] = 0.0f;
-      if (u < a.kt && a.base && tig < 2) {
-        const long long row = tile_row0 + lane_row[u];
-        if (whole || row + LROWS <= a.D) {
+      if (a.base && tig < 2) {
+        const int row = tile_row0 + lane_row[u];
+        if (whole || row <= D - LROWS) {
           if (LROWS == 2) {
             const float2 x = *reinterpret_cast<const float2*>(a.base + row);
             bv[u][0] = x.x; bv[u][1] = x.y;
@@ -502,7 +504,7 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
         } else {
 #pragma unroll
           for (int i = 0; i < LROWS; ++i)
-            if (row + i < a.D) bv[u][i] = a.base[row + i];
+            if (row + i < D) bv[u][i] = a.base[row + i];
         }
       }
     }
@@ -511,12 +513,12 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
       break;
     }
     const uint32_t tile_base = twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes);
-    float keep[2][LROWS];
+    float keep[KT][LROWS];
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < KT; ++u) {
 #pragma unroll
       for (int i = 0; i < LROWS; ++i) keep[u][i] = 0.0f;
-      if (u < a.kt) {
+      {
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
           int acc0[4] = {0, 0, 0, 0};                   // 8-bit: rows 2gid, 2gid+1; 4-bit: rows 4gid, 4gid+2
@@ -569,10 +571,10 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
     __syncwarp();
     if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      if (u < a.kt && tig < 2) {
-        const long long row = tile_row0 + lane_row[u];
-        if (whole || row + LROWS <= a.D) {
+    for (int u = 0; u < KT; ++u) {
+      if (tig < 2) {
+        const int row = tile_row0 + lane_row[u];
+        if (whole || row <= D - LROWS) {
           if (LROWS == 2) {
             *reinterpret_cast<float2*>(a.out + row) =
                 make_float2(bv[u][0] + keep[u][0] + poison, bv[u][1] + keep[u][1] + poison);
@@ -584,7 +586,7 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
         } else {
 #pragma unroll
           for (int i = 0; i < LROWS; ++i)
-            if (row + i < a.D) a.out[row + i] = bv[u][i] + keep[u][i] + poison;
+            if (row + i < D) a.out[row + i] = bv[u][i] + keep[u][i] + poison;
         }
       }
     }
@@ -645,9 +647,9 @@ int round_up_i(int x, int m) { return (x + m - 1) / m * m; }
 template <int BITS, bool GBF16, int MT>
 int launch_project_mma_t(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg,
                          const ProjectMmaArgs& a, int grid, int smem) {
-  auto kern = twa_project_mma_kernel<BITS, GBF16, MT>;
-  static int smem_limit[64] = {0};   // per device
-  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[ctx->device & 63], smem);
+  auto kern = a.kt == 2 ? twa_project_mma_kernel<BITS, GBF16, MT, 2> : twa_project_mma_kernel<BITS, GBF16, MT, 1>;
+  static int smem_limit[2][64] = {{0}};   // per tile height and device
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[a.kt - 1][ctx->device & 63], smem);
   if (rc) return rc;
   kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, mg, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
@@ -660,9 +662,9 @@ int launch_project_mma_mt(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap
 
 template <int BITS, int KS>
 int launch_lift_mma_t(twa_ctx* ctx, const CUtensorMap& mp, const LiftMmaArgs& a, int grid, int smem) {
-  auto kern = twa_lift_mma_kernel<BITS, KS>;
-  static int smem_limit[64] = {0};   // per device
-  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[ctx->device & 63], smem);
+  auto kern = a.kt == 2 ? twa_lift_mma_kernel<BITS, KS, 2> : twa_lift_mma_kernel<BITS, KS, 1>;
+  static int smem_limit[2][64] = {{0}};   // per tile height and device
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[a.kt - 1][ctx->device & 63], smem);
   if (rc) return rc;
   kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
