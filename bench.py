@@ -70,6 +70,24 @@ def read_traffic(key):
     return None
 
 
+def max_over_ranks(values, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group):
+    a job is as slow as its slowest replica."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_gbps(world, bytes_per_step_per_rank, ms_per_step):
+    """Throughput of the whole job: every rank runs its own replica of the workload (the path has
+    no exchange step), so the bytes add up and the time is the slowest rank's."""
+    return world * bytes_per_step_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 class ClockSampler:
     """nvidia-smi samples of one GPU's clocks and throttle reasons while a region runs."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -319,18 +337,15 @@ def run_ours(args):
     e2e_ms = t0.elapsed_time(t1) / e2e_steps
 
     # ---- max over ranks ------------------------------------------------------------------
-    stats = torch.tensor([total_ms, e2e_ms, proj_ms, lift_ms, build_ms, quant_ms],
-                         dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms, proj_ms, lift_ms, build_ms, quant_ms = stats.tolist()
+    total_ms, e2e_ms, proj_ms, lift_ms, build_ms, quant_ms = max_over_ranks(
+        [total_ms, e2e_ms, proj_ms, lift_ms, build_ms, quant_ms], dev)
 
     if rank == 0:
         peak, peak_kind = load_peaks()
         sb = step_bytes(D, n, bits, g_bytes)
         kb = kernel_bytes(D, n, bits, g_bytes)
         ms_per_step = total_ms / args.steps
-        value = world * sb / (ms_per_step * 1e-3) / 1e9
+        value = whole_job_gbps(world, sb, ms_per_step)
         suffix = "_mma" if args.dequant_path == 0 and bits != 32 else ""
         dom = "project" if proj_ms >= lift_ms else "lift"
         dom_ms = (proj_ms if dom == "project" else lift_ms) / max(rec, 1)

@@ -115,6 +115,11 @@ enum { TWA_TUNE_PROJECT_WARPS = 1, TWA_TUNE_LIFT_WARPS = 2, TWA_TUNE_STAGES = 3,
        TWA_TUNE_WAIT_LIMIT_MS = 4, TWA_TUNE_DEQUANT_PATH = 5, TWA_TUNE_TILE_SEGMENTS = 6 };
 int twa_set_tuning(twa_ctx* ctx, int key, int value);
 
+/* Exercises the bounded wait every streaming kernel uses, without any fault: enqueues one block
+ * that waits (TWA_TUNE_WAIT_LIMIT_MS) for a barrier phase nothing completes.  The kernel then
+ * returns normally and twa_get_status reports TWA_ERR_TIMEOUT; the context stays usable. */
+int twa_selftest_wait(twa_ctx* ctx);
+
 /* Per-kernel timing of twa_step for measurements.  twa_profile_enable(ctx, max_steps > 0)
  * creates CUDA events; from then on each twa_step records three of them (before the
  * projection kernel, between the two kernels, after the lift kernel) until max_steps steps

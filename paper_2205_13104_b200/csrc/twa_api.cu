@@ -17,7 +17,32 @@ bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) 
 
 }  // namespace
 
+namespace {
+// One block waits, with the library's bounded wait, for an mbarrier phase that nothing completes.
+__global__ void wait_selftest_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    twa_mbar_init(twa_smem_u32(&bar), 1);
+    abort_flag = 0;
+    twa_fence_barrier_init();
+  }
+  __syncthreads();
+  if (!twa_mbar_wait(twa_smem_u32(&bar), 0, &abort_flag, limit_ns)) {
+    if (threadIdx.x == 0) twa_set_status(status, TWA_ERR_TIMEOUT, -1);
+  }
+}
+}  // namespace
+
 extern "C" {
+
+int twa_selftest_wait(twa_ctx* ctx) {
+  if (!ctx) return TWA_ERR_INVALID_ARG;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  wait_selftest_kernel<<<1, 64, 0, ctx->stream>>>(ctx->d_status, ctx->wait_limit_ns);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
 
 int twa_create(twa_ctx** out, int device, void* cuda_stream) {
   if (!out) return TWA_ERR_INVALID_ARG;

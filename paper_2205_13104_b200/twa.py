@@ -40,7 +40,7 @@ TWA_TUNE_TILE_SEGMENTS = 6
 
 EXPORTS = [
     "twa_create", "twa_destroy", "twa_get_status", "twa_clear_status", "twa_strerror",
-    "twa_last_error", "twa_set_tuning", "twa_profile_enable", "twa_profile_read",
+    "twa_last_error", "twa_set_tuning", "twa_selftest_wait", "twa_profile_enable", "twa_profile_read",
     "twa_basis_col_stride", "twa_basis_bytes",
     "twa_workspace_bytes", "twa_build_basis", "twa_build_workspace_bytes", "twa_build_begin",
     "twa_build_feed", "twa_build_end_pass", "twa_mean", "twa_quantize_basis",
@@ -109,6 +109,7 @@ def load():
         "twa_strerror": (ctypes.c_char_p, [i32]),
         "twa_last_error": (ctypes.c_char_p, [vp]),
         "twa_set_tuning": (i32, [vp, i32, i32]),
+        "twa_selftest_wait": (i32, [vp]),
         "twa_profile_enable": (i32, [vp, i32]),
         "twa_profile_read": (i32, [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                    ctypes.POINTER(i32)]),
@@ -219,6 +220,10 @@ def twa_clear_status(ctx):
 
 def twa_set_tuning(ctx, key, value):
     _check(load().twa_set_tuning(ctx, int(key), int(value)), "twa_set_tuning", ctx)
+
+
+def twa_selftest_wait(ctx):
+    _check(load().twa_selftest_wait(ctx), "twa_selftest_wait", ctx)
 
 
 def twa_profile_enable(ctx, max_steps):

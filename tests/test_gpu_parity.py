@@ -472,3 +472,27 @@ def test_tile_segments_knob(env, D, n, bits, segments):
         assert torch.all(w[D:] == 5.0)
     finally:
         twa.twa_set_tuning(ctx, twa.TWA_TUNE_TILE_SEGMENTS, 0)
+
+
+def test_bounded_wait_runs_out_cleanly_and_the_context_stays_usable(env):
+    """A wait that nothing satisfies ends after its limit with a status, not a hang or a fault."""
+    ctx, ws = env
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_WAIT_LIMIT_MS, 20)
+    try:
+        twa.twa_selftest_wait(ctx)
+        code, detail = twa.twa_get_status(ctx)
+        assert code == twa.TWA_ERR_TIMEOUT
+    finally:
+        twa.twa_set_tuning(ctx, twa.TWA_TUNE_WAIT_LIMIT_MS, 0)
+        twa.twa_clear_status(ctx)
+    status_ok(ctx)
+    D, n = 4099, 5
+    P = random_basis(D, n, 4)
+    B = twa.twa_quantize_basis(ctx, twa.basis_from_tensor(P, D), 8, ws)
+    g = torch.randn(D, device=DEV)
+    c = torch.empty(n, device=DEV)
+    twa.twa_project(ctx, B, g, c, ws)
+    codes, s = twa.twa_basis_export(ctx, B)
+    co = orc.unpack_codes(codes.cpu().numpy(), D, 8)
+    assert rel(c.cpu().numpy(), orc.project(co, s.cpu().numpy(), g.cpu().numpy())) <= TOL
+    status_ok(ctx)
