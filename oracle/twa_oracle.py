@@ -275,3 +275,129 @@ def step_f32(P32, g, alpha, wbar, lr, lam=0.0):
     alpha_new = sgd_update(alpha, c, lr, lam)
     w_new = lift_f32(P32, alpha_new, wbar)
     return alpha_new, w_new, c
+
+
+# --------------------------------------------------------------------------- #
+# The paper's default construction: decentralise + normalise, layer by layer,
+# per-layer min-max (affine) B-bit codes, one coefficient per (layer, model).
+# `layers` is the list of row offsets [0 = o_0 < o_1 < ... < o_L = D]: layer l
+# owns rows o_l .. o_{l+1}-1 of the flat parameter vector (Section 4.5).
+# --------------------------------------------------------------------------- #
+def center_normalize(W, layers):
+    """e_i^l = (w_i^l - w_bar^l) / ||w_i^l - w_bar^l||_2 for every layer l
+    (Section 4.1, the subspace-construction equation, applied per layer as in
+    Section 4.5; Algorithm 1).  A layer in which a candidate equals the mean
+    gives a zero vector (the paper does not say; such a direction cannot move
+    the weights).  Returns (P float64 (D, n), w_bar float64 (D,))."""
+    W = np.asarray(W)
+    D, n = W.shape
+    wbar = mean(W)
+    P = np.zeros((D, n), dtype=np.float64, order="F")
+    for l in range(len(layers) - 1):
+        a, b = layers[l], layers[l + 1]
+        for i in range(n):
+            v = W[a:b, i].astype(np.float64) - wbar[a:b]
+            nv = float(np.sqrt(np.dot(v, v)))
+            if nv > 0.0:
+                P[a:b, i] = v / nv
+    return P, wbar
+
+
+def affine_factors(P32, layers, bits):
+    """Per-layer factors of the uniform min-max quantiser (Section 4.6):
+    b^l = min(P^l), a^l = fl32(fl32(max(P^l) - min(P^l)) / (2^B - 1)), over all
+    n columns of the layer.  Returns (a float32 (L,), b float32 (L,))."""
+    P32 = np.asarray(P32)
+    assert P32.dtype == np.float32
+    L = len(layers) - 1
+    a = np.zeros(L, dtype=np.float32)
+    b = np.zeros(L, dtype=np.float32)
+    levels = float(2 ** bits - 1)
+    for l in range(L):
+        blk = P32[layers[l]:layers[l + 1], :]
+        lo, hi = np.float32(blk.min()), np.float32(blk.max())
+        span = np.float32(hi - lo)                               # float32 subtraction
+        a[l] = np.float32(np.float64(span) / levels)             # = IEEE float32 division
+        b[l] = lo
+    return a, b
+
+
+def affine_encode(P32, layers, a, b, bits):
+    """code = clamp(round_half_even(fl32(fl32(p - b^l) / a^l)), 0, 2^B - 1); a
+    layer with a^l == 0 (constant layer) is all zeros.  Section 4.6, with the
+    subtraction and the division both rounded to float32 and ties to even (the
+    paper leaves precision and rounding mode open).  Returns uint8 code VALUES
+    of shape (D, n)."""
+    P32 = np.asarray(P32)
+    assert P32.dtype == np.float32
+    D, n = P32.shape
+    top = 2 ** bits - 1
+    codes = np.zeros((D, n), dtype=np.uint8, order="F")
+    for l in range(len(layers) - 1):
+        if a[l] == 0:
+            continue
+        r0, r1 = layers[l], layers[l + 1]
+        d = (P32[r0:r1, :] - np.float32(b[l])).astype(np.float32)          # float32 subtraction
+        t = (d.astype(np.float64) / np.float64(a[l])).astype(np.float32)    # float32 division
+        codes[r0:r1, :] = np.clip(np.rint(t), 0, top).astype(np.uint8)
+    return codes
+
+
+def affine_quantize(P32, layers, bits):
+    a, b = affine_factors(P32, layers, bits)
+    return affine_encode(P32, layers, a, b, bits), a, b
+
+
+def affine_dequantize(codes, layers, a, b):
+    """P~^l = a^l * code + b^l in float64 (Section 4.6)."""
+    codes = np.asarray(codes)
+    out = np.zeros(codes.shape, dtype=np.float64, order="F")
+    for l in range(len(layers) - 1):
+        r0, r1 = layers[l], layers[l + 1]
+        out[r0:r1, :] = np.float64(a[l]) * codes[r0:r1, :].astype(np.float64) + np.float64(b[l])
+    return out
+
+
+def project_layerwise(codes, layers, a, b, g):
+    """c[l, i] = sum_{r in layer l} P~[r, i] g[r] with P~ = a^l code + b^l
+    (Algorithm 1, the update of the variables of layer l).  Returns (L, n)."""
+    codes = np.asarray(codes)
+    g64 = np.asarray(g).astype(np.float64)
+    L, n = len(layers) - 1, codes.shape[1]
+    c = np.zeros((L, n), dtype=np.float64)
+    for l in range(L):
+        r0, r1 = layers[l], layers[l + 1]
+        gl = g64[r0:r1]
+        sg = float(np.sum(gl))
+        for i in range(n):
+            c[l, i] = np.float64(a[l]) * np.dot(codes[r0:r1, i].astype(np.float64), gl) + np.float64(b[l]) * sg
+    return c
+
+
+def lift_layerwise(codes, layers, a, b, beta, base=None):
+    """w^l = base^l + P~^l beta^l (Algorithm 1, the update of the weights of layer
+    l); beta has shape (L, n)."""
+    codes = np.asarray(codes)
+    D, n = codes.shape
+    w = np.zeros(D, dtype=np.float64) if base is None else np.asarray(base).astype(np.float64).copy()
+    for l in range(len(layers) - 1):
+        r0, r1 = layers[l], layers[l + 1]
+        for i in range(n):
+            w[r0:r1] += np.float64(beta[l, i]) * (np.float64(a[l]) * codes[r0:r1, i].astype(np.float64)
+                                                  + np.float64(b[l]))
+    return w
+
+
+def step_layerwise(codes, layers, a, b, g, beta, wbar, lr, lam=0.0):
+    """One iteration of the loop body of Algorithm 1 with its inner loop over the
+    layers.  Returns (beta_new (L, n), w_new, c (L, n))."""
+    c = project_layerwise(codes, layers, a, b, g)
+    beta_new = sgd_update(beta, c, lr, lam)
+    w_new = lift_layerwise(codes, layers, a, b, beta_new, wbar)
+    return beta_new, w_new, c
+
+
+def paper_affine_storage_bytes(D, n, bits, L):
+    """Table "memory_projection" (Section 4.6): n*B*D/8 code bytes plus two
+    4-byte factors per layer."""
+    return n * bits * D / 8 + 8 * L
