@@ -246,6 +246,56 @@ int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host /* host *
                   twa_dtype g_dtype, float lr, float lambda, float* alpha, const float* wbar,
                   float* w, float* w_host /* host */, void* g_stage, void* ws, size_t ws_bytes);
 
+/* ---- the paper's default construction: layer-wise, affine B-bit codes -------------------- */
+
+/* Layers are given as L+1 row offsets of the flat parameter vector on the HOST,
+ * 0 = o_0 < o_1 < ... < o_L = D; layer l owns rows o_l .. o_{l+1}-1 (Section 4.5).
+ *
+ * A layered basis stores P~^l = a^l * code + b^l with unsigned B-bit codes and one (a^l, b^l)
+ * pair per layer (Section 4.6: a^l = (max P^l - min P^l) / (2^B - 1), b^l = min P^l, code =
+ * round((P - b^l) / a^l); here with float32 subtraction and division and round-half-to-even).
+ * The codes use the same column-major chunk-permuted bytes as twa_basis, except that every layer
+ * starts on a 64-byte granule of the column; `granules` maps each granule back to {layer, valid
+ * rows, first flat row, 0}.  All pointers are device pointers into the one buffer `mem` the
+ * caller passed to twa_quantize_affine. */
+typedef struct {
+  twa_basis codes;            /* D = padded rows, bits 8 or 4, scales == NULL                  */
+  float* a;                   /* L scaling factors                                              */
+  float* b;                   /* L zero factors                                                 */
+  int32_t* granules;          /* 4 ints per 64-byte granule of a column                         */
+  int64_t* flat_offsets;      /* L+1 row offsets of the layers in the flat parameter vector     */
+  int64_t* internal_offsets;  /* L+1 row offsets of the layers in the padded storage            */
+  int64_t D;                  /* flat rows                                                      */
+  int32_t L;                  /* layers                                                         */
+} twa_layered_basis;
+
+/* Scratch for the two construction calls below (device, 16-byte aligned). */
+size_t twa_layered_workspace_bytes(const int64_t* offsets_host, int L, int n);
+/* Padded row count and size of `mem` for a layered basis. */
+int64_t twa_layered_rows(const int64_t* offsets_host, int L, int bits);
+size_t twa_layered_basis_bytes(const int64_t* offsets_host, int L, int n, int bits);
+
+/* w_bar and, in place of the candidates, e_i^l = (w_i^l - w_bar^l) / ||w_i^l - w_bar^l||_2 for every
+ * layer l and candidate i (Section 4.1 construction equation applied per layer, Section 4.5;
+ * Algorithm 1).  A layer in which a candidate equals the mean gives a zero vector.  W, ldw,
+ * wbar_out, P32_out as for twa_build_basis.  Synchronises the stream once (uploads the layer
+ * tables from pageable host memory).  Device-side error: TWA_ERR_NONFINITE. */
+int twa_build_centered(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw,
+                       const int64_t* offsets_host, int L, float* wbar_out, twa_basis* P32_out,
+                       void* lws, size_t lws_bytes);
+
+/* Per-layer min-max quantisation of a float32 basis (Section 4.6), bits 8 or 4.
+ *  mem  device buffer of twa_layered_basis_bytes, 256-byte aligned; *out points into it.
+ * Device-side error: TWA_ERR_NONFINITE (detail = layer). */
+int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offsets_host, int L,
+                        int bits, void* mem, size_t mem_bytes, twa_layered_basis* out, void* lws,
+                        size_t lws_bytes);
+
+/* Canonical image for parity checks: unsigned codes in flat row order, n x ceil(D*bits/8) bytes
+ * (4 bits: row 2k low nibble, row 2k+1 high nibble), and the L factors a, b.  Device pointers. */
+int twa_layered_export(twa_ctx* ctx, const twa_layered_basis* lb, void* codes_out, float* a_out,
+                       float* b_out);
+
 /* ---- projection without any allocation ----------------------------------------------- */
 
 /* (No counterpart in the paper: this entry point exists for the way some programs manage

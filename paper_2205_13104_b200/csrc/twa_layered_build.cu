@@ -1,0 +1,479 @@
+// The paper's default construction (Sections 4.1, 4.5, 4.6; Algorithm 1): per layer l,
+// e_i^l = (w_i^l - w_bar^l) / ||w_i^l - w_bar^l||, quantised with the uniform min-max scheme
+// code = round((P - b^l) / a^l), a^l = (max - min) / (2^B - 1), b^l = min, one (a, b) pair per layer.
+//
+// Storage of the codes ("layered basis"): the same column-major, chunk-permuted bytes as the
+// per-column format, but every layer starts on a 64-byte granule of the column, so that a warp's
+// share of a tile always lies in one layer.  A table with one entry per granule maps it back to
+// (layer, first flat row, number of valid rows).
+#include <math.h>
+#include <stdio.h>
+
+#include <algorithm>
+#include <vector>
+
+#include "twa_common.cuh"
+
+namespace {
+
+constexpr int BLOCK = 256;
+constexpr long long ITEM_ROWS = 8192;       // rows of one layer handled by one block
+
+struct Item { int layer; long long r0, r1; };   // flat rows [r0, r1) of one layer
+
+long long granule_rows(int bits) { return 64LL * 8 / bits; }
+
+// host view of the layer partition
+struct Partition {
+  std::vector<long long> flat, internal;     // L+1 offsets each
+  std::vector<Item> items;
+  std::vector<int> first_item;               // L+1
+  long long D_int;
+};
+
+int make_partition(const int64_t* offsets, int L, long long D, int bits, Partition* p) {
+  if (!offsets || L < 1 || offsets[0] != 0 || offsets[L] != D) return TWA_ERR_INVALID_ARG;
+  const long long gr = granule_rows(bits);
+  p->flat.assign(offsets, offsets + L + 1);
+  p->internal.resize(L + 1);
+  p->first_item.resize(L + 1);
+  p->items.clear();
+  long long io = 0;
+  for (int l = 0; l < L; ++l) {
+    const long long len = offsets[l + 1] - offsets[l];
+    if (len < 1) return TWA_ERR_INVALID_ARG;
+    p->internal[l] = io;
+    p->first_item[l] = static_cast<int>(p->items.size());
+    for (long long r = offsets[l]; r < offsets[l + 1]; r += ITEM_ROWS)
+      p->items.push_back({l, r, r + ITEM_ROWS < offsets[l + 1] ? r + ITEM_ROWS : offsets[l + 1]});
+    io += (len + gr - 1) / gr * gr;
+  }
+  p->internal[L] = io;
+  p->first_item[L] = static_cast<int>(p->items.size());
+  p->D_int = io;
+  return io < (1LL << 31) ? TWA_OK : TWA_ERR_UNSUPPORTED;
+}
+
+// ---- kernels ------------------------------------------------------------------------------
+__device__ __forceinline__ double block_sum_d(double v, double* sh) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+  __syncthreads();
+  double t = 0;
+  if (threadIdx.x == 0)
+    for (int w = 0; w < BLOCK / 32; ++w) t += sh[w];
+  return t;
+}
+
+// partial[item][i] = sum over the item's rows of (w - w_bar)^2
+__global__ void __launch_bounds__(BLOCK) centred_sumsq_kernel(const float* __restrict__ W, long long ldw,
+                                                              const float* __restrict__ wbar,
+                                                              const Item* __restrict__ items, int n,
+                                                              double* __restrict__ partial) {
+  __shared__ double sh[BLOCK / 32];
+  const Item it = items[blockIdx.x];
+  const float* col = W + blockIdx.y * ldw;
+  double s = 0;
+  for (long long r = it.r0 + threadIdx.x; r < it.r1; r += BLOCK) {
+    const double v = static_cast<double>(col[r]) - static_cast<double>(wbar[r]);
+    s += v * v;
+  }
+  const double t = block_sum_d(s, sh);
+  if (threadIdx.x == 0) partial[static_cast<size_t>(blockIdx.x) * n + blockIdx.y] = t;
+}
+
+// inv[l][i] = 1 / sqrt(sum of the layer's partials in item order), 0 for a zero vector
+__global__ void inv_norm_kernel(const double* __restrict__ partial, const int* __restrict__ first_item,
+                                int L, int n, double* __restrict__ inv, int* status) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= L * n) return;
+  const int l = idx / n, i = idx - l * n;
+  double s = 0;
+  for (int k = first_item[l]; k < first_item[l + 1]; ++k) s += partial[static_cast<size_t>(k) * n + i];
+  if (!isfinite(s)) twa_set_status(status, TWA_ERR_NONFINITE, i);
+  inv[idx] = (s > 0.0 && isfinite(s)) ? 1.0 / sqrt(s) : 0.0;
+}
+
+__global__ void __launch_bounds__(BLOCK) centre_scale_kernel(float* __restrict__ W, long long ldw,
+                                                             const float* __restrict__ wbar,
+                                                             const Item* __restrict__ items, int n,
+                                                             const double* __restrict__ inv) {
+  const Item it = items[blockIdx.x];
+  float* col = W + blockIdx.y * ldw;
+  const double f = inv[static_cast<size_t>(it.layer) * n + blockIdx.y];
+  for (long long r = it.r0 + threadIdx.x; r < it.r1; r += BLOCK)
+    col[r] = static_cast<float>((static_cast<double>(col[r]) - static_cast<double>(wbar[r])) * f);
+}
+
+// partial min / max of one item over one column
+__global__ void __launch_bounds__(BLOCK) minmax_kernel(const float* __restrict__ P, long long ld,
+                                                       const Item* __restrict__ items, int n,
+                                                       float* __restrict__ pmin, float* __restrict__ pmax) {
+  __shared__ float smin[BLOCK / 32], smax[BLOCK / 32];
+  const Item it = items[blockIdx.x];
+  const float* col = P + blockIdx.y * ld;
+  float lo = INFINITY, hi = -INFINITY;
+  bool bad = false;                              // fmin / fmax drop NaN: track non-finite input apart
+  for (long long r = it.r0 + threadIdx.x; r < it.r1; r += BLOCK) {
+    const float v = col[r];
+    lo = fminf(lo, v);
+    hi = fmaxf(hi, v);
+    bad |= !isfinite(v);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, off));
+    hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, off));
+  }
+  bad = __any_sync(0xFFFFFFFFu, bad);
+  if ((threadIdx.x & 31) == 0) {
+    smin[threadIdx.x >> 5] = bad ? NAN : lo;
+    smax[threadIdx.x >> 5] = hi;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 0; w < BLOCK / 32; ++w) {
+      bad |= isnan(smin[w]);
+      lo = fminf(lo, smin[w]);
+      hi = fmaxf(hi, smax[w]);
+    }
+    pmin[static_cast<size_t>(blockIdx.x) * n + blockIdx.y] = bad ? NAN : lo;
+    pmax[static_cast<size_t>(blockIdx.x) * n + blockIdx.y] = hi;
+  }
+}
+
+// a[l] = (max - min) / (2^B - 1), b[l] = min over the layer's items and all columns
+__global__ void factors_kernel(const float* __restrict__ pmin, const float* __restrict__ pmax,
+                               const int* __restrict__ first_item, int L, int n, float levels,
+                               float* __restrict__ a, float* __restrict__ b, int* status) {
+  const int l = blockIdx.x * blockDim.x + threadIdx.x;
+  if (l >= L) return;
+  float lo = INFINITY, hi = -INFINITY;
+  bool bad = false;
+  for (int k = first_item[l]; k < first_item[l + 1]; ++k)
+    for (int i = 0; i < n; ++i) {
+      const float x = pmin[static_cast<size_t>(k) * n + i], y = pmax[static_cast<size_t>(k) * n + i];
+      bad |= isnan(x) || isnan(y);
+      lo = fminf(lo, x);
+      hi = fmaxf(hi, y);
+    }
+  if (bad) {
+    twa_set_status(status, TWA_ERR_NONFINITE, l);
+    a[l] = 0.0f;
+    b[l] = 0.0f;
+    return;
+  }
+  a[l] = __fdiv_rn(__fsub_rn(hi, lo), levels);
+  b[l] = lo;
+}
+
+// One thread writes one 16-byte chunk of one column: 16 rows (8-bit) or 32 rows (4-bit) of a layer,
+// rows past the layer's end get the code 0.
+template <int BITS>
+__global__ void __launch_bounds__(BLOCK) affine_encode_kernel(const float* __restrict__ P, long long ld,
+                                                              const long long* __restrict__ flat,
+                                                              const long long* __restrict__ internal,
+                                                              const float* __restrict__ a,
+                                                              const float* __restrict__ b,
+                                                              unsigned char* __restrict__ out,
+                                                              long long out_stride) {
+  constexpr int RPC = 128 / BITS;
+  constexpr float TOP = BITS == 8 ? 255.0f : 15.0f;
+  const int l = blockIdx.z, j = blockIdx.y;
+  const long long len = flat[l + 1] - flat[l];
+  const long long chunks = (internal[l + 1] - internal[l]) / RPC;
+  const float al = a[l], bl = b[l];
+  const float* col = P + j * ld + flat[l];
+  uint4* dst = reinterpret_cast<uint4*>(out + j * out_stride);
+  for (long long c = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; c < chunks;
+       c += static_cast<long long>(gridDim.x) * BLOCK) {
+    uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int k = 0; k < RPC; ++k) {
+      const long long r = c * RPC + k;
+      uint32_t u = 0;
+      if (r < len && al != 0.0f) {
+        float q = rintf(__fdiv_rn(__fsub_rn(col[r], bl), al));
+        q = fminf(fmaxf(q, 0.0f), TOP);
+        u = static_cast<uint32_t>(q);
+      }
+      if (BITS == 8) w[k >> 2] |= u << (8 * (k & 3));
+      else w[k >> 3] |= u << (4 * (k & 7));
+    }
+    const long long q = internal[l] / RPC + c;
+    dst[(q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j)] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+// fills the tail of every column (rows from the last layer's end to the column stride) with code 0
+__global__ void tail_zero_kernel(unsigned char* out, long long out_stride, long long first_chunk,
+                                 long long chunks) {
+  const int j = blockIdx.y;
+  uint4* dst = reinterpret_cast<uint4*>(out + j * out_stride);
+  for (long long q = first_chunk + blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; q < chunks;
+       q += static_cast<long long>(gridDim.x) * blockDim.x)
+    dst[(q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j)] = make_uint4(0, 0, 0, 0);
+}
+
+// canonical image for parity: unsigned codes in flat row order, n x ceil(D*bits/8) bytes
+template <int BITS>
+__global__ void __launch_bounds__(BLOCK) layered_export_kernel(const unsigned char* __restrict__ in,
+                                                               long long in_stride,
+                                                               const long long* __restrict__ flat,
+                                                               const long long* __restrict__ internal, int L,
+                                                               long long D, unsigned char* __restrict__ out,
+                                                               long long row_bytes) {
+  const int j = blockIdx.y;
+  const unsigned char* src = in + j * in_stride;
+  unsigned char* dst = out + j * row_bytes;
+  for (long long ob = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; ob < row_bytes;
+       ob += static_cast<long long>(gridDim.x) * BLOCK) {
+    unsigned v = 0;
+#pragma unroll
+    for (int h = 0; h < 8 / BITS; ++h) {
+      const long long r = ob * (8 / BITS) + h;
+      if (r >= D) break;
+      int lo = 0, hi = L;                       // layer of flat row r: last l with flat[l] <= r
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (flat[mid] <= r) lo = mid; else hi = mid;
+      }
+      const long long ir = internal[lo] + (r - flat[lo]);
+      const long long ib = ir * BITS / 8;
+      const long long q = ib >> 4;
+      const unsigned char byte = src[(((q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j)) << 4) | (ib & 15)];
+      const unsigned code = BITS == 8 ? byte : ((byte >> (4 * (ir & 1))) & 0xF);
+      v |= code << (BITS == 8 ? 0 : 4 * h);
+    }
+    dst[ob] = static_cast<unsigned char>(v);
+  }
+}
+
+// device layout of the construction workspace
+struct LwsLayout { size_t items, first_item, flat, internal, partial, pmin, pmax, inv, total; };
+LwsLayout lws_layout(size_t n_items, int L, int n) {
+  LwsLayout w;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = (o + bytes + 255) / 256 * 256; return at; };
+  w.items = take(sizeof(Item) * n_items);
+  w.first_item = take(sizeof(int) * (L + 1));
+  w.flat = take(sizeof(long long) * (L + 1));
+  w.internal = take(sizeof(long long) * (L + 1));
+  w.partial = take(sizeof(double) * n_items * n);
+  w.pmin = take(sizeof(float) * n_items * n);
+  w.pmax = take(sizeof(float) * n_items * n);
+  w.inv = take(sizeof(double) * static_cast<size_t>(L) * n);
+  w.total = o;
+  return w;
+}
+
+int upload_partition(twa_ctx* ctx, const Partition& p, int L, char* lws, const LwsLayout& w) {
+  TWA_CUDA_OK(ctx, cudaMemcpyAsync(lws + w.items, p.items.data(), sizeof(Item) * p.items.size(),
+                                   cudaMemcpyHostToDevice, ctx->stream));
+  TWA_CUDA_OK(ctx, cudaMemcpyAsync(lws + w.first_item, p.first_item.data(), sizeof(int) * (L + 1),
+                                   cudaMemcpyHostToDevice, ctx->stream));
+  TWA_CUDA_OK(ctx, cudaMemcpyAsync(lws + w.flat, p.flat.data(), sizeof(long long) * (L + 1),
+                                   cudaMemcpyHostToDevice, ctx->stream));
+  TWA_CUDA_OK(ctx, cudaMemcpyAsync(lws + w.internal, p.internal.data(), sizeof(long long) * (L + 1),
+                                   cudaMemcpyHostToDevice, ctx->stream));
+  // the host vectors are pageable: the copies above have completed on return, but be explicit
+  TWA_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));
+  return TWA_OK;
+}
+
+size_t count_items(const int64_t* offsets, int L) {
+  size_t k = 0;
+  for (int l = 0; l < L; ++l) k += static_cast<size_t>((offsets[l + 1] - offsets[l] + ITEM_ROWS - 1) / ITEM_ROWS);
+  return k;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t twa_layered_workspace_bytes(const int64_t* offsets_host, int L, int n) {
+  if (!offsets_host || L < 1 || n < 1) return 0;
+  return lws_layout(count_items(offsets_host, L), L, n).total;
+}
+
+int64_t twa_layered_rows(const int64_t* offsets_host, int L, int bits) {
+  if (!offsets_host || L < 1 || (bits != 8 && bits != 4)) return 0;
+  const long long gr = granule_rows(bits);
+  long long io = 0;
+  for (int l = 0; l < L; ++l) io += (offsets_host[l + 1] - offsets_host[l] + gr - 1) / gr * gr;
+  return io;
+}
+
+size_t twa_layered_basis_bytes(const int64_t* offsets_host, int L, int n, int bits) {
+  const int64_t rows = twa_layered_rows(offsets_host, L, bits);
+  if (rows < 1 || n < 1) return 0;
+  const size_t codes = twa_basis_bytes(rows, n, bits);
+  const size_t granules = static_cast<size_t>(twa_basis_col_stride(rows, bits) / 64);
+  return codes + 256 + 2 * ((sizeof(float) * L + 255) / 256 * 256) + 16 * granules +
+         (sizeof(long long) * (L + 1) + 255) / 256 * 256 * 2;
+}
+
+int twa_build_centered(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, const int64_t* offsets_host,
+                       int L, float* wbar_out, twa_basis* P32_out, void* lws, size_t lws_bytes) {
+  if (!ctx || !W || !wbar_out || !P32_out || !offsets_host) return TWA_ERR_INVALID_ARG;
+  if (D < 1 || D >= (1LL << 31) || n < 1 || ldw < D) return TWA_ERR_INVALID_ARG;
+  if (n > TWA_MAX_N) return TWA_ERR_UNSUPPORTED;
+  Partition p;
+  int rc = make_partition(offsets_host, L, D, 8, &p);
+  if (rc) return rc;
+  const LwsLayout w = lws_layout(p.items.size(), L, n);
+  if (!lws || lws_bytes < w.total) return TWA_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(W) & 15) || (ldw & 3) || (reinterpret_cast<uintptr_t>(lws) & 15))
+    return TWA_ERR_MISALIGNED;
+  rc = twa_mean(ctx, W, D, n, ldw, wbar_out);
+  if (rc) return rc;
+  char* ws = static_cast<char*>(lws);
+  rc = upload_partition(ctx, p, L, ws, w);
+  if (rc) return rc;
+  const Item* items = reinterpret_cast<const Item*>(ws + w.items);
+  const int* first_item = reinterpret_cast<const int*>(ws + w.first_item);
+  double* partial = reinterpret_cast<double*>(ws + w.partial);
+  double* inv = reinterpret_cast<double*>(ws + w.inv);
+  const dim3 grid(static_cast<unsigned>(p.items.size()), static_cast<unsigned>(n));
+  centred_sumsq_kernel<<<grid, BLOCK, 0, ctx->stream>>>(W, ldw, wbar_out, items, n, partial);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  inv_norm_kernel<<<(L * n + 255) / 256, 256, 0, ctx->stream>>>(partial, first_item, L, n, inv, ctx->d_status);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  centre_scale_kernel<<<grid, BLOCK, 0, ctx->stream>>>(W, ldw, wbar_out, items, n, inv);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  *P32_out = twa_basis{W, nullptr, D, 4 * ldw, n, 32};
+  return TWA_OK;
+}
+
+int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offsets_host, int L, int bits,
+                        void* mem, size_t mem_bytes, twa_layered_basis* out, void* lws, size_t lws_bytes) {
+  if (!ctx || !P32 || !out || !offsets_host || !mem) return TWA_ERR_INVALID_ARG;
+  if (bits != 8 && bits != 4) return TWA_ERR_UNSUPPORTED;
+  int rc = twa_check_basis(P32);
+  if (rc) return rc;
+  if (P32->bits != 32) return TWA_ERR_INVALID_ARG;
+  const long long D = P32->D;
+  const int n = P32->n;
+  Partition p;
+  rc = make_partition(offsets_host, L, D, bits, &p);
+  if (rc) return rc;
+  const LwsLayout w = lws_layout(p.items.size(), L, n);
+  if (!lws || lws_bytes < w.total) return TWA_ERR_WORKSPACE;
+  if (mem_bytes < twa_layered_basis_bytes(offsets_host, L, n, bits)) return TWA_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(mem) & 255) || (reinterpret_cast<uintptr_t>(lws) & 15)) return TWA_ERR_MISALIGNED;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  char* ws = static_cast<char*>(lws);
+  rc = upload_partition(ctx, p, L, ws, w);
+  if (rc) return rc;
+
+  // carve the caller's buffer: codes | a | b | granule table | flat offsets | internal offsets
+  char* m = static_cast<char*>(mem);
+  const long long stride = twa_basis_col_stride(p.D_int, bits);
+  const size_t codes_bytes = static_cast<size_t>(stride) * n;
+  const size_t fl = (sizeof(float) * L + 255) / 256 * 256;
+  const size_t n_gran = static_cast<size_t>(stride / 64);
+  const size_t off_bytes = (sizeof(long long) * (L + 1) + 255) / 256 * 256;
+  size_t o = (codes_bytes + 255) / 256 * 256;
+  float* a = reinterpret_cast<float*>(m + o); o += fl;
+  float* b = reinterpret_cast<float*>(m + o); o += fl;
+  int* gran = reinterpret_cast<int*>(m + o); o += 16 * n_gran;
+  long long* d_flat = reinterpret_cast<long long*>(m + o); o += off_bytes;
+  long long* d_int = reinterpret_cast<long long*>(m + o);
+
+  // granule table: layer, valid rows, first flat row of every 64-byte granule of a column
+  {
+    const long long gr = granule_rows(bits);
+    std::vector<int> tab(4 * n_gran, 0);
+    for (size_t k = 0; k < n_gran; ++k) tab[4 * k] = -1;              // granules behind the last layer
+    for (int l = 0; l < L; ++l) {
+      const long long len = p.flat[l + 1] - p.flat[l];
+      for (long long k0 = 0; k0 < len; k0 += gr) {
+        const size_t gidx = static_cast<size_t>((p.internal[l] + k0) / gr);
+        tab[4 * gidx] = l;
+        tab[4 * gidx + 1] = static_cast<int>(len - k0 < gr ? len - k0 : gr);
+        tab[4 * gidx + 2] = static_cast<int>(p.flat[l] + k0);
+      }
+    }
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(gran, tab.data(), sizeof(int) * tab.size(), cudaMemcpyHostToDevice,
+                                     ctx->stream));
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_flat, p.flat.data(), sizeof(long long) * (L + 1),
+                                     cudaMemcpyHostToDevice, ctx->stream));
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_int, p.internal.data(), sizeof(long long) * (L + 1),
+                                     cudaMemcpyHostToDevice, ctx->stream));
+    TWA_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));
+  }
+
+  const Item* items = reinterpret_cast<const Item*>(ws + w.items);
+  const int* first_item = reinterpret_cast<const int*>(ws + w.first_item);
+  float* pmin = reinterpret_cast<float*>(ws + w.pmin);
+  float* pmax = reinterpret_cast<float*>(ws + w.pmax);
+  const float* P = static_cast<const float*>(P32->data);
+  const long long ld = P32->col_stride / 4;
+  const dim3 grid(static_cast<unsigned>(p.items.size()), static_cast<unsigned>(n));
+  minmax_kernel<<<grid, BLOCK, 0, ctx->stream>>>(P, ld, items, n, pmin, pmax);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  factors_kernel<<<(L + 127) / 128, 128, 0, ctx->stream>>>(pmin, pmax, first_item, L, n,
+                                                           bits == 8 ? 255.0f : 15.0f, a, b, ctx->d_status);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  long long max_len = 0;
+  for (int l = 0; l < L; ++l) max_len = std::max(max_len, p.internal[l + 1] - p.internal[l]);
+  const int rpc = 128 / bits;
+  long long gx = (max_len / rpc + BLOCK - 1) / BLOCK;
+  if (gx > 64) gx = 64;
+  if (gx < 1) gx = 1;
+  if (L > 65535) return TWA_ERR_UNSUPPORTED;
+  const dim3 egrid(static_cast<unsigned>(gx), static_cast<unsigned>(n), static_cast<unsigned>(L));
+  unsigned char* codes = reinterpret_cast<unsigned char*>(m);
+  const long long* fl_d = reinterpret_cast<const long long*>(ws + w.flat);
+  const long long* in_d = reinterpret_cast<const long long*>(ws + w.internal);
+  if (bits == 8)
+    affine_encode_kernel<8><<<egrid, BLOCK, 0, ctx->stream>>>(P, ld, fl_d, in_d, a, b, codes, stride);
+  else
+    affine_encode_kernel<4><<<egrid, BLOCK, 0, ctx->stream>>>(P, ld, fl_d, in_d, a, b, codes, stride);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  const long long total_chunks = stride / 16, first_tail = p.D_int / rpc;
+  if (first_tail < total_chunks) {
+    tail_zero_kernel<<<dim3(1, n), 64, 0, ctx->stream>>>(codes, stride, first_tail, total_chunks);
+    TWA_CUDA_OK(ctx, cudaGetLastError());
+  }
+  out->codes = twa_basis{codes, nullptr, p.D_int, stride, n, bits};
+  out->a = a;
+  out->b = b;
+  out->granules = gran;
+  out->flat_offsets = reinterpret_cast<int64_t*>(d_flat);
+  out->internal_offsets = reinterpret_cast<int64_t*>(d_int);
+  out->D = D;
+  out->L = L;
+  return TWA_OK;
+}
+
+int twa_layered_export(twa_ctx* ctx, const twa_layered_basis* lb, void* codes_out, float* a_out,
+                       float* b_out) {
+  if (!ctx || !lb || !codes_out || !a_out || !b_out) return TWA_ERR_INVALID_ARG;
+  if (lb->codes.bits != 8 && lb->codes.bits != 4) return TWA_ERR_UNSUPPORTED;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  const int bits = lb->codes.bits, n = lb->codes.n;
+  const long long row_bytes = (lb->D * bits + 7) / 8;
+  long long gx = (row_bytes + BLOCK * 8 - 1) / (BLOCK * 8);
+  if (gx > 1024) gx = 1024;
+  const dim3 grid(static_cast<unsigned>(gx), static_cast<unsigned>(n));
+  if (bits == 8)
+    layered_export_kernel<8><<<grid, BLOCK, 0, ctx->stream>>>(
+        static_cast<const unsigned char*>(lb->codes.data), lb->codes.col_stride,
+        reinterpret_cast<const long long*>(lb->flat_offsets),
+        reinterpret_cast<const long long*>(lb->internal_offsets), lb->L, lb->D,
+        static_cast<unsigned char*>(codes_out), row_bytes);
+  else
+    layered_export_kernel<4><<<grid, BLOCK, 0, ctx->stream>>>(
+        static_cast<const unsigned char*>(lb->codes.data), lb->codes.col_stride,
+        reinterpret_cast<const long long*>(lb->flat_offsets),
+        reinterpret_cast<const long long*>(lb->internal_offsets), lb->L, lb->D,
+        static_cast<unsigned char*>(codes_out), row_bytes);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  TWA_CUDA_OK(ctx, cudaMemcpyAsync(a_out, lb->a, sizeof(float) * lb->L, cudaMemcpyDeviceToDevice, ctx->stream));
+  TWA_CUDA_OK(ctx, cudaMemcpyAsync(b_out, lb->b, sizeof(float) * lb->L, cudaMemcpyDeviceToDevice, ctx->stream));
+  return TWA_OK;
+}
+
+}  // extern "C"

@@ -16,8 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libtwa.so")
 CSRC = os.path.join(_HERE, "csrc")
-SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_chunked.cu", "twa_stream.cu", "twa_stream_mma.cu",
-           "twa_noalloc.cu"]
+SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_chunked.cu", "twa_layered_build.cu", "twa_stream.cu",
+           "twa_stream_mma.cu", "twa_noalloc.cu"]
 
 TWA_MAX_N = 128
 TWA_OK = 0
@@ -45,7 +45,8 @@ EXPORTS = [
     "twa_workspace_bytes", "twa_build_basis", "twa_build_workspace_bytes", "twa_build_begin",
     "twa_build_feed", "twa_build_end_pass", "twa_mean", "twa_quantize_basis",
     "twa_basis_export", "twa_basis_import", "twa_project", "twa_lift", "twa_step",
-    "twa_step_host", "twa_project_noalloc", "twa_noalloc_last_error", "twa_noalloc_scratch_bytes",
+    "twa_step_host", "twa_layered_workspace_bytes", "twa_layered_rows", "twa_layered_basis_bytes",
+    "twa_build_centered", "twa_quantize_affine", "twa_layered_export", "twa_project_noalloc", "twa_noalloc_last_error", "twa_noalloc_scratch_bytes",
 ]
 
 
@@ -54,6 +55,13 @@ class twa_basis(ctypes.Structure):
     _fields_ = [("data", ctypes.c_void_p), ("scales", ctypes.c_void_p),
                 ("D", ctypes.c_int64), ("col_stride", ctypes.c_int64),
                 ("n", ctypes.c_int32), ("bits", ctypes.c_int32)]
+
+
+class twa_layered_basis(ctypes.Structure):
+    """Mirror of the C struct twa_layered_basis."""
+    _fields_ = [("codes", twa_basis), ("a", ctypes.c_void_p), ("b", ctypes.c_void_p),
+                ("granules", ctypes.c_void_p), ("flat_offsets", ctypes.c_void_p),
+                ("internal_offsets", ctypes.c_void_p), ("D", ctypes.c_int64), ("L", ctypes.c_int32)]
 
 
 class TwaError(RuntimeError):
@@ -129,6 +137,13 @@ def load():
         "twa_lift": (i32, [vp, bp, vp, vp, vp, vp, szt]),
         "twa_step": (i32, [vp, bp, vp, i32, f32, f32, vp, vp, vp, vp, vp, szt]),
         "twa_step_host": (i32, [vp, bp, vp, i32, f32, f32, vp, vp, vp, vp, vp, vp, szt]),
+        "twa_layered_workspace_bytes": (szt, [ctypes.POINTER(ctypes.c_int64), i32, i32]),
+        "twa_layered_rows": (i64, [ctypes.POINTER(ctypes.c_int64), i32, i32]),
+        "twa_layered_basis_bytes": (szt, [ctypes.POINTER(ctypes.c_int64), i32, i32, i32]),
+        "twa_build_centered": (i32, [vp, vp, i64, i32, i64, ctypes.POINTER(ctypes.c_int64), i32, vp, bp, vp, szt]),
+        "twa_quantize_affine": (i32, [vp, bp, ctypes.POINTER(ctypes.c_int64), i32, i32, vp, szt,
+                                      ctypes.POINTER(twa_layered_basis), vp, szt]),
+        "twa_layered_export": (i32, [vp, ctypes.POINTER(twa_layered_basis), vp, vp, vp]),
         "twa_project_noalloc": (i32, [i32, vp, bp, vp, i32, vp, vp]),
         "twa_noalloc_last_error": (ctypes.c_char_p, []),
         "twa_noalloc_scratch_bytes": (szt, []),
@@ -415,3 +430,78 @@ def twa_project_noalloc(device, stream, P, g, c_out, status_out=None):
     if rc != TWA_OK:
         raise TwaError(rc, "twa_project_noalloc", twa_noalloc_last_error())
     return c_out
+
+
+# --------------------------------------------------------------------------------------
+# the paper's default construction: layer-wise, affine B-bit codes
+# --------------------------------------------------------------------------------------
+def _offsets(layers):
+    arr = (ctypes.c_int64 * len(layers))(*[int(x) for x in layers])
+    return arr, len(layers) - 1
+
+
+class LayeredBasis:
+    """A twa_layered_basis descriptor with the tensor that owns its memory."""
+
+    def __init__(self, desc, mem, layers):
+        self.desc = desc
+        self.mem = mem
+        self.layers = list(layers)
+
+    D = property(lambda self: self.desc.D)
+    L = property(lambda self: self.desc.L)
+    n = property(lambda self: self.desc.codes.n)
+    bits = property(lambda self: self.desc.codes.bits)
+
+
+def twa_layered_workspace_bytes(layers, n):
+    arr, L = _offsets(layers)
+    return int(load().twa_layered_workspace_bytes(arr, L, int(n)))
+
+
+def twa_layered_rows(layers, bits):
+    arr, L = _offsets(layers)
+    return int(load().twa_layered_rows(arr, L, int(bits)))
+
+
+def twa_layered_basis_bytes(layers, n, bits):
+    arr, L = _offsets(layers)
+    return int(load().twa_layered_basis_bytes(arr, L, int(n), int(bits)))
+
+
+def new_layered_workspace(layers, n, device):
+    return torch.empty(twa_layered_workspace_bytes(layers, n), dtype=torch.uint8, device=device)
+
+
+def twa_build_centered(ctx, W, D, layers, wbar_out, lws):
+    assert W.dtype == torch.float32 and W.is_contiguous()
+    n, ldw = W.shape
+    arr, L = _offsets(layers)
+    desc = twa_basis()
+    rc = load().twa_build_centered(ctx, _ptr(W), int(D), int(n), int(ldw), arr, L, _ptr(wbar_out),
+                                   ctypes.byref(desc), _ptr(lws), lws.numel())
+    _check(rc, "twa_build_centered", ctx)
+    return Basis(desc, W, None)
+
+
+def twa_quantize_affine(ctx, P32, layers, bits, lws):
+    arr, L = _offsets(layers)
+    mem = torch.empty(twa_layered_basis_bytes(layers, P32.n, bits), dtype=torch.uint8,
+                      device=P32.data.device)
+    desc = twa_layered_basis()
+    rc = load().twa_quantize_affine(ctx, ctypes.byref(P32.desc), arr, L, int(bits), _ptr(mem),
+                                    mem.numel(), ctypes.byref(desc), _ptr(lws), lws.numel())
+    _check(rc, "twa_quantize_affine", ctx)
+    return LayeredBasis(desc, mem, layers)
+
+
+def twa_layered_export(ctx, lb):
+    """Canonical unsigned codes (n, ceil(D*bits/8)) uint8 in flat row order and the factors a, b."""
+    row_bytes = (lb.D * lb.bits + 7) // 8
+    dev = lb.mem.device
+    codes = torch.empty((lb.n, row_bytes), dtype=torch.uint8, device=dev)
+    a = torch.empty(lb.L, dtype=torch.float32, device=dev)
+    b = torch.empty(lb.L, dtype=torch.float32, device=dev)
+    _check(load().twa_layered_export(ctx, ctypes.byref(lb.desc), _ptr(codes), _ptr(a), _ptr(b)),
+           "twa_layered_export", ctx)
+    return codes, a, b
