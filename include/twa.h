@@ -267,6 +267,13 @@ typedef struct {
   int64_t* internal_offsets;  /* L+1 row offsets of the layers in the padded storage            */
   int64_t D;                  /* flat rows                                                      */
   int32_t L;                  /* layers                                                         */
+  /* Work split of the step kernels, fixed when the basis is quantised (it depends on the GPU's
+   * multiprocessor count and on the tile height in force then): block k owns tiles
+   * k*tiles_per_cta .. of `tiles`, meets layers cta_first_layer[k] .. and keeps one row of
+   * partial sums per layer it meets, rows cta_run_base[k] .. cta_run_base[k+1]-1. */
+  int32_t cta_count, kt, tiles, tiles_per_cta, total_runs;
+  int32_t* cta_first_layer;   /* cta_count ints                                                 */
+  int32_t* cta_run_base;      /* cta_count + 1 ints                                             */
 } twa_layered_basis;
 
 /* Scratch for the two construction calls below (device, 16-byte aligned). */
@@ -295,6 +302,27 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
  * (4 bits: row 2k low nibble, row 2k+1 high nibble), and the L factors a, b.  Device pointers. */
 int twa_layered_export(twa_ctx* ctx, const twa_layered_basis* lb, void* codes_out, float* a_out,
                        float* b_out);
+
+/* Layer-wise subspace step (Algorithm 1 with the loop over layers of Section 4.5; quantised
+ * basis of Section 4.6).  beta, c_out: L x n floats, layer-major (row l = coefficients of layer
+ * l's n basis vectors).  g, wbar, base, w: D elements in flat row order.  sws: device scratch of
+ * twa_layered_step_workspace_bytes, 256-byte aligned; it carries nothing between calls.
+ *
+ *   project: c^l_i   = sum_r (a^l code[r,i] + b^l) g[r]   over the rows r of layer l
+ *   lift:    w_out[r] = base[r] + sum_i (a^l code[r,i] + b^l) beta^l_i   (base may be NULL)
+ *   step:    c = project(g); beta <- (1 - lr*lambda) beta - lr c; w = lift(beta, wbar)
+ *
+ * Integer dot products are exact; float32 partial sums per warp and layer are combined in
+ * float64 in a fixed order.  Device-side errors: TWA_ERR_NONFINITE (detail = layer),
+ * TWA_ERR_TIMEOUT. */
+size_t twa_layered_step_workspace_bytes(const twa_layered_basis* lb);
+int twa_layered_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype,
+                        float* c_out, void* sws, size_t sws_bytes);
+int twa_layered_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* beta, const float* base,
+                     float* w_out, void* sws, size_t sws_bytes);
+int twa_layered_step(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype,
+                     float lr, float lambda, float* beta, const float* wbar, float* w, float* c_out,
+                     void* sws, size_t sws_bytes);
 
 /* ---- projection without any allocation ----------------------------------------------- */
 

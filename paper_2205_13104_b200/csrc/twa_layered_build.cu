@@ -22,6 +22,8 @@ constexpr long long ITEM_ROWS = 8192;       // rows of one layer handled by one 
 struct Item { int layer; long long r0, r1; };   // flat rows [r0, r1) of one layer
 
 long long granule_rows(int bits) { return 64LL * 8 / bits; }
+constexpr int MAX_CTAS = 1024;                              // blocks of a step kernel
+constexpr size_t CTA_TABLE_BYTES = (sizeof(int) * (MAX_CTAS + 1) + 255) / 256 * 256;
 
 // host view of the layer partition
 struct Partition {
@@ -311,7 +313,7 @@ size_t twa_layered_basis_bytes(const int64_t* offsets_host, int L, int n, int bi
   const size_t codes = twa_basis_bytes(rows, n, bits);
   const size_t granules = static_cast<size_t>(twa_basis_col_stride(rows, bits) / 64);
   return codes + 256 + 2 * ((sizeof(float) * L + 255) / 256 * 256) + 16 * granules +
-         (sizeof(long long) * (L + 1) + 255) / 256 * 256 * 2;
+         (sizeof(long long) * (L + 1) + 255) / 256 * 256 * 2 + 2 * CTA_TABLE_BYTES;
 }
 
 int twa_build_centered(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, const int64_t* offsets_host,
@@ -379,8 +381,33 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
   float* b = reinterpret_cast<float*>(m + o); o += fl;
   int* gran = reinterpret_cast<int*>(m + o); o += 16 * n_gran;
   long long* d_flat = reinterpret_cast<long long*>(m + o); o += off_bytes;
-  long long* d_int = reinterpret_cast<long long*>(m + o);
+  long long* d_int = reinterpret_cast<long long*>(m + o); o += off_bytes;
+  int* d_cta_first = reinterpret_cast<int*>(m + o); o += CTA_TABLE_BYTES;
+  int* d_cta_base = reinterpret_cast<int*>(m + o);
 
+  // work split of the step kernels: contiguous tile ranges, and the layers each range meets
+  const int kt = (ctx->tune_tile_segments == 1 || ctx->tune_tile_segments == 2) ? ctx->tune_tile_segments
+                                                                                : (n <= 64 ? 2 : 1);
+  const long long tile_rows = 512LL * 8 / bits * kt;
+  const int tiles = static_cast<int>((p.D_int + tile_rows - 1) / tile_rows);
+  int ctas = ctx->sm_count < tiles ? ctx->sm_count : tiles;
+  if (ctas > MAX_CTAS) ctas = MAX_CTAS;
+  const int tpc = (tiles + ctas - 1) / ctas;
+  ctas = (tiles + tpc - 1) / tpc;
+  std::vector<int> cta_first(ctas), cta_base(ctas + 1, 0);
+  {
+    int l = 0;
+    for (int k = 0; k < ctas; ++k) {
+      const long long r0 = static_cast<long long>(k) * tpc * tile_rows;       // < D_int
+      long long r1 = r0 + tpc * tile_rows;
+      if (r1 > p.D_int) r1 = p.D_int;
+      while (p.internal[l + 1] <= r0) ++l;
+      cta_first[k] = l;
+      int last = l;
+      while (p.internal[last + 1] < r1) ++last;
+      cta_base[k + 1] = cta_base[k] + (last - l + 1);
+    }
+  }
   // granule table: layer, valid rows, first flat row of every 64-byte granule of a column
   {
     const long long gr = granule_rows(bits);
@@ -400,6 +427,10 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
     TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_flat, p.flat.data(), sizeof(long long) * (L + 1),
                                      cudaMemcpyHostToDevice, ctx->stream));
     TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_int, p.internal.data(), sizeof(long long) * (L + 1),
+                                     cudaMemcpyHostToDevice, ctx->stream));
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_cta_first, cta_first.data(), sizeof(int) * ctas, cudaMemcpyHostToDevice,
+                                     ctx->stream));
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_cta_base, cta_base.data(), sizeof(int) * (ctas + 1),
                                      cudaMemcpyHostToDevice, ctx->stream));
     TWA_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));
   }
@@ -445,6 +476,13 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
   out->internal_offsets = reinterpret_cast<int64_t*>(d_int);
   out->D = D;
   out->L = L;
+  out->cta_count = ctas;
+  out->kt = kt;
+  out->tiles = tiles;
+  out->tiles_per_cta = tpc;
+  out->total_runs = cta_base[ctas];
+  out->cta_first_layer = d_cta_first;
+  out->cta_run_base = d_cta_base;
   return TWA_OK;
 }
 

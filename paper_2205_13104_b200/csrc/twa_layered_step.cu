@@ -1,0 +1,679 @@
+// Subspace step for the paper's default construction (Algorithm 1 with its loop over the layers;
+// Sections 4.2, 4.3, 4.5, 4.6): for every layer l
+//     c^l = P~^l^T g^l,   beta^l <- (1 - eta*lambda) beta^l - eta c^l,   w^l = w_bar^l + P~^l beta^l,
+// with P~^l = a^l * code + b^l, unsigned B-bit codes.
+//
+// Same data path as twa_stream_mma.cu (TMA tiles of the codes, integer MMAs against base-128
+// digits of g and of the coefficients).  What the layers add:
+//  * every block owns a contiguous range of tiles, so it meets few layers; a warp's share of a
+//    tile (32*KT bytes of every column) lies inside one 64-byte granule, hence inside one layer,
+//    and the granule table gives its layer, its first flat row and how many of its rows exist;
+//  * g, w_bar and w are addressed by flat row (layers start anywhere), so they move through
+//    ordinary loads and stores, prefetched one tile ahead;
+//  * projection sums are kept per (block, warp, layer) and combined in a fixed order by a small
+//    second kernel, which also applies a^l, b^l * sum(g^l) and the coefficient update;
+//  * the lift takes its digit fragments per layer from a table made by a third small kernel,
+//    and adds the constant b^l * sum_i beta_i^l.
+#include <stdio.h>
+
+#include <vector>
+
+#include "twa_mma.cuh"
+
+namespace {
+
+constexpr int ROW_FLOATS = 132;                 // one partial row: 128 column sums, sum of g, padding
+
+struct LProjectArgs {
+  int n, stages, tiles, tpc, n_gran;
+  unsigned stage_bytes, tx_bytes, scratch_off;
+  const int4* gran;
+  const void* g;
+  const int* cta_first;
+  const int* cta_base;
+  float* partials;
+  int* status;
+  unsigned long long wait_limit_ns;
+};
+
+struct LLiftArgs {
+  int n, stages, tiles, tpc, n_gran;
+  unsigned stage_bytes, tx_bytes;
+  const int4* gran;
+  const unsigned char* dig;      // [L][4][128] digit bytes of a^l * beta^l_i
+  const int* ebits;              // [L] exponent field of the layer's largest |coefficient|
+  const float* konst;            // [L] b^l * sum_i beta^l_i
+  const float* base;
+  float* out;
+  int* status;
+  unsigned long long wait_limit_ns;
+};
+
+// ------------------------------------------------------------------------------------------------
+template <int BITS, bool GBF16, int MT, int KT>
+__global__ void __launch_bounds__(MMA_THREADS, 1)
+layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProjectArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
+  constexpr int RB = 32 * 8 / BITS;                    // rows behind 32 bytes of a column
+  constexpr int GPT = 8 * KT;                          // granules of a column per tile
+  twa_smem_header* hdr = reinterpret_cast<twa_smem_header*>(smem);
+  unsigned char* ring = smem + TWA_SMEM_HEADER;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gid = lane >> 2, tig = lane & 3;
+  init_barriers(hdr, a.stages);
+  __syncthreads();
+  const int t_first = blockIdx.x * a.tpc;
+  const int t_count = (a.tiles - t_first) < a.tpc ? (a.tiles - t_first) : a.tpc;
+
+  if (warp == MMA_WARPS) {
+    if (lane == 0)
+      producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, KT, 0, 0,
+                        0, 0, a.tx_bytes, false, a.status, a.wait_limit_ns);
+    return;
+  }
+  unsigned char* digw = smem + a.scratch_off + warp * DIGIT_SCRATCH;
+  const int lm = lane >> 3, lr = lane & 7;
+  const int jmax = a.n - 1;
+  constexpr int col_bytes = TWA_TILE_COL_BYTES * KT;
+  uint32_t aoff[KT][MT];
+#pragma unroll
+  for (int u = 0; u < KT; ++u)
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      int j = mt * 16 + lr + 8 * (lm & 1);
+      j = j < jmax ? j : jmax;
+      const int chunk = (warp * KT + u) * 2 + (lm >> 1);
+      aoff[u][mt] = static_cast<uint32_t>(j * col_bytes + ((chunk >> 5) << 9) + (twa_chunk_slot(chunk & 31, j) << 4));
+    }
+  const int wb = warp * 32 * KT;                       // first byte of the warp's share of a tile column
+  const int gran_in_tile = wb >> 6;
+  const int rig0 = (wb & 63) * 8 / BITS;               // first row of the share inside its granule
+  const unsigned short* g16 = static_cast<const unsigned short*>(a.g);
+  const float* g32 = static_cast<const float*>(a.g);
+
+  // the granule entry and the gradient values of one tile
+  int4 e_next;
+  float gn0[KT], gn1[KT];
+  auto fetch = [&](int tile) {
+    const int gi = tile * GPT + gran_in_tile;
+    e_next = gi < a.n_gran ? __ldg(a.gran + gi) : make_int4(-1, 0, 0, 0);
+#pragma unroll
+    for (int u = 0; u < KT; ++u) {
+      gn0[u] = gn1[u] = 0.0f;
+      if (e_next.x >= 0) {
+        const int r = rig0 + u * RB + (BITS == 8 ? lane : 2 * lane);
+        const long long f = static_cast<long long>(e_next.z) + r;
+        if (r < e_next.y) gn0[u] = GBF16 ? __uint_as_float(static_cast<uint32_t>(__ldg(g16 + f)) << 16) : __ldg(g32 + f);
+        if (BITS == 4 && r + 1 < e_next.y)
+          gn1[u] = GBF16 ? __uint_as_float(static_cast<uint32_t>(__ldg(g16 + f + 1)) << 16) : __ldg(g32 + f + 1);
+      }
+    }
+  };
+
+  float facc[MT][2];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) facc[mt][0] = facc[mt][1] = 0.0f;
+  float gsum = 0.0f;
+  int cur_layer = -1;
+  bool bad = false;
+  const int my_first = a.cta_first[blockIdx.x], my_base = a.cta_base[blockIdx.x];
+  auto flush = [&]() {
+    float* row = a.partials + (static_cast<size_t>(my_base + cur_layer - my_first) * MMA_WARPS + warp) * ROW_FLOATS;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      float v0 = facc[mt][0], v1 = facc[mt][1];
+      v0 += __shfl_xor_sync(0xFFFFFFFFu, v0, 1);
+      v1 += __shfl_xor_sync(0xFFFFFFFFu, v1, 1);
+      v0 += __shfl_xor_sync(0xFFFFFFFFu, v0, 2);
+      v1 += __shfl_xor_sync(0xFFFFFFFFu, v1, 2);
+      if (tig == 0) {
+        row[mt * 16 + gid] = bad ? __int_as_float(0x7FC00000) : v0;
+        row[mt * 16 + gid + 8] = bad ? __int_as_float(0x7FC00000) : v1;
+      }
+      facc[mt][0] = facc[mt][1] = 0.0f;
+    }
+    float gs = gsum;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) gs += __shfl_xor_sync(0xFFFFFFFFu, gs, off);
+    if (lane == 0) row[128] = gs;
+    gsum = 0.0f;
+    bad = false;
+  };
+
+  volatile int* abort_flag = &hdr->abort_flag;
+  int s = 0;
+  unsigned phase = 0;
+  fetch(t_first);
+  for (int k = 0; k < t_count; ++k) {
+    const int4 e = e_next;
+    float g0[KT], g1[KT];
+#pragma unroll
+    for (int u = 0; u < KT; ++u) { g0[u] = gn0[u]; g1[u] = gn1[u]; }
+    if (k + 1 < t_count) fetch(t_first + k + 1);
+    if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
+      twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+      break;
+    }
+    if (e.x != cur_layer) {
+      if (cur_layer >= 0) flush();
+      cur_layer = e.x;
+    }
+    if (e.x >= 0) {
+      const uint32_t tile_base = twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes);
+      unsigned mb = 0u;
+#pragma unroll
+      for (int u = 0; u < KT; ++u) {
+        mb = max(mb, __float_as_uint(g0[u]) & 0x7FFFFFFFu);
+        if (BITS == 4) mb = max(mb, __float_as_uint(g1[u]) & 0x7FFFFFFFu);
+        gsum += g0[u] + g1[u];
+      }
+      mb = __reduce_max_sync(0xFFFFFFFFu, mb);
+      const unsigned ebits = mb >> 23;
+      if (ebits >= 255u) bad = true;
+      if (ebits >= 5u && ebits < 255u) {
+        const float up = __uint_as_float((259u - ebits) << 23);
+        const float w0 = (ebits >= 6u) ? __uint_as_float((ebits - 5u) << 23) : 5.877471754e-39f;
+        const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
+        float wa = tig == 0 ? w0 : (tig == 1 ? w2 : 0.0f);
+        float wb_ = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);
+        if (BITS == 4) { wa *= 0.0625f; wb_ *= 0.0625f; }
+        int c[MT][4];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) c[mt][0] = c[mt][1] = c[mt][2] = c[mt][3] = 0;
+#pragma unroll
+        for (int u = 0; u < KT; ++u) {
+          const uint32_t d0 = cut_digits(g0[u] * up);
+          uint32_t b0, b1, b2 = 0, b3 = 0;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) digw[q * 32 + lane] = static_cast<unsigned char>(d0 >> (8 * q));
+          if (BITS == 4) {
+            const uint32_t d1 = cut_digits(g1[u] * up);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) digw[128 + q * 32 + lane] = static_cast<unsigned char>(d1 >> (8 * q));
+          }
+          __syncwarp();
+          b0 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 4 * tig) : 0u;
+          b1 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 16 + 4 * tig) : 0u;
+          if (BITS == 4) {
+            b2 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 4 * tig) : 0u;
+            b3 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 16 + 4 * tig) : 0u;
+          }
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            uint32_t r[4];
+            ldmatrix_x4(tile_base + aoff[u][mt], r);
+            if (BITS == 8) {
+              mma_u8s8(c[mt], r, b0, b1);
+            } else {
+              uint32_t ev[4], od[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                ev[i] = (r[i] << 4) & 0xF0F0F0F0u;       // even rows: 16 * code, unsigned
+                od[i] = r[i] & 0xF0F0F0F0u;              // odd rows
+              }
+              mma_u8s8(c[mt], ev, b0, b1);
+              mma_u8s8(c[mt], od, b2, b3);
+            }
+          }
+          __syncwarp();
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          facc[mt][0] = fmaf(small_int_to_float(c[mt][0]), wa, facc[mt][0]);
+          facc[mt][0] = fmaf(small_int_to_float(c[mt][1]), wb_, facc[mt][0]);
+          facc[mt][1] = fmaf(small_int_to_float(c[mt][2]), wa, facc[mt][1]);
+          facc[mt][1] = fmaf(small_int_to_float(c[mt][3]), wb_, facc[mt][1]);
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
+    if (++s == a.stages) {
+      s = 0;
+      phase ^= 1u;
+    }
+  }
+  if (cur_layer >= 0) flush();
+}
+
+// One block per layer: fixed-order sum of the layer's partial rows, c = a S + b sum(g), update.
+__global__ void layered_combine_kernel(const float* __restrict__ partials, const int* __restrict__ cta_first,
+                                       const int* __restrict__ cta_base, int ctas, int n,
+                                       const float* __restrict__ a, const float* __restrict__ b,
+                                       float* c_out, float* beta, float lr, float lambda, int* status) {
+  const int l = blockIdx.x, i = threadIdx.x;
+  double S = 0.0, Sg = 0.0;
+  for (int cta = 0; cta < ctas; ++cta) {
+    const int f = cta_first[cta], cnt = cta_base[cta + 1] - cta_base[cta];
+    if (l < f || l >= f + cnt) continue;
+    const float* rows = partials + static_cast<size_t>(cta_base[cta] + l - f) * MMA_WARPS * ROW_FLOATS;
+    for (int w = 0; w < MMA_WARPS; ++w) {
+      if (i < n) S += static_cast<double>(__ldcg(rows + w * ROW_FLOATS + i));
+      Sg += static_cast<double>(__ldcg(rows + w * ROW_FLOATS + 128));
+    }
+  }
+  if (i >= n) return;
+  const double c = static_cast<double>(a[l]) * S + static_cast<double>(b[l]) * Sg;
+  if (!isfinite(c)) twa_set_status(status, TWA_ERR_NONFINITE, l);
+  if (c_out) c_out[static_cast<size_t>(l) * n + i] = static_cast<float>(c);
+  if (beta) {
+    const double decay = 1.0 - static_cast<double>(lr) * static_cast<double>(lambda);
+    beta[static_cast<size_t>(l) * n + i] =
+        static_cast<float>(decay * static_cast<double>(beta[static_cast<size_t>(l) * n + i]) - static_cast<double>(lr) * c);
+  }
+}
+
+// One block (128 threads) per layer: digits of a^l * beta^l_i on the layer's common scale, and
+// the constant b^l * sum_i beta^l_i.
+__global__ void layered_coef_kernel(const float* __restrict__ beta, int n, const float* __restrict__ a,
+                                    const float* __restrict__ b, float mult, unsigned char* __restrict__ dig,
+                                    int* __restrict__ ebits_out, float* __restrict__ konst, int* status) {
+  __shared__ unsigned amax;
+  const int l = blockIdx.x, i = threadIdx.x;
+  if (i == 0) amax = 0u;
+  __syncthreads();
+  float coef = 0.0f;
+  if (i < n) coef = beta[static_cast<size_t>(l) * n + i] * mult * a[l];
+  atomicMax(&amax, __float_as_uint(coef) & 0x7FFFFFFFu);
+  __syncthreads();
+  const unsigned ebits = amax >> 23;
+  const bool bad = ebits >= 255u, live = ebits >= 5u && !bad;
+  uint32_t d = 0;
+  if (live) d = cut_digits(coef * __uint_as_float((259u - ebits) << 23));
+#pragma unroll
+  for (int k = 0; k < 4; ++k) dig[static_cast<size_t>(l) * 512 + k * 128 + i] = static_cast<unsigned char>(d >> (8 * k));
+  if (i == 0) {
+    double sb = 0.0;
+    for (int q = 0; q < n; ++q) sb += static_cast<double>(beta[static_cast<size_t>(l) * n + q]);
+    const double kk = static_cast<double>(b[l]) * static_cast<double>(mult) * sb;
+    if (bad || !isfinite(kk)) twa_set_status(status, TWA_ERR_NONFINITE, l);
+    konst[l] = static_cast<float>(kk);
+    ebits_out[l] = bad ? -1 : (live ? static_cast<int>(ebits) : 0);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+template <int BITS, int KS, int KT>
+__global__ void __launch_bounds__(MMA_THREADS, 1)
+layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
+  constexpr int LROWS = BITS == 8 ? 2 : 4;
+  constexpr int RB = 32 * 8 / BITS;
+  constexpr int GPT = 8 * KT;
+  twa_smem_header* hdr = reinterpret_cast<twa_smem_header*>(smem);
+  unsigned char* ring = smem + TWA_SMEM_HEADER;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gid = lane >> 2, tig = lane & 3;
+  init_barriers(hdr, a.stages);
+  __syncthreads();
+  const int t_first = blockIdx.x * a.tpc;
+  const int t_count = (a.tiles - t_first) < a.tpc ? (a.tiles - t_first) : a.tpc;
+  if (warp == MMA_WARPS) {
+    if (lane == 0)
+      producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, KT, 0, 0,
+                        0, 0, a.tx_bytes, true, a.status, a.wait_limit_ns);
+    return;
+  }
+  const int lm = lane >> 3, lr = lane & 7;
+  const int jmax = a.n - 1;
+  constexpr int col_bytes = TWA_TILE_COL_BYTES * KT;
+  uint32_t loff[KT][2][KS];
+#pragma unroll
+  for (int u = 0; u < KT; ++u)
+#pragma unroll
+    for (int ch = 0; ch < 2; ++ch)
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        int j = ks * 32 + lm * 8 + lr;
+        j = j < jmax ? j : jmax;
+        const int chunk = (warp * KT + u) * 2 + ch;
+        loff[u][ch][ks] = static_cast<uint32_t>(j * col_bytes + ((chunk >> 5) << 9) + (twa_chunk_slot(chunk & 31, j) << 4));
+      }
+  const int wb = warp * 32 * KT;
+  const int gran_in_tile = wb >> 6;
+  const int rig0 = (wb & 63) * 8 / BITS;
+  // rows (inside the granule) this lane finishes for block u: chunk tig, LROWS rows from LROWS * gid
+  int rrow[KT];
+#pragma unroll
+  for (int u = 0; u < KT; ++u) rrow[u] = rig0 + u * RB + 16 * tig * (8 / BITS) + LROWS * gid;
+
+  int4 e_next;
+  float bn[KT][LROWS];
+  auto fetch = [&](int tile) {
+    const int gi = tile * GPT + gran_in_tile;
+    e_next = gi < a.n_gran ? __ldg(a.gran + gi) : make_int4(-1, 0, 0, 0);
+#pragma unroll
+    for (int u = 0; u < KT; ++u)
+#pragma unroll
+      for (int i = 0; i < LROWS; ++i) {
+        bn[u][i] = 0.0f;
+        if (a.base && tig < 2 && e_next.x >= 0 && rrow[u] + i < e_next.y)
+          bn[u][i] = a.base[static_cast<long long>(e_next.z) + rrow[u] + i];
+      }
+  };
+
+  uint32_t bfrag[KS][2];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) bfrag[ks][0] = bfrag[ks][1] = 0u;
+  float wa = 0.0f, wbw = 0.0f, kon = 0.0f;
+  int cur_layer = -1;
+  volatile int* abort_flag = &hdr->abort_flag;
+  int s = 0;
+  unsigned phase = 0;
+  fetch(t_first + t_count - 1);
+  for (int k = 0; k < t_count; ++k) {                   // backwards, like the producer
+    const int4 e = e_next;
+    float bv[KT][LROWS];
+#pragma unroll
+    for (int u = 0; u < KT; ++u)
+#pragma unroll
+      for (int i = 0; i < LROWS; ++i) bv[u][i] = bn[u][i];
+    if (k + 1 < t_count) fetch(t_first + t_count - 2 - k);
+    if (e.x != cur_layer && e.x >= 0) {                  // new layer: its digit fragments and factors
+      cur_layer = e.x;
+      const int eb = a.ebits[cur_layer];
+      const float w0 = eb <= 0 ? 0.0f : (eb >= 6 ? __uint_as_float(static_cast<uint32_t>(eb - 5) << 23) : 5.877471754e-39f);
+      const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
+      wa = tig == 0 ? w0 : (tig == 1 ? w2 : 0.0f);
+      wbw = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);
+      if (BITS == 4) { wa *= 0.0625f; wbw *= 0.0625f; }
+      kon = eb < 0 ? __int_as_float(0x7FC00000) : a.konst[cur_layer];
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        bfrag[ks][0] = bfrag[ks][1] = 0u;
+        if (gid < 4) {
+          const unsigned char* tk = a.dig + static_cast<size_t>(cur_layer) * 512 + gid * 128 + ks * 32 + 2 * tig;
+          bfrag[ks][0] = static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(tk)) |
+                         (static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(tk + 8)) << 16);
+          bfrag[ks][1] = static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(tk + 16)) |
+                         (static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(tk + 24)) << 16);
+        }
+      }
+    }
+    if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
+      twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+      break;
+    }
+    const uint32_t tile_base = twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes);
+    float keep[KT][LROWS];
+#pragma unroll
+    for (int u = 0; u < KT; ++u) {
+#pragma unroll
+      for (int i = 0; i < LROWS; ++i) keep[u][i] = 0.0f;
+      if (e.x >= 0) {
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch) {
+          int acc0[4] = {0, 0, 0, 0};
+          int acc1[4] = {0, 0, 0, 0};
+#pragma unroll
+          for (int ks = 0; ks < KS; ++ks) {
+            uint32_t r[4];
+            ldmatrix_x4_trans(tile_base + loff[u][ch][ks], r);
+            if (BITS == 8) {
+              const uint32_t af[4] = {__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[0], r[1], 0x7531),
+                                      __byte_perm(r[2], r[3], 0x6420), __byte_perm(r[2], r[3], 0x7531)};
+              mma_u8s8(acc0, af, bfrag[ks][0], bfrag[ks][1]);
+            } else {
+              uint32_t ev[4], od[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                ev[i] = (r[i] << 4) & 0xF0F0F0F0u;
+                od[i] = r[i] & 0xF0F0F0F0u;
+              }
+              const uint32_t ae[4] = {__byte_perm(ev[0], ev[1], 0x6420), __byte_perm(ev[0], ev[1], 0x7531),
+                                      __byte_perm(ev[2], ev[3], 0x6420), __byte_perm(ev[2], ev[3], 0x7531)};
+              const uint32_t ao[4] = {__byte_perm(od[0], od[1], 0x6420), __byte_perm(od[0], od[1], 0x7531),
+                                      __byte_perm(od[2], od[3], 0x6420), __byte_perm(od[2], od[3], 0x7531)};
+              mma_u8s8(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
+              mma_u8s8(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
+            }
+          }
+          float v[LROWS];
+          if (BITS == 8) {
+            v[0] = fmaf(small_int_to_float(acc0[1]), wbw, small_int_to_float(acc0[0]) * wa);
+            v[1] = fmaf(small_int_to_float(acc0[3]), wbw, small_int_to_float(acc0[2]) * wa);
+          } else {
+            v[0] = fmaf(small_int_to_float(acc0[1]), wbw, small_int_to_float(acc0[0]) * wa);
+            v[2] = fmaf(small_int_to_float(acc0[3]), wbw, small_int_to_float(acc0[2]) * wa);
+            v[1] = fmaf(small_int_to_float(acc1[1]), wbw, small_int_to_float(acc1[0]) * wa);
+            v[3] = fmaf(small_int_to_float(acc1[3]), wbw, small_int_to_float(acc1[2]) * wa);
+          }
+#pragma unroll
+          for (int i = 0; i < LROWS; ++i) {
+            v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 1);
+            if (tig == ch) keep[u][i] = v[i];
+          }
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
+    if (e.x >= 0 && tig < 2) {
+#pragma unroll
+      for (int u = 0; u < KT; ++u)
+#pragma unroll
+        for (int i = 0; i < LROWS; ++i)
+          if (rrow[u] + i < e.y) a.out[static_cast<long long>(e.z) + rrow[u] + i] = bv[u][i] + keep[u][i] + kon;
+    }
+    if (++s == a.stages) {
+      s = 0;
+      phase ^= 1u;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+int encode_codes_map(twa_ctx* ctx, const twa_basis* P, int kt, CUtensorMap* map) {
+  long long row_bytes = (P->D * P->bits + 7) / 8;
+  row_bytes = (row_bytes + 511) / 512 * 512;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(row_bytes / 4), static_cast<cuuint64_t>(P->n)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(P->col_stride)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(TWA_TILE_COL_WORDS * kt), static_cast<cuuint32_t>(P->n)};
+  cuuint32_t es[2] = {1, 1};
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, P->data, dims, strides, box, es,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(ctx->last_error, sizeof(ctx->last_error), "cuTensorMapEncodeTiled(layered codes) failed: %d",
+             static_cast<int>(r));
+    return TWA_ERR_CUDA;
+  }
+  return TWA_OK;
+}
+
+struct StepLayout { size_t partials, dig, ebits, konst, total; };
+StepLayout step_layout(const twa_layered_basis* lb) {
+  StepLayout w;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = (o + bytes + 255) / 256 * 256; return at; };
+  w.partials = take(sizeof(float) * static_cast<size_t>(lb->total_runs) * MMA_WARPS * ROW_FLOATS);
+  w.dig = take(static_cast<size_t>(lb->L) * 512);
+  w.ebits = take(sizeof(int) * lb->L);
+  w.konst = take(sizeof(float) * lb->L);
+  w.total = o;
+  return w;
+}
+
+template <int BITS, bool GBF16, int MT>
+int launch_lproject_t(twa_ctx* ctx, const CUtensorMap& mp, const LProjectArgs& a, int kt, int grid, int smem) {
+  auto kern = kt == 2 ? layered_project_kernel<BITS, GBF16, MT, 2> : layered_project_kernel<BITS, GBF16, MT, 1>;
+  static int smem_limit[2][64] = {{0}};
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[kt - 1][ctx->device & 63], smem);
+  if (rc) return rc;
+  kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, a);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+template <int BITS, bool GBF16>
+int launch_lproject(twa_ctx* ctx, const CUtensorMap& mp, const LProjectArgs& a, int kt, int grid, int smem) {
+  switch ((a.n + 15) >> 4) {
+    case 1: return launch_lproject_t<BITS, GBF16, 1>(ctx, mp, a, kt, grid, smem);
+    case 2: return launch_lproject_t<BITS, GBF16, 2>(ctx, mp, a, kt, grid, smem);
+    case 3: return launch_lproject_t<BITS, GBF16, 3>(ctx, mp, a, kt, grid, smem);
+    case 4: return launch_lproject_t<BITS, GBF16, 4>(ctx, mp, a, kt, grid, smem);
+    case 5: return launch_lproject_t<BITS, GBF16, 5>(ctx, mp, a, kt, grid, smem);
+    case 6: return launch_lproject_t<BITS, GBF16, 6>(ctx, mp, a, kt, grid, smem);
+    case 7: return launch_lproject_t<BITS, GBF16, 7>(ctx, mp, a, kt, grid, smem);
+    default: return launch_lproject_t<BITS, GBF16, 8>(ctx, mp, a, kt, grid, smem);
+  }
+}
+
+template <int BITS, int KS>
+int launch_llift_t(twa_ctx* ctx, const CUtensorMap& mp, const LLiftArgs& a, int kt, int grid, int smem) {
+  auto kern = kt == 2 ? layered_lift_kernel<BITS, KS, 2> : layered_lift_kernel<BITS, KS, 1>;
+  static int smem_limit[2][64] = {{0}};
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[kt - 1][ctx->device & 63], smem);
+  if (rc) return rc;
+  kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, a);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+template <int BITS>
+int launch_llift(twa_ctx* ctx, const CUtensorMap& mp, const LLiftArgs& a, int kt, int grid, int smem) {
+  switch ((a.n + 31) >> 5) {
+    case 1: return launch_llift_t<BITS, 1>(ctx, mp, a, kt, grid, smem);
+    case 2: return launch_llift_t<BITS, 2>(ctx, mp, a, kt, grid, smem);
+    case 3: return launch_llift_t<BITS, 3>(ctx, mp, a, kt, grid, smem);
+    default: return launch_llift_t<BITS, 4>(ctx, mp, a, kt, grid, smem);
+  }
+}
+
+int stage_count(const twa_ctx* ctx, int fixed, int stage_bytes) {
+  int s = (ctx->smem_optin - fixed) / stage_bytes;
+  if (s > TWA_MAX_STAGES) s = TWA_MAX_STAGES;
+  return s;
+}
+
+int do_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype, float* c_out,
+               float* beta, float lr, float lambda, char* sws) {
+  const StepLayout w = step_layout(lb);
+  const int n = lb->codes.n, kt = lb->kt;
+  CUtensorMap mp;
+  int rc = encode_codes_map(ctx, &lb->codes, kt, &mp);
+  if (rc) return rc;
+  LProjectArgs a;
+  a.n = n;
+  a.tiles = lb->tiles;
+  a.tpc = lb->tiles_per_cta;
+  a.n_gran = static_cast<int>(lb->codes.col_stride / 64);
+  a.tx_bytes = static_cast<unsigned>(n) * TWA_TILE_COL_BYTES * kt;
+  a.stage_bytes = (a.tx_bytes + 1023) / 1024 * 1024;
+  a.stages = stage_count(ctx, TWA_SMEM_HEADER + MMA_WARPS * DIGIT_SCRATCH + 1024, static_cast<int>(a.stage_bytes));
+  if (a.stages < 2) return TWA_ERR_UNSUPPORTED;
+  a.scratch_off = TWA_SMEM_HEADER + static_cast<unsigned>(a.stages) * a.stage_bytes;
+  a.gran = reinterpret_cast<const int4*>(lb->granules);
+  a.g = g;
+  a.cta_first = lb->cta_first_layer;
+  a.cta_base = lb->cta_run_base;
+  a.partials = reinterpret_cast<float*>(sws + w.partials);
+  a.status = ctx->d_status;
+  a.wait_limit_ns = ctx->wait_limit_ns;
+  TWA_CUDA_OK(ctx, cudaMemsetAsync(a.partials, 0, w.dig - w.partials, ctx->stream));
+  const int smem = static_cast<int>(a.scratch_off) + MMA_WARPS * DIGIT_SCRATCH + 1024;
+  const bool bf16 = g_dtype == TWA_BF16;
+  if (lb->codes.bits == 8)
+    rc = bf16 ? launch_lproject<8, true>(ctx, mp, a, kt, lb->cta_count, smem)
+              : launch_lproject<8, false>(ctx, mp, a, kt, lb->cta_count, smem);
+  else
+    rc = bf16 ? launch_lproject<4, true>(ctx, mp, a, kt, lb->cta_count, smem)
+              : launch_lproject<4, false>(ctx, mp, a, kt, lb->cta_count, smem);
+  if (rc) return rc;
+  layered_combine_kernel<<<lb->L, 128, 0, ctx->stream>>>(a.partials, lb->cta_first_layer, lb->cta_run_base,
+                                                       lb->cta_count, n, lb->a, lb->b, c_out, beta, lr, lambda,
+                                                       ctx->d_status);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+int do_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* beta, const float* base, float* out,
+            char* sws) {
+  const StepLayout w = step_layout(lb);
+  const int n = lb->codes.n, kt = lb->kt;
+  unsigned char* dig = reinterpret_cast<unsigned char*>(sws + w.dig);
+  int* ebits = reinterpret_cast<int*>(sws + w.ebits);
+  float* konst = reinterpret_cast<float*>(sws + w.konst);
+  layered_coef_kernel<<<lb->L, 128, 0, ctx->stream>>>(beta, n, lb->a, lb->b, 1.0f, dig, ebits, konst, ctx->d_status);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  CUtensorMap mp;
+  int rc = encode_codes_map(ctx, &lb->codes, kt, &mp);
+  if (rc) return rc;
+  LLiftArgs a;
+  a.n = n;
+  a.tiles = lb->tiles;
+  a.tpc = lb->tiles_per_cta;
+  a.n_gran = static_cast<int>(lb->codes.col_stride / 64);
+  a.tx_bytes = static_cast<unsigned>(n) * TWA_TILE_COL_BYTES * kt;
+  a.stage_bytes = (a.tx_bytes + 1023) / 1024 * 1024;
+  a.stages = stage_count(ctx, TWA_SMEM_HEADER + 1024, static_cast<int>(a.stage_bytes));
+  if (a.stages < 2) return TWA_ERR_UNSUPPORTED;
+  a.gran = reinterpret_cast<const int4*>(lb->granules);
+  a.dig = dig;
+  a.ebits = ebits;
+  a.konst = konst;
+  a.base = base;
+  a.out = out;
+  a.status = ctx->d_status;
+  a.wait_limit_ns = ctx->wait_limit_ns;
+  const int smem = TWA_SMEM_HEADER + a.stages * static_cast<int>(a.stage_bytes) + 1024;
+  return lb->codes.bits == 8 ? launch_llift<8>(ctx, mp, a, kt, lb->cta_count, smem)
+                             : launch_llift<4>(ctx, mp, a, kt, lb->cta_count, smem);
+}
+
+int check_step_args(twa_ctx* ctx, const twa_layered_basis* lb, const void* sws, size_t sws_bytes) {
+  if (!ctx || !lb || !lb->codes.data || !lb->a || !lb->b || !lb->granules || !lb->cta_first_layer ||
+      !lb->cta_run_base)
+    return TWA_ERR_INVALID_ARG;
+  if (lb->codes.bits != 8 && lb->codes.bits != 4) return TWA_ERR_UNSUPPORTED;
+  if (lb->codes.n < 1 || lb->codes.n > TWA_MAX_N || lb->L < 1 || lb->cta_count < 1 || (lb->kt != 1 && lb->kt != 2))
+    return TWA_ERR_INVALID_ARG;
+  if (!sws || sws_bytes < step_layout(lb).total) return TWA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(sws) & 255) return TWA_ERR_MISALIGNED;
+  return TWA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t twa_layered_step_workspace_bytes(const twa_layered_basis* lb) {
+  if (!lb || lb->L < 1 || lb->total_runs < 1) return 0;
+  return step_layout(lb).total;
+}
+
+int twa_layered_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype,
+                        float* c_out, void* sws, size_t sws_bytes) {
+  int rc = check_step_args(ctx, lb, sws, sws_bytes);
+  if (rc) return rc;
+  if (!g || !c_out || (g_dtype != TWA_F32 && g_dtype != TWA_BF16)) return TWA_ERR_INVALID_ARG;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  return do_project(ctx, lb, g, g_dtype, c_out, nullptr, 0.0f, 0.0f, static_cast<char*>(sws));
+}
+
+int twa_layered_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* beta, const float* base,
+                     float* w_out, void* sws, size_t sws_bytes) {
+  int rc = check_step_args(ctx, lb, sws, sws_bytes);
+  if (rc) return rc;
+  if (!beta || !w_out) return TWA_ERR_INVALID_ARG;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  return do_lift(ctx, lb, beta, base, w_out, static_cast<char*>(sws));
+}
+
+int twa_layered_step(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype, float lr,
+                     float lambda, float* beta, const float* wbar, float* w, float* c_out, void* sws,
+                     size_t sws_bytes) {
+  int rc = check_step_args(ctx, lb, sws, sws_bytes);
+  if (rc) return rc;
+  if (!g || !beta || !wbar || !w || (g_dtype != TWA_F32 && g_dtype != TWA_BF16)) return TWA_ERR_INVALID_ARG;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  rc = do_project(ctx, lb, g, g_dtype, c_out, beta, lr, lambda, static_cast<char*>(sws));
+  if (rc) return rc;
+  return do_lift(ctx, lb, beta, wbar, w, static_cast<char*>(sws));
+}
+
+}  // extern "C"

@@ -27,14 +27,9 @@
 // never wait for one another inside the tile loop.
 #include <stdio.h>
 
-#include "twa_common.cuh"
+#include "twa_mma.cuh"
 
 namespace {
-
-constexpr int MMA_WARPS = 16;
-constexpr int MMA_THREADS = (MMA_WARPS + 1) * 32;
-constexpr int DIGIT_SCRATCH = 256;             // bytes of digit scratch per warp
-constexpr float RND = 12582912.0f;             // 2^23 + 2^22: x + RND rounds x to an integer (ties to even)
 
 struct ProjectMmaArgs {
   long long D;
@@ -67,107 +62,6 @@ struct LiftMmaArgs {
   unsigned long long wait_limit_ns;
 };
 
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"(addr));
-}
-
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"(addr));
-}
-
-// d += a (16 x 32, s8) * b (32 x 8, s8), int32 accumulation
-__device__ __forceinline__ void mma_s8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// |v| < 2^22 -> float, exactly, without the conversion unit
-__device__ __forceinline__ float small_int_to_float(int v) {
-  return __int_as_float(0x4B400000 + v) - RND;
-}
-
-// Four signed base-128 digits of t (|t| <= 64): t = d0 + d1/128 + d2/128^2 + d3/128^3 + eps,
-// |eps| <= 2^-22, every digit in [-64, 64].  Returned packed, digit k in byte k.
-__device__ __forceinline__ uint32_t cut_digits(float t) {
-  const float m0 = t + RND;
-  t = (t - (m0 - RND)) * 128.0f;
-  const float m1 = t + RND;
-  t = (t - (m1 - RND)) * 128.0f;
-  const float m2 = t + RND;
-  t = (t - (m2 - RND)) * 128.0f;
-  const float m3 = t + RND;
-  const uint32_t lo = __byte_perm(__float_as_uint(m0), __float_as_uint(m1), 0x0040);  // bytes m0.b0, m1.b0
-  const uint32_t hi = __byte_perm(__float_as_uint(m2), __float_as_uint(m3), 0x0040);
-  return __byte_perm(lo, hi, 0x5410);
-}
-
-// g_boxes 1-D boxes of 256 gradient elements follow the tile of P~ in a stage (project only).
-__device__ __forceinline__ void producer_loop_mma(twa_smem_header* hdr, unsigned char* ring,
-                                                  const CUtensorMap* map_p, const CUtensorMap* map_g,
-                                                  int tiles, int stages, unsigned stage_bytes, int kt,
-                                                  int g_boxes, int g_elem_bytes, int tile_rows,
-                                                  unsigned g_off, unsigned tx_bytes,
-                                                  bool reverse, int* status, unsigned long long limit) {
-  twa_prefetch_tensormap(map_p);
-  if (g_boxes > 0) twa_prefetch_tensormap(map_g);
-  volatile int* abort_flag = &hdr->abort_flag;
-  int s = 0, issued = 0;
-  unsigned phase = 0;
-  bool ok = true;
-  for (int t = blockIdx.x; t < tiles; t += gridDim.x) {
-    if (issued >= stages) {
-      if (!twa_mbar_wait(twa_smem_u32(&hdr->empty[s]), phase, abort_flag, limit)) {
-        ok = false;
-        break;
-      }
-    }
-    const int tile = reverse ? (tiles - 1 - t) : t;
-    const uint32_t fb = twa_smem_u32(&hdr->full[s]);
-    const uint32_t dst = twa_smem_u32(ring + static_cast<size_t>(s) * stage_bytes);
-    twa_mbar_expect_tx(fb, tx_bytes);
-    twa_tma_load_2d(dst, map_p, tile * TWA_TILE_COL_WORDS * kt, 0, fb);
-    for (int b = 0; b < g_boxes; ++b)
-      twa_tma_load_1d(dst + g_off + b * 256 * g_elem_bytes, map_g, tile * tile_rows + b * 256, fb);
-    ++issued;
-    if (++s == stages) {
-      s = 0;
-      if (issued > stages) phase ^= 1u;
-    }
-  }
-  if (!ok) {
-    twa_set_status(status, TWA_ERR_TIMEOUT, -1);
-    const int live = issued < stages ? issued : stages;
-    for (int q = 0; q < live; ++q) {      // let the copies already issued land
-      const int last = ((issued - 1 - q) / stages) * stages + q;
-      const unsigned par = static_cast<unsigned>(last / stages) & 1u;
-      const unsigned long long t0 = twa_globaltimer();
-      while (!twa_mbar_try_wait(twa_smem_u32(&hdr->full[q]), par)) {
-        if (twa_globaltimer() - t0 > limit) break;
-      }
-    }
-  }
-}
-
-__device__ __forceinline__ void init_barriers(twa_smem_header* hdr, int stages) {
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < stages; ++s) {
-      twa_mbar_init(twa_smem_u32(&hdr->full[s]), 1);
-      twa_mbar_init(twa_smem_u32(&hdr->empty[s]), MMA_WARPS);
-    }
-    hdr->abort_flag = 0;
-    hdr->last_flag = 0;
-    hdr->bad_flag = 0;
-    hdr->amax_bits = 0;
-    twa_fence_barrier_init();
-  }
-}
-
 // =================================================================================================
 // project
 // =================================================================================================
@@ -198,9 +92,11 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
 
   if (warp == MMA_WARPS) {
     if (lane == 0)
-      producer_loop_mma(hdr, ring, &map_p, &map_g, a.tiles, a.stages, a.stage_bytes, KT,
-                        SROWS * KT / 256, GSZ, SROWS * KT, a.g_off, a.tx_bytes, false, a.status,
-                        a.wait_limit_ns);
+      producer_loop_mma(hdr, ring, &map_p, &map_g, blockIdx.x, gridDim.x,
+                        (a.tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
+                            static_cast<int>(gridDim.x),
+                        a.stages, a.stage_bytes, KT, SROWS * KT / 256, GSZ, SROWS * KT, a.g_off,
+                        a.tx_bytes, false, a.status, a.wait_limit_ns);
   } else {
     unsigned char* digw = smem + a.scratch_off + warp * DIGIT_SCRATCH;   // this warp's digit bytes
     const int lm = lane >> 3, lr = lane & 7;            // ldmatrix: matrix and row this lane addresses
@@ -425,8 +321,11 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
 
   if (warp == MMA_WARPS) {
     if (lane == 0)
-      producer_loop_mma(hdr, ring, &map_p, nullptr, a.tiles, a.stages, a.stage_bytes, KT, 0, 0, 0, 0,
-                        a.tx_bytes, a.reverse != 0, a.status, a.wait_limit_ns);
+      producer_loop_mma(hdr, ring, &map_p, nullptr, blockIdx.x, gridDim.x,
+                        (a.tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
+                            static_cast<int>(gridDim.x),
+                        a.stages, a.stage_bytes, KT, 0, 0, 0, 0, a.tx_bytes, a.reverse != 0, a.status,
+                        a.wait_limit_ns);
     return;
   }
   if (bad && tid == 0) twa_set_status(a.status, TWA_ERR_NONFINITE, -1);
@@ -482,8 +381,11 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
   volatile int* abort_flag = &hdr->abort_flag;
   int s = 0;
   unsigned phase = 0;
-  for (int t = blockIdx.x; t < a.tiles; t += gridDim.x) {
-    const int tile = a.reverse ? (a.tiles - 1 - t) : t;
+  // the same tile sequence as the producer: this block's tiles, backwards when `reverse`
+  const int t_count = (a.tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
+                      static_cast<int>(gridDim.x);
+  for (int k = 0; k < t_count; ++k) {
+    const int tile = static_cast<int>(blockIdx.x) + (a.reverse ? (t_count - 1 - k) : k) * static_cast<int>(gridDim.x);
     const int tile_row0 = tile * tile_rows;               // < D < 2^31
     const bool whole = tile_row0 <= D - tile_rows;        // no row of the tile lies past D
     float bv[KT][LROWS];

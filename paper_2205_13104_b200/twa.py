@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libtwa.so")
 CSRC = os.path.join(_HERE, "csrc")
-SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_chunked.cu", "twa_layered_build.cu", "twa_stream.cu",
+SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_chunked.cu", "twa_layered_build.cu", "twa_layered_step.cu", "twa_stream.cu",
            "twa_stream_mma.cu", "twa_noalloc.cu"]
 
 TWA_MAX_N = 128
@@ -46,7 +46,9 @@ EXPORTS = [
     "twa_build_feed", "twa_build_end_pass", "twa_mean", "twa_quantize_basis",
     "twa_basis_export", "twa_basis_import", "twa_project", "twa_lift", "twa_step",
     "twa_step_host", "twa_layered_workspace_bytes", "twa_layered_rows", "twa_layered_basis_bytes",
-    "twa_build_centered", "twa_quantize_affine", "twa_layered_export", "twa_project_noalloc", "twa_noalloc_last_error", "twa_noalloc_scratch_bytes",
+    "twa_build_centered", "twa_quantize_affine", "twa_layered_export",
+    "twa_layered_step_workspace_bytes", "twa_layered_project", "twa_layered_lift", "twa_layered_step",
+    "twa_project_noalloc", "twa_noalloc_last_error", "twa_noalloc_scratch_bytes",
 ]
 
 
@@ -61,7 +63,10 @@ class twa_layered_basis(ctypes.Structure):
     """Mirror of the C struct twa_layered_basis."""
     _fields_ = [("codes", twa_basis), ("a", ctypes.c_void_p), ("b", ctypes.c_void_p),
                 ("granules", ctypes.c_void_p), ("flat_offsets", ctypes.c_void_p),
-                ("internal_offsets", ctypes.c_void_p), ("D", ctypes.c_int64), ("L", ctypes.c_int32)]
+                ("internal_offsets", ctypes.c_void_p), ("D", ctypes.c_int64), ("L", ctypes.c_int32),
+                ("cta_count", ctypes.c_int32), ("kt", ctypes.c_int32), ("tiles", ctypes.c_int32),
+                ("tiles_per_cta", ctypes.c_int32), ("total_runs", ctypes.c_int32),
+                ("cta_first_layer", ctypes.c_void_p), ("cta_run_base", ctypes.c_void_p)]
 
 
 class TwaError(RuntimeError):
@@ -144,6 +149,11 @@ def load():
         "twa_quantize_affine": (i32, [vp, bp, ctypes.POINTER(ctypes.c_int64), i32, i32, vp, szt,
                                       ctypes.POINTER(twa_layered_basis), vp, szt]),
         "twa_layered_export": (i32, [vp, ctypes.POINTER(twa_layered_basis), vp, vp, vp]),
+        "twa_layered_step_workspace_bytes": (szt, [ctypes.POINTER(twa_layered_basis)]),
+        "twa_layered_project": (i32, [vp, ctypes.POINTER(twa_layered_basis), vp, i32, vp, vp, szt]),
+        "twa_layered_lift": (i32, [vp, ctypes.POINTER(twa_layered_basis), vp, vp, vp, vp, szt]),
+        "twa_layered_step": (i32, [vp, ctypes.POINTER(twa_layered_basis), vp, i32, f32, f32, vp, vp, vp, vp,
+                                   vp, szt]),
         "twa_project_noalloc": (i32, [i32, vp, bp, vp, i32, vp, vp]),
         "twa_noalloc_last_error": (ctypes.c_char_p, []),
         "twa_noalloc_scratch_bytes": (szt, []),
@@ -505,3 +515,33 @@ def twa_layered_export(ctx, lb):
     _check(load().twa_layered_export(ctx, ctypes.byref(lb.desc), _ptr(codes), _ptr(a), _ptr(b)),
            "twa_layered_export", ctx)
     return codes, a, b
+
+
+def twa_layered_step_workspace_bytes(lb):
+    return int(load().twa_layered_step_workspace_bytes(ctypes.byref(lb.desc)))
+
+
+def new_layered_step_workspace(lb):
+    return torch.empty(twa_layered_step_workspace_bytes(lb), dtype=torch.uint8, device=lb.mem.device)
+
+
+def twa_layered_project(ctx, lb, g, c_out, sws):
+    """c_out: (L, n) float32, layer-major."""
+    rc = load().twa_layered_project(ctx, ctypes.byref(lb.desc), _ptr(g), _dtype_code(g), _ptr(c_out),
+                                    _ptr(sws), sws.numel())
+    _check(rc, "twa_layered_project", ctx)
+    return c_out
+
+
+def twa_layered_lift(ctx, lb, beta, base, w_out, sws):
+    rc = load().twa_layered_lift(ctx, ctypes.byref(lb.desc), _ptr(beta), _ptr(base), _ptr(w_out),
+                                 _ptr(sws), sws.numel())
+    _check(rc, "twa_layered_lift", ctx)
+    return w_out
+
+
+def twa_layered_step(ctx, lb, g, lr, lam, beta, wbar, w, sws, c_out=None):
+    rc = load().twa_layered_step(ctx, ctypes.byref(lb.desc), _ptr(g), _dtype_code(g), float(lr), float(lam),
+                                 _ptr(beta), _ptr(wbar), _ptr(w), _ptr(c_out), _ptr(sws), sws.numel())
+    _check(rc, "twa_layered_step", ctx)
+    return w

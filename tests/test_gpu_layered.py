@@ -108,3 +108,144 @@ def test_affine_nonfinite_is_reported(env):
     code, detail = twa.twa_get_status(ctx)
     assert (code, detail) == (twa.TWA_ERR_NONFINITE, 1)
     twa.twa_clear_status(ctx)
+
+
+# ------------------------------------------------------------------ layer-wise step
+def _random_layers(D, count, seed):
+    rng = np.random.default_rng(seed)
+    cuts = np.unique(rng.integers(1, D, size=count - 1))
+    return [0] + [int(x) for x in cuts] + [D]
+
+
+STEP_CASES = CASES + [
+    (3_000_017, 33, _random_layers(3_000_017, 60, 1)),        # two 512-byte segments per tile column
+    (2_500_003, 100, _random_layers(2_500_003, 40, 2)),       # one segment per tile column
+    (1_200_000, 128, [0, 5, 6, 70, 1_200_000]),
+]
+
+
+def _layered_basis(ctx, D, n, layers, bits, seed):
+    W = inputs.trajectory_candidates(D, n, 0.005, 0.001, seed, DEV, ld=inputs.padded_ld(D, 4))
+    wbar = torch.empty(D, device=DEV)
+    lws = twa.new_layered_workspace(layers, n, DEV)
+    P32 = twa.twa_build_centered(ctx, W, D, layers, wbar, lws)
+    lb = twa.twa_quantize_affine(ctx, P32, layers, bits, lws)
+    codes_g, a_g, b_g = twa.twa_layered_export(ctx, lb)
+    status_ok(ctx)
+    codes = unpack_unsigned(codes_g.cpu().numpy(), D, bits)
+    return lb, wbar, codes, a_g.cpu().numpy(), b_g.cpu().numpy()
+
+
+def _term_scale(codes, layers, a, b, g64):
+    """Per (layer, column) sum of the magnitudes of the terms of c: the size rounding errors scale with."""
+    L, n = len(layers) - 1, codes.shape[1]
+    s = np.zeros((L, n))
+    ag = np.abs(g64)
+    for l in range(L):
+        r0, r1 = layers[l], layers[l + 1]
+        s[l] = abs(float(a[l])) * (codes[r0:r1].astype(np.float64).T @ ag[r0:r1]) + abs(float(b[l])) * ag[r0:r1].sum()
+    return s
+
+
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("D,n,layers", STEP_CASES)
+def test_layered_project(env, D, n, layers, bits, g_dtype):
+    ctx, _ = env
+    lb, _, codes, a, b = _layered_basis(ctx, D, n, layers, bits, 51)
+    L = len(layers) - 1
+    g = inputs.gradient(D, 1e-3, 7, 0, g_dtype, DEV)
+    sws = twa.new_layered_step_workspace(lb)
+    c = torch.full((L, n), float("nan"), device=DEV)
+    twa.twa_layered_project(ctx, lb, g, c, sws)
+    status_ok(ctx)
+    g64 = g.float().cpu().numpy().astype(np.float64)
+    c_o = orc.project_layerwise(codes, layers, a, b, g64)
+    c_g = c.cpu().numpy()
+    assert rel(c_g, c_o) <= TOL
+    assert np.all(np.abs(c_g - c_o) <= 2e-6 * _term_scale(codes, layers, a, b, g64) + 1e-30)
+    # same call again: bitwise the same result (fixed summation order)
+    c2 = torch.empty_like(c)
+    twa.twa_layered_project(ctx, lb, g, c2, sws)
+    assert torch.equal(c, c2)
+
+
+@pytest.mark.parametrize("with_base", [True, False])
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("D,n,layers", STEP_CASES)
+def test_layered_lift(env, D, n, layers, bits, with_base):
+    ctx, _ = env
+    lb, wbar, codes, a, b = _layered_basis(ctx, D, n, layers, bits, 52)
+    L = len(layers) - 1
+    gen = torch.Generator(device="cpu").manual_seed(5)
+    beta = (torch.randn((L, n), generator=gen) * 0.3).to(DEV)
+    if L > 2:
+        beta[1] = 0.0                                          # a layer that stays at its mean
+    sws = twa.new_layered_step_workspace(lb)
+    w = torch.full((D,), float("nan"), device=DEV)
+    twa.twa_layered_lift(ctx, lb, beta, wbar if with_base else None, w, sws)
+    status_ok(ctx)
+    base = wbar.cpu().numpy() if with_base else None
+    w_o = orc.lift_layerwise(codes, layers, a, b, beta.cpu().numpy(), base)
+    w_g = w.cpu().numpy()
+    assert rel(w_g, w_o) <= TOL
+    d_o = w_o - (base.astype(np.float64) if with_base else 0.0)
+    d_g = w_g.astype(np.float64) - (base.astype(np.float64) if with_base else 0.0)
+    assert np.linalg.norm(d_g - d_o) <= (2e-5 if with_base else TOL) * np.linalg.norm(d_o)
+    if L > 2 and with_base:
+        r0, r1 = layers[1], layers[2]
+        np.testing.assert_array_equal(w_g[r0:r1], base[r0:r1])
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("D,n,layers", STEP_CASES[1:2] + STEP_CASES[4:6])
+def test_layered_step_matches_oracle_over_iterations(env, D, n, layers, bits):
+    ctx, _ = env
+    lb, wbar, codes, a, b = _layered_basis(ctx, D, n, layers, bits, 53)
+    L = len(layers) - 1
+    sws = twa.new_layered_step_workspace(lb)
+    beta = torch.zeros((L, n), device=DEV)
+    w = torch.empty(D, device=DEV)
+    c = torch.empty((L, n), device=DEV)
+    beta_o = np.zeros((L, n))
+    wbar_o = wbar.cpu().numpy()
+    lr, lam = 0.5, 1e-2
+    for it in range(3):
+        g = inputs.gradient(D, 1e-2, 9, it, torch.bfloat16, DEV)
+        twa.twa_layered_step(ctx, lb, g, lr, lam, beta, wbar, w, sws, c_out=c)
+        status_ok(ctx)
+        # the oracle continues from the GPU's float32 coefficients, so errors do not compound
+        beta_new_o, w_o, c_o = orc.step_layerwise(codes, layers, a, b, g.float().cpu().numpy(), beta_o, wbar_o,
+                                                  lr, lam)
+        assert rel(c.cpu().numpy(), c_o) <= TOL
+        assert rel(beta.cpu().numpy(), beta_new_o) <= TOL
+        w_from_gpu_beta = orc.lift_layerwise(codes, layers, a, b, beta.cpu().numpy(), wbar_o)
+        assert rel(w.cpu().numpy(), w_from_gpu_beta) <= TOL
+        assert rel(w.cpu().numpy(), w_o) <= 2e-5
+        beta_o = beta.cpu().numpy().astype(np.float64)
+
+
+def test_layered_step_reports_nonfinite_and_bad_arguments(env):
+    ctx, _ = env
+    D, n, layers = 40000, 5, [0, 100, 20000, 40000]
+    lb, wbar, _, _, _ = _layered_basis(ctx, D, n, layers, 8, 54)
+    sws = twa.new_layered_step_workspace(lb)
+    g = inputs.gradient(D, 1e-3, 7, 0, torch.float32, DEV)
+    g[30000] = float("inf")
+    c = torch.empty((3, n), device=DEV)
+    twa.twa_layered_project(ctx, lb, g, c, sws)
+    code, detail = twa.twa_get_status(ctx)
+    assert (code, detail) == (twa.TWA_ERR_NONFINITE, 2)
+    twa.twa_clear_status(ctx)
+    assert torch.isfinite(c[:2]).all() and torch.isnan(c[2]).all()
+    beta = torch.zeros((3, n), device=DEV)
+    beta[1, 2] = float("nan")
+    w = torch.empty(D, device=DEV)
+    twa.twa_layered_lift(ctx, lb, beta, wbar, w, sws)
+    code, detail = twa.twa_get_status(ctx)
+    assert (code, detail) == (twa.TWA_ERR_NONFINITE, 1)
+    twa.twa_clear_status(ctx)
+    assert torch.isnan(w[100:20000]).all() and torch.isfinite(w[:100]).all() and torch.isfinite(w[20000:]).all()
+    with pytest.raises(twa.TwaError) as e:
+        twa.twa_layered_project(ctx, lb, g, c, sws[: sws.numel() - 256])
+    assert e.value.code == twa.TWA_ERR_WORKSPACE
