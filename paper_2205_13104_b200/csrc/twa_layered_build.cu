@@ -22,6 +22,7 @@ constexpr long long ITEM_ROWS = 8192;       // rows of one layer handled by one 
 struct Item { int layer; long long r0, r1; };   // flat rows [r0, r1) of one layer
 
 long long granule_rows(int bits) { return 64LL * 8 / bits; }
+constexpr size_t TABLE_SLACK = 8;                           // granule entries past the last column byte
 constexpr int MAX_CTAS = 1024;                              // blocks of a step kernel
 constexpr size_t CTA_TABLE_BYTES = (sizeof(int) * (MAX_CTAS + 1) + 255) / 256 * 256;
 
@@ -312,7 +313,7 @@ size_t twa_layered_basis_bytes(const int64_t* offsets_host, int L, int n, int bi
   if (rows < 1 || n < 1) return 0;
   const size_t codes = twa_basis_bytes(rows, n, bits);
   const size_t granules = static_cast<size_t>(twa_basis_col_stride(rows, bits) / 64);
-  return codes + 256 + 2 * ((sizeof(float) * L + 255) / 256 * 256) + 16 * granules +
+  return codes + 256 + 2 * ((sizeof(float) * L + 255) / 256 * 256) + 16 * (granules + TABLE_SLACK) +
          (sizeof(long long) * (L + 1) + 255) / 256 * 256 * 2 + 2 * CTA_TABLE_BYTES;
 }
 
@@ -379,7 +380,7 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
   size_t o = (codes_bytes + 255) / 256 * 256;
   float* a = reinterpret_cast<float*>(m + o); o += fl;
   float* b = reinterpret_cast<float*>(m + o); o += fl;
-  int* gran = reinterpret_cast<int*>(m + o); o += 16 * n_gran;
+  int* gran = reinterpret_cast<int*>(m + o); o += 16 * (n_gran + TABLE_SLACK);
   long long* d_flat = reinterpret_cast<long long*>(m + o); o += off_bytes;
   long long* d_int = reinterpret_cast<long long*>(m + o); o += off_bytes;
   int* d_cta_first = reinterpret_cast<int*>(m + o); o += CTA_TABLE_BYTES;
@@ -411,8 +412,9 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
   // granule table: layer, valid rows, first flat row of every 64-byte granule of a column
   {
     const long long gr = granule_rows(bits);
-    std::vector<int> tab(4 * n_gran, 0);
-    for (size_t k = 0; k < n_gran; ++k) tab[4 * k] = -1;              // granules behind the last layer
+    // (with slack, so that the last tile of a two-segment tiling finds entries for all its granules)
+    std::vector<int> tab(4 * (n_gran + TABLE_SLACK), 0);
+    for (size_t k = 0; k < n_gran + TABLE_SLACK; ++k) tab[4 * k] = -1;   // granules behind the last layer
     for (int l = 0; l < L; ++l) {
       const long long len = p.flat[l + 1] - p.flat[l];
       for (long long k0 = 0; k0 < len; k0 += gr) {

@@ -8,8 +8,10 @@
 //  * every block owns a contiguous range of tiles, so it meets few layers; a warp's share of a
 //    tile (32*KT bytes of every column) lies inside one 64-byte granule, hence inside one layer,
 //    and the granule table gives its layer, its first flat row and how many of its rows exist;
-//  * g, w_bar and w are addressed by flat row (layers start anywhere), so they move through
-//    ordinary loads and stores, prefetched one tile ahead;
+//  * g, w_bar and w are addressed by flat row (layers start anywhere, so bulk copies cannot be
+//    aligned): four helper warps stage the tile's granule entries and its rows of g (or w_bar)
+//    in the stage beside the codes, each helper several tiles ahead of the MMA warps, and
+//    signal the stage's "full" barrier together with the bulk copy;
 //  * projection sums are kept per (block, warp, layer) and combined in a fixed order by a small
 //    second kernel, which also applies a^l, b^l * sum(g^l) and the coefficient update;
 //  * the lift takes its digit fragments per layer from a table made by a third small kernel,
@@ -23,10 +25,12 @@
 namespace {
 
 constexpr int ROW_FLOATS = 132;                 // one partial row: 128 column sums, sum of g, padding
+constexpr int L_THREADS = (MMA_WARPS + 2) * 32; // MMA warps, the bulk-copy warp, the helper warp
 
 struct LProjectArgs {
-  int n, stages, tiles, tpc, n_gran;
-  unsigned stage_bytes, tx_bytes, scratch_off;
+  int n, stages, tiles, tpc;
+  long long D;
+  unsigned stage_bytes, tx_bytes, scratch_off, aux_off, ering_off;
   const int4* gran;
   const void* g;
   const int* cta_first;
@@ -37,31 +41,167 @@ struct LProjectArgs {
 };
 
 struct LLiftArgs {
-  int n, stages, tiles, tpc, n_gran;
-  unsigned stage_bytes, tx_bytes;
+  int n, stages, tiles, tpc;
+  long long D;
+  unsigned stage_bytes, tx_bytes, aux_off, ering_off;
   const int4* gran;
   const unsigned char* dig;      // [L][4][128] digit bytes of a^l * beta^l_i
   const int* ebits;              // [L] exponent field of the layer's largest |coefficient|
   const float* konst;            // [L] b^l * sum_i beta^l_i
   const float* base;
   float* out;
+  int out_vector_ok;             // out is 16-byte aligned
   int* status;
   unsigned long long wait_limit_ns;
 };
 
+__device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src, int src_bytes) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_16_zfill(uint32_t dst, const void* src, int src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+// The barrier receives one arrival from this thread once all its copies issued so far have landed.
+__device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void init_barriers_layered(twa_smem_header* hdr, int stages) {
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      twa_mbar_init(twa_smem_u32(&hdr->full[s]), 33);           // the bulk copy and the 32 helper lanes
+      twa_mbar_init(twa_smem_u32(&hdr->empty[s]), MMA_WARPS);
+    }
+    hdr->abort_flag = 0;
+    hdr->last_flag = 0;
+    hdr->bad_flag = 0;
+    twa_fence_barrier_init();
+  }
+}
+
+// What a stage holds beside the codes: the tile's granule entries (16 bytes each), then one
+// segment per granule with the granule's rows of the flat vector (g or w_bar).  A segment starts
+// at the 4-byte word that holds the granule's first element, so a bfloat16 granule that starts at
+// an odd flat row sits one element into its segment.
+__host__ __device__ constexpr int granule_rows(int bits) { return 64 * 8 / bits; }
+__host__ __device__ constexpr int segment_bytes(int bits) { return granule_rows(bits) * 4 + 16; }
+__host__ __device__ constexpr int aux_bytes(int bits, int kt) { return 8 * kt * (16 + segment_bytes(bits)); }
+
+constexpr int ENTRY_DEPTH = 16;                                  // tiles the helper reads entries ahead
+constexpr int ENTRY_RING_BYTES = ENTRY_DEPTH * 16 * 16;          // up to 16 granules per tile
+
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// The helper warp: for every tile of the block's sequence, asynchronous copies of the granule
+// entries and of the rows of `src` the tile's granules cover (flat rows have no alignment
+// guarantee, which rules out bulk copies), straight into the tile's stage; each lane's copies report to the stage's "full"
+// barrier.  The copies' addresses come from the entries, which the warp therefore fetches
+// ENTRY_DEPTH tiles ahead into a ring of its own (`ering`), also asynchronously, so that it
+// never waits for a load issued recently.  src may be NULL (only entries are staged).
+template <int BITS, int KT, int ES>
+__device__ __forceinline__ void helper_loop(twa_smem_header* hdr, unsigned char* ring, unsigned stage_bytes,
+                                            unsigned aux_off, int stages, int t_first, int t_count,
+                                            bool reverse, const int4* __restrict__ gran, const void* src,
+                                            long long D, int4* ering, int lane, int* status,
+                                            unsigned long long limit) {
+  constexpr int GR = granule_rows(BITS);
+  constexpr int GPT = 8 * KT;
+  constexpr int SEG = segment_bytes(BITS);
+  constexpr int QW = GR * ES / 16;                     // 16-byte pieces of a granule's rows
+  constexpr int TQ = GPT * QW;                         // and of a tile's: a multiple of 32
+  static_assert(TQ % 32 == 0, "pieces per tile");
+  volatile int* abort_flag = &hdr->abort_flag;
+  const char* sbytes = static_cast<const char*>(src);
+  const long long total_bytes = D * ES;
+  auto entries_of = [&](int k) {
+    return gran + static_cast<size_t>(t_first + (reverse ? (t_count - 1 - k) : k)) * GPT + lane;
+  };
+  for (int j = 0; j < ENTRY_DEPTH; ++j) {              // one group per tile, also when it is empty
+    if (lane < GPT && j < t_count) cp_async_16(twa_smem_u32(ering + j * GPT + lane), entries_of(j));
+    cp_async_commit();
+  }
+  int s = 0, use = 0, slot = 0;
+  for (int k = 0; k < t_count; ++k) {
+    cp_async_wait_group<ENTRY_DEPTH - 1>();            // the group that brought tile k's entries
+    __syncwarp();
+    const int4* ep = ering + slot * GPT;
+    if (use > 0 && !twa_mbar_wait(twa_smem_u32(&hdr->empty[s]), static_cast<unsigned>(use - 1) & 1u, abort_flag, limit)) {
+      twa_set_status(status, TWA_ERR_TIMEOUT, -1);
+      break;
+    }
+    const uint32_t aux = twa_smem_u32(ring + static_cast<size_t>(s) * stage_bytes + aux_off);
+    if (lane < GPT) cp_async_16(aux + lane * 16, entries_of(k));
+    if (src) {
+      // The tile's rows in 16-byte pieces, one per lane and pass.  A granule whose first row sits
+      // on a 16-byte boundary of src (every granule, when the layers' sizes are multiples of 8)
+      // is copied 16 bytes at a time; any other granule 4 bytes at a time.
+#pragma unroll
+      for (int i = 0; i < TQ / 32; ++i) {
+        const int x = i * 32 + lane, q = x / QW, j = x % QW;
+        const int4 e = ep[q];
+        if (e.x < 0) continue;
+        const long long gbyte = static_cast<long long>(e.z) * ES;            // the granule's first row in src
+        const uint32_t seg = aux + GPT * 16 + q * SEG;
+        if ((gbyte & 15) == 0) {
+          const int nbytes = e.y * ES - j * 16;                                // bytes of existing rows from here on
+          if (nbytes > 0) cp_async_16_zfill(seg + j * 16, sbytes + gbyte + j * 16, nbytes < 16 ? nbytes : 16);
+        } else {
+          const long long byte0 = gbyte & ~3LL;                                // word holding the first row
+          const int shift = ES == 2 ? (e.z & 1) : 0;
+#pragma unroll
+          for (int t = 0; t < (ES == 2 ? 5 : 4); ++t) {
+            if (t == 4 && j != QW - 1) continue;                               // the one word past a shifted granule
+            const int w = 4 * j + t;
+            const int first = ES == 2 ? 2 * w - shift : w;                     // first row the word holds
+            if (first < e.y) {
+              const long long off = byte0 + 4LL * w;
+              const long long rem = total_bytes - off;
+              cp_async_4(seg + 4 * w, sbytes + off, rem >= 4 ? 4 : static_cast<int>(rem));
+            }
+          }
+        }
+      }
+    }
+    cp_async_arrive_noinc(twa_smem_u32(&hdr->full[s]));
+    __syncwarp();                                      // every lane has read the ring slot
+    if (lane < GPT && k + ENTRY_DEPTH < t_count)
+      cp_async_16(twa_smem_u32(ering + slot * GPT + lane), entries_of(k + ENTRY_DEPTH));
+    cp_async_commit();
+    if (++slot == ENTRY_DEPTH) slot = 0;
+    if (++s == stages) {
+      s = 0;
+      ++use;
+    }
+  }
+  cp_async_wait_group<0>();                            // nothing of this warp is in flight when it leaves
+}
+
 // ------------------------------------------------------------------------------------------------
 template <int BITS, bool GBF16, int MT, int KT>
-__global__ void __launch_bounds__(MMA_THREADS, 1)
+__global__ void __launch_bounds__(L_THREADS, 1)
 layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProjectArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
   constexpr int RB = 32 * 8 / BITS;                    // rows behind 32 bytes of a column
-  constexpr int GPT = 8 * KT;                          // granules of a column per tile
   twa_smem_header* hdr = reinterpret_cast<twa_smem_header*>(smem);
   unsigned char* ring = smem + TWA_SMEM_HEADER;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gid = lane >> 2, tig = lane & 3;
-  init_barriers(hdr, a.stages);
+  init_barriers_layered(hdr, a.stages);
+  const int my_first = a.cta_first[blockIdx.x], my_base = a.cta_base[blockIdx.x];
+  {
+    // a warp writes a row of partial sums only for the layers it meets: the rest must read as zero
+    float* mine = a.partials + static_cast<size_t>(my_base) * MMA_WARPS * ROW_FLOATS;
+    const int count = (a.cta_base[blockIdx.x + 1] - my_base) * MMA_WARPS * ROW_FLOATS;
+    for (int i = threadIdx.x; i < count; i += blockDim.x) mine[i] = 0.0f;
+  }
   __syncthreads();
   const int t_first = blockIdx.x * a.tpc;
   const int t_count = (a.tiles - t_first) < a.tpc ? (a.tiles - t_first) : a.tpc;
@@ -70,6 +210,12 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
     if (lane == 0)
       producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, KT, 0, 0,
                         0, 0, a.tx_bytes, false, a.status, a.wait_limit_ns);
+    return;
+  }
+  if (warp > MMA_WARPS) {
+    helper_loop<BITS, KT, (GBF16 ? 2 : 4)>(hdr, ring, a.stage_bytes, a.aux_off, a.stages, t_first, t_count, false,
+                                           a.gran, a.g, a.D, reinterpret_cast<int4*>(smem + a.ering_off), lane,
+                                           a.status, a.wait_limit_ns);
     return;
   }
   unsigned char* digw = smem + a.scratch_off + warp * DIGIT_SCRATCH;
@@ -86,38 +232,15 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
       const int chunk = (warp * KT + u) * 2 + (lm >> 1);
       aoff[u][mt] = static_cast<uint32_t>(j * col_bytes + ((chunk >> 5) << 9) + (twa_chunk_slot(chunk & 31, j) << 4));
     }
-  const int wb = warp * 32 * KT;                       // first byte of the warp's share of a tile column
-  const int gran_in_tile = wb >> 6;
-  const int rig0 = (wb & 63) * 8 / BITS;               // first row of the share inside its granule
-  const unsigned short* g16 = static_cast<const unsigned short*>(a.g);
-  const float* g32 = static_cast<const float*>(a.g);
-
-  // the granule entry and the gradient values of one tile
-  int4 e_next;
-  float gn0[KT], gn1[KT];
-  auto fetch = [&](int tile) {
-    const int gi = tile * GPT + gran_in_tile;
-    e_next = gi < a.n_gran ? __ldg(a.gran + gi) : make_int4(-1, 0, 0, 0);
-#pragma unroll
-    for (int u = 0; u < KT; ++u) {
-      gn0[u] = gn1[u] = 0.0f;
-      if (e_next.x >= 0) {
-        const int r = rig0 + u * RB + (BITS == 8 ? lane : 2 * lane);
-        const long long f = static_cast<long long>(e_next.z) + r;
-        if (r < e_next.y) gn0[u] = GBF16 ? __uint_as_float(static_cast<uint32_t>(__ldg(g16 + f)) << 16) : __ldg(g32 + f);
-        if (BITS == 4 && r + 1 < e_next.y)
-          gn1[u] = GBF16 ? __uint_as_float(static_cast<uint32_t>(__ldg(g16 + f + 1)) << 16) : __ldg(g32 + f + 1);
-      }
-    }
-  };
-
+  const int gran_in_tile = (warp * 32 * KT) >> 6;      // the granule holding the warp's share of a column
+  const int rig0 = ((warp * 32 * KT) & 63) * 8 / BITS; // first row of the share inside the granule
+  const unsigned seg_off = a.aux_off + 8 * KT * 16 + gran_in_tile * segment_bytes(BITS);
   float facc[MT][2];
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt) facc[mt][0] = facc[mt][1] = 0.0f;
   float gsum = 0.0f;
   int cur_layer = -1;
   bool bad = false;
-  const int my_first = a.cta_first[blockIdx.x], my_base = a.cta_base[blockIdx.x];
   auto flush = [&]() {
     float* row = a.partials + (static_cast<size_t>(my_base + cur_layer - my_first) * MMA_WARPS + warp) * ROW_FLOATS;
 #pragma unroll
@@ -144,23 +267,37 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
   volatile int* abort_flag = &hdr->abort_flag;
   int s = 0;
   unsigned phase = 0;
-  fetch(t_first);
   for (int k = 0; k < t_count; ++k) {
-    const int4 e = e_next;
-    float g0[KT], g1[KT];
-#pragma unroll
-    for (int u = 0; u < KT; ++u) { g0[u] = gn0[u]; g1[u] = gn1[u]; }
-    if (k + 1 < t_count) fetch(t_first + k + 1);
     if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
       twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
       break;
+    }
+    const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
+    const int4 e = reinterpret_cast<const int4*>(st + a.aux_off)[gran_in_tile];
+    // the granule's rows of g, staged by the helper; rows past the layer's end hold nothing
+    float g0[KT], g1[KT];
+#pragma unroll
+    for (int u = 0; u < KT; ++u) {
+      const int r = rig0 + u * RB + (BITS == 8 ? lane : 2 * lane);
+      float x0, x1 = 0.0f;
+      if (GBF16) {
+        const unsigned short* gs = reinterpret_cast<const unsigned short*>(st + seg_off) + (e.z & 1);
+        x0 = __uint_as_float(static_cast<uint32_t>(gs[r]) << 16);
+        if (BITS == 4) x1 = __uint_as_float(static_cast<uint32_t>(gs[r + 1]) << 16);
+      } else {
+        const float* gs = reinterpret_cast<const float*>(st + seg_off);
+        x0 = gs[r];
+        if (BITS == 4) x1 = gs[r + 1];
+      }
+      g0[u] = r < e.y ? x0 : 0.0f;
+      g1[u] = (BITS == 4 && r + 1 < e.y) ? x1 : 0.0f;
     }
     if (e.x != cur_layer) {
       if (cur_layer >= 0) flush();
       cur_layer = e.x;
     }
     if (e.x >= 0) {
-      const uint32_t tile_base = twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes);
+      const uint32_t tile_base = twa_smem_u32(st);
       unsigned mb = 0u;
 #pragma unroll
       for (int u = 0; u < KT; ++u) {
@@ -237,47 +374,16 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
   if (cur_layer >= 0) flush();
 }
 
-// One block per layer: fixed-order sum of the layer's partial rows, c = a S + b sum(g), update.
-__global__ void layered_combine_kernel(const float* __restrict__ partials, const int* __restrict__ cta_first,
-                                       const int* __restrict__ cta_base, int ctas, int n,
-                                       const float* __restrict__ a, const float* __restrict__ b,
-                                       float* c_out, float* beta, float lr, float lambda, int* status) {
-  const int l = blockIdx.x, i = threadIdx.x;
-  double S = 0.0, Sg = 0.0;
-  for (int cta = 0; cta < ctas; ++cta) {
-    const int f = cta_first[cta], cnt = cta_base[cta + 1] - cta_base[cta];
-    if (l < f || l >= f + cnt) continue;
-    const float* rows = partials + static_cast<size_t>(cta_base[cta] + l - f) * MMA_WARPS * ROW_FLOATS;
-    for (int w = 0; w < MMA_WARPS; ++w) {
-      if (i < n) S += static_cast<double>(__ldcg(rows + w * ROW_FLOATS + i));
-      Sg += static_cast<double>(__ldcg(rows + w * ROW_FLOATS + 128));
-    }
-  }
-  if (i >= n) return;
-  const double c = static_cast<double>(a[l]) * S + static_cast<double>(b[l]) * Sg;
-  if (!isfinite(c)) twa_set_status(status, TWA_ERR_NONFINITE, l);
-  if (c_out) c_out[static_cast<size_t>(l) * n + i] = static_cast<float>(c);
-  if (beta) {
-    const double decay = 1.0 - static_cast<double>(lr) * static_cast<double>(lambda);
-    beta[static_cast<size_t>(l) * n + i] =
-        static_cast<float>(decay * static_cast<double>(beta[static_cast<size_t>(l) * n + i]) - static_cast<double>(lr) * c);
-  }
-}
-
-// One block (128 threads) per layer: digits of a^l * beta^l_i on the layer's common scale, and
-// the constant b^l * sum_i beta^l_i.
-__global__ void layered_coef_kernel(const float* __restrict__ beta, int n, const float* __restrict__ a,
-                                    const float* __restrict__ b, float mult, unsigned char* __restrict__ dig,
-                                    int* __restrict__ ebits_out, float* __restrict__ konst, int* status) {
-  __shared__ unsigned amax;
-  const int l = blockIdx.x, i = threadIdx.x;
-  if (i == 0) amax = 0u;
-  __syncthreads();
-  float coef = 0.0f;
-  if (i < n) coef = beta[static_cast<size_t>(l) * n + i] * mult * a[l];
-  atomicMax(&amax, __float_as_uint(coef) & 0x7FFFFFFFu);
-  __syncthreads();
-  const unsigned ebits = amax >> 23;
+// Digits of the layer's coefficients a^l * beta^l_i on their common scale, and the constant
+// b^l * sum_i beta^l_i.  Called by the first 128 threads of a block; `amax` is shared and zero.
+__device__ __forceinline__ void layer_coefficients(int l, int i, int n, float beta_i, float al, float bl,
+                                                   const float* beta_row, unsigned* amax,
+                                                   unsigned char* __restrict__ dig, int* __restrict__ ebits_out,
+                                                   float* __restrict__ konst, int* status) {
+  const float coef = i < n ? beta_i * al : 0.0f;
+  atomicMax(amax, __float_as_uint(coef) & 0x7FFFFFFFu);
+  asm volatile("bar.sync 1, 128;" ::: "memory");
+  const unsigned ebits = *amax >> 23;
   const bool bad = ebits >= 255u, live = ebits >= 5u && !bad;
   uint32_t d = 0;
   if (live) d = cut_digits(coef * __uint_as_float((259u - ebits) << 23));
@@ -285,28 +391,115 @@ __global__ void layered_coef_kernel(const float* __restrict__ beta, int n, const
   for (int k = 0; k < 4; ++k) dig[static_cast<size_t>(l) * 512 + k * 128 + i] = static_cast<unsigned char>(d >> (8 * k));
   if (i == 0) {
     double sb = 0.0;
-    for (int q = 0; q < n; ++q) sb += static_cast<double>(beta[static_cast<size_t>(l) * n + q]);
-    const double kk = static_cast<double>(b[l]) * static_cast<double>(mult) * sb;
+    for (int q = 0; q < n; ++q) sb += static_cast<double>(beta_row[q]);
+    const double kk = static_cast<double>(bl) * sb;
     if (bad || !isfinite(kk)) twa_set_status(status, TWA_ERR_NONFINITE, l);
     konst[l] = static_cast<float>(kk);
     ebits_out[l] = bad ? -1 : (live ? static_cast<int>(ebits) : 0);
   }
 }
 
+constexpr int COMBINE_PARTS = 4;
+
+// One block of 128 * COMBINE_PARTS threads per layer: fixed-order sum of the layer's partial rows,
+// c = a S + b sum(g), the coefficient update, and (dig != NULL) the lift's coefficient digits.
+// Part p sums a contiguous quarter of the blocks that met the layer; the parts are added in order.
+__global__ void __launch_bounds__(128 * COMBINE_PARTS)
+layered_combine_kernel(const float* __restrict__ partials, const int* __restrict__ cta_first,
+                       const int* __restrict__ cta_base, int ctas, int n, const float* __restrict__ a,
+                       const float* __restrict__ b, float* c_out, float* beta, float lr, float lambda,
+                       unsigned char* dig, int* ebits_out, float* konst, int* status) {
+  __shared__ int range[2];
+  __shared__ unsigned amax;
+  __shared__ double part_s[COMBINE_PARTS][128], part_g[COMBINE_PARTS];
+  __shared__ float beta_new[128];
+  const int l = blockIdx.x, i = threadIdx.x & 127, p = threadIdx.x >> 7;
+  if (threadIdx.x == 0) {
+    range[0] = ctas;
+    range[1] = -1;
+    amax = 0u;
+  }
+  __syncthreads();
+  for (int cta = threadIdx.x; cta < ctas; cta += blockDim.x) {        // which blocks met this layer
+    const int f = cta_first[cta], cnt = cta_base[cta + 1] - cta_base[cta];
+    if (l >= f && l < f + cnt) {
+      atomicMin(&range[0], cta);
+      atomicMax(&range[1], cta);
+    }
+  }
+  __syncthreads();
+  const int c0 = range[0], c1 = range[1] + 1;                          // contiguous: blocks own tile ranges in order
+  const int per = (c1 - c0 + COMBINE_PARTS - 1) / COMBINE_PARTS;
+  const int lo = c0 + p * per, hi = (lo + per) < c1 ? (lo + per) : c1;
+  double S = 0.0, Sg = 0.0;
+  for (int cta = lo; cta < hi; ++cta) {
+    const float* rows = partials + static_cast<size_t>(cta_base[cta] + l - cta_first[cta]) * MMA_WARPS * ROW_FLOATS;
+    float v[MMA_WARPS], vg[MMA_WARPS];
+#pragma unroll
+    for (int w = 0; w < MMA_WARPS; ++w) {
+      v[w] = i < n ? __ldcg(rows + w * ROW_FLOATS + i) : 0.0f;
+      vg[w] = __ldcg(rows + w * ROW_FLOATS + 128);
+    }
+#pragma unroll
+    for (int w = 0; w < MMA_WARPS; ++w) {
+      S += static_cast<double>(v[w]);
+      Sg += static_cast<double>(vg[w]);
+    }
+  }
+  part_s[p][i] = S;
+  if (i == 0) part_g[p] = Sg;
+  __syncthreads();
+  if (p != 0) return;
+  S = 0.0;
+  Sg = 0.0;
+#pragma unroll
+  for (int q = 0; q < COMBINE_PARTS; ++q) {
+    S += part_s[q][i];
+    Sg += part_g[q];
+  }
+  float bnew = 0.0f;
+  if (i < n) {
+    const double c = static_cast<double>(a[l]) * S + static_cast<double>(b[l]) * Sg;
+    if (!isfinite(c)) twa_set_status(status, TWA_ERR_NONFINITE, l);
+    if (c_out) c_out[static_cast<size_t>(l) * n + i] = static_cast<float>(c);
+    if (beta) {
+      const double decay = 1.0 - static_cast<double>(lr) * static_cast<double>(lambda);
+      bnew = static_cast<float>(decay * static_cast<double>(beta[static_cast<size_t>(l) * n + i]) - static_cast<double>(lr) * c);
+      beta[static_cast<size_t>(l) * n + i] = bnew;
+    }
+  }
+  if (dig) {                                                           // only with beta: the step
+    beta_new[i] = bnew;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    layer_coefficients(l, i, n, bnew, a[l], b[l], beta_new, &amax, dig, ebits_out, konst, status);
+  }
+}
+
+// One block (128 threads) per layer: the lift's coefficient digits from given coefficients.
+__global__ void layered_coef_kernel(const float* __restrict__ beta, int n, const float* __restrict__ a,
+                                    const float* __restrict__ b, unsigned char* __restrict__ dig,
+                                    int* __restrict__ ebits_out, float* __restrict__ konst, int* status) {
+  __shared__ unsigned amax;
+  const int l = blockIdx.x, i = threadIdx.x;
+  if (i == 0) amax = 0u;
+  __syncthreads();
+  const float bi = i < n ? beta[static_cast<size_t>(l) * n + i] : 0.0f;
+  layer_coefficients(l, i, n, bi, a[l], b[l], beta + static_cast<size_t>(l) * n, &amax, dig, ebits_out, konst, status);
+}
+
 // ------------------------------------------------------------------------------------------------
 template <int BITS, int KS, int KT>
-__global__ void __launch_bounds__(MMA_THREADS, 1)
+__global__ void __launch_bounds__(L_THREADS, 1)
 layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
   constexpr int LROWS = BITS == 8 ? 2 : 4;
   constexpr int RB = 32 * 8 / BITS;
-  constexpr int GPT = 8 * KT;
   twa_smem_header* hdr = reinterpret_cast<twa_smem_header*>(smem);
   unsigned char* ring = smem + TWA_SMEM_HEADER;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gid = lane >> 2, tig = lane & 3;
-  init_barriers(hdr, a.stages);
+  init_barriers_layered(hdr, a.stages);
   __syncthreads();
   const int t_first = blockIdx.x * a.tpc;
   const int t_count = (a.tiles - t_first) < a.tpc ? (a.tiles - t_first) : a.tpc;
@@ -314,6 +507,11 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
     if (lane == 0)
       producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, KT, 0, 0,
                         0, 0, a.tx_bytes, true, a.status, a.wait_limit_ns);
+    return;
+  }
+  if (warp > MMA_WARPS) {
+    helper_loop<BITS, KT, 4>(hdr, ring, a.stage_bytes, a.aux_off, a.stages, t_first, t_count, true, a.gran, a.base,
+                             a.D, reinterpret_cast<int4*>(smem + a.ering_off), lane, a.status, a.wait_limit_ns);
     return;
   }
   const int lm = lane >> 3, lr = lane & 7;
@@ -334,25 +532,11 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
   const int wb = warp * 32 * KT;
   const int gran_in_tile = wb >> 6;
   const int rig0 = (wb & 63) * 8 / BITS;
+  const unsigned seg_off = a.aux_off + 8 * KT * 16 + gran_in_tile * segment_bytes(BITS);
   // rows (inside the granule) this lane finishes for block u: chunk tig, LROWS rows from LROWS * gid
   int rrow[KT];
 #pragma unroll
   for (int u = 0; u < KT; ++u) rrow[u] = rig0 + u * RB + 16 * tig * (8 / BITS) + LROWS * gid;
-
-  int4 e_next;
-  float bn[KT][LROWS];
-  auto fetch = [&](int tile) {
-    const int gi = tile * GPT + gran_in_tile;
-    e_next = gi < a.n_gran ? __ldg(a.gran + gi) : make_int4(-1, 0, 0, 0);
-#pragma unroll
-    for (int u = 0; u < KT; ++u)
-#pragma unroll
-      for (int i = 0; i < LROWS; ++i) {
-        bn[u][i] = 0.0f;
-        if (a.base && tig < 2 && e_next.x >= 0 && rrow[u] + i < e_next.y)
-          bn[u][i] = a.base[static_cast<long long>(e_next.z) + rrow[u] + i];
-      }
-  };
 
   uint32_t bfrag[KS][2];
 #pragma unroll
@@ -362,15 +546,28 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
   volatile int* abort_flag = &hdr->abort_flag;
   int s = 0;
   unsigned phase = 0;
-  fetch(t_first + t_count - 1);
   for (int k = 0; k < t_count; ++k) {                   // backwards, like the producer
-    const int4 e = e_next;
+    if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
+      twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+      break;
+    }
+    const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
+    const int4 e = reinterpret_cast<const int4*>(st + a.aux_off)[gran_in_tile];
+    const float* gs = reinterpret_cast<const float*>(st + seg_off);        // the granule's rows of base, staged
     float bv[KT][LROWS];
 #pragma unroll
-    for (int u = 0; u < KT; ++u)
+    for (int u = 0; u < KT; ++u) {
+      if (!a.base) {
 #pragma unroll
-      for (int i = 0; i < LROWS; ++i) bv[u][i] = bn[u][i];
-    if (k + 1 < t_count) fetch(t_first + t_count - 2 - k);
+        for (int i = 0; i < LROWS; ++i) bv[u][i] = 0.0f;
+      } else if (LROWS == 2) {
+        const float2 x = *reinterpret_cast<const float2*>(gs + rrow[u]);
+        bv[u][0] = x.x; bv[u][1] = x.y;
+      } else {
+        const float4 x = *reinterpret_cast<const float4*>(gs + rrow[u]);
+        bv[u][0] = x.x; bv[u][1] = x.y; bv[u][LROWS - 2] = x.z; bv[u][LROWS - 1] = x.w;
+      }
+    }
     if (e.x != cur_layer && e.x >= 0) {                  // new layer: its digit fragments and factors
       cur_layer = e.x;
       const int eb = a.ebits[cur_layer];
@@ -392,11 +589,7 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
         }
       }
     }
-    if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
-      twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
-      break;
-    }
-    const uint32_t tile_base = twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes);
+    const uint32_t tile_base = twa_smem_u32(st);
     float keep[KT][LROWS];
 #pragma unroll
     for (int u = 0; u < KT; ++u) {
@@ -451,11 +644,22 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
     __syncwarp();
     if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
     if (e.x >= 0 && tig < 2) {
+      const bool aligned = (e.z & (LROWS - 1)) == 0 && a.out_vector_ok;   // the lane's rows start on a vector boundary
 #pragma unroll
-      for (int u = 0; u < KT; ++u)
+      for (int u = 0; u < KT; ++u) {
+        float* dst = a.out + static_cast<long long>(e.z) + rrow[u];
+        float r[LROWS];
 #pragma unroll
-        for (int i = 0; i < LROWS; ++i)
-          if (rrow[u] + i < e.y) a.out[static_cast<long long>(e.z) + rrow[u] + i] = bv[u][i] + keep[u][i] + kon;
+        for (int i = 0; i < LROWS; ++i) r[i] = bv[u][i] + keep[u][i] + kon;
+        if (aligned && rrow[u] + LROWS <= e.y) {
+          if (LROWS == 2) *reinterpret_cast<float2*>(dst) = make_float2(r[0], r[1]);
+          else *reinterpret_cast<float4*>(dst) = make_float4(r[0], r[1], r[LROWS - 2], r[LROWS - 1]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < LROWS; ++i)
+            if (rrow[u] + i < e.y) dst[i] = r[i];
+        }
+      }
     }
     if (++s == a.stages) {
       s = 0;
@@ -504,7 +708,7 @@ int launch_lproject_t(twa_ctx* ctx, const CUtensorMap& mp, const LProjectArgs& a
   static int smem_limit[2][64] = {{0}};
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[kt - 1][ctx->device & 63], smem);
   if (rc) return rc;
-  kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, a);
+  kern<<<grid, L_THREADS, smem, ctx->stream>>>(mp, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
 }
@@ -529,7 +733,7 @@ int launch_llift_t(twa_ctx* ctx, const CUtensorMap& mp, const LLiftArgs& a, int 
   static int smem_limit[2][64] = {{0}};
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[kt - 1][ctx->device & 63], smem);
   if (rc) return rc;
-  kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, a);
+  kern<<<grid, L_THREADS, smem, ctx->stream>>>(mp, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
 }
@@ -551,7 +755,7 @@ int stage_count(const twa_ctx* ctx, int fixed, int stage_bytes) {
 }
 
 int do_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype, float* c_out,
-               float* beta, float lr, float lambda, char* sws) {
+               float* beta, float lr, float lambda, bool with_digits, char* sws) {
   const StepLayout w = step_layout(lb);
   const int n = lb->codes.n, kt = lb->kt;
   CUtensorMap mp;
@@ -561,12 +765,15 @@ int do_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dty
   a.n = n;
   a.tiles = lb->tiles;
   a.tpc = lb->tiles_per_cta;
-  a.n_gran = static_cast<int>(lb->codes.col_stride / 64);
+  a.D = lb->D;
   a.tx_bytes = static_cast<unsigned>(n) * TWA_TILE_COL_BYTES * kt;
-  a.stage_bytes = (a.tx_bytes + 1023) / 1024 * 1024;
-  a.stages = stage_count(ctx, TWA_SMEM_HEADER + MMA_WARPS * DIGIT_SCRATCH + 1024, static_cast<int>(a.stage_bytes));
+  a.aux_off = a.tx_bytes;
+  a.stage_bytes = (a.aux_off + aux_bytes(lb->codes.bits, kt) + 1023) / 1024 * 1024;
+  a.stages = stage_count(ctx, TWA_SMEM_HEADER + MMA_WARPS * DIGIT_SCRATCH + ENTRY_RING_BYTES + 1024,
+                         static_cast<int>(a.stage_bytes));
   if (a.stages < 2) return TWA_ERR_UNSUPPORTED;
   a.scratch_off = TWA_SMEM_HEADER + static_cast<unsigned>(a.stages) * a.stage_bytes;
+  a.ering_off = a.scratch_off + MMA_WARPS * DIGIT_SCRATCH;
   a.gran = reinterpret_cast<const int4*>(lb->granules);
   a.g = g;
   a.cta_first = lb->cta_first_layer;
@@ -574,8 +781,7 @@ int do_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dty
   a.partials = reinterpret_cast<float*>(sws + w.partials);
   a.status = ctx->d_status;
   a.wait_limit_ns = ctx->wait_limit_ns;
-  TWA_CUDA_OK(ctx, cudaMemsetAsync(a.partials, 0, w.dig - w.partials, ctx->stream));
-  const int smem = static_cast<int>(a.scratch_off) + MMA_WARPS * DIGIT_SCRATCH + 1024;
+  const int smem = static_cast<int>(a.ering_off) + ENTRY_RING_BYTES + 1024;
   const bool bf16 = g_dtype == TWA_BF16;
   if (lb->codes.bits == 8)
     rc = bf16 ? launch_lproject<8, true>(ctx, mp, a, kt, lb->cta_count, smem)
@@ -584,22 +790,25 @@ int do_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dty
     rc = bf16 ? launch_lproject<4, true>(ctx, mp, a, kt, lb->cta_count, smem)
               : launch_lproject<4, false>(ctx, mp, a, kt, lb->cta_count, smem);
   if (rc) return rc;
-  layered_combine_kernel<<<lb->L, 128, 0, ctx->stream>>>(a.partials, lb->cta_first_layer, lb->cta_run_base,
-                                                       lb->cta_count, n, lb->a, lb->b, c_out, beta, lr, lambda,
-                                                       ctx->d_status);
+  layered_combine_kernel<<<lb->L, 128 * COMBINE_PARTS, 0, ctx->stream>>>(
+      a.partials, lb->cta_first_layer, lb->cta_run_base, lb->cta_count, n, lb->a, lb->b, c_out, beta, lr, lambda,
+      with_digits ? reinterpret_cast<unsigned char*>(sws + w.dig) : nullptr, reinterpret_cast<int*>(sws + w.ebits),
+      reinterpret_cast<float*>(sws + w.konst), ctx->d_status);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
 }
 
 int do_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* beta, const float* base, float* out,
-            char* sws) {
+            bool digits_ready, char* sws) {
   const StepLayout w = step_layout(lb);
   const int n = lb->codes.n, kt = lb->kt;
   unsigned char* dig = reinterpret_cast<unsigned char*>(sws + w.dig);
   int* ebits = reinterpret_cast<int*>(sws + w.ebits);
   float* konst = reinterpret_cast<float*>(sws + w.konst);
-  layered_coef_kernel<<<lb->L, 128, 0, ctx->stream>>>(beta, n, lb->a, lb->b, 1.0f, dig, ebits, konst, ctx->d_status);
-  TWA_CUDA_OK(ctx, cudaGetLastError());
+  if (!digits_ready) {
+    layered_coef_kernel<<<lb->L, 128, 0, ctx->stream>>>(beta, n, lb->a, lb->b, dig, ebits, konst, ctx->d_status);
+    TWA_CUDA_OK(ctx, cudaGetLastError());
+  }
   CUtensorMap mp;
   int rc = encode_codes_map(ctx, &lb->codes, kt, &mp);
   if (rc) return rc;
@@ -607,20 +816,23 @@ int do_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* beta, const 
   a.n = n;
   a.tiles = lb->tiles;
   a.tpc = lb->tiles_per_cta;
-  a.n_gran = static_cast<int>(lb->codes.col_stride / 64);
+  a.D = lb->D;
   a.tx_bytes = static_cast<unsigned>(n) * TWA_TILE_COL_BYTES * kt;
-  a.stage_bytes = (a.tx_bytes + 1023) / 1024 * 1024;
-  a.stages = stage_count(ctx, TWA_SMEM_HEADER + 1024, static_cast<int>(a.stage_bytes));
+  a.aux_off = a.tx_bytes;
+  a.stage_bytes = (a.aux_off + aux_bytes(lb->codes.bits, kt) + 1023) / 1024 * 1024;
+  a.stages = stage_count(ctx, TWA_SMEM_HEADER + ENTRY_RING_BYTES + 1024, static_cast<int>(a.stage_bytes));
   if (a.stages < 2) return TWA_ERR_UNSUPPORTED;
+  a.ering_off = TWA_SMEM_HEADER + static_cast<unsigned>(a.stages) * a.stage_bytes;
   a.gran = reinterpret_cast<const int4*>(lb->granules);
   a.dig = dig;
   a.ebits = ebits;
   a.konst = konst;
   a.base = base;
   a.out = out;
+  a.out_vector_ok = (reinterpret_cast<uintptr_t>(out) & 15) == 0;
   a.status = ctx->d_status;
   a.wait_limit_ns = ctx->wait_limit_ns;
-  const int smem = TWA_SMEM_HEADER + a.stages * static_cast<int>(a.stage_bytes) + 1024;
+  const int smem = static_cast<int>(a.ering_off) + ENTRY_RING_BYTES + 1024;
   return lb->codes.bits == 8 ? launch_llift<8>(ctx, mp, a, kt, lb->cta_count, smem)
                              : launch_llift<4>(ctx, mp, a, kt, lb->cta_count, smem);
 }
@@ -651,8 +863,9 @@ int twa_layered_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g
   int rc = check_step_args(ctx, lb, sws, sws_bytes);
   if (rc) return rc;
   if (!g || !c_out || (g_dtype != TWA_F32 && g_dtype != TWA_BF16)) return TWA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(g) & 3) return TWA_ERR_MISALIGNED;         // staged in 4-byte words
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-  return do_project(ctx, lb, g, g_dtype, c_out, nullptr, 0.0f, 0.0f, static_cast<char*>(sws));
+  return do_project(ctx, lb, g, g_dtype, c_out, nullptr, 0.0f, 0.0f, false, static_cast<char*>(sws));
 }
 
 int twa_layered_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* beta, const float* base,
@@ -660,8 +873,9 @@ int twa_layered_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* bet
   int rc = check_step_args(ctx, lb, sws, sws_bytes);
   if (rc) return rc;
   if (!beta || !w_out) return TWA_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(base) & 3) || (reinterpret_cast<uintptr_t>(w_out) & 3)) return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-  return do_lift(ctx, lb, beta, base, w_out, static_cast<char*>(sws));
+  return do_lift(ctx, lb, beta, base, w_out, false, static_cast<char*>(sws));
 }
 
 int twa_layered_step(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype, float lr,
@@ -670,10 +884,13 @@ int twa_layered_step(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, t
   int rc = check_step_args(ctx, lb, sws, sws_bytes);
   if (rc) return rc;
   if (!g || !beta || !wbar || !w || (g_dtype != TWA_F32 && g_dtype != TWA_BF16)) return TWA_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(g) & 3) || (reinterpret_cast<uintptr_t>(wbar) & 3) ||
+      (reinterpret_cast<uintptr_t>(w) & 3))
+    return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-  rc = do_project(ctx, lb, g, g_dtype, c_out, beta, lr, lambda, static_cast<char*>(sws));
+  rc = do_project(ctx, lb, g, g_dtype, c_out, beta, lr, lambda, true, static_cast<char*>(sws));
   if (rc) return rc;
-  return do_lift(ctx, lb, beta, wbar, w, static_cast<char*>(sws));
+  return do_lift(ctx, lb, beta, wbar, w, true, static_cast<char*>(sws));
 }
 
 }  // extern "C"

@@ -177,3 +177,78 @@ WORKLOADS = {
     "decoder1p3b": Workload("decoder1p3b", 1_315_758_080, 32, 0.002, 0.0005, 1e-4, "bf16",
                             (8, 4), 50, chunked_build=True),
 }
+
+
+# --------------------------------------------------------------------------------------
+# Layer partitions: the sizes of the parameter tensors of the architectures the workloads
+# stand for, in definition order; each tensor is one "layer" of the layer-wise method.
+# --------------------------------------------------------------------------------------
+def _offsets_from_sizes(sizes):
+    out = [0]
+    for s in sizes:
+        out.append(out[-1] + int(s))
+    return out
+
+
+def _vit_b16_sizes():
+    d, mlp, patch, tokens, classes = 768, 3072, 16, 197, 1000
+    s = [d, tokens * d, d * 3 * patch * patch, d]                # class token, positions, patch embedding
+    for _ in range(12):
+        s += [d, d, 3 * d * d, 3 * d, d * d, d, d, d, mlp * d, mlp, d * mlp, d]
+    s += [d, d, d * classes, classes]
+    return s
+
+
+def _decoder_1p3b_sizes():
+    d, ffn, vocab, positions = 2048, 8192, 50272, 2050
+    s = [vocab * d, positions * d]
+    for _ in range(24):
+        s += [d * d, d] * 4 + [d, d, ffn * d, ffn, d * ffn, d, d, d]
+    s += [d, d]
+    return s
+
+
+def _resnet18_sizes():
+    # 3x3 stem, four stages of two basic blocks, 10 classes
+    s = [64 * 3 * 9, 64, 64]
+    cin = 64
+    for cout, stride in ((64, 1), (128, 2), (256, 2), (512, 2)):
+        for b in range(2):
+            s += [cout * cin * 9, cout, cout, cout * cout * 9, cout, cout]
+            if b == 0 and (stride != 1 or cin != cout):
+                s += [cout * cin, cout, cout]
+            cin = cout
+    s += [512 * 10, 10]
+    return s
+
+
+def _resnet50_sizes():
+    # 7x7 stem, bottleneck stages of 3, 4, 6, 3 blocks, 1000 classes
+    s = [64 * 3 * 49, 64, 64]
+    cin = 64
+    for width, blocks in ((64, 3), (128, 4), (256, 6), (512, 3)):
+        cout = 4 * width
+        for b in range(blocks):
+            s += [width * cin, width, width, width * width * 9, width, width, cout * width, cout, cout]
+            if b == 0:
+                s += [cout * cin, cout, cout]
+            cin = cout
+    s += [2048 * 1000, 1000]
+    return s
+
+
+_LAYER_SIZES = {"vitb16": _vit_b16_sizes, "decoder1p3b": _decoder_1p3b_sizes,
+                "resnet18": _resnet18_sizes, "resnet50": _resnet50_sizes}
+
+
+def layer_offsets(name, D=None):
+    """L+1 row offsets of the layers of workload `name`.  With D given and different from the
+    workload's size (a cut-down run), the partition is cut at D (or its last layer extended)."""
+    if name in _LAYER_SIZES:
+        off = _offsets_from_sizes(_LAYER_SIZES[name]())
+    else:
+        total = WORKLOADS[name].D
+        off = _offsets_from_sizes([total // 8] * 7 + [total - 7 * (total // 8)])
+    if D is not None and D != off[-1]:
+        off = [o for o in off if o < D] + [D]
+    return off
