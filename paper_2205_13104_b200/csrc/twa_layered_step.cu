@@ -61,6 +61,17 @@ __device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src, int sr
 __device__ __forceinline__ void cp_async_16_zfill(uint32_t dst, const void* src, int src_bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
+// Untiled bulk copy global -> shared, completion counted in bytes on an mbarrier; both addresses
+// 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, unsigned bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+// More bytes to expect on the barrier's current phase, without an arrival.
+__device__ __forceinline__ void twa_mbar_expect_tx_only(uint32_t bar, unsigned bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
@@ -139,31 +150,51 @@ __device__ __forceinline__ void helper_loop(twa_smem_header* hdr, unsigned char*
     const uint32_t aux = twa_smem_u32(ring + static_cast<size_t>(s) * stage_bytes + aux_off);
     if (lane < GPT) cp_async_16(aux + lane * 16, entries_of(k));
     if (src) {
-      // The tile's rows in 16-byte pieces, one per lane and pass.  A granule whose first row sits
-      // on a 16-byte boundary of src (every granule, when the layers' sizes are multiples of 8)
-      // is copied 16 bytes at a time; any other granule 4 bytes at a time.
+      // Lane q looks after granule q.  A granule whose rows start on a 16-byte boundary of src and
+      // fill a multiple of 16 bytes (every granule, when the layers' sizes are multiples of 8 rows)
+      // goes as one bulk copy counted in bytes on the stage's barrier.
+      const uint32_t fb = twa_smem_u32(&hdr->full[s]);
+      bool settled = true;
+      if (lane < GPT) {
+        const int4 e = ep[lane];
+        if (e.x >= 0) {
+          const char* from = sbytes + static_cast<long long>(e.z) * ES;
+          const unsigned bytes = static_cast<unsigned>(e.y) * ES;
+          if (((reinterpret_cast<uintptr_t>(from) | bytes) & 15) == 0) {
+            twa_mbar_expect_tx_only(fb, bytes);
+            bulk_copy_g2s(aux + GPT * 16 + lane * SEG, from, bytes, fb);
+          } else {
+            settled = false;
+          }
+        }
+      }
+      const unsigned todo = ~__ballot_sync(0xFFFFFFFFu, settled);
+      if (todo) {
+        // The other granules in 16-byte pieces, one per lane and pass: 16 bytes at a time where
+        // the granule starts on a 16-byte boundary, else 4 bytes at a time.
+#pragma unroll 1
+        for (int i = 0; i < TQ / 32; ++i) {
+          const int x = i * 32 + lane, q = x / QW, j = x % QW;
+          if (!((todo >> q) & 1u)) continue;
+          const int4 e = ep[q];
+          const long long gbyte = static_cast<long long>(e.z) * ES;            // the granule's first row in src
+          const uint32_t seg = aux + GPT * 16 + q * SEG;
+          if (((reinterpret_cast<uintptr_t>(sbytes) + gbyte) & 15) == 0) {
+            const int nbytes = e.y * ES - j * 16;                              // bytes of existing rows from here on
+            if (nbytes > 0) cp_async_16_zfill(seg + j * 16, sbytes + gbyte + j * 16, nbytes < 16 ? nbytes : 16);
+          } else {
+            const long long byte0 = gbyte & ~3LL;                              // word holding the first row
+            const int shift = ES == 2 ? (e.z & 1) : 0;
 #pragma unroll
-      for (int i = 0; i < TQ / 32; ++i) {
-        const int x = i * 32 + lane, q = x / QW, j = x % QW;
-        const int4 e = ep[q];
-        if (e.x < 0) continue;
-        const long long gbyte = static_cast<long long>(e.z) * ES;            // the granule's first row in src
-        const uint32_t seg = aux + GPT * 16 + q * SEG;
-        if ((gbyte & 15) == 0) {
-          const int nbytes = e.y * ES - j * 16;                                // bytes of existing rows from here on
-          if (nbytes > 0) cp_async_16_zfill(seg + j * 16, sbytes + gbyte + j * 16, nbytes < 16 ? nbytes : 16);
-        } else {
-          const long long byte0 = gbyte & ~3LL;                                // word holding the first row
-          const int shift = ES == 2 ? (e.z & 1) : 0;
-#pragma unroll
-          for (int t = 0; t < (ES == 2 ? 5 : 4); ++t) {
-            if (t == 4 && j != QW - 1) continue;                               // the one word past a shifted granule
-            const int w = 4 * j + t;
-            const int first = ES == 2 ? 2 * w - shift : w;                     // first row the word holds
-            if (first < e.y) {
-              const long long off = byte0 + 4LL * w;
-              const long long rem = total_bytes - off;
-              cp_async_4(seg + 4 * w, sbytes + off, rem >= 4 ? 4 : static_cast<int>(rem));
+            for (int t = 0; t < (ES == 2 ? 5 : 4); ++t) {
+              if (t == 4 && j != QW - 1) continue;                             // the one word past a shifted granule
+              const int w = 4 * j + t;
+              const int first = ES == 2 ? 2 * w - shift : w;                   // first row the word holds
+              if (first < e.y) {
+                const long long off = byte0 + 4LL * w;
+                const long long rem = total_bytes - off;
+                cp_async_4(seg + 4 * w, sbytes + off, rem >= 4 ? 4 : static_cast<int>(rem));
+              }
             }
           }
         }
@@ -181,6 +212,11 @@ __device__ __forceinline__ void helper_loop(twa_smem_header* hdr, unsigned char*
     }
   }
   cp_async_wait_group<0>();                            // nothing of this warp is in flight when it leaves
+  if (*abort_flag) {                                   // a wait ran out: give the bulk copies issued so far time to land
+    const unsigned long long t0 = twa_globaltimer();
+    while (twa_globaltimer() - t0 < 200000ull) {
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
