@@ -294,3 +294,96 @@ def test_workload_decoder_chunked_build_sampled(env):
     seg = 512
     check_step_sampled(ctx, ws, wl, Pq, wbar, bits, col_blocks=[24],
                        row_ranges=[(0, 2 * seg), ((D // 2 // seg) * seg, 2 * seg), (D - seg, seg)])
+
+
+# ------------------------------------------------------------------ the layer-wise construction, full size
+def _unpack_rows(packed, r0, r1, bits):
+    """Unsigned codes of flat rows r0..r1-1 (r0 even) from the canonical export, shape (rows, n)."""
+    if bits == 8:
+        return np.asfortranarray(packed[:, r0:r1].cpu().numpy().T)
+    b = packed[:, r0 // 2:(r1 + 1) // 2].cpu().numpy()
+    inter = np.empty((b.shape[0], 2 * b.shape[1]), dtype=np.uint8)
+    inter[:, 0::2], inter[:, 1::2] = b & 0xF, b >> 4
+    return np.asfortranarray(inter[:, :r1 - r0].T)
+
+
+@pytest.mark.parametrize("name,bits_list", [("resnet50", (8,)), ("vitb16", (8, 4))])
+def test_workload_layerwise_sampled(env, name, bits_list):
+    """The paper's default construction on the workload's own layer partition: per-layer factors
+    and sampled codes bit-exact, one layer-wise step checked on sampled layers, columns and rows."""
+    ctx, _ = env
+    wl = inputs.WORKLOADS[name]
+    D, n = wl.D, wl.n
+    layers = inputs.layer_offsets(name)
+    L = len(layers) - 1
+    sizes = np.diff(layers)
+    W = wl.candidates(DEV)
+    wbar = torch.empty(D, device=DEV)
+    lws = twa.new_layered_workspace(layers, n, DEV)
+    P32 = twa.twa_build_centered(ctx, W, D, layers, wbar, lws)
+    status_ok(ctx)
+    # every column of every layer has unit norm (sampled layers: smallest, largest, first, last)
+    pick = sorted({0, L - 1, int(np.argmin(sizes)), int(np.argmax(sizes)), L // 2})
+    for l in pick:
+        blk = W[:, layers[l]:layers[l + 1]].double()
+        assert torch.max(torch.abs((blk * blk).sum(dim=1) - 1.0)).item() <= TOL
+    g = wl.gradient(0, DEV)
+    g_host = g.float().cpu().numpy().astype(np.float64)
+    for bits in bits_list:
+        lb = twa.twa_quantize_affine(ctx, P32, layers, bits, lws)
+        status_ok(ctx)
+        packed, a_g, b_g = twa.twa_layered_export(ctx, lb)
+        a_h, b_h = a_g.cpu().numpy(), b_g.cpu().numpy()
+        cols = [0, n // 2, n - 1]
+        for l in pick:
+            r0, r1 = layers[l], layers[l + 1]
+            blk = np.asfortranarray(W[:, r0:r1].cpu().numpy().T)
+            a_o, b_o = orc.affine_factors(blk, [0, r1 - r0], bits)
+            assert (a_h[l], b_h[l]) == (a_o[0], b_o[0])
+            codes_o = orc.affine_encode(np.asfortranarray(blk[:, cols]), [0, r1 - r0], a_o, b_o, bits)
+            lo = r0 - (r0 % 2)
+            got = _unpack_rows(packed, lo, r1, bits)[r0 - lo:, :]
+            np.testing.assert_array_equal(got[:, cols], codes_o)
+        # one step from beta = 0
+        sws = twa.new_layered_step_workspace(lb)
+        beta = torch.zeros((L, n), device=DEV)
+        c = torch.empty((L, n), device=DEV)
+        w = torch.empty(D, device=DEV)
+        twa.twa_layered_step(ctx, lb, g, LR, 0.0, beta, wbar, w, sws, c_out=c)
+        status_ok(ctx)
+        c_h, beta_h = c.cpu().numpy(), beta.cpu().numpy()
+        np.testing.assert_allclose(beta_h, -LR * c_h.astype(np.float64), rtol=1e-6, atol=1e-30)
+        for l in pick:
+            r0, r1 = layers[l], layers[l + 1]
+            lo = r0 - (r0 % 2)
+            codes = _unpack_rows(packed, lo, r1, bits)[r0 - lo:, :][:, cols]
+            c_o = orc.project_layerwise(codes, [0, r1 - r0], a_h[l:l + 1], b_h[l:l + 1], g_host[r0:r1])
+            scale = abs(float(a_h[l])) * (codes.astype(np.float64).T @ np.abs(g_host[r0:r1])) \
+                + abs(float(b_h[l])) * np.abs(g_host[r0:r1]).sum()
+            assert np.all(np.abs(c_h[l, cols] - c_o[0]) <= 2e-6 * scale + 1e-30)
+        # rows of the lifted weights inside each sampled layer (its first, a middle and its last rows):
+        # with the base point, then the lift alone, whose bound is not carried by w_bar
+        for base in (wbar, None):
+            if base is None:
+                twa.twa_layered_lift(ctx, lb, beta, None, w, sws)
+                status_ok(ctx)
+            for l in pick:
+                r0, r1 = layers[l], layers[l + 1]
+                span = min(r1 - r0, 3001)
+                for s0 in sorted({r0, r0 + (r1 - r0 - span) // 2, r1 - span}):
+                    lo = s0 - (s0 % 2)
+                    rows_codes = _unpack_rows(packed, lo, s0 + span, bits)[s0 - lo:, :]
+                    w_o = orc.lift_layerwise(rows_codes, [0, span], a_h[l:l + 1], b_h[l:l + 1], beta_h[l:l + 1],
+                                             None if base is None else base[s0:s0 + span].cpu().numpy())
+                    assert rel(w[s0:s0 + span].cpu().numpy(), w_o) <= TOL
+        # all layers at once, cheaply: sum_l c[l, i] equals the flat projection of column i
+        i = n // 2
+        col = _unpack_rows(packed, 0, D, bits)[:, i].astype(np.float64) if D <= 30_000_000 else None
+        if col is not None:
+            total = 0.0
+            for l in range(L):
+                r0, r1 = layers[l], layers[l + 1]
+                total += float(a_h[l]) * np.dot(col[r0:r1], g_host[r0:r1]) + float(b_h[l]) * g_host[r0:r1].sum()
+            assert abs(c_h[:, i].astype(np.float64).sum() - total) <= 1e-5 * np.abs(c_h[:, i]).sum()
+        del lb, packed, sws
+        torch.cuda.empty_cache()
