@@ -217,6 +217,20 @@ def project(codes, scales, g):
     return c
 
 
+def project_batch(codes, scales, G):
+    """Coefficient gradients of several gradient vectors at once: column b of the
+    result is P~^T g_b (Section 4.2, the chain-rule equation, applied to each
+    column of G).  G has shape (D, B); returns (n, B) in float64."""
+    codes = np.asarray(codes)
+    G64 = np.asarray(G).astype(np.float64)
+    n, B = codes.shape[1], G64.shape[1]
+    C = np.zeros((n, B), dtype=np.float64)
+    for b in range(B):
+        for j in range(n):
+            C[j, b] = np.float64(scales[j]) * np.dot(codes[:, j].astype(np.float64), G64[:, b])
+    return C
+
+
 def project_f32(P32, g):
     """c = P^T g for an unquantised float32 basis, in float64."""
     P32 = np.asarray(P32)

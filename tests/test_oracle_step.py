@@ -118,3 +118,27 @@ def test_step_f32_matches_quantised_step_up_to_quantisation_error():
     a2, w2, c2 = orc.step(codes, s, g, np.zeros(n), np.zeros(D, dtype=np.float32), 0.1)
     assert np.linalg.norm(c1 - c2) <= 0.05 * np.linalg.norm(c1)
     assert np.linalg.norm(w1 - w2) <= 0.1 * np.linalg.norm(w1)
+
+
+# ------------------------------------------------------------------ several gradients at once
+def test_project_batch_brute_force_and_dense_product():
+    # integers small enough for exact float64 arithmetic: a hand-computed 3 x 2 x 2 case
+    codes = np.array([[1, -2], [3, 0], [-1, 4]], dtype=np.int8)
+    s = np.array([0.5, 2.0], dtype=np.float32)
+    G = np.array([[2.0, -1.0], [1.0, 0.0], [4.0, 3.0]], dtype=np.float32)
+    # column 0: 0.5*(2+3-4)=0.5 ; 2*(-4+0+16)=24     column 1: 0.5*(-1+0-3)=-2 ; 2*(2+0+12)=28
+    np.testing.assert_array_equal(orc.project_batch(codes, s, G), [[0.5, -2.0], [24.0, 28.0]])
+    rng = np.random.default_rng(3)
+    codes = rng.integers(-127, 128, size=(500, 7)).astype(np.int8)
+    s = rng.random(7).astype(np.float32)
+    G = rng.standard_normal((500, 5)).astype(np.float32)
+    dense = (codes.astype(np.float64) * s.astype(np.float64)).T @ G.astype(np.float64)
+    np.testing.assert_allclose(orc.project_batch(codes, s, G), dense, rtol=1e-12, atol=1e-12)
+    # the projection of a sum of gradients is the sum of the columns (why accumulation needs no batch)
+    np.testing.assert_allclose(orc.project(codes, s, G.astype(np.float64).sum(axis=1)),
+                               orc.project_batch(codes, s, G).sum(axis=1), rtol=1e-11, atol=1e-11)
+    # a transposed operand or a dropped scale fails: column b of G only meets column b of the result
+    G2 = G.copy()
+    G2[:, 3] = 0
+    out = orc.project_batch(codes, s, G2)
+    assert np.all(out[:, 3] == 0) and np.all(out[:, [0, 1, 2, 4]] == orc.project_batch(codes, s, G)[:, [0, 1, 2, 4]])
