@@ -520,6 +520,80 @@ def run_layered(args):
         dist.destroy_process_group()
 
 
+def run_project_batch(args):
+    """Projection of --project-batch gradients per call (P~ read once per group) beside the same
+    number of single-gradient calls, on the workload's column shape; D may be cut with --rows."""
+    import dataclasses
+    import torch
+    from paper_2205_13104_b200 import inputs, twa
+
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    twa.load()
+    wl = inputs.WORKLOADS[args.workload]
+    if args.rows:
+        wl = dataclasses.replace(wl, name=f"{wl.name}[rows={args.rows}]", D=args.rows)
+    D, n, bits, B = wl.D, wl.n, args.bits, args.project_batch
+    gdt = torch.bfloat16 if wl.g_dtype == "bf16" else torch.float32
+    g_bytes = 2 if wl.g_dtype == "bf16" else 4
+    ctx = twa.twa_create(0)
+    ws = twa.new_workspace(dev)
+    # the projection does the same work on any values: codes of a random matrix
+    if 4 * n * D > 120e9:
+        raise SystemExit("the float32 matrix to quantise does not fit: cut D with --rows")
+    W = torch.randn((n, inputs.padded_ld(D, 128)), device=dev) / (D ** 0.5)
+    Pq = twa.twa_quantize_basis(ctx, twa.basis_from_tensor(W, D), bits, ws)
+    del W
+    torch.cuda.empty_cache()
+    ld = inputs.padded_ld(D, 8)
+    G = torch.empty((B, ld), dtype=gdt, device=dev)
+    for b in range(B):
+        G[b, :D] = wl.gradient(b, dev)
+    C = torch.empty((B, n), dtype=torch.float32, device=dev)
+    c1 = torch.empty(n, dtype=torch.float32, device=dev)
+
+    def timed(fn):
+        for _ in range(args.warmup):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+
+    def singles():
+        for b in range(B):
+            twa.twa_project(ctx, Pq, G[b, :D], c1, ws)
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    batch_ms = timed(lambda: twa.twa_project_batch(ctx, Pq, G, C, ws))
+    clocks = sampler.stop()
+    single_ms = timed(singles)
+    code, detail = twa.twa_get_status(ctx)
+    if code != 0:
+        raise RuntimeError(f"projection failed: {twa.twa_strerror(code)} {detail}")
+    group = twa.twa_project_batch_group(ctx, Pq, gdt)
+    p_bytes = n * ((D * bits + 7) // 8)
+    moved = -(-B // group) * p_bytes + B * D * g_bytes
+    peak, peak_kind = load_peaks()
+    print(json.dumps({
+        "metric": f"twa_project_batch_gradients_per_s_int{bits}", "value": B / (batch_ms * 1e-3), "unit": "gradients/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": batch_ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{wl.name}: D={D} n={n} int{bits} P, {wl.g_dtype} g, {B} gradients per call, "
+                               f"groups of {group}", "l2": f"inputs larger than L2: P~ is {p_bytes / 1e6:.0f} MB"},
+        "single_calls_ms": single_ms, "speedup_over_single_calls": single_ms / batch_ms,
+        "roofline": {"bound": "hbm", "kernel": "twa_project_batch_kernel", "achieved": moved / (batch_ms * 1e-3) / 1e9,
+                     "peak": peak, "unit": "GB/s", "frac": moved / (batch_ms * 1e-3) / 1e9 / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None, "bytes_per_launch": moved // -(-B // group)},
+        "cpu_baseline": None, "gpu_launches": -(-B // group) * args.steps, "clocks": clocks}))
+    twa.twa_destroy(ctx)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -539,8 +613,12 @@ def main():
                     help="profiling aid: quantise a random matrix instead of building the basis")
     ap.add_argument("--layered", action="store_true",
                     help="the layer-wise construction with per-layer affine codes instead of the default workload")
+    ap.add_argument("--project-batch", type=int, default=0,
+                    help="time the projection of this many gradients per call instead of the fused step")
     args = ap.parse_args()
-    if args.layered and args.impl == "ours":
+    if args.project_batch and args.impl == "ours":
+        run_project_batch(args)
+    elif args.layered and args.impl == "ours":
         run_layered(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -224,6 +224,18 @@ int twa_basis_import(twa_ctx* ctx, const void* codes, const float* scales, int64
 int twa_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
                 float* c_out, void* ws, size_t ws_bytes);
 
+/* The projection for `batch` gradients at once (Section 4.2's chain-rule equation for every row of
+ * G): C_out[b*n + j] = s_j * sum_r code[r,j] * G[b*ldg + r].  P~ is read once per group of
+ * twa_project_batch_group(ctx, P, g_dtype) gradients (8 when three stages of that shape fit in shared
+ * memory, else 4; 1 for a float32 basis, which is projected gradient by gradient),
+ * two gradients sharing every integer MMA.
+ *  G      in: batch rows of ldg elements of g_dtype, ldg >= D; G and ldg*sizeof(element) 16-byte
+ *         aligned.   C_out  out: batch x n floats.
+ * Device-side errors: TWA_ERR_NONFINITE (detail = index of the gradient), TWA_ERR_TIMEOUT. */
+int twa_project_batch(twa_ctx* ctx, const twa_basis* P, const void* G, int64_t ldg, int batch,
+                      twa_dtype g_dtype, float* C_out, void* ws, size_t ws_bytes);
+int twa_project_batch_group(twa_ctx* ctx, const twa_basis* P, twa_dtype g_dtype);
+
 /* w_out[r] = base[r] + sum_j (s_j * alpha[j]) * code[r,j].
  *  alpha  in: n floats.   base  in: D floats, or NULL for 0.
  *  w_out  out: D floats; may be the same buffer as base, must not overlap P. */

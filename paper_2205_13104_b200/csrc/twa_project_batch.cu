@@ -1,0 +1,461 @@
+// Projection of several gradients at once: C[b][j] = s_j * sum_r code[r,j] * G[b][r]
+// (Section 4.2, the chain-rule equation, for every row of G), P~ read once per group of gradients.
+//
+// Same data path as the single-gradient kernel in twa_stream_mma.cu.  What the batch adds: the
+// m16n8k32 integer MMA has eight result columns and one gradient's four base-128 digits fill only
+// four of them, so two gradients share every MMA (columns 0-3: digits of the first, 4-7: digits of
+// the second).  A tile of P~ in shared memory serves NP such pairs before its stage is released;
+// the gradients of a group arrive as [NB][256] boxes of one 2-D tensor map over G (rows past the
+// batch read as zero).
+#include <stdio.h>
+
+#include "twa_mma.cuh"
+
+namespace {
+
+constexpr int PAIR_SCRATCH = 512;               // digit bytes per warp: two gradients x (even, odd rows) x [4][32]
+
+struct BatchArgs {
+  long long D;
+  int n, stages, tiles, b0, batch;
+  unsigned stage_bytes, g_off, tx_bytes, scratch_off;
+  const float* scales;
+  float* partials;              // [grid][NB][n]
+  unsigned* ticket;
+  int* status;
+  float* c_out;                 // [batch][n]
+  unsigned long long wait_limit_ns;
+};
+
+template <int KT, int NB>
+__device__ __forceinline__ void producer_loop_batch(twa_smem_header* hdr, unsigned char* ring,
+                                                    const CUtensorMap* map_p, const CUtensorMap* map_g,
+                                                    const BatchArgs& a, int tile_rows, int g_elem_bytes) {
+  twa_prefetch_tensormap(map_p);
+  twa_prefetch_tensormap(map_g);
+  volatile int* abort_flag = &hdr->abort_flag;
+  int s = 0, issued = 0;
+  unsigned phase = 0;
+  bool ok = true;
+  for (int tile = blockIdx.x; tile < a.tiles; tile += gridDim.x) {
+    if (issued >= a.stages) {
+      if (!twa_mbar_wait(twa_smem_u32(&hdr->empty[s]), phase, abort_flag, a.wait_limit_ns)) {
+        ok = false;
+        break;
+      }
+    }
+    const uint32_t fb = twa_smem_u32(&hdr->full[s]);
+    const uint32_t dst = twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes);
+    twa_mbar_expect_tx(fb, a.tx_bytes);
+    twa_tma_load_2d(dst, map_p, tile * TWA_TILE_COL_WORDS * KT, 0, fb);
+    for (int q = 0; q < tile_rows / 256; ++q)
+      twa_tma_load_2d(dst + a.g_off + q * NB * 256 * g_elem_bytes, map_g, tile * tile_rows + q * 256, a.b0, fb);
+    ++issued;
+    if (++s == a.stages) {
+      s = 0;
+      if (issued > a.stages) phase ^= 1u;
+    }
+  }
+  if (!ok) {
+    twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+    const int live = issued < a.stages ? issued : a.stages;
+    for (int q = 0; q < live; ++q) {      // let the copies already issued land
+      const int last = ((issued - 1 - q) / a.stages) * a.stages + q;
+      const unsigned par = static_cast<unsigned>(last / a.stages) & 1u;
+      const unsigned long long t0 = twa_globaltimer();
+      while (!twa_mbar_try_wait(twa_smem_u32(&hdr->full[q]), par)) {
+        if (twa_globaltimer() - t0 > a.wait_limit_ns) break;
+      }
+    }
+  }
+}
+
+// NP pairs of gradients per launch (NB = 2 NP); MT, KT as in the single-gradient kernel.
+template <int BITS, bool GBF16, int MT, int KT, int NP>
+__global__ void __launch_bounds__(MMA_THREADS, 1)
+twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_g,
+                         const BatchArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
+  constexpr int NB = 2 * NP;
+  constexpr int SROWS = twa_tile_rows(BITS);           // rows behind one 512-byte segment
+  constexpr int GSZ = GBF16 ? 2 : 4;
+  twa_smem_header* hdr = reinterpret_cast<twa_smem_header*>(smem);
+  unsigned char* ring = smem + TWA_SMEM_HEADER;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gid = lane >> 2, tig = lane & 3;
+
+  init_barriers(hdr, a.stages);
+  __syncthreads();
+
+  float facc[NP][MT][2];
+#pragma unroll
+  for (int p = 0; p < NP; ++p)
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) facc[p][mt][0] = facc[p][mt][1] = 0.0f;
+
+  if (warp == MMA_WARPS) {
+    if (lane == 0) producer_loop_batch<KT, NB>(hdr, ring, &map_p, &map_g, a, SROWS * KT, GSZ);
+  } else {
+    unsigned char* digw = smem + a.scratch_off + warp * PAIR_SCRATCH;
+    const int lm = lane >> 3, lr = lane & 7;
+    const int jmax = a.n - 1;
+    constexpr int col_bytes = TWA_TILE_COL_BYTES * KT;
+    uint32_t aoff[KT][MT];
+#pragma unroll
+    for (int u = 0; u < KT; ++u)
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        int j = mt * 16 + lr + 8 * (lm & 1);
+        j = j < jmax ? j : jmax;
+        const int chunk = (warp * KT + u) * 2 + (lm >> 1);
+        aoff[u][mt] = static_cast<uint32_t>(j * col_bytes + ((chunk >> 5) << 9) + (twa_chunk_slot(chunk & 31, j) << 4));
+      }
+    // element offsets, inside one gradient's [256] slices of the stage, of this lane's rows for block u:
+    // row r of the tile lives in box r / 256 at position r % 256
+    int goff[KT];
+#pragma unroll
+    for (int u = 0; u < KT; ++u) {
+      const int r = (warp * KT + u) * (SROWS / MMA_WARPS) + (BITS == 8 ? lane : 2 * lane);
+      goff[u] = (r >> 8) * NB * 256 + (r & 255);
+    }
+    volatile int* abort_flag = &hdr->abort_flag;
+    int s = 0;
+    unsigned phase = 0;
+    unsigned bad = 0u;                                   // bit b: gradient b of the group is not finite
+    for (int t = blockIdx.x; t < a.tiles; t += gridDim.x) {
+      if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
+        twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+        break;
+      }
+      const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
+      const uint32_t tile_base = twa_smem_u32(st);
+#pragma unroll
+      for (int p = 0; p < NP; ++p) {
+        // ---- the warp's rows of the pair's two gradients ---------------------------------------
+        float g0[2][KT], g1[2][KT];
+        unsigned mb[2] = {0u, 0u};
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int u = 0; u < KT; ++u) {
+            const int e = goff[u] + (2 * p + h) * 256;
+            g1[h][u] = 0.0f;
+            if (GBF16) {
+              const unsigned short* gs = reinterpret_cast<const unsigned short*>(st + a.g_off);
+              g0[h][u] = __uint_as_float(static_cast<uint32_t>(gs[e]) << 16);
+              if (BITS == 4) g1[h][u] = __uint_as_float(static_cast<uint32_t>(gs[e + 1]) << 16);
+            } else {
+              const float* gs = reinterpret_cast<const float*>(st + a.g_off);
+              g0[h][u] = gs[e];
+              if (BITS == 4) g1[h][u] = gs[e + 1];
+            }
+            mb[h] = max(mb[h], max(__float_as_uint(g0[h][u]) & 0x7FFFFFFFu, __float_as_uint(g1[h][u]) & 0x7FFFFFFFu));
+          }
+        mb[0] = __reduce_max_sync(0xFFFFFFFFu, mb[0]);
+        mb[1] = __reduce_max_sync(0xFFFFFFFFu, mb[1]);
+        const unsigned eb0 = mb[0] >> 23, eb1 = mb[1] >> 23;
+        if (eb0 >= 255u) bad |= 1u << (2 * p);
+        if (eb1 >= 255u) bad |= 1u << (2 * p + 1);
+        const bool live0 = eb0 >= 5u && eb0 < 255u, live1 = eb1 >= 5u && eb1 < 255u;
+        if (!live0 && !live1) continue;                  // nothing representable in either gradient here
+        const float up0 = live0 ? __uint_as_float((259u - eb0) << 23) : 0.0f;
+        const float up1 = live1 ? __uint_as_float((259u - eb1) << 23) : 0.0f;
+        // lanes tig 0,1 finish the first gradient's digits, tig 2,3 the second's
+        const unsigned ebm = (tig < 2) ? eb0 : eb1;
+        const bool livem = (tig < 2) ? live0 : live1;
+        const float w0 = !livem ? 0.0f : (ebm >= 6u ? __uint_as_float((ebm - 5u) << 23) : 5.877471754e-39f);
+        const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
+        float wa = (tig & 1) == 0 ? w0 : w2;
+        float wb = (tig & 1) == 0 ? w1 : w3;
+        if (BITS == 4) { wa *= 0.0625f; wb *= 0.0625f; }
+        int c[MT][4];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) c[mt][0] = c[mt][1] = c[mt][2] = c[mt][3] = 0;
+#pragma unroll
+        for (int u = 0; u < KT; ++u) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const bool lv = h ? live1 : live0;            // a dead or non-finite gradient contributes zero digits
+            const uint32_t d0 = cut_digits(lv ? g0[h][u] * (h ? up1 : up0) : 0.0f);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) digw[h * 256 + k * 32 + lane] = static_cast<unsigned char>(d0 >> (8 * k));
+            if (BITS == 4) {
+              const uint32_t d1 = cut_digits(lv ? g1[h][u] * (h ? up1 : up0) : 0.0f);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) digw[h * 256 + 128 + k * 32 + lane] = static_cast<unsigned char>(d1 >> (8 * k));
+            }
+          }
+          __syncwarp();
+          // B fragment: result column gid = digit gid of the first gradient (gid < 4) or digit gid - 4 of the second
+          const unsigned char* dg = digw + (gid >> 2) * 256 + (gid & 3) * 32 + 4 * tig;
+          const uint32_t b0 = *reinterpret_cast<const uint32_t*>(dg);
+          const uint32_t b1 = *reinterpret_cast<const uint32_t*>(dg + 16);
+          uint32_t b2 = 0, b3 = 0;
+          if (BITS == 4) {
+            b2 = *reinterpret_cast<const uint32_t*>(dg + 128);
+            b3 = *reinterpret_cast<const uint32_t*>(dg + 128 + 16);
+          }
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            uint32_t r[4];
+            ldmatrix_x4(tile_base + aoff[u][mt], r);
+            if (BITS == 8) {
+              mma_s8(c[mt], r, b0, b1);
+            } else {
+              uint32_t e[4], o[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                e[i] = (r[i] << 4) & 0xF0F0F0F0u;         // even rows: 16 * code
+                o[i] = r[i] & 0xF0F0F0F0u;                // odd rows:  16 * code
+              }
+              mma_s8(c[mt], e, b0, b1);
+              mma_s8(c[mt], o, b2, b3);
+            }
+          }
+          __syncwarp();                                  // the digit scratch is rewritten next
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          facc[p][mt][0] = fmaf(small_int_to_float(c[mt][0]), wa, facc[p][mt][0]);
+          facc[p][mt][0] = fmaf(small_int_to_float(c[mt][1]), wb, facc[p][mt][0]);
+          facc[p][mt][1] = fmaf(small_int_to_float(c[mt][2]), wa, facc[p][mt][1]);
+          facc[p][mt][1] = fmaf(small_int_to_float(c[mt][3]), wb, facc[p][mt][1]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
+      if (++s == a.stages) {
+        s = 0;
+        phase ^= 1u;
+      }
+    }
+    if (bad) atomicOr(&hdr->bad_flag, static_cast<int>(bad));
+  }
+  __syncthreads();                                       // every stage consumed; the ring is free
+
+  // ---- sums of the block: lanes -> warps -> block, in a fixed order --------------------------
+  float* part = reinterpret_cast<float*>(ring);         // [MMA_WARPS][NB][TWA_MAX_N]
+  if (warp < MMA_WARPS) {
+#pragma unroll
+    for (int p = 0; p < NP; ++p)
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        float v0 = facc[p][mt][0], v1 = facc[p][mt][1];
+        v0 += __shfl_xor_sync(0xFFFFFFFFu, v0, 1);
+        v1 += __shfl_xor_sync(0xFFFFFFFFu, v1, 1);
+        if ((tig & 1) == 0) {                            // tig 0: first gradient of the pair, tig 2: second
+          float* row = part + (warp * NB + 2 * p + (tig >> 1)) * TWA_MAX_N;
+          row[mt * 16 + gid] = v0;
+          row[mt * 16 + gid + 8] = v1;
+        }
+      }
+  }
+  __syncthreads();
+  const int tid = threadIdx.x;
+  const int outs = NB * a.n;
+  for (int idx = tid; idx < outs; idx += blockDim.x) {
+    const int b = idx / a.n, j = idx - b * a.n;
+    float sum = 0.0f;
+#pragma unroll
+    for (int w = 0; w < MMA_WARPS; ++w) sum += part[(w * NB + b) * TWA_MAX_N + j];
+    if ((hdr->bad_flag >> b) & 1) sum = __int_as_float(0x7FC00000);
+    a.partials[static_cast<size_t>(blockIdx.x) * outs + idx] = sum;
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned ticket = atomicAdd(a.ticket, 1u);
+    hdr->last_flag = (ticket == gridDim.x - 1) ? 1 : 0;
+  }
+  __syncthreads();
+  if (hdr->last_flag) {
+    __threadfence();
+    for (int idx = tid; idx < outs; idx += blockDim.x) {
+      const int b = idx / a.n, j = idx - b * a.n;
+      if (a.b0 + b >= a.batch) continue;
+      double sum = 0.0;
+      for (unsigned k = 0; k < gridDim.x; ++k)
+        sum += static_cast<double>(__ldcg(&a.partials[static_cast<size_t>(k) * outs + idx]));
+      const double c = sum * static_cast<double>(a.scales[j]);
+      if (!isfinite(c)) twa_set_status(a.status, TWA_ERR_NONFINITE, a.b0 + b);
+      a.c_out[static_cast<size_t>(a.b0 + b) * a.n + j] = static_cast<float>(c);
+    }
+    if (tid == 0) *a.ticket = 0u;
+  }
+}
+
+int encode_codes_map(twa_ctx* ctx, const twa_basis* P, int kt, CUtensorMap* map) {
+  long long row_bytes = (P->D * P->bits + 7) / 8;
+  row_bytes = (row_bytes + 511) / 512 * 512;             // whole, internally permuted 512-byte segments
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(row_bytes / 4), static_cast<cuuint64_t>(P->n)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(P->col_stride)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(TWA_TILE_COL_WORDS * kt), static_cast<cuuint32_t>(P->n)};
+  cuuint32_t es[2] = {1, 1};
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, P->data, dims, strides, box, es,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(ctx->last_error, sizeof(ctx->last_error), "cuTensorMapEncodeTiled(P~) failed: %d", static_cast<int>(r));
+    return TWA_ERR_CUDA;
+  }
+  return TWA_OK;
+}
+
+int encode_batch_map(twa_ctx* ctx, const void* G, long long D, long long ldg, int batch, bool bf16, int nb,
+                     CUtensorMap* map) {
+  const int gsz = bf16 ? 2 : 4;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(batch)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldg * gsz)};
+  cuuint32_t box[2] = {256, static_cast<cuuint32_t>(nb)};
+  cuuint32_t es[2] = {1, 1};
+  CUresult r = ctx->encode_tiled(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                                 const_cast<void*>(G), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(ctx->last_error, sizeof(ctx->last_error), "cuTensorMapEncodeTiled(G) failed: %d", static_cast<int>(r));
+    return TWA_ERR_CUDA;
+  }
+  return TWA_OK;
+}
+
+template <int BITS, bool GBF16, int MT, int KT, int NP>
+int launch_one(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg, const BatchArgs& a, int grid, int smem) {
+  auto kern = twa_project_batch_kernel<BITS, GBF16, MT, KT, NP>;
+  static int smem_limit[64] = {0};
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[ctx->device & 63], smem);
+  if (rc) return rc;
+  kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, mg, a);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+// Shapes of a pass: four pairs of gradients when at least three such stages fit in shared memory
+// (with two 512-byte segments per tile column for n <= 64, one for wider bases), else two pairs
+// and one segment.
+template <int BITS, bool GBF16>
+int launch_mt(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg, const BatchArgs& a, int kt, int nb, int grid,
+              int smem) {
+  const int mt = (a.n + 15) >> 4;
+  if (nb == 8 && kt == 2) {
+    switch (mt) {
+      case 1: return launch_one<BITS, GBF16, 1, 2, 4>(ctx, mp, mg, a, grid, smem);
+      case 2: return launch_one<BITS, GBF16, 2, 2, 4>(ctx, mp, mg, a, grid, smem);
+      case 3: return launch_one<BITS, GBF16, 3, 2, 4>(ctx, mp, mg, a, grid, smem);
+      default: return launch_one<BITS, GBF16, 4, 2, 4>(ctx, mp, mg, a, grid, smem);
+    }
+  }
+  if (nb == 8) {
+    switch (mt) {
+      case 5: return launch_one<BITS, GBF16, 5, 1, 4>(ctx, mp, mg, a, grid, smem);
+      case 6: return launch_one<BITS, GBF16, 6, 1, 4>(ctx, mp, mg, a, grid, smem);
+      case 7: return launch_one<BITS, GBF16, 7, 1, 4>(ctx, mp, mg, a, grid, smem);
+      default: return launch_one<BITS, GBF16, 8, 1, 4>(ctx, mp, mg, a, grid, smem);
+    }
+  }
+  switch (mt) {
+    case 1: return launch_one<BITS, GBF16, 1, 1, 2>(ctx, mp, mg, a, grid, smem);
+    case 2: return launch_one<BITS, GBF16, 2, 1, 2>(ctx, mp, mg, a, grid, smem);
+    case 3: return launch_one<BITS, GBF16, 3, 1, 2>(ctx, mp, mg, a, grid, smem);
+    case 4: return launch_one<BITS, GBF16, 4, 1, 2>(ctx, mp, mg, a, grid, smem);
+    case 5: return launch_one<BITS, GBF16, 5, 1, 2>(ctx, mp, mg, a, grid, smem);
+    case 6: return launch_one<BITS, GBF16, 6, 1, 2>(ctx, mp, mg, a, grid, smem);
+    case 7: return launch_one<BITS, GBF16, 7, 1, 2>(ctx, mp, mg, a, grid, smem);
+    default: return launch_one<BITS, GBF16, 8, 1, 2>(ctx, mp, mg, a, grid, smem);
+  }
+}
+
+constexpr int FIXED_SMEM = TWA_SMEM_HEADER + MMA_WARPS * PAIR_SCRATCH + 1024;
+
+unsigned stage_bytes_of(const twa_basis* P, int gsz, int kt, int nb) {
+  const unsigned tx = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt + twa_tile_rows(P->bits) * kt * gsz * nb;
+  return (tx + 1023) / 1024 * 1024;
+}
+
+// (segments per tile column, gradients per pass) for this basis, gradient type and device
+void pass_shape(const twa_ctx* ctx, const twa_basis* P, int gsz, int* kt, int* nb) {
+  const int kt8 = P->n <= 64 ? 2 : 1;
+  const bool fits = (ctx->smem_optin - FIXED_SMEM) / static_cast<int>(stage_bytes_of(P, gsz, kt8, 8)) >= 3;
+  const bool partials_fit = static_cast<size_t>(ctx->sm_count) * 8 * P->n <= static_cast<size_t>(TWA_MAX_GRID) * TWA_MAX_N;
+  if (fits && partials_fit) {
+    *kt = kt8;
+    *nb = 8;
+  } else {
+    *kt = 1;
+    *nb = 4;
+  }
+}
+
+}  // namespace
+
+extern "C" int twa_project_batch_group(twa_ctx* ctx, const twa_basis* P, twa_dtype g_dtype) {
+  if (!ctx || !P || P->bits == 32) return 1;
+  int kt, nb;
+  pass_shape(ctx, P, g_dtype == TWA_BF16 ? 2 : 4, &kt, &nb);
+  return nb;
+}
+
+extern "C" int twa_project_batch(twa_ctx* ctx, const twa_basis* P, const void* G, int64_t ldg, int batch,
+                                 twa_dtype g_dtype, float* C_out, void* ws, size_t ws_bytes) {
+  if (!ctx || !P || !G || !C_out || batch < 1) return TWA_ERR_INVALID_ARG;
+  if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
+  int rc = twa_check_basis(P);
+  if (rc) return rc;
+  if (ldg < P->D) return TWA_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < TWA_WS_BYTES) return TWA_ERR_WORKSPACE;
+  const bool bf16 = g_dtype == TWA_BF16;
+  const int gsz = bf16 ? 2 : 4;
+  if ((reinterpret_cast<uintptr_t>(G) & 15) || ((ldg * gsz) & 15)) return TWA_ERR_MISALIGNED;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  if (P->bits == 32) {
+    // a float32 basis (the build's own format) has no integer path: one projection per gradient
+    for (int b = 0; b < batch; ++b) {
+      rc = twa_project(ctx, P, static_cast<const char*>(G) + static_cast<size_t>(b) * ldg * gsz, g_dtype,
+                       C_out + static_cast<size_t>(b) * P->n, ws, ws_bytes);
+      if (rc) return rc;
+    }
+    return TWA_OK;
+  }
+  int kt, nb;
+  pass_shape(ctx, P, gsz, &kt, &nb);
+  const int rows = twa_tile_rows(P->bits) * kt;
+  CUtensorMap mp, mg;
+  rc = encode_codes_map(ctx, P, kt, &mp);
+  if (rc) return rc;
+  rc = encode_batch_map(ctx, G, P->D, ldg, batch, bf16, nb, &mg);
+  if (rc) return rc;
+  BatchArgs a;
+  a.D = P->D;
+  a.n = P->n;
+  a.tiles = static_cast<int>((P->D + rows - 1) / rows);
+  a.batch = batch;
+  a.g_off = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt;
+  a.tx_bytes = a.g_off + static_cast<unsigned>(rows * gsz * nb);
+  a.stage_bytes = (a.tx_bytes + 1023) / 1024 * 1024;
+  int stages = (ctx->smem_optin - FIXED_SMEM) / static_cast<int>(a.stage_bytes);
+  if (stages > TWA_MAX_STAGES) stages = TWA_MAX_STAGES;
+  if (stages < 2) return TWA_ERR_UNSUPPORTED;
+  // the ring is reused for the block's [16][NB][128] float sums after the tile loop
+  if (static_cast<size_t>(stages) * a.stage_bytes < sizeof(float) * MMA_WARPS * nb * TWA_MAX_N) return TWA_ERR_UNSUPPORTED;
+  a.stages = stages;
+  a.scratch_off = TWA_SMEM_HEADER + static_cast<unsigned>(stages) * a.stage_bytes;
+  a.scales = P->scales;
+  a.partials = reinterpret_cast<float*>(static_cast<char*>(ws) + TWA_WS_PARTIALS);
+  a.ticket = ctx->d_ticket;
+  a.status = ctx->d_status;
+  a.c_out = C_out;
+  a.wait_limit_ns = ctx->wait_limit_ns;
+  int grid = ctx->sm_count < a.tiles ? ctx->sm_count : a.tiles;
+  while (static_cast<size_t>(grid) * nb * P->n > static_cast<size_t>(TWA_MAX_GRID) * TWA_MAX_N) --grid;
+  const int smem = static_cast<int>(a.scratch_off) + MMA_WARPS * PAIR_SCRATCH + 1024;
+  for (int b0 = 0; b0 < batch; b0 += nb) {
+    a.b0 = b0;
+    if (P->bits == 8)
+      rc = bf16 ? launch_mt<8, true>(ctx, mp, mg, a, kt, nb, grid, smem) : launch_mt<8, false>(ctx, mp, mg, a, kt, nb, grid, smem);
+    else
+      rc = bf16 ? launch_mt<4, true>(ctx, mp, mg, a, kt, nb, grid, smem) : launch_mt<4, false>(ctx, mp, mg, a, kt, nb, grid, smem);
+    if (rc) return rc;
+  }
+  return TWA_OK;
+}

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libtwa.so")
 CSRC = os.path.join(_HERE, "csrc")
-SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_chunked.cu", "twa_layered_build.cu", "twa_layered_step.cu", "twa_stream.cu",
+SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_chunked.cu", "twa_layered_build.cu", "twa_layered_step.cu", "twa_project_batch.cu", "twa_stream.cu",
            "twa_stream_mma.cu", "twa_noalloc.cu"]
 
 TWA_MAX_N = 128
@@ -45,7 +45,7 @@ EXPORTS = [
     "twa_workspace_bytes", "twa_build_basis", "twa_build_workspace_bytes", "twa_build_begin",
     "twa_build_feed", "twa_build_end_pass", "twa_mean", "twa_quantize_basis",
     "twa_basis_export", "twa_basis_import", "twa_project", "twa_lift", "twa_step",
-    "twa_step_host", "twa_layered_workspace_bytes", "twa_layered_rows", "twa_layered_basis_bytes",
+    "twa_step_host", "twa_project_batch", "twa_project_batch_group", "twa_layered_workspace_bytes", "twa_layered_rows", "twa_layered_basis_bytes",
     "twa_build_centered", "twa_quantize_affine", "twa_layered_export",
     "twa_layered_step_workspace_bytes", "twa_layered_project", "twa_layered_lift", "twa_layered_step",
     "twa_project_noalloc", "twa_noalloc_last_error", "twa_noalloc_scratch_bytes",
@@ -142,6 +142,8 @@ def load():
         "twa_lift": (i32, [vp, bp, vp, vp, vp, vp, szt]),
         "twa_step": (i32, [vp, bp, vp, i32, f32, f32, vp, vp, vp, vp, vp, szt]),
         "twa_step_host": (i32, [vp, bp, vp, i32, f32, f32, vp, vp, vp, vp, vp, vp, szt]),
+        "twa_project_batch": (i32, [vp, bp, vp, i64, i32, i32, vp, vp, szt]),
+        "twa_project_batch_group": (i32, [vp, bp, i32]),
         "twa_layered_workspace_bytes": (szt, [ctypes.POINTER(ctypes.c_int64), i32, i32]),
         "twa_layered_rows": (i64, [ctypes.POINTER(ctypes.c_int64), i32, i32]),
         "twa_layered_basis_bytes": (szt, [ctypes.POINTER(ctypes.c_int64), i32, i32, i32]),
@@ -394,6 +396,20 @@ def twa_project(ctx, P, g, c_out, ws):
                             _ptr(ws), ws.numel())
     _check(rc, "twa_project", ctx)
     return c_out
+
+
+def twa_project_batch(ctx, P, G, C_out, ws):
+    """G: (batch, ldg) gradients, one per row; C_out: (batch, n) float32."""
+    assert G.dim() == 2 and G.is_contiguous() and C_out.is_contiguous()
+    rc = load().twa_project_batch(ctx, ctypes.byref(P.desc), _ptr(G), int(G.shape[1]), int(G.shape[0]),
+                                  _dtype_code(G), _ptr(C_out), _ptr(ws), ws.numel())
+    _check(rc, "twa_project_batch", ctx)
+    return C_out
+
+
+def twa_project_batch_group(ctx, P, g_dtype=torch.bfloat16):
+    code = _dtype_code(torch.empty(0, dtype=g_dtype))
+    return int(load().twa_project_batch_group(ctx, ctypes.byref(P.desc), code))
 
 
 def twa_lift(ctx, P, alpha, base, w_out, ws):
