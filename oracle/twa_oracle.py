@@ -250,6 +250,46 @@ def sgd_update(alpha, c, lr, lam=0.0):
     return (1.0 - float(lr) * float(lam)) * alpha - float(lr) * c
 
 
+def adam_update(alpha, m, v, c, lr, t, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0):
+    """One Adam step on the coefficients with decoupled weight decay (the base
+    optimiser the paper uses on the coefficients of transformer models, Section 5
+    training details; Adam as published by Kingma & Ba, the decay applied to the
+    variable itself as in AdamW).  t is the 1-based step count.
+        alpha <- (1 - lr*wd) alpha
+        m <- beta1 m + (1-beta1) c ;  v <- beta2 v + (1-beta2) c^2
+        alpha <- alpha - lr * (m / (1-beta1^t)) / (sqrt(v / (1-beta2^t)) + eps)
+    Returns (alpha, m, v) in float64."""
+    alpha = np.asarray(alpha, dtype=np.float64)
+    m = np.asarray(m, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    c = np.asarray(c, dtype=np.float64)
+    alpha = alpha * (1.0 - float(lr) * float(weight_decay))
+    m = float(beta1) * m + (1.0 - float(beta1)) * c
+    v = float(beta2) * v + (1.0 - float(beta2)) * c * c
+    m_hat = m / (1.0 - float(beta1) ** int(t))
+    v_hat = v / (1.0 - float(beta2) ** int(t))
+    alpha = alpha - float(lr) * m_hat / (np.sqrt(v_hat) + float(eps))
+    return alpha, m, v
+
+
+def cosine_lr(base_lr, step, total_steps, min_lr=0.0):
+    """Cosine learning-rate schedule (the schedule of the paper's TWA runs on
+    transformers): base at step 0, min_lr at step total_steps."""
+    x = min(max(float(step) / float(total_steps), 0.0), 1.0)
+    return float(min_lr) + 0.5 * (float(base_lr) - float(min_lr)) * (1.0 + np.cos(np.pi * x))
+
+
+def weighted_average(W, weights):
+    """Fixed-weight average w = sum_i weights_i w_i of the candidates (SWA: equal
+    weights; LAWA: equal weights on the last t; EMA: geometric weights -- the
+    comparison methods of Section 2), in float64."""
+    W = np.asarray(W)
+    out = np.zeros(W.shape[0], dtype=np.float64)
+    for i in range(W.shape[1]):
+        out += np.float64(weights[i]) * W[:, i].astype(np.float64)
+    return out
+
+
 def lift(codes, scales, alpha, base=None):
     """w = base + P~ alpha (Section 4.3: w_twa = w_bar + P beta; Algorithm 1,
     the update of the weights).  base None means 0.
