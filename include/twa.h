@@ -250,6 +250,30 @@ int twa_step(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
              float lambda, float* alpha, const float* wbar, float* w, float* c_out, void* ws,
              size_t ws_bytes);
 
+/* The same iteration with Adam on the coefficients and decoupled weight decay (the base optimiser
+ * of the paper's transformer runs, Section 5; Adam as published by Kingma & Ba):
+ *   m <- beta1 m + (1-beta1) c;  v <- beta2 v + (1-beta2) c^2;
+ *   alpha <- (1 - lr*weight_decay) alpha - lr (m / (1-beta1^step)) / (sqrt(v / (1-beta2^step)) + eps)
+ * `opt` is read on the HOST at call time; `step` is the 1-based count of this update.  m, v: n floats
+ * on the device, zero before the first step, updated in place.  A learning-rate schedule is the
+ * caller's: pass the step's rate in opt->lr (twa_cosine_lr gives the cosine schedule). */
+typedef struct {
+  float lr, beta1, beta2, eps, weight_decay;
+  int32_t step;
+} twa_adam;
+int twa_step_adam(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype, const twa_adam* opt,
+                  float* alpha, float* m, float* v, const float* wbar, float* w, float* c_out, void* ws,
+                  size_t ws_bytes);
+/* Host function: min_lr + (base_lr - min_lr) (1 + cos(pi step/total_steps)) / 2, step clamped to
+ * [0, total_steps]. */
+float twa_cosine_lr(float base_lr, int step, int total_steps, float min_lr);
+
+/* Fixed-weight average of the candidates, w_out = sum_i weights[i] * w_i (Section 2's comparison
+ * methods: SWA = equal weights, LAWA = equal weights on the last t, EMA = geometric weights), one
+ * streaming pass over W.  W, ldw as for twa_build_basis (not modified); weights: n floats, device. */
+int twa_weighted_average(twa_ctx* ctx, const float* W, int64_t D, int n, int64_t ldw, const float* weights,
+                         float* w_out, void* ws, size_t ws_bytes);
+
 /* The same iteration for a caller whose gradient and weights live in HOST memory (pinned
  * memory makes the copies asynchronous): copies g_host (D elements) into the device
  * staging buffer g_stage, runs twa_step into the device buffer w, and copies w back to
@@ -335,6 +359,11 @@ int twa_layered_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* bet
 int twa_layered_step(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype,
                      float lr, float lambda, float* beta, const float* wbar, float* w, float* c_out,
                      void* sws, size_t sws_bytes);
+
+/* The layer-wise step with Adam on every layer's coefficients (m, v: L x n floats, as twa_step_adam). */
+int twa_layered_step_adam(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype,
+                          const twa_adam* opt, float* beta, float* m, float* v, const float* wbar, float* w,
+                          float* c_out, void* sws, size_t sws_bytes);
 
 /* ---- projection without any allocation ----------------------------------------------- */
 

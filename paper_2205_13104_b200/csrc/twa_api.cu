@@ -1,4 +1,5 @@
 // C entry points: context, status, and the per-step calls (project, lift, step).
+#include <math.h>
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
@@ -33,6 +34,21 @@ __global__ void wait_selftest_kernel(int* status, unsigned long long limit_ns) {
   }
 }
 }  // namespace
+
+int twa_adam_device_args(const twa_adam* opt, float* m, float* v, twa_adam_args* out) {
+  if (!opt || !m || !v || !out) return TWA_ERR_INVALID_ARG;
+  if (opt->step < 1 || !(opt->beta1 >= 0.0f && opt->beta1 < 1.0f) || !(opt->beta2 >= 0.0f && opt->beta2 < 1.0f) ||
+      !(opt->eps >= 0.0f))
+    return TWA_ERR_INVALID_ARG;
+  out->m = m;
+  out->v = v;
+  out->beta1 = opt->beta1;
+  out->beta2 = opt->beta2;
+  out->eps = opt->eps;
+  out->bc1 = static_cast<float>(1.0 - pow(static_cast<double>(opt->beta1), opt->step));
+  out->bc2 = static_cast<float>(1.0 - pow(static_cast<double>(opt->beta2), opt->step));
+  return TWA_OK;
+}
 
 extern "C" {
 
@@ -186,8 +202,9 @@ int twa_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, const float* 
   return twa_launch_lift(ctx, P, alpha, 1.0f, base, w_out, false);
 }
 
-int twa_step(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype, float lr, float lambda,
-             float* alpha, const float* wbar, float* w, float* c_out, void* ws, size_t ws_bytes) {
+static int step_impl(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype, float lr, float lambda,
+                     const twa_adam_args& adam, float* alpha, const float* wbar, float* w, float* c_out, void* ws,
+                     size_t ws_bytes) {
   if (!ctx || !g || !alpha || !wbar || !w) return TWA_ERR_INVALID_ARG;
   if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
   int rc = twa_check_basis(P);
@@ -196,7 +213,7 @@ int twa_step(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
   if (rc) return rc;
   if (misaligned16(g) || misaligned16(w) || misaligned16(wbar)) return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-  twa_project_epilogue epi = {c_out, alpha, lr, lambda, -1};
+  twa_project_epilogue epi = {c_out, alpha, lr, lambda, -1, adam};
   cudaEvent_t* ev = nullptr;
   if (ctx->prof_events && ctx->prof_count < ctx->prof_cap) ev = ctx->prof_events + 3 * ctx->prof_count;
   if (ev) TWA_CUDA_OK(ctx, cudaEventRecord(ev[0], ctx->stream));
@@ -212,6 +229,35 @@ int twa_step(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
     ctx->prof_count++;
   }
   return TWA_OK;
+}
+
+int twa_step(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype, float lr, float lambda,
+             float* alpha, const float* wbar, float* w, float* c_out, void* ws, size_t ws_bytes) {
+  return step_impl(ctx, P, g, g_dtype, lr, lambda, twa_adam_args{}, alpha, wbar, w, c_out, ws, ws_bytes);
+}
+
+int twa_step_adam(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype, const twa_adam* opt,
+                  float* alpha, float* m, float* v, const float* wbar, float* w, float* c_out, void* ws,
+                  size_t ws_bytes) {
+  twa_adam_args ad;
+  int rc = twa_adam_device_args(opt, m, v, &ad);
+  if (rc) return rc;
+  return step_impl(ctx, P, g, g_dtype, opt->lr, opt->weight_decay, ad, alpha, wbar, w, c_out, ws, ws_bytes);
+}
+
+float twa_cosine_lr(float base_lr, int step, int total_steps, float min_lr) {
+  double x = total_steps > 0 ? static_cast<double>(step) / static_cast<double>(total_steps) : 1.0;
+  x = x < 0.0 ? 0.0 : (x > 1.0 ? 1.0 : x);
+  return static_cast<float>(static_cast<double>(min_lr) +
+                            0.5 * (static_cast<double>(base_lr) - static_cast<double>(min_lr)) *
+                                (1.0 + cos(3.14159265358979323846 * x)));
+}
+
+int twa_weighted_average(twa_ctx* ctx, const float* W, int64_t D, int n, int64_t ldw, const float* weights,
+                         float* w_out, void* ws, size_t ws_bytes) {
+  if (!W || !weights) return TWA_ERR_INVALID_ARG;
+  const twa_basis cand = {const_cast<float*>(W), nullptr, D, 4 * ldw, n, 32};
+  return twa_lift(ctx, &cand, weights, nullptr, w_out, ws, ws_bytes);
 }
 
 int twa_profile_enable(twa_ctx* ctx, int max_steps) {

@@ -216,14 +216,43 @@ __device__ __forceinline__ float twa_bf16_hi(uint32_t pair) { return __uint_as_f
 
 #endif  // __CUDACC__
 
+// Adam moments and constants for the coefficient update (m == null: plain gradient descent).
+// bc1 = 1 - beta1^t and bc2 = 1 - beta2^t for the 1-based step t, computed on the host.
+struct twa_adam_args {
+  float* m;
+  float* v;
+  float beta1, beta2, eps, bc1, bc2;
+};
+
+#ifdef __CUDACC__
+// The optimiser step on one coefficient after the projection gave its gradient c:
+//   gradient descent  x <- (1 - lr*lambda) x - lr c                      (Section 4.2, Algorithm 1)
+//   Adam, decoupled decay  m <- b1 m + (1-b1) c,  v <- b2 v + (1-b2) c^2,
+//                          x <- (1 - lr*lambda) x - lr (m/bc1) / (sqrt(v/bc2) + eps)
+// in float64 on float32 state; idx addresses the moments.
+__device__ __forceinline__ float twa_coefficient_update(float x, double c, float lr, float lambda,
+                                                        const twa_adam_args& ad, size_t idx) {
+  const double decay = 1.0 - static_cast<double>(lr) * static_cast<double>(lambda);
+  if (!ad.m) return static_cast<float>(decay * static_cast<double>(x) - static_cast<double>(lr) * c);
+  const double b1 = ad.beta1, b2 = ad.beta2;
+  const double m = b1 * static_cast<double>(ad.m[idx]) + (1.0 - b1) * c;
+  const double v = b2 * static_cast<double>(ad.v[idx]) + (1.0 - b2) * c * c;
+  ad.m[idx] = static_cast<float>(m);
+  ad.v[idx] = static_cast<float>(v);
+  const double step = (m / static_cast<double>(ad.bc1)) / (sqrt(v / static_cast<double>(ad.bc2)) + static_cast<double>(ad.eps));
+  return static_cast<float>(decay * static_cast<double>(x) - static_cast<double>(lr) * step);
+}
+#endif
+
 // ------------------------------------------------------------------------------------------
 // Internal launchers (defined in the .cu files)
 // ------------------------------------------------------------------------------------------
 struct twa_project_epilogue {
   float* c_out;        // n floats or null
-  float* alpha;        // when non-null: alpha <- (1 - lr*lambda) alpha - lr c
+  float* alpha;        // when non-null: alpha <- (1 - lr*lambda) alpha - lr c, or the Adam step below
   float lr, lambda;
   int nonfinite_detail; // detail reported with TWA_ERR_NONFINITE; -1 = index of the coefficient
+  twa_adam_args adam;  // m == null: plain gradient descent
 };
 
 int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
@@ -231,6 +260,8 @@ int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtyp
 int twa_launch_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
                     const float* base, float* out, bool reverse_tiles);
 int twa_check_basis(const twa_basis* P);
+// Validates the optimiser constants and fills the kernel-side Adam arguments (bias corrections for opt->step).
+int twa_adam_device_args(const twa_adam* opt, float* m, float* v, twa_adam_args* out);
 // scales[j] = absmax_j / qmax from the bit patterns of the column maxima; flags NaN/Inf
 int twa_launch_scales(twa_ctx* ctx, const unsigned* absmax, int n, int bits, float* scales);
 // Variants of the two launchers for 8- and 4-bit storage that compute the integer dot

@@ -444,7 +444,7 @@ __global__ void __launch_bounds__(128 * COMBINE_PARTS)
 layered_combine_kernel(const float* __restrict__ partials, const int* __restrict__ cta_first,
                        const int* __restrict__ cta_base, int ctas, int n, const float* __restrict__ a,
                        const float* __restrict__ b, float* c_out, float* beta, float lr, float lambda,
-                       unsigned char* dig, int* ebits_out, float* konst, int* status) {
+                       const twa_adam_args adam, unsigned char* dig, int* ebits_out, float* konst, int* status) {
   __shared__ int range[2];
   __shared__ unsigned amax;
   __shared__ double part_s[COMBINE_PARTS][128], part_g[COMBINE_PARTS];
@@ -499,9 +499,9 @@ layered_combine_kernel(const float* __restrict__ partials, const int* __restrict
     if (!isfinite(c)) twa_set_status(status, TWA_ERR_NONFINITE, l);
     if (c_out) c_out[static_cast<size_t>(l) * n + i] = static_cast<float>(c);
     if (beta) {
-      const double decay = 1.0 - static_cast<double>(lr) * static_cast<double>(lambda);
-      bnew = static_cast<float>(decay * static_cast<double>(beta[static_cast<size_t>(l) * n + i]) - static_cast<double>(lr) * c);
-      beta[static_cast<size_t>(l) * n + i] = bnew;
+      const size_t at = static_cast<size_t>(l) * n + i;
+      bnew = twa_coefficient_update(beta[at], c, lr, lambda, adam, at);
+      beta[at] = bnew;
     }
   }
   if (dig) {                                                           // only with beta: the step
@@ -791,7 +791,7 @@ int stage_count(const twa_ctx* ctx, int fixed, int stage_bytes) {
 }
 
 int do_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype, float* c_out,
-               float* beta, float lr, float lambda, bool with_digits, char* sws) {
+               float* beta, float lr, float lambda, const twa_adam_args& adam, bool with_digits, char* sws) {
   const StepLayout w = step_layout(lb);
   const int n = lb->codes.n, kt = lb->kt;
   CUtensorMap mp;
@@ -828,7 +828,7 @@ int do_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dty
   if (rc) return rc;
   layered_combine_kernel<<<lb->L, 128 * COMBINE_PARTS, 0, ctx->stream>>>(
       a.partials, lb->cta_first_layer, lb->cta_run_base, lb->cta_count, n, lb->a, lb->b, c_out, beta, lr, lambda,
-      with_digits ? reinterpret_cast<unsigned char*>(sws + w.dig) : nullptr, reinterpret_cast<int*>(sws + w.ebits),
+      adam, with_digits ? reinterpret_cast<unsigned char*>(sws + w.dig) : nullptr, reinterpret_cast<int*>(sws + w.ebits),
       reinterpret_cast<float*>(sws + w.konst), ctx->d_status);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
@@ -901,7 +901,7 @@ int twa_layered_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g
   if (!g || !c_out || (g_dtype != TWA_F32 && g_dtype != TWA_BF16)) return TWA_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(g) & 3) return TWA_ERR_MISALIGNED;         // staged in 4-byte words
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-  return do_project(ctx, lb, g, g_dtype, c_out, nullptr, 0.0f, 0.0f, false, static_cast<char*>(sws));
+  return do_project(ctx, lb, g, g_dtype, c_out, nullptr, 0.0f, 0.0f, twa_adam_args{}, false, static_cast<char*>(sws));
 }
 
 int twa_layered_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* beta, const float* base,
@@ -914,9 +914,9 @@ int twa_layered_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* bet
   return do_lift(ctx, lb, beta, base, w_out, false, static_cast<char*>(sws));
 }
 
-int twa_layered_step(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype, float lr,
-                     float lambda, float* beta, const float* wbar, float* w, float* c_out, void* sws,
-                     size_t sws_bytes) {
+static int layered_step_impl(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype, float lr,
+                             float lambda, const twa_adam_args& adam, float* beta, const float* wbar, float* w,
+                             float* c_out, void* sws, size_t sws_bytes) {
   int rc = check_step_args(ctx, lb, sws, sws_bytes);
   if (rc) return rc;
   if (!g || !beta || !wbar || !w || (g_dtype != TWA_F32 && g_dtype != TWA_BF16)) return TWA_ERR_INVALID_ARG;
@@ -924,9 +924,24 @@ int twa_layered_step(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, t
       (reinterpret_cast<uintptr_t>(w) & 3))
     return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-  rc = do_project(ctx, lb, g, g_dtype, c_out, beta, lr, lambda, true, static_cast<char*>(sws));
+  rc = do_project(ctx, lb, g, g_dtype, c_out, beta, lr, lambda, adam, true, static_cast<char*>(sws));
   if (rc) return rc;
   return do_lift(ctx, lb, beta, wbar, w, true, static_cast<char*>(sws));
+}
+
+int twa_layered_step(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype, float lr,
+                     float lambda, float* beta, const float* wbar, float* w, float* c_out, void* sws,
+                     size_t sws_bytes) {
+  return layered_step_impl(ctx, lb, g, g_dtype, lr, lambda, twa_adam_args{}, beta, wbar, w, c_out, sws, sws_bytes);
+}
+
+int twa_layered_step_adam(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dtype g_dtype,
+                          const twa_adam* opt, float* beta, float* m, float* v, const float* wbar, float* w,
+                          float* c_out, void* sws, size_t sws_bytes) {
+  twa_adam_args ad;
+  int rc = twa_adam_device_args(opt, m, v, &ad);
+  if (rc) return rc;
+  return layered_step_impl(ctx, lb, g, g_dtype, opt->lr, opt->weight_decay, ad, beta, wbar, w, c_out, sws, sws_bytes);
 }
 
 }  // extern "C"

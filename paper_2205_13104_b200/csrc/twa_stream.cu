@@ -23,6 +23,7 @@ struct ProjectArgs {
   float* c_out;
   float* alpha;
   float lr, lambda;
+  twa_adam_args adam;
   int nonfinite_detail;
   unsigned long long wait_limit_ns;
 };
@@ -258,11 +259,7 @@ twa_project_kernel(const __grid_constant__ CUtensorMap map_p,
       if (!isfinite(c))
         twa_set_status(a.status, TWA_ERR_NONFINITE, a.nonfinite_detail >= 0 ? a.nonfinite_detail : tid);
       if (a.c_out) a.c_out[tid] = static_cast<float>(c);
-      if (a.alpha) {
-        const double decay = 1.0 - static_cast<double>(a.lr) * static_cast<double>(a.lambda);
-        a.alpha[tid] = static_cast<float>(decay * static_cast<double>(a.alpha[tid]) -
-                                          static_cast<double>(a.lr) * c);
-      }
+      if (a.alpha) a.alpha[tid] = twa_coefficient_update(a.alpha[tid], c, a.lr, a.lambda, a.adam, tid);
     }
     if (tid == 0) *a.ticket = 0u;
   }
@@ -565,6 +562,7 @@ int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtyp
   a.alpha = epi.alpha;
   a.lr = epi.lr;
   a.lambda = epi.lambda;
+  a.adam = epi.adam;
   a.nonfinite_detail = epi.nonfinite_detail;
   a.wait_limit_ns = ctx->wait_limit_ns;
   int grid = ctx->sm_count < a.tiles ? ctx->sm_count : a.tiles;

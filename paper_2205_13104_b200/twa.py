@@ -45,7 +45,7 @@ EXPORTS = [
     "twa_workspace_bytes", "twa_build_basis", "twa_build_workspace_bytes", "twa_build_begin",
     "twa_build_feed", "twa_build_end_pass", "twa_mean", "twa_quantize_basis",
     "twa_basis_export", "twa_basis_import", "twa_project", "twa_lift", "twa_step",
-    "twa_step_host", "twa_project_batch", "twa_project_batch_group", "twa_layered_workspace_bytes", "twa_layered_rows", "twa_layered_basis_bytes",
+    "twa_step_host", "twa_step_adam", "twa_cosine_lr", "twa_weighted_average", "twa_layered_step_adam", "twa_project_batch", "twa_project_batch_group", "twa_layered_workspace_bytes", "twa_layered_rows", "twa_layered_basis_bytes",
     "twa_build_centered", "twa_quantize_affine", "twa_layered_export",
     "twa_layered_step_workspace_bytes", "twa_layered_project", "twa_layered_lift", "twa_layered_step",
     "twa_project_noalloc", "twa_noalloc_last_error", "twa_noalloc_scratch_bytes",
@@ -57,6 +57,12 @@ class twa_basis(ctypes.Structure):
     _fields_ = [("data", ctypes.c_void_p), ("scales", ctypes.c_void_p),
                 ("D", ctypes.c_int64), ("col_stride", ctypes.c_int64),
                 ("n", ctypes.c_int32), ("bits", ctypes.c_int32)]
+
+
+class twa_adam(ctypes.Structure):
+    """Mirror of the C struct twa_adam."""
+    _fields_ = [("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float),
+                ("eps", ctypes.c_float), ("weight_decay", ctypes.c_float), ("step", ctypes.c_int32)]
 
 
 class twa_layered_basis(ctypes.Structure):
@@ -142,6 +148,11 @@ def load():
         "twa_lift": (i32, [vp, bp, vp, vp, vp, vp, szt]),
         "twa_step": (i32, [vp, bp, vp, i32, f32, f32, vp, vp, vp, vp, vp, szt]),
         "twa_step_host": (i32, [vp, bp, vp, i32, f32, f32, vp, vp, vp, vp, vp, vp, szt]),
+        "twa_step_adam": (i32, [vp, bp, vp, i32, ctypes.POINTER(twa_adam), vp, vp, vp, vp, vp, vp, vp, szt]),
+        "twa_cosine_lr": (f32, [f32, i32, i32, f32]),
+        "twa_weighted_average": (i32, [vp, vp, i64, i32, i64, vp, vp, vp, szt]),
+        "twa_layered_step_adam": (i32, [vp, ctypes.POINTER(twa_layered_basis), vp, i32, ctypes.POINTER(twa_adam), vp, vp,
+                                        vp, vp, vp, vp, vp, szt]),
         "twa_project_batch": (i32, [vp, bp, vp, i64, i32, i32, vp, vp, szt]),
         "twa_project_batch_group": (i32, [vp, bp, i32]),
         "twa_layered_workspace_bytes": (szt, [ctypes.POINTER(ctypes.c_int64), i32, i32]),
@@ -561,3 +572,39 @@ def twa_layered_step(ctx, lb, g, lr, lam, beta, wbar, w, sws, c_out=None):
                                  _ptr(beta), _ptr(wbar), _ptr(w), _ptr(c_out), _ptr(sws), sws.numel())
     _check(rc, "twa_layered_step", ctx)
     return w
+
+
+def _adam(lr, step, beta1, beta2, eps, weight_decay):
+    return twa_adam(float(lr), float(beta1), float(beta2), float(eps), float(weight_decay), int(step))
+
+
+def twa_step_adam(ctx, P, g, lr, step, alpha, m, v, wbar, w, ws, beta1=0.9, beta2=0.999, eps=1e-8,
+                  weight_decay=0.0, c_out=None):
+    opt = _adam(lr, step, beta1, beta2, eps, weight_decay)
+    rc = load().twa_step_adam(ctx, ctypes.byref(P.desc), _ptr(g), _dtype_code(g), ctypes.byref(opt), _ptr(alpha),
+                              _ptr(m), _ptr(v), _ptr(wbar), _ptr(w), _ptr(c_out), _ptr(ws), ws.numel())
+    _check(rc, "twa_step_adam", ctx)
+    return w
+
+
+def twa_layered_step_adam(ctx, lb, g, lr, step, beta, m, v, wbar, w, sws, beta1=0.9, beta2=0.999, eps=1e-8,
+                          weight_decay=0.0, c_out=None):
+    opt = _adam(lr, step, beta1, beta2, eps, weight_decay)
+    rc = load().twa_layered_step_adam(ctx, ctypes.byref(lb.desc), _ptr(g), _dtype_code(g), ctypes.byref(opt),
+                                      _ptr(beta), _ptr(m), _ptr(v), _ptr(wbar), _ptr(w), _ptr(c_out), _ptr(sws),
+                                      sws.numel())
+    _check(rc, "twa_layered_step_adam", ctx)
+    return w
+
+
+def twa_cosine_lr(base_lr, step, total_steps, min_lr=0.0):
+    return float(load().twa_cosine_lr(float(base_lr), int(step), int(total_steps), float(min_lr)))
+
+
+def twa_weighted_average(ctx, W, D, weights, w_out, ws):
+    """W: (n, ldw) float32 candidates, one per row; weights: (n,) float32 on the device."""
+    assert W.dtype == torch.float32 and W.is_contiguous()
+    rc = load().twa_weighted_average(ctx, _ptr(W), int(D), int(W.shape[0]), int(W.shape[1]), _ptr(weights),
+                                     _ptr(w_out), _ptr(ws), ws.numel())
+    _check(rc, "twa_weighted_average", ctx)
+    return w_out
