@@ -110,9 +110,11 @@ const char* twa_last_error(const twa_ctx* ctx);
  *      1 = code -> float32 conversion and float32 FMA.  The warp and stage knobs act on the
  *      float path and on 32-bit bases only.
  *  TWA_TUNE_TILE_SEGMENTS: tensor-pipe path, 512-byte segments of a column per tile: 1 or 2
- *      (default: 2 for n <= 64, else 1).                                                */
+ *      (default: 2 for n <= 64, else 1).
+ *  TWA_TUNE_BUILD_PANEL: twa_build_basis: 0 = panels of 8 columns (default), 1 = column by column. */
 enum { TWA_TUNE_PROJECT_WARPS = 1, TWA_TUNE_LIFT_WARPS = 2, TWA_TUNE_STAGES = 3,
-       TWA_TUNE_WAIT_LIMIT_MS = 4, TWA_TUNE_DEQUANT_PATH = 5, TWA_TUNE_TILE_SEGMENTS = 6 };
+       TWA_TUNE_WAIT_LIMIT_MS = 4, TWA_TUNE_DEQUANT_PATH = 5, TWA_TUNE_TILE_SEGMENTS = 6,
+       TWA_TUNE_BUILD_PANEL = 7 };
 int twa_set_tuning(twa_ctx* ctx, int key, int value);
 
 /* Exercises the bounded wait every streaming kernel uses, without any fault: enqueues one block

@@ -165,6 +165,10 @@ int twa_set_tuning(twa_ctx* ctx, int key, int value) {
       if (value > 2) return TWA_ERR_INVALID_ARG;
       ctx->tune_tile_segments = value;
       return TWA_OK;
+    case TWA_TUNE_BUILD_PANEL:
+      if (value > 1) return TWA_ERR_INVALID_ARG;
+      ctx->tune_build_panel = value;
+      return TWA_OK;
     case TWA_TUNE_DEQUANT_PATH:
       if (value > 1) return TWA_ERR_INVALID_ARG;
       ctx->tune_dequant_path = value;

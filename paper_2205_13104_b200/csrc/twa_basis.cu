@@ -83,11 +83,124 @@ __global__ void __launch_bounds__(BLOCK) sumsq_kernel(const float* __restrict__ 
   }
 }
 
+// ---- sweeps inside a panel: a column against at most 7 earlier columns -------------------------
+constexpr int INPANEL = 7;
+
+// coef[i] = sum_r Q_i[r] v[r], i < cnt: products and sums in float64, blocks combined in block order.
+__global__ void __launch_bounds__(BLOCK) inpanel_dots_kernel(const float* __restrict__ Q0, long long ld, int cnt,
+                                                             const float* __restrict__ v, long long D,
+                                                             double* __restrict__ dpart, float* __restrict__ coef,
+                                                             unsigned* __restrict__ ticket, int* status, int detail) {
+  __shared__ double sh[INPANEL][BLOCK / 32];
+  __shared__ int last;
+  const long long nvec = D >> 2;
+  double s[INPANEL];
+#pragma unroll
+  for (int i = 0; i < INPANEL; ++i) s[i] = 0.0;
+  for (long long t = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; t < nvec;
+       t += static_cast<long long>(gridDim.x) * BLOCK) {
+    const float4 x = reinterpret_cast<const float4*>(v)[t];
+#pragma unroll
+    for (int i = 0; i < INPANEL; ++i) {
+      if (i < cnt) {
+        const float4 q = __ldcs(reinterpret_cast<const float4*>(Q0 + i * ld) + t);
+        s[i] += static_cast<double>(x.x) * q.x + static_cast<double>(x.y) * q.y + static_cast<double>(x.z) * q.z +
+                static_cast<double>(x.w) * q.w;
+      }
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (D & 3)) {
+    const long long r = (nvec << 2) + threadIdx.x;
+    for (int i = 0; i < cnt; ++i) s[i] += static_cast<double>(v[r]) * Q0[i * ld + r];
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+  for (int i = 0; i < INPANEL; ++i) {
+    double t = s[i];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, off);
+    if (lane == 0) sh[i][warp] = t;
+  }
+  __syncthreads();
+  if (threadIdx.x < INPANEL) {
+    double t = 0;
+    for (int w = 0; w < BLOCK / 32; ++w) t += sh[threadIdx.x][w];
+    dpart[static_cast<size_t>(blockIdx.x) * 8 + threadIdx.x] = t;
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (last) {
+    __threadfence();
+    if (threadIdx.x < cnt) {
+      double t = 0;
+      for (unsigned b = 0; b < gridDim.x; ++b) t += __ldcg(&dpart[static_cast<size_t>(b) * 8 + threadIdx.x]);
+      if (!isfinite(t)) twa_set_status(status, TWA_ERR_NONFINITE, detail);
+      coef[threadIdx.x] = static_cast<float>(t);
+    }
+    if (threadIdx.x == 0) *ticket = 0u;
+  }
+}
+
+// v <- v - sum_i coef[i] Q_i (float32, the coefficients applied in index order), and
+// *result = sum of the squares of the stored values (float64).
+__global__ void __launch_bounds__(BLOCK) inpanel_update_kernel(const float* __restrict__ Q0, long long ld, int cnt,
+                                                               float* __restrict__ v, long long D,
+                                                               const float* __restrict__ coef,
+                                                               double* __restrict__ dpart, double* __restrict__ result,
+                                                               unsigned* __restrict__ ticket) {
+  __shared__ double sh[BLOCK / 32];
+  __shared__ int last;
+  float c[INPANEL];
+#pragma unroll
+  for (int i = 0; i < INPANEL; ++i) c[i] = i < cnt ? coef[i] : 0.0f;
+  const long long nvec = D >> 2;
+  double s = 0;
+  for (long long t = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; t < nvec;
+       t += static_cast<long long>(gridDim.x) * BLOCK) {
+    float4 x = reinterpret_cast<const float4*>(v)[t];
+#pragma unroll
+    for (int i = 0; i < INPANEL; ++i) {
+      if (i < cnt) {
+        const float4 q = __ldcs(reinterpret_cast<const float4*>(Q0 + i * ld) + t);
+        x.x = fmaf(-c[i], q.x, x.x); x.y = fmaf(-c[i], q.y, x.y);
+        x.z = fmaf(-c[i], q.z, x.z); x.w = fmaf(-c[i], q.w, x.w);
+      }
+    }
+    reinterpret_cast<float4*>(v)[t] = x;
+    s += static_cast<double>(x.x) * x.x + static_cast<double>(x.y) * x.y + static_cast<double>(x.z) * x.z +
+         static_cast<double>(x.w) * x.w;
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (D & 3)) {
+    const long long r = (nvec << 2) + threadIdx.x;
+    float x = v[r];
+    for (int i = 0; i < cnt; ++i) x = fmaf(-c[i], Q0[i * ld + r], x);
+    v[r] = x;
+    s += static_cast<double>(x) * x;
+  }
+  const double bs = block_sum(s, sh);
+  if (threadIdx.x == 0) {
+    dpart[blockIdx.x] = bs;
+    __threadfence();
+    last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (last && threadIdx.x == 0) {
+    __threadfence();
+    double t = 0;
+    for (unsigned b = 0; b < gridDim.x; ++b) t += __ldcg(&dpart[b]);
+    *result = t;
+    *ticket = 0u;
+  }
+}
+
 // ---- normalise a column: v <- v / |v|, with the rank and finiteness checks -------------------
 __global__ void __launch_bounds__(BLOCK) normalise_kernel(float* __restrict__ v, long long D,
-                                                          const double* __restrict__ norms, int column,
+                                                          const double* __restrict__ norm_before,
+                                                          const double* __restrict__ norm_after, int column,
                                                           int* status) {
-  const double na = norms[0], nv = norms[1];
+  const double na = *norm_before, nv = *norm_after;
   double f;
   if (!isfinite(na) || !isfinite(nv)) {
     if (blockIdx.x == 0 && threadIdx.x == 0) twa_set_status(status, TWA_ERR_NONFINITE, column);
@@ -234,11 +347,10 @@ int grid_for(const twa_ctx* ctx, long long items, int per_block, int blocks_per_
   return static_cast<int>(g);
 }
 
-int launch_sumsq(twa_ctx* ctx, const float* v, long long D, void* ws, int slot) {
+int launch_sumsq(twa_ctx* ctx, const float* v, long long D, void* ws, double* result) {
   char* w = static_cast<char*>(ws);
   const int grid = grid_for(ctx, D, BLOCK * 16, 4);
-  sumsq_kernel<<<grid, BLOCK, 0, ctx->stream>>>(v, D, reinterpret_cast<double*>(w + TWA_WS_DPART),
-                                                reinterpret_cast<double*>(w + TWA_WS_NORMS) + slot,
+  sumsq_kernel<<<grid, BLOCK, 0, ctx->stream>>>(v, D, reinterpret_cast<double*>(w + TWA_WS_DPART), result,
                                                 ctx->d_ticket);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
@@ -293,26 +405,86 @@ int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float
 
   char* w = static_cast<char*>(ws);
   float* coef = reinterpret_cast<float*>(w + TWA_WS_COEF);
-  const double* norms = reinterpret_cast<const double*>(w + TWA_WS_NORMS);
+  double* norms = reinterpret_cast<double*>(w + TWA_WS_NORMS);          // [0]: after the sweep
+  // squared norms of a panel's columns as given: the last doubles of the workspace's float region
+  double* given = reinterpret_cast<double*>(w + TWA_WS_PARTIALS + sizeof(float) * TWA_MAX_GRID * TWA_MAX_N) - 8;
   const int egrid = grid_for(ctx, D, BLOCK * 16, 4);
-  for (int j = 0; j < n; ++j) {
-    float* col = W + j * ldw;
-    rc = launch_sumsq(ctx, col, D, ws, 0);                       // |a_j|^2
-    if (rc) return rc;
-    if (j > 0) {
-      twa_basis Q = {W, nullptr, D, 4 * ldw, j, 32};
-      twa_project_epilogue epi = {coef, nullptr, 0.0f, 0.0f, j};
-      for (int pass = 0; pass < 2; ++pass) {
-        rc = twa_launch_project(ctx, &Q, col, TWA_F32, epi, ws);  // c = Q^T v, all from the same v
-        if (rc) return rc;
-        rc = twa_launch_lift(ctx, &Q, coef, -1.0f, col, col, false);   // v <- v - Q c
+  const int width = ctx->tune_build_panel == 1 ? 1 : 8;
+
+  // One Gram-Schmidt sweep of column k against columns first .. k-1 (all coefficients from the same
+  // vector), then its squared norm.
+  auto sweep = [&](int first, int k) -> int {
+    float* col = W + k * ldw;
+    if (k > first) {
+      twa_basis Q = {W + first * ldw, nullptr, D, 4 * ldw, k - first, 32};
+      twa_project_epilogue epi = {coef, nullptr, 0.0f, 0.0f, k};
+      int r = twa_launch_project(ctx, &Q, col, TWA_F32, epi, ws);         // c = Q^T v
+      if (r) return r;
+      r = twa_launch_lift(ctx, &Q, coef, -1.0f, col, col, false);         // v <- v - Q c
+      if (r) return r;
+    }
+    return launch_sumsq(ctx, col, D, ws, norms);
+  };
+
+  if (width == 1) {
+    // column by column: two sweeps against everything before, then normalise
+    for (int j = 0; j < n; ++j) {
+      float* col = W + j * ldw;
+      rc = launch_sumsq(ctx, col, D, ws, given);                       // |a_j|^2
+      if (rc) return rc;
+      rc = sweep(0, j);
+      if (rc) return rc;
+      if (j > 0) {
+        rc = sweep(0, j);
         if (rc) return rc;
       }
+      normalise_kernel<<<egrid, BLOCK, 0, ctx->stream>>>(col, D, given, norms, j, ctx->d_status);
+      TWA_CUDA_OK(ctx, cudaGetLastError());
     }
-    rc = launch_sumsq(ctx, col, D, ws, 1);                       // |v|^2
-    if (rc) return rc;
-    normalise_kernel<<<egrid, BLOCK, 0, ctx->stream>>>(col, D, norms, j, ctx->d_status);
-    TWA_CUDA_OK(ctx, cudaGetLastError());
+  } else {
+    // Panels of up to 8 columns.  Twice: remove the earlier basis vectors from the whole panel in one
+    // pass over them (projection of the panel, then update), then sweep and normalise the panel's
+    // columns among themselves.  The first round makes the panel orthonormal up to the rounding its
+    // cancellation amplifies; the second round, applied to unit vectors, removes that.
+    for (int j0 = 0; j0 < n; j0 += width) {
+      const int pb = n - j0 < width ? n - j0 : width;
+      for (int q = 0; q < pb; ++q) {
+        rc = launch_sumsq(ctx, W + (j0 + q) * ldw, D, ws, given + q);   // |a_j|^2 as given
+        if (rc) return rc;
+      }
+      for (int round = 0; round < 2; ++round) {
+        if (j0 > 0) {
+          rc = twa_launch_panel_project(ctx, W, D, ldw, j0, pb, ws);
+          if (rc) return rc;
+          rc = twa_launch_panel_lift(ctx, W, D, ldw, j0, pb, ws);
+          if (rc) return rc;
+        }
+        for (int q = 0; q < pb; ++q) {
+          const int k = j0 + q;
+          float* col = W + k * ldw;
+          if (round == 1) {
+            rc = launch_sumsq(ctx, col, D, ws, given + q);              // 1, or 0 for a column found dependent
+            if (rc) return rc;
+          }
+          if (q > 0) {
+            // one sweep against the panel's earlier columns, fused with the squared norm of the result
+            double* dpart = reinterpret_cast<double*>(w + TWA_WS_DPART);
+            double* dots_part = reinterpret_cast<double*>(w + TWA_WS_PARTIALS);   // [egrid][8], start of the float region
+            inpanel_dots_kernel<<<egrid, BLOCK, 0, ctx->stream>>>(W + j0 * ldw, ldw, q, col, D, dots_part, coef,
+                                                                  ctx->d_ticket, ctx->d_status, k);
+            TWA_CUDA_OK(ctx, cudaGetLastError());
+            inpanel_update_kernel<<<egrid, BLOCK, 0, ctx->stream>>>(W + j0 * ldw, ldw, q, col, D, coef, dpart, norms,
+                                                                    ctx->d_ticket);
+            TWA_CUDA_OK(ctx, cudaGetLastError());
+          } else {
+            rc = launch_sumsq(ctx, col, D, ws, norms);
+            if (rc) return rc;
+          }
+          normalise_kernel<<<egrid, BLOCK, 0, ctx->stream>>>(col, D, given + q, norms, k, ctx->d_status);
+          TWA_CUDA_OK(ctx, cudaGetLastError());
+        }
+      }
+    }
   }
   P32_out->data = W;
   P32_out->scales = nullptr;

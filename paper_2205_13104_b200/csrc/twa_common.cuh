@@ -29,6 +29,7 @@ struct twa_ctx {
   int tune_project_warps, tune_lift_warps, tune_stages;
   int tune_dequant_path;      // 0 = integer tensor-pipe dot products, 1 = float FMA
   int tune_tile_segments;     // tensor-pipe path: 512-byte segments per tile column (0 = choose)
+  int tune_build_panel;       // resident basis build: 0 = panels of 8 columns, 1 = column by column
   cudaEvent_t* prof_events;   // 3 per recorded step, or null
   int prof_cap, prof_count;   // steps
   // state of a row-chunked basis build (twa_build_begin .. twa_build_end_pass)
@@ -260,6 +261,10 @@ int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtyp
 int twa_launch_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
                     const float* base, float* out, bool reverse_tiles);
 int twa_check_basis(const twa_basis* P);
+// Panel steps of the blocked basis build on the float32 matrix W (columns of stride ldw):
+// C = Q^T A_p into the workspace, then A_p <- A_p - Q C; Q = columns 0..nq-1, A_p = the next pb <= 8.
+int twa_launch_panel_project(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws);
+int twa_launch_panel_lift(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws);
 // Validates the optimiser constants and fills the kernel-side Adam arguments (bias corrections for opt->step).
 int twa_adam_device_args(const twa_adam* opt, float* m, float* v, twa_adam_args* out);
 // scales[j] = absmax_j / qmax from the bit patterns of the column maxima; flags NaN/Inf

@@ -1,0 +1,386 @@
+// Panel steps of the blocked Gram-Schmidt build (Section 4.1 of the paper: Schmidt
+// orthogonalisation of {w_i}): a panel of up to 8 candidate columns is orthogonalised against all
+// earlier basis vectors at once, so the earlier vectors are read once per panel instead of once
+// per column.
+//     C = Q^T A_p        (twa_launch_panel_project)   Q: columns 0 .. nq-1, A_p: columns nq .. nq+pb-1
+//     A_p <- A_p - Q C   (twa_launch_panel_lift)
+// The projection streams tiles of 64 rows x (nq + pb) columns of the float32 matrix through a TMA
+// ring (one box per stage: the panel's columns are simply the last columns of the tile).
+//  * projection: warp w owns columns w, w+16, ...; a lane owns 2 rows; 8 x 8 accumulators per lane;
+//    lanes -> block -> last block to finish, float64 over blocks in block order.
+//  * update: a lane owns one row of a block of 512 rows and walks all nq columns as they stream past
+//    in chunks of 8, so there is no reduction at all.
+#include <stdio.h>
+
+#include "twa_common.cuh"
+
+namespace {
+
+constexpr int PANEL = 8;                         // columns per panel at most
+constexpr int PROWS = 64;                        // rows per tile
+constexpr int PCOL_BYTES = PROWS * 4;
+constexpr int PWARPS = 16;                       // consumer warps
+constexpr int PTHREADS = (PWARPS + 1) * 32;
+constexpr int CPART_BYTES = 4096;                // block's sums / coefficients: TWA_MAX_N x PANEL floats
+constexpr int MAX_Q_PER_WARP = TWA_MAX_N / PWARPS;
+
+struct PanelArgs {
+  long long D, ldw;
+  int nq, pb, tiles, stages, detail;
+  unsigned stage_bytes, tx_bytes;
+  float* panel;                // first column of the panel
+  float* partials;             // [grid][nq * PANEL]
+  float* C;                    // [nq][PANEL]
+  unsigned* ticket;
+  int* status;
+  unsigned long long wait_limit_ns;
+};
+
+__device__ __forceinline__ void panel_producer(twa_smem_header* hdr, unsigned char* ring, const CUtensorMap* map,
+                                               const PanelArgs& a) {
+  twa_prefetch_tensormap(map);
+  volatile int* abort_flag = &hdr->abort_flag;
+  int issued = 0;
+  bool ok = true;
+  for (int tile = blockIdx.x; tile < a.tiles; tile += gridDim.x, ++issued) {
+    const int s = issued % a.stages, use = issued / a.stages;
+    if (use > 0 && !twa_mbar_wait(twa_smem_u32(&hdr->empty[s]), static_cast<unsigned>(use - 1) & 1u, abort_flag,
+                                  a.wait_limit_ns)) {
+      ok = false;
+      break;
+    }
+    const uint32_t fb = twa_smem_u32(&hdr->full[s]);
+    twa_mbar_expect_tx(fb, a.tx_bytes);
+    twa_tma_load_2d(twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes), map, tile * PROWS, 0, fb);
+  }
+  if (!ok) {
+    twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+    const int live = issued < a.stages ? issued : a.stages;
+    for (int q = 0; q < live; ++q) {      // let the copies already issued land
+      const int last = ((issued - 1 - q) / a.stages) * a.stages + q;
+      const unsigned par = static_cast<unsigned>(last / a.stages) & 1u;
+      const unsigned long long t0 = twa_globaltimer();
+      while (!twa_mbar_try_wait(twa_smem_u32(&hdr->full[q]), par)) {
+        if (twa_globaltimer() - t0 > a.wait_limit_ns) break;
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(PTHREADS, 1)
+panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
+  twa_smem_header* hdr = reinterpret_cast<twa_smem_header*>(smem);
+  float* cpart = reinterpret_cast<float*>(smem + TWA_SMEM_HEADER);
+  unsigned char* ring = smem + TWA_SMEM_HEADER + CPART_BYTES;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < a.stages; ++s) {
+      twa_mbar_init(twa_smem_u32(&hdr->full[s]), 1);
+      twa_mbar_init(twa_smem_u32(&hdr->empty[s]), PWARPS);
+    }
+    hdr->abort_flag = 0;
+    hdr->last_flag = 0;
+    twa_fence_barrier_init();
+  }
+  __syncthreads();
+
+  if (warp == PWARPS) {
+    if (lane == 0) panel_producer(hdr, ring, &map, a);
+  } else {
+    const int cpw = warp < a.nq ? (a.nq - warp + PWARPS - 1) / PWARPS : 0;       // columns warp, warp + 16, ...
+    float acc[MAX_Q_PER_WARP][PANEL];
+#pragma unroll
+    for (int k = 0; k < MAX_Q_PER_WARP; ++k)
+#pragma unroll
+      for (int q = 0; q < PANEL; ++q) acc[k][q] = 0.0f;
+    volatile int* abort_flag = &hdr->abort_flag;
+    int k_tile = 0;
+    for (int tile = blockIdx.x; tile < a.tiles; tile += gridDim.x, ++k_tile) {
+      const int s = k_tile % a.stages;
+      if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), static_cast<unsigned>(k_tile / a.stages) & 1u, abort_flag,
+                         a.wait_limit_ns)) {
+        twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+        break;
+      }
+      const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
+      float2 g[PANEL];
+#pragma unroll
+      for (int q = 0; q < PANEL; ++q)
+        g[q] = q < a.pb ? *reinterpret_cast<const float2*>(st + (a.nq + q) * PCOL_BYTES + lane * 8) : make_float2(0.f, 0.f);
+#pragma unroll
+      for (int k = 0; k < MAX_Q_PER_WARP; ++k) {
+        if (k < cpw) {
+          const float2 p = *reinterpret_cast<const float2*>(st + (warp + k * PWARPS) * PCOL_BYTES + lane * 8);
+#pragma unroll
+          for (int q = 0; q < PANEL; ++q) acc[k][q] = fmaf(p.x, g[q].x, fmaf(p.y, g[q].y, acc[k][q]));
+        }
+      }
+      __syncwarp();
+      if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
+    }
+    // lanes -> one value per (column, panel column); every pair belongs to exactly one warp
+#pragma unroll
+    for (int k = 0; k < MAX_Q_PER_WARP; ++k) {
+      if (k < cpw) {
+#pragma unroll
+        for (int q = 0; q < PANEL; ++q) {
+          float v = acc[k][q];
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+          if (lane == 0) cpart[(warp + k * PWARPS) * PANEL + q] = v;
+        }
+      }
+    }
+  }
+  __syncthreads();
+  const int tid = threadIdx.x, outs = a.nq * PANEL;
+  for (int i = tid; i < outs; i += blockDim.x) a.partials[static_cast<size_t>(blockIdx.x) * outs + i] = cpart[i];
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned ticket = atomicAdd(a.ticket, 1u);
+    hdr->last_flag = (ticket == gridDim.x - 1) ? 1 : 0;
+  }
+  __syncthreads();
+  if (hdr->last_flag) {
+    __threadfence();
+    for (int i = tid; i < outs; i += blockDim.x) {
+      double sum = 0.0;
+      for (unsigned b = 0; b < gridDim.x; ++b) sum += static_cast<double>(__ldcg(&a.partials[static_cast<size_t>(b) * outs + i]));
+      if (!isfinite(sum)) twa_set_status(a.status, TWA_ERR_NONFINITE, a.detail + (i % PANEL));
+      a.C[i] = static_cast<float>(sum);
+    }
+    if (tid == 0) *a.ticket = 0u;
+  }
+}
+
+// Update kernel.  A block walks blocks of 512 rows; a lane owns one row of the block (16 warps x 32
+// lanes) and accumulates its 8 results while the columns of Q stream past in chunks of 8 (one stage
+// = 512 rows x 8 columns, two boxes of 256 rows); the chunk after the last one of Q is the panel
+// itself, whose old values the lane then updates and stores.  Every consumer warp consumes every
+// stage, in order: the plain ring protocol, no reduction anywhere.
+constexpr int LROWS_BLOCK = PWARPS * 32;                     // 512 rows per row block
+constexpr int LCHUNK = PANEL;                                // columns per stage
+constexpr unsigned LSTAGE_BYTES = LROWS_BLOCK * LCHUNK * 4;  // 16 KB
+
+struct PanelLiftArgs {
+  long long D, ldw;
+  int nq, pb, row_blocks, stages;
+  float* panel;
+  const float* C;
+  int* status;
+  unsigned long long wait_limit_ns;
+};
+
+__global__ void __launch_bounds__(PTHREADS, 1)
+panel_lift_kernel(const __grid_constant__ CUtensorMap map, const PanelLiftArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
+  twa_smem_header* hdr = reinterpret_cast<twa_smem_header*>(smem);
+  float* Cs = reinterpret_cast<float*>(smem + TWA_SMEM_HEADER);        // [nq][PANEL]
+  unsigned char* ring = smem + TWA_SMEM_HEADER + CPART_BYTES;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < a.stages; ++s) {
+      twa_mbar_init(twa_smem_u32(&hdr->full[s]), 1);
+      twa_mbar_init(twa_smem_u32(&hdr->empty[s]), PWARPS);
+    }
+    hdr->abort_flag = 0;
+    twa_fence_barrier_init();
+  }
+  for (int i = threadIdx.x; i < a.nq * PANEL; i += blockDim.x) Cs[i] = a.C[i];
+  __syncthreads();
+  volatile int* abort_flag = &hdr->abort_flag;
+  const int chunks = a.nq / LCHUNK + 1;                                // chunks of Q, then the panel
+  if (warp == PWARPS) {
+    if (lane != 0) return;
+    twa_prefetch_tensormap(&map);
+    int it = 0;
+    bool ok = true;
+    for (int rb = blockIdx.x; rb < a.row_blocks && ok; rb += gridDim.x) {
+      for (int c = 0; c < chunks; ++c, ++it) {
+        const int s = it % a.stages, use = it / a.stages;
+        if (use > 0 && !twa_mbar_wait(twa_smem_u32(&hdr->empty[s]), static_cast<unsigned>(use - 1) & 1u, abort_flag,
+                                      a.wait_limit_ns)) {
+          ok = false;
+          break;
+        }
+        const uint32_t fb = twa_smem_u32(&hdr->full[s]);
+        const uint32_t dst = twa_smem_u32(ring + static_cast<size_t>(s) * LSTAGE_BYTES);
+        twa_mbar_expect_tx(fb, LSTAGE_BYTES);
+        twa_tma_load_2d(dst, &map, rb * LROWS_BLOCK, c * LCHUNK, fb);
+        twa_tma_load_2d(dst + LSTAGE_BYTES / 2, &map, rb * LROWS_BLOCK + 256, c * LCHUNK, fb);
+      }
+    }
+    if (!ok) {
+      twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+      const int live = it < a.stages ? it : a.stages;
+      for (int q = 0; q < live; ++q) {      // let the copies already issued land
+        const int last = ((it - 1 - q) / a.stages) * a.stages + q;
+        const unsigned par = static_cast<unsigned>(last / a.stages) & 1u;
+        const unsigned long long t0 = twa_globaltimer();
+        while (!twa_mbar_try_wait(twa_smem_u32(&hdr->full[q]), par)) {
+          if (twa_globaltimer() - t0 > a.wait_limit_ns) break;
+        }
+      }
+    }
+    return;
+  }
+  // element (column c of the chunk, row r of the block) sits at ((r >> 8) * 8 + c) * 256 + (r & 255)
+  const int r = warp * 32 + lane;
+  const int base = (r >> 8) * LCHUNK * 256 + (r & 255);
+  int it = 0;
+  bool alive = true;
+  for (int rb = blockIdx.x; rb < a.row_blocks && alive; rb += gridDim.x) {
+    float acc[PANEL];
+#pragma unroll
+    for (int q = 0; q < PANEL; ++q) acc[q] = 0.0f;
+    for (int c = 0; c < chunks; ++c, ++it) {
+      const int s = it % a.stages;
+      if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), static_cast<unsigned>(it / a.stages) & 1u, abort_flag,
+                         a.wait_limit_ns)) {
+        twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+        alive = false;
+        break;
+      }
+      const float* st = reinterpret_cast<const float*>(ring + static_cast<size_t>(s) * LSTAGE_BYTES) + base;
+      if (c < chunks - 1) {
+#pragma unroll
+        for (int u = 0; u < LCHUNK; ++u) {
+          const float x = st[u * 256];
+          const float4 c0 = *reinterpret_cast<const float4*>(Cs + (c * LCHUNK + u) * PANEL);
+          const float4 c1 = *reinterpret_cast<const float4*>(Cs + (c * LCHUNK + u) * PANEL + 4);
+          acc[0] = fmaf(x, c0.x, acc[0]); acc[1] = fmaf(x, c0.y, acc[1]);
+          acc[2] = fmaf(x, c0.z, acc[2]); acc[3] = fmaf(x, c0.w, acc[3]);
+          acc[4] = fmaf(x, c1.x, acc[4]); acc[5] = fmaf(x, c1.y, acc[5]);
+          acc[6] = fmaf(x, c1.z, acc[6]); acc[7] = fmaf(x, c1.w, acc[7]);
+        }
+        __syncwarp();
+        if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
+      } else {
+        float old[PANEL];
+#pragma unroll
+        for (int q = 0; q < PANEL; ++q) old[q] = st[q * 256];
+        __syncwarp();
+        if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
+        const long long row = static_cast<long long>(rb) * LROWS_BLOCK + r;
+        if (row < a.D) {
+#pragma unroll
+          for (int q = 0; q < PANEL; ++q)
+            if (q < a.pb) a.panel[q * a.ldw + row] = old[q] - acc[q];
+        }
+      }
+    }
+  }
+}
+
+int encode_panel_map(twa_ctx* ctx, const float* W, long long D, long long ldw, int cols, CUtensorMap* map) {
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(cols)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldw * 4)};
+  cuuint32_t box[2] = {PROWS, static_cast<cuuint32_t>(cols)};
+  cuuint32_t es[2] = {1, 1};
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(W), dims, strides, box, es,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(ctx->last_error, sizeof(ctx->last_error), "cuTensorMapEncodeTiled(panel) failed: %d", static_cast<int>(r));
+    return TWA_ERR_CUDA;
+  }
+  return TWA_OK;
+}
+
+int fill_args(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws, PanelArgs* a, int* grid,
+              int* smem) {
+  if (nq < 1 || pb < 1 || pb > PANEL || nq + pb > TWA_MAX_N) return TWA_ERR_INVALID_ARG;
+  a->D = D;
+  a->ldw = ldw;
+  a->nq = nq;
+  a->pb = pb;
+  a->detail = nq;
+  a->tiles = static_cast<int>((D + PROWS - 1) / PROWS);
+  a->tx_bytes = static_cast<unsigned>(nq + pb) * PCOL_BYTES;
+  a->stage_bytes = (a->tx_bytes + 1023) / 1024 * 1024;
+  const int fixed = TWA_SMEM_HEADER + CPART_BYTES + 1024;
+  int stages = (ctx->smem_optin - fixed) / static_cast<int>(a->stage_bytes);
+  if (stages > TWA_MAX_STAGES) stages = TWA_MAX_STAGES;
+  if (stages < 2) return TWA_ERR_UNSUPPORTED;
+  a->stages = stages;
+  a->panel = W + static_cast<long long>(nq) * ldw;
+  // the float region of the workspace: per-block sums, then the coefficients (1024 floats), then
+  // 16 floats the caller keeps for itself
+  float* region = reinterpret_cast<float*>(static_cast<char*>(ws) + TWA_WS_PARTIALS);
+  const size_t region_floats = static_cast<size_t>(TWA_MAX_GRID) * TWA_MAX_N;
+  a->partials = region;
+  a->C = region + region_floats - 1040;
+  a->ticket = ctx->d_ticket;
+  a->status = ctx->d_status;
+  a->wait_limit_ns = ctx->wait_limit_ns;
+  int g = ctx->sm_count < a->tiles ? ctx->sm_count : a->tiles;
+  const size_t per_block = static_cast<size_t>(nq) * PANEL;
+  if (static_cast<size_t>(g) * per_block > region_floats - 1040) g = static_cast<int>((region_floats - 1040) / per_block);
+  *grid = g;
+  *smem = fixed + stages * static_cast<int>(a->stage_bytes);
+  return TWA_OK;
+}
+
+}  // namespace
+
+int twa_launch_panel_project(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws) {
+  PanelArgs a;
+  int grid, smem;
+  int rc = fill_args(ctx, W, D, ldw, nq, pb, ws, &a, &grid, &smem);
+  if (rc) return rc;
+  CUtensorMap map;
+  rc = encode_panel_map(ctx, W, D, ldw, nq + pb, &map);
+  if (rc) return rc;
+  static int smem_limit[64] = {0};
+  rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(panel_project_kernel), &smem_limit[ctx->device & 63], smem);
+  if (rc) return rc;
+  panel_project_kernel<<<grid, PTHREADS, smem, ctx->stream>>>(map, a);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+int twa_launch_panel_lift(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws) {
+  if (nq < LCHUNK || (nq % LCHUNK) != 0 || pb < 1 || pb > PANEL || nq + pb > TWA_MAX_N) return TWA_ERR_INVALID_ARG;
+  PanelLiftArgs a;
+  a.D = D;
+  a.ldw = ldw;
+  a.nq = nq;
+  a.pb = pb;
+  a.row_blocks = static_cast<int>((D + LROWS_BLOCK - 1) / LROWS_BLOCK);
+  const int fixed = TWA_SMEM_HEADER + CPART_BYTES + 1024;
+  int stages = (ctx->smem_optin - fixed) / static_cast<int>(LSTAGE_BYTES);
+  if (stages > TWA_MAX_STAGES) stages = TWA_MAX_STAGES;
+  if (stages < 2) return TWA_ERR_UNSUPPORTED;
+  a.stages = stages;
+  a.panel = W + static_cast<long long>(nq) * ldw;
+  const float* region = reinterpret_cast<const float*>(static_cast<const char*>(ws) + TWA_WS_PARTIALS);
+  a.C = region + static_cast<size_t>(TWA_MAX_GRID) * TWA_MAX_N - 1040;      // where the projection left it
+  a.status = ctx->d_status;
+  a.wait_limit_ns = ctx->wait_limit_ns;
+  // boxes of 256 rows x 8 columns over the matrix's first nq + pb columns (columns past them read as zero)
+  CUtensorMap map;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(nq + pb)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldw * 4)};
+  cuuint32_t box[2] = {256, LCHUNK};
+  cuuint32_t es[2] = {1, 1};
+  CUresult r = ctx->encode_tiled(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, W, dims, strides, box, es,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(ctx->last_error, sizeof(ctx->last_error), "cuTensorMapEncodeTiled(panel update) failed: %d",
+             static_cast<int>(r));
+    return TWA_ERR_CUDA;
+  }
+  const int grid = ctx->sm_count < a.row_blocks ? ctx->sm_count : a.row_blocks;
+  const int smem = fixed + stages * static_cast<int>(LSTAGE_BYTES);
+  static int smem_limit[64] = {0};
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(panel_lift_kernel), &smem_limit[ctx->device & 63], smem);
+  if (rc) return rc;
+  panel_lift_kernel<<<grid, PTHREADS, smem, ctx->stream>>>(map, a);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libtwa.so")
 CSRC = os.path.join(_HERE, "csrc")
-SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_chunked.cu", "twa_layered_build.cu", "twa_layered_step.cu", "twa_project_batch.cu", "twa_stream.cu",
+SOURCES = ["twa_api.cu", "twa_basis.cu", "twa_chunked.cu", "twa_layered_build.cu", "twa_layered_step.cu", "twa_project_batch.cu", "twa_panel.cu", "twa_stream.cu",
            "twa_stream_mma.cu", "twa_noalloc.cu"]
 
 TWA_MAX_N = 128
@@ -37,6 +37,7 @@ TWA_TUNE_STAGES = 3
 TWA_TUNE_WAIT_LIMIT_MS = 4
 TWA_TUNE_DEQUANT_PATH = 5
 TWA_TUNE_TILE_SEGMENTS = 6
+TWA_TUNE_BUILD_PANEL = 7
 
 EXPORTS = [
     "twa_create", "twa_destroy", "twa_get_status", "twa_clear_status", "twa_strerror",

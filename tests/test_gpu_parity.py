@@ -496,3 +496,54 @@ def test_bounded_wait_runs_out_cleanly_and_the_context_stays_usable(env):
     co = orc.unpack_codes(codes.cpu().numpy(), D, 8)
     assert rel(c.cpu().numpy(), orc.project(co, s.cpu().numpy(), g.cpu().numpy())) <= TOL
     status_ok(ctx)
+
+
+# ------------------------------------------------------------------ panel build against the column-wise build
+@pytest.mark.parametrize("D,n,step", [(50001, 24, 0.005), (50001, 24, 0.0002), (120007, 77, 0.002), (9001, 9, 0.01)])
+def test_panel_build_agrees_with_column_build_and_oracle(env, D, n, step):
+    ctx, ws = env
+    wbar = torch.empty(D, device=DEV)
+    out = {}
+    for mode in (1, 0):                                   # 1: column by column, 0: panels of 8 (default)
+        W = inputs.trajectory_candidates(D, n, step, 0.001, 31, DEV, ld=inputs.padded_ld(D, 4))
+        A = host_cols(W, D).copy()
+        twa.twa_set_tuning(ctx, twa.TWA_TUNE_BUILD_PANEL, mode)
+        try:
+            twa.twa_build_basis(ctx, W, D, wbar, ws)
+        finally:
+            twa.twa_set_tuning(ctx, twa.TWA_TUNE_BUILD_PANEL, 0)
+        status_ok(ctx)
+        out[mode] = host_cols(W, D).astype(np.float64)
+    Q, _, bad = orc.cgs2(A)
+    assert bad is None
+    kappa = np.linalg.cond(A.astype(np.float64))
+    for mode, Pg in out.items():
+        assert np.max(np.abs(Pg.T @ Pg - np.eye(n))) <= 1e-5, mode
+        assert np.max(np.linalg.norm(Pg - Q, axis=0)) <= 10 * kappa * np.finfo(np.float32).eps, mode
+        T = Pg.T @ A.astype(np.float64)
+        assert np.all(np.diag(T) > 0) and np.max(np.abs(np.tril(T, -1))) <= 2e-5 * np.max(np.abs(T))
+    # the two schedules reach the same vectors to the accuracy either reaches the oracle
+    assert np.max(np.linalg.norm(out[0] - out[1], axis=0)) <= 20 * kappa * np.finfo(np.float32).eps
+
+
+def test_panel_build_finds_dependence_across_and_inside_panels(env):
+    ctx, ws = env
+    D, n = 30001, 20
+    wbar = torch.empty(D, device=DEV)
+    for bad_col, src in ((13, 3), (14, 9), (7, 0)):       # earlier panel; same panel; first panel
+        W = inputs.trajectory_candidates(D, n, 0.01, 0.002, 2, DEV, ld=inputs.padded_ld(D, 4))
+        W[bad_col] = W[src] * -2.0
+        twa.twa_build_basis(ctx, W, D, wbar, ws)
+        code, detail = twa.twa_get_status(ctx)
+        assert (code, detail) == (twa.TWA_ERR_RANK_DEFICIENT, bad_col)
+        twa.twa_clear_status(ctx)
+        Pg = host_cols(W, D).astype(np.float64)
+        keep = [j for j in range(n) if j != bad_col]
+        assert np.all(Pg[:, bad_col] == 0)                 # the dependent column is zeroed, the rest is a basis
+        assert np.max(np.abs(Pg[:, keep].T @ Pg[:, keep] - np.eye(n - 1))) <= 1e-5
+    W = inputs.trajectory_candidates(D, n, 0.01, 0.002, 2, DEV, ld=inputs.padded_ld(D, 4))
+    W[11, 222] = float("nan")
+    twa.twa_build_basis(ctx, W, D, wbar, ws)
+    code, detail = twa.twa_get_status(ctx)
+    assert code == twa.TWA_ERR_NONFINITE and 8 <= detail <= 15      # reported for the panel that holds it
+    twa.twa_clear_status(ctx)
