@@ -4,9 +4,9 @@
 // per column.
 //     C = Q^T A_p        (twa_launch_panel_project)   Q: columns 0 .. nq-1, A_p: columns nq .. nq+pb-1
 //     A_p <- A_p - Q C   (twa_launch_panel_lift)
-// The projection streams tiles of 64 rows x (nq + pb) columns of the float32 matrix through a TMA
+// The projection streams tiles of 128 rows x (nq + pb) columns of the float32 matrix through a TMA
 // ring (one box per stage: the panel's columns are simply the last columns of the tile).
-//  * projection: warp w owns columns w, w+16, ...; a lane owns 2 rows; 8 x 8 accumulators per lane;
+//  * projection: warp w owns columns w, w+16, ...; a lane owns 4 rows; 8 x 8 accumulators per lane;
 //    lanes -> block -> last block to finish, float64 over blocks in block order.
 //  * update: a lane owns one row of a block of 512 rows and walks all nq columns as they stream past
 //    in chunks of 8, so there is no reduction at all.
@@ -17,7 +17,7 @@
 namespace {
 
 constexpr int PANEL = 8;                         // columns per panel at most
-constexpr int PROWS = 64;                        // rows per tile
+constexpr int PROWS = 128;                       // rows per tile of the projection
 constexpr int PCOL_BYTES = PROWS * 4;
 constexpr int PWARPS = 16;                       // consumer warps
 constexpr int PTHREADS = (PWARPS + 1) * 32;
@@ -105,16 +105,22 @@ panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a)
         break;
       }
       const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
-      float2 g[PANEL];
 #pragma unroll
-      for (int q = 0; q < PANEL; ++q)
-        g[q] = q < a.pb ? *reinterpret_cast<const float2*>(st + (a.nq + q) * PCOL_BYTES + lane * 8) : make_float2(0.f, 0.f);
+      for (int half = 0; half < 2; ++half) {             // four panel columns at a time (registers)
+        float4 g[4];
 #pragma unroll
-      for (int k = 0; k < MAX_Q_PER_WARP; ++k) {
-        if (k < cpw) {
-          const float2 p = *reinterpret_cast<const float2*>(st + (warp + k * PWARPS) * PCOL_BYTES + lane * 8);
+        for (int q = 0; q < 4; ++q)
+          g[q] = half * 4 + q < a.pb ? *reinterpret_cast<const float4*>(st + (a.nq + half * 4 + q) * PCOL_BYTES + lane * 16)
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-          for (int q = 0; q < PANEL; ++q) acc[k][q] = fmaf(p.x, g[q].x, fmaf(p.y, g[q].y, acc[k][q]));
+        for (int k = 0; k < MAX_Q_PER_WARP; ++k) {
+          if (k < cpw) {
+            const float4 p = *reinterpret_cast<const float4*>(st + (warp + k * PWARPS) * PCOL_BYTES + lane * 16);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              acc[k][half * 4 + q] =
+                  fmaf(p.x, g[q].x, fmaf(p.y, g[q].y, fmaf(p.z, g[q].z, fmaf(p.w, g[q].w, acc[k][half * 4 + q]))));
+          }
         }
       }
       __syncwarp();
