@@ -398,6 +398,48 @@ twa_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LiftArgs a) {
   if (*abort_flag && tid == 0) twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
 }
 
+// ---- lift on a float32 basis ---------------------------------------------------------------------
+// out[r] = base[r] + sum_j (alpha_j * mult) P_j[r]: a thread owns four consecutive rows and walks the
+// columns in index order, products and sums in float64 (the sum is rounded once).  No shared-memory
+// staging: every byte is used once and consecutive threads read consecutive 16-byte pieces of a column.
+constexpr int LIFT32_BLOCK = 256;
+
+__global__ void __launch_bounds__(LIFT32_BLOCK)
+twa_lift32_kernel(const float* __restrict__ P, long long ld, int n, const float* __restrict__ alpha, float mult,
+                  const float* base, float* out, long long D, int* status) {
+  __shared__ float coef[TWA_MAX_N];
+  if (threadIdx.x < n) {
+    const float c = alpha[threadIdx.x] * mult;
+    if (!isfinite(c) && blockIdx.x == 0) twa_set_status(status, TWA_ERR_NONFINITE, -1);
+    coef[threadIdx.x] = c;
+  }
+  __syncthreads();
+  const long long nvec = D >> 2;
+  for (long long v = blockIdx.x * static_cast<long long>(LIFT32_BLOCK) + threadIdx.x; v < nvec;
+       v += static_cast<long long>(gridDim.x) * LIFT32_BLOCK) {
+    double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+    if (base) {
+      const float4 b = reinterpret_cast<const float4*>(base)[v];
+      s0 = b.x; s1 = b.y; s2 = b.z; s3 = b.w;
+    }
+#pragma unroll 8
+    for (int j = 0; j < n; ++j) {
+      const float4 x = __ldcs(reinterpret_cast<const float4*>(P + j * ld) + v);
+      const double c = coef[j];
+      s0 = fma(c, static_cast<double>(x.x), s0); s1 = fma(c, static_cast<double>(x.y), s1);
+      s2 = fma(c, static_cast<double>(x.z), s2); s3 = fma(c, static_cast<double>(x.w), s3);
+    }
+    reinterpret_cast<float4*>(out)[v] = make_float4(static_cast<float>(s0), static_cast<float>(s1),
+                                                    static_cast<float>(s2), static_cast<float>(s3));
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (D & 3)) {
+    const long long r = (nvec << 2) + threadIdx.x;
+    double s = base ? static_cast<double>(base[r]) : 0.0;
+    for (int j = 0; j < n; ++j) s = fma(static_cast<double>(coef[j]), static_cast<double>(P[j * ld + r]), s);
+    out[r] = static_cast<float>(s);
+  }
+}
+
 // ---- host side ----------------------------------------------------------------------------
 int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
@@ -586,6 +628,17 @@ int twa_launch_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, float 
                     const float* base, float* out, bool reverse_tiles) {
   if (P->bits != 32 && ctx->tune_dequant_path == 0)
     return twa_launch_lift_mma(ctx, P, alpha, alpha_mult, base, out, reverse_tiles);
+  if (P->bits == 32) {
+    const long long nvec = P->D >> 2;
+    long long g = (nvec + LIFT32_BLOCK - 1) / LIFT32_BLOCK;
+    const long long cap = static_cast<long long>(ctx->sm_count) * 8;
+    if (g > cap) g = cap;
+    if (g < 1) g = 1;
+    twa_lift32_kernel<<<static_cast<int>(g), LIFT32_BLOCK, 0, ctx->stream>>>(
+        static_cast<const float*>(P->data), P->col_stride / 4, P->n, alpha, alpha_mult, base, out, P->D, ctx->d_status);
+    TWA_CUDA_OK(ctx, cudaGetLastError());
+    return TWA_OK;
+  }
   const int rows = twa_tile_rows(P->bits);
   CUtensorMap mp;
   int rc = encode_basis_map(ctx, P, &mp);
