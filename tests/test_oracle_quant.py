@@ -99,7 +99,7 @@ def test_storage_accounting_against_the_papers_tables():
     assert abs(orc.paper_storage_bytes(D, n, 32) - extra_fp32) / extra_fp32 < 0.05
     assert abs(orc.paper_storage_bytes(D, n, 4, L=161) - extra_q4) / extra_q4 < 0.05
     assert abs(extra_fp32 / extra_q4 - 8.0) < 1e-9                  # "around 8x"
-    # this build's per-column format: same code bytes, 4n instead of 8L for the factors
+    # the per-column format: same code bytes, 4n instead of 8L for the factors
     assert orc.storage_bytes(D, n, 32) == 4 * n * D
     assert orc.storage_bytes(D, n, 4) == n * D // 2 + 4 * n
     assert orc.storage_bytes(D, n, 8) == n * D + 4 * n
