@@ -228,6 +228,7 @@ def run_ours(args):
     g_bytes = 2 if wl.g_dtype == "bf16" else 4
     ctx = twa.twa_create(local)
     twa.twa_set_tuning(ctx, twa.TWA_TUNE_DEQUANT_PATH, args.dequant_path)
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_LIFT_VECTORS, args.lift_vectors)
     ws = twa.new_workspace(dev)
 
     # ---- basis build and quantisation, timed once each -------------------------------
@@ -606,6 +607,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--reference-rows", type=int, default=1 << 21)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--lift-vectors", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="TWA_TUNE_LIFT_VECTORS: how base and output travel in the 8/4-bit lift (0 = built-in choice)")
     ap.add_argument("--dequant-path", type=int, default=0, choices=[0, 1],
                     help="0: integer dot products on the tensor pipe (default); 1: float32 FMA path")
     ap.add_argument("--rows", type=int, default=0, help="override D (smaller cases for profiler captures)")

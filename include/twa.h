@@ -111,10 +111,15 @@ const char* twa_last_error(const twa_ctx* ctx);
  *      float path and on 32-bit bases only.
  *  TWA_TUNE_TILE_SEGMENTS: tensor-pipe path, 512-byte segments of a column per tile: 1 or 2
  *      (default: 2 for n <= 64, else 1).
- *  TWA_TUNE_BUILD_PANEL: twa_build_basis: 0 = panels of 8 columns (default), 1 = column by column. */
+ *  TWA_TUNE_BUILD_PANEL: twa_build_basis: 0 = panels of 8 columns (default), 1 = column by column.
+ *  TWA_TUNE_LIFT_VECTORS: lift on 8/4-bit codes, how the rows of `base` and of `w_out` travel:
+ *      1 = every lane loads and stores its own rows; 2 = `base` comes through the shared-memory
+ *      ring beside the codes; 3 = as 2, and the results leave through bulk stores from shared
+ *      memory; 0 = built-in choice by the share of the two vectors in the bytes moved
+ *      (n * bits <= 192: 2, <= 320: 3, else 1). */
 enum { TWA_TUNE_PROJECT_WARPS = 1, TWA_TUNE_LIFT_WARPS = 2, TWA_TUNE_STAGES = 3,
        TWA_TUNE_WAIT_LIMIT_MS = 4, TWA_TUNE_DEQUANT_PATH = 5, TWA_TUNE_TILE_SEGMENTS = 6,
-       TWA_TUNE_BUILD_PANEL = 7 };
+       TWA_TUNE_BUILD_PANEL = 7, TWA_TUNE_LIFT_VECTORS = 8 };
 int twa_set_tuning(twa_ctx* ctx, int key, int value);
 
 /* Exercises the bounded wait every streaming kernel uses, without any fault: enqueues one block

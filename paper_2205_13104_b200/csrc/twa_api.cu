@@ -169,6 +169,10 @@ int twa_set_tuning(twa_ctx* ctx, int key, int value) {
       if (value > 1) return TWA_ERR_INVALID_ARG;
       ctx->tune_build_panel = value;
       return TWA_OK;
+    case TWA_TUNE_LIFT_VECTORS:
+      if (value > 3) return TWA_ERR_INVALID_ARG;
+      ctx->tune_lift_base_path = value;
+      return TWA_OK;
     case TWA_TUNE_DEQUANT_PATH:
       if (value > 1) return TWA_ERR_INVALID_ARG;
       ctx->tune_dequant_path = value;

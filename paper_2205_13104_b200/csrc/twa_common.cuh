@@ -30,6 +30,7 @@ struct twa_ctx {
   int tune_dequant_path;      // 0 = integer tensor-pipe dot products, 1 = float FMA
   int tune_tile_segments;     // tensor-pipe path: 512-byte segments per tile column (0 = choose)
   int tune_build_panel;       // resident basis build: 0 = panels of 8 columns, 1 = column by column
+  int tune_lift_base_path;    // tensor-pipe lift, base / output vectors: 0 = choose, 1 = lanes, 2 = base through the ring, 3 = both
   cudaEvent_t* prof_events;   // 3 per recorded step, or null
   int prof_cap, prof_count;   // steps
   // state of a row-chunked basis build (twa_build_begin .. twa_build_end_pass)
@@ -183,6 +184,27 @@ __device__ __forceinline__ void twa_tma_load_1d(uint32_t dst, const CUtensorMap*
       "cp.async.bulk.tensor.1d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2}], [%3];"
       ::"r"(dst), "l"(map), "r"(x), "r"(bar)
       : "memory");
+}
+
+// Bulk tensor store from this block's shared memory, clipped by the tensor map; completion is
+// tracked by the issuing thread's bulk async-group.
+__device__ __forceinline__ void twa_tma_store_1d(const CUtensorMap* map, int x, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.1d.global.shared::cta.bulk_group [%0, {%1}], [%2];"
+               ::"l"(map), "r"(x), "r"(src)
+               : "memory");
+}
+
+__device__ __forceinline__ void twa_bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+
+// Waits until all but the newest N bulk groups of this thread have finished reading shared memory.
+template <int N>
+__device__ __forceinline__ void twa_bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+
+// Orders this thread's earlier shared-memory writes before later reads by the bulk-copy engine.
+__device__ __forceinline__ void twa_fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
 __device__ __forceinline__ void twa_prefetch_tensormap(const CUtensorMap* map) {

@@ -53,6 +53,7 @@ struct LiftMmaArgs {
   int n, stages, tiles;
   int kt;                      // 512-byte segments of a column per tile (1 or 2)
   unsigned stage_bytes, tx_bytes, table_off;
+  unsigned base_off;           // offset of the tile's rows of the base vector inside a stage (BTMA)
   const float* scales;
   const float* alpha;
   float alpha_mult;
@@ -281,9 +282,19 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
 // lift
 // =================================================================================================
 // KS = number of 32-column steps, ceil(n / 32), a compile-time constant.
-template <int BITS, int KS, int KT>
+// VEC says how the rows of the base vector and of the output travel:
+//   0  every lane loads its base rows and stores its results itself;
+//   1  the tile's base rows ride the ring beside the codes (1-D boxes of 256 floats, zero past D),
+//      so their latency is hidden by the depth of the ring and not by one tile of look-ahead;
+//   2  as 1, and the results are written over the base rows in the stage and leave through one
+//      bulk tensor store per warp and tile (clipped at D by the tensor map); the stage is handed
+//      back one tile later, once that store has read it.
+// 1 and 2 need 16-byte aligned vectors.
+template <int BITS, int KS, int KT, int VEC>
 __global__ void __launch_bounds__(MMA_THREADS, 1)
-twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs a) {
+twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_b,
+                    const __grid_constant__ CUtensorMap map_o, const LiftMmaArgs a) {
+  constexpr bool BTMA = VEC >= 1, STMA = VEC == 2;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
   constexpr int ROWS = twa_tile_rows(BITS);
@@ -318,11 +329,11 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
 
   if (warp == MMA_WARPS) {
     if (lane == 0)
-      producer_loop_mma(hdr, ring, &map_p, nullptr, blockIdx.x, gridDim.x,
+      producer_loop_mma(hdr, ring, &map_p, &map_b, blockIdx.x, gridDim.x,
                         (a.tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
                             static_cast<int>(gridDim.x),
-                        a.stages, a.stage_bytes, KT, 0, 0, 0, 0, a.tx_bytes, a.reverse != 0, a.status,
-                        a.wait_limit_ns);
+                        a.stages, a.stage_bytes, KT, BTMA ? ROWS * KT / 256 : 0, 4, ROWS * KT, a.base_off,
+                        a.tx_bytes, a.reverse != 0, a.status, a.wait_limit_ns);
     return;
   }
   if (bad && tid == 0) twa_set_status(a.status, TWA_ERR_NONFINITE, -1);
@@ -390,7 +401,7 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
     for (int u = 0; u < KT; ++u) {
 #pragma unroll
       for (int i = 0; i < LROWS; ++i) bv[u][i] = 0.0f;
-      if (a.base && tig < 2) {
+      if (!BTMA && a.base && tig < 2) {
         const int row = tile_row0 + lane_row[u];
         if (whole || row <= D - LROWS) {
           if (LROWS == 2) {
@@ -412,6 +423,19 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
       break;
     }
     const uint32_t tile_base = twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes);
+    if (BTMA && tig < 2) {
+      const float* sb = reinterpret_cast<const float*>(ring + static_cast<size_t>(s) * a.stage_bytes + a.base_off);
+#pragma unroll
+      for (int u = 0; u < KT; ++u) {
+        if (LROWS == 2) {
+          const float2 x = *reinterpret_cast<const float2*>(sb + lane_row[u]);
+          bv[u][0] = x.x; bv[u][1] = x.y;
+        } else {
+          const float4 x = *reinterpret_cast<const float4*>(sb + lane_row[u]);
+          bv[u][0] = x.x; bv[u][1] = x.y; bv[u][2] = x.z; bv[u][3] = x.w;
+        }
+      }
+    }
     float keep[KT][LROWS];
 #pragma unroll
     for (int u = 0; u < KT; ++u) {
@@ -467,6 +491,51 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
         }
       }
     }
+    if (STMA) {
+      float* sb = reinterpret_cast<float*>(ring + static_cast<size_t>(s) * a.stage_bytes + a.base_off);
+      if (tig < 2) {
+#pragma unroll
+        for (int u = 0; u < KT; ++u) {
+          if (LROWS == 2) {
+            *reinterpret_cast<float2*>(sb + lane_row[u]) =
+                make_float2(bv[u][0] + keep[u][0] + poison, bv[u][1] + keep[u][1] + poison);
+          } else {
+            *reinterpret_cast<float4*>(sb + lane_row[u]) =
+                make_float4(bv[u][0] + keep[u][0] + poison, bv[u][1] + keep[u][1] + poison,
+                            bv[u][2] + keep[u][2] + poison, bv[u][3] + keep[u][3] + poison);
+          }
+        }
+        twa_fence_proxy_async();                          // the lanes' writes, before the bulk store reads them
+        // The bulk store clips in units of 16 bytes, so its tensor map ends at the last multiple of
+        // four rows; the up to three rows after that are stored by the lanes that own them.
+        if (!whole) {
+#pragma unroll
+          for (int u = 0; u < KT; ++u)
+#pragma unroll
+            for (int i = 0; i < LROWS; ++i) {
+              const int row = tile_row0 + lane_row[u] + i;
+              if (row >= (D & ~3) && row < D) a.out[row] = bv[u][i] + keep[u][i] + poison;
+            }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) {
+        // the warp's rows of the tile are contiguous: [warp * KT * 32 * (8 / BITS), + KT * 32 * (8 / BITS))
+        constexpr int wrows = KT * 32 * (8 / BITS);
+        if (tile_row0 + warp * wrows < (D & ~3))          // no store starts past the end of the map
+          twa_tma_store_1d(&map_o, tile_row0 + warp * wrows, twa_smem_u32(sb + warp * wrows));
+        twa_bulk_commit();
+        if (k > 0) {                                      // the previous tile's store has read its stage
+          twa_bulk_wait_read<1>();
+          twa_mbar_arrive(twa_smem_u32(&hdr->empty[s == 0 ? a.stages - 1 : s - 1]));
+        }
+      }
+      if (++s == a.stages) {
+        s = 0;
+        phase ^= 1u;
+      }
+      continue;
+    }
     __syncwarp();
     if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
 #pragma unroll
@@ -494,6 +563,7 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const LiftMmaArgs
       phase ^= 1u;
     }
   }
+  if (STMA && lane == 0) twa_bulk_wait_read<0>();         // shared memory must outlive the stores' reads
 }
 
 // =================================================================================================
@@ -559,13 +629,17 @@ template <int BITS, bool GBF16>
 int launch_project_mma_mt(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg,
                           const ProjectMmaArgs& a, int grid, int smem);
 
-template <int BITS, int KS>
-int launch_lift_mma_t(twa_ctx* ctx, const CUtensorMap& mp, const LiftMmaArgs& a, int grid, int smem) {
-  auto kern = a.kt == 2 ? twa_lift_mma_kernel<BITS, KS, 2> : twa_lift_mma_kernel<BITS, KS, 1>;
+struct LiftMaps {
+  CUtensorMap p, b, o;
+};
+
+template <int BITS, int KS, int VEC>
+int launch_lift_mma_t(twa_ctx* ctx, const LiftMaps& m, const LiftMmaArgs& a, int grid, int smem) {
+  auto kern = a.kt == 2 ? twa_lift_mma_kernel<BITS, KS, 2, VEC> : twa_lift_mma_kernel<BITS, KS, 1, VEC>;
   static int smem_limit[2][64] = {{0}};   // per tile height and device
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[a.kt - 1][ctx->device & 63], smem);
   if (rc) return rc;
-  kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, a);
+  kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(m.p, m.b, m.o, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
 }
@@ -585,14 +659,40 @@ int launch_project_mma_mt(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap
   }
 }
 
-template <int BITS>
-int launch_lift_mma_ks(twa_ctx* ctx, const CUtensorMap& mp, const LiftMmaArgs& a, int grid, int smem) {
+template <int BITS, int VEC>
+int launch_lift_mma_ks(twa_ctx* ctx, const LiftMaps& m, const LiftMmaArgs& a, int grid, int smem) {
   switch ((a.n + 31) >> 5) {
-    case 1: return launch_lift_mma_t<BITS, 1>(ctx, mp, a, grid, smem);
-    case 2: return launch_lift_mma_t<BITS, 2>(ctx, mp, a, grid, smem);
-    case 3: return launch_lift_mma_t<BITS, 3>(ctx, mp, a, grid, smem);
-    default: return launch_lift_mma_t<BITS, 4>(ctx, mp, a, grid, smem);
+    case 1: return launch_lift_mma_t<BITS, 1, VEC>(ctx, m, a, grid, smem);
+    case 2: return launch_lift_mma_t<BITS, 2, VEC>(ctx, m, a, grid, smem);
+    case 3: return launch_lift_mma_t<BITS, 3, VEC>(ctx, m, a, grid, smem);
+    default: return launch_lift_mma_t<BITS, 4, VEC>(ctx, m, a, grid, smem);
   }
+}
+
+template <int BITS>
+int launch_lift_mma_vec(twa_ctx* ctx, const LiftMaps& m, const LiftMmaArgs& a, int grid, int smem, int vec) {
+  switch (vec) {
+    case 2: return launch_lift_mma_ks<BITS, 2>(ctx, m, a, grid, smem);
+    case 1: return launch_lift_mma_ks<BITS, 1>(ctx, m, a, grid, smem);
+    default: return launch_lift_mma_ks<BITS, 0>(ctx, m, a, grid, smem);
+  }
+}
+
+// 1-D tensor map over a float vector of D elements with boxes of `box` elements
+int encode_vector_map(twa_ctx* ctx, const float* v, long long D, int box, CUtensorMap* map) {
+  cuuint64_t dims[1] = {static_cast<cuuint64_t>(D)};
+  cuuint64_t strides[1] = {0};
+  cuuint32_t bx[1] = {static_cast<cuuint32_t>(box)};
+  cuuint32_t es[1] = {1};
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 1, const_cast<float*>(v), dims, strides, bx, es,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(ctx->last_error, sizeof(ctx->last_error), "cuTensorMapEncodeTiled(vector) failed: %d",
+             static_cast<int>(r));
+    return TWA_ERR_CUDA;
+  }
+  return TWA_OK;
 }
 
 }  // namespace
@@ -659,7 +759,35 @@ int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, fl
   a.n = P->n;
   a.tiles = static_cast<int>((P->D + rows - 1) / rows);
   a.kt = kt;
-  a.tx_bytes = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt;
+  // How base and output travel (see the kernel): through the ring and bulk stores when tensor maps
+  // can describe them (16-byte aligned starts) and the two vectors are a large share of the bytes
+  // moved, 64 / (n * bits + 64).  Measured on B200: a third (n = 16 at 8 bits, n = 32 at 4 bits): base
+  // through the ring 6.6 / 6.3 TB/s against 4.3 / 5.5 with the lanes' own loads, bulk stores in between;
+  // a fifth (n = 32 at 8 bits): ring and bulk stores 6.7 against 6.45 (ring alone) and 6.3 (lanes);
+  // a seventh and less (n >= 50 at 8 bits): the lanes' loads are hidden behind the wait for the codes
+  // and the ring alone costs 3-4 %.
+  const int nb = P->n * P->bits;
+  int vec = ctx->tune_lift_base_path == 0 ? (nb <= 192 ? 1 : (nb <= 320 ? 2 : 0)) : ctx->tune_lift_base_path - 1;
+  if (base == nullptr || ((reinterpret_cast<uintptr_t>(base) | reinterpret_cast<uintptr_t>(out)) & 15u) != 0) vec = 0;
+  const bool btma = vec >= 1;
+  LiftMaps maps;
+  maps.p = mp;
+  maps.b = mp;
+  maps.o = mp;
+  if (btma) {
+    rc = encode_vector_map(ctx, base, P->D, 256, &maps.b);
+    if (rc) return rc;
+  }
+  if (vec == 2) {
+    if (P->D < 4) vec = 1;                                // nothing for a bulk store to write
+  }
+  if (vec == 2) {
+    // rows [D & ~3, D) are stored by the lanes: a bulk store clips in units of 16 bytes
+    rc = encode_vector_map(ctx, out, P->D & ~3ll, kt * 32 * (8 / P->bits), &maps.o);
+    if (rc) return rc;
+  }
+  a.base_off = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt;
+  a.tx_bytes = a.base_off + (btma ? static_cast<unsigned>(rows) * 4u : 0u);
   a.stage_bytes = static_cast<unsigned>(round_up_i(static_cast<int>(a.tx_bytes), 1024));
   const int fixed = TWA_SMEM_HEADER + 4 * TWA_MAX_N + 1024;               // 1024: alignment slack
   int stages = (ctx->smem_optin - fixed) / static_cast<int>(a.stage_bytes);
@@ -678,6 +806,6 @@ int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, fl
   a.wait_limit_ns = ctx->wait_limit_ns;
   const int grid = ctx->sm_count < a.tiles ? ctx->sm_count : a.tiles;
   const int smem = static_cast<int>(a.table_off) + 4 * TWA_MAX_N + 1024;
-  return P->bits == 8 ? launch_lift_mma_ks<8>(ctx, mp, a, grid, smem)
-                      : launch_lift_mma_ks<4>(ctx, mp, a, grid, smem);
+  return P->bits == 8 ? launch_lift_mma_vec<8>(ctx, maps, a, grid, smem, vec)
+                      : launch_lift_mma_vec<4>(ctx, maps, a, grid, smem, vec);
 }

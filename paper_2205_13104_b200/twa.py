@@ -38,6 +38,7 @@ TWA_TUNE_WAIT_LIMIT_MS = 4
 TWA_TUNE_DEQUANT_PATH = 5
 TWA_TUNE_TILE_SEGMENTS = 6
 TWA_TUNE_BUILD_PANEL = 7
+TWA_TUNE_LIFT_VECTORS = 8
 
 EXPORTS = [
     "twa_create", "twa_destroy", "twa_get_status", "twa_clear_status", "twa_strerror",
@@ -85,24 +86,52 @@ class TwaError(RuntimeError):
         super().__init__(msg)
 
 
+def _nvcc():
+    return os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+
+
+NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+              "-Xcompiler", "-fPIC", "-I", os.path.join(_ROOT, "include")]
+
+
 def build_command(out=LIB_PATH):
-    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    return [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(_ROOT, "include"),
-            "-o", out] + [os.path.join(CSRC, s) for s in SOURCES]
+    """The one-line form of the build (every source in one nvcc call)."""
+    return [_nvcc()] + NVCC_FLAGS + ["-shared", "-o", out] + [os.path.join(CSRC, s) for s in SOURCES]
 
 
 def build_library(force=False, verbose=False):
     """Compiles the CUDA library for sm_100a next to this file (nvcc cross-compiles without
-    a GPU).  Skipped when the library is newer than every source."""
+    a GPU): one object per source, compiled side by side, then one link.  Skipped when the
+    library is newer than every source; an object is reused while it is newer than every
+    source and header."""
+    from concurrent.futures import ThreadPoolExecutor
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(_ROOT, "include", "twa.h")]
-    if not force and os.path.exists(LIB_PATH) and \
-            all(os.path.getmtime(LIB_PATH) >= os.path.getmtime(d) for d in deps):
+    newest = max(os.path.getmtime(d) for d in deps)
+    if not force and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= newest:
         return LIB_PATH
-    cmd = build_command()
+    obj_dir = os.path.join(_HERE, "_build")
+    os.makedirs(obj_dir, exist_ok=True)
+    headers = [d for d in deps if not d.endswith(".cu")]
+    newest_header = max(os.path.getmtime(h) for h in headers)
+
+    def compile_one(src):
+        obj = os.path.join(obj_dir, os.path.splitext(src)[0] + ".o")
+        path = os.path.join(CSRC, src)
+        if not force and os.path.exists(obj) and \
+                os.path.getmtime(obj) >= max(os.path.getmtime(path), newest_header):
+            return obj
+        cmd = [_nvcc()] + NVCC_FLAGS + ["-c", path, "-o", obj]
+        if verbose:
+            print(" ".join(cmd), flush=True)
+        subprocess.run(cmd, check=True)
+        return obj
+
+    with ThreadPoolExecutor(max_workers=min(len(SOURCES), os.cpu_count() or 1)) as pool:
+        objs = list(pool.map(compile_one, SOURCES))
+    link = [_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB_PATH] + objs
     if verbose:
-        print(" ".join(cmd))
-    subprocess.run(cmd, check=True)
+        print(" ".join(link), flush=True)
+    subprocess.run(link, check=True)
     return LIB_PATH
 
 

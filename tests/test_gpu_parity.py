@@ -474,6 +474,37 @@ def test_tile_segments_knob(env, D, n, bits, segments):
         twa.twa_set_tuning(ctx, twa.TWA_TUNE_TILE_SEGMENTS, 0)
 
 
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("D,n", [(1, 1), (4099, 33), (70001, 100), (131075, 8), (600001, 32)])
+def test_lift_vectors_knob(env, D, n, bits):
+    """The lift's ways of moving `base` and the output (loaded and stored by the lanes, or through
+    the shared-memory ring and bulk stores) do the same arithmetic: identical bits, all matching the oracle."""
+    ctx, ws = env
+    P = random_basis(D, n, 1700 + D + n)
+    B = twa.twa_quantize_basis(ctx, twa.basis_from_tensor(P, D), bits, ws)
+    codes, s = twa.twa_basis_export(ctx, B)
+    co, so = orc.unpack_codes(codes.cpu().numpy(), D, bits), s.cpu().numpy()
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(D + 3 * n + bits)
+    alpha = torch.randn(n, generator=gen, device=DEV)
+    base = torch.randn(D + 8, generator=gen, device=DEV)
+    base[D:] = float("nan")                         # must never reach the output
+    out = []
+    try:
+        for mode in (1, 2, 3):
+            twa.twa_set_tuning(ctx, twa.TWA_TUNE_LIFT_VECTORS, mode)
+            w = torch.full((D + 8,), 5.0, device=DEV)
+            twa.twa_lift(ctx, B, alpha, base[:D], w, ws)
+            status_ok(ctx)
+            assert torch.all(w[D:] == 5.0)
+            out.append(w[:D].clone())
+    finally:
+        twa.twa_set_tuning(ctx, twa.TWA_TUNE_LIFT_VECTORS, 0)
+    assert torch.equal(out[0], out[1]) and torch.equal(out[0], out[2])
+    w_ref = orc.lift(co, so, alpha.cpu().numpy(), base[:D].cpu().numpy())
+    assert rel(out[0].cpu().numpy(), w_ref) <= TOL
+
+
 def test_bounded_wait_runs_out_cleanly_and_the_context_stays_usable(env):
     """A wait that nothing satisfies ends after its limit with a status, not a hang or a fault."""
     ctx, ws = env
