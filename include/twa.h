@@ -111,7 +111,9 @@ const char* twa_last_error(const twa_ctx* ctx);
  *      float path and on 32-bit bases only.
  *  TWA_TUNE_TILE_SEGMENTS: tensor-pipe path, 512-byte segments of a column per tile: 1 or 2
  *      (default: 2 for n <= 64, else 1).
- *  TWA_TUNE_BUILD_PANEL: twa_build_basis: 0 = panels of 8 columns (default), 1 = column by column.
+ *  TWA_TUNE_BUILD_PANEL: twa_build_basis: 0 = panels of 8 columns, the Gram-Schmidt coefficients
+ *      inside a panel taken from the panel's Gram matrix (default); 1 = column by column;
+ *      2 = panels of 8 columns with column-by-column sweeps inside a panel.
  *  TWA_TUNE_LIFT_VECTORS: lift on 8/4-bit codes, how the rows of `base` and of `w_out` travel:
  *      1 = every lane loads and stores its own rows; 2 = `base` comes through the shared-memory
  *      ring beside the codes; 3 = as 2, and the results leave through bulk stores from shared

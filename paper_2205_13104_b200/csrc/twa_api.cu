@@ -166,7 +166,7 @@ int twa_set_tuning(twa_ctx* ctx, int key, int value) {
       ctx->tune_tile_segments = value;
       return TWA_OK;
     case TWA_TUNE_BUILD_PANEL:
-      if (value > 1) return TWA_ERR_INVALID_ARG;
+      if (value > 2) return TWA_ERR_INVALID_ARG;
       ctx->tune_build_panel = value;
       return TWA_OK;
     case TWA_TUNE_LIFT_VECTORS:

@@ -443,8 +443,8 @@ int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float
     }
   } else {
     // Panels of up to 8 columns.  Twice: remove the earlier basis vectors from the whole panel in one
-    // pass over them (projection of the panel, then update), then sweep and normalise the panel's
-    // columns among themselves.  The first round makes the panel orthonormal up to the rounding its
+    // pass over them (projection of the panel, then update), then orthonormalise the panel's columns
+    // among themselves (Gram form, or column sweeps and normalisations with TWA_TUNE_BUILD_PANEL = 2).  The first round makes the panel orthonormal up to the rounding its
     // cancellation amplifies; the second round, applied to unit vectors, removes that.
     for (int j0 = 0; j0 < n; j0 += width) {
       const int pb = n - j0 < width ? n - j0 : width;
@@ -458,6 +458,15 @@ int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float
           if (rc) return rc;
           rc = twa_launch_panel_lift(ctx, W, D, ldw, j0, pb, ws);
           if (rc) return rc;
+        }
+        if (ctx->tune_build_panel == 0) {
+          // Gram form inside the panel: all coefficients of the panel's own Gram-Schmidt from its
+          // Gram matrix in one pass, the new columns in a second; in the second round the rank test
+          // compares against the columns' norms as this round found them (1, or 0 for a column
+          // already found dependent).
+          rc = twa_launch_panel_gram(ctx, W, D, ldw, j0, pb, ws, given, round == 1);
+          if (rc) return rc;
+          continue;
         }
         for (int q = 0; q < pb; ++q) {
           const int k = j0 + q;

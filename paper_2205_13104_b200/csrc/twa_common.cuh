@@ -29,7 +29,7 @@ struct twa_ctx {
   int tune_project_warps, tune_lift_warps, tune_stages;
   int tune_dequant_path;      // 0 = integer tensor-pipe dot products, 1 = float FMA
   int tune_tile_segments;     // tensor-pipe path: 512-byte segments per tile column (0 = choose)
-  int tune_build_panel;       // resident basis build: 0 = panels of 8 columns, 1 = column by column
+  int tune_build_panel;       // resident basis build: 0 = panels of 8 columns, Gram form inside; 1 = column by column; 2 = panels, column sweeps inside
   int tune_lift_base_path;    // tensor-pipe lift, base / output vectors: 0 = choose, 1 = lanes, 2 = base through the ring, 3 = both
   cudaEvent_t* prof_events;   // 3 per recorded step, or null
   int prof_cap, prof_count;   // steps
@@ -287,6 +287,10 @@ int twa_check_basis(const twa_basis* P);
 // C = Q^T A_p into the workspace, then A_p <- A_p - Q C; Q = columns 0..nq-1, A_p = the next pb <= 8.
 int twa_launch_panel_project(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws);
 int twa_launch_panel_lift(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws);
+// Gram-Schmidt among the panel's own columns in Gram form: the coefficients from the panel's Gram
+// matrix (one pass), then A_p <- A_p T (one pass); rank and finiteness tests against `given`.
+int twa_launch_panel_gram(twa_ctx* ctx, float* W, long long D, long long ldw, int j0, int pb, void* ws, double* given,
+                          bool given_from_diagonal);
 // Validates the optimiser constants and fills the kernel-side Adam arguments (bias corrections for opt->step).
 int twa_adam_device_args(const twa_adam* opt, float* m, float* v, twa_adam_args* out);
 // scales[j] = absmax_j / qmax from the bit patterns of the column maxima; flags NaN/Inf

@@ -282,6 +282,172 @@ panel_lift_kernel(const __grid_constant__ CUtensorMap map, const PanelLiftArgs a
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Gram form of the sweeps inside a panel.  Gram-Schmidt on the panel's columns a_0 .. a_{pb-1} gives
+// q_j = (a_j - sum_{k<j} r_kj q_k) / r_jj with r_kj = <q_k, a_j>; every q_k is a combination of the
+// a's, so all r_kj follow from the panel's Gram matrix G = A_p^T A_p: they are the entries of its
+// Cholesky factor, and Q_p = A_p T with T = R^-1 upper triangular.  One pass takes the 36 dot
+// products <a_i, a_j> (float64 products and sums, warp shuffles, blocks combined in block order);
+// the block that finishes last factorises G in float64, applies the rank and finiteness tests of
+// the column-by-column schedule (r_jj <= 1e-5 |a_j| as given: the column becomes zero and is
+// reported) and leaves T; a second pass writes A_p T.  Twelve column passes per panel and round
+// instead of the 52 of the column sweeps.
+constexpr int GRAM_BLOCK = 256;
+constexpr int NPAIR = PANEL * (PANEL + 1) / 2;                     // 36
+__host__ __device__ constexpr int pair_index(int i, int j) { return j * (j + 1) / 2 + i; }   // i <= j
+
+__global__ void __launch_bounds__(GRAM_BLOCK) panel_gram_kernel(const float* __restrict__ A0, long long ld, int pb,
+                                                               long long D, double* __restrict__ gpart,
+                                                               double* __restrict__ given, int given_from_diagonal,
+                                                               double* __restrict__ T, unsigned* __restrict__ ticket,
+                                                               int* status, int col0) {
+  __shared__ double sh[NPAIR][GRAM_BLOCK / 32];
+  __shared__ double G[NPAIR];
+  __shared__ int last;
+  double s[NPAIR];
+#pragma unroll
+  for (int p = 0; p < NPAIR; ++p) s[p] = 0.0;
+  const long long nvec = D >> 2;
+  for (long long t = blockIdx.x * static_cast<long long>(GRAM_BLOCK) + threadIdx.x; t < nvec;
+       t += static_cast<long long>(gridDim.x) * GRAM_BLOCK) {
+    float4 x[PANEL];
+#pragma unroll
+    for (int j = 0; j < PANEL; ++j)
+      x[j] = j < pb ? __ldcs(reinterpret_cast<const float4*>(A0 + j * ld) + t) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int comp = 0; comp < 4; ++comp) {
+      double v[PANEL];
+#pragma unroll
+      for (int j = 0; j < PANEL; ++j)
+        v[j] = static_cast<double>(comp == 0 ? x[j].x : comp == 1 ? x[j].y : comp == 2 ? x[j].z : x[j].w);
+#pragma unroll
+      for (int j = 0; j < PANEL; ++j)
+#pragma unroll
+        for (int i = 0; i <= j; ++i) s[pair_index(i, j)] = fma(v[i], v[j], s[pair_index(i, j)]);
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (D & 3)) {
+    const long long r = (nvec << 2) + threadIdx.x;
+    double v[PANEL];
+#pragma unroll
+    for (int j = 0; j < PANEL; ++j) v[j] = j < pb ? static_cast<double>(A0[j * ld + r]) : 0.0;
+#pragma unroll
+    for (int j = 0; j < PANEL; ++j)
+#pragma unroll
+      for (int i = 0; i <= j; ++i) s[pair_index(i, j)] = fma(v[i], v[j], s[pair_index(i, j)]);
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+  for (int p = 0; p < NPAIR; ++p) {
+    double t = s[p];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, off);
+    if (lane == 0) sh[p][warp] = t;
+  }
+  __syncthreads();
+  if (threadIdx.x < NPAIR) {
+    double t = 0;
+    for (int w = 0; w < GRAM_BLOCK / 32; ++w) t += sh[threadIdx.x][w];
+    gpart[static_cast<size_t>(blockIdx.x) * NPAIR + threadIdx.x] = t;
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!last) return;
+  __threadfence();
+  if (threadIdx.x < NPAIR) {
+    double t = 0;
+    for (unsigned b = 0; b < gridDim.x; ++b) t += __ldcg(&gpart[static_cast<size_t>(b) * NPAIR + threadIdx.x]);
+    G[threadIdx.x] = t;
+  }
+  __syncthreads();
+  if (threadIdx.x != 0) return;
+  *ticket = 0u;
+  // R (upper triangular, r[pair_index(k, j)] = r_kj) and T = R^-1, column by column
+  double r[NPAIR], tm[PANEL][PANEL];
+  bool dead[PANEL];
+  for (int j = 0; j < PANEL; ++j)
+    for (int i = 0; i < PANEL; ++i) tm[i][j] = 0.0;
+  for (int j = 0; j < pb; ++j) {
+    double d = G[pair_index(j, j)];
+    const double na = given_from_diagonal ? d : given[j];
+    for (int k = 0; k < j; ++k) {
+      double c = 0.0;
+      if (!dead[k]) {
+        c = G[pair_index(k, j)];
+        for (int i = 0; i < k; ++i) c -= r[pair_index(i, k)] * r[pair_index(i, j)];
+        c /= r[pair_index(k, k)];
+      }
+      r[pair_index(k, j)] = c;
+      d -= c * c;
+    }
+    const double rjj = d > 0.0 ? sqrt(d) : 0.0;
+    dead[j] = false;
+    if (!isfinite(na) || !isfinite(d)) {
+      twa_set_status(status, TWA_ERR_NONFINITE, col0 + j);
+      dead[j] = true;
+    } else if (!(rjj > 1e-5 * sqrt(na))) {
+      twa_set_status(status, TWA_ERR_RANK_DEFICIENT, col0 + j);
+      dead[j] = true;
+    }
+    r[pair_index(j, j)] = dead[j] ? 1.0 : rjj;
+    if (!dead[j]) {
+      // T[:, j] = (e_j - sum_{k<j} r_kj T[:, k]) / r_jj
+      for (int i = 0; i <= j; ++i) {
+        double v = i == j ? 1.0 : 0.0;
+        for (int k = i; k < j; ++k) v -= r[pair_index(k, j)] * tm[i][k];
+        tm[i][j] = v / rjj;
+      }
+    }
+    if (given_from_diagonal) given[j] = na;
+  }
+  for (int j = 0; j < PANEL; ++j)
+    for (int i = 0; i < PANEL; ++i) T[j * PANEL + i] = tm[i][j];
+}
+
+// A_p <- A_p T (T upper triangular, [column j][row i] at T[j * 8 + i]); float64 sums, one rounding per stored value.
+__global__ void __launch_bounds__(GRAM_BLOCK) panel_apply_kernel(float* __restrict__ A0, long long ld, int pb, long long D,
+                                                                const double* __restrict__ T) {
+  __shared__ double Ts[PANEL * PANEL];
+  if (threadIdx.x < PANEL * PANEL) Ts[threadIdx.x] = T[threadIdx.x];
+  __syncthreads();
+  const long long nvec = D >> 2;
+  for (long long t = blockIdx.x * static_cast<long long>(GRAM_BLOCK) + threadIdx.x; t < nvec;
+       t += static_cast<long long>(gridDim.x) * GRAM_BLOCK) {
+    float4 x[PANEL], y[PANEL];
+#pragma unroll
+    for (int j = 0; j < PANEL; ++j)
+      x[j] = j < pb ? __ldcs(reinterpret_cast<const float4*>(A0 + j * ld) + t) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < PANEL; ++j) {
+      double a = 0.0, b = 0.0, c = 0.0, d = 0.0;
+#pragma unroll
+      for (int i = 0; i <= j; ++i) {
+        const double w = Ts[j * PANEL + i];
+        a = fma(static_cast<double>(x[i].x), w, a);
+        b = fma(static_cast<double>(x[i].y), w, b);
+        c = fma(static_cast<double>(x[i].z), w, c);
+        d = fma(static_cast<double>(x[i].w), w, d);
+      }
+      y[j] = make_float4(static_cast<float>(a), static_cast<float>(b), static_cast<float>(c), static_cast<float>(d));
+    }
+#pragma unroll
+    for (int j = 0; j < PANEL; ++j)
+      if (j < pb) reinterpret_cast<float4*>(A0 + j * ld)[t] = y[j];
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (D & 3)) {
+    const long long r = (nvec << 2) + threadIdx.x;
+    double x[PANEL];
+    for (int j = 0; j < PANEL; ++j) x[j] = j < pb ? static_cast<double>(A0[j * ld + r]) : 0.0;
+    for (int j = 0; j < pb; ++j) {
+      double a = 0.0;
+      for (int i = 0; i <= j; ++i) a = fma(x[i], Ts[j * PANEL + i], a);
+      A0[j * ld + r] = static_cast<float>(a);
+    }
+  }
+}
+
 int encode_panel_map(twa_ctx* ctx, const float* W, long long D, long long ldw, int cols, CUtensorMap* map) {
   cuuint64_t dims[2] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(cols)};
   cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldw * 4)};
@@ -387,6 +553,31 @@ int twa_launch_panel_lift(twa_ctx* ctx, float* W, long long D, long long ldw, in
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(panel_lift_kernel), &smem_limit[ctx->device & 63], smem);
   if (rc) return rc;
   panel_lift_kernel<<<grid, PTHREADS, smem, ctx->stream>>>(map, a);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+// Orthonormalises the panel's pb <= 8 columns among themselves in Gram form (see panel_gram_kernel).
+// `given`: device array of 8 doubles, the squared norms the rank test compares against; with
+// given_from_diagonal they are taken from (and written as) the diagonal of this pass's Gram matrix.
+int twa_launch_panel_gram(twa_ctx* ctx, float* W, long long D, long long ldw, int j0, int pb, void* ws, double* given,
+                          bool given_from_diagonal) {
+  if (pb < 1 || pb > PANEL) return TWA_ERR_INVALID_ARG;
+  char* w = static_cast<char*>(ws);
+  double* gpart = reinterpret_cast<double*>(w + TWA_WS_PARTIALS);           // [grid][36], start of the float region
+  double* T = reinterpret_cast<double*>(w + TWA_WS_COEF);                    // 64 doubles
+  static_assert(sizeof(float) * TWA_MAX_N >= sizeof(double) * PANEL * PANEL, "coefficient area too small for T");
+  long long g = (D / 4 + GRAM_BLOCK - 1) / GRAM_BLOCK;
+  const long long cap = static_cast<long long>(ctx->sm_count) * 4;
+  if (g > cap) g = cap;
+  if (g > TWA_MAX_GRID) g = TWA_MAX_GRID;
+  if (g < 1) g = 1;
+  const int grid = static_cast<int>(g);
+  float* A0 = W + static_cast<long long>(j0) * ldw;
+  panel_gram_kernel<<<grid, GRAM_BLOCK, 0, ctx->stream>>>(A0, ldw, pb, D, gpart, given, given_from_diagonal ? 1 : 0, T,
+                                                          ctx->d_ticket, ctx->d_status, j0);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  panel_apply_kernel<<<grid, GRAM_BLOCK, 0, ctx->stream>>>(A0, ldw, pb, D, T);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
 }

@@ -535,7 +535,7 @@ def test_panel_build_agrees_with_column_build_and_oracle(env, D, n, step):
     ctx, ws = env
     wbar = torch.empty(D, device=DEV)
     out = {}
-    for mode in (1, 0):                                   # 1: column by column, 0: panels of 8 (default)
+    for mode in (1, 2, 0):       # 1: column by column; 2: panels of 8, sweeps inside; 0: panels, Gram form inside (default)
         W = inputs.trajectory_candidates(D, n, step, 0.001, 31, DEV, ld=inputs.padded_ld(D, 4))
         A = host_cols(W, D).copy()
         twa.twa_set_tuning(ctx, twa.TWA_TUNE_BUILD_PANEL, mode)
@@ -553,17 +553,26 @@ def test_panel_build_agrees_with_column_build_and_oracle(env, D, n, step):
         assert np.max(np.linalg.norm(Pg - Q, axis=0)) <= 10 * kappa * np.finfo(np.float32).eps, mode
         T = Pg.T @ A.astype(np.float64)
         assert np.all(np.diag(T) > 0) and np.max(np.abs(np.tril(T, -1))) <= 2e-5 * np.max(np.abs(T))
-    # the two schedules reach the same vectors to the accuracy either reaches the oracle
-    assert np.max(np.linalg.norm(out[0] - out[1], axis=0)) <= 20 * kappa * np.finfo(np.float32).eps
+    # the schedules reach the same vectors to the accuracy each reaches the oracle
+    for mode in (0, 2):
+        assert np.max(np.linalg.norm(out[mode] - out[1], axis=0)) <= 20 * kappa * np.finfo(np.float32).eps, mode
 
 
-def test_panel_build_finds_dependence_across_and_inside_panels(env):
+@pytest.fixture(params=[0, 2], ids=["gram-in-panel", "sweeps-in-panel"])
+def panel_mode(request, env):
+    ctx, _ = env
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_BUILD_PANEL, request.param)
+    yield request.param
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_BUILD_PANEL, 0)
+
+
+def test_panel_build_finds_dependence_across_and_inside_panels(env, panel_mode):
     ctx, ws = env
     D, n = 30001, 20
     wbar = torch.empty(D, device=DEV)
-    for bad_col, src in ((13, 3), (14, 9), (7, 0)):       # earlier panel; same panel; first panel
+    for bad_col, src in ((13, 3), (14, 9), (7, 0), (0, None), (19, 18)):   # earlier panel; same panel; first panel; zero first column; last
         W = inputs.trajectory_candidates(D, n, 0.01, 0.002, 2, DEV, ld=inputs.padded_ld(D, 4))
-        W[bad_col] = W[src] * -2.0
+        W[bad_col] = W[src] * -2.0 if src is not None else 0.0
         twa.twa_build_basis(ctx, W, D, wbar, ws)
         code, detail = twa.twa_get_status(ctx)
         assert (code, detail) == (twa.TWA_ERR_RANK_DEFICIENT, bad_col)
