@@ -22,7 +22,6 @@ constexpr int PCOL_BYTES = PROWS * 4;
 constexpr int PWARPS = 16;                       // consumer warps
 constexpr int PTHREADS = (PWARPS + 1) * 32;
 constexpr int CPART_BYTES = 4096;                // block's sums / coefficients: TWA_MAX_N x PANEL floats
-constexpr int MAX_Q_PER_WARP = TWA_MAX_N / PWARPS;
 
 struct PanelArgs {
   long long D, ldw;
@@ -67,6 +66,10 @@ __device__ __forceinline__ void panel_producer(twa_smem_header* hdr, unsigned ch
   }
 }
 
+// CPW = columns of Q a warp owns at most, ceil(nq / 16): a compile-time constant, so that the loops
+// over a warp's columns carry no guards (a warp with fewer columns repeats column 0 and drops the
+// result).  With run-time bounds the same kernel spent four times the instructions at nq = 16.
+template <int CPW>
 __global__ void __launch_bounds__(PTHREADS, 1)
 panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -89,18 +92,21 @@ panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a)
   if (warp == PWARPS) {
     if (lane == 0) panel_producer(hdr, ring, &map, a);
   } else {
-    const int cpw = warp < a.nq ? (a.nq - warp + PWARPS - 1) / PWARPS : 0;       // columns warp, warp + 16, ...
-    float acc[MAX_Q_PER_WARP][PANEL];
+    // columns warp, warp + 16, ...: byte offset of this lane's four rows of each inside a tile
+    // (all but the last always exist, at a constant stride; the last may not: it then repeats column 0)
+    const int qbase = warp * PCOL_BYTES + lane * 16;
+    const int qlast = (warp + (CPW - 1) * PWARPS < a.nq ? warp + (CPW - 1) * PWARPS : 0) * PCOL_BYTES + lane * 16;
+    const int goff = a.nq * PCOL_BYTES + lane * 16;
+    float acc[CPW][PANEL];
 #pragma unroll
-    for (int k = 0; k < MAX_Q_PER_WARP; ++k)
+    for (int k = 0; k < CPW; ++k)
 #pragma unroll
       for (int q = 0; q < PANEL; ++q) acc[k][q] = 0.0f;
     volatile int* abort_flag = &hdr->abort_flag;
-    int k_tile = 0;
-    for (int tile = blockIdx.x; tile < a.tiles; tile += gridDim.x, ++k_tile) {
-      const int s = k_tile % a.stages;
-      if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), static_cast<unsigned>(k_tile / a.stages) & 1u, abort_flag,
-                         a.wait_limit_ns)) {
+    int s = 0;
+    unsigned phase = 0;
+    for (int tile = blockIdx.x; tile < a.tiles; tile += gridDim.x) {
+      if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
         twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
         break;
       }
@@ -110,33 +116,33 @@ panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a)
         float4 g[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q)
-          g[q] = half * 4 + q < a.pb ? *reinterpret_cast<const float4*>(st + (a.nq + half * 4 + q) * PCOL_BYTES + lane * 16)
+          g[q] = half * 4 + q < a.pb ? *reinterpret_cast<const float4*>(st + goff + (half * 4 + q) * PCOL_BYTES)
                                      : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int k = 0; k < MAX_Q_PER_WARP; ++k) {
-          if (k < cpw) {
-            const float4 p = *reinterpret_cast<const float4*>(st + (warp + k * PWARPS) * PCOL_BYTES + lane * 16);
+        for (int k = 0; k < CPW; ++k) {
+          const float4 p = *reinterpret_cast<const float4*>(st + (k < CPW - 1 ? qbase + k * PWARPS * PCOL_BYTES : qlast));
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-              acc[k][half * 4 + q] =
-                  fmaf(p.x, g[q].x, fmaf(p.y, g[q].y, fmaf(p.z, g[q].z, fmaf(p.w, g[q].w, acc[k][half * 4 + q]))));
-          }
+          for (int q = 0; q < 4; ++q)
+            acc[k][half * 4 + q] =
+                fmaf(p.x, g[q].x, fmaf(p.y, g[q].y, fmaf(p.z, g[q].z, fmaf(p.w, g[q].w, acc[k][half * 4 + q]))));
         }
       }
       __syncwarp();
       if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
+      if (++s == a.stages) {
+        s = 0;
+        phase ^= 1u;
+      }
     }
     // lanes -> one value per (column, panel column); every pair belongs to exactly one warp
 #pragma unroll
-    for (int k = 0; k < MAX_Q_PER_WARP; ++k) {
-      if (k < cpw) {
+    for (int k = 0; k < CPW; ++k) {
 #pragma unroll
-        for (int q = 0; q < PANEL; ++q) {
-          float v = acc[k][q];
+      for (int q = 0; q < PANEL; ++q) {
+        float v = acc[k][q];
 #pragma unroll
-          for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
-          if (lane == 0) cpart[(warp + k * PWARPS) * PANEL + q] = v;
-        }
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+        if (lane == 0 && warp + k * PWARPS < a.nq) cpart[(warp + k * PWARPS) * PANEL + q] = v;
       }
     }
   }
@@ -296,7 +302,7 @@ constexpr int GRAM_BLOCK = 256;
 constexpr int NPAIR = PANEL * (PANEL + 1) / 2;                     // 36
 __host__ __device__ constexpr int pair_index(int i, int j) { return j * (j + 1) / 2 + i; }   // i <= j
 
-__global__ void __launch_bounds__(GRAM_BLOCK) panel_gram_kernel(const float* __restrict__ A0, long long ld, int pb,
+__global__ void __launch_bounds__(GRAM_BLOCK, 2) panel_gram_kernel(const float* __restrict__ A0, long long ld, int pb,
                                                                long long D, double* __restrict__ gpart,
                                                                double* __restrict__ given, int given_from_diagonal,
                                                                double* __restrict__ T, unsigned* __restrict__ ticket,
@@ -497,6 +503,16 @@ int fill_args(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb
   return TWA_OK;
 }
 
+template <int CPW>
+int launch_panel_project(twa_ctx* ctx, const CUtensorMap& map, const PanelArgs& a, int grid, int smem) {
+  static int smem_limit[64] = {0};
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(panel_project_kernel<CPW>), &smem_limit[ctx->device & 63], smem);
+  if (rc) return rc;
+  panel_project_kernel<CPW><<<grid, PTHREADS, smem, ctx->stream>>>(map, a);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
 }  // namespace
 
 int twa_launch_panel_project(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws) {
@@ -507,12 +523,17 @@ int twa_launch_panel_project(twa_ctx* ctx, float* W, long long D, long long ldw,
   CUtensorMap map;
   rc = encode_panel_map(ctx, W, D, ldw, nq + pb, &map);
   if (rc) return rc;
-  static int smem_limit[64] = {0};
-  rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(panel_project_kernel), &smem_limit[ctx->device & 63], smem);
-  if (rc) return rc;
-  panel_project_kernel<<<grid, PTHREADS, smem, ctx->stream>>>(map, a);
-  TWA_CUDA_OK(ctx, cudaGetLastError());
-  return TWA_OK;
+  const int cpw = (nq + PWARPS - 1) / PWARPS;
+  switch (cpw) {
+    case 1: return launch_panel_project<1>(ctx, map, a, grid, smem);
+    case 2: return launch_panel_project<2>(ctx, map, a, grid, smem);
+    case 3: return launch_panel_project<3>(ctx, map, a, grid, smem);
+    case 4: return launch_panel_project<4>(ctx, map, a, grid, smem);
+    case 5: return launch_panel_project<5>(ctx, map, a, grid, smem);
+    case 6: return launch_panel_project<6>(ctx, map, a, grid, smem);
+    case 7: return launch_panel_project<7>(ctx, map, a, grid, smem);
+    default: return launch_panel_project<8>(ctx, map, a, grid, smem);
+  }
 }
 
 int twa_launch_panel_lift(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws) {
