@@ -6,10 +6,12 @@
 //     A_p <- A_p - Q C   (twa_launch_panel_lift)
 // The projection streams tiles of 128 rows x (nq + pb) columns of the float32 matrix through a TMA
 // ring (one box per stage: the panel's columns are simply the last columns of the tile).
-//  * projection: warp w owns columns w, w+16, ...; a lane owns 4 rows; 8 x 8 accumulators per lane;
+//  * projection: warp w of 15 owns columns w, w+15, ...; a lane owns 4 rows; up to 8 x 8 accumulators per lane;
 //    lanes -> block -> last block to finish, float64 over blocks in block order.
-//  * update: a lane owns one row of a block of 512 rows and walks all nq columns as they stream past
+//  * update: a lane owns two rows of a block of 1024 rows and walks all nq columns as they stream past
 //    in chunks of 8, so there is no reduction at all.
+//  * inside the panel: the Gram-Schmidt coefficients from the panel's Gram matrix (one pass), the new
+//    columns as A_p T (a second pass).
 #include <stdio.h>
 
 #include "twa_common.cuh"
@@ -21,6 +23,11 @@ constexpr int PROWS = 128;                       // rows per tile of the project
 constexpr int PCOL_BYTES = PROWS * 4;
 constexpr int PWARPS = 16;                       // consumer warps
 constexpr int PTHREADS = (PWARPS + 1) * 32;
+// The projection runs 15 consumer warps and the producer: 16 warps, four per scheduler, leave 128
+// registers per thread for up to 8 x 8 accumulators (with 17 warps one scheduler holds five and the
+// limit is 96: the kernels for six and more columns per warp spilled).
+constexpr int PJWARPS = 15;
+constexpr int PJTHREADS = (PJWARPS + 1) * 32;
 constexpr int CPART_BYTES = 4096;                // block's sums / coefficients: TWA_MAX_N x PANEL floats
 
 struct PanelArgs {
@@ -66,11 +73,11 @@ __device__ __forceinline__ void panel_producer(twa_smem_header* hdr, unsigned ch
   }
 }
 
-// CPW = columns of Q a warp owns at most, ceil(nq / 16): a compile-time constant, so that the loops
+// CPW = columns of Q a warp owns at most, ceil(nq / 15): a compile-time constant, so that the loops
 // over a warp's columns carry no guards (a warp with fewer columns repeats column 0 and drops the
 // result).  With run-time bounds the same kernel spent four times the instructions at nq = 16.
 template <int CPW>
-__global__ void __launch_bounds__(PTHREADS, 1)
+__global__ void __launch_bounds__(PJTHREADS, 1)
 panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -81,7 +88,7 @@ panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a)
   if (threadIdx.x == 0) {
     for (int s = 0; s < a.stages; ++s) {
       twa_mbar_init(twa_smem_u32(&hdr->full[s]), 1);
-      twa_mbar_init(twa_smem_u32(&hdr->empty[s]), PWARPS);
+      twa_mbar_init(twa_smem_u32(&hdr->empty[s]), PJWARPS);
     }
     hdr->abort_flag = 0;
     hdr->last_flag = 0;
@@ -89,13 +96,13 @@ panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a)
   }
   __syncthreads();
 
-  if (warp == PWARPS) {
+  if (warp == PJWARPS) {
     if (lane == 0) panel_producer(hdr, ring, &map, a);
   } else {
-    // columns warp, warp + 16, ...: byte offset of this lane's four rows of each inside a tile
+    // columns warp, warp + 15, ...: byte offset of this lane's four rows of each inside a tile
     // (all but the last always exist, at a constant stride; the last may not: it then repeats column 0)
     const int qbase = warp * PCOL_BYTES + lane * 16;
-    const int qlast = (warp + (CPW - 1) * PWARPS < a.nq ? warp + (CPW - 1) * PWARPS : 0) * PCOL_BYTES + lane * 16;
+    const int qlast = (warp + (CPW - 1) * PJWARPS < a.nq ? warp + (CPW - 1) * PJWARPS : 0) * PCOL_BYTES + lane * 16;
     const int goff = a.nq * PCOL_BYTES + lane * 16;
     float acc[CPW][PANEL];
 #pragma unroll
@@ -111,20 +118,21 @@ panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a)
         break;
       }
       const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
+      constexpr int GQ = 4;                               // panel columns in registers at a time
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {             // four panel columns at a time (registers)
-        float4 g[4];
+      for (int part = 0; part < PANEL / GQ; ++part) {
+        float4 g[GQ];
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-          g[q] = half * 4 + q < a.pb ? *reinterpret_cast<const float4*>(st + goff + (half * 4 + q) * PCOL_BYTES)
-                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int q = 0; q < GQ; ++q)
+          g[q] = part * GQ + q < a.pb ? *reinterpret_cast<const float4*>(st + goff + (part * GQ + q) * PCOL_BYTES)
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int k = 0; k < CPW; ++k) {
-          const float4 p = *reinterpret_cast<const float4*>(st + (k < CPW - 1 ? qbase + k * PWARPS * PCOL_BYTES : qlast));
+          const float4 p = *reinterpret_cast<const float4*>(st + (k < CPW - 1 ? qbase + k * PJWARPS * PCOL_BYTES : qlast));
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
-            acc[k][half * 4 + q] =
-                fmaf(p.x, g[q].x, fmaf(p.y, g[q].y, fmaf(p.z, g[q].z, fmaf(p.w, g[q].w, acc[k][half * 4 + q]))));
+          for (int q = 0; q < GQ; ++q)
+            acc[k][part * GQ + q] =
+                fmaf(p.x, g[q].x, fmaf(p.y, g[q].y, fmaf(p.z, g[q].z, fmaf(p.w, g[q].w, acc[k][part * GQ + q]))));
         }
       }
       __syncwarp();
@@ -142,7 +150,7 @@ panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a)
         float v = acc[k][q];
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
-        if (lane == 0 && warp + k * PWARPS < a.nq) cpart[(warp + k * PWARPS) * PANEL + q] = v;
+        if (lane == 0 && warp + k * PJWARPS < a.nq) cpart[(warp + k * PJWARPS) * PANEL + q] = v;
       }
     }
   }
@@ -522,7 +530,7 @@ int launch_panel_project(twa_ctx* ctx, const CUtensorMap& map, const PanelArgs& 
   static int smem_limit[64] = {0};
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(panel_project_kernel<CPW>), &smem_limit[ctx->device & 63], smem);
   if (rc) return rc;
-  panel_project_kernel<CPW><<<grid, PTHREADS, smem, ctx->stream>>>(map, a);
+  panel_project_kernel<CPW><<<grid, PJTHREADS, smem, ctx->stream>>>(map, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
 }
@@ -537,7 +545,7 @@ int twa_launch_panel_project(twa_ctx* ctx, float* W, long long D, long long ldw,
   CUtensorMap map;
   rc = encode_panel_map(ctx, W, D, ldw, nq + pb, &map);
   if (rc) return rc;
-  const int cpw = (nq + PWARPS - 1) / PWARPS;
+  const int cpw = (nq + PJWARPS - 1) / PJWARPS;
   switch (cpw) {
     case 1: return launch_panel_project<1>(ctx, map, a, grid, smem);
     case 2: return launch_panel_project<2>(ctx, map, a, grid, smem);
