@@ -343,6 +343,30 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
                         int bits, void* mem, size_t mem_bytes, twa_layered_basis* out, void* lws,
                         size_t lws_bytes);
 
+/* Row-chunked form of twa_build_centered + twa_quantize_affine (same Sections 4.1, 4.5, 4.6) for
+ * candidate sets that do not fit in device memory: the caller feeds every row chunk of the
+ * candidates once per pass, in any order inside a pass, and never holds more than one chunk.
+ *   begin           carves `mem` (twa_layered_basis_bytes, 256-byte aligned), fills *out, clears the
+ *                   accumulators in lws (twa_layered_workspace_bytes) and the codes; synchronises
+ *                   the stream once (uploads the layer tables)
+ *   pass 0: feed    w_bar rows of the chunk into wbar[row0 ..], sums of (w - w_bar)^2 per layer and
+ *                   candidate;            end_pass(0): the norms
+ *   pass 1: feed    min / max of e = (w - w_bar) / ||.|| per layer; q32_out (optional, rows x n,
+ *                   column stride ldq) receives e as float32;   end_pass(1): the factors a, b
+ *   pass 2: feed    codes of e (computed with the arithmetic of pass 1, so they are exactly the
+ *                   quantiser applied to the float32 values of pass 1);   end_pass(2): nothing
+ * chunk: rows x n float32, candidate i at chunk[i * ld + (r - row0)] for flat row r; 16-byte aligned,
+ * ld and row0 multiples of 4.  offsets_host, lws: as passed to begin.  wbar: D floats, the same
+ * buffer in every call.  The same chunking need not be used in every pass.  Errors as for the
+ * resident calls (TWA_ERR_NONFINITE: detail = candidate in pass 0, layer in pass 1). */
+int twa_layered_build_begin(twa_ctx* ctx, int64_t D, int n, const int64_t* offsets_host, int L, int bits,
+                            void* mem, size_t mem_bytes, twa_layered_basis* out, void* lws, size_t lws_bytes);
+int twa_layered_build_feed(twa_ctx* ctx, const twa_layered_basis* lb, const int64_t* offsets_host, int pass,
+                           const float* chunk, int64_t ld, int64_t row0, int64_t rows, float* wbar,
+                           float* q32_out, int64_t ldq, void* lws, size_t lws_bytes);
+int twa_layered_build_end_pass(twa_ctx* ctx, const twa_layered_basis* lb, const int64_t* offsets_host,
+                               int pass, void* lws, size_t lws_bytes);
+
 /* Canonical image for parity checks: unsigned codes in flat row order, n x ceil(D*bits/8) bytes
  * (4 bits: row 2k low nibble, row 2k+1 high nibble), and the L factors a, b.  Device pointers. */
 int twa_layered_export(twa_ctx* ctx, const twa_layered_basis* lb, void* codes_out, float* a_out,

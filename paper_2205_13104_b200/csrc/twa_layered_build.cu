@@ -209,6 +209,130 @@ __global__ void __launch_bounds__(BLOCK) affine_encode_kernel(const float* __res
   }
 }
 
+// ---- row-chunked construction: the same arithmetic on rows [row0, row1) of the flat vector --------
+// chunk[i * ld + (r - row0)] is candidate i at flat row r.  An item (at most 8192 rows of one layer)
+// may straddle two chunks: its partial results are merged by the calls in stream order.
+__global__ void __launch_bounds__(BLOCK) chunk_centred_sumsq_kernel(const float* __restrict__ chunk, long long ld,
+                                                                    long long row0, long long row1,
+                                                                    const float* __restrict__ wbar,
+                                                                    const Item* __restrict__ items, int n,
+                                                                    double* __restrict__ partial) {
+  __shared__ double sh[BLOCK / 32];
+  const Item it = items[blockIdx.x];
+  const long long r0 = it.r0 > row0 ? it.r0 : row0, r1 = it.r1 < row1 ? it.r1 : row1;
+  const float* col = chunk + blockIdx.y * ld - row0;
+  double s = 0;
+  for (long long r = r0 + threadIdx.x; r < r1; r += BLOCK) {
+    const double v = static_cast<double>(col[r]) - static_cast<double>(wbar[r]);
+    s += v * v;
+  }
+  const double t = block_sum_d(s, sh);
+  if (threadIdx.x == 0) partial[static_cast<size_t>(blockIdx.x) * n + blockIdx.y] += t;
+}
+
+// e = (w - w_bar) / ||.|| for the chunk's rows (the expression of centre_scale_kernel), its min / max
+// per item merged into pmin / pmax, and optionally the values themselves.
+__global__ void __launch_bounds__(BLOCK) chunk_minmax_kernel(const float* __restrict__ chunk, long long ld,
+                                                             long long row0, long long row1,
+                                                             const float* __restrict__ wbar,
+                                                             const Item* __restrict__ items, int n,
+                                                             const double* __restrict__ inv, float* __restrict__ pmin,
+                                                             float* __restrict__ pmax, float* __restrict__ q32,
+                                                             long long ldq) {
+  __shared__ float smin[BLOCK / 32], smax[BLOCK / 32];
+  const Item it = items[blockIdx.x];
+  const long long r0 = it.r0 > row0 ? it.r0 : row0, r1 = it.r1 < row1 ? it.r1 : row1;
+  const float* col = chunk + blockIdx.y * ld - row0;
+  const double f = inv[static_cast<size_t>(it.layer) * n + blockIdx.y];
+  float lo = INFINITY, hi = -INFINITY;
+  bool bad = false;
+  for (long long r = r0 + threadIdx.x; r < r1; r += BLOCK) {
+    const float v = static_cast<float>((static_cast<double>(col[r]) - static_cast<double>(wbar[r])) * f);
+    if (q32) q32[blockIdx.y * ldq + (r - row0)] = v;
+    lo = fminf(lo, v);
+    hi = fmaxf(hi, v);
+    bad |= !isfinite(v);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, off));
+    hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, off));
+  }
+  bad = __any_sync(0xFFFFFFFFu, bad);
+  if ((threadIdx.x & 31) == 0) {
+    smin[threadIdx.x >> 5] = bad ? NAN : lo;
+    smax[threadIdx.x >> 5] = hi;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 0; w < BLOCK / 32; ++w) {
+      bad |= isnan(smin[w]);
+      lo = fminf(lo, smin[w]);
+      hi = fmaxf(hi, smax[w]);
+    }
+    const size_t at = static_cast<size_t>(blockIdx.x) * n + blockIdx.y;
+    const float old_lo = pmin[at], old_hi = pmax[at];
+    bad |= isnan(old_lo);
+    pmin[at] = bad ? NAN : fminf(lo, old_lo);
+    pmax[at] = fmaxf(hi, old_hi);
+  }
+}
+
+__global__ void fill_kernel(float* p, size_t count, float v) {
+  for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < count;
+       i += static_cast<size_t>(gridDim.x) * blockDim.x)
+    p[i] = v;
+}
+
+// Codes of the chunk's rows.  A 16-byte group of codes (16 or 32 rows counted from the layer's first
+// row) may straddle two chunks: the storage starts as zeros and every call ORs its rows in.
+template <int BITS>
+__global__ void __launch_bounds__(BLOCK) chunk_affine_encode_kernel(const float* __restrict__ chunk, long long ld,
+                                                                    long long row0, long long row1,
+                                                                    const float* __restrict__ wbar,
+                                                                    const double* __restrict__ inv, int n,
+                                                                    const long long* __restrict__ flat,
+                                                                    const long long* __restrict__ internal,
+                                                                    const float* __restrict__ a,
+                                                                    const float* __restrict__ b,
+                                                                    unsigned char* __restrict__ out,
+                                                                    long long out_stride, int first_layer) {
+  constexpr int RPC = 128 / BITS;
+  constexpr float TOP = BITS == 8 ? 255.0f : 15.0f;
+  const int l = first_layer + blockIdx.z, j = blockIdx.y;
+  const long long lay0 = flat[l], lay1 = flat[l + 1];
+  const long long f0 = (lay0 > row0 ? lay0 : row0) - lay0, f1 = (lay1 < row1 ? lay1 : row1) - lay0;   // rows of the layer
+  if (f1 <= f0) return;
+  const long long c0 = f0 / RPC, c1 = (f1 + RPC - 1) / RPC;
+  const float al = a[l], bl = b[l];
+  const double f = inv[static_cast<size_t>(l) * n + j];
+  const float* col = chunk + j * ld - row0 + lay0;
+  const float* wb = wbar + lay0;
+  uint4* dst = reinterpret_cast<uint4*>(out + j * out_stride);
+  for (long long c = c0 + blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; c < c1;
+       c += static_cast<long long>(gridDim.x) * BLOCK) {
+    uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int k = 0; k < RPC; ++k) {
+      const long long r = c * RPC + k;
+      uint32_t u = 0;
+      if (r >= f0 && r < f1 && al != 0.0f) {
+        const float e = static_cast<float>((static_cast<double>(col[r]) - static_cast<double>(wb[r])) * f);
+        float q = rintf(__fdiv_rn(__fsub_rn(e, bl), al));
+        q = fminf(fmaxf(q, 0.0f), TOP);
+        u = static_cast<uint32_t>(q);
+      }
+      if (BITS == 8) w[k >> 2] |= u << (8 * (k & 3));
+      else w[k >> 3] |= u << (4 * (k & 7));
+    }
+    const long long q = internal[l] / RPC + c;
+    uint4* at = dst + ((q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j));
+    uint4 old = *at;
+    old.x |= w[0]; old.y |= w[1]; old.z |= w[2]; old.w |= w[3];
+    *at = old;
+  }
+}
+
 // fills the tail of every column (rows from the last layer's end to the column stride) with code 0
 __global__ void tail_zero_kernel(unsigned char* out, long long out_stride, long long first_chunk,
                                  long long chunks) {
@@ -291,6 +415,96 @@ size_t count_items(const int64_t* offsets, int L) {
   return k;
 }
 
+// Carves the caller's buffer of a layered basis (codes | a | b | granule table | flat offsets |
+// internal offsets | block tables), builds and uploads the tables, and fills the descriptor.
+int prepare_layered_storage(twa_ctx* ctx, const Partition& p, long long D, int L, int n, int bits, void* mem,
+                            twa_layered_basis* out) {
+  // carve the caller's buffer: codes | a | b | granule table | flat offsets | internal offsets
+  char* m = static_cast<char*>(mem);
+  const long long stride = twa_basis_col_stride(p.D_int, bits);
+  const size_t codes_bytes = static_cast<size_t>(stride) * n;
+  const size_t fl = (sizeof(float) * L + 255) / 256 * 256;
+  const size_t n_gran = static_cast<size_t>(stride / 64);
+  const size_t off_bytes = (sizeof(long long) * (L + 1) + 255) / 256 * 256;
+  size_t o = (codes_bytes + 255) / 256 * 256;
+  float* a = reinterpret_cast<float*>(m + o); o += fl;
+  float* b = reinterpret_cast<float*>(m + o); o += fl;
+  int* gran = reinterpret_cast<int*>(m + o); o += 16 * (n_gran + TABLE_SLACK);
+  long long* d_flat = reinterpret_cast<long long*>(m + o); o += off_bytes;
+  long long* d_int = reinterpret_cast<long long*>(m + o); o += off_bytes;
+  int* d_cta_first = reinterpret_cast<int*>(m + o); o += CTA_TABLE_BYTES;
+  int* d_cta_base = reinterpret_cast<int*>(m + o);
+
+  // work split of the step kernels: contiguous tile ranges, and the layers each range meets
+  const int kt = (ctx->tune_tile_segments == 1 || ctx->tune_tile_segments == 2) ? ctx->tune_tile_segments
+                                                                                : (n <= 64 ? 2 : 1);
+  const long long tile_rows = 512LL * 8 / bits * kt;
+  const int tiles = static_cast<int>((p.D_int + tile_rows - 1) / tile_rows);
+  int ctas = ctx->sm_count < tiles ? ctx->sm_count : tiles;
+  if (ctas > MAX_CTAS) ctas = MAX_CTAS;
+  const int tpc = (tiles + ctas - 1) / ctas;
+  ctas = (tiles + tpc - 1) / tpc;
+  std::vector<int> cta_first(ctas), cta_base(ctas + 1, 0);
+  {
+    int l = 0;
+    for (int k = 0; k < ctas; ++k) {
+      const long long r0 = static_cast<long long>(k) * tpc * tile_rows;       // < D_int
+      long long r1 = r0 + tpc * tile_rows;
+      if (r1 > p.D_int) r1 = p.D_int;
+      while (p.internal[l + 1] <= r0) ++l;
+      cta_first[k] = l;
+      int last = l;
+      while (p.internal[last + 1] < r1) ++last;
+      cta_base[k + 1] = cta_base[k] + (last - l + 1);
+    }
+  }
+  // granule table: layer, valid rows, first flat row of every 64-byte granule of a column
+  {
+    const long long gr = granule_rows(bits);
+    // (with slack, so that the last tile of a two-segment tiling finds entries for all its granules)
+    std::vector<int> tab(4 * (n_gran + TABLE_SLACK), 0);
+    for (size_t k = 0; k < n_gran + TABLE_SLACK; ++k) tab[4 * k] = -1;   // granules behind the last layer
+    for (int l = 0; l < L; ++l) {
+      const long long len = p.flat[l + 1] - p.flat[l];
+      for (long long k0 = 0; k0 < len; k0 += gr) {
+        const size_t gidx = static_cast<size_t>((p.internal[l] + k0) / gr);
+        tab[4 * gidx] = l;
+        tab[4 * gidx + 1] = static_cast<int>(len - k0 < gr ? len - k0 : gr);
+        tab[4 * gidx + 2] = static_cast<int>(p.flat[l] + k0);
+      }
+    }
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(gran, tab.data(), sizeof(int) * tab.size(), cudaMemcpyHostToDevice,
+                                     ctx->stream));
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_flat, p.flat.data(), sizeof(long long) * (L + 1),
+                                     cudaMemcpyHostToDevice, ctx->stream));
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_int, p.internal.data(), sizeof(long long) * (L + 1),
+                                     cudaMemcpyHostToDevice, ctx->stream));
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_cta_first, cta_first.data(), sizeof(int) * ctas, cudaMemcpyHostToDevice,
+                                     ctx->stream));
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_cta_base, cta_base.data(), sizeof(int) * (ctas + 1),
+                                     cudaMemcpyHostToDevice, ctx->stream));
+    TWA_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));
+  }
+
+  unsigned char* codes = reinterpret_cast<unsigned char*>(m);
+  out->codes = twa_basis{codes, nullptr, p.D_int, stride, n, bits};
+  out->a = a;
+  out->b = b;
+  out->granules = gran;
+  out->flat_offsets = reinterpret_cast<int64_t*>(d_flat);
+  out->internal_offsets = reinterpret_cast<int64_t*>(d_int);
+  out->D = D;
+  out->L = L;
+  out->cta_count = ctas;
+  out->kt = kt;
+  out->tiles = tiles;
+  out->tiles_per_cta = tpc;
+  out->total_runs = cta_base[ctas];
+  out->cta_first_layer = d_cta_first;
+  out->cta_run_base = d_cta_base;
+  return TWA_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -370,72 +584,11 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
   rc = upload_partition(ctx, p, L, ws, w);
   if (rc) return rc;
 
-  // carve the caller's buffer: codes | a | b | granule table | flat offsets | internal offsets
-  char* m = static_cast<char*>(mem);
-  const long long stride = twa_basis_col_stride(p.D_int, bits);
-  const size_t codes_bytes = static_cast<size_t>(stride) * n;
-  const size_t fl = (sizeof(float) * L + 255) / 256 * 256;
-  const size_t n_gran = static_cast<size_t>(stride / 64);
-  const size_t off_bytes = (sizeof(long long) * (L + 1) + 255) / 256 * 256;
-  size_t o = (codes_bytes + 255) / 256 * 256;
-  float* a = reinterpret_cast<float*>(m + o); o += fl;
-  float* b = reinterpret_cast<float*>(m + o); o += fl;
-  int* gran = reinterpret_cast<int*>(m + o); o += 16 * (n_gran + TABLE_SLACK);
-  long long* d_flat = reinterpret_cast<long long*>(m + o); o += off_bytes;
-  long long* d_int = reinterpret_cast<long long*>(m + o); o += off_bytes;
-  int* d_cta_first = reinterpret_cast<int*>(m + o); o += CTA_TABLE_BYTES;
-  int* d_cta_base = reinterpret_cast<int*>(m + o);
-
-  // work split of the step kernels: contiguous tile ranges, and the layers each range meets
-  const int kt = (ctx->tune_tile_segments == 1 || ctx->tune_tile_segments == 2) ? ctx->tune_tile_segments
-                                                                                : (n <= 64 ? 2 : 1);
-  const long long tile_rows = 512LL * 8 / bits * kt;
-  const int tiles = static_cast<int>((p.D_int + tile_rows - 1) / tile_rows);
-  int ctas = ctx->sm_count < tiles ? ctx->sm_count : tiles;
-  if (ctas > MAX_CTAS) ctas = MAX_CTAS;
-  const int tpc = (tiles + ctas - 1) / ctas;
-  ctas = (tiles + tpc - 1) / tpc;
-  std::vector<int> cta_first(ctas), cta_base(ctas + 1, 0);
-  {
-    int l = 0;
-    for (int k = 0; k < ctas; ++k) {
-      const long long r0 = static_cast<long long>(k) * tpc * tile_rows;       // < D_int
-      long long r1 = r0 + tpc * tile_rows;
-      if (r1 > p.D_int) r1 = p.D_int;
-      while (p.internal[l + 1] <= r0) ++l;
-      cta_first[k] = l;
-      int last = l;
-      while (p.internal[last + 1] < r1) ++last;
-      cta_base[k + 1] = cta_base[k] + (last - l + 1);
-    }
-  }
-  // granule table: layer, valid rows, first flat row of every 64-byte granule of a column
-  {
-    const long long gr = granule_rows(bits);
-    // (with slack, so that the last tile of a two-segment tiling finds entries for all its granules)
-    std::vector<int> tab(4 * (n_gran + TABLE_SLACK), 0);
-    for (size_t k = 0; k < n_gran + TABLE_SLACK; ++k) tab[4 * k] = -1;   // granules behind the last layer
-    for (int l = 0; l < L; ++l) {
-      const long long len = p.flat[l + 1] - p.flat[l];
-      for (long long k0 = 0; k0 < len; k0 += gr) {
-        const size_t gidx = static_cast<size_t>((p.internal[l] + k0) / gr);
-        tab[4 * gidx] = l;
-        tab[4 * gidx + 1] = static_cast<int>(len - k0 < gr ? len - k0 : gr);
-        tab[4 * gidx + 2] = static_cast<int>(p.flat[l] + k0);
-      }
-    }
-    TWA_CUDA_OK(ctx, cudaMemcpyAsync(gran, tab.data(), sizeof(int) * tab.size(), cudaMemcpyHostToDevice,
-                                     ctx->stream));
-    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_flat, p.flat.data(), sizeof(long long) * (L + 1),
-                                     cudaMemcpyHostToDevice, ctx->stream));
-    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_int, p.internal.data(), sizeof(long long) * (L + 1),
-                                     cudaMemcpyHostToDevice, ctx->stream));
-    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_cta_first, cta_first.data(), sizeof(int) * ctas, cudaMemcpyHostToDevice,
-                                     ctx->stream));
-    TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_cta_base, cta_base.data(), sizeof(int) * (ctas + 1),
-                                     cudaMemcpyHostToDevice, ctx->stream));
-    TWA_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));
-  }
+  rc = prepare_layered_storage(ctx, p, D, L, n, bits, mem, out);
+  if (rc) return rc;
+  float* a = out->a;
+  float* b = out->b;
+  const long long stride = out->codes.col_stride;
 
   const Item* items = reinterpret_cast<const Item*>(ws + w.items);
   const int* first_item = reinterpret_cast<const int*>(ws + w.first_item);
@@ -457,7 +610,7 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
   if (gx < 1) gx = 1;
   if (L > 65535) return TWA_ERR_UNSUPPORTED;
   const dim3 egrid(static_cast<unsigned>(gx), static_cast<unsigned>(n), static_cast<unsigned>(L));
-  unsigned char* codes = reinterpret_cast<unsigned char*>(m);
+  unsigned char* codes = static_cast<unsigned char*>(out->codes.data);
   const long long* fl_d = reinterpret_cast<const long long*>(ws + w.flat);
   const long long* in_d = reinterpret_cast<const long long*>(ws + w.internal);
   if (bits == 8)
@@ -470,21 +623,6 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
     tail_zero_kernel<<<dim3(1, n), 64, 0, ctx->stream>>>(codes, stride, first_tail, total_chunks);
     TWA_CUDA_OK(ctx, cudaGetLastError());
   }
-  out->codes = twa_basis{codes, nullptr, p.D_int, stride, n, bits};
-  out->a = a;
-  out->b = b;
-  out->granules = gran;
-  out->flat_offsets = reinterpret_cast<int64_t*>(d_flat);
-  out->internal_offsets = reinterpret_cast<int64_t*>(d_int);
-  out->D = D;
-  out->L = L;
-  out->cta_count = ctas;
-  out->kt = kt;
-  out->tiles = tiles;
-  out->tiles_per_cta = tpc;
-  out->total_runs = cta_base[ctas];
-  out->cta_first_layer = d_cta_first;
-  out->cta_run_base = d_cta_base;
   return TWA_OK;
 }
 
@@ -513,6 +651,132 @@ int twa_layered_export(twa_ctx* ctx, const twa_layered_basis* lb, void* codes_ou
   TWA_CUDA_OK(ctx, cudaGetLastError());
   TWA_CUDA_OK(ctx, cudaMemcpyAsync(a_out, lb->a, sizeof(float) * lb->L, cudaMemcpyDeviceToDevice, ctx->stream));
   TWA_CUDA_OK(ctx, cudaMemcpyAsync(b_out, lb->b, sizeof(float) * lb->L, cudaMemcpyDeviceToDevice, ctx->stream));
+  return TWA_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Row-chunked form of twa_build_centered + twa_quantize_affine
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+// items [k0, k1) and layers [l0, l1] that meet flat rows [row0, row1)
+void chunk_range(const Partition& p, int L, long long row0, long long row1, int* k0, int* k1, int* l0, int* l1) {
+  auto by_end = [](const Item& it, long long r) { return it.r1 <= r; };
+  auto by_start = [](const Item& it, long long r) { return it.r0 < r; };
+  *k0 = static_cast<int>(std::lower_bound(p.items.begin(), p.items.end(), row0, by_end) - p.items.begin());
+  *k1 = static_cast<int>(std::lower_bound(p.items.begin(), p.items.end(), row1, by_start) - p.items.begin());
+  *l0 = static_cast<int>(std::upper_bound(p.flat.begin(), p.flat.end(), row0) - p.flat.begin()) - 1;
+  *l1 = static_cast<int>(std::lower_bound(p.flat.begin(), p.flat.end(), row1) - p.flat.begin()) - 1;
+  if (*l1 > L - 1) *l1 = L - 1;
+}
+
+}  // namespace
+
+extern "C" {
+
+int twa_layered_build_begin(twa_ctx* ctx, int64_t D, int n, const int64_t* offsets_host, int L, int bits, void* mem,
+                            size_t mem_bytes, twa_layered_basis* out, void* lws, size_t lws_bytes) {
+  if (!ctx || !out || !offsets_host || !mem) return TWA_ERR_INVALID_ARG;
+  if (bits != 8 && bits != 4) return TWA_ERR_UNSUPPORTED;
+  if (D < 1 || D >= (1LL << 31) || n < 1) return TWA_ERR_INVALID_ARG;
+  if (n > TWA_MAX_N || L > 65535) return TWA_ERR_UNSUPPORTED;
+  Partition p;
+  int rc = make_partition(offsets_host, L, D, bits, &p);
+  if (rc) return rc;
+  const LwsLayout w = lws_layout(p.items.size(), L, n);
+  if (!lws || lws_bytes < w.total) return TWA_ERR_WORKSPACE;
+  if (mem_bytes < twa_layered_basis_bytes(offsets_host, L, n, bits)) return TWA_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(mem) & 255) || (reinterpret_cast<uintptr_t>(lws) & 15)) return TWA_ERR_MISALIGNED;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  char* ws = static_cast<char*>(lws);
+  rc = upload_partition(ctx, p, L, ws, w);
+  if (rc) return rc;
+  rc = prepare_layered_storage(ctx, p, D, L, n, bits, mem, out);
+  if (rc) return rc;
+  const size_t cells = p.items.size() * static_cast<size_t>(n);
+  TWA_CUDA_OK(ctx, cudaMemsetAsync(ws + w.partial, 0, sizeof(double) * cells, ctx->stream));
+  fill_kernel<<<64, 256, 0, ctx->stream>>>(reinterpret_cast<float*>(ws + w.pmin), cells, INFINITY);
+  fill_kernel<<<64, 256, 0, ctx->stream>>>(reinterpret_cast<float*>(ws + w.pmax), cells, -INFINITY);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  TWA_CUDA_OK(ctx, cudaMemsetAsync(out->codes.data, 0, static_cast<size_t>(out->codes.col_stride) * n, ctx->stream));
+  return TWA_OK;
+}
+
+int twa_layered_build_feed(twa_ctx* ctx, const twa_layered_basis* lb, const int64_t* offsets_host, int pass,
+                           const float* chunk, int64_t ld, int64_t row0, int64_t rows, float* wbar,
+                           float* q32_out, int64_t ldq, void* lws, size_t lws_bytes) {
+  if (!ctx || !lb || !offsets_host || !chunk || !wbar || pass < 0 || pass > 2) return TWA_ERR_INVALID_ARG;
+  const long long D = lb->D;
+  const int n = lb->codes.n, L = lb->L, bits = lb->codes.bits;
+  if (rows < 1 || row0 < 0 || row0 + rows > D || ld < rows) return TWA_ERR_INVALID_ARG;
+  if (q32_out && (pass != 1 || ldq < rows)) return TWA_ERR_INVALID_ARG;
+  // the mean of the chunk is written with 16-byte stores at wbar + row0
+  if ((reinterpret_cast<uintptr_t>(chunk) & 15) || (ld & 3) || (row0 & 3) || (reinterpret_cast<uintptr_t>(wbar) & 15))
+    return TWA_ERR_MISALIGNED;
+  Partition p;
+  int rc = make_partition(offsets_host, L, D, bits, &p);
+  if (rc) return rc;
+  const LwsLayout w = lws_layout(p.items.size(), L, n);
+  if (!lws || lws_bytes < w.total) return TWA_ERR_WORKSPACE;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  char* ws = static_cast<char*>(lws);
+  const long long row1 = row0 + rows;
+  int k0, k1, l0, l1;
+  chunk_range(p, L, row0, row1, &k0, &k1, &l0, &l1);
+  if (k1 <= k0 || l1 < l0) return TWA_ERR_INVALID_ARG;
+  const Item* items = reinterpret_cast<const Item*>(ws + w.items) + k0;
+  const size_t cell0 = static_cast<size_t>(k0) * n;
+  const dim3 grid(static_cast<unsigned>(k1 - k0), static_cast<unsigned>(n));
+  const double* inv = reinterpret_cast<const double*>(ws + w.inv);
+  if (pass == 0) {
+    rc = twa_mean(ctx, chunk, rows, n, ld, wbar + row0);
+    if (rc) return rc;
+    chunk_centred_sumsq_kernel<<<grid, BLOCK, 0, ctx->stream>>>(chunk, ld, row0, row1, wbar, items, n,
+                                                                reinterpret_cast<double*>(ws + w.partial) + cell0);
+  } else if (pass == 1) {
+    chunk_minmax_kernel<<<grid, BLOCK, 0, ctx->stream>>>(chunk, ld, row0, row1, wbar, items, n, inv,
+                                                         reinterpret_cast<float*>(ws + w.pmin) + cell0,
+                                                         reinterpret_cast<float*>(ws + w.pmax) + cell0, q32_out, ldq);
+  } else {
+    const int rpc = 128 / bits;
+    long long gx = (rows / rpc + 2 + BLOCK - 1) / BLOCK;
+    if (gx > 64) gx = 64;
+    const dim3 egrid(static_cast<unsigned>(gx), static_cast<unsigned>(n), static_cast<unsigned>(l1 - l0 + 1));
+    const long long* fl_d = reinterpret_cast<const long long*>(ws + w.flat);
+    const long long* in_d = reinterpret_cast<const long long*>(ws + w.internal);
+    unsigned char* codes = static_cast<unsigned char*>(lb->codes.data);
+    if (bits == 8)
+      chunk_affine_encode_kernel<8><<<egrid, BLOCK, 0, ctx->stream>>>(chunk, ld, row0, row1, wbar, inv, n, fl_d, in_d,
+                                                                      lb->a, lb->b, codes, lb->codes.col_stride, l0);
+    else
+      chunk_affine_encode_kernel<4><<<egrid, BLOCK, 0, ctx->stream>>>(chunk, ld, row0, row1, wbar, inv, n, fl_d, in_d,
+                                                                      lb->a, lb->b, codes, lb->codes.col_stride, l0);
+  }
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+int twa_layered_build_end_pass(twa_ctx* ctx, const twa_layered_basis* lb, const int64_t* offsets_host, int pass,
+                               void* lws, size_t lws_bytes) {
+  if (!ctx || !lb || !offsets_host || pass < 0 || pass > 2) return TWA_ERR_INVALID_ARG;
+  const int n = lb->codes.n, L = lb->L, bits = lb->codes.bits;
+  const LwsLayout w = lws_layout(count_items(offsets_host, L), L, n);
+  if (!lws || lws_bytes < w.total) return TWA_ERR_WORKSPACE;
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  char* ws = static_cast<char*>(lws);
+  const int* first_item = reinterpret_cast<const int*>(ws + w.first_item);
+  if (pass == 0) {
+    inv_norm_kernel<<<(L * n + 255) / 256, 256, 0, ctx->stream>>>(reinterpret_cast<const double*>(ws + w.partial),
+                                                                 first_item, L, n, reinterpret_cast<double*>(ws + w.inv),
+                                                                 ctx->d_status);
+  } else if (pass == 1) {
+    factors_kernel<<<(L + 127) / 128, 128, 0, ctx->stream>>>(reinterpret_cast<const float*>(ws + w.pmin),
+                                                             reinterpret_cast<const float*>(ws + w.pmax), first_item, L, n,
+                                                             bits == 8 ? 255.0f : 15.0f, lb->a, lb->b, ctx->d_status);
+  }
+  TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
 }
 

@@ -49,6 +49,7 @@ EXPORTS = [
     "twa_basis_export", "twa_basis_import", "twa_project", "twa_lift", "twa_step",
     "twa_step_host", "twa_step_adam", "twa_cosine_lr", "twa_weighted_average", "twa_layered_step_adam", "twa_project_batch", "twa_project_batch_group", "twa_layered_workspace_bytes", "twa_layered_rows", "twa_layered_basis_bytes",
     "twa_build_centered", "twa_quantize_affine", "twa_layered_export",
+    "twa_layered_build_begin", "twa_layered_build_feed", "twa_layered_build_end_pass",
     "twa_layered_step_workspace_bytes", "twa_layered_project", "twa_layered_lift", "twa_layered_step",
     "twa_project_noalloc", "twa_noalloc_last_error", "twa_noalloc_scratch_bytes",
 ]
@@ -192,6 +193,12 @@ def load():
         "twa_quantize_affine": (i32, [vp, bp, ctypes.POINTER(ctypes.c_int64), i32, i32, vp, szt,
                                       ctypes.POINTER(twa_layered_basis), vp, szt]),
         "twa_layered_export": (i32, [vp, ctypes.POINTER(twa_layered_basis), vp, vp, vp]),
+        "twa_layered_build_begin": (i32, [vp, i64, i32, ctypes.POINTER(ctypes.c_int64), i32, i32, vp, szt,
+                                          ctypes.POINTER(twa_layered_basis), vp, szt]),
+        "twa_layered_build_feed": (i32, [vp, ctypes.POINTER(twa_layered_basis), ctypes.POINTER(ctypes.c_int64), i32,
+                                         vp, i64, i64, i64, vp, vp, i64, vp, szt]),
+        "twa_layered_build_end_pass": (i32, [vp, ctypes.POINTER(twa_layered_basis), ctypes.POINTER(ctypes.c_int64),
+                                             i32, vp, szt]),
         "twa_layered_step_workspace_bytes": (szt, [ctypes.POINTER(twa_layered_basis)]),
         "twa_layered_project": (i32, [vp, ctypes.POINTER(twa_layered_basis), vp, i32, vp, vp, szt]),
         "twa_layered_lift": (i32, [vp, ctypes.POINTER(twa_layered_basis), vp, vp, vp, vp, szt]),
@@ -560,6 +567,34 @@ def twa_quantize_affine(ctx, P32, layers, bits, lws):
                                     mem.numel(), ctypes.byref(desc), _ptr(lws), lws.numel())
     _check(rc, "twa_quantize_affine", ctx)
     return LayeredBasis(desc, mem, layers)
+
+
+def twa_layered_build_begin(ctx, D, n, layers, bits, lws, device):
+    """Starts a row-chunked layer-wise build; returns the (still empty) LayeredBasis."""
+    arr, L = _offsets(layers)
+    mem = torch.empty(twa_layered_basis_bytes(layers, n, bits), dtype=torch.uint8, device=device)
+    desc = twa_layered_basis()
+    rc = load().twa_layered_build_begin(ctx, int(D), int(n), arr, L, int(bits), _ptr(mem), mem.numel(),
+                                        ctypes.byref(desc), _ptr(lws), lws.numel())
+    _check(rc, "twa_layered_build_begin", ctx)
+    return LayeredBasis(desc, mem, layers)
+
+
+def twa_layered_build_feed(ctx, lb, pass_index, chunk, row0, rows, wbar, lws, q32_out=None):
+    """chunk: (n, ld) float32 CUDA tensor, candidate i's rows row0 .. row0+rows-1 in chunk[i, :rows]."""
+    assert chunk.dtype == torch.float32 and chunk.stride(1) == 1
+    arr, _ = _offsets(lb.layers)
+    ldq = q32_out.stride(0) if q32_out is not None else 0
+    rc = load().twa_layered_build_feed(ctx, ctypes.byref(lb.desc), arr, int(pass_index), _ptr(chunk),
+                                       int(chunk.stride(0)), int(row0), int(rows), _ptr(wbar), _ptr(q32_out),
+                                       int(ldq), _ptr(lws), lws.numel())
+    _check(rc, "twa_layered_build_feed", ctx)
+
+
+def twa_layered_build_end_pass(ctx, lb, pass_index, lws):
+    arr, _ = _offsets(lb.layers)
+    rc = load().twa_layered_build_end_pass(ctx, ctypes.byref(lb.desc), arr, int(pass_index), _ptr(lws), lws.numel())
+    _check(rc, "twa_layered_build_end_pass", ctx)
 
 
 def twa_layered_export(ctx, lb):

@@ -98,6 +98,89 @@ def test_quantize_affine_bit_exact(env, D, n, layers, bits):
     assert codes_g.numel() == n * ((D * bits + 7) // 8)
 
 
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("D,n,layers,chunk_rows", [
+    (1777, 6, [0, 7, 300, 301, 1000, 1777], 500),              # chunk edges inside layers and inside 16-byte code groups
+    (70001, 33, [0, 64, 1000, 1001, 30000, 30017, 65536, 70001], 8192),
+    (70001, 33, [0, 64, 1000, 1001, 30000, 30017, 65536, 70001], 70004),   # one chunk
+    (300000, 20, [0, 300000], 65536),
+    (5, 2, [0, 1, 5], 4),
+])
+def test_chunked_layered_build_matches_oracle_and_resident_build(env, D, n, layers, chunk_rows, bits):
+    """The row-chunked build gives the mean bit for bit, float32 vectors equal to the resident build's
+    up to the last bit (the norms are summed in another grouping), and codes and factors that are
+    exactly the oracle's quantiser applied to the float32 vectors of its own pass 1."""
+    ctx, _ = env
+    ld = inputs.padded_ld(D, 4)
+    W = inputs.trajectory_candidates(D, n, 0.005, 0.001, 43, DEV, ld=ld)
+    A = W[:, :D].cpu().numpy().T.copy()
+    lws = twa.new_layered_workspace(layers, n, DEV)
+    wbar = torch.full((D + 3,), 7.0, device=DEV)[:D]
+    lb = twa.twa_layered_build_begin(ctx, D, n, layers, bits, lws, DEV)
+    Q = torch.zeros((n, ld), device=DEV)
+    # the second pass runs over another chunking: the result may not depend on it
+    sizes = [chunk_rows, max(4, (chunk_rows // 3) // 4 * 4), chunk_rows]
+    for p in range(3):
+        for r0 in range(0, D, sizes[p]):
+            rows = min(sizes[p], D - r0)
+            chunk = W[:, r0:r0 + rows]                    # a view: column stride ld, 16-byte aligned start
+            twa.twa_layered_build_feed(ctx, lb, p, chunk, r0, rows, wbar, lws,
+                                       q32_out=Q[:, r0:r0 + rows] if p == 1 else None)
+        twa.twa_layered_build_end_pass(ctx, lb, p, lws)
+    status_ok(ctx)
+    P_o, wbar_o = orc.center_normalize(A, layers)
+    np.testing.assert_array_equal(wbar.cpu().numpy(), wbar_o.astype(np.float32))
+    Qg = np.asfortranarray(Q[:, :D].cpu().numpy().T)
+    # against the resident build on the same candidates
+    W2 = W.clone()
+    wbar2 = torch.empty(D, device=DEV)
+    twa.twa_build_centered(ctx, W2, D, layers, wbar2, lws)
+    Pr = W2[:, :D].cpu().numpy().T
+    assert np.max(np.abs(Qg - Pr)) <= 2 * np.finfo(np.float32).eps * max(1e-30, np.max(np.abs(Pr)))
+    scale = np.abs(A).max()
+    for l in range(len(layers) - 1):
+        r0, r1 = layers[l], layers[l + 1]
+        norms = np.linalg.norm(A[r0:r1].astype(np.float64) - wbar_o[r0:r1, None], axis=0)
+        tol = 4 * np.finfo(np.float32).eps * np.maximum(1.0, scale * np.sqrt(r1 - r0) / np.maximum(norms, 1e-300))
+        assert np.all(np.abs(Qg[r0:r1] - P_o[r0:r1]).max(axis=0) <= tol)
+    codes_g, a_g, b_g = twa.twa_layered_export(ctx, lb)
+    codes_o, a_o, b_o = orc.affine_quantize(Qg, layers, bits)
+    np.testing.assert_array_equal(a_g.cpu().numpy(), a_o)
+    np.testing.assert_array_equal(b_g.cpu().numpy(), b_o)
+    np.testing.assert_array_equal(unpack_unsigned(codes_g.cpu().numpy(), D, bits), codes_o)
+    # the basis steps like any other layered basis
+    sws = twa.new_layered_step_workspace(lb)
+    L = len(layers) - 1
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(D + n)
+    g = torch.randn(D, generator=gen, device=DEV) * 1e-3
+    c = torch.empty((L, n), device=DEV)
+    twa.twa_layered_project(ctx, lb, g, c, sws)
+    status_ok(ctx)
+    c_o = orc.project_layerwise(codes_o, layers, a_o, b_o, g.cpu().numpy())
+    scale_c = _term_scale(codes_o, layers, a_o, b_o, g.double().cpu().numpy())
+    assert np.all(np.abs(c.cpu().numpy() - c_o) <= 1e-5 * np.maximum(scale_c, 1e-30))
+
+
+def test_chunked_layered_build_rejects_bad_arguments(env):
+    ctx, _ = env
+    D, n, layers = 5000, 3, [0, 100, 5000]
+    lws = twa.new_layered_workspace(layers, n, DEV)
+    lb = twa.twa_layered_build_begin(ctx, D, n, layers, 8, lws, DEV)
+    chunk = torch.zeros((n, 1024), device=DEV)
+    wbar = torch.empty(D, device=DEV)
+    with pytest.raises(twa.TwaError) as e:
+        twa.twa_layered_build_feed(ctx, lb, 0, chunk, 4990, 1024, wbar, lws)       # past the end
+    assert e.value.code == twa.TWA_ERR_INVALID_ARG
+    with pytest.raises(twa.TwaError) as e:
+        twa.twa_layered_build_feed(ctx, lb, 0, chunk, 1022, 1024, wbar, lws)       # row0 not a multiple of 4
+    assert e.value.code == twa.TWA_ERR_MISALIGNED
+    with pytest.raises(twa.TwaError) as e:
+        twa.twa_layered_build_feed(ctx, lb, 3, chunk, 0, 1024, wbar, lws)          # no such pass
+    assert e.value.code == twa.TWA_ERR_INVALID_ARG
+    status_ok(ctx)
+
+
 def test_affine_nonfinite_is_reported(env):
     ctx, _ = env
     D, n, layers = 5000, 3, [0, 100, 5000]
