@@ -661,15 +661,29 @@ int twa_layered_export(twa_ctx* ctx, const twa_layered_basis* lb, void* codes_ou
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-// items [k0, k1) and layers [l0, l1] that meet flat rows [row0, row1)
-void chunk_range(const Partition& p, int L, long long row0, long long row1, int* k0, int* k1, int* l0, int* l1) {
-  auto by_end = [](const Item& it, long long r) { return it.r1 <= r; };
-  auto by_start = [](const Item& it, long long r) { return it.r0 < r; };
-  *k0 = static_cast<int>(std::lower_bound(p.items.begin(), p.items.end(), row0, by_end) - p.items.begin());
-  *k1 = static_cast<int>(std::lower_bound(p.items.begin(), p.items.end(), row1, by_start) - p.items.begin());
-  *l0 = static_cast<int>(std::upper_bound(p.flat.begin(), p.flat.end(), row0) - p.flat.begin()) - 1;
-  *l1 = static_cast<int>(std::lower_bound(p.flat.begin(), p.flat.end(), row1) - p.flat.begin()) - 1;
-  if (*l1 > L - 1) *l1 = L - 1;
+// Items [k0, k1) and layers [l0, l1] that meet flat rows [row0, row1), and the number of items in all,
+// from the layer offsets alone (make_partition's numbering: a layer's items follow one another,
+// ITEM_ROWS rows each).  Returns false for offsets make_partition would reject.
+bool chunk_range(const int64_t* offsets, int L, long long D, long long row0, long long row1, int* k0, int* k1,
+                 int* l0, int* l1, size_t* n_items) {
+  if (!offsets || L < 1 || offsets[0] != 0 || offsets[L] != D) return false;
+  size_t first = 0;
+  *l0 = *l1 = -1;
+  for (int l = 0; l < L; ++l) {
+    const long long a = offsets[l], b = offsets[l + 1];
+    if (b <= a) return false;
+    if (row0 >= a && row0 < b) {
+      *l0 = l;
+      *k0 = static_cast<int>(first + static_cast<size_t>((row0 - a) / ITEM_ROWS));
+    }
+    if (row1 - 1 >= a && row1 - 1 < b) {
+      *l1 = l;
+      *k1 = static_cast<int>(first + static_cast<size_t>((row1 - 1 - a) / ITEM_ROWS)) + 1;
+    }
+    first += static_cast<size_t>((b - a + ITEM_ROWS - 1) / ITEM_ROWS);
+  }
+  *n_items = first;
+  return *l0 >= 0 && *l1 >= *l0;
 }
 
 }  // namespace
@@ -715,17 +729,14 @@ int twa_layered_build_feed(twa_ctx* ctx, const twa_layered_basis* lb, const int6
   // the mean of the chunk is written with 16-byte stores at wbar + row0
   if ((reinterpret_cast<uintptr_t>(chunk) & 15) || (ld & 3) || (row0 & 3) || (reinterpret_cast<uintptr_t>(wbar) & 15))
     return TWA_ERR_MISALIGNED;
-  Partition p;
-  int rc = make_partition(offsets_host, L, D, bits, &p);
-  if (rc) return rc;
-  const LwsLayout w = lws_layout(p.items.size(), L, n);
+  const long long row1 = row0 + rows;
+  int k0 = 0, k1 = 0, l0, l1, rc;
+  size_t n_items;
+  if (!chunk_range(offsets_host, L, D, row0, row1, &k0, &k1, &l0, &l1, &n_items) || k1 <= k0) return TWA_ERR_INVALID_ARG;
+  const LwsLayout w = lws_layout(n_items, L, n);
   if (!lws || lws_bytes < w.total) return TWA_ERR_WORKSPACE;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
   char* ws = static_cast<char*>(lws);
-  const long long row1 = row0 + rows;
-  int k0, k1, l0, l1;
-  chunk_range(p, L, row0, row1, &k0, &k1, &l0, &l1);
-  if (k1 <= k0 || l1 < l0) return TWA_ERR_INVALID_ARG;
   const Item* items = reinterpret_cast<const Item*>(ws + w.items) + k0;
   const size_t cell0 = static_cast<size_t>(k0) * n;
   const dim3 grid(static_cast<unsigned>(k1 - k0), static_cast<unsigned>(n));
