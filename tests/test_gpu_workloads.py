@@ -387,3 +387,85 @@ def test_workload_layerwise_sampled(env, name, bits_list):
             assert abs(c_h[:, i].astype(np.float64).sum() - total) <= 1e-5 * np.abs(c_h[:, i]).sum()
         del lb, packed, sws
         torch.cuda.empty_cache()
+
+
+def test_workload_decoder_layerwise_chunked_sampled(env):
+    """The paper's default construction at the 1.3 B size, built from row chunks: mean rows, per-layer
+    factors and sampled codes bit-exact against the oracle on the float32 vectors of the build's own
+    second pass; one layer-wise step checked on sampled layers, columns and rows."""
+    ctx, _ = env
+    wl = inputs.WORKLOADS["decoder1p3b"]
+    D, n, bits = wl.D, wl.n, 8
+    layers = inputs.layer_offsets("decoder1p3b")
+    L = len(layers) - 1
+    sizes = np.diff(layers)
+    CH = inputs.CHUNK_ROWS
+    # a bias (2048 rows), a 2048 x 2048 matrix, the layer after the embedding, the last layer
+    pick = sorted({1, int(np.argmin(sizes)), int(np.where(sizes == 4194304)[0][len(sizes) // 8]), L - 1})
+    blocks = {l: np.empty((layers[l + 1] - layers[l], n), dtype=np.float32, order="F") for l in pick}
+    first_rows = {}
+    lws = twa.new_layered_workspace(layers, n, DEV)
+    wbar = torch.empty(D, device=DEV)
+    lb = twa.twa_layered_build_begin(ctx, D, n, layers, bits, lws, DEV)
+    buf = torch.empty((n, CH), device=DEV)
+    qbuf = torch.empty((n, CH), device=DEV)
+    for p in range(3):
+        for r0 in range(0, D, CH):
+            rows = min(CH, D - r0)
+            inputs.trajectory_rows(D, n, wl.step, wl.drift, wl.seed, DEV, row0=r0, rows=rows, out=buf[:, :rows])
+            hit = [l for l in pick if layers[l] < r0 + rows and layers[l + 1] > r0] if p == 1 else []
+            twa.twa_layered_build_feed(ctx, lb, p, buf, r0, rows, wbar, lws, q32_out=qbuf if hit else None)
+            for l in hit:
+                a0, a1 = max(layers[l], r0), min(layers[l + 1], r0 + rows)
+                blocks[l][a0 - layers[l]:a1 - layers[l]] = qbuf[:, a0 - r0:a1 - r0].cpu().numpy().T
+            if p == 0 and r0 in (0, (D // CH) * CH):
+                first_rows[r0] = buf[:, :min(rows, 100000)].cpu().numpy().T.copy()
+        twa.twa_layered_build_end_pass(ctx, lb, p, lws)
+    status_ok(ctx)
+    del buf, qbuf
+    torch.cuda.empty_cache()
+    for r0, a_rows in first_rows.items():
+        np.testing.assert_array_equal(wbar[r0:r0 + a_rows.shape[0]].cpu().numpy(), orc.mean(a_rows).astype(np.float32))
+    packed, a_g, b_g = twa.twa_layered_export(ctx, lb)
+    a_h, b_h = a_g.cpu().numpy(), b_g.cpu().numpy()
+    cols = [0, n // 2, n - 1]
+    for l in pick:
+        r0, r1 = layers[l], layers[l + 1]
+        blk = blocks[l]
+        # unit columns per layer, factors and codes of the oracle's quantiser on these float32 values
+        assert np.max(np.abs(np.sum(blk.astype(np.float64) ** 2, axis=0) - 1.0)) <= TOL
+        a_o, b_o = orc.affine_factors(blk, [0, r1 - r0], bits)
+        assert (a_h[l], b_h[l]) == (a_o[0], b_o[0])
+        codes_o = orc.affine_encode(np.asfortranarray(blk[:, cols]), [0, r1 - r0], a_o, b_o, bits)
+        np.testing.assert_array_equal(_unpack_rows(packed, r0, r1, bits)[:, cols], codes_o)
+    blocks.clear()
+    # one step from beta = 0
+    g = wl.gradient(0, DEV)
+    sws = twa.new_layered_step_workspace(lb)
+    beta = torch.zeros((L, n), device=DEV)
+    c = torch.empty((L, n), device=DEV)
+    w = torch.empty(D, device=DEV)
+    twa.twa_layered_step(ctx, lb, g, LR, 0.0, beta, wbar, w, sws, c_out=c)
+    status_ok(ctx)
+    c_h, beta_h = c.cpu().numpy(), beta.cpu().numpy()
+    np.testing.assert_allclose(beta_h, -LR * c_h.astype(np.float64), rtol=1e-6, atol=1e-30)
+    for l in pick:
+        r0, r1 = layers[l], layers[l + 1]
+        g_l = g[r0:r1].float().cpu().numpy().astype(np.float64)
+        codes = _unpack_rows(packed, r0, r1, bits)[:, cols]
+        c_o = orc.project_layerwise(codes, [0, r1 - r0], a_h[l:l + 1], b_h[l:l + 1], g_l)
+        scale = abs(float(a_h[l])) * (codes.astype(np.float64).T @ np.abs(g_l)) + abs(float(b_h[l])) * np.abs(g_l).sum()
+        assert np.all(np.abs(c_h[l, cols] - c_o[0]) <= 2e-6 * scale + 1e-30)
+    for base in (wbar, None):
+        if base is None:
+            twa.twa_layered_lift(ctx, lb, beta, None, w, sws)
+            status_ok(ctx)
+        for l in pick:
+            r0, r1 = layers[l], layers[l + 1]
+            span = min(r1 - r0, 3001)
+            for s0 in sorted({r0, r0 + (r1 - r0 - span) // 2, r1 - span}):
+                lo = s0 - (s0 % 2)
+                rows_codes = _unpack_rows(packed, lo, s0 + span, bits)[s0 - lo:, :]
+                w_o = orc.lift_layerwise(rows_codes, [0, span], a_h[l:l + 1], b_h[l:l + 1], beta_h[l:l + 1],
+                                         None if base is None else base[s0:s0 + span].cpu().numpy())
+                assert rel(w[s0:s0 + span].cpu().numpy(), w_o) <= TOL
