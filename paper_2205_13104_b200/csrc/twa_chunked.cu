@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
   extern __shared__ __align__(16) unsigned char sm[];
   float* As = reinterpret_cast<float*>(sm);                                   // [NP][ASTR]
   double* Ms = reinterpret_cast<double*>(sm + sizeof(float) * NP * ASTR + 8); // [NP][NP]
-  double* T = Ms + NP * NP;                                                   // [NP][ASTR] (mode 1)
+  double* T = Ms + NP * NP;                                                   // [NP][ASTR] (mode 1; mode 0 keeps its copy at Ms)
   float* Tq = reinterpret_cast<float*>(T);                                    // [NP][ASTR] (mode 3)
   __shared__ unsigned smax[NP];
   const int tid = threadIdx.x;
@@ -85,9 +85,13 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
   for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     const long long r = tile * RT + tid;            // row inside the chunk
     const bool valid = r < a.rows;
-#pragma unroll 4
-    for (int j = 0; j < NP; ++j)
-      As[j * ASTR + tid] = (j < a.n && valid) ? __ldcs(a.A + j * a.ld + r) : 0.0f;
+    // all of the row's loads are issued before the first is used: with four in flight per thread the
+    // passes ran at a tenth of the memory rate
+    float row[NP];
+#pragma unroll
+    for (int j = 0; j < NP; ++j) row[j] = (j < a.n && valid) ? __ldcs(a.A + j * a.ld + r) : 0.0f;
+#pragma unroll
+    for (int j = 0; j < NP; ++j) As[j * ASTR + tid] = row[j];
     __syncthreads();
 
     if (MODE == 0) {
@@ -96,13 +100,19 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
         for (int j = 0; j < a.n; ++j) s += As[j * ASTR + tid];
         a.wbar[a.row0 + r] = static_cast<float>(s / static_cast<double>(a.n));
       }
+      // the tile once more as float64 (Ms is free in this mode): one conversion per element instead
+      // of six per product group in the loop below, which made this pass the slowest of the four
+      double* T0 = Ms;
+#pragma unroll
+      for (int j = 0; j < NP; ++j) T0[j * ASTR + tid] = static_cast<double>(row[j]);
+      __syncthreads();
 #pragma unroll 2
       for (int k = 0; k < RT; ++k) {
         double x[IB], y[JB];
 #pragma unroll
-        for (int u = 0; u < IB; ++u) x[u] = As[(ti + 8 * u) * ASTR + k];
+        for (int u = 0; u < IB; ++u) x[u] = T0[(ti + 8 * u) * ASTR + k];
 #pragma unroll
-        for (int v = 0; v < JB; ++v) y[v] = As[(tj + 16 * v) * ASTR + k];
+        for (int v = 0; v < JB; ++v) y[v] = T0[(tj + 16 * v) * ASTR + k];
 #pragma unroll
         for (int u = 0; u < IB; ++u)
 #pragma unroll
@@ -261,7 +271,7 @@ template <int NP, int MODE>
 int launch_chunk(twa_ctx* ctx, const ChunkArgs& a, int grid) {
   size_t smem = sizeof(float) * NP * ASTR + 8;
   if (MODE >= 1) smem += sizeof(double) * NP * NP;
-  if (MODE == 1) smem += sizeof(double) * NP * ASTR;
+  if (MODE <= 1) smem += sizeof(double) * NP * ASTR;      // the tile (mode 0) or A*M (mode 1) as float64
   if (MODE == 3) smem += sizeof(float) * NP * ASTR;
   auto kern = chunk_kernel<NP, MODE>;
   static int smem_limit[64] = {0};
