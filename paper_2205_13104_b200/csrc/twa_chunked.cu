@@ -21,6 +21,7 @@ namespace {
 
 constexpr int RT = 128;                 // rows per tile = threads per block
 constexpr int ASTR = RT + 1;            // padded strides: conflict-free column-strided reads
+constexpr int DSTR = RT + 4;            // stride of the float64 tile: the matrix-fragment loads below are conflict-free
 constexpr int MAX_BLOCKS = 512;
 constexpr int BUILD_MAX_N = 64;
 
@@ -57,6 +58,40 @@ BuildLayout layout_for(int np) {
 }
 int padded_n(int n) { return (n + 15) / 16 * 16; }
 
+// d += a (8 x 4, row-major) * b (4 x 8, column-major) in float64 on the tensor pipe: lane l holds
+// a[l >> 2][l & 3], b[l & 3][l >> 2] and d[l >> 2][2 * (l & 3) + {0, 1}].
+__device__ __forceinline__ void dmma_8x8x4(double (&d)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+               : "+d"(d[0]), "+d"(d[1])
+               : "d"(a), "d"(b));
+}
+
+// Gram matrix of a tile held column by column in float64 (T[c * DSTR + r], RT rows, NP columns):
+// warp w takes the 8-row bands w, w + 4, ... of G and all NP / 8 column blocks of each; one
+// tensor-pipe product per 8 x 8 block and 4 rows, the rows in order.  With scalar float64 FMAs this
+// loop issued seven times the instructions and the Gram passes ran at a quarter of the float64 rate.
+template <int NP>
+__device__ __forceinline__ void gram_accumulate(const double* T, double (&acc)[(NP / 8 + 3) / 4][NP / 8][2], int warp,
+                                                int lane) {
+  constexpr int NB = NP / 8, IBW = (NB + 3) / 4;
+  const int off = (lane >> 2) * DSTR + (lane & 3);
+#pragma unroll 2
+  for (int k0 = 0; k0 < RT; k0 += 4) {
+    double b[NB];
+#pragma unroll
+    for (int jb = 0; jb < NB; ++jb) b[jb] = T[jb * 8 * DSTR + off + k0];
+#pragma unroll
+    for (int u = 0; u < IBW; ++u) {
+      const int ib = warp + 4 * u;
+      if (ib < NB) {
+        const double av = T[ib * 8 * DSTR + off + k0];
+#pragma unroll
+        for (int jb = 0; jb < NB; ++jb) dmma_8x8x4(acc[u][jb], av, b[jb]);
+      }
+    }
+  }
+}
+
 // MODE 0: mean rows + Gram of A.  MODE 1: Gram of A*M.  MODE 2: absmax (and float32 copy) of A*M.
 // MODE 3: codes of A*M.
 template <int NP, int MODE>
@@ -64,22 +99,36 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
   extern __shared__ __align__(16) unsigned char sm[];
   float* As = reinterpret_cast<float*>(sm);                                   // [NP][ASTR]
   double* Ms = reinterpret_cast<double*>(sm + sizeof(float) * NP * ASTR + 8); // [NP][NP]
-  double* T = Ms + NP * NP;                                                   // [NP][ASTR] (mode 1; mode 0 keeps its copy at Ms)
-  float* Tq = reinterpret_cast<float*>(T);                                    // [NP][ASTR] (mode 3)
+  double* T = Ms + NP * NP;                                                   // [NP][DSTR] (mode 1; mode 0 keeps its copy at Ms)
+  float* Tq = reinterpret_cast<float*>(T);                                    // [NP][ASTR] (modes 2, 3)
   __shared__ unsigned smax[NP];
   const int tid = threadIdx.x;
-  constexpr int IB = NP / 8, JB = NP / 16;
-  const int ti = tid >> 4, tj = tid & 15;          // Gram: rows ti + 8a, columns tj + 16b
+  constexpr int NB = NP / 8, IBW = (NB + 3) / 4;   // Gram: 8 x 8 blocks; bands of G per warp
+  const int warp = tid >> 5, lane = tid & 31;
 
   if (MODE >= 1)
     for (int i = tid; i < NP * NP; i += RT) Ms[i] = a.M[i];
   if (MODE == 2 && tid < NP) smax[tid] = 0u;
-  double acc[IB][JB];
+  // Fragment (kb, jb) of M for the products below: M[4 kb + (lane & 3)][8 jb + (lane >> 2)]; kept in
+  // registers for NP <= 32 (20 values), read from shared memory for wider bases.
+  constexpr bool MREG = NP <= 32;
+  double mreg[MREG ? NB * (NP / 4) : 1] = {0.0};
+  auto mfrag = [&](int kb, int jb) -> double {
+    return MREG ? mreg[jb * (NP / 4) + kb] : Ms[(kb * 4 + (lane & 3)) * NP + jb * 8 + (lane >> 2)];
+  };
+  double acc[IBW][NB][2];
 #pragma unroll
-  for (int x = 0; x < IB; ++x)
+  for (int x = 0; x < IBW; ++x)
 #pragma unroll
-    for (int y = 0; y < JB; ++y) acc[x][y] = 0.0;
+    for (int y = 0; y < NB; ++y) acc[x][y][0] = acc[x][y][1] = 0.0;
   __syncthreads();
+  if (MODE >= 1 && MREG) {
+#pragma unroll
+    for (int jb = 0; jb < NB; ++jb)
+#pragma unroll
+      for (int kb = 0; kb < NP / 4; ++kb)
+        mreg[jb * (NP / 4) + kb] = kb <= 2 * jb + 1 ? Ms[(kb * 4 + (lane & 3)) * NP + jb * 8 + (lane >> 2)] : 0.0;
+  }
 
   const long long ntiles = (a.rows_padded + RT - 1) / RT;
   for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
@@ -100,65 +149,55 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
         for (int j = 0; j < a.n; ++j) s += As[j * ASTR + tid];
         a.wbar[a.row0 + r] = static_cast<float>(s / static_cast<double>(a.n));
       }
-      // the tile once more as float64 (Ms is free in this mode): one conversion per element instead
-      // of six per product group in the loop below, which made this pass the slowest of the four
+      // the tile once more as float64 (Ms is free in this mode)
       double* T0 = Ms;
 #pragma unroll
-      for (int j = 0; j < NP; ++j) T0[j * ASTR + tid] = static_cast<double>(row[j]);
+      for (int j = 0; j < NP; ++j) T0[j * DSTR + tid] = static_cast<double>(row[j]);
       __syncthreads();
-#pragma unroll 2
-      for (int k = 0; k < RT; ++k) {
-        double x[IB], y[JB];
-#pragma unroll
-        for (int u = 0; u < IB; ++u) x[u] = T0[(ti + 8 * u) * ASTR + k];
-#pragma unroll
-        for (int v = 0; v < JB; ++v) y[v] = T0[(tj + 16 * v) * ASTR + k];
-#pragma unroll
-        for (int u = 0; u < IB; ++u)
-#pragma unroll
-          for (int v = 0; v < JB; ++v) acc[u][v] = fma(x[u], y[v], acc[u][v]);
-      }
+      gram_accumulate<NP>(T0, acc, warp, lane);
     } else {
-      // this thread's row of A*M: q[j] = sum_{i <= j} a_i M[i][j]
-      double q[NP];
+      // the tile's rows of A*M, q[r][j] = sum_{i <= j} a[r][i] M[i][j], as float64 tensor-pipe products:
+      // warp w takes the 8-row bands 4w .. 4w+3 of the tile; a band's fragment of A serves all column
+      // blocks; blocks of M below the diagonal are skipped.  (One thread per row with scalar FMAs
+      // took 528 shared-memory reads and as many FMAs per row at n = 32.)
+#pragma unroll 1
+      for (int u = 0; u < RT / 32; ++u) {
+        const int r0 = (warp * (RT / 32) + u) * 8;
+        double c[NB][2];
 #pragma unroll
-      for (int j = 0; j < NP; ++j) q[j] = 0.0;
+        for (int jb = 0; jb < NB; ++jb) c[jb][0] = c[jb][1] = 0.0;
 #pragma unroll
-      for (int i = 0; i < NP; ++i) {
-        const double ai = As[i * ASTR + tid];
+        for (int kb = 0; kb < NP / 4; ++kb) {
+          const double av = static_cast<double>(As[(kb * 4 + (lane & 3)) * ASTR + r0 + (lane >> 2)]);
 #pragma unroll
-        for (int j = i; j < NP; ++j) q[j] = fma(ai, Ms[i * NP + j], q[j]);
-      }
-      if (MODE == 1) {
-#pragma unroll
-        for (int j = 0; j < NP; ++j) T[j * ASTR + tid] = q[j];
-        __syncthreads();
-#pragma unroll 2
-        for (int k = 0; k < RT; ++k) {
-          double x[IB], y[JB];
-#pragma unroll
-          for (int u = 0; u < IB; ++u) x[u] = T[(ti + 8 * u) * ASTR + k];
-#pragma unroll
-          for (int v = 0; v < JB; ++v) y[v] = T[(tj + 16 * v) * ASTR + k];
-#pragma unroll
-          for (int u = 0; u < IB; ++u)
-#pragma unroll
-            for (int v = 0; v < JB; ++v) acc[u][v] = fma(x[u], y[v], acc[u][v]);
+          for (int jb = kb >> 1; jb < NB; ++jb) dmma_8x8x4(c[jb], av, mfrag(kb, jb));
         }
+#pragma unroll
+        for (int jb = 0; jb < NB; ++jb) {
+          const int col = jb * 8 + 2 * (lane & 3), rr = r0 + (lane >> 2);
+          if (MODE == 1) {
+            T[col * DSTR + rr] = c[jb][0];
+            T[(col + 1) * DSTR + rr] = c[jb][1];
+          } else {
+            Tq[col * ASTR + rr] = static_cast<float>(c[jb][0]);
+            Tq[(col + 1) * ASTR + rr] = static_cast<float>(c[jb][1]);
+          }
+        }
+      }
+      __syncthreads();
+      if (MODE == 1) {
+        gram_accumulate<NP>(T, acc, warp, lane);
       } else {
 #pragma unroll
         for (int j = 0; j < NP; ++j) {
-          const float qf = static_cast<float>(q[j]);
+          const float qf = Tq[j * ASTR + tid];
           if (a.q32 && valid && j < a.n) a.q32[j * a.ldq + r] = qf;
           if (MODE == 2) {
             const unsigned m = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(qf) & 0x7FFFFFFFu);
             if ((tid & 31) == 0 && j < a.n) atomicMax(&smax[j], m);
-          } else {
-            Tq[j * ASTR + tid] = qf;
           }
         }
         if (MODE == 3) {
-          __syncthreads();
           // 16 output bytes per task: 16 rows (8-bit) or 32 rows (4-bit) of one column
           const int rows_per_chunk = 128 / a.bits;
           const int chunks_per_col = RT / rows_per_chunk;
@@ -190,9 +229,17 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
   if (MODE <= 1) {
     double* out = a.partials + static_cast<size_t>(blockIdx.x) * NP * NP;
 #pragma unroll
-    for (int u = 0; u < IB; ++u)
+    for (int u = 0; u < IBW; ++u) {
+      const int ib = warp + 4 * u;
+      if (ib < NB) {
 #pragma unroll
-      for (int v = 0; v < JB; ++v) out[(ti + 8 * u) * NP + tj + 16 * v] = acc[u][v];
+        for (int jb = 0; jb < NB; ++jb) {
+          double* at = out + (ib * 8 + (lane >> 2)) * NP + jb * 8 + 2 * (lane & 3);
+          at[0] = acc[u][jb][0];
+          at[1] = acc[u][jb][1];
+        }
+      }
+    }
   }
   if (MODE == 2) {
     __syncthreads();
@@ -271,8 +318,8 @@ template <int NP, int MODE>
 int launch_chunk(twa_ctx* ctx, const ChunkArgs& a, int grid) {
   size_t smem = sizeof(float) * NP * ASTR + 8;
   if (MODE >= 1) smem += sizeof(double) * NP * NP;
-  if (MODE <= 1) smem += sizeof(double) * NP * ASTR;      // the tile (mode 0) or A*M (mode 1) as float64
-  if (MODE == 3) smem += sizeof(float) * NP * ASTR;
+  if (MODE <= 1) smem += sizeof(double) * NP * DSTR;      // the tile (mode 0) or A*M (mode 1) as float64
+  if (MODE >= 2) smem += sizeof(float) * NP * ASTR;        // A*M as float32
   auto kern = chunk_kernel<NP, MODE>;
   static int smem_limit[64] = {0};
   if (smem > 48 * 1024) {
