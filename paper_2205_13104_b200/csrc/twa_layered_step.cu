@@ -601,7 +601,7 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
   uint32_t bfrag[KS][2];
 #pragma unroll
   for (int ks = 0; ks < KS; ++ks) bfrag[ks][0] = bfrag[ks][1] = 0u;
-  float wa = 0.0f, wbw = 0.0f, kon = 0.0f;
+  float wbw = 0.0f, kon = 0.0f;
   int cur_layer = -1;
   volatile int* abort_flag = &hdr->abort_flag;
   int s = 0;
@@ -635,9 +635,8 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
       const int eb = a.ebits[cur_layer];
       const float w0 = eb <= 0 ? 0.0f : (eb >= 6 ? __uint_as_float(static_cast<uint32_t>(eb - 5) << 23) : 5.877471754e-39f);
       const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
-      wa = tig == 0 ? w0 : (tig == 1 ? w2 : 0.0f);
-      wbw = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);
-      if (BITS == 4) { wa *= 0.0625f; wbw *= 0.0625f; }
+      wbw = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);      // weight of the lower digit of this lane's pair
+      if (BITS == 4) wbw *= 0.0625f;
       kon = eb < 0 ? __int_as_float(0x7FC00000) : a.konst[cur_layer];
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
@@ -686,14 +685,14 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
             }
           }
           float v[LROWS];
-          if (BITS == 8) {
-            v[0] = fmaf(small_int_to_float(acc0[1]), wbw, small_int_to_float(acc0[0]) * wa);
-            v[1] = fmaf(small_int_to_float(acc0[3]), wbw, small_int_to_float(acc0[2]) * wa);
+          if (BITS == 8) {                                // digit pairs (0,1) in lanes tig = 0, (2,3) in tig = 1
+            v[0] = digit_pair_to_float(acc0[0], acc0[1], wbw);
+            v[1] = digit_pair_to_float(acc0[2], acc0[3], wbw);
           } else {
-            v[0] = fmaf(small_int_to_float(acc0[1]), wbw, small_int_to_float(acc0[0]) * wa);
-            v[2] = fmaf(small_int_to_float(acc0[3]), wbw, small_int_to_float(acc0[2]) * wa);
-            v[1] = fmaf(small_int_to_float(acc1[1]), wbw, small_int_to_float(acc1[0]) * wa);
-            v[3] = fmaf(small_int_to_float(acc1[3]), wbw, small_int_to_float(acc1[2]) * wa);
+            v[0] = digit_pair_to_float(acc0[0], acc0[1], wbw);
+            v[2] = digit_pair_to_float(acc0[2], acc0[3], wbw);
+            v[1] = digit_pair_to_float(acc1[0], acc1[1], wbw);
+            v[3] = digit_pair_to_float(acc1[2], acc1[3], wbw);
           }
 #pragma unroll
           for (int i = 0; i < LROWS; ++i) {

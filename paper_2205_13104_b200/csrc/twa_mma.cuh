@@ -42,6 +42,12 @@ __device__ __forceinline__ float small_int_to_float(int v) {
   return __int_as_float(0x4B400000 + v) - RND;
 }
 
+// Two neighbouring digit sums as one float: (128 * hi + lo) * w_lo, w_lo the weight of the lower digit.
+// The integer has up to 27 bits; its conversion rounds once (2^-24 relative).
+__device__ __forceinline__ float digit_pair_to_float(int hi, int lo, float w_lo) {
+  return static_cast<float>(hi * 128 + lo) * w_lo;
+}
+
 // Four signed base-128 digits of t (|t| <= 64): t = d0 + d1/128 + d2/128^2 + d3/128^3 + eps,
 // |eps| <= 2^-22, every digit in [-64, 64].  Returned packed, digit k in byte k.
 __device__ __forceinline__ uint32_t cut_digits(float t) {

@@ -340,9 +340,8 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
 
   const float w0 = !live ? 0.0f : (ebits >= 6u ? __uint_as_float((ebits - 5u) << 23) : 5.877471754e-39f);
   const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
-  float wa = tig == 0 ? w0 : (tig == 1 ? w2 : 0.0f);
-  float wb = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);
-  if (BITS == 4) { wa *= 0.0625f; wb *= 0.0625f; }
+  float wb = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);    // weight of the lower digit of this lane's pair
+  if (BITS == 4) wb *= 0.0625f;                         // 4-bit codes enter the MMA times 16
   const float poison = bad ? __int_as_float(0x7FC00000) : 0.0f;
 
   // B fragments: k-slot 4*tig+i of a 32-column step holds column j0 + {2tig, 2tig+1, 8+2tig, 9+2tig}[i]
@@ -474,14 +473,16 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
           // digit sums -> float; the four digits of a row sit in lanes tig = 0 and 1 of its quad,
           // and only those two lanes need the total
           float v[LROWS];
+          // lane tig = 0 holds the sums of digits 0 and 1 of its rows, tig = 1 those of digits 2 and 3
+          // (wb is the weight of the lower digit of the pair; 0 in lanes tig >= 2)
           if (BITS == 8) {
-            v[0] = fmaf(small_int_to_float(acc0[1]), wb, small_int_to_float(acc0[0]) * wa);
-            v[1] = fmaf(small_int_to_float(acc0[3]), wb, small_int_to_float(acc0[2]) * wa);
+            v[0] = digit_pair_to_float(acc0[0], acc0[1], wb);
+            v[1] = digit_pair_to_float(acc0[2], acc0[3], wb);
           } else {
-            v[0] = fmaf(small_int_to_float(acc0[1]), wb, small_int_to_float(acc0[0]) * wa);
-            v[2] = fmaf(small_int_to_float(acc0[3]), wb, small_int_to_float(acc0[2]) * wa);
-            v[1] = fmaf(small_int_to_float(acc1[1]), wb, small_int_to_float(acc1[0]) * wa);
-            v[3] = fmaf(small_int_to_float(acc1[3]), wb, small_int_to_float(acc1[2]) * wa);
+            v[0] = digit_pair_to_float(acc0[0], acc0[1], wb);
+            v[2] = digit_pair_to_float(acc0[2], acc0[3], wb);
+            v[1] = digit_pair_to_float(acc1[0], acc1[1], wb);
+            v[3] = digit_pair_to_float(acc1[2], acc1[3], wb);
           }
 #pragma unroll
           for (int i = 0; i < LROWS; ++i) {
