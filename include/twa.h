@@ -104,7 +104,10 @@ const char* twa_last_error(const twa_ctx* ctx);
 /* Tuning knobs for measurements; value 0 restores the built-in choice.
  *  TWA_TUNE_PROJECT_WARPS / TWA_TUNE_LIFT_WARPS: consumer warps per block (8..20; lift: even, >= 16)
  *  TWA_TUNE_STAGES: depth of the shared-memory ring (2..16)
- *  TWA_TUNE_WAIT_LIMIT_MS: bound of every in-kernel wait (default 2000 ms)
+ *  TWA_TUNE_WAIT_LIMIT_MS: bound of every in-kernel wait (default 2000 ms).  The limit is
+ *      wall-clock time (%globaltimer), not time the kernel was running: where the GPU is
+ *      time-sliced with other contexts, or a tool serialises kernels, a block that was off the
+ *      GPU for longer reports TWA_ERR_TIMEOUT with nothing wrong -- raise the limit there.
  *  TWA_TUNE_DEQUANT_PATH: how 8/4-bit codes meet g and alpha: 0 = exact integer dot products
  *      on the tensor pipe against block-fixed-point digits of g / alpha (default),
  *      1 = code -> float32 conversion and float32 FMA.  The warp and stage knobs act on the
@@ -154,8 +157,14 @@ size_t twa_workspace_bytes(int64_t D, int n, int bits);
 /* w_bar and the orthonormal basis of the n candidates.
  *  W        in/out: D x n float32 candidates, column i = w_i, column stride ldw ELEMENTS
  *           (ldw >= D, ldw % 4 == 0).  Overwritten by the basis: on return column j holds
- *           e_j, obtained by classical Gram-Schmidt with one re-orthogonalisation, column
- *           after column in the given order, each normalised to unit length.
+ *           e_j, the j-th vector of the Gram-Schmidt orthonormalisation of the candidates in
+ *           the given order (the factor Q of A = QR with positive diagonal).  Schedule: block
+ *           classical Gram-Schmidt with one re-orthogonalisation -- panels of 8 columns are
+ *           first made orthogonal to all earlier vectors (twice), then orthonormalised among
+ *           themselves from the panel's float64 Gram matrix (its Cholesky factor holds the
+ *           Gram-Schmidt coefficients), twice.  TWA_TUNE_BUILD_PANEL = 1 selects the literal
+ *           column-after-column schedule (two projection passes per column); both give the
+ *           same factor up to rounding.
  *  wbar_out out: D floats, the mean of the candidates (written before W is overwritten).
  *  P32_out  out (host struct): filled with {W, NULL, D, 4*ldw, n, 32}.
  * Device-side errors: TWA_ERR_NONFINITE, TWA_ERR_RANK_DEFICIENT (a column whose remainder
@@ -189,6 +198,9 @@ int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float
  *          the whole basis pass base + row0 and the full column stride).  With bits == 32
  *          this is the only output and pass 3 is not run.
  *  Pq      the caller sets data (twa_basis_bytes) and scales before twa_build_end_pass(2).
+ *          Several widths from one build: call twa_build_end_pass(ctx, 2, bits, Pq) once per
+ *          width (each takes its scales from the same column absmax) and feed every chunk of
+ *          pass 3 once per Pq; the rule "each row range once per pass" then holds per Pq.
  *  bws     device scratch of twa_build_workspace_bytes(n) bytes, alive until the last call.
  * Device-side errors: TWA_ERR_RANK_DEFICIENT (same 1e-5 rule as twa_build_basis),
  * TWA_ERR_NONFINITE.  Codes are exactly the quantiser applied to the float32 rows of pass 2. */
@@ -254,7 +266,10 @@ int twa_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, const float* 
 /* One training iteration of the subspace: c = P~^T g; alpha <- (1 - lr*lambda) alpha - lr c;
  * w = wbar + P~ alpha.  alpha (n floats) is updated in place; w (D floats) is overwritten and
  * may be the same buffer as wbar only if the caller wants wbar replaced.  c_out (n floats)
- * receives c and may be NULL. */
+ * receives c and may be NULL.  alpha is state that outlives the call: when any coefficient of c is
+ * not finite (TWA_ERR_NONFINITE) or a wait ran out in the projection (TWA_ERR_TIMEOUT) alpha is left
+ * as it was (w is then lifted from the old alpha), so the step can be repeated after
+ * twa_clear_status. */
 int twa_step(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype, float lr,
              float lambda, float* alpha, const float* wbar, float* w, float* c_out, void* ws,
              size_t ws_bytes);
@@ -418,7 +433,9 @@ int twa_layered_step_adam(twa_ctx* ctx, const twa_layered_basis* lb, const void*
  *  status_out           device, 2 ints, or NULL: receives {TWA_OK or the device-side error,
  *                       detail} when the kernel has run.
  * Limits: n <= TWA_MAX_N (128) columns and at most 256 blocks of partial sums; a larger n is
- * rejected with TWA_ERR_UNSUPPORTED and a message in twa_noalloc_last_error().
+ * rejected with TWA_ERR_UNSUPPORTED.  twa_noalloc_last_error() gives the reason of the calling
+ * thread's last rejected call; it is meaningful only right after a negative return value (a
+ * call that is accepted clears it).
  * The first call on a device looks up the device address of the array and the driver entry
  * point it needs; make that first call before any stream capture begins.
  * All calls on one device share the array: the call clears the counter and the status on the

@@ -169,6 +169,31 @@ __device__ __forceinline__ bool twa_mbar_wait(uint32_t bar, uint32_t parity, vol
   }
 }
 
+// Called by the thread that filled a ring of `stages` stages `issued` times, once it has issued its
+// last copy: waits (for at most `limit_ns` per stage) until the newest fill of every stage has
+// landed, so that no bulk copy is still writing this block's shared memory when the block reuses the
+// ring or exits -- also when the consumers gave up on a wait of their own.  Returns false if a
+// fill did not land in time.
+__device__ __forceinline__ bool twa_drain_ring(twa_smem_header* hdr, int issued, int stages,
+                                               unsigned long long limit_ns) {
+  bool landed = true;
+  const int live = issued < stages ? issued : stages;
+  for (int q = 0; q < live; ++q) {
+    const int last = ((issued - 1 - q) / stages) * stages + q;   // newest fill of stage q
+    const unsigned par = static_cast<unsigned>(last / stages) & 1u;
+    const uint32_t bar = twa_smem_u32(&hdr->full[q]);
+    if (twa_mbar_try_wait(bar, par)) continue;
+    const unsigned long long t0 = twa_globaltimer();
+    while (!twa_mbar_try_wait(bar, par)) {
+      if (twa_globaltimer() - t0 > limit_ns) {
+        landed = false;
+        break;
+      }
+    }
+  }
+  return landed;
+}
+
 // Bulk tensor copies global -> this block's shared memory, completion counted on an mbarrier.
 __device__ __forceinline__ void twa_tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
                                                 uint32_t bar) {

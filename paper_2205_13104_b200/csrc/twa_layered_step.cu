@@ -273,7 +273,12 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
                                            a.status, a.wait_limit_ns);
     return;
   }
-  unsigned char* digw = smem + a.scratch_off + warp * DIGIT_SCRATCH;
+  unsigned char* digw = smem + a.scratch_off + warp * BYTE_DIGIT_SCRATCH;   // this warp's digit matrices
+  constexpr bool FOUR = !GBF16;                        // float32 gradients carry a fourth byte digit
+  byte_digit_init<FOUR>(digw, lane);
+  __syncwarp();
+  const uint32_t dig_addr = byte_digit_ldmatrix_addr(digw, lane);
+  const int dmult = byte_digit_mult(tig);
   const int lm = lane >> 3, lr = lane & 7;
   const int jmax = a.n - 1;
   constexpr int col_bytes = TWA_TILE_COL_BYTES * KT;
@@ -365,42 +370,33 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
         gsum += g0[u] + g1[u];
       }
       mb = __reduce_max_sync(0xFFFFFFFFu, mb);
-      const unsigned ebits = mb >> 23;
-      if (ebits >= 255u) bad = true;
-      if (ebits >= 5u && ebits < 255u) {
-        const float up = __uint_as_float((259u - ebits) << 23);
-        const float w0 = (ebits >= 6u) ? __uint_as_float((ebits - 5u) << 23) : 5.877471754e-39f;
-        const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
-        float wa = tig == 0 ? w0 : (tig == 1 ? w2 : 0.0f);
-        float wb_ = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);
-        if (BITS == 4) { wa *= 0.0625f; wb_ *= 0.0625f; }
+      const ByteDigitScale ds = byte_digit_scale(mb);
+      if (ds.bad) bad = true;
+      if (ds.live) {
+        // 4-bit codes enter the MMA times 16
+        const float wl = byte_digit_weight(tig, BITS == 4 ? ds.w0 * 0.0625f : ds.w0);
         int c[MT][4];
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) c[mt][0] = c[mt][1] = c[mt][2] = c[mt][3] = 0;
 #pragma unroll
         for (int u = 0; u < KT; ++u) {
-          const uint32_t d0 = cut_digits(g0[u] * up);
-          uint32_t b0, b1, b2 = 0, b3 = 0;
-#pragma unroll
-          for (int q = 0; q < 4; ++q) digw[q * 32 + lane] = static_cast<unsigned char>(d0 >> (8 * q));
-          if (BITS == 4) {
-            const uint32_t d1 = cut_digits(g1[u] * up);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) digw[128 + q * 32 + lane] = static_cast<unsigned char>(d1 >> (8 * q));
-          }
+          byte_digit_store<FOUR>(digw, 0, lane, g0[u], ds.up);
+          if (BITS == 4) byte_digit_store<FOUR>(digw, 1, lane, g1[u], ds.up);
           __syncwarp();
-          b0 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 4 * tig) : 0u;
-          b1 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 16 + 4 * tig) : 0u;
-          if (BITS == 4) {
-            b2 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 4 * tig) : 0u;
-            b3 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 16 + 4 * tig) : 0u;
+          uint32_t b0, b1, b2 = 0, b3 = 0;
+          if (BITS == 8) {
+            ldmatrix_x2(dig_addr, b0, b1);
+          } else {
+            uint32_t bb[4];
+            ldmatrix_x4(dig_addr, bb);
+            b0 = bb[0]; b1 = bb[1]; b2 = bb[2]; b3 = bb[3];   // second matrix pair: the odd rows
           }
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
             uint32_t r[4];
             ldmatrix_x4(tile_base + aoff[u][mt], r);
             if (BITS == 8) {
-              mma_u8s8(c[mt], r, b0, b1);
+              mma_u8u8(c[mt], r, b0, b1);
             } else {
               uint32_t ev[4], od[4];
 #pragma unroll
@@ -408,18 +404,17 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
                 ev[i] = (r[i] << 4) & 0xF0F0F0F0u;       // even rows: 16 * code, unsigned
                 od[i] = r[i] & 0xF0F0F0F0u;              // odd rows
               }
-              mma_u8s8(c[mt], ev, b0, b1);
-              mma_u8s8(c[mt], od, b2, b3);
+              mma_u8u8(c[mt], ev, b0, b1);
+              mma_u8u8(c[mt], od, b2, b3);
             }
           }
           __syncwarp();
         }
+        // digit sums -> float: |sum| < 2^31 (at most 128 rows x 255 x 240 per digit, times 257)
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-          facc[mt][0] = fmaf(small_int_to_float(c[mt][0]), wa, facc[mt][0]);
-          facc[mt][0] = fmaf(small_int_to_float(c[mt][1]), wb_, facc[mt][0]);
-          facc[mt][1] = fmaf(small_int_to_float(c[mt][2]), wa, facc[mt][1]);
-          facc[mt][1] = fmaf(small_int_to_float(c[mt][3]), wb_, facc[mt][1]);
+          facc[mt][0] = fmaf(static_cast<float>(c[mt][0] + dmult * c[mt][1]), wl, facc[mt][0]);
+          facc[mt][1] = fmaf(static_cast<float>(c[mt][2] + dmult * c[mt][3]), wl, facc[mt][1]);
         }
       }
     }
@@ -522,9 +517,14 @@ layered_combine_kernel(const float* __restrict__ partials, const int* __restrict
     if (!isfinite(c)) twa_set_status(status, TWA_ERR_NONFINITE, l);
     if (c_out) c_out[static_cast<size_t>(l) * n + i] = static_cast<float>(c);
     if (beta) {
+      // the coefficients are state that outlives the call: a coefficient whose c is not finite, and
+      // every coefficient after a wait ran out in the projection, stays as it was
       const size_t at = static_cast<size_t>(l) * n + i;
-      bnew = twa_coefficient_update(beta[at], c, lr, lambda, adam, at);
-      beta[at] = bnew;
+      bnew = beta[at];
+      if (isfinite(c) && __ldcg(status) != TWA_ERR_TIMEOUT) {
+        bnew = twa_coefficient_update(bnew, c, lr, lambda, adam, at);
+        beta[at] = bnew;
+      }
     }
   }
   if (dig) {                                                           // only with beta: the step
@@ -830,11 +830,11 @@ int do_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dty
   a.tx_bytes = static_cast<unsigned>(n) * TWA_TILE_COL_BYTES * kt;
   a.aux_off = a.tx_bytes;
   a.stage_bytes = (a.aux_off + aux_bytes(lb->codes.bits, kt) + 1023) / 1024 * 1024;
-  a.stages = stage_count(ctx, TWA_SMEM_HEADER + MMA_WARPS * DIGIT_SCRATCH + ENTRY_RING_BYTES + 1024,
+  a.stages = stage_count(ctx, TWA_SMEM_HEADER + MMA_WARPS * BYTE_DIGIT_SCRATCH + ENTRY_RING_BYTES + 1024,
                          static_cast<int>(a.stage_bytes));
   if (a.stages < 2) return TWA_ERR_UNSUPPORTED;
   a.scratch_off = TWA_SMEM_HEADER + static_cast<unsigned>(a.stages) * a.stage_bytes;
-  a.ering_off = a.scratch_off + MMA_WARPS * DIGIT_SCRATCH;
+  a.ering_off = a.scratch_off + MMA_WARPS * BYTE_DIGIT_SCRATCH;
   a.gran = reinterpret_cast<const int4*>(lb->granules);
   a.g = g;
   a.cta_first = lb->cta_first_layer;

@@ -37,6 +37,14 @@ __device__ __forceinline__ void mma_s8(int (&d)[4], const uint32_t (&a)[4], uint
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// d = a (16 x 32, s8) * b (32 x 8, s8): the first product of a sum, no accumulator to clear
+__device__ __forceinline__ void mma_s8_first(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(0));
+}
+
 // |v| < 2^22 -> float, exactly, without the conversion unit
 __device__ __forceinline__ float small_int_to_float(int v) {
   return __int_as_float(0x4B400000 + v) - RND;
@@ -61,6 +69,104 @@ __device__ __forceinline__ uint32_t cut_digits(float t) {
   const uint32_t lo = __byte_perm(__float_as_uint(m0), __float_as_uint(m1), 0x0040);  // bytes m0.b0, m1.b0
   const uint32_t hi = __byte_perm(__float_as_uint(m2), __float_as_uint(m3), 0x0040);
   return __byte_perm(lo, hi, 0x5410);
+}
+
+// d += a (16 x 32, s8) * b (32 x 8, u8), int32 accumulation
+__device__ __forceinline__ void mma_s8u8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.s8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// d += a (16 x 32, u8) * b (32 x 8, u8), int32 accumulation
+__device__ __forceinline__ void mma_u8u8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void ldmatrix_x2(uint32_t addr, uint32_t& r0, uint32_t& r1) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
+}
+
+// ---- byte digits of the gradient (projection kernels) ---------------------------------------------
+// A block of gradient values with largest magnitude below 2^(e-126) (e = its biased exponent) is
+// turned into integers q = round(g * 2^sexp), |q| <= 2^22, by ONE fused multiply-add with the
+// constant RND = 1.5 * 2^23: the float RND + q has the bit pattern 0x4B400000 + q, so its three low
+// bytes are the base-256 digits of q + 2^22:
+//     q = u0 + 256 u1 + 65536 (u2 - 64),   u0, u1 in [0, 255], u2 in [0, 128].
+// The integer MMAs take the three bytes as unsigned operands next to a column of ones, whose dot
+// product (the sum of the codes) removes the offset 64 of the top byte.  For float32 gradients a
+// fourth byte carries the remainder: r = round((g * 2^sexp - q) * 254) in [-127, 127], stored as
+// r + 128, again next to a column of ones.  Error of the cut: 2^-23 (three bytes) or 2^-31 (four)
+// of the power of two above the block's largest magnitude.
+constexpr int BYTE_DIGIT_ROWS = 8;              // rows of a digit matrix: u0, u1, u2, ones, r + 128, ones, 0, 0
+constexpr int BYTE_DIGIT_SET = BYTE_DIGIT_ROWS * 32;      // bytes: one row of 32 gradient rows per digit
+constexpr int BYTE_DIGIT_SCRATCH = 2 * BYTE_DIGIT_SET;    // per warp: even and odd rows (4-bit codes)
+
+struct ByteDigitScale {
+  float up;        // 2^sexp
+  float w0;        // 2^-sexp, the weight of u0
+  bool live;       // false: every value of the block is below 2^-122 and contributes nothing
+  bool bad;        // NaN or Inf among the values
+};
+
+// mb = largest |g| of the block as a bit pattern
+__device__ __forceinline__ ByteDigitScale byte_digit_scale(unsigned mb) {
+  const int ebits = static_cast<int>(mb >> 23);
+  ByteDigitScale s;
+  s.bad = ebits >= 255;
+  s.live = ebits >= 5 && ebits < 255;
+  int sexp = 148 - ebits;                                  // |g| 2^sexp < 2^22
+  sexp = sexp > 126 ? 126 : sexp;
+  s.up = __uint_as_float(static_cast<unsigned>(127 + sexp) << 23);
+  s.w0 = __uint_as_float(static_cast<unsigned>(127 - sexp) << 23);
+  return s;
+}
+
+// Fills the constant rows of a warp's digit matrices (ones in row 3, and in row 5 with four-byte
+// digits; zeros elsewhere); rows 0-2 (and 4) are rewritten for every block of rows.
+template <bool FOUR>
+__device__ __forceinline__ void byte_digit_init(unsigned char* digw, int lane) {
+  uint32_t* w = reinterpret_cast<uint32_t*>(digw);
+#pragma unroll
+  for (int i = 0; i < BYTE_DIGIT_SCRATCH / 128; ++i) {
+    const int idx = lane + 32 * i;                         // word of the scratch
+    const int row = (idx % (BYTE_DIGIT_SET / 4)) / 8;
+    w[idx] = (row == 3 || (FOUR && row == 5)) ? 0x01010101u : 0u;
+  }
+}
+
+// Writes the digits of the lane's value of gradient row `lane` into digit matrix `set`.
+template <bool FOUR>
+__device__ __forceinline__ void byte_digit_store(unsigned char* digw, int set, int lane, float g, float up) {
+  const float y = fmaf(g, up, RND);
+  const uint32_t b = __float_as_uint(y);
+  unsigned char* d = digw + set * BYTE_DIGIT_SET + lane;
+  d[0] = static_cast<unsigned char>(b);
+  d[32] = static_cast<unsigned char>(b >> 8);
+  d[64] = static_cast<unsigned char>(b >> 16);
+  if (FOUR) {
+    const float rem = fmaf(g, up, -(y - RND));             // exact: g * up - q
+    d[128] = static_cast<unsigned char>(__float_as_uint(fmaf(rem, 254.0f, RND + 128.0f)));
+  }
+}
+
+// Address a lane hands to ldmatrix for the warp's digit matrices: matrix m = lane / 8 is the (m & 1)-th
+// half (gradient rows 16 (m & 1) ...) of set m / 2, row lane % 8 is digit lane % 8.
+__device__ __forceinline__ uint32_t byte_digit_ldmatrix_addr(const unsigned char* digw, int lane) {
+  const int m = lane >> 3;
+  return twa_smem_u32(digw + (m >> 1) * BYTE_DIGIT_SET + (lane & 7) * 32 + (m & 1) * 16);
+}
+
+// Lane constants of the recombination: the accumulator columns of lane tig hold digits 2 tig, 2 tig + 1.
+//   tig 0: u0 + 256 u1, weight w0;  tig 1: u2 - 64 ones, weight 65536 w0;
+//   tig 2: (r + 128) - 128 ones, weight w0 / 254;  tig 3: nothing.
+__device__ __forceinline__ int byte_digit_mult(int tig) { return tig == 0 ? 256 : (tig == 1 ? -64 : (tig == 2 ? -128 : 0)); }
+__device__ __forceinline__ float byte_digit_weight(int tig, float w0) {
+  return tig == 0 ? w0 : (tig == 1 ? w0 * 65536.0f : (tig == 2 ? w0 * (1.0f / 254.0f) : 0.0f));
 }
 
 // Producer loop: tile k of this block's sequence is t_first + k * t_step (k < t_count); with
@@ -99,18 +205,9 @@ __device__ __forceinline__ void producer_loop_mma(twa_smem_header* hdr, unsigned
       if (issued > stages) phase ^= 1u;
     }
   }
-  if (!ok) {
-    twa_set_status(status, TWA_ERR_TIMEOUT, -1);
-    const int live = issued < stages ? issued : stages;
-    for (int q = 0; q < live; ++q) {      // let the copies already issued land
-      const int last = ((issued - 1 - q) / stages) * stages + q;
-      const unsigned par = static_cast<unsigned>(last / stages) & 1u;
-      const unsigned long long t0 = twa_globaltimer();
-      while (!twa_mbar_try_wait(twa_smem_u32(&hdr->full[q]), par)) {
-        if (twa_globaltimer() - t0 > limit) break;
-      }
-    }
-  }
+  // every copy issued has landed before this lane leaves, whatever the consumers did meanwhile
+  if (!twa_drain_ring(hdr, issued, stages, limit)) ok = false;
+  if (!ok) twa_set_status(status, TWA_ERR_TIMEOUT, -1);
 }
 
 __device__ __forceinline__ void init_barriers(twa_smem_header* hdr, int stages) {

@@ -36,7 +36,13 @@ struct DeviceSetup {
 constexpr int MAX_DEVICES = 64;
 DeviceSetup g_setup[MAX_DEVICES];
 std::mutex g_setup_lock;
-char g_noalloc_error[256] = "";
+// Text of the calling thread's last rejected call ("" after a call that was accepted).
+thread_local char g_noalloc_error[256] = "";
+
+int reject(int code, const char* why) {
+  snprintf(g_noalloc_error, sizeof(g_noalloc_error), "%s", why);
+  return code;
+}
 
 int fail(int code, const char* what, cudaError_t e) {
   snprintf(g_noalloc_error, sizeof(g_noalloc_error), "%s: %s", what, cudaGetErrorString(e));
@@ -81,17 +87,18 @@ extern "C" {
 
 int twa_project_noalloc(int device, void* cuda_stream, const twa_basis* P, const void* g,
                         twa_dtype g_dtype, float* c_out, int* status_out) {
-  if (!P || !g || !c_out) return TWA_ERR_INVALID_ARG;
-  if (device < 0 || device >= MAX_DEVICES) return TWA_ERR_INVALID_ARG;
-  if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
+  g_noalloc_error[0] = 0;
+  if (!P || !g || !c_out) return reject(TWA_ERR_INVALID_ARG, "P, g and c_out must not be null");
+  if (device < 0 || device >= MAX_DEVICES) return reject(TWA_ERR_INVALID_ARG, "device index out of range");
+  if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return reject(TWA_ERR_INVALID_ARG, "g_dtype is neither TWA_F32 nor TWA_BF16");
   if (P->n > TWA_MAX_N) {
     snprintf(g_noalloc_error, sizeof(g_noalloc_error),
              "n = %d exceeds the %d columns the static scratch holds", P->n, TWA_MAX_N);
     return TWA_ERR_UNSUPPORTED;
   }
   int rc = twa_check_basis(P);
-  if (rc) return rc;
-  if (reinterpret_cast<uintptr_t>(g) & 15) return TWA_ERR_MISALIGNED;
+  if (rc) return reject(rc, "the basis descriptor is not valid (sizes, width, alignment)");
+  if (reinterpret_cast<uintptr_t>(g) & 15) return reject(TWA_ERR_MISALIGNED, "g is not 16-byte aligned");
   cudaError_t e = cudaSetDevice(device);
   if (e != cudaSuccess) return fail(TWA_ERR_CUDA, "cudaSetDevice", e);
   DeviceSetup* s = nullptr;

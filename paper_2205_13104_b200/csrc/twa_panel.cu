@@ -59,18 +59,9 @@ __device__ __forceinline__ void panel_producer(twa_smem_header* hdr, unsigned ch
     twa_mbar_expect_tx(fb, a.tx_bytes);
     twa_tma_load_2d(twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes), map, tile * PROWS, 0, fb);
   }
-  if (!ok) {
-    twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
-    const int live = issued < a.stages ? issued : a.stages;
-    for (int q = 0; q < live; ++q) {      // let the copies already issued land
-      const int last = ((issued - 1 - q) / a.stages) * a.stages + q;
-      const unsigned par = static_cast<unsigned>(last / a.stages) & 1u;
-      const unsigned long long t0 = twa_globaltimer();
-      while (!twa_mbar_try_wait(twa_smem_u32(&hdr->full[q]), par)) {
-        if (twa_globaltimer() - t0 > a.wait_limit_ns) break;
-      }
-    }
-  }
+  // every copy issued has landed before this lane leaves, whatever the consumers did meanwhile
+  if (!twa_drain_ring(hdr, issued, a.stages, a.wait_limit_ns)) ok = false;
+  if (!ok) twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
 }
 
 // CPW = columns of Q a warp owns at most, ceil(nq / 15): a compile-time constant, so that the loops
@@ -239,18 +230,9 @@ panel_lift_kernel(const __grid_constant__ CUtensorMap map, const PanelLiftArgs a
           twa_tma_load_2d(dst + b * LBOX_BYTES, &map, rb * LROWS_BLOCK + b * 256, c * LCHUNK, fb);
       }
     }
-    if (!ok) {
-      twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
-      const int live = it < a.stages ? it : a.stages;
-      for (int q = 0; q < live; ++q) {      // let the copies already issued land
-        const int last = ((it - 1 - q) / a.stages) * a.stages + q;
-        const unsigned par = static_cast<unsigned>(last / a.stages) & 1u;
-        const unsigned long long t0 = twa_globaltimer();
-        while (!twa_mbar_try_wait(twa_smem_u32(&hdr->full[q]), par)) {
-          if (twa_globaltimer() - t0 > a.wait_limit_ns) break;
-        }
-      }
-    }
+    // every copy issued has landed before this lane leaves, whatever the consumers did meanwhile
+    if (!twa_drain_ring(hdr, it, a.stages, a.wait_limit_ns)) ok = false;
+    if (!ok) twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
     return;
   }
   // element (column c of the chunk, row r of the block) sits at ((r >> 8) * 8 + c) * 256 + (r & 255)

@@ -2,9 +2,11 @@
 // (Section 4.2, the chain-rule equation, for every row of G), P~ read once per group of gradients.
 //
 // Same data path as the single-gradient kernel in twa_stream_mma.cu.  What the batch adds: the
-// m16n8k32 integer MMA has eight result columns and one gradient's four base-128 digits fill only
-// four of them, so two gradients share every MMA (columns 0-3: digits of the first, 4-7: digits of
-// the second).  A tile of P~ in shared memory serves NP such pairs before its stage is released;
+// m16n8k32 integer MMA has eight result columns and one gradient's three byte digits and the
+// column of ones that goes with them fill only four, so two gradients share every MMA (columns
+// 0-3: the first, 4-7: the second; float32 gradients are cut to three bytes here too: 2^-23 of the
+// largest magnitude of a warp's rows).  A tile of P~ in shared memory serves NP such pairs before
+// its stage is released;
 // the gradients of a group arrive as [NB][256] boxes of one 2-D tensor map over G (rows past the
 // batch read as zero).
 #include <stdio.h>
@@ -13,7 +15,27 @@
 
 namespace {
 
-constexpr int PAIR_SCRATCH = 512;               // digit bytes per warp: two gradients x (even, odd rows) x [4][32]
+constexpr int PAIR_SCRATCH = BYTE_DIGIT_SCRATCH;  // per warp: (even, odd rows) x [8 digit rows][32 gradient rows]
+
+// Digit matrix of a pair of gradients: rows u0, u1, u2, ones of the first, then of the second.
+__device__ __forceinline__ void pair_digit_init(unsigned char* digw, int lane) {
+  uint32_t* w = reinterpret_cast<uint32_t*>(digw);
+#pragma unroll
+  for (int i = 0; i < PAIR_SCRATCH / 128; ++i) {
+    const int idx = lane + 32 * i;
+    const int row = (idx % (BYTE_DIGIT_SET / 4)) / 8;
+    w[idx] = (row & 3) == 3 ? 0x01010101u : 0u;
+  }
+}
+
+// The three byte digits of gradient h's value for gradient row `lane` into digit matrix `set`.
+__device__ __forceinline__ void pair_digit_store(unsigned char* digw, int set, int h, int lane, float g, float up) {
+  const uint32_t b = __float_as_uint(fmaf(g, up, RND));
+  unsigned char* d = digw + set * BYTE_DIGIT_SET + h * 128 + lane;
+  d[0] = static_cast<unsigned char>(b);
+  d[32] = static_cast<unsigned char>(b >> 8);
+  d[64] = static_cast<unsigned char>(b >> 16);
+}
 
 struct BatchArgs {
   long long D;
@@ -56,18 +78,9 @@ __device__ __forceinline__ void producer_loop_batch(twa_smem_header* hdr, unsign
       if (issued > a.stages) phase ^= 1u;
     }
   }
-  if (!ok) {
-    twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
-    const int live = issued < a.stages ? issued : a.stages;
-    for (int q = 0; q < live; ++q) {      // let the copies already issued land
-      const int last = ((issued - 1 - q) / a.stages) * a.stages + q;
-      const unsigned par = static_cast<unsigned>(last / a.stages) & 1u;
-      const unsigned long long t0 = twa_globaltimer();
-      while (!twa_mbar_try_wait(twa_smem_u32(&hdr->full[q]), par)) {
-        if (twa_globaltimer() - t0 > a.wait_limit_ns) break;
-      }
-    }
-  }
+  // every copy issued has landed before this lane leaves, whatever the consumers did meanwhile
+  if (!twa_drain_ring(hdr, issued, a.stages, a.wait_limit_ns)) ok = false;
+  if (!ok) twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
 }
 
 // NP pairs of gradients per launch (NB = 2 NP); MT, KT as in the single-gradient kernel.
@@ -98,6 +111,10 @@ twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
     if (lane == 0) producer_loop_batch<KT, NB>(hdr, ring, &map_p, &map_g, a, SROWS * KT, GSZ);
   } else {
     unsigned char* digw = smem + a.scratch_off + warp * PAIR_SCRATCH;
+    pair_digit_init(digw, lane);
+    __syncwarp();
+    const uint32_t dig_addr = byte_digit_ldmatrix_addr(digw, lane);
+    const int dmult = (tig & 1) ? -64 : 256;
     const int lm = lane >> 3, lr = lane & 7;
     const int jmax = a.n - 1;
     constexpr int col_bytes = TWA_TILE_COL_BYTES * KT;
@@ -154,21 +171,17 @@ twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
           }
         mb[0] = __reduce_max_sync(0xFFFFFFFFu, mb[0]);
         mb[1] = __reduce_max_sync(0xFFFFFFFFu, mb[1]);
-        const unsigned eb0 = mb[0] >> 23, eb1 = mb[1] >> 23;
-        if (eb0 >= 255u) bad |= 1u << (2 * p);
-        if (eb1 >= 255u) bad |= 1u << (2 * p + 1);
-        const bool live0 = eb0 >= 5u && eb0 < 255u, live1 = eb1 >= 5u && eb1 < 255u;
-        if (!live0 && !live1) continue;                  // nothing representable in either gradient here
-        const float up0 = live0 ? __uint_as_float((259u - eb0) << 23) : 0.0f;
-        const float up1 = live1 ? __uint_as_float((259u - eb1) << 23) : 0.0f;
-        // lanes tig 0,1 finish the first gradient's digits, tig 2,3 the second's
-        const unsigned ebm = (tig < 2) ? eb0 : eb1;
-        const bool livem = (tig < 2) ? live0 : live1;
-        const float w0 = !livem ? 0.0f : (ebm >= 6u ? __uint_as_float((ebm - 5u) << 23) : 5.877471754e-39f);
-        const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
-        float wa = (tig & 1) == 0 ? w0 : w2;
-        float wb = (tig & 1) == 0 ? w1 : w3;
-        if (BITS == 4) { wa *= 0.0625f; wb *= 0.0625f; }
+        const ByteDigitScale ds0 = byte_digit_scale(mb[0]), ds1 = byte_digit_scale(mb[1]);
+        if (ds0.bad) bad |= 1u << (2 * p);
+        if (ds1.bad) bad |= 1u << (2 * p + 1);
+        if (!ds0.live && !ds1.live) continue;            // nothing representable in either gradient here
+        // a dead or non-finite gradient is cut with scale 0: its digits are those of zero
+        const float up0 = ds0.live ? ds0.up : 0.0f, up1 = ds1.live ? ds1.up : 0.0f;
+        // lanes tig 0,1 finish the first gradient's digits (columns u0 u1 | u2 ones), tig 2,3 the second's
+        const bool livem = (tig < 2) ? ds0.live : ds1.live;
+        float wl = !livem ? 0.0f : ((tig < 2) ? ds0.w0 : ds1.w0);
+        if (tig & 1) wl *= 65536.0f;
+        if (BITS == 4) wl *= 0.0625f;                    // 4-bit codes enter the MMA times 16
         int c[MT][4];
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) c[mt][0] = c[mt][1] = c[mt][2] = c[mt][3] = 0;
@@ -176,32 +189,25 @@ twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
         for (int u = 0; u < KT; ++u) {
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
-            const bool lv = h ? live1 : live0;            // a dead or non-finite gradient contributes zero digits
-            const uint32_t d0 = cut_digits(lv ? g0[h][u] * (h ? up1 : up0) : 0.0f);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) digw[h * 256 + k * 32 + lane] = static_cast<unsigned char>(d0 >> (8 * k));
-            if (BITS == 4) {
-              const uint32_t d1 = cut_digits(lv ? g1[h][u] * (h ? up1 : up0) : 0.0f);
-#pragma unroll
-              for (int k = 0; k < 4; ++k) digw[h * 256 + 128 + k * 32 + lane] = static_cast<unsigned char>(d1 >> (8 * k));
-            }
+            pair_digit_store(digw, 0, h, lane, g0[h][u], h ? up1 : up0);
+            if (BITS == 4) pair_digit_store(digw, 1, h, lane, g1[h][u], h ? up1 : up0);
           }
           __syncwarp();
-          // B fragment: result column gid = digit gid of the first gradient (gid < 4) or digit gid - 4 of the second
-          const unsigned char* dg = digw + (gid >> 2) * 256 + (gid & 3) * 32 + 4 * tig;
-          const uint32_t b0 = *reinterpret_cast<const uint32_t*>(dg);
-          const uint32_t b1 = *reinterpret_cast<const uint32_t*>(dg + 16);
-          uint32_t b2 = 0, b3 = 0;
-          if (BITS == 4) {
-            b2 = *reinterpret_cast<const uint32_t*>(dg + 128);
-            b3 = *reinterpret_cast<const uint32_t*>(dg + 128 + 16);
+          // B fragment: result columns 0-3 = u0, u1, u2, ones of the first gradient, 4-7 of the second
+          uint32_t b0, b1, b2 = 0, b3 = 0;
+          if (BITS == 8) {
+            ldmatrix_x2(dig_addr, b0, b1);
+          } else {
+            uint32_t bb[4];
+            ldmatrix_x4(dig_addr, bb);
+            b0 = bb[0]; b1 = bb[1]; b2 = bb[2]; b3 = bb[3];   // second matrix pair: the odd rows
           }
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
             uint32_t r[4];
             ldmatrix_x4(tile_base + aoff[u][mt], r);
             if (BITS == 8) {
-              mma_s8(c[mt], r, b0, b1);
+              mma_s8u8(c[mt], r, b0, b1);
             } else {
               uint32_t e[4], o[4];
 #pragma unroll
@@ -209,18 +215,16 @@ twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
                 e[i] = (r[i] << 4) & 0xF0F0F0F0u;         // even rows: 16 * code
                 o[i] = r[i] & 0xF0F0F0F0u;                // odd rows:  16 * code
               }
-              mma_s8(c[mt], e, b0, b1);
-              mma_s8(c[mt], o, b2, b3);
+              mma_s8u8(c[mt], e, b0, b1);
+              mma_s8u8(c[mt], o, b2, b3);
             }
           }
-          __syncwarp();                                  // the digit scratch is rewritten next
+          __syncwarp();                                  // the digit matrices are rewritten next
         }
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-          facc[p][mt][0] = fmaf(small_int_to_float(c[mt][0]), wa, facc[p][mt][0]);
-          facc[p][mt][0] = fmaf(small_int_to_float(c[mt][1]), wb, facc[p][mt][0]);
-          facc[p][mt][1] = fmaf(small_int_to_float(c[mt][2]), wa, facc[p][mt][1]);
-          facc[p][mt][1] = fmaf(small_int_to_float(c[mt][3]), wb, facc[p][mt][1]);
+          facc[p][mt][0] = fmaf(static_cast<float>(c[mt][0] + dmult * c[mt][1]), wl, facc[p][mt][0]);
+          facc[p][mt][1] = fmaf(static_cast<float>(c[mt][2] + dmult * c[mt][3]), wl, facc[p][mt][1]);
         }
       }
       __syncwarp();

@@ -81,19 +81,9 @@ __device__ __forceinline__ void producer_loop(SmemHeader* hdr, unsigned char* ri
       if (issued > stages) phase ^= 1u;
     }
   }
-  if (!ok) {
-    // Let every copy already issued land before the block may exit.
-    twa_set_status(status, TWA_ERR_TIMEOUT, -1);
-    const int live = issued < stages ? issued : stages;
-    for (int q = 0; q < live; ++q) {
-      const int last = ((issued - 1 - q) / stages) * stages + q;   // last issue into stage q
-      const unsigned par = static_cast<unsigned>(last / stages) & 1u;
-      const unsigned long long t0 = twa_globaltimer();
-      while (!twa_mbar_try_wait(twa_smem_u32(&hdr->full[q]), par)) {
-        if (twa_globaltimer() - t0 > limit) break;
-      }
-    }
-  }
+  // every copy issued has landed before this lane leaves, whatever the consumers did meanwhile
+  if (!twa_drain_ring(hdr, issued, stages, limit)) ok = false;
+  if (!ok) twa_set_status(status, TWA_ERR_TIMEOUT, -1);
 }
 
 // ---- project ------------------------------------------------------------------------------
@@ -251,16 +241,22 @@ twa_project_kernel(const __grid_constant__ CUtensorMap map_p,
   __syncthreads();
   if (hdr->last_flag) {
     __threadfence();
+    double c = 0.0;
     if (tid < a.n) {
       double sum = 0.0;
       for (unsigned b = 0; b < gridDim.x; ++b)
         sum += static_cast<double>(__ldcg(&a.partials[static_cast<size_t>(b) * a.n + tid]));
-      const double c = (BITS == 32) ? sum : sum * static_cast<double>(a.scales[tid]);
+      c = (BITS == 32) ? sum : sum * static_cast<double>(a.scales[tid]);
       if (!isfinite(c))
         twa_set_status(a.status, TWA_ERR_NONFINITE, a.nonfinite_detail >= 0 ? a.nonfinite_detail : tid);
       if (a.c_out) a.c_out[tid] = static_cast<float>(c);
-      if (a.alpha) a.alpha[tid] = twa_coefficient_update(a.alpha[tid], c, a.lr, a.lambda, a.adam, tid);
     }
+    // The coefficients are state that outlives the call: they are left as they were when any c is not
+    // finite or a wait ran out in some block (whose partial sums are then incomplete), so that the
+    // caller can clear the status and repeat the step.
+    const int unusable = __syncthreads_or(!isfinite(c)) | (__ldcg(a.status) == TWA_ERR_TIMEOUT);
+    if (tid < a.n && a.alpha && !unusable)
+      a.alpha[tid] = twa_coefficient_update(a.alpha[tid], c, a.lr, a.lambda, a.adam, tid);
     if (tid == 0) *a.ticket = 0u;
   }
 }

@@ -100,7 +100,12 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
                         a.stages, a.stage_bytes, KT, SROWS * KT / 256, GSZ, SROWS * KT, a.g_off,
                         a.tx_bytes, false, a.status, a.wait_limit_ns);
   } else {
-    unsigned char* digw = smem + a.scratch_off + warp * DIGIT_SCRATCH;   // this warp's digit bytes
+    unsigned char* digw = smem + a.scratch_off + warp * BYTE_DIGIT_SCRATCH;   // this warp's digit matrices
+    constexpr bool FOUR = !GBF16;                       // float32 gradients carry a fourth byte digit
+    byte_digit_init<FOUR>(digw, lane);
+    __syncwarp();
+    const uint32_t dig_addr = byte_digit_ldmatrix_addr(digw, lane);
+    const int dmult = byte_digit_mult(tig);
     const int lm = lane >> 3, lr = lane & 7;            // ldmatrix: matrix and row this lane addresses
     const int jmax = a.n - 1;                           // last column that exists in shared memory
     constexpr int col_bytes = TWA_TILE_COL_BYTES * KT;
@@ -134,89 +139,72 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
       unsigned mb = 0u;
 #pragma unroll
       for (int u = 0; u < KT; ++u) {
-        {
-          g1[u] = 0.0f;
-          const int vw = warp * KT + u;                 // index of the 32-byte block in the column
-          if (BITS == 8) {
-            if (GBF16) g0[u] = __uint_as_float(static_cast<uint32_t>(
-                           reinterpret_cast<const unsigned short*>(st + a.g_off)[vw * WROWS + lane]) << 16);
-            else g0[u] = reinterpret_cast<const float*>(st + a.g_off)[vw * WROWS + lane];
+        g1[u] = 0.0f;
+        const int vw = warp * KT + u;                   // index of the 32-byte block in the column
+        if (BITS == 8) {
+          if (GBF16) g0[u] = __uint_as_float(static_cast<uint32_t>(
+                         reinterpret_cast<const unsigned short*>(st + a.g_off)[vw * WROWS + lane]) << 16);
+          else g0[u] = reinterpret_cast<const float*>(st + a.g_off)[vw * WROWS + lane];
+        } else {
+          if (GBF16) {
+            const uint32_t pr = reinterpret_cast<const uint32_t*>(st + a.g_off)[vw * 32 + lane];
+            g0[u] = twa_bf16_lo(pr);
+            g1[u] = twa_bf16_hi(pr);
           } else {
-            if (GBF16) {
-              const uint32_t pr = reinterpret_cast<const uint32_t*>(st + a.g_off)[vw * 32 + lane];
-              g0[u] = twa_bf16_lo(pr);
-              g1[u] = twa_bf16_hi(pr);
-            } else {
-              const float2 pr = reinterpret_cast<const float2*>(st + a.g_off)[vw * 32 + lane];
-              g0[u] = pr.x;
-              g1[u] = pr.y;
-            }
-            mb = max(mb, __float_as_uint(g1[u]) & 0x7FFFFFFFu);
+            const float2 pr = reinterpret_cast<const float2*>(st + a.g_off)[vw * 32 + lane];
+            g0[u] = pr.x;
+            g1[u] = pr.y;
           }
-          mb = max(mb, __float_as_uint(g0[u]) & 0x7FFFFFFFu);
+          mb = max(mb, __float_as_uint(g1[u]) & 0x7FFFFFFFu);
         }
+        mb = max(mb, __float_as_uint(g0[u]) & 0x7FFFFFFFu);
       }
       mb = __reduce_max_sync(0xFFFFFFFFu, mb);          // one digit scale for the warp's rows of the tile
-      const unsigned ebits = mb >> 23;
-      if (ebits >= 255u) bad = true;                    // NaN or Inf in g
-      // Rows whose largest |g| is below 2^-122 contribute nothing representable: skipped.
-      if (ebits >= 5u && ebits < 255u) {
-        // |g| < 2^(ebits-126) here; t = g * 2^(132-ebits) lies in (-64, 64)
-        const float up = __uint_as_float((259u - ebits) << 23);
-        // weight of digit k: 2^(ebits-132) / 128^k
-        const float w0 = (ebits >= 6u) ? __uint_as_float((ebits - 5u) << 23) : 5.877471754e-39f;
-        const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
-        float wa = tig == 0 ? w0 : (tig == 1 ? w2 : 0.0f);        // digits 2*tig, 2*tig+1 sit in this lane's
-        float wb = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);        // accumulator columns
-        if (BITS == 4) { wa *= 0.0625f; wb *= 0.0625f; }          // 4-bit codes enter the MMA times 16
+      const ByteDigitScale ds = byte_digit_scale(mb);
+      if (ds.bad) bad = true;                           // NaN or Inf in g
+      if (ds.live) {
+        // 4-bit codes enter the MMA times 16
+        const float wl = byte_digit_weight(tig, BITS == 4 ? ds.w0 * 0.0625f : ds.w0);
         int c[MT][4];
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) c[mt][0] = c[mt][1] = c[mt][2] = c[mt][3] = 0;
 #pragma unroll
         for (int u = 0; u < KT; ++u) {
-          {
-            const uint32_t d0 = cut_digits(g0[u] * up);
-            uint32_t b0, b1, b2 = 0, b3 = 0;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) digw[k * 32 + lane] = static_cast<unsigned char>(d0 >> (8 * k));
-            if (BITS == 4) {
-              const uint32_t d1 = cut_digits(g1[u] * up);
-#pragma unroll
-              for (int k = 0; k < 4; ++k) digw[128 + k * 32 + lane] = static_cast<unsigned char>(d1 >> (8 * k));
-            }
-            __syncwarp();
-            b0 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 4 * tig) : 0u;
-            b1 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + gid * 32 + 16 + 4 * tig) : 0u;
-            if (BITS == 4) {                              // second scratch half: the odd rows
-              b2 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 4 * tig) : 0u;
-              b3 = gid < 4 ? *reinterpret_cast<const uint32_t*>(digw + 128 + gid * 32 + 16 + 4 * tig) : 0u;
-            }
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-              uint32_t r[4];
-              ldmatrix_x4(tile_base + aoff[u][mt], r);
-              if (BITS == 8) {
-                mma_s8(c[mt], r, b0, b1);
-              } else {
-                uint32_t e[4], o[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  e[i] = (r[i] << 4) & 0xF0F0F0F0u;       // even rows: 16 * code
-                  o[i] = r[i] & 0xF0F0F0F0u;              // odd rows:  16 * code
-                }
-                mma_s8(c[mt], e, b0, b1);
-                mma_s8(c[mt], o, b2, b3);
-              }
-            }
-            __syncwarp();                                // the digit scratch is rewritten by the next block
+          byte_digit_store<FOUR>(digw, 0, lane, g0[u], ds.up);
+          if (BITS == 4) byte_digit_store<FOUR>(digw, 1, lane, g1[u], ds.up);
+          __syncwarp();
+          uint32_t b0, b1, b2 = 0, b3 = 0;
+          if (BITS == 8) {
+            ldmatrix_x2(dig_addr, b0, b1);
+          } else {
+            uint32_t bb[4];
+            ldmatrix_x4(dig_addr, bb);
+            b0 = bb[0]; b1 = bb[1]; b2 = bb[2]; b3 = bb[3];   // second matrix pair: the odd rows
           }
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            uint32_t r[4];
+            ldmatrix_x4(tile_base + aoff[u][mt], r);
+            if (BITS == 8) {
+              mma_s8u8(c[mt], r, b0, b1);
+            } else {
+              uint32_t e[4], o[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                e[i] = (r[i] << 4) & 0xF0F0F0F0u;       // even rows: 16 * code
+                o[i] = r[i] & 0xF0F0F0F0u;              // odd rows:  16 * code
+              }
+              mma_s8u8(c[mt], e, b0, b1);
+              mma_s8u8(c[mt], o, b2, b3);
+            }
+          }
+          __syncwarp();                                  // the digit matrices are rewritten by the next block
         }
+        // digit sums -> float: |sum| < 2^31 always (at most 128 rows x 255 x 127 per digit, times 257)
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-          facc[mt][0] = fmaf(small_int_to_float(c[mt][0]), wa, facc[mt][0]);
-          facc[mt][0] = fmaf(small_int_to_float(c[mt][1]), wb, facc[mt][0]);
-          facc[mt][1] = fmaf(small_int_to_float(c[mt][2]), wa, facc[mt][1]);
-          facc[mt][1] = fmaf(small_int_to_float(c[mt][3]), wb, facc[mt][1]);
+          facc[mt][0] = fmaf(static_cast<float>(c[mt][0] + dmult * c[mt][1]), wl, facc[mt][0]);
+          facc[mt][1] = fmaf(static_cast<float>(c[mt][2] + dmult * c[mt][3]), wl, facc[mt][1]);
         }
       }
       __syncwarp();
@@ -264,16 +252,22 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
   __syncthreads();
   if (hdr->last_flag) {
     __threadfence();
+    double c = 0.0;
     if (tid < a.n) {
       double sum = 0.0;
       for (unsigned b = 0; b < gridDim.x; ++b)
         sum += static_cast<double>(__ldcg(&a.partials[static_cast<size_t>(b) * a.n + tid]));
-      const double c = sum * static_cast<double>(a.scales[tid]);
+      c = sum * static_cast<double>(a.scales[tid]);
       if (!isfinite(c))
         twa_set_status(a.status, TWA_ERR_NONFINITE, a.nonfinite_detail >= 0 ? a.nonfinite_detail : tid);
       if (a.c_out) a.c_out[tid] = static_cast<float>(c);
-      if (a.alpha) a.alpha[tid] = twa_coefficient_update(a.alpha[tid], c, a.lr, a.lambda, a.adam, tid);
     }
+    // The coefficients are state that outlives the call: they are left as they were when any c is not
+    // finite or a wait ran out in some block (whose partial sums are then incomplete), so that the
+    // caller can clear the status and repeat the step.
+    const int unusable = __syncthreads_or(!isfinite(c)) | (__ldcg(a.status) == TWA_ERR_TIMEOUT);
+    if (tid < a.n && a.alpha && !unusable)
+      a.alpha[tid] = twa_coefficient_update(a.alpha[tid], c, a.lr, a.lambda, a.adam, tid);
     if (tid == 0) *a.ticket = 0u;
   }
 }
@@ -342,7 +336,7 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
   const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
   float wb = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);    // weight of the lower digit of this lane's pair
   if (BITS == 4) wb *= 0.0625f;                         // 4-bit codes enter the MMA times 16
-  const float poison = bad ? __int_as_float(0x7FC00000) : 0.0f;
+  if (bad) wb = __int_as_float(0x7FC00000);             // NaN or Inf among the coefficients poisons every row
 
   // B fragments: k-slot 4*tig+i of a 32-column step holds column j0 + {2tig, 2tig+1, 8+2tig, 9+2tig}[i]
   // (and the same + 16 for the second register), the order the transposing loads deliver.
@@ -438,58 +432,56 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
     float keep[KT][LROWS];
 #pragma unroll
     for (int u = 0; u < KT; ++u) {
+      float v[2][LROWS];                                // per 16-byte chunk of the block
 #pragma unroll
-      for (int i = 0; i < LROWS; ++i) keep[u][i] = 0.0f;
-      {
+      for (int ch = 0; ch < 2; ++ch) {
+        int acc0[4];                                    // 8-bit: rows 2gid, 2gid+1; 4-bit: rows 4gid, 4gid+2
+        int acc1[4];                                    // 4-bit only: rows 4gid+1, 4gid+3
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          int acc0[4] = {0, 0, 0, 0};                   // 8-bit: rows 2gid, 2gid+1; 4-bit: rows 4gid, 4gid+2
-          int acc1[4] = {0, 0, 0, 0};                   // 4-bit only: rows 4gid+1, 4gid+3
+        for (int ks = 0; ks < KS; ++ks) {
+          uint32_t r[4];
+          ldmatrix_x4_trans(tile_base + loff[u][ch][ks], r);
+          // the transposing load delivers byte pairs of two columns: regroup to four columns per register
+          const uint32_t af[4] = {__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[0], r[1], 0x7531),
+                                  __byte_perm(r[2], r[3], 0x6420), __byte_perm(r[2], r[3], 0x7531)};
+          if (BITS == 8) {
+            if (ks == 0) mma_s8_first(acc0, af, bfrag[ks][0], bfrag[ks][1]);
+            else mma_s8(acc0, af, bfrag[ks][0], bfrag[ks][1]);
+          } else {
+            uint32_t ae[4], ao[4];
 #pragma unroll
-          for (int ks = 0; ks < KS; ++ks) {
-            {
-              uint32_t r[4];
-              ldmatrix_x4_trans(tile_base + loff[u][ch][ks], r);
-              if (BITS == 8) {
-                const uint32_t af[4] = {__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[0], r[1], 0x7531),
-                                        __byte_perm(r[2], r[3], 0x6420), __byte_perm(r[2], r[3], 0x7531)};
-                mma_s8(acc0, af, bfrag[ks][0], bfrag[ks][1]);
-              } else {
-                uint32_t e[4], o[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  e[i] = (r[i] << 4) & 0xF0F0F0F0u;
-                  o[i] = r[i] & 0xF0F0F0F0u;
-                }
-                const uint32_t ae[4] = {__byte_perm(e[0], e[1], 0x6420), __byte_perm(e[0], e[1], 0x7531),
-                                        __byte_perm(e[2], e[3], 0x6420), __byte_perm(e[2], e[3], 0x7531)};
-                const uint32_t ao[4] = {__byte_perm(o[0], o[1], 0x6420), __byte_perm(o[0], o[1], 0x7531),
-                                        __byte_perm(o[2], o[3], 0x6420), __byte_perm(o[2], o[3], 0x7531)};
-                mma_s8(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
-                mma_s8(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
-              }
+            for (int i = 0; i < 4; ++i) {
+              ae[i] = (af[i] << 4) & 0xF0F0F0F0u;       // even rows: 16 * code
+              ao[i] = af[i] & 0xF0F0F0F0u;              // odd rows:  16 * code
+            }
+            if (ks == 0) {
+              mma_s8_first(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
+              mma_s8_first(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
+            } else {
+              mma_s8(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
+              mma_s8(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
             }
           }
-          // digit sums -> float; the four digits of a row sit in lanes tig = 0 and 1 of its quad,
-          // and only those two lanes need the total
-          float v[LROWS];
-          // lane tig = 0 holds the sums of digits 0 and 1 of its rows, tig = 1 those of digits 2 and 3
-          // (wb is the weight of the lower digit of the pair; 0 in lanes tig >= 2)
-          if (BITS == 8) {
-            v[0] = digit_pair_to_float(acc0[0], acc0[1], wb);
-            v[1] = digit_pair_to_float(acc0[2], acc0[3], wb);
-          } else {
-            v[0] = digit_pair_to_float(acc0[0], acc0[1], wb);
-            v[2] = digit_pair_to_float(acc0[2], acc0[3], wb);
-            v[1] = digit_pair_to_float(acc1[0], acc1[1], wb);
-            v[3] = digit_pair_to_float(acc1[2], acc1[3], wb);
-          }
-#pragma unroll
-          for (int i = 0; i < LROWS; ++i) {
-            v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 1);
-            if (tig == ch) keep[u][i] = v[i];
-          }
         }
+        // digit sums -> float: lane tig = 0 holds the sums of digits 0 and 1 of its rows, tig = 1 those of
+        // digits 2 and 3 (wb is the weight of the lower digit of the pair; 0 in lanes tig >= 2)
+        if (BITS == 8) {
+          v[ch][0] = digit_pair_to_float(acc0[0], acc0[1], wb);
+          v[ch][1] = digit_pair_to_float(acc0[2], acc0[3], wb);
+        } else {
+          v[ch][0] = digit_pair_to_float(acc0[0], acc0[1], wb);
+          v[ch][2] = digit_pair_to_float(acc0[2], acc0[3], wb);
+          v[ch][1] = digit_pair_to_float(acc1[0], acc1[1], wb);
+          v[ch][3] = digit_pair_to_float(acc1[2], acc1[3], wb);
+        }
+      }
+      // The four digits of a row sit in lanes tig = 0 and 1 of its quad; lane tig = 0 finishes the rows of
+      // chunk 0 and lane tig = 1 those of chunk 1: each hands the other the half it does not keep.
+#pragma unroll
+      for (int i = 0; i < LROWS; ++i) {
+        const float mine = (tig & 1) ? v[1][i] : v[0][i];
+        const float theirs = (tig & 1) ? v[0][i] : v[1][i];
+        keep[u][i] = mine + __shfl_xor_sync(0xFFFFFFFFu, theirs, 1);
       }
     }
     if (STMA) {
@@ -499,11 +491,11 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
         for (int u = 0; u < KT; ++u) {
           if (LROWS == 2) {
             *reinterpret_cast<float2*>(sb + lane_row[u]) =
-                make_float2(bv[u][0] + keep[u][0] + poison, bv[u][1] + keep[u][1] + poison);
+                make_float2(bv[u][0] + keep[u][0], bv[u][1] + keep[u][1]);
           } else {
             *reinterpret_cast<float4*>(sb + lane_row[u]) =
-                make_float4(bv[u][0] + keep[u][0] + poison, bv[u][1] + keep[u][1] + poison,
-                            bv[u][2] + keep[u][2] + poison, bv[u][3] + keep[u][3] + poison);
+                make_float4(bv[u][0] + keep[u][0], bv[u][1] + keep[u][1],
+                            bv[u][2] + keep[u][2], bv[u][3] + keep[u][3]);
           }
         }
         twa_fence_proxy_async();                          // the lanes' writes, before the bulk store reads them
@@ -515,7 +507,7 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
 #pragma unroll
             for (int i = 0; i < LROWS; ++i) {
               const int row = tile_row0 + lane_row[u] + i;
-              if (row >= (D & ~3) && row < D) a.out[row] = bv[u][i] + keep[u][i] + poison;
+              if (row >= (D & ~3) && row < D) a.out[row] = bv[u][i] + keep[u][i];
             }
         }
       }
@@ -546,16 +538,16 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
         if (whole || row <= D - LROWS) {
           if (LROWS == 2) {
             *reinterpret_cast<float2*>(a.out + row) =
-                make_float2(bv[u][0] + keep[u][0] + poison, bv[u][1] + keep[u][1] + poison);
+                make_float2(bv[u][0] + keep[u][0], bv[u][1] + keep[u][1]);
           } else {
             *reinterpret_cast<float4*>(a.out + row) =
-                make_float4(bv[u][0] + keep[u][0] + poison, bv[u][1] + keep[u][1] + poison,
-                            bv[u][2] + keep[u][2] + poison, bv[u][3] + keep[u][3] + poison);
+                make_float4(bv[u][0] + keep[u][0], bv[u][1] + keep[u][1],
+                            bv[u][2] + keep[u][2], bv[u][3] + keep[u][3]);
           }
         } else {
 #pragma unroll
           for (int i = 0; i < LROWS; ++i)
-            if (row + i < D) a.out[row + i] = bv[u][i] + keep[u][i] + poison;
+            if (row + i < D) a.out[row + i] = bv[u][i] + keep[u][i];
         }
       }
     }
@@ -718,7 +710,7 @@ int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_
   a.g_off = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt;
   a.tx_bytes = a.g_off + static_cast<unsigned>(rows * gsz);
   a.stage_bytes = static_cast<unsigned>(round_up_i(static_cast<int>(a.tx_bytes), 1024));
-  const int fixed = TWA_SMEM_HEADER + MMA_WARPS * DIGIT_SCRATCH + 1024;   // 1024: alignment slack
+  const int fixed = TWA_SMEM_HEADER + MMA_WARPS * BYTE_DIGIT_SCRATCH + 1024;   // 1024: alignment slack
   int stages = (ctx->smem_optin - fixed) / static_cast<int>(a.stage_bytes);
   if (stages > TWA_MAX_STAGES) stages = TWA_MAX_STAGES;
   if (ctx->tune_stages >= 2 && ctx->tune_stages < stages) stages = ctx->tune_stages;
@@ -740,7 +732,7 @@ int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_
   a.wait_limit_ns = ctx->wait_limit_ns;
   int grid = ctx->sm_count < a.tiles ? ctx->sm_count : a.tiles;
   if (grid > TWA_MAX_GRID) grid = TWA_MAX_GRID;
-  const int smem = static_cast<int>(a.scratch_off) + MMA_WARPS * DIGIT_SCRATCH + 1024;
+  const int smem = static_cast<int>(a.scratch_off) + MMA_WARPS * BYTE_DIGIT_SCRATCH + 1024;
   if (P->bits == 8)
     return bf16 ? launch_project_mma_mt<8, true>(ctx, mp, mg, a, grid, smem)
                 : launch_project_mma_mt<8, false>(ctx, mp, mg, a, grid, smem);

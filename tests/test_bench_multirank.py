@@ -60,7 +60,8 @@ def test_reference_arm_prints_only_on_rank_zero(monkeypatch):
     import argparse
     import bench
     monkeypatch.setenv("RANK", "1")
-    args = argparse.Namespace(workload="tiny", bits=8, steps=1, warmup=0, gpus=2, reference_rows=4096)
+    args = argparse.Namespace(workload="tiny", bits=8, steps=2, warmup=0, gpus=2, reference_rows=4096,
+                              reference_max_steps=20)
     buf = io.StringIO()
     with redirect_stdout(buf):
         bench.run_reference(args)
@@ -72,6 +73,28 @@ def test_reference_arm_prints_only_on_rank_zero(monkeypatch):
     line = json.loads(buf.getvalue())
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["value"] > 0
+    # the record says what really ran: seconds timed, threads used, one-thread figure, the host
+    cpu = line["cpu_baseline"]
+    assert cpu["timed_seconds"] > 0 and cpu["single_thread"]["threads"] == 1 and cpu["host_cores"] >= 1
+    assert line["config"]["workload"] == bench.workload_label(bench_inputs().WORKLOADS["tiny"], 1048576, 8)
+
+
+def bench_inputs():
+    from paper_2205_13104_b200 import inputs
+    return inputs
+
+
+def test_series_statistics_and_clock_windows():
+    import bench
+    st = bench.series_stats([3.0, 1.0, 2.0, 10.0])
+    assert st == {"mean": 4.0, "median": 2.5, "min": 1.0, "max": 10.0}
+    s = bench.ClockSampler(0)
+    s.samples = [(10.0, 1900.0, 1965.0, 900.0, []), (10.5, 1500.0, 1965.0, 1000.0, ["sw_power_cap"]),
+                 (11.0, 1600.0, 1965.0, 990.0, ["sw_power_cap"])]
+    assert s.summary(10.4, 11.1)["sm_mhz"] == 1600.0 and s.summary(10.4, 11.1)["reasons"] == ["sw_power_cap"]
+    assert s.summary(9.0, 10.1) == {"sm_mhz": 1900.0, "sm_max_mhz": 1965.0, "samples": 1, "power_w_max": 900.0,
+                                    "reasons": []}
+    assert s.summary(20.0, 21.0)["sm_mhz"] == 1600.0           # no sample inside: the nearest one
 
 
 def test_step_byte_accounting():

@@ -587,3 +587,88 @@ def test_panel_build_finds_dependence_across_and_inside_panels(env, panel_mode):
     code, detail = twa.twa_get_status(ctx)
     assert code == twa.TWA_ERR_NONFINITE and 8 <= detail <= 15      # reported for the panel that holds it
     twa.twa_clear_status(ctx)
+
+
+@pytest.mark.parametrize("ratio,deficient", [(3e-5, False), (3e-6, True)])
+def test_nearly_dependent_column_inside_a_panel_all_schedules_agree(env, ratio, deficient):
+    """One candidate of the second panel is its neighbour plus a small step, so that its remainder
+    after orthogonalisation is `ratio` times its length: just above the float32 rank rule (1e-5)
+    the three schedules and the oracle give the same orthonormal basis, just below it all three
+    report that column (the oracle, run with the same rule, names the same one)."""
+    ctx, ws = env
+    D, n, col = 60001, 20, 11
+    wbar = torch.empty(D, device=DEV)
+
+    def candidates():
+        W = inputs.trajectory_candidates(D, n, 0.01, 0.002, 5, DEV, ld=inputs.padded_ld(D, 4))
+        gen = torch.Generator(device=DEV)
+        gen.manual_seed(77)
+        xi = torch.randn(D, generator=gen, device=DEV)
+        W[col, :D] = W[col - 1, :D] + xi * (ratio * W[col - 1, :D].norm() / xi.norm())
+        return W
+
+    A = host_cols(candidates(), D).copy()
+    Q, _, bad = orc.cgs2(A, rel_tol=1e-5)                       # the GPU build's rule
+    assert (bad == col) if deficient else (bad is None)
+    kappa = np.linalg.cond(A.astype(np.float64))
+    out = {}
+    for mode in (1, 2, 0):
+        W = candidates()
+        twa.twa_set_tuning(ctx, twa.TWA_TUNE_BUILD_PANEL, mode)
+        try:
+            twa.twa_build_basis(ctx, W, D, wbar, ws)
+        finally:
+            twa.twa_set_tuning(ctx, twa.TWA_TUNE_BUILD_PANEL, 0)
+        code, detail = twa.twa_get_status(ctx)
+        twa.twa_clear_status(ctx)
+        Pg = host_cols(W, D).astype(np.float64)
+        if deficient:
+            assert (code, detail) == (twa.TWA_ERR_RANK_DEFICIENT, col), mode
+            keep = [j for j in range(n) if j != col]
+            assert np.all(Pg[:, col] == 0)
+            assert np.max(np.abs(Pg[:, keep].T @ Pg[:, keep] - np.eye(n - 1))) <= 1e-5, mode
+        else:
+            assert code == 0, (mode, code, detail)
+            assert np.max(np.abs(Pg.T @ Pg - np.eye(n))) <= 1e-5, mode
+            assert np.max(np.linalg.norm(Pg - Q, axis=0)) <= 10 * kappa * np.finfo(np.float32).eps, mode
+        out[mode] = Pg
+    if not deficient:
+        for mode in (0, 2):
+            assert np.max(np.linalg.norm(out[mode] - out[1], axis=0)) <= 20 * kappa * np.finfo(np.float32).eps
+
+
+def test_step_keeps_the_coefficients_when_the_gradient_is_not_finite(env):
+    """alpha is state that outlives a call: a step whose projection is not finite reports
+    TWA_ERR_NONFINITE, leaves alpha as it was and lifts w from that alpha; after clearing the status
+    the next step continues as if the bad one had not been made."""
+    ctx, ws = env
+    D, n = 20011, 12
+    for bits in (8, 32):
+        P = random_basis(D, n, 21)
+        B = twa.basis_from_tensor(P, D)
+        if bits != 32:
+            B = twa.twa_quantize_basis(ctx, B, bits, ws)
+        wbar = torch.randn(D, device=DEV)
+        alpha = torch.zeros(n, device=DEV)
+        w = torch.empty(D, device=DEV)
+        g = inputs.gradient(D, 1e-3, 4, 0, torch.float32, DEV)
+        twa.twa_step(ctx, B, g, 0.1, 0.0, alpha, wbar, w, ws)
+        status_ok(ctx)
+        before, w_before = alpha.clone(), w.clone()
+        g_bad = g.clone()
+        g_bad[1234] = float("nan")
+        c = torch.empty(n, device=DEV)
+        twa.twa_step(ctx, B, g_bad, 0.1, 0.0, alpha, wbar, w, ws, c_out=c)
+        code, _ = twa.twa_get_status(ctx)
+        assert code == twa.TWA_ERR_NONFINITE
+        assert torch.isnan(c).any()
+        assert torch.equal(alpha, before)
+        if bits != 32:
+            assert torch.equal(w, w_before)                 # lifted from the unchanged alpha
+        twa.twa_clear_status(ctx)
+        # the same good step twice from the same state gives the same alpha as stepping once more
+        ref = before.clone()
+        twa.twa_step(ctx, B, g, 0.1, 0.0, ref, wbar, torch.empty(D, device=DEV), ws)
+        twa.twa_step(ctx, B, g, 0.1, 0.0, alpha, wbar, w, ws)
+        status_ok(ctx)
+        assert torch.equal(alpha, ref)

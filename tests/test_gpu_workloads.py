@@ -14,6 +14,7 @@ import pytest
 import torch
 
 from oracle import twa_oracle as orc
+from oracle_stream import HostColumns, WeightedGradientSum, project_f32_columns, project_packed
 from paper_2205_13104_b200 import inputs, twa
 
 pytestmark = pytest.mark.gpu
@@ -49,55 +50,171 @@ def host_col(t, j, D):
     return t[j, :D].cpu().numpy()
 
 
-def oracle_project_chunked(codes, scales, g, chunk=1 << 24):
-    """oracle.project summed over row chunks (it is linear in the rows)."""
-    D = codes.shape[0]
-    c = np.zeros(codes.shape[1])
-    for r0 in range(0, D, chunk):
-        c += orc.project(codes[r0:r0 + chunk], scales, g[r0:r0 + chunk])
-    return c
+def oracle_project_all(ctx, basis, gs, block=8):
+    """The oracle's projection of ALL n columns at full size, for every gradient of the list gs in
+    one pass: the canonical codes leave the device eight columns at a time and go through
+    oracle.project in row chunks (tests/oracle_stream.py); a float32 basis goes through
+    oracle.project_f32 the same way.  Returns C (n, len(gs)) and, per column, a lower bound of
+    ||p~_j||: |s_j| qmax (the element that set the scale has the code +-qmax), or for float32 the
+    largest |entry|."""
+    D, n, bits = basis.D, basis.n, basis.bits
+    cs, low = [], []
+    for j0 in range(0, n, block):
+        cols = min(block, n - j0)
+        if bits == 32:
+            vals = np.asfortranarray(np.stack([basis.data[j, :D].cpu().numpy() for j in range(j0, j0 + cols)], axis=1))
+            cs.append(project_f32_columns(vals, gs))
+            low.append(np.abs(vals).max(axis=0).astype(np.float64))
+            continue
+        codes, s = twa.twa_basis_export(ctx, twa.basis_view(basis, col0=j0, cols=cols))
+        packed = codes.cpu().numpy()
+        del codes
+        s_h = s.cpu().numpy()
+        cs.append(project_packed(packed, s_h, D, bits, gs))
+        low.append(np.abs(s_h.astype(np.float64)) * orc.QMAX[bits])
+        del packed
+    return np.concatenate(cs, axis=0), np.concatenate(low)
 
 
-def check_step_sampled(ctx, ws, wl, Pq, wbar, bits, col_blocks, row_ranges):
-    """One fused step from alpha = 0 on the full workload; oracle on sampled columns / rows."""
-    D, n = wl.D, wl.n
-    g = wl.gradient(0, DEV)
-    alpha = torch.zeros(n, device=DEV)
-    w = torch.empty(D, device=DEV)
-    c = torch.empty(n, device=DEV)
-    twa.twa_step(ctx, Pq, g, LR, 0.0, alpha, wbar, w, ws, c_out=c)
-    status_ok(ctx)
-    g_host = g.float().cpu().numpy()
-    c_host, a_host = c.cpu().numpy(), alpha.cpu().numpy()
+def assert_coefficients(c_got, c_ref, norm_low, g_norm):
+    """Every one of the n coefficients against the oracle: the stated relative L2 bound, and element
+    by element (a single wrong column cannot hide under the norm) 1e-5 of the largest coefficient
+    and 1e-5 ||p~_j|| ||g|| with ||p~_j|| replaced by a lower bound of it."""
+    c_got = np.asarray(c_got, dtype=np.float64)
+    assert rel(c_got, c_ref) <= TOL
+    err = np.abs(c_got - c_ref)
+    assert np.all(err <= TOL * np.max(np.abs(c_ref)))
+    assert np.all(err <= TOL * norm_low * g_norm)
+
+
+def check_lift_rows(ctx, Pq, bits, w, alpha64, wbar, row_ranges, offset=None):
+    """Rows of w against the oracle's lift with the given float64 coefficients: relative L2 and,
+    with a base point, a few float32 ulps element by element.  w is the device vector, or (with
+    `offset`) a host copy of the rows from `offset` on."""
+    D = Pq.D
     seg = 512 * 8 // bits
-    for j0 in col_blocks:
-        cols = min(8, n - j0)
-        codes, s = twa.twa_basis_export(ctx, twa.basis_view(Pq, col0=j0, cols=cols))
-        co = orc.unpack_codes(codes.cpu().numpy(), D, bits)
-        so = s.cpu().numpy()
-        pick = [0, cols - 1] if cols > 1 else [0]
-        c_ref = oracle_project_chunked(co[:, pick], so[pick], g_host)
-        assert rel(c_host[[j0 + k for k in pick]], c_ref) <= TOL
-        np.testing.assert_allclose(a_host[[j0 + k for k in pick]], -LR * c_ref, rtol=2e-5, atol=0)
-        del codes, co
     for r0, rows in row_ranges:
         assert r0 % seg == 0
         rows = min(rows, D - r0)
         codes, s = twa.twa_basis_export(ctx, twa.basis_view(Pq, row0=r0, rows=rows))
         co = orc.unpack_codes(codes.cpu().numpy(), rows, bits)
-        base = wbar[r0:r0 + rows].cpu().numpy()
-        w_ref = orc.lift(co, s.cpu().numpy(), a_host.astype(np.float64), base)
-        w_got = w[r0:r0 + rows].cpu().numpy()
+        base = None if wbar is None else wbar[r0:r0 + rows].cpu().numpy()
+        w_ref = orc.lift(co, s.cpu().numpy(), alpha64, base)
+        w_got = w[r0:r0 + rows].cpu().numpy() if offset is None else w[r0 - offset:r0 - offset + rows]
         assert rel(w_got, w_ref) <= TOL
-        assert np.max(np.abs(w_got - w_ref.astype(np.float32))) <= 4 * np.spacing(np.float32(np.abs(w_ref).max()))
-    # the lift alone, without the base point: the bound that is not carried by w_bar
-    twa.twa_lift(ctx, Pq, alpha, None, w, ws)
-    for r0, rows in row_ranges[:1]:
-        rows = min(rows, D - r0)
-        codes, s = twa.twa_basis_export(ctx, twa.basis_view(Pq, row0=r0, rows=rows))
-        co = orc.unpack_codes(codes.cpu().numpy(), rows, bits)
-        assert rel(w[r0:r0 + rows].cpu().numpy(), orc.lift(co, s.cpu().numpy(), a_host.astype(np.float64), None)) <= TOL
+        if wbar is not None:
+            assert np.max(np.abs(w_got - w_ref.astype(np.float32))) <= 4 * np.spacing(np.float32(np.abs(w_ref).max()))
+
+
+def sampled_row_ranges(D, bits, n):
+    """Row ranges of the lift to compare: the first tiles, the tiles where the second and a middle
+    sweep of the persistent grid begin, a range across row 2^30 (where it exists), the middle, the
+    last whole tile and the ragged end.  All start on a 512-byte segment of the codes."""
+    seg = 512 * 8 // bits
+    tile = seg * (2 if n <= 64 else 1)
+    last = ((D - 1) // seg) * seg
+    out = [(0, 2 * tile + seg), ((D // 2 // seg) * seg, 3 * seg), (max(0, last - 2 * tile), 2 * tile), (last, seg)]
+    for t in (148, 148 * 37 + 5):
+        if (t + 2) * tile < D:
+            out.append((t * tile - seg, 2 * tile))
+    if D > (1 << 30) + 2 * tile:
+        out.append(((1 << 30) - tile, 2 * tile))
+    return sorted(set(out))
+
+
+def host_columns(ctx, basis, cols):
+    """The given columns of a basis on the host for the step-by-step oracle (cols None = all)."""
+    D, n = basis.D, basis.n
+    cols = list(range(n)) if cols is None else list(cols)
+    if not cols:
+        return None, cols
+    if basis.bits == 32:
+        vals = np.asfortranarray(np.stack([basis.data[j, :D].cpu().numpy() for j in cols], axis=1))
+        return HostColumns(vals, None, 32), cols
+    vals, scales = [], []
+    for j in cols:
+        codes, s = twa.twa_basis_export(ctx, twa.basis_view(basis, col0=j - j % 8, cols=min(8, n - (j - j % 8))))
+        vals.append(orc.unpack_codes(codes[j % 8:j % 8 + 1].cpu().numpy(), D, basis.bits)[:, 0])
+        scales.append(s[j % 8].item())
+        del codes
+    return HostColumns(np.asfortranarray(np.stack(vals, axis=1)), np.array(scales, dtype=np.float32), basis.bits), cols
+
+
+def run_sequence(ctx, ws, wl, bases, wbar, T, sample_cols):
+    """T fused steps from alpha = 0 with a fresh gradient every step (the loop of Algorithm 1 as the
+    workload states it), on every basis of `bases` side by side, in the launch configuration the
+    benchmark times.  Against the oracle:
+      * step 1: all n coefficients c and alpha element by element, rows of w on sampled ranges;
+      * every step: the oracle steps the sampled columns (all columns when sample_cols is None, none
+        when it is empty) through project + update; the library's alpha on those columns is compared
+        on the way;
+      * after step T: all n coefficients against alpha_T = -lr P~^T G, G the weighted sum of the T
+        gradients (the oracle's own stepped columns must agree with it to 1e-9), rows of w against
+        the oracle's lift with that alpha_T, and the lift alone without the base point."""
+    D, n = wl.D, wl.n
+    state = []
+    for basis in bases:
+        cols_h, cols = host_columns(ctx, basis, sample_cols)
+        state.append(dict(basis=basis, alpha=torch.zeros(n, device=DEV), w=torch.empty(D, device=DEV),
+                          c=torch.empty(n, device=DEV), cols_h=cols_h, cols=cols, a_or=np.zeros(len(cols))))
+    gdt = torch.bfloat16 if wl.g_dtype == "bf16" else torch.float32
+    g = torch.empty(D, dtype=gdt, device=DEV)
+    g32 = torch.empty(D, device=DEV) if gdt != torch.float32 else None
+    g_pin = torch.empty(D, dtype=torch.float32).pin_memory()
+    g_host = g_pin.numpy()
+    gsum = WeightedGradientSum(D, T, LR, 0.0)
+    g0 = None
+    for t in range(T):
+        wl.gradient(t, DEV, out=g)
+        for st in state:
+            twa.twa_step(ctx, st["basis"], g, LR, 0.0, st["alpha"], wbar, st["w"], ws, c_out=st["c"])
+        if g32 is not None:
+            g32.copy_(g)                                   # exact widening of bfloat16
+        g_pin.copy_(g if g32 is None else g32)
+        torch.cuda.synchronize()
+        gsum.add(g_host)
+        for st in state:
+            if len(st["cols"]):
+                c_or = st["cols_h"].project(g_host)
+                st["a_or"] = orc.sgd_update(st["a_or"], c_or, LR, 0.0)
+        if t == 0:
+            g0 = g_host.copy()
+            for st in state:
+                bits = st["basis"].bits
+                st["c0"], st["a0"] = st["c"].cpu().numpy(), st["alpha"].cpu().numpy()
+                if bits != 32:
+                    st["ranges"] = sampled_row_ranges(D, bits, n)
+                    st["w0"] = [st["w"][r0:r0 + rows].cpu().numpy() for r0, rows in st["ranges"]]
+        if t in (0, T // 3, (2 * T) // 3, T - 1):
+            for st in state:
+                if len(st["cols"]):
+                    assert rel(st["alpha"].cpu().numpy()[st["cols"]], st["a_or"]) <= TOL
     status_ok(ctx)
+    G = gsum.result()
+    g0_norm = float(np.sqrt(np.dot(g0.astype(np.float64), g0.astype(np.float64))))
+    for st in state:
+        basis, bits = st["basis"], st["basis"].bits
+        a_T = st["alpha"].cpu().numpy()
+        C, norm_low = oracle_project_all(ctx, basis, [g0, G])
+        c0_ref, a_lin = C[:, 0], -LR * C[:, 1]
+        assert_coefficients(st["c0"], c0_ref, norm_low, g0_norm)
+        a0_ref = orc.sgd_update(np.zeros(n), c0_ref, LR, 0.0)
+        assert_coefficients(st["a0"], a0_ref, LR * norm_low, g0_norm)
+        if len(st["cols"]):
+            assert rel(st["a_or"], a_lin[st["cols"]]) <= 1e-9   # the oracle with itself: stepped = linear form
+        assert rel(a_T, a_lin) <= TOL
+        assert np.all(np.abs(a_T - a_lin) <= TOL * np.max(np.abs(a_lin)))
+        st["a_lin"] = a_lin
+        if bits == 32:
+            continue                                        # the caller compares the whole of w
+        for (r0, rows), w_got in zip(st["ranges"], st["w0"]):
+            check_lift_rows(ctx, basis, bits, w_got, a0_ref, wbar, [(r0, rows)], offset=r0)
+        check_lift_rows(ctx, basis, bits, st["w"], a_lin, wbar, st["ranges"])
+        # the lift alone, without the base point: the bound that is not carried by w_bar
+        twa.twa_lift(ctx, basis, st["alpha"], None, st["w"], ws)
+        check_lift_rows(ctx, basis, bits, st["w"], a_T.astype(np.float64), None, st["ranges"][:3])
+        status_ok(ctx)
+    return state
 
 
 def check_codes_sampled(ctx, P32, Pq, bits, cols):
@@ -193,20 +310,19 @@ def test_workload_resnet18_float32_and_int8(env):
     codes_o, s_o = orc.quantize(np.asfortranarray(Pg), 8)
     np.testing.assert_array_equal(s_g.cpu().numpy(), s_o)
     np.testing.assert_array_equal(codes_g.cpu().numpy(), orc.pack_codes(codes_o, 8))
-    for basis, ostep in ((P32, lambda g, a: orc.step_f32(Pg, g, a, wbar.cpu().numpy(), LR)),
-                         (Pq, lambda g, a: orc.step(codes_o, s_o, g, a, wbar.cpu().numpy(), LR))):
-        alpha = torch.zeros(n, device=DEV)
-        w = torch.empty(D, device=DEV)
-        c = torch.empty(n, device=DEV)
-        a_o = np.zeros(n)
-        for t in range(3):                                # fresh gradient every step
-            g = wl.gradient(t, DEV)
-            twa.twa_step(ctx, basis, g, LR, 0.0, alpha, wbar, w, ws, c_out=c)
-            a_o, w_o, c_o = ostep(g.cpu().numpy(), a_o)
-            assert rel(c.cpu().numpy(), c_o) <= TOL
-            assert rel(alpha.cpu().numpy(), a_o) <= TOL
-            assert rel(w.cpu().numpy(), w_o) <= TOL
-        status_ok(ctx)
+    # the workload's 100 steps with a fresh gradient each, float32 and int8 basis side by side; the
+    # oracle steps every column; after the last step the whole of w, element by element
+    state = run_sequence(ctx, ws, wl, [P32, Pq], wbar, wl.steps, [0, 7, n - 1])
+    wbar_h = wbar.cpu().numpy()
+    for st, w_o in ((state[0], orc.lift_f32(Pg, state[0]["a_lin"], wbar_h)),
+                    (state[1], orc.lift(codes_o, s_o, state[1]["a_lin"], wbar_h))):
+        w_g = st["w"].cpu().numpy() if st["basis"].bits == 32 else None
+        if w_g is None:                                   # run_sequence ended the int8 leg with a lift without base
+            twa.twa_lift(ctx, Pq, st["alpha"], wbar, st["w"], ws)
+            w_g = st["w"].cpu().numpy()
+        assert rel(w_g, w_o) <= TOL
+        assert np.max(np.abs(w_g - w_o.astype(np.float32))) <= 4 * np.spacing(np.float32(np.abs(w_o).max()))
+    status_ok(ctx)
 
 
 # ------------------------------------------------------------------ ResNet-50- and ViT-B-sized: sampled
@@ -228,29 +344,34 @@ def test_workload_resident_build_sampled(env, name, bits_list):
         np.testing.assert_array_equal(wbar[r0:r0 + 4099].cpu().numpy(), orc.mean(blk).astype(np.float32))
     del A
     torch.cuda.empty_cache()
+    bases = []
     for bits in bits_list:
-        seg = 512 * 8 // bits
         Pq = twa.twa_quantize_basis(ctx, P32, bits, ws)
         status_ok(ctx)
         check_codes_sampled(ctx, P32, Pq, bits, [0, n // 2 + 1, n - 1])
-        last = (D // seg) * seg                           # the ragged last segment
-        check_step_sampled(ctx, ws, wl, Pq, wbar, bits, col_blocks=[0, ((n - 1) // 8) * 8],
-                           row_ranges=[(0, 2 * seg), ((D // 2 // seg) * seg, 3 * seg), (last, seg)])
-        del Pq
-        torch.cuda.empty_cache()
+        bases.append(Pq)
+    del P32, W
+    torch.cuda.empty_cache()
+    # the workload's 100 steps; the oracle steps two sampled columns
+    run_sequence(ctx, ws, wl, bases, wbar, wl.steps, [17, n - 1])
+    del bases
+    torch.cuda.empty_cache()
 
 
 # ------------------------------------------------------------------ 1.3 B-sized: chunked build, sampled
 def test_workload_decoder_chunked_build_sampled(env):
+    """The 1.3 B-sized workload: one row-chunked build gives the int8 and the int4 basis (the scales
+    of both widths come from the absmax of pass 2, the codes of both from the chunks of pass 3);
+    then the workload's 50 steps on both, checked as run_sequence describes."""
     ctx, ws = env
     wl = inputs.WORKLOADS["decoder1p3b"]
-    D, n, bits = wl.D, wl.n, 8
+    D, n = wl.D, wl.n
     CH = inputs.CHUNK_ROWS
     starts = list(range(0, D, CH))
     sampled = {starts[0]: None, starts[len(starts) // 2]: None, starts[-1]: None}
     bws = torch.empty(twa.twa_build_workspace_bytes(n), dtype=torch.uint8, device=DEV)
     wbar = torch.empty(D, device=DEV)
-    Pq = twa.new_quantised_basis(D, n, bits, DEV)
+    bases = {bits: twa.new_quantised_basis(D, n, bits, DEV) for bits in (8, 4)}
     buf = torch.empty((n, CH), device=DEV)
     qbuf = torch.empty((n, CH), device=DEV)
     twa.twa_build_begin(ctx, D, n, wbar, bws)
@@ -259,25 +380,39 @@ def test_workload_decoder_chunked_build_sampled(env):
             rows = min(CH, D - r0)
             inputs.trajectory_rows(D, n, wl.step, wl.drift, wl.seed, DEV, row0=r0, rows=rows, out=buf[:, :rows])
             keep = p == 3 and r0 in sampled
-            twa.twa_build_feed(ctx, p, buf, r0, rows, Pq=Pq if p == 3 else None, q32_out=qbuf if keep else None)
+            if p < 3:
+                twa.twa_build_feed(ctx, p, buf, r0, rows)
+            else:
+                twa.twa_build_feed(ctx, p, buf, r0, rows, Pq=bases[8], q32_out=qbuf if keep else None)
+                twa.twa_build_feed(ctx, p, buf, r0, rows, Pq=bases[4])
             if keep:
                 sampled[r0] = (qbuf[:, :rows].cpu().numpy().T.copy(), buf[:, :rows].cpu().numpy().T.copy())
-        twa.twa_build_end_pass(ctx, p, bits if p == 2 else 0, Pq if p == 2 else None)
+        if p == 2:
+            twa.twa_build_end_pass(ctx, p, 8, bases[8])
+            twa.twa_build_end_pass(ctx, p, 4, bases[4])
+        else:
+            twa.twa_build_end_pass(ctx, p, 0, None)
     status_ok(ctx)
     del buf, qbuf, bws
     torch.cuda.empty_cache()
-    scales = Pq.scales.cpu().numpy()
+    for bits, Pq in bases.items():
+        scales = Pq.scales.cpu().numpy()
+        qmax = orc.QMAX[bits]
+        for r0, (q32, a_rows) in sampled.items():
+            rows = q32.shape[0]
+            # codes of the chunk = the oracle's encoder on the chunk's float32 rows with the global scales
+            codes, _ = twa.twa_basis_export(ctx, twa.basis_view(Pq, row0=r0, rows=rows))
+            co = orc.encode(np.asfortranarray(q32), scales, bits)
+            np.testing.assert_array_equal(codes.cpu().numpy(), orc.pack_codes(co, bits))
+            assert np.all(np.abs(q32).max(axis=0) <= scales * qmax * (1 + 1e-6))
+            del codes, co
+    M0 = None
     for r0, (q32, a_rows) in sampled.items():
         rows = q32.shape[0]
-        # codes of the chunk = the oracle's encoder on the chunk's float32 rows with the global scales
-        codes, _ = twa.twa_basis_export(ctx, twa.basis_view(Pq, row0=r0, rows=rows))
-        co = orc.encode(np.asfortranarray(q32), scales, bits)
-        np.testing.assert_array_equal(codes.cpu().numpy(), orc.pack_codes(co, bits))
-        assert np.all(np.abs(q32).max(axis=0) <= scales * 127 * (1 + 1e-6))
         # w_bar rows = the oracle's mean of the candidate rows
         np.testing.assert_array_equal(wbar[r0:r0 + rows].cpu().numpy(), orc.mean(a_rows).astype(np.float32))
         # rows of Q are rows of A times one upper-triangular matrix: the same M for every chunk
-        if r0 == 0:
+        if M0 is None:
             M0, *_ = np.linalg.lstsq(a_rows[:65536].astype(np.float64), q32[:65536].astype(np.float64), rcond=None)
             assert np.max(np.abs(np.tril(M0, -1))) <= 1e-3 * np.max(np.abs(M0))
             assert np.all(np.diag(M0) > 0)
@@ -286,14 +421,12 @@ def test_workload_decoder_chunked_build_sampled(env):
             assert np.linalg.norm(resid) <= 1e-5 * np.linalg.norm(q32[:65536])
     sampled.clear()
     # unit columns: the dequantised basis has norm 1 up to the quantisation error (oracle on one column)
-    codes, s = twa.twa_basis_export(ctx, twa.basis_view(Pq, col0=24, cols=8))
+    codes, s = twa.twa_basis_export(ctx, twa.basis_view(bases[8], col0=24, cols=8))
     col = codes[7].cpu().numpy().view(np.int8)[:D].astype(np.float64)
     assert abs(np.sqrt(np.dot(col, col)) * float(s[7]) - 1.0) <= 2e-3
-    del codes
+    del codes, col
     torch.cuda.empty_cache()
-    seg = 512
-    check_step_sampled(ctx, ws, wl, Pq, wbar, bits, col_blocks=[24],
-                       row_ranges=[(0, 2 * seg), ((D // 2 // seg) * seg, 2 * seg), (D - seg, seg)])
+    run_sequence(ctx, ws, wl, [bases[8], bases[4]], wbar, wl.steps, [])
 
 
 # ------------------------------------------------------------------ the layer-wise construction, full size
@@ -389,13 +522,14 @@ def test_workload_layerwise_sampled(env, name, bits_list):
         torch.cuda.empty_cache()
 
 
-def test_workload_decoder_layerwise_chunked_sampled(env):
+@pytest.mark.parametrize("bits", [8, 4])
+def test_workload_decoder_layerwise_chunked_sampled(env, bits):
     """The paper's default construction at the 1.3 B size, built from row chunks: mean rows, per-layer
-    factors and sampled codes bit-exact against the oracle on the float32 vectors of the build's own
-    second pass; one layer-wise step checked on sampled layers, columns and rows."""
+    factors and codes of sampled layers bit-exact against the oracle on the float32 vectors of the
+    build's own second pass; one layer-wise step checked on sampled layers (all n columns) and rows."""
     ctx, _ = env
     wl = inputs.WORKLOADS["decoder1p3b"]
-    D, n, bits = wl.D, wl.n, 8
+    D, n = wl.D, wl.n
     layers = inputs.layer_offsets("decoder1p3b")
     L = len(layers) - 1
     sizes = np.diff(layers)
@@ -428,7 +562,7 @@ def test_workload_decoder_layerwise_chunked_sampled(env):
         np.testing.assert_array_equal(wbar[r0:r0 + a_rows.shape[0]].cpu().numpy(), orc.mean(a_rows).astype(np.float32))
     packed, a_g, b_g = twa.twa_layered_export(ctx, lb)
     a_h, b_h = a_g.cpu().numpy(), b_g.cpu().numpy()
-    cols = [0, n // 2, n - 1]
+    cols = list(range(n))
     for l in pick:
         r0, r1 = layers[l], layers[l + 1]
         blk = blocks[l]

@@ -142,3 +142,29 @@ def test_project_batch_brute_force_and_dense_product():
     G2[:, 3] = 0
     out = orc.project_batch(codes, s, G2)
     assert np.all(out[:, 3] == 0) and np.all(out[:, [0, 1, 2, 4]] == orc.project_batch(codes, s, G)[:, [0, 1, 2, 4]])
+
+
+# ------------------------------------------------------------------ many steps in a row
+def test_many_steps_end_at_the_projection_of_the_weighted_gradient_sum():
+    """T steps of Algorithm 1's loop from alpha = 0 end at alpha_T = -eta P~^T G with
+    G = sum_t (1 - eta*lambda)^(T-1-t) g_t, and w_T = w_bar + P~ alpha_T: the form the full-size
+    sequence tests use where stepping the oracle through every gradient is out of reach."""
+    from oracle_stream import weighted_gradient_sum
+    D, n, T = 700, 6, 40
+    _, _, codes, s = _quantised_basis(D, n, 8, seed=7)
+    rng = np.random.default_rng(8)
+    wbar = rng.standard_normal(D).astype(np.float32)
+    for lr, lam in ((0.1, 0.0), (0.05, 0.3)):
+        grads = [(rng.standard_normal(D) * 1e-3).astype(np.float32) for _ in range(T)]
+        alpha = np.zeros(n)
+        for g in grads:
+            alpha, w, _ = orc.step(codes, s, g, alpha, wbar, lr, lam)
+        G = weighted_gradient_sum(grads, lr, lam)
+        a_lin = -lr * orc.project(codes, s, G)
+        np.testing.assert_allclose(alpha, a_lin, rtol=1e-12, atol=1e-18)
+        np.testing.assert_allclose(w, orc.lift(codes, s, a_lin, wbar), rtol=1e-13, atol=1e-15)
+    # a dropped decay factor or a reversed order of the weights does not pass
+    bad = np.zeros(D)
+    for t, g in enumerate(grads):
+        bad += (1.0 - 0.05 * 0.3) ** t * g.astype(np.float64)
+    assert np.linalg.norm(-0.05 * orc.project(codes, s, bad) - alpha) > 1e-6 * np.linalg.norm(alpha)

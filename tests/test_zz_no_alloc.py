@@ -1,8 +1,8 @@
 """twa_project_noalloc: the projection for callers that cannot allocate device memory when
 they call (an allocator that owns the whole device, a loop that may not synchronise, a
-plug-in given only its buffers).  It must give what twa_project gives, call after call,
-although it has no context and no workspace and keeps its scratch in a fixed array of the
-library's device image that every call reuses.
+plug-in given only its buffers).  It must give what twa_project gives -- and what the float64
+oracle gives on the same bytes -- call after call, although it has no context and no workspace
+and keeps its scratch in a fixed array of the library's device image that every call reuses.
 
 Collected last on purpose: a failure here cannot hide the result of any other test.
 """
@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import twa_oracle as orc
 from paper_2205_13104_b200 import twa
 
 pytestmark = pytest.mark.gpu
@@ -37,6 +38,11 @@ def test_noalloc_projection_matches_twa_project_twice_in_a_row(bits, gdt):
     B = twa.basis_from_tensor(P, D)
     if bits != 32:
         B = twa.twa_quantize_basis(ctx, B, bits, ws)
+    if bits != 32:                             # the oracle's view of the same basis: canonical codes and scales
+        codes, scales = twa.twa_basis_export(ctx, B)
+        codes_h, scales_h = orc.unpack_codes(codes.cpu().numpy(), D, bits), scales.cpu().numpy()
+    else:
+        P_h = P[:, :D].cpu().numpy().T
     status = torch.full((2,), 99, dtype=torch.int32, device=DEV)
     for call in range(2):                      # the second call meets the first one's leftovers
         g = (torch.randn(D, generator=gen, device=DEV) * 1e-3).to(gdt)
@@ -48,6 +54,10 @@ def test_noalloc_projection_matches_twa_project_twice_in_a_row(bits, gdt):
         assert status[0].item() == 0
         assert _rel(got[:n], want) <= TOL
         assert torch.all(got[n:] == 5.0)
+        g_h = g.float().cpu().numpy()
+        c_o = orc.project(codes_h, scales_h, g_h) if bits != 32 else orc.project_f32(P_h, g_h)
+        assert _rel(got[:n].cpu(), torch.from_numpy(c_o)) <= TOL
+        assert _rel(want.cpu(), torch.from_numpy(c_o)) <= TOL
     assert twa.twa_get_status(ctx)[0] == 0
     twa.twa_destroy(ctx)
 
