@@ -657,48 +657,53 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
 #pragma unroll
       for (int i = 0; i < LROWS; ++i) keep[u][i] = 0.0f;
       if (e.x >= 0) {
+        float v[2][LROWS];                                // per 16-byte chunk of the block
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
-          int acc0[4] = {0, 0, 0, 0};
-          int acc1[4] = {0, 0, 0, 0};
+          int acc0[4], acc1[4];
 #pragma unroll
           for (int ks = 0; ks < KS; ++ks) {
             uint32_t r[4];
             ldmatrix_x4_trans(tile_base + loff[u][ch][ks], r);
+            // the transposing load delivers byte pairs of two columns: regroup to four columns per register
+            const uint32_t af[4] = {__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[0], r[1], 0x7531),
+                                    __byte_perm(r[2], r[3], 0x6420), __byte_perm(r[2], r[3], 0x7531)};
             if (BITS == 8) {
-              const uint32_t af[4] = {__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[0], r[1], 0x7531),
-                                      __byte_perm(r[2], r[3], 0x6420), __byte_perm(r[2], r[3], 0x7531)};
-              mma_u8s8(acc0, af, bfrag[ks][0], bfrag[ks][1]);
+              if (ks == 0) mma_u8s8_first(acc0, af, bfrag[ks][0], bfrag[ks][1]);
+              else mma_u8s8(acc0, af, bfrag[ks][0], bfrag[ks][1]);
             } else {
-              uint32_t ev[4], od[4];
+              uint32_t ae[4], ao[4];
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
-                ev[i] = (r[i] << 4) & 0xF0F0F0F0u;
-                od[i] = r[i] & 0xF0F0F0F0u;
+                ae[i] = (af[i] << 4) & 0xF0F0F0F0u;       // even rows: 16 * code, unsigned
+                ao[i] = af[i] & 0xF0F0F0F0u;              // odd rows
               }
-              const uint32_t ae[4] = {__byte_perm(ev[0], ev[1], 0x6420), __byte_perm(ev[0], ev[1], 0x7531),
-                                      __byte_perm(ev[2], ev[3], 0x6420), __byte_perm(ev[2], ev[3], 0x7531)};
-              const uint32_t ao[4] = {__byte_perm(od[0], od[1], 0x6420), __byte_perm(od[0], od[1], 0x7531),
-                                      __byte_perm(od[2], od[3], 0x6420), __byte_perm(od[2], od[3], 0x7531)};
-              mma_u8s8(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
-              mma_u8s8(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
+              if (ks == 0) {
+                mma_u8s8_first(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
+                mma_u8s8_first(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
+              } else {
+                mma_u8s8(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
+                mma_u8s8(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
+              }
             }
           }
-          float v[LROWS];
           if (BITS == 8) {                                // digit pairs (0,1) in lanes tig = 0, (2,3) in tig = 1
-            v[0] = digit_pair_to_float(acc0[0], acc0[1], wbw);
-            v[1] = digit_pair_to_float(acc0[2], acc0[3], wbw);
+            v[ch][0] = digit_pair_to_float(acc0[0], acc0[1], wbw);
+            v[ch][1] = digit_pair_to_float(acc0[2], acc0[3], wbw);
           } else {
-            v[0] = digit_pair_to_float(acc0[0], acc0[1], wbw);
-            v[2] = digit_pair_to_float(acc0[2], acc0[3], wbw);
-            v[1] = digit_pair_to_float(acc1[0], acc1[1], wbw);
-            v[3] = digit_pair_to_float(acc1[2], acc1[3], wbw);
+            v[ch][0] = digit_pair_to_float(acc0[0], acc0[1], wbw);
+            v[ch][2] = digit_pair_to_float(acc0[2], acc0[3], wbw);
+            v[ch][1] = digit_pair_to_float(acc1[0], acc1[1], wbw);
+            v[ch][3] = digit_pair_to_float(acc1[2], acc1[3], wbw);
           }
+        }
+        // lane tig = 0 finishes the rows of chunk 0, lane tig = 1 those of chunk 1: each hands the other
+        // the digit-pair sums it does not keep
 #pragma unroll
-          for (int i = 0; i < LROWS; ++i) {
-            v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 1);
-            if (tig == ch) keep[u][i] = v[i];
-          }
+        for (int i = 0; i < LROWS; ++i) {
+          const float mine = (tig & 1) ? v[1][i] : v[0][i];
+          const float theirs = (tig & 1) ? v[0][i] : v[1][i];
+          keep[u][i] = mine + __shfl_xor_sync(0xFFFFFFFFu, theirs, 1);
         }
       }
     }

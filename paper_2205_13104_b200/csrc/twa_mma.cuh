@@ -45,6 +45,14 @@ __device__ __forceinline__ void mma_s8_first(int (&d)[4], const uint32_t (&a)[4]
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(0));
 }
 
+// d = a (16 x 32, u8) * b (32 x 8, s8): the first product of a sum, no accumulator to clear
+__device__ __forceinline__ void mma_u8s8_first(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(0));
+}
+
 // |v| < 2^22 -> float, exactly, without the conversion unit
 __device__ __forceinline__ float small_int_to_float(int v) {
   return __int_as_float(0x4B400000 + v) - RND;
@@ -103,7 +111,10 @@ __device__ __forceinline__ void ldmatrix_x2(uint32_t addr, uint32_t& r0, uint32_
 // r + 128, again next to a column of ones.  Error of the cut: 2^-23 (three bytes) or 2^-31 (four)
 // of the power of two above the block's largest magnitude.
 constexpr int BYTE_DIGIT_ROWS = 8;              // rows of a digit matrix: u0, u1, u2, ones, r + 128, ones, 0, 0
-constexpr int BYTE_DIGIT_SET = BYTE_DIGIT_ROWS * 32;      // bytes: one row of 32 gradient rows per digit
+constexpr int BYTE_DIGIT_STRIDE = 48;           // bytes between digit rows: 32 gradient rows + 16 of padding, so
+                                                // that the eight 16-byte rows of a matrix load fall into
+                                                // eight different groups of four banks
+constexpr int BYTE_DIGIT_SET = BYTE_DIGIT_ROWS * BYTE_DIGIT_STRIDE;
 constexpr int BYTE_DIGIT_SCRATCH = 2 * BYTE_DIGIT_SET;    // per warp: even and odd rows (4-bit codes)
 
 struct ByteDigitScale {
@@ -134,7 +145,7 @@ __device__ __forceinline__ void byte_digit_init(unsigned char* digw, int lane) {
 #pragma unroll
   for (int i = 0; i < BYTE_DIGIT_SCRATCH / 128; ++i) {
     const int idx = lane + 32 * i;                         // word of the scratch
-    const int row = (idx % (BYTE_DIGIT_SET / 4)) / 8;
+    const int row = (idx % (BYTE_DIGIT_SET / 4)) / (BYTE_DIGIT_STRIDE / 4);
     w[idx] = (row == 3 || (FOUR && row == 5)) ? 0x01010101u : 0u;
   }
 }
@@ -146,11 +157,11 @@ __device__ __forceinline__ void byte_digit_store(unsigned char* digw, int set, i
   const uint32_t b = __float_as_uint(y);
   unsigned char* d = digw + set * BYTE_DIGIT_SET + lane;
   d[0] = static_cast<unsigned char>(b);
-  d[32] = static_cast<unsigned char>(b >> 8);
-  d[64] = static_cast<unsigned char>(b >> 16);
+  d[BYTE_DIGIT_STRIDE] = static_cast<unsigned char>(b >> 8);
+  d[2 * BYTE_DIGIT_STRIDE] = static_cast<unsigned char>(b >> 16);
   if (FOUR) {
     const float rem = fmaf(g, up, -(y - RND));             // exact: g * up - q
-    d[128] = static_cast<unsigned char>(__float_as_uint(fmaf(rem, 254.0f, RND + 128.0f)));
+    d[4 * BYTE_DIGIT_STRIDE] = static_cast<unsigned char>(__float_as_uint(fmaf(rem, 254.0f, RND + 128.0f)));
   }
 }
 
@@ -158,7 +169,7 @@ __device__ __forceinline__ void byte_digit_store(unsigned char* digw, int set, i
 // half (gradient rows 16 (m & 1) ...) of set m / 2, row lane % 8 is digit lane % 8.
 __device__ __forceinline__ uint32_t byte_digit_ldmatrix_addr(const unsigned char* digw, int lane) {
   const int m = lane >> 3;
-  return twa_smem_u32(digw + (m >> 1) * BYTE_DIGIT_SET + (lane & 7) * 32 + (m & 1) * 16);
+  return twa_smem_u32(digw + (m >> 1) * BYTE_DIGIT_SET + (lane & 7) * BYTE_DIGIT_STRIDE + (m & 1) * 16);
 }
 
 // Lane constants of the recombination: the accumulator columns of lane tig hold digits 2 tig, 2 tig + 1.

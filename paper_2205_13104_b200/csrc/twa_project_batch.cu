@@ -23,7 +23,7 @@ __device__ __forceinline__ void pair_digit_init(unsigned char* digw, int lane) {
 #pragma unroll
   for (int i = 0; i < PAIR_SCRATCH / 128; ++i) {
     const int idx = lane + 32 * i;
-    const int row = (idx % (BYTE_DIGIT_SET / 4)) / 8;
+    const int row = (idx % (BYTE_DIGIT_SET / 4)) / (BYTE_DIGIT_STRIDE / 4);
     w[idx] = (row & 3) == 3 ? 0x01010101u : 0u;
   }
 }
@@ -31,10 +31,10 @@ __device__ __forceinline__ void pair_digit_init(unsigned char* digw, int lane) {
 // The three byte digits of gradient h's value for gradient row `lane` into digit matrix `set`.
 __device__ __forceinline__ void pair_digit_store(unsigned char* digw, int set, int h, int lane, float g, float up) {
   const uint32_t b = __float_as_uint(fmaf(g, up, RND));
-  unsigned char* d = digw + set * BYTE_DIGIT_SET + h * 128 + lane;
+  unsigned char* d = digw + set * BYTE_DIGIT_SET + h * 4 * BYTE_DIGIT_STRIDE + lane;
   d[0] = static_cast<unsigned char>(b);
-  d[32] = static_cast<unsigned char>(b >> 8);
-  d[64] = static_cast<unsigned char>(b >> 16);
+  d[BYTE_DIGIT_STRIDE] = static_cast<unsigned char>(b >> 8);
+  d[2 * BYTE_DIGIT_STRIDE] = static_cast<unsigned char>(b >> 16);
 }
 
 struct BatchArgs {
