@@ -380,20 +380,73 @@ def affine_encode(P32, layers, a, b, bits):
     """code = clamp(round_half_even(fl32(fl32(p - b^l) / a^l)), 0, 2^B - 1); a
     layer with a^l == 0 (constant layer) is all zeros.  Section 4.6, with the
     subtraction and the division both rounded to float32 and ties to even (the
-    paper leaves precision and rounding mode open).  Returns uint8 code VALUES
-    of shape (D, n)."""
+    paper leaves precision and rounding mode open).  Returns the code VALUES of
+    shape (D, n), uint8 (uint16 for B = 16)."""
     P32 = np.asarray(P32)
     assert P32.dtype == np.float32
     D, n = P32.shape
     top = 2 ** bits - 1
-    codes = np.zeros((D, n), dtype=np.uint8, order="F")
+    dt = np.uint16 if bits > 8 else np.uint8
+    codes = np.zeros((D, n), dtype=dt, order="F")
     for l in range(len(layers) - 1):
         if a[l] == 0:
             continue
         r0, r1 = layers[l], layers[l + 1]
         d = (P32[r0:r1, :] - np.float32(b[l])).astype(np.float32)          # float32 subtraction
         t = (d.astype(np.float64) / np.float64(a[l])).astype(np.float32)    # float32 division
-        codes[r0:r1, :] = np.clip(np.rint(t), 0, top).astype(np.uint8)
+        codes[r0:r1, :] = np.clip(np.rint(t), 0, top).astype(dt)
+    return codes
+
+
+SLOT_BITS = {1: 1, 2: 2, 3: 4, 4: 4, 8: 8, 16: 16}
+
+
+def pack_unsigned(codes, bits):
+    """Canonical byte image of unsigned B-bit codes (Section 4.6 stores the quantised matrix
+    as B-bit integers), one row of bytes per column.  A code occupies a slot of 1, 2, 4, 8 or
+    16 bits (3-bit codes sit in 4-bit slots): with S slots per byte, byte k of column j holds
+    rows S*k .. S*k+S-1, row S*k+s in bits [s*slot, (s+1)*slot); 16-bit codes take two bytes,
+    low byte first.  Unused bits are 0.  Returns uint8 of shape (n, ceil(D*slot/8))."""
+    codes = np.asarray(codes)
+    D, n = codes.shape
+    slot = SLOT_BITS[bits]
+    if slot == 16:
+        out = np.zeros((n, 2 * D), dtype=np.uint8)
+        for j in range(n):
+            col = codes[:, j].astype(np.uint32)
+            out[j, 0::2] = (col & 0xFF).astype(np.uint8)
+            out[j, 1::2] = (col >> 8).astype(np.uint8)
+        return out
+    per = 8 // slot
+    nb = (D + per - 1) // per
+    out = np.zeros((n, nb), dtype=np.uint8)
+    for j in range(n):
+        col = codes[:, j].astype(np.uint16)
+        for s_ in range(per):
+            part = col[s_::per]
+            out[j, : part.size] |= (part << (s_ * slot)).astype(np.uint8)
+    return out
+
+
+def unpack_unsigned(packed, D, bits):
+    """Inverse of pack_unsigned: (n, bytes) uint8 -> code values (D, n), uint16."""
+    packed = np.asarray(packed, dtype=np.uint8)
+    n = packed.shape[0]
+    slot = SLOT_BITS[bits]
+    codes = np.zeros((D, n), dtype=np.uint16, order="F")
+    if slot == 16:
+        for j in range(n):
+            b = packed[j].astype(np.uint16)
+            codes[:, j] = (b[0::2] | (b[1::2] << 8))[:D]
+        return codes
+    per = 8 // slot
+    mask = (1 << slot) - 1
+    for j in range(n):
+        b = packed[j].astype(np.uint16)
+        inter = np.empty(per * b.size, dtype=np.uint16)
+        for s_ in range(per):
+            inter[s_::per] = (b >> (s_ * slot)) & mask
+        codes[:, j] = inter[:D]
     return codes
 
 

@@ -142,3 +142,45 @@ def test_layerwise_step_equals_per_layer_weight_space_recursion():
             np.testing.assert_allclose(w, dev, rtol=1e-9, atol=1e-12)
     c0 = orc.project_layerwise(codes, LAYERS, a, b, g)
     np.testing.assert_allclose(orc.step_layerwise(codes, LAYERS, a, b, g, np.zeros((L, n)), wbar, 0.1)[0], -0.1 * c0)
+
+
+def test_unsigned_packing_hand_bytes_and_roundtrip():
+    """The canonical image of unsigned B-bit codes, against bytes worked out by hand."""
+    codes = np.array([[1, 0], [0, 1], [1, 1], [1, 0], [0, 0], [0, 1], [1, 0], [1, 1], [1, 1]], dtype=np.uint8)
+    # 1 bit, column 0 rows 0..8 = 1,0,1,1,0,0,1,1 | 1  -> bits 0,2,3,6,7 = 0xCD, then 0x01
+    np.testing.assert_array_equal(orc.pack_unsigned(codes, 1), [[0xCD, 0x01], [0xA6, 0x01]])
+    c2 = np.array([[3], [0], [2], [1], [1]], dtype=np.uint8)
+    # 2 bits: 3 | 0<<2 | 2<<4 | 1<<6 = 0x63, then 0x01
+    np.testing.assert_array_equal(orc.pack_unsigned(c2, 2), [[0x63, 0x01]])
+    c3 = np.array([[7], [5], [2]], dtype=np.uint8)
+    # 3-bit codes in 4-bit slots: 7 | 5<<4 = 0x57, then 0x02
+    np.testing.assert_array_equal(orc.pack_unsigned(c3, 3), [[0x57, 0x02]])
+    np.testing.assert_array_equal(orc.pack_unsigned(c3, 4), [[0x57, 0x02]])
+    np.testing.assert_array_equal(orc.pack_unsigned(c3, 8), [[7, 5, 2]])
+    c16 = np.array([[0x1234], [0xFFFF], [7]], dtype=np.uint16)
+    np.testing.assert_array_equal(orc.pack_unsigned(c16, 16), [[0x34, 0x12, 0xFF, 0xFF, 0x07, 0x00]])
+    rng = np.random.default_rng(11)
+    for bits in (1, 2, 3, 4, 8, 16):
+        for D in (1, 7, 8, 9, 1001):
+            c = rng.integers(0, 2 ** bits, size=(D, 3)).astype(np.uint16)
+            p = orc.pack_unsigned(c, bits)
+            assert p.shape == (3, (D * orc.SLOT_BITS[bits] + 7) // 8)
+            np.testing.assert_array_equal(orc.unpack_unsigned(p, D, bits), c)
+
+
+def test_affine_quantiser_at_every_width_of_the_ablation():
+    """B in {1, 2, 3, 4, 8, 16} (the paper's bits ablation): codes stay in range, the half-step
+    bound holds, and a two-level layer at 1 bit maps its minimum to 0 and its maximum to 1."""
+    rng = np.random.default_rng(5)
+    P = rng.standard_normal((500, 4)).astype(np.float32)
+    for bits in (1, 2, 3, 4, 8, 16):
+        codes, a, b = orc.affine_quantize(P, [0, 200, 500], bits)
+        assert codes.max() <= 2 ** bits - 1 and codes.min() >= 0
+        deq = orc.affine_dequantize(codes, [0, 200, 500], a, b)
+        step = np.repeat(a.astype(np.float64), [200, 300])[:, None]
+        # half a step, plus the float32 roundings of the subtraction and of the quotient
+        assert np.all(np.abs(deq - P) <= 0.5 * step + 8 * np.finfo(np.float32).eps * np.abs(P).max())
+    two = np.array([[-1.0], [3.0], [3.0], [-1.0]], dtype=np.float32)
+    codes, a, b = orc.affine_quantize(two, [0, 4], 1)
+    assert a[0] == 4.0 and b[0] == -1.0
+    np.testing.assert_array_equal(codes[:, 0], [0, 1, 1, 0])
