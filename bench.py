@@ -721,6 +721,9 @@ def run_layered(args):
     if args.rows:
         wl = dataclasses.replace(wl, name=f"{wl.name}[rows={args.rows}]", D=args.rows)
     D, n, bits, L = wl.D, wl.n, args.bits, len(layers) - 1
+    if bits == 16 and n > 64:
+        raise SystemExit("16-bit codes are stored as two 8-bit planes: at most 64 candidates")
+    slot = {16: 16, 8: 8, 4: 4, 3: 4, 2: 2, 1: 1}[bits]   # bits of device memory per code
     g_bytes = 2 if wl.g_dtype == "bf16" else 4
     ctx = twa.twa_create(env.local)
     wbar = torch.empty(D, dtype=torch.float32, device=dev)
@@ -789,8 +792,8 @@ def run_layered(args):
     build_ms, quant_ms = max_over_ranks([build_ms, quant_ms], dev)
     if rank == 0:
         peak, peak_kind = load_peaks()
-        sb = step_bytes(D, n, bits, g_bytes)
-        kb = kernel_bytes(D, n, bits, g_bytes)
+        sb = step_bytes(D, n, slot, g_bytes)
+        kb = kernel_bytes(D, n, slot, g_bytes)
         stats = series_stats(series)
         ms_per_step = stats["mean"]
         value = whole_job_gbps(world, sb, ms_per_step)
@@ -805,7 +808,8 @@ def run_layered(args):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": f"{wl.name}: D={D} n={n} L={L} layers, per-layer affine int{bits} P, "
                                    f"{wl.g_dtype} g, lr={LR} lambda={LAM}",
-                       "l2": f"inputs larger than L2: P~ is {n * ((D * bits + 7) // 8) / 1e6:.0f} MB per pass",
+                       "l2": f"inputs larger than L2: P~ is {n * ((D * slot + 7) // 8) / 1e6:.0f} MB per pass "
+                             f"({slot} bits of device memory per code)",
                        "gradients": f"{len(pool)} distinct gradients generated before the timed region, cycled",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "bytes_per_step": sb,
@@ -902,7 +906,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vitb16")
-    ap.add_argument("--bits", type=int, default=8, choices=[32, 8, 4])
+    ap.add_argument("--bits", type=int, default=8, choices=[32, 16, 8, 4, 3, 2, 1],
+                    help="storage width of P: 32 / 8 / 4 for the per-column path; the layer-wise path (--layered)\n"
+                         "takes every width of the paper's ablation: 16, 8, 4, 3, 2, 1")
     ap.add_argument("--g-pool", type=int, default=8)
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--min-timed-ms", type=float, default=1000.0,
@@ -929,6 +935,8 @@ def main():
     args = ap.parse_args()
     if args.steps < 1:
         raise SystemExit("--steps must be at least 1")
+    if args.bits in (16, 3, 2, 1) and not (args.layered and args.impl == "ours"):
+        raise SystemExit("widths 16, 3, 2 and 1 exist for the layer-wise construction only: add --layered")
     if args.project_batch and args.impl == "ours":
         run_project_batch(args)
     elif args.layered and args.impl == "ours":

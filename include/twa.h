@@ -314,12 +314,17 @@ int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host /* host *
  * A layered basis stores P~^l = a^l * code + b^l with unsigned B-bit codes and one (a^l, b^l)
  * pair per layer (Section 4.6: a^l = (max P^l - min P^l) / (2^B - 1), b^l = min P^l, code =
  * round((P - b^l) / a^l); here with float32 subtraction and division and round-half-to-even).
- * The codes use the same column-major chunk-permuted bytes as twa_basis, except that every layer
- * starts on a 64-byte granule of the column; `granules` maps each granule back to {layer, valid
- * rows, first flat row, 0}.  All pointers are device pointers into the one buffer `mem` the
- * caller passed to twa_quantize_affine. */
+ * B is 1, 2, 3, 4, 8 or 16, the widths of the paper's ablation on quantisation bits (Section 5.5).
+ * A code occupies a slot of 1, 2, 4 or 8 bits of a column byte (3-bit codes sit in 4-bit slots;
+ * with S slots per byte, row S k + s of a column is in bits [s * slot, (s+1) * slot) of byte k);
+ * 16-bit codes are stored as two 8-bit planes, the high bytes in columns 0..n-1 and the low bytes
+ * in columns n..2n-1 of `codes` (so n <= 64 there).  Device memory per candidate and row: the slot
+ * width, i.e. B bits except for B = 3 (4 bits).  The columns use the same column-major
+ * chunk-permuted bytes as twa_basis, except that every layer starts on a 64-byte granule of the
+ * column; `granules` maps each granule back to {layer, valid rows, first flat row, 0}.  All
+ * pointers are device pointers into the one buffer `mem` the caller passed to twa_quantize_affine. */
 typedef struct {
-  twa_basis codes;            /* D = padded rows, bits 8 or 4, scales == NULL                  */
+  twa_basis codes;            /* D = padded rows, bits = slot width 8, 4, 2 or 1, scales == NULL */
   float* a;                   /* L scaling factors                                              */
   float* b;                   /* L zero factors                                                 */
   int32_t* granules;          /* 4 ints per 64-byte granule of a column                         */
@@ -334,6 +339,9 @@ typedef struct {
   int32_t cta_count, kt, tiles, tiles_per_cta, total_runs;
   int32_t* cta_first_layer;   /* cta_count ints                                                 */
   int32_t* cta_run_base;      /* cta_count + 1 ints                                             */
+  int32_t code_bits;          /* B of the quantiser: 1, 2, 3, 4, 8 or 16 (codes.bits is the slot) */
+  int32_t planes;             /* 1, or 2 for B = 16: codes.n = 2 n, columns 0..n-1 the high     */
+                              /* bytes of the codes, columns n..2n-1 the low bytes              */
 } twa_layered_basis;
 
 /* Scratch for the two construction calls below (device, 16-byte aligned). */
@@ -351,7 +359,8 @@ int twa_build_centered(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw,
                        const int64_t* offsets_host, int L, float* wbar_out, twa_basis* P32_out,
                        void* lws, size_t lws_bytes);
 
-/* Per-layer min-max quantisation of a float32 basis (Section 4.6), bits 8 or 4.
+/* Per-layer min-max quantisation of a float32 basis (Section 4.6), bits = B in {1, 2, 3, 4, 8, 16}
+ * (P32->n <= 64 for B = 16).
  *  mem  device buffer of twa_layered_basis_bytes, 256-byte aligned; *out points into it.
  * Device-side error: TWA_ERR_NONFINITE (detail = layer). */
 int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offsets_host, int L,
@@ -382,8 +391,10 @@ int twa_layered_build_feed(twa_ctx* ctx, const twa_layered_basis* lb, const int6
 int twa_layered_build_end_pass(twa_ctx* ctx, const twa_layered_basis* lb, const int64_t* offsets_host,
                                int pass, void* lws, size_t lws_bytes);
 
-/* Canonical image for parity checks: unsigned codes in flat row order, n x ceil(D*bits/8) bytes
- * (4 bits: row 2k low nibble, row 2k+1 high nibble), and the L factors a, b.  Device pointers. */
+/* Canonical image for parity checks and checkpoints: unsigned codes in flat row order, n rows of
+ * ceil(D*slot/8) bytes (slot = 1, 2, 4, 8 as above: row S k + s in bits [s*slot, (s+1)*slot) of byte
+ * k; B = 3 uses 4-bit slots, so its image has D/2 bytes per candidate; B = 16: 2 D bytes per
+ * candidate, low byte first), and the L factors a, b.  Device pointers. */
 int twa_layered_export(twa_ctx* ctx, const twa_layered_basis* lb, void* codes_out, float* a_out,
                        float* b_out);
 

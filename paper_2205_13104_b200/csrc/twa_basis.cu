@@ -367,7 +367,7 @@ int twa_launch_scales(twa_ctx* ctx, const unsigned* absmax, int n, int bits, flo
 extern "C" {
 
 int64_t twa_basis_col_stride(int64_t D, int bits) {
-  if (D < 1 || (bits != 32 && bits != 8 && bits != 4)) return 0;
+  if (D < 1 || (bits != 32 && bits != 8 && bits != 4 && bits != 2 && bits != 1)) return 0;
   const int64_t row_bytes = (D * bits + 7) / 8;
   if (bits == 32) return (row_bytes + 127) / 128 * 128;
   return (row_bytes + 511) / 512 * 512;      // whole 512-byte segments: see twa_chunk_slot

@@ -22,6 +22,20 @@ constexpr long long ITEM_ROWS = 8192;       // rows of one layer handled by one 
 struct Item { int layer; long long r0, r1; };   // flat rows [r0, r1) of one layer
 
 long long granule_rows(int bits) { return 64LL * 8 / bits; }
+// Code width B of the quantiser (Section 4.6) -> width of the slot a code occupies in the stored
+// columns, and the number of byte planes: 3-bit codes sit in 4-bit slots; 16-bit codes are two 8-bit
+// planes (columns 0..n-1 hold the high bytes, n..2n-1 the low bytes).  0 = width not supported.
+int slot_bits(int code_bits) {
+  switch (code_bits) {
+    case 1: return 1;
+    case 2: return 2;
+    case 3: case 4: return 4;
+    case 8: case 16: return 8;
+    default: return 0;
+  }
+}
+int plane_count(int code_bits) { return code_bits == 16 ? 2 : 1; }
+float top_code(int code_bits) { return static_cast<float>((1 << code_bits) - 1); }
 constexpr size_t TABLE_SLACK = 8;                           // granule entries past the last column byte
 constexpr int MAX_CTAS = 1024;                              // blocks of a step kernel
 constexpr size_t CTA_TABLE_BYTES = (sizeof(int) * (MAX_CTAS + 1) + 255) / 256 * 256;
@@ -171,41 +185,55 @@ __global__ void factors_kernel(const float* __restrict__ pmin, const float* __re
   b[l] = lo;
 }
 
-// One thread writes one 16-byte chunk of one column: 16 rows (8-bit) or 32 rows (4-bit) of a layer,
-// rows past the layer's end get the code 0.
-template <int BITS>
+// Puts code u (k-th of a 16-byte chunk, slots of W bits) into the chunk's words.
+template <int W>
+__device__ __forceinline__ void put_code(uint32_t (&w)[4], int k, uint32_t u) {
+  constexpr int PER_WORD = 32 / W;
+  w[k / PER_WORD] |= u << (W * (k % PER_WORD));
+}
+
+// One thread writes one 16-byte chunk of one column: 128 / W rows of a layer (W = slot width), rows
+// past the layer's end get the code 0.  PLANES == 2 (16-bit codes): the chunk of the high bytes goes
+// to column j, that of the low bytes to column n + j.
+template <int W, int PLANES>
 __global__ void __launch_bounds__(BLOCK) affine_encode_kernel(const float* __restrict__ P, long long ld,
                                                               const long long* __restrict__ flat,
                                                               const long long* __restrict__ internal,
                                                               const float* __restrict__ a,
-                                                              const float* __restrict__ b,
+                                                              const float* __restrict__ b, float top, int n,
                                                               unsigned char* __restrict__ out,
                                                               long long out_stride) {
-  constexpr int RPC = 128 / BITS;
-  constexpr float TOP = BITS == 8 ? 255.0f : 15.0f;
+  constexpr int RPC = 128 / W;
   const int l = blockIdx.z, j = blockIdx.y;
   const long long len = flat[l + 1] - flat[l];
   const long long chunks = (internal[l + 1] - internal[l]) / RPC;
   const float al = a[l], bl = b[l];
   const float* col = P + j * ld + flat[l];
   uint4* dst = reinterpret_cast<uint4*>(out + j * out_stride);
+  uint4* dst_lo = reinterpret_cast<uint4*>(out + (static_cast<long long>(n) + j) * out_stride);
   for (long long c = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; c < chunks;
        c += static_cast<long long>(gridDim.x) * BLOCK) {
-    uint32_t w[4] = {0, 0, 0, 0};
+    uint32_t w[4] = {0, 0, 0, 0}, wl[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int k = 0; k < RPC; ++k) {
       const long long r = c * RPC + k;
       uint32_t u = 0;
       if (r < len && al != 0.0f) {
         float q = rintf(__fdiv_rn(__fsub_rn(col[r], bl), al));
-        q = fminf(fmaxf(q, 0.0f), TOP);
+        q = fminf(fmaxf(q, 0.0f), top);
         u = static_cast<uint32_t>(q);
       }
-      if (BITS == 8) w[k >> 2] |= u << (8 * (k & 3));
-      else w[k >> 3] |= u << (4 * (k & 7));
+      if (PLANES == 2) {
+        put_code<W>(w, k, u >> 8);
+        put_code<W>(wl, k, u & 0xFFu);
+      } else {
+        put_code<W>(w, k, u);
+      }
     }
     const long long q = internal[l] / RPC + c;
     dst[(q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j)] = make_uint4(w[0], w[1], w[2], w[3]);
+    if (PLANES == 2)
+      dst_lo[(q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), n + j)] = make_uint4(wl[0], wl[1], wl[2], wl[3]);
   }
 }
 
@@ -286,7 +314,7 @@ __global__ void fill_kernel(float* p, size_t count, float v) {
 
 // Codes of the chunk's rows.  A 16-byte group of codes (16 or 32 rows counted from the layer's first
 // row) may straddle two chunks: the storage starts as zeros and every call ORs its rows in.
-template <int BITS>
+template <int W, int PLANES>
 __global__ void __launch_bounds__(BLOCK) chunk_affine_encode_kernel(const float* __restrict__ chunk, long long ld,
                                                                     long long row0, long long row1,
                                                                     const float* __restrict__ wbar,
@@ -294,11 +322,10 @@ __global__ void __launch_bounds__(BLOCK) chunk_affine_encode_kernel(const float*
                                                                     const long long* __restrict__ flat,
                                                                     const long long* __restrict__ internal,
                                                                     const float* __restrict__ a,
-                                                                    const float* __restrict__ b,
+                                                                    const float* __restrict__ b, float top,
                                                                     unsigned char* __restrict__ out,
                                                                     long long out_stride, int first_layer) {
-  constexpr int RPC = 128 / BITS;
-  constexpr float TOP = BITS == 8 ? 255.0f : 15.0f;
+  constexpr int RPC = 128 / W;
   const int l = first_layer + blockIdx.z, j = blockIdx.y;
   const long long lay0 = flat[l], lay1 = flat[l + 1];
   const long long f0 = (lay0 > row0 ? lay0 : row0) - lay0, f1 = (lay1 < row1 ? lay1 : row1) - lay0;   // rows of the layer
@@ -309,9 +336,10 @@ __global__ void __launch_bounds__(BLOCK) chunk_affine_encode_kernel(const float*
   const float* col = chunk + j * ld - row0 + lay0;
   const float* wb = wbar + lay0;
   uint4* dst = reinterpret_cast<uint4*>(out + j * out_stride);
+  uint4* dst_lo = reinterpret_cast<uint4*>(out + (static_cast<long long>(n) + j) * out_stride);
   for (long long c = c0 + blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; c < c1;
        c += static_cast<long long>(gridDim.x) * BLOCK) {
-    uint32_t w[4] = {0, 0, 0, 0};
+    uint32_t w[4] = {0, 0, 0, 0}, wl[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int k = 0; k < RPC; ++k) {
       const long long r = c * RPC + k;
@@ -319,17 +347,27 @@ __global__ void __launch_bounds__(BLOCK) chunk_affine_encode_kernel(const float*
       if (r >= f0 && r < f1 && al != 0.0f) {
         const float e = static_cast<float>((static_cast<double>(col[r]) - static_cast<double>(wb[r])) * f);
         float q = rintf(__fdiv_rn(__fsub_rn(e, bl), al));
-        q = fminf(fmaxf(q, 0.0f), TOP);
+        q = fminf(fmaxf(q, 0.0f), top);
         u = static_cast<uint32_t>(q);
       }
-      if (BITS == 8) w[k >> 2] |= u << (8 * (k & 3));
-      else w[k >> 3] |= u << (4 * (k & 7));
+      if (PLANES == 2) {
+        put_code<W>(w, k, u >> 8);
+        put_code<W>(wl, k, u & 0xFFu);
+      } else {
+        put_code<W>(w, k, u);
+      }
     }
     const long long q = internal[l] / RPC + c;
     uint4* at = dst + ((q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j));
     uint4 old = *at;
     old.x |= w[0]; old.y |= w[1]; old.z |= w[2]; old.w |= w[3];
     *at = old;
+    if (PLANES == 2) {
+      at = dst_lo + ((q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), n + j));
+      old = *at;
+      old.x |= wl[0]; old.y |= wl[1]; old.z |= wl[2]; old.w |= wl[3];
+      *at = old;
+    }
   }
 }
 
@@ -343,23 +381,29 @@ __global__ void tail_zero_kernel(unsigned char* out, long long out_stride, long 
     dst[(q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j)] = make_uint4(0, 0, 0, 0);
 }
 
-// canonical image for parity: unsigned codes in flat row order, n x ceil(D*bits/8) bytes
-template <int BITS>
+// Canonical image for parity and checkpoints: unsigned codes in flat row order, one row of bytes per
+// candidate; slots of W bits, row (8/W) k + s of a column in bits [s W, (s+1) W) of byte k.  PLANES == 2
+// (16-bit codes): two bytes per row, low byte first, from the low-byte column n + j and the high-byte
+// column j.
+template <int W, int PLANES>
 __global__ void __launch_bounds__(BLOCK) layered_export_kernel(const unsigned char* __restrict__ in,
                                                                long long in_stride,
                                                                const long long* __restrict__ flat,
                                                                const long long* __restrict__ internal, int L,
-                                                               long long D, unsigned char* __restrict__ out,
+                                                               long long D, int n, unsigned char* __restrict__ out,
                                                                long long row_bytes) {
+  constexpr int PER = 8 / W;
   const int j = blockIdx.y;
-  const unsigned char* src = in + j * in_stride;
   unsigned char* dst = out + j * row_bytes;
   for (long long ob = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; ob < row_bytes;
        ob += static_cast<long long>(gridDim.x) * BLOCK) {
+    // PLANES == 2: output byte ob is the low (ob even) or high (ob odd) byte of row ob / 2
+    const int col = PLANES == 2 ? ((ob & 1) ? j : n + j) : j;
+    const unsigned char* src = in + col * in_stride;
     unsigned v = 0;
 #pragma unroll
-    for (int h = 0; h < 8 / BITS; ++h) {
-      const long long r = ob * (8 / BITS) + h;
+    for (int h = 0; h < PER; ++h) {
+      const long long r = PLANES == 2 ? (ob >> 1) : ob * PER + h;
       if (r >= D) break;
       int lo = 0, hi = L;                       // layer of flat row r: last l with flat[l] <= r
       while (hi - lo > 1) {
@@ -367,11 +411,11 @@ __global__ void __launch_bounds__(BLOCK) layered_export_kernel(const unsigned ch
         if (flat[mid] <= r) lo = mid; else hi = mid;
       }
       const long long ir = internal[lo] + (r - flat[lo]);
-      const long long ib = ir * BITS / 8;
+      const long long ib = ir * W / 8;
       const long long q = ib >> 4;
-      const unsigned char byte = src[(((q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j)) << 4) | (ib & 15)];
-      const unsigned code = BITS == 8 ? byte : ((byte >> (4 * (ir & 1))) & 0xF);
-      v |= code << (BITS == 8 ? 0 : 4 * h);
+      const unsigned char byte = src[(((q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), col)) << 4) | (ib & 15)];
+      const unsigned code = (byte >> (W * (ir % PER))) & ((1u << W) - 1u);
+      v |= code << (W * h);
     }
     dst[ob] = static_cast<unsigned char>(v);
   }
@@ -417,10 +461,12 @@ size_t count_items(const int64_t* offsets, int L) {
 
 // Carves the caller's buffer of a layered basis (codes | a | b | granule table | flat offsets |
 // internal offsets | block tables), builds and uploads the tables, and fills the descriptor.
-int prepare_layered_storage(twa_ctx* ctx, const Partition& p, long long D, int L, int n, int bits, void* mem,
-                            twa_layered_basis* out) {
+int prepare_layered_storage(twa_ctx* ctx, const Partition& p, long long D, int L, int n_cand, int code_bits,
+                            void* mem, twa_layered_basis* out) {
   // carve the caller's buffer: codes | a | b | granule table | flat offsets | internal offsets
   char* m = static_cast<char*>(mem);
+  const int bits = slot_bits(code_bits), planes = plane_count(code_bits);
+  const int n = n_cand * planes;                       // stored columns
   const long long stride = twa_basis_col_stride(p.D_int, bits);
   const size_t codes_bytes = static_cast<size_t>(stride) * n;
   const size_t fl = (sizeof(float) * L + 255) / 256 * 256;
@@ -436,8 +482,10 @@ int prepare_layered_storage(twa_ctx* ctx, const Partition& p, long long D, int L
   int* d_cta_base = reinterpret_cast<int*>(m + o);
 
   // work split of the step kernels: contiguous tile ranges, and the layers each range meets
-  const int kt = (ctx->tune_tile_segments == 1 || ctx->tune_tile_segments == 2) ? ctx->tune_tile_segments
-                                                                                : (n <= 64 ? 2 : 1);
+  // (slots below 4 bits: one segment per tile -- a tile of 1-bit codes already covers 4096 rows)
+  const int kt = bits < 4 ? 1
+                          : ((ctx->tune_tile_segments == 1 || ctx->tune_tile_segments == 2) ? ctx->tune_tile_segments
+                                                                                           : (n <= 64 ? 2 : 1));
   const long long tile_rows = 512LL * 8 / bits * kt;
   const int tiles = static_cast<int>((p.D_int + tile_rows - 1) / tile_rows);
   int ctas = ctx->sm_count < tiles ? ctx->sm_count : tiles;
@@ -495,6 +543,8 @@ int prepare_layered_storage(twa_ctx* ctx, const Partition& p, long long D, int L
   out->internal_offsets = reinterpret_cast<int64_t*>(d_int);
   out->D = D;
   out->L = L;
+  out->code_bits = code_bits;
+  out->planes = planes;
   out->cta_count = ctas;
   out->kt = kt;
   out->tiles = tiles;
@@ -515,8 +565,8 @@ size_t twa_layered_workspace_bytes(const int64_t* offsets_host, int L, int n) {
 }
 
 int64_t twa_layered_rows(const int64_t* offsets_host, int L, int bits) {
-  if (!offsets_host || L < 1 || (bits != 8 && bits != 4)) return 0;
-  const long long gr = granule_rows(bits);
+  if (!offsets_host || L < 1 || slot_bits(bits) == 0) return 0;
+  const long long gr = granule_rows(slot_bits(bits));
   long long io = 0;
   for (int l = 0; l < L; ++l) io += (offsets_host[l + 1] - offsets_host[l] + gr - 1) / gr * gr;
   return io;
@@ -525,8 +575,9 @@ int64_t twa_layered_rows(const int64_t* offsets_host, int L, int bits) {
 size_t twa_layered_basis_bytes(const int64_t* offsets_host, int L, int n, int bits) {
   const int64_t rows = twa_layered_rows(offsets_host, L, bits);
   if (rows < 1 || n < 1) return 0;
-  const size_t codes = twa_basis_bytes(rows, n, bits);
-  const size_t granules = static_cast<size_t>(twa_basis_col_stride(rows, bits) / 64);
+  const int w = slot_bits(bits);
+  const size_t codes = twa_basis_bytes(rows, n * plane_count(bits), w);
+  const size_t granules = static_cast<size_t>(twa_basis_col_stride(rows, w) / 64);
   return codes + 256 + 2 * ((sizeof(float) * L + 255) / 256 * 256) + 16 * (granules + TABLE_SLACK) +
          (sizeof(long long) * (L + 1) + 255) / 256 * 256 * 2 + 2 * CTA_TABLE_BYTES;
 }
@@ -566,14 +617,16 @@ int twa_build_centered(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, co
 int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offsets_host, int L, int bits,
                         void* mem, size_t mem_bytes, twa_layered_basis* out, void* lws, size_t lws_bytes) {
   if (!ctx || !P32 || !out || !offsets_host || !mem) return TWA_ERR_INVALID_ARG;
-  if (bits != 8 && bits != 4) return TWA_ERR_UNSUPPORTED;
+  const int wbits = slot_bits(bits), planes = plane_count(bits);
+  if (wbits == 0) return TWA_ERR_UNSUPPORTED;
   int rc = twa_check_basis(P32);
   if (rc) return rc;
   if (P32->bits != 32) return TWA_ERR_INVALID_ARG;
   const long long D = P32->D;
   const int n = P32->n;
+  if (n * planes > TWA_MAX_N) return TWA_ERR_UNSUPPORTED;
   Partition p;
-  rc = make_partition(offsets_host, L, D, bits, &p);
+  rc = make_partition(offsets_host, L, D, wbits, &p);
   if (rc) return rc;
   const LwsLayout w = lws_layout(p.items.size(), L, n);
   if (!lws || lws_bytes < w.total) return TWA_ERR_WORKSPACE;
@@ -599,12 +652,12 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
   const dim3 grid(static_cast<unsigned>(p.items.size()), static_cast<unsigned>(n));
   minmax_kernel<<<grid, BLOCK, 0, ctx->stream>>>(P, ld, items, n, pmin, pmax);
   TWA_CUDA_OK(ctx, cudaGetLastError());
-  factors_kernel<<<(L + 127) / 128, 128, 0, ctx->stream>>>(pmin, pmax, first_item, L, n,
-                                                           bits == 8 ? 255.0f : 15.0f, a, b, ctx->d_status);
+  const float top = top_code(bits);
+  factors_kernel<<<(L + 127) / 128, 128, 0, ctx->stream>>>(pmin, pmax, first_item, L, n, top, a, b, ctx->d_status);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   long long max_len = 0;
   for (int l = 0; l < L; ++l) max_len = std::max(max_len, p.internal[l + 1] - p.internal[l]);
-  const int rpc = 128 / bits;
+  const int rpc = 128 / wbits;
   long long gx = (max_len / rpc + BLOCK - 1) / BLOCK;
   if (gx > 64) gx = 64;
   if (gx < 1) gx = 1;
@@ -613,14 +666,20 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
   unsigned char* codes = static_cast<unsigned char*>(out->codes.data);
   const long long* fl_d = reinterpret_cast<const long long*>(ws + w.flat);
   const long long* in_d = reinterpret_cast<const long long*>(ws + w.internal);
-  if (bits == 8)
-    affine_encode_kernel<8><<<egrid, BLOCK, 0, ctx->stream>>>(P, ld, fl_d, in_d, a, b, codes, stride);
+  if (planes == 2)
+    affine_encode_kernel<8, 2><<<egrid, BLOCK, 0, ctx->stream>>>(P, ld, fl_d, in_d, a, b, top, n, codes, stride);
+  else if (wbits == 8)
+    affine_encode_kernel<8, 1><<<egrid, BLOCK, 0, ctx->stream>>>(P, ld, fl_d, in_d, a, b, top, n, codes, stride);
+  else if (wbits == 4)
+    affine_encode_kernel<4, 1><<<egrid, BLOCK, 0, ctx->stream>>>(P, ld, fl_d, in_d, a, b, top, n, codes, stride);
+  else if (wbits == 2)
+    affine_encode_kernel<2, 1><<<egrid, BLOCK, 0, ctx->stream>>>(P, ld, fl_d, in_d, a, b, top, n, codes, stride);
   else
-    affine_encode_kernel<4><<<egrid, BLOCK, 0, ctx->stream>>>(P, ld, fl_d, in_d, a, b, codes, stride);
+    affine_encode_kernel<1, 1><<<egrid, BLOCK, 0, ctx->stream>>>(P, ld, fl_d, in_d, a, b, top, n, codes, stride);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   const long long total_chunks = stride / 16, first_tail = p.D_int / rpc;
   if (first_tail < total_chunks) {
-    tail_zero_kernel<<<dim3(1, n), 64, 0, ctx->stream>>>(codes, stride, first_tail, total_chunks);
+    tail_zero_kernel<<<dim3(1, n * planes), 64, 0, ctx->stream>>>(codes, stride, first_tail, total_chunks);
     TWA_CUDA_OK(ctx, cudaGetLastError());
   }
   return TWA_OK;
@@ -629,25 +688,24 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
 int twa_layered_export(twa_ctx* ctx, const twa_layered_basis* lb, void* codes_out, float* a_out,
                        float* b_out) {
   if (!ctx || !lb || !codes_out || !a_out || !b_out) return TWA_ERR_INVALID_ARG;
-  if (lb->codes.bits != 8 && lb->codes.bits != 4) return TWA_ERR_UNSUPPORTED;
+  const int bits = lb->codes.bits, planes = lb->planes;
+  if ((bits != 8 && bits != 4 && bits != 2 && bits != 1) || (planes != 1 && planes != 2)) return TWA_ERR_UNSUPPORTED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-  const int bits = lb->codes.bits, n = lb->codes.n;
-  const long long row_bytes = (lb->D * bits + 7) / 8;
+  const int n = lb->codes.n / planes;
+  const long long row_bytes = planes == 2 ? 2 * lb->D : (lb->D * bits + 7) / 8;
   long long gx = (row_bytes + BLOCK * 8 - 1) / (BLOCK * 8);
   if (gx > 1024) gx = 1024;
   const dim3 grid(static_cast<unsigned>(gx), static_cast<unsigned>(n));
-  if (bits == 8)
-    layered_export_kernel<8><<<grid, BLOCK, 0, ctx->stream>>>(
-        static_cast<const unsigned char*>(lb->codes.data), lb->codes.col_stride,
-        reinterpret_cast<const long long*>(lb->flat_offsets),
-        reinterpret_cast<const long long*>(lb->internal_offsets), lb->L, lb->D,
-        static_cast<unsigned char*>(codes_out), row_bytes);
-  else
-    layered_export_kernel<4><<<grid, BLOCK, 0, ctx->stream>>>(
-        static_cast<const unsigned char*>(lb->codes.data), lb->codes.col_stride,
-        reinterpret_cast<const long long*>(lb->flat_offsets),
-        reinterpret_cast<const long long*>(lb->internal_offsets), lb->L, lb->D,
-        static_cast<unsigned char*>(codes_out), row_bytes);
+  const unsigned char* in = static_cast<const unsigned char*>(lb->codes.data);
+  const long long* fl = reinterpret_cast<const long long*>(lb->flat_offsets);
+  const long long* il = reinterpret_cast<const long long*>(lb->internal_offsets);
+  unsigned char* o = static_cast<unsigned char*>(codes_out);
+  const long long st = lb->codes.col_stride;
+  if (planes == 2) layered_export_kernel<8, 2><<<grid, BLOCK, 0, ctx->stream>>>(in, st, fl, il, lb->L, lb->D, n, o, row_bytes);
+  else if (bits == 8) layered_export_kernel<8, 1><<<grid, BLOCK, 0, ctx->stream>>>(in, st, fl, il, lb->L, lb->D, n, o, row_bytes);
+  else if (bits == 4) layered_export_kernel<4, 1><<<grid, BLOCK, 0, ctx->stream>>>(in, st, fl, il, lb->L, lb->D, n, o, row_bytes);
+  else if (bits == 2) layered_export_kernel<2, 1><<<grid, BLOCK, 0, ctx->stream>>>(in, st, fl, il, lb->L, lb->D, n, o, row_bytes);
+  else layered_export_kernel<1, 1><<<grid, BLOCK, 0, ctx->stream>>>(in, st, fl, il, lb->L, lb->D, n, o, row_bytes);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   TWA_CUDA_OK(ctx, cudaMemcpyAsync(a_out, lb->a, sizeof(float) * lb->L, cudaMemcpyDeviceToDevice, ctx->stream));
   TWA_CUDA_OK(ctx, cudaMemcpyAsync(b_out, lb->b, sizeof(float) * lb->L, cudaMemcpyDeviceToDevice, ctx->stream));
@@ -693,11 +751,11 @@ extern "C" {
 int twa_layered_build_begin(twa_ctx* ctx, int64_t D, int n, const int64_t* offsets_host, int L, int bits, void* mem,
                             size_t mem_bytes, twa_layered_basis* out, void* lws, size_t lws_bytes) {
   if (!ctx || !out || !offsets_host || !mem) return TWA_ERR_INVALID_ARG;
-  if (bits != 8 && bits != 4) return TWA_ERR_UNSUPPORTED;
+  if (slot_bits(bits) == 0) return TWA_ERR_UNSUPPORTED;
   if (D < 1 || D >= (1LL << 31) || n < 1) return TWA_ERR_INVALID_ARG;
-  if (n > TWA_MAX_N || L > 65535) return TWA_ERR_UNSUPPORTED;
+  if (n * plane_count(bits) > TWA_MAX_N || L > 65535) return TWA_ERR_UNSUPPORTED;
   Partition p;
-  int rc = make_partition(offsets_host, L, D, bits, &p);
+  int rc = make_partition(offsets_host, L, D, slot_bits(bits), &p);
   if (rc) return rc;
   const LwsLayout w = lws_layout(p.items.size(), L, n);
   if (!lws || lws_bytes < w.total) return TWA_ERR_WORKSPACE;
@@ -714,7 +772,8 @@ int twa_layered_build_begin(twa_ctx* ctx, int64_t D, int n, const int64_t* offse
   fill_kernel<<<64, 256, 0, ctx->stream>>>(reinterpret_cast<float*>(ws + w.pmin), cells, INFINITY);
   fill_kernel<<<64, 256, 0, ctx->stream>>>(reinterpret_cast<float*>(ws + w.pmax), cells, -INFINITY);
   TWA_CUDA_OK(ctx, cudaGetLastError());
-  TWA_CUDA_OK(ctx, cudaMemsetAsync(out->codes.data, 0, static_cast<size_t>(out->codes.col_stride) * n, ctx->stream));
+  TWA_CUDA_OK(ctx, cudaMemsetAsync(out->codes.data, 0, static_cast<size_t>(out->codes.col_stride) * out->codes.n,
+                                   ctx->stream));
   return TWA_OK;
 }
 
@@ -723,7 +782,8 @@ int twa_layered_build_feed(twa_ctx* ctx, const twa_layered_basis* lb, const int6
                            float* q32_out, int64_t ldq, void* lws, size_t lws_bytes) {
   if (!ctx || !lb || !offsets_host || !chunk || !wbar || pass < 0 || pass > 2) return TWA_ERR_INVALID_ARG;
   const long long D = lb->D;
-  const int n = lb->codes.n, L = lb->L, bits = lb->codes.bits;
+  const int planes = lb->planes == 2 ? 2 : 1;
+  const int n = lb->codes.n / planes, L = lb->L, bits = lb->codes.bits;
   if (rows < 1 || row0 < 0 || row0 + rows > D || ld < rows) return TWA_ERR_INVALID_ARG;
   if (q32_out && (pass != 1 || ldq < rows)) return TWA_ERR_INVALID_ARG;
   // the mean of the chunk is written with 16-byte stores at wbar + row0
@@ -758,12 +818,17 @@ int twa_layered_build_feed(twa_ctx* ctx, const twa_layered_basis* lb, const int6
     const long long* fl_d = reinterpret_cast<const long long*>(ws + w.flat);
     const long long* in_d = reinterpret_cast<const long long*>(ws + w.internal);
     unsigned char* codes = static_cast<unsigned char*>(lb->codes.data);
-    if (bits == 8)
-      chunk_affine_encode_kernel<8><<<egrid, BLOCK, 0, ctx->stream>>>(chunk, ld, row0, row1, wbar, inv, n, fl_d, in_d,
-                                                                      lb->a, lb->b, codes, lb->codes.col_stride, l0);
-    else
-      chunk_affine_encode_kernel<4><<<egrid, BLOCK, 0, ctx->stream>>>(chunk, ld, row0, row1, wbar, inv, n, fl_d, in_d,
-                                                                      lb->a, lb->b, codes, lb->codes.col_stride, l0);
+    const float top = top_code(lb->code_bits);
+    const long long st = lb->codes.col_stride;
+#define TWA_CHUNK_ENCODE(W, PL) \
+    chunk_affine_encode_kernel<W, PL><<<egrid, BLOCK, 0, ctx->stream>>>(chunk, ld, row0, row1, wbar, inv, n, fl_d, in_d, \
+                                                                        lb->a, lb->b, top, codes, st, l0)
+    if (planes == 2) TWA_CHUNK_ENCODE(8, 2);
+    else if (bits == 8) TWA_CHUNK_ENCODE(8, 1);
+    else if (bits == 4) TWA_CHUNK_ENCODE(4, 1);
+    else if (bits == 2) TWA_CHUNK_ENCODE(2, 1);
+    else TWA_CHUNK_ENCODE(1, 1);
+#undef TWA_CHUNK_ENCODE
   }
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
@@ -772,7 +837,7 @@ int twa_layered_build_feed(twa_ctx* ctx, const twa_layered_basis* lb, const int6
 int twa_layered_build_end_pass(twa_ctx* ctx, const twa_layered_basis* lb, const int64_t* offsets_host, int pass,
                                void* lws, size_t lws_bytes) {
   if (!ctx || !lb || !offsets_host || pass < 0 || pass > 2) return TWA_ERR_INVALID_ARG;
-  const int n = lb->codes.n, L = lb->L, bits = lb->codes.bits;
+  const int n = lb->codes.n / (lb->planes == 2 ? 2 : 1), L = lb->L;
   const LwsLayout w = lws_layout(count_items(offsets_host, L), L, n);
   if (!lws || lws_bytes < w.total) return TWA_ERR_WORKSPACE;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
@@ -785,7 +850,7 @@ int twa_layered_build_end_pass(twa_ctx* ctx, const twa_layered_basis* lb, const 
   } else if (pass == 1) {
     factors_kernel<<<(L + 127) / 128, 128, 0, ctx->stream>>>(reinterpret_cast<const float*>(ws + w.pmin),
                                                              reinterpret_cast<const float*>(ws + w.pmax), first_item, L, n,
-                                                             bits == 8 ? 255.0f : 15.0f, lb->a, lb->b, ctx->d_status);
+                                                             top_code(lb->code_bits), lb->a, lb->b, ctx->d_status);
   }
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;

@@ -101,6 +101,10 @@ __host__ __device__ constexpr int granule_rows(int bits) { return 64 * 8 / bits;
 __host__ __device__ constexpr int segment_bytes(int bits) { return granule_rows(bits) * 4 + 16; }
 __host__ __device__ constexpr int aux_bytes(int bits, int kt) { return 8 * kt * (16 + segment_bytes(bits)); }
 
+// digit matrices of a projection warp: one per code slot of a byte (at least the two of the shared helpers)
+__host__ __device__ constexpr int digit_sets(int bits) { return 8 / bits < 2 ? 2 : 8 / bits; }
+__host__ __device__ constexpr int digit_scratch(int bits) { return digit_sets(bits) * BYTE_DIGIT_SET; }
+
 constexpr int ENTRY_DEPTH = 16;                                  // tiles the helper reads entries ahead
 constexpr int ENTRY_RING_BYTES = ENTRY_DEPTH * 16 * 16;          // up to 16 granules per tile
 
@@ -273,9 +277,10 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
                                            a.status, a.wait_limit_ns);
     return;
   }
-  unsigned char* digw = smem + a.scratch_off + warp * BYTE_DIGIT_SCRATCH;   // this warp's digit matrices
+  constexpr int SUB = 8 / BITS;                        // codes per byte: one digit matrix each
+  unsigned char* digw = smem + a.scratch_off + warp * digit_scratch(BITS);   // this warp's digit matrices
   constexpr bool FOUR = !GBF16;                        // float32 gradients carry a fourth byte digit
-  byte_digit_init<FOUR>(digw, lane);
+  byte_digit_init<FOUR, digit_sets(BITS)>(digw, lane);
   __syncwarp();
   const uint32_t dig_addr = byte_digit_ldmatrix_addr(digw, lane);
   const int dmult = byte_digit_mult(tig);
@@ -338,23 +343,23 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
     const int4* entries = reinterpret_cast<const int4*>(st + a.aux_off);
     const int4 e = entries[gran_in_tile];
     const unsigned seg_off = tile_is_packed<BITS, KT, GES>(entries, a.g) ? seg_off_packed : seg_off_loose;
-    // the granule's rows of g, staged by the helper; rows past the layer's end hold nothing
-    float g0[KT], g1[KT];
+    // the granule's rows of g, staged by the helper; rows past the layer's end hold nothing.  Lane l
+    // holds the SUB rows behind byte l of the warp's 32-byte block: row SUB * l + s meets code slot s.
+    float gv[KT][SUB];
 #pragma unroll
     for (int u = 0; u < KT; ++u) {
-      const int r = rig0 + u * RB + (BITS == 8 ? lane : 2 * lane);
-      float x0, x1 = 0.0f;
-      if (GBF16) {
-        const unsigned short* gs = reinterpret_cast<const unsigned short*>(st + seg_off) + (e.z & 1);
-        x0 = __uint_as_float(static_cast<uint32_t>(gs[r]) << 16);
-        if (BITS == 4) x1 = __uint_as_float(static_cast<uint32_t>(gs[r + 1]) << 16);
-      } else {
-        const float* gs = reinterpret_cast<const float*>(st + seg_off);
-        x0 = gs[r];
-        if (BITS == 4) x1 = gs[r + 1];
+      const int r = rig0 + u * RB + SUB * lane;
+#pragma unroll
+      for (int q = 0; q < SUB; ++q) {
+        float x;
+        if (GBF16) {
+          const unsigned short* gs = reinterpret_cast<const unsigned short*>(st + seg_off) + (e.z & 1);
+          x = __uint_as_float(static_cast<uint32_t>(gs[r + q]) << 16);
+        } else {
+          x = reinterpret_cast<const float*>(st + seg_off)[r + q];
+        }
+        gv[u][q] = r + q < e.y ? x : 0.0f;
       }
-      g0[u] = r < e.y ? x0 : 0.0f;
-      g1[u] = (BITS == 4 && r + 1 < e.y) ? x1 : 0.0f;
     }
     if (e.x != cur_layer) {
       if (cur_layer >= 0) flush();
@@ -364,11 +369,12 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
       const uint32_t tile_base = twa_smem_u32(st);
       unsigned mb = 0u;
 #pragma unroll
-      for (int u = 0; u < KT; ++u) {
-        mb = max(mb, __float_as_uint(g0[u]) & 0x7FFFFFFFu);
-        if (BITS == 4) mb = max(mb, __float_as_uint(g1[u]) & 0x7FFFFFFFu);
-        gsum += g0[u] + g1[u];
-      }
+      for (int u = 0; u < KT; ++u)
+#pragma unroll
+        for (int q = 0; q < SUB; ++q) {
+          mb = max(mb, __float_as_uint(gv[u][q]) & 0x7FFFFFFFu);
+          gsum += gv[u][q];
+        }
       mb = __reduce_max_sync(0xFFFFFFFFu, mb);
       const ByteDigitScale ds = byte_digit_scale(mb);
       if (ds.bad) bad = true;
@@ -380,32 +386,44 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
         for (int mt = 0; mt < MT; ++mt) c[mt][0] = c[mt][1] = c[mt][2] = c[mt][3] = 0;
 #pragma unroll
         for (int u = 0; u < KT; ++u) {
-          byte_digit_store<FOUR>(digw, 0, lane, g0[u], ds.up);
-          if (BITS == 4) byte_digit_store<FOUR>(digw, 1, lane, g1[u], ds.up);
+#pragma unroll
+          for (int q = 0; q < SUB; ++q) byte_digit_store<FOUR>(digw, q, lane, gv[u][q], ds.up);
           __syncwarp();
-          uint32_t b0, b1, b2 = 0, b3 = 0;
-          if (BITS == 8) {
-            ldmatrix_x2(dig_addr, b0, b1);
+          uint32_t bf[SUB < 2 ? 2 : SUB][2];             // B fragments: digit matrix q meets code slot q
+          if (SUB == 1) {
+            ldmatrix_x2(dig_addr, bf[0][0], bf[0][1]);
           } else {
-            uint32_t bb[4];
-            ldmatrix_x4(dig_addr, bb);
-            b0 = bb[0]; b1 = bb[1]; b2 = bb[2]; b3 = bb[3];   // second matrix pair: the odd rows
+#pragma unroll
+            for (int q = 0; q < SUB / 2; ++q) {
+              uint32_t bb[4];
+              ldmatrix_x4(dig_addr + q * 2 * BYTE_DIGIT_SET, bb);
+              bf[2 * q][0] = bb[0]; bf[2 * q][1] = bb[1]; bf[2 * q + 1][0] = bb[2]; bf[2 * q + 1][1] = bb[3];
+            }
           }
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
             uint32_t r[4];
             ldmatrix_x4(tile_base + aoff[u][mt], r);
             if (BITS == 8) {
-              mma_u8u8(c[mt], r, b0, b1);
-            } else {
+              mma_u8u8(c[mt], r, bf[0][0], bf[0][1]);
+            } else if (BITS == 4) {
               uint32_t ev[4], od[4];
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
                 ev[i] = (r[i] << 4) & 0xF0F0F0F0u;       // even rows: 16 * code, unsigned
                 od[i] = r[i] & 0xF0F0F0F0u;              // odd rows
               }
-              mma_u8u8(c[mt], ev, b0, b1);
-              mma_u8u8(c[mt], od, b2, b3);
+              mma_u8u8(c[mt], ev, bf[0][0], bf[0][1]);
+              mma_u8u8(c[mt], od, bf[1][0], bf[1][1]);
+            } else {
+              constexpr uint32_t MASK = 0x01010101u * ((1u << BITS) - 1u);
+#pragma unroll
+              for (int q = 0; q < SUB; ++q) {            // slot q of every byte: rows SUB * byte + q
+                uint32_t x[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) x[i] = (r[i] >> (BITS * q)) & MASK;
+                mma_u8u8(c[mt], x, bf[q][0], bf[q][1]);
+              }
             }
           }
           __syncwarp();
@@ -428,13 +446,18 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
   if (cur_layer >= 0) flush();
 }
 
-// Digits of the layer's coefficients a^l * beta^l_i on their common scale, and the constant
-// b^l * sum_i beta^l_i.  Called by the first 128 threads of a block; `amax` is shared and zero.
-__device__ __forceinline__ void layer_coefficients(int l, int i, int n, float beta_i, float al, float bl,
+// Digits of the layer's coefficients on their common scale, one per stored column, and the constant
+// b^l * sum_i beta^l_i.  One plane: column i carries a^l beta^l_i.  Two planes (16-bit codes, high
+// bytes in columns 0..n-1, low bytes in n..2n-1): column i carries 256 a^l beta^l_i, column n + i
+// carries a^l beta^l_i.  Called by the first 128 threads of a block; `amax` is shared and zero;
+// beta_row holds the layer's n coefficients.
+__device__ __forceinline__ void layer_coefficients(int l, int i, int n, int planes, float al, float bl,
                                                    const float* beta_row, unsigned* amax,
                                                    unsigned char* __restrict__ dig, int* __restrict__ ebits_out,
                                                    float* __restrict__ konst, int* status) {
-  const float coef = i < n ? beta_i * al : 0.0f;
+  float coef = 0.0f;
+  if (i < n) coef = beta_row[i] * al * (planes == 2 ? 256.0f : 1.0f);
+  else if (planes == 2 && i < 2 * n) coef = beta_row[i - n] * al;
   atomicMax(amax, __float_as_uint(coef) & 0x7FFFFFFFu);
   asm volatile("bar.sync 1, 128;" ::: "memory");
   const unsigned ebits = *amax >> 23;
@@ -460,7 +483,7 @@ constexpr int COMBINE_PARTS = 4;
 // Part p sums a contiguous quarter of the blocks that met the layer; the parts are added in order.
 __global__ void __launch_bounds__(128 * COMBINE_PARTS)
 layered_combine_kernel(const float* __restrict__ partials, const int* __restrict__ cta_first,
-                       const int* __restrict__ cta_base, int ctas, int n, const float* __restrict__ a,
+                       const int* __restrict__ cta_base, int ctas, int n, int planes, const float* __restrict__ a,
                        const float* __restrict__ b, float* c_out, float* beta, float lr, float lambda,
                        const twa_adam_args adam, unsigned char* dig, int* ebits_out, float* konst, int* status) {
   __shared__ int range[2];
@@ -491,7 +514,7 @@ layered_combine_kernel(const float* __restrict__ partials, const int* __restrict
     float v[MMA_WARPS], vg[MMA_WARPS];
 #pragma unroll
     for (int w = 0; w < MMA_WARPS; ++w) {
-      v[w] = i < n ? __ldcg(rows + w * ROW_FLOATS + i) : 0.0f;
+      v[w] = i < n * planes ? __ldcg(rows + w * ROW_FLOATS + i) : 0.0f;
       vg[w] = __ldcg(rows + w * ROW_FLOATS + 128);
     }
 #pragma unroll
@@ -510,6 +533,11 @@ layered_combine_kernel(const float* __restrict__ partials, const int* __restrict
   for (int q = 0; q < COMBINE_PARTS; ++q) {
     S += part_s[q][i];
     Sg += part_g[q];
+  }
+  if (planes == 2) {                                                   // S of candidate i = 256 S_high + S_low
+    part_s[0][i] = S;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (i < n) S = 256.0 * S + part_s[0][n + i];
   }
   float bnew = 0.0f;
   if (i < n) {
@@ -530,20 +558,21 @@ layered_combine_kernel(const float* __restrict__ partials, const int* __restrict
   if (dig) {                                                           // only with beta: the step
     beta_new[i] = bnew;
     asm volatile("bar.sync 1, 128;" ::: "memory");
-    layer_coefficients(l, i, n, bnew, a[l], b[l], beta_new, &amax, dig, ebits_out, konst, status);
+    layer_coefficients(l, i, n, planes, a[l], b[l], beta_new, &amax, dig, ebits_out, konst, status);
   }
 }
 
 // One block (128 threads) per layer: the lift's coefficient digits from given coefficients.
-__global__ void layered_coef_kernel(const float* __restrict__ beta, int n, const float* __restrict__ a,
+__global__ void layered_coef_kernel(const float* __restrict__ beta, int n, int planes, const float* __restrict__ a,
                                     const float* __restrict__ b, unsigned char* __restrict__ dig,
                                     int* __restrict__ ebits_out, float* __restrict__ konst, int* status) {
   __shared__ unsigned amax;
+  __shared__ float row[128];
   const int l = blockIdx.x, i = threadIdx.x;
   if (i == 0) amax = 0u;
+  row[i] = i < n ? beta[static_cast<size_t>(l) * n + i] : 0.0f;
   __syncthreads();
-  const float bi = i < n ? beta[static_cast<size_t>(l) * n + i] : 0.0f;
-  layer_coefficients(l, i, n, bi, a[l], b[l], beta + static_cast<size_t>(l) * n, &amax, dig, ebits_out, konst, status);
+  layer_coefficients(l, i, n, planes, a[l], b[l], row, &amax, dig, ebits_out, konst, status);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -552,7 +581,10 @@ __global__ void __launch_bounds__(L_THREADS, 1)
 layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (twa_smem_u32(smem_raw) & 1023u)) & 1023u);
-  constexpr int LROWS = BITS == 8 ? 2 : 4;
+  constexpr int SUB = 8 / BITS;                        // codes per byte
+  constexpr int LROWS = 2 * SUB;                       // rows a lane finishes per 16-byte chunk
+  constexpr int SG = SUB > 4 ? 4 : SUB;                // code slots handled together (bounds the live registers)
+  constexpr int NG = SUB / SG;
   constexpr int RB = 32 * 8 / BITS;
   twa_smem_header* hdr = reinterpret_cast<twa_smem_header*>(smem);
   unsigned char* ring = smem + TWA_SMEM_HEADER;
@@ -626,8 +658,11 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
         const float2 x = *reinterpret_cast<const float2*>(gs + rrow[u]);
         bv[u][0] = x.x; bv[u][1] = x.y;
       } else {
-        const float4 x = *reinterpret_cast<const float4*>(gs + rrow[u]);
-        bv[u][0] = x.x; bv[u][1] = x.y; bv[u][LROWS - 2] = x.z; bv[u][LROWS - 1] = x.w;
+#pragma unroll
+        for (int v4 = 0; v4 < LROWS / 4; ++v4) {
+          const float4 x = *reinterpret_cast<const float4*>(gs + rrow[u] + 4 * v4);
+          bv[u][4 * v4] = x.x; bv[u][4 * v4 + 1] = x.y; bv[u][4 * v4 + 2] = x.z; bv[u][4 * v4 + 3] = x.w;
+        }
       }
     }
     if (e.x != cur_layer && e.x >= 0) {                  // new layer: its digit fragments and factors
@@ -636,7 +671,7 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
       const float w0 = eb <= 0 ? 0.0f : (eb >= 6 ? __uint_as_float(static_cast<uint32_t>(eb - 5) << 23) : 5.877471754e-39f);
       const float w1 = w0 * 0.0078125f, w2 = w1 * 0.0078125f, w3 = w2 * 0.0078125f;
       wbw = tig == 0 ? w1 : (tig == 1 ? w3 : 0.0f);      // weight of the lower digit of this lane's pair
-      if (BITS == 4) wbw *= 0.0625f;
+      if (BITS == 4) wbw *= 0.0625f;                     // 4-bit codes enter the MMA times 16
       kon = eb < 0 ? __int_as_float(0x7FC00000) : a.konst[cur_layer];
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
@@ -657,60 +692,73 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
 #pragma unroll
       for (int i = 0; i < LROWS; ++i) keep[u][i] = 0.0f;
       if (e.x >= 0) {
-        float v[2][LROWS];                                // per 16-byte chunk of the block
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          int acc0[4], acc1[4];
+        for (int grp = 0; grp < NG; ++grp) {              // code slots grp * SG .. grp * SG + SG - 1 of every byte
+          float v[2][2 * SG];                             // per 16-byte chunk of the block
 #pragma unroll
-          for (int ks = 0; ks < KS; ++ks) {
-            uint32_t r[4];
-            ldmatrix_x4_trans(tile_base + loff[u][ch][ks], r);
-            // the transposing load delivers byte pairs of two columns: regroup to four columns per register
-            const uint32_t af[4] = {__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[0], r[1], 0x7531),
-                                    __byte_perm(r[2], r[3], 0x6420), __byte_perm(r[2], r[3], 0x7531)};
-            if (BITS == 8) {
-              if (ks == 0) mma_u8s8_first(acc0, af, bfrag[ks][0], bfrag[ks][1]);
-              else mma_u8s8(acc0, af, bfrag[ks][0], bfrag[ks][1]);
-            } else {
-              uint32_t ae[4], ao[4];
+          for (int ch = 0; ch < 2; ++ch) {
+            // acc[q]: (c0, c1) row SUB * (2 gid) + slot, (c2, c3) row SUB * (2 gid + 1) + slot
+            int acc[SG][4];
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                ae[i] = (af[i] << 4) & 0xF0F0F0F0u;       // even rows: 16 * code, unsigned
-                ao[i] = af[i] & 0xF0F0F0F0u;              // odd rows
-              }
-              if (ks == 0) {
-                mma_u8s8_first(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
-                mma_u8s8_first(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
+            for (int ks = 0; ks < KS; ++ks) {
+              uint32_t r[4];
+              ldmatrix_x4_trans(tile_base + loff[u][ch][ks], r);
+              // the transposing load delivers byte pairs of two columns: regroup to four columns per register
+              const uint32_t af[4] = {__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[0], r[1], 0x7531),
+                                      __byte_perm(r[2], r[3], 0x6420), __byte_perm(r[2], r[3], 0x7531)};
+              if (BITS == 8) {
+                if (ks == 0) mma_u8s8_first(acc[0], af, bfrag[ks][0], bfrag[ks][1]);
+                else mma_u8s8(acc[0], af, bfrag[ks][0], bfrag[ks][1]);
+              } else if (BITS == 4) {
+                uint32_t ae[4], ao[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  ae[i] = (af[i] << 4) & 0xF0F0F0F0u;     // even rows: 16 * code, unsigned
+                  ao[i] = af[i] & 0xF0F0F0F0u;            // odd rows
+                }
+                if (ks == 0) {
+                  mma_u8s8_first(acc[0], ae, bfrag[ks][0], bfrag[ks][1]);
+                  mma_u8s8_first(acc[SG - 1], ao, bfrag[ks][0], bfrag[ks][1]);
+                } else {
+                  mma_u8s8(acc[0], ae, bfrag[ks][0], bfrag[ks][1]);
+                  mma_u8s8(acc[SG - 1], ao, bfrag[ks][0], bfrag[ks][1]);
+                }
               } else {
-                mma_u8s8(acc0, ae, bfrag[ks][0], bfrag[ks][1]);
-                mma_u8s8(acc1, ao, bfrag[ks][0], bfrag[ks][1]);
+                constexpr uint32_t MASK = 0x01010101u * ((1u << BITS) - 1u);
+#pragma unroll
+                for (int q = 0; q < SG; ++q) {
+                  uint32_t x[4];
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) x[i] = (af[i] >> (BITS * (grp * SG + q))) & MASK;
+                  if (ks == 0) mma_u8s8_first(acc[q], x, bfrag[ks][0], bfrag[ks][1]);
+                  else mma_u8s8(acc[q], x, bfrag[ks][0], bfrag[ks][1]);
+                }
               }
             }
-          }
-          if (BITS == 8) {                                // digit pairs (0,1) in lanes tig = 0, (2,3) in tig = 1
-            v[ch][0] = digit_pair_to_float(acc0[0], acc0[1], wbw);
-            v[ch][1] = digit_pair_to_float(acc0[2], acc0[3], wbw);
-          } else {
-            v[ch][0] = digit_pair_to_float(acc0[0], acc0[1], wbw);
-            v[ch][2] = digit_pair_to_float(acc0[2], acc0[3], wbw);
-            v[ch][1] = digit_pair_to_float(acc1[0], acc1[1], wbw);
-            v[ch][3] = digit_pair_to_float(acc1[2], acc1[3], wbw);
-          }
-        }
-        // lane tig = 0 finishes the rows of chunk 0, lane tig = 1 those of chunk 1: each hands the other
-        // the digit-pair sums it does not keep
+            // digit pairs (0,1) in lanes tig = 0, (2,3) in tig = 1
 #pragma unroll
-        for (int i = 0; i < LROWS; ++i) {
-          const float mine = (tig & 1) ? v[1][i] : v[0][i];
-          const float theirs = (tig & 1) ? v[0][i] : v[1][i];
-          keep[u][i] = mine + __shfl_xor_sync(0xFFFFFFFFu, theirs, 1);
+            for (int q = 0; q < SG; ++q) {
+              v[ch][q] = digit_pair_to_float(acc[q][0], acc[q][1], wbw);
+              v[ch][SG + q] = digit_pair_to_float(acc[q][2], acc[q][3], wbw);
+            }
+          }
+          // lane tig = 0 finishes the rows of chunk 0, lane tig = 1 those of chunk 1: each hands the other
+          // the digit-pair sums it does not keep
+#pragma unroll
+          for (int q = 0; q < 2 * SG; ++q) {
+            const float mine = (tig & 1) ? v[1][q] : v[0][q];
+            const float theirs = (tig & 1) ? v[0][q] : v[1][q];
+            // row inside the lane's LROWS: SUB * (q / SG) + slot
+            keep[u][SUB * (q / SG) + grp * SG + (q % SG)] = mine + __shfl_xor_sync(0xFFFFFFFFu, theirs, 1);
+          }
         }
       }
     }
     __syncwarp();
     if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
     if (e.x >= 0 && tig < 2) {
-      const bool aligned = (e.z & (LROWS - 1)) == 0 && a.out_vector_ok;   // the lane's rows start on a vector boundary
+      constexpr int VW = LROWS < 4 ? LROWS : 4;            // floats per vector store
+      const bool aligned = (e.z & (VW - 1)) == 0 && a.out_vector_ok;      // the lane's rows start on a vector boundary
 #pragma unroll
       for (int u = 0; u < KT; ++u) {
         float* dst = a.out + static_cast<long long>(e.z) + rrow[u];
@@ -718,8 +766,13 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
 #pragma unroll
         for (int i = 0; i < LROWS; ++i) r[i] = bv[u][i] + keep[u][i] + kon;
         if (aligned && rrow[u] + LROWS <= e.y) {
-          if (LROWS == 2) *reinterpret_cast<float2*>(dst) = make_float2(r[0], r[1]);
-          else *reinterpret_cast<float4*>(dst) = make_float4(r[0], r[1], r[LROWS - 2], r[LROWS - 1]);
+          if (LROWS == 2) {
+            *reinterpret_cast<float2*>(dst) = make_float2(r[0], r[1]);
+          } else {
+#pragma unroll
+            for (int v4 = 0; v4 < LROWS / 4; ++v4)
+              *reinterpret_cast<float4*>(dst + 4 * v4) = make_float4(r[4 * v4], r[4 * v4 + 1], r[4 * v4 + 2], r[4 * v4 + 3]);
+          }
         } else {
 #pragma unroll
           for (int i = 0; i < LROWS; ++i)
@@ -770,7 +823,9 @@ StepLayout step_layout(const twa_layered_basis* lb) {
 
 template <int BITS, bool GBF16, int MT>
 int launch_lproject_t(twa_ctx* ctx, const CUtensorMap& mp, const LProjectArgs& a, int kt, int grid, int smem) {
-  auto kern = kt == 2 ? layered_project_kernel<BITS, GBF16, MT, 2> : layered_project_kernel<BITS, GBF16, MT, 1>;
+  // slots below 4 bits are tiled with one segment only
+  auto kern = (BITS >= 4 && kt == 2) ? layered_project_kernel<BITS, GBF16, MT, (BITS >= 4 ? 2 : 1)>
+                                     : layered_project_kernel<BITS, GBF16, MT, 1>;
   static int smem_limit[2][64] = {{0}};
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[kt - 1][ctx->device & 63], smem);
   if (rc) return rc;
@@ -795,7 +850,7 @@ int launch_lproject(twa_ctx* ctx, const CUtensorMap& mp, const LProjectArgs& a, 
 
 template <int BITS, int KS>
 int launch_llift_t(twa_ctx* ctx, const CUtensorMap& mp, const LLiftArgs& a, int kt, int grid, int smem) {
-  auto kern = kt == 2 ? layered_lift_kernel<BITS, KS, 2> : layered_lift_kernel<BITS, KS, 1>;
+  auto kern = (BITS >= 4 && kt == 2) ? layered_lift_kernel<BITS, KS, (BITS >= 4 ? 2 : 1)> : layered_lift_kernel<BITS, KS, 1>;
   static int smem_limit[2][64] = {{0}};
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[kt - 1][ctx->device & 63], smem);
   if (rc) return rc;
@@ -835,11 +890,11 @@ int do_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dty
   a.tx_bytes = static_cast<unsigned>(n) * TWA_TILE_COL_BYTES * kt;
   a.aux_off = a.tx_bytes;
   a.stage_bytes = (a.aux_off + aux_bytes(lb->codes.bits, kt) + 1023) / 1024 * 1024;
-  a.stages = stage_count(ctx, TWA_SMEM_HEADER + MMA_WARPS * BYTE_DIGIT_SCRATCH + ENTRY_RING_BYTES + 1024,
+  a.stages = stage_count(ctx, TWA_SMEM_HEADER + MMA_WARPS * digit_scratch(lb->codes.bits) + ENTRY_RING_BYTES + 1024,
                          static_cast<int>(a.stage_bytes));
   if (a.stages < 2) return TWA_ERR_UNSUPPORTED;
   a.scratch_off = TWA_SMEM_HEADER + static_cast<unsigned>(a.stages) * a.stage_bytes;
-  a.ering_off = a.scratch_off + MMA_WARPS * BYTE_DIGIT_SCRATCH;
+  a.ering_off = a.scratch_off + MMA_WARPS * digit_scratch(lb->codes.bits);
   a.gran = reinterpret_cast<const int4*>(lb->granules);
   a.g = g;
   a.cta_first = lb->cta_first_layer;
@@ -849,15 +904,20 @@ int do_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dty
   a.wait_limit_ns = ctx->wait_limit_ns;
   const int smem = static_cast<int>(a.ering_off) + ENTRY_RING_BYTES + 1024;
   const bool bf16 = g_dtype == TWA_BF16;
-  if (lb->codes.bits == 8)
-    rc = bf16 ? launch_lproject<8, true>(ctx, mp, a, kt, lb->cta_count, smem)
-              : launch_lproject<8, false>(ctx, mp, a, kt, lb->cta_count, smem);
-  else
-    rc = bf16 ? launch_lproject<4, true>(ctx, mp, a, kt, lb->cta_count, smem)
-              : launch_lproject<4, false>(ctx, mp, a, kt, lb->cta_count, smem);
+  switch (lb->codes.bits) {
+    case 8: rc = bf16 ? launch_lproject<8, true>(ctx, mp, a, kt, lb->cta_count, smem)
+                      : launch_lproject<8, false>(ctx, mp, a, kt, lb->cta_count, smem); break;
+    case 4: rc = bf16 ? launch_lproject<4, true>(ctx, mp, a, kt, lb->cta_count, smem)
+                      : launch_lproject<4, false>(ctx, mp, a, kt, lb->cta_count, smem); break;
+    case 2: rc = bf16 ? launch_lproject<2, true>(ctx, mp, a, kt, lb->cta_count, smem)
+                      : launch_lproject<2, false>(ctx, mp, a, kt, lb->cta_count, smem); break;
+    default: rc = bf16 ? launch_lproject<1, true>(ctx, mp, a, kt, lb->cta_count, smem)
+                       : launch_lproject<1, false>(ctx, mp, a, kt, lb->cta_count, smem); break;
+  }
   if (rc) return rc;
+  const int planes = lb->planes == 2 ? 2 : 1;
   layered_combine_kernel<<<lb->L, 128 * COMBINE_PARTS, 0, ctx->stream>>>(
-      a.partials, lb->cta_first_layer, lb->cta_run_base, lb->cta_count, n, lb->a, lb->b, c_out, beta, lr, lambda,
+      a.partials, lb->cta_first_layer, lb->cta_run_base, lb->cta_count, n / planes, planes, lb->a, lb->b, c_out, beta, lr, lambda,
       adam, with_digits ? reinterpret_cast<unsigned char*>(sws + w.dig) : nullptr, reinterpret_cast<int*>(sws + w.ebits),
       reinterpret_cast<float*>(sws + w.konst), ctx->d_status);
   TWA_CUDA_OK(ctx, cudaGetLastError());
@@ -872,7 +932,9 @@ int do_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* beta, const 
   int* ebits = reinterpret_cast<int*>(sws + w.ebits);
   float* konst = reinterpret_cast<float*>(sws + w.konst);
   if (!digits_ready) {
-    layered_coef_kernel<<<lb->L, 128, 0, ctx->stream>>>(beta, n, lb->a, lb->b, dig, ebits, konst, ctx->d_status);
+    const int planes = lb->planes == 2 ? 2 : 1;
+    layered_coef_kernel<<<lb->L, 128, 0, ctx->stream>>>(beta, n / planes, planes, lb->a, lb->b, dig, ebits, konst,
+                                                        ctx->d_status);
     TWA_CUDA_OK(ctx, cudaGetLastError());
   }
   CUtensorMap mp;
@@ -899,16 +961,22 @@ int do_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* beta, const 
   a.status = ctx->d_status;
   a.wait_limit_ns = ctx->wait_limit_ns;
   const int smem = static_cast<int>(a.ering_off) + ENTRY_RING_BYTES + 1024;
-  return lb->codes.bits == 8 ? launch_llift<8>(ctx, mp, a, kt, lb->cta_count, smem)
-                             : launch_llift<4>(ctx, mp, a, kt, lb->cta_count, smem);
+  switch (lb->codes.bits) {
+    case 8: return launch_llift<8>(ctx, mp, a, kt, lb->cta_count, smem);
+    case 4: return launch_llift<4>(ctx, mp, a, kt, lb->cta_count, smem);
+    case 2: return launch_llift<2>(ctx, mp, a, kt, lb->cta_count, smem);
+    default: return launch_llift<1>(ctx, mp, a, kt, lb->cta_count, smem);
+  }
 }
 
 int check_step_args(twa_ctx* ctx, const twa_layered_basis* lb, const void* sws, size_t sws_bytes) {
   if (!ctx || !lb || !lb->codes.data || !lb->a || !lb->b || !lb->granules || !lb->cta_first_layer ||
       !lb->cta_run_base)
     return TWA_ERR_INVALID_ARG;
-  if (lb->codes.bits != 8 && lb->codes.bits != 4) return TWA_ERR_UNSUPPORTED;
-  if (lb->codes.n < 1 || lb->codes.n > TWA_MAX_N || lb->L < 1 || lb->cta_count < 1 || (lb->kt != 1 && lb->kt != 2))
+  const int wb = lb->codes.bits;
+  if (wb != 8 && wb != 4 && wb != 2 && wb != 1) return TWA_ERR_UNSUPPORTED;
+  if (lb->codes.n < 1 || lb->codes.n > TWA_MAX_N || lb->L < 1 || lb->cta_count < 1 || (lb->kt != 1 && lb->kt != 2) ||
+      (wb < 4 && lb->kt != 1) || (lb->planes == 2 && (lb->codes.n & 1)))
     return TWA_ERR_INVALID_ARG;
   if (!sws || sws_bytes < step_layout(lb).total) return TWA_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(sws) & 255) return TWA_ERR_MISALIGNED;

@@ -139,11 +139,11 @@ __device__ __forceinline__ ByteDigitScale byte_digit_scale(unsigned mb) {
 
 // Fills the constant rows of a warp's digit matrices (ones in row 3, and in row 5 with four-byte
 // digits; zeros elsewhere); rows 0-2 (and 4) are rewritten for every block of rows.
-template <bool FOUR>
+template <bool FOUR, int SETS = 2>
 __device__ __forceinline__ void byte_digit_init(unsigned char* digw, int lane) {
   uint32_t* w = reinterpret_cast<uint32_t*>(digw);
 #pragma unroll
-  for (int i = 0; i < BYTE_DIGIT_SCRATCH / 128; ++i) {
+  for (int i = 0; i < SETS * BYTE_DIGIT_SET / 128; ++i) {
     const int idx = lane + 32 * i;                         // word of the scratch
     const int row = (idx % (BYTE_DIGIT_SET / 4)) / (BYTE_DIGIT_STRIDE / 4);
     w[idx] = (row == 3 || (FOUR && row == 5)) ? 0x01010101u : 0u;

@@ -75,7 +75,8 @@ class twa_layered_basis(ctypes.Structure):
                 ("internal_offsets", ctypes.c_void_p), ("D", ctypes.c_int64), ("L", ctypes.c_int32),
                 ("cta_count", ctypes.c_int32), ("kt", ctypes.c_int32), ("tiles", ctypes.c_int32),
                 ("tiles_per_cta", ctypes.c_int32), ("total_runs", ctypes.c_int32),
-                ("cta_first_layer", ctypes.c_void_p), ("cta_run_base", ctypes.c_void_p)]
+                ("cta_first_layer", ctypes.c_void_p), ("cta_run_base", ctypes.c_void_p),
+                ("code_bits", ctypes.c_int32), ("planes", ctypes.c_int32)]
 
 
 class TwaError(RuntimeError):
@@ -524,8 +525,9 @@ class LayeredBasis:
 
     D = property(lambda self: self.desc.D)
     L = property(lambda self: self.desc.L)
-    n = property(lambda self: self.desc.codes.n)
-    bits = property(lambda self: self.desc.codes.bits)
+    n = property(lambda self: self.desc.codes.n // max(1, self.desc.planes))     # candidates
+    bits = property(lambda self: self.desc.code_bits)                            # B of the quantiser
+    slot_bits = property(lambda self: 16 if self.desc.planes == 2 else self.desc.codes.bits)
 
 
 def twa_layered_workspace_bytes(layers, n):
@@ -598,8 +600,9 @@ def twa_layered_build_end_pass(ctx, lb, pass_index, lws):
 
 
 def twa_layered_export(ctx, lb):
-    """Canonical unsigned codes (n, ceil(D*bits/8)) uint8 in flat row order and the factors a, b."""
-    row_bytes = (lb.D * lb.bits + 7) // 8
+    """Canonical unsigned codes (n, ceil(D*slot/8)) uint8 in flat row order (slot = 1, 2, 4, 8 or 16
+    bits per code; 3-bit codes sit in 4-bit slots, 16-bit codes low byte first) and the factors a, b."""
+    row_bytes = (lb.D * lb.slot_bits + 7) // 8
     dev = lb.mem.device
     codes = torch.empty((lb.n, row_bytes), dtype=torch.uint8, device=dev)
     a = torch.empty(lb.L, dtype=torch.float32, device=dev)

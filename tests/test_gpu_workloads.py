@@ -431,16 +431,15 @@ def test_workload_decoder_chunked_build_sampled(env):
 
 # ------------------------------------------------------------------ the layer-wise construction, full size
 def _unpack_rows(packed, r0, r1, bits):
-    """Unsigned codes of flat rows r0..r1-1 (r0 even) from the canonical export, shape (rows, n)."""
-    if bits == 8:
-        return np.asfortranarray(packed[:, r0:r1].cpu().numpy().T)
-    b = packed[:, r0 // 2:(r1 + 1) // 2].cpu().numpy()
-    inter = np.empty((b.shape[0], 2 * b.shape[1]), dtype=np.uint8)
-    inter[:, 0::2], inter[:, 1::2] = b & 0xF, b >> 4
-    return np.asfortranarray(inter[:, :r1 - r0].T)
+    """Unsigned codes of flat rows r0..r1-1 (r0 a multiple of the codes per byte) from the canonical
+    export, shape (rows, n), by the oracle's definition of that image."""
+    slot = orc.SLOT_BITS[bits]
+    assert (r0 * slot) % 8 == 0
+    b = packed[:, r0 * slot // 8:(r1 * slot + 7) // 8].cpu().numpy()
+    return orc.unpack_unsigned(b, r1 - r0, bits)
 
 
-@pytest.mark.parametrize("name,bits_list", [("resnet50", (8,)), ("vitb16", (8, 4))])
+@pytest.mark.parametrize("name,bits_list", [("resnet50", (8, 16)), ("vitb16", (8, 4, 3, 2, 1))])
 def test_workload_layerwise_sampled(env, name, bits_list):
     """The paper's default construction on the workload's own layer partition: per-layer factors
     and sampled codes bit-exact, one layer-wise step checked on sampled layers, columns and rows."""
@@ -474,7 +473,7 @@ def test_workload_layerwise_sampled(env, name, bits_list):
             a_o, b_o = orc.affine_factors(blk, [0, r1 - r0], bits)
             assert (a_h[l], b_h[l]) == (a_o[0], b_o[0])
             codes_o = orc.affine_encode(np.asfortranarray(blk[:, cols]), [0, r1 - r0], a_o, b_o, bits)
-            lo = r0 - (r0 % 2)
+            lo = r0 - (r0 % 8)
             got = _unpack_rows(packed, lo, r1, bits)[r0 - lo:, :]
             np.testing.assert_array_equal(got[:, cols], codes_o)
         # one step from beta = 0
@@ -488,7 +487,7 @@ def test_workload_layerwise_sampled(env, name, bits_list):
         np.testing.assert_allclose(beta_h, -LR * c_h.astype(np.float64), rtol=1e-6, atol=1e-30)
         for l in pick:
             r0, r1 = layers[l], layers[l + 1]
-            lo = r0 - (r0 % 2)
+            lo = r0 - (r0 % 8)
             codes = _unpack_rows(packed, lo, r1, bits)[r0 - lo:, :][:, cols]
             c_o = orc.project_layerwise(codes, [0, r1 - r0], a_h[l:l + 1], b_h[l:l + 1], g_host[r0:r1])
             scale = abs(float(a_h[l])) * (codes.astype(np.float64).T @ np.abs(g_host[r0:r1])) \
@@ -504,7 +503,7 @@ def test_workload_layerwise_sampled(env, name, bits_list):
                 r0, r1 = layers[l], layers[l + 1]
                 span = min(r1 - r0, 3001)
                 for s0 in sorted({r0, r0 + (r1 - r0 - span) // 2, r1 - span}):
-                    lo = s0 - (s0 % 2)
+                    lo = s0 - (s0 % 8)
                     rows_codes = _unpack_rows(packed, lo, s0 + span, bits)[s0 - lo:, :]
                     w_o = orc.lift_layerwise(rows_codes, [0, span], a_h[l:l + 1], b_h[l:l + 1], beta_h[l:l + 1],
                                              None if base is None else base[s0:s0 + span].cpu().numpy())
@@ -598,7 +597,7 @@ def test_workload_decoder_layerwise_chunked_sampled(env, bits):
             r0, r1 = layers[l], layers[l + 1]
             span = min(r1 - r0, 3001)
             for s0 in sorted({r0, r0 + (r1 - r0 - span) // 2, r1 - span}):
-                lo = s0 - (s0 % 2)
+                lo = s0 - (s0 % 8)
                 rows_codes = _unpack_rows(packed, lo, s0 + span, bits)[s0 - lo:, :]
                 w_o = orc.lift_layerwise(rows_codes, [0, span], a_h[l:l + 1], b_h[l:l + 1], beta_h[l:l + 1],
                                          None if base is None else base[s0:s0 + span].cpu().numpy())
