@@ -299,9 +299,16 @@ int twa_weighted_average(twa_ctx* ctx, const float* W, int64_t D, int n, int64_t
                          float* w_out, void* ws, size_t ws_bytes);
 
 /* The same iteration for a caller whose gradient and weights live in HOST memory (pinned
- * memory makes the copies asynchronous): copies g_host (D elements) into the device
- * staging buffer g_stage, runs twa_step into the device buffer w, and copies w back to
- * w_host (D floats).  All three operations are enqueued on the context's stream. */
+ * memory makes the copies asynchronous): g_host (D elements) goes to the device staging
+ * buffer g_stage, the step runs into the device buffer w, and w goes back to w_host (D floats).
+ * From 2^22 rows on the work is cut into up to 16 row chunks so that the three parts overlap:
+ * the projection of a chunk starts when its rows of g have arrived, and every chunk of w leaves
+ * for the host while the next one is lifted; the copies run on a second stream the context
+ * creates at the first such call, ordered with the context's stream by events (work enqueued on
+ * the context's stream after the call starts after the last copy).  The coefficients' gradient
+ * is then the float64 sum of the chunks' projections in chunk order: equal to twa_step's within
+ * the rounding of the float32 partial sums, not bit for bit.  Smaller problems run the three
+ * operations back to back on the context's stream and give twa_step's result exactly. */
 int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host /* host */,
                   twa_dtype g_dtype, float lr, float lambda, float* alpha, const float* wbar,
                   float* w, float* w_host /* host */, void* g_stage, void* ws, size_t ws_bytes);

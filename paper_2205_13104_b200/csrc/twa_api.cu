@@ -35,6 +35,22 @@ __global__ void wait_selftest_kernel(int* status, unsigned long long limit_ns) {
 }
 }  // namespace
 
+namespace {
+// twa_step_host: the coefficients' gradient is the sum of the chunks' projections (float64, chunk
+// order), then the update of Algorithm 1.  One block of TWA_MAX_N threads.
+__global__ void chunk_combine_kernel(const float* __restrict__ chunk_c, int chunks, int n, float* alpha, float lr,
+                                     float lambda, int* status) {
+  const int j = threadIdx.x;
+  double c = 0.0;
+  if (j < n)
+    for (int k = 0; k < chunks; ++k) c += static_cast<double>(chunk_c[static_cast<size_t>(k) * TWA_MAX_N + j]);
+  if (j < n && !isfinite(c)) twa_set_status(status, TWA_ERR_NONFINITE, j);
+  // alpha stays as it was when the projection is unusable (see twa_step)
+  const int unusable = __syncthreads_or(!isfinite(c)) | (__ldcg(status) == TWA_ERR_TIMEOUT);
+  if (j < n && !unusable) alpha[j] = twa_coefficient_update(alpha[j], c, lr, lambda, twa_adam_args{}, j);
+}
+}  // namespace
+
 int twa_adam_device_args(const twa_adam* opt, float* m, float* v, twa_adam_args* out) {
   if (!opt || !m || !v || !out) return TWA_ERR_INVALID_ARG;
   if (opt->step < 1 || !(opt->beta1 >= 0.0f && opt->beta1 < 1.0f) || !(opt->beta2 >= 0.0f && opt->beta2 < 1.0f) ||
@@ -115,6 +131,12 @@ void twa_destroy(twa_ctx* ctx) {
   if (ctx->prof_events) {
     for (int i = 0; i < 3 * ctx->prof_cap; ++i) cudaEventDestroy(ctx->prof_events[i]);
     free(ctx->prof_events);
+  }
+  if (ctx->copy_events) {
+    cudaStreamSynchronize(ctx->copy_stream);
+    for (int i = 0; i < 2 * TWA_HOST_CHUNKS + 2; ++i) cudaEventDestroy(ctx->copy_events[i]);
+    free(ctx->copy_events);
+    cudaStreamDestroy(ctx->copy_stream);
   }
   if (ctx->d_status) cudaFree(ctx->d_status);
   free(ctx);
@@ -313,12 +335,85 @@ int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host, twa_dtyp
   if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
   if (P->D < 1) return TWA_ERR_INVALID_ARG;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-  const size_t gbytes = static_cast<size_t>(P->D) * (g_dtype == TWA_BF16 ? 2 : 4);
-  TWA_CUDA_OK(ctx, cudaMemcpyAsync(g_stage, g_host, gbytes, cudaMemcpyHostToDevice, ctx->stream));
-  int rc = twa_step(ctx, P, g_stage, g_dtype, lr, lambda, alpha, wbar, w, nullptr, ws, ws_bytes);
+  const size_t gsz = g_dtype == TWA_BF16 ? 2 : 4;
+  const long long D = P->D;
+  // Row chunks: multiples of 2^16 rows (whole tiles of every storage width), at most TWA_HOST_CHUNKS.
+  // Below 2^22 rows the copies are too short to be worth splitting.
+  long long chunk_rows = (D + TWA_HOST_CHUNKS - 1) / TWA_HOST_CHUNKS;
+  chunk_rows = (chunk_rows + 65535) / 65536 * 65536;
+  const int chunks = static_cast<int>((D + chunk_rows - 1) / chunk_rows);
+  if (D < (1LL << 22) || chunks < 2) {
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(g_stage, g_host, static_cast<size_t>(D) * gsz, cudaMemcpyHostToDevice, ctx->stream));
+    int rc = twa_step(ctx, P, g_stage, g_dtype, lr, lambda, alpha, wbar, w, nullptr, ws, ws_bytes);
+    if (rc) return rc;
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(w_host, w, static_cast<size_t>(D) * 4, cudaMemcpyDeviceToHost, ctx->stream));
+    return TWA_OK;
+  }
+  if (!alpha || !wbar || !w) return TWA_ERR_INVALID_ARG;
+  int rc = twa_check_basis(P);
   if (rc) return rc;
-  TWA_CUDA_OK(ctx, cudaMemcpyAsync(w_host, w, static_cast<size_t>(P->D) * 4, cudaMemcpyDeviceToHost,
-                                   ctx->stream));
+  rc = check_ws(ws, ws_bytes);
+  if (rc) return rc;
+  if (misaligned16(g_stage) || misaligned16(w) || misaligned16(wbar)) return TWA_ERR_MISALIGNED;
+  if (!ctx->copy_events) {
+    TWA_CUDA_OK(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    const int count = 2 * TWA_HOST_CHUNKS + 2;
+    cudaEvent_t* ev = static_cast<cudaEvent_t*>(calloc(count, sizeof(cudaEvent_t)));
+    if (!ev) return TWA_ERR_INVALID_ARG;
+    for (int i = 0; i < count; ++i) TWA_CUDA_OK(ctx, cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming));
+    ctx->copy_events = ev;
+  }
+  cudaEvent_t* ev_up = ctx->copy_events;                       // gradient chunk k is on the device
+  cudaEvent_t* ev_lift = ctx->copy_events + TWA_HOST_CHUNKS;   // rows of chunk k of w are final
+  cudaEvent_t ev_begin = ctx->copy_events[2 * TWA_HOST_CHUNKS], ev_end = ctx->copy_events[2 * TWA_HOST_CHUNKS + 1];
+  float* chunk_c = reinterpret_cast<float*>(static_cast<char*>(ws) + TWA_WS_CHUNK_COEF);
+  const char* gh = static_cast<const char*>(g_host);
+  char* gs = static_cast<char*>(g_stage);
+  auto view = [&](int k, twa_basis* v, long long* r0) {
+    *r0 = static_cast<long long>(k) * chunk_rows;
+    const long long rows = (*r0 + chunk_rows < D) ? chunk_rows : D - *r0;
+    *v = *P;
+    v->data = static_cast<char*>(P->data) + (*r0 * P->bits) / 8;
+    v->D = rows;
+  };
+  // the copies wait for everything enqueued on the context's stream so far (g_stage and w may be in use)
+  TWA_CUDA_OK(ctx, cudaEventRecord(ev_begin, ctx->stream));
+  TWA_CUDA_OK(ctx, cudaStreamWaitEvent(ctx->copy_stream, ev_begin, 0));
+  for (int k = 0; k < chunks; ++k) {
+    twa_basis v;
+    long long r0;
+    view(k, &v, &r0);
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(gs + r0 * gsz, gh + r0 * gsz, static_cast<size_t>(v.D) * gsz, cudaMemcpyHostToDevice,
+                                     ctx->copy_stream));
+    TWA_CUDA_OK(ctx, cudaEventRecord(ev_up[k], ctx->copy_stream));
+  }
+  // projection of every chunk as soon as its rows of g have arrived
+  for (int k = 0; k < chunks; ++k) {
+    twa_basis v;
+    long long r0;
+    view(k, &v, &r0);
+    TWA_CUDA_OK(ctx, cudaStreamWaitEvent(ctx->stream, ev_up[k], 0));
+    twa_project_epilogue epi = {chunk_c + static_cast<size_t>(k) * TWA_MAX_N, nullptr, 0.0f, 0.0f, -1};
+    rc = twa_launch_project(ctx, &v, gs + r0 * gsz, g_dtype, epi, ws);
+    if (rc) return rc;
+  }
+  chunk_combine_kernel<<<1, TWA_MAX_N, 0, ctx->stream>>>(chunk_c, chunks, P->n, alpha, lr, lambda, ctx->d_status);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  // lift chunk by chunk; every chunk of w leaves for the host while the next one is computed
+  for (int k = 0; k < chunks; ++k) {
+    twa_basis v;
+    long long r0;
+    view(k, &v, &r0);
+    rc = twa_launch_lift(ctx, &v, alpha, 1.0f, wbar + r0, w + r0, false);
+    if (rc) return rc;
+    TWA_CUDA_OK(ctx, cudaEventRecord(ev_lift[k], ctx->stream));
+    TWA_CUDA_OK(ctx, cudaStreamWaitEvent(ctx->copy_stream, ev_lift[k], 0));
+    TWA_CUDA_OK(ctx, cudaMemcpyAsync(w_host + r0, w + r0, static_cast<size_t>(v.D) * 4, cudaMemcpyDeviceToHost,
+                                     ctx->copy_stream));
+  }
+  // later work on the context's stream (and a caller waiting for it) sees w_host complete
+  TWA_CUDA_OK(ctx, cudaEventRecord(ev_end, ctx->copy_stream));
+  TWA_CUDA_OK(ctx, cudaStreamWaitEvent(ctx->stream, ev_end, 0));
   return TWA_OK;
 }
 

@@ -38,6 +38,10 @@ struct twa_ctx {
   int build_n;
   float* build_wbar;
   char* build_ws;
+  // twa_step_host: a second stream for the host copies and the events that order it with `stream`
+  // (created by the first call that needs them)
+  cudaStream_t copy_stream;
+  cudaEvent_t* copy_events;   // 2 * TWA_HOST_CHUNKS + 2
   char last_error[256];
 };
 
@@ -63,7 +67,10 @@ constexpr size_t TWA_WS_NORMS = TWA_WS_COEF + sizeof(float) * TWA_MAX_N;
 constexpr size_t TWA_WS_DPART = TWA_WS_NORMS + 64;       // double [TWA_MAX_GRID] partial sums
 constexpr size_t TWA_WS_ABSMAX = TWA_WS_DPART + sizeof(double) * TWA_MAX_GRID;
                                                          // uint  [TWA_MAX_N]  bit patterns of column absmax
-constexpr size_t TWA_WS_BYTES = TWA_WS_ABSMAX + sizeof(unsigned) * TWA_MAX_N;
+constexpr int TWA_HOST_CHUNKS = 16;                      // row chunks of twa_step_host at most
+constexpr size_t TWA_WS_CHUNK_COEF = TWA_WS_ABSMAX + sizeof(unsigned) * TWA_MAX_N;
+                                                         // float [TWA_HOST_CHUNKS][TWA_MAX_N]  per-chunk projections
+constexpr size_t TWA_WS_BYTES = TWA_WS_CHUNK_COEF + sizeof(float) * TWA_HOST_CHUNKS * TWA_MAX_N;
 
 // ------------------------------------------------------------------------------------------
 // Streaming-kernel geometry

@@ -249,6 +249,49 @@ def test_step_host_matches_device_step(env):
     assert torch.equal(a1, a2) and torch.equal(w1, w2) and torch.equal(w_host, w1.cpu())
 
 
+@pytest.mark.parametrize("bits,gdt", [(8, torch.bfloat16), (4, torch.float32), (32, torch.float32)])
+def test_step_host_in_row_chunks_matches_device_step_and_oracle(env, bits, gdt):
+    """From 2^22 rows on twa_step_host cuts the step into row chunks that overlap with the host copies
+    (a second stream, events): the coefficients are the sum of the chunks' projections, so they agree
+    with twa_step within rounding, w with the oracle's lift of those coefficients; two calls in a row
+    reuse the staging buffer and the events."""
+    ctx, ws = env
+    D, n = (1 << 22) + 70001, 5
+    P = random_basis(D, n, 78)
+    B = twa.basis_from_tensor(P, D)
+    if bits != 32:
+        B = twa.twa_quantize_basis(ctx, B, bits, ws)
+        codes, s = twa.twa_basis_export(ctx, B)
+        co, so = orc.unpack_codes(codes.cpu().numpy(), D, bits), s.cpu().numpy()
+    else:
+        Ph = host_cols(P, D)
+    wbar = torch.randn(D, device=DEV)
+    a_dev = torch.zeros(n, device=DEV)
+    a_host = torch.zeros(n, device=DEV)
+    w_dev = torch.empty(D, device=DEV)
+    w_stage = torch.empty(D, device=DEV)
+    w_host = torch.empty(D, dtype=torch.float32).pin_memory()
+    g_stage = torch.empty(D, dtype=gdt, device=DEV)
+    a_o = np.zeros(n)
+    for t in range(2):
+        g = inputs.gradient(D, 1e-3, 5, t, gdt, DEV)
+        g_pinned = g.cpu().pin_memory()
+        twa.twa_step(ctx, B, g, 0.1, 0.0, a_dev, wbar, w_dev, ws)
+        twa.twa_step_host(ctx, B, g_pinned, 0.1, 0.0, a_host, wbar, w_stage, w_host, g_stage, ws)
+        status_ok(ctx)                                    # waits for the context's stream, hence for the copies
+        gh = g.float().cpu().numpy()
+        if bits != 32:
+            a_o, w_o, _ = orc.step(co, so, gh, a_o, wbar.cpu().numpy(), 0.1)
+        else:
+            a_o, w_o, _ = orc.step_f32(Ph, gh, a_o, wbar.cpu().numpy(), 0.1)
+        assert torch.equal(g_stage, g)
+        assert rel(a_host.cpu().numpy(), a_o) <= TOL
+        assert rel(a_host.cpu().numpy(), a_dev.cpu().numpy()) <= 1e-6
+        assert torch.equal(w_host, w_stage.cpu())
+        assert rel(w_host.numpy(), w_o) <= TOL
+        assert np.max(np.abs(w_host.numpy() - w_o.astype(np.float32))) <= 4 * np.spacing(np.float32(np.abs(w_o).max()))
+
+
 # ------------------------------------------------------------------ basis
 @pytest.mark.parametrize("D,n", [(1, 1), (130, 2), (5003, 3), (70001, 33), (200004, 100), (40001, 128)])
 def test_build_basis(env, D, n):
