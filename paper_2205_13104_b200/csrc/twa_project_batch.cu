@@ -15,13 +15,16 @@
 
 namespace {
 
-constexpr int PAIR_SCRATCH = BYTE_DIGIT_SCRATCH;  // per warp: (even, odd rows) x [8 digit rows][32 gradient rows]
+// Digit matrices of one pair of gradients: [8 digit rows][32 gradient rows]; with 4-bit codes one for
+// the even and one for the odd rows.  A warp keeps one such set per pair of the group.
+__host__ __device__ constexpr int pair_bytes(int bits) { return (bits == 8 ? 1 : 2) * BYTE_DIGIT_SET; }
 
 // Digit matrix of a pair of gradients: rows u0, u1, u2, ones of the first, then of the second.
+template <int BITS>
 __device__ __forceinline__ void pair_digit_init(unsigned char* digw, int lane) {
   uint32_t* w = reinterpret_cast<uint32_t*>(digw);
 #pragma unroll
-  for (int i = 0; i < PAIR_SCRATCH / 128; ++i) {
+  for (int i = 0; i < pair_bytes(BITS) / 128; ++i) {
     const int idx = lane + 32 * i;
     const int row = (idx % (BYTE_DIGIT_SET / 4)) / (BYTE_DIGIT_STRIDE / 4);
     w[idx] = (row & 3) == 3 ? 0x01010101u : 0u;
@@ -110,8 +113,9 @@ twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
   if (warp == MMA_WARPS) {
     if (lane == 0) producer_loop_batch<KT, NB>(hdr, ring, &map_p, &map_g, a, SROWS * KT, GSZ);
   } else {
-    unsigned char* digw = smem + a.scratch_off + warp * PAIR_SCRATCH;
-    pair_digit_init(digw, lane);
+    constexpr int PAIR_BYTES = pair_bytes(BITS);         // digit matrices of one pair of gradients
+    unsigned char* digw = smem + a.scratch_off + warp * PAIR_BYTES;   // reused pair after pair
+    pair_digit_init<BITS>(digw, lane);
     __syncwarp();
     const uint32_t dig_addr = byte_digit_ldmatrix_addr(digw, lane);
     const int dmult = (tig & 1) ? -64 : 256;
@@ -148,83 +152,81 @@ twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
       const uint32_t tile_base = twa_smem_u32(st);
 #pragma unroll
-      for (int p = 0; p < NP; ++p) {
-        // ---- the warp's rows of the pair's two gradients ---------------------------------------
-        float g0[2][KT], g1[2][KT];
-        unsigned mb[2] = {0u, 0u};
+      for (int u = 0; u < KT; ++u) {
+        // ---- digits of the warp's rows of every gradient of the group, one matrix per pair ------
+        float wl[NP];                                    // this lane's weight for pair p (0: nothing to add)
+        uint32_t bf[NP][4];                              // B fragments of every pair
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-          for (int u = 0; u < KT; ++u) {
-            const int e = goff[u] + (2 * p + h) * 256;
-            g1[h][u] = 0.0f;
-            if (GBF16) {
-              const unsigned short* gs = reinterpret_cast<const unsigned short*>(st + a.g_off);
-              g0[h][u] = __uint_as_float(static_cast<uint32_t>(gs[e]) << 16);
-              if (BITS == 4) g1[h][u] = __uint_as_float(static_cast<uint32_t>(gs[e + 1]) << 16);
-            } else {
-              const float* gs = reinterpret_cast<const float*>(st + a.g_off);
-              g0[h][u] = gs[e];
-              if (BITS == 4) g1[h][u] = gs[e + 1];
-            }
-            mb[h] = max(mb[h], max(__float_as_uint(g0[h][u]) & 0x7FFFFFFFu, __float_as_uint(g1[h][u]) & 0x7FFFFFFFu));
-          }
-        mb[0] = __reduce_max_sync(0xFFFFFFFFu, mb[0]);
-        mb[1] = __reduce_max_sync(0xFFFFFFFFu, mb[1]);
-        const ByteDigitScale ds0 = byte_digit_scale(mb[0]), ds1 = byte_digit_scale(mb[1]);
-        if (ds0.bad) bad |= 1u << (2 * p);
-        if (ds1.bad) bad |= 1u << (2 * p + 1);
-        if (!ds0.live && !ds1.live) continue;            // nothing representable in either gradient here
-        // a dead or non-finite gradient is cut with scale 0: its digits are those of zero
-        const float up0 = ds0.live ? ds0.up : 0.0f, up1 = ds1.live ? ds1.up : 0.0f;
-        // lanes tig 0,1 finish the first gradient's digits (columns u0 u1 | u2 ones), tig 2,3 the second's
-        const bool livem = (tig < 2) ? ds0.live : ds1.live;
-        float wl = !livem ? 0.0f : ((tig < 2) ? ds0.w0 : ds1.w0);
-        if (tig & 1) wl *= 65536.0f;
-        if (BITS == 4) wl *= 0.0625f;                    // 4-bit codes enter the MMA times 16
-        int c[MT][4];
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt) c[mt][0] = c[mt][1] = c[mt][2] = c[mt][3] = 0;
-#pragma unroll
-        for (int u = 0; u < KT; ++u) {
+        for (int p = 0; p < NP; ++p) {
+          float g0[2], g1[2];
+          unsigned mb[2];
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
-            pair_digit_store(digw, 0, h, lane, g0[h][u], h ? up1 : up0);
-            if (BITS == 4) pair_digit_store(digw, 1, h, lane, g1[h][u], h ? up1 : up0);
+            const int e = goff[u] + (2 * p + h) * 256;
+            g1[h] = 0.0f;
+            if (GBF16) {
+              const unsigned short* gs = reinterpret_cast<const unsigned short*>(st + a.g_off);
+              g0[h] = __uint_as_float(static_cast<uint32_t>(gs[e]) << 16);
+              if (BITS == 4) g1[h] = __uint_as_float(static_cast<uint32_t>(gs[e + 1]) << 16);
+            } else {
+              const float* gs = reinterpret_cast<const float*>(st + a.g_off);
+              g0[h] = gs[e];
+              if (BITS == 4) g1[h] = gs[e + 1];
+            }
+            mb[h] = max(__float_as_uint(g0[h]) & 0x7FFFFFFFu, __float_as_uint(g1[h]) & 0x7FFFFFFFu);
+          }
+          // one digit scale per gradient for the warp's rows of this 32-byte block
+          mb[0] = __reduce_max_sync(0xFFFFFFFFu, mb[0]);
+          mb[1] = __reduce_max_sync(0xFFFFFFFFu, mb[1]);
+          const ByteDigitScale ds0 = byte_digit_scale(mb[0]), ds1 = byte_digit_scale(mb[1]);
+          if (ds0.bad) bad |= 1u << (2 * p);
+          if (ds1.bad) bad |= 1u << (2 * p + 1);
+          // a dead or non-finite gradient is cut with scale 0: its digits are those of zero
+          const float up0 = ds0.live ? ds0.up : 0.0f, up1 = ds1.live ? ds1.up : 0.0f;
+          // lanes tig 0,1 finish the first gradient's digits (columns u0 u1 | u2 ones), tig 2,3 the second's
+          const bool livem = (tig < 2) ? ds0.live : ds1.live;
+          float w = !livem ? 0.0f : ((tig < 2) ? ds0.w0 : ds1.w0);
+          if (tig & 1) w *= 65536.0f;
+          if (BITS == 4) w *= 0.0625f;                   // 4-bit codes enter the MMA times 16
+          wl[p] = w;
+          pair_digit_store(digw, 0, 0, lane, g0[0], up0);
+          pair_digit_store(digw, 0, 1, lane, g0[1], up1);
+          if (BITS == 4) {
+            pair_digit_store(digw, 1, 0, lane, g1[0], up0);
+            pair_digit_store(digw, 1, 1, lane, g1[1], up1);
           }
           __syncwarp();
-          // B fragment: result columns 0-3 = u0, u1, u2, ones of the first gradient, 4-7 of the second
-          uint32_t b0, b1, b2 = 0, b3 = 0;
+          // B fragments: result columns 0-3 = u0, u1, u2, ones of the pair's first gradient, 4-7 of its second
           if (BITS == 8) {
-            ldmatrix_x2(dig_addr, b0, b1);
+            ldmatrix_x2(dig_addr, bf[p][0], bf[p][1]);
           } else {
             uint32_t bb[4];
             ldmatrix_x4(dig_addr, bb);
-            b0 = bb[0]; b1 = bb[1]; b2 = bb[2]; b3 = bb[3];   // second matrix pair: the odd rows
+            bf[p][0] = bb[0]; bf[p][1] = bb[1]; bf[p][2] = bb[2]; bf[p][3] = bb[3];   // second pair: the odd rows
           }
-#pragma unroll
-          for (int mt = 0; mt < MT; ++mt) {
-            uint32_t r[4];
-            ldmatrix_x4(tile_base + aoff[u][mt], r);
-            if (BITS == 8) {
-              mma_s8u8(c[mt], r, b0, b1);
-            } else {
-              uint32_t e[4], o[4];
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                e[i] = (r[i] << 4) & 0xF0F0F0F0u;         // even rows: 16 * code
-                o[i] = r[i] & 0xF0F0F0F0u;                // odd rows:  16 * code
-              }
-              mma_s8u8(c[mt], e, b0, b1);
-              mma_s8u8(c[mt], o, b2, b3);
-            }
-          }
-          __syncwarp();                                  // the digit matrices are rewritten next
+          __syncwarp();                                  // the digit matrices are rewritten by the next pair
         }
+        // ---- every 16-column group of the tile is loaded (and unpacked) once for all pairs -------
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-          facc[p][mt][0] = fmaf(static_cast<float>(c[mt][0] + dmult * c[mt][1]), wl, facc[p][mt][0]);
-          facc[p][mt][1] = fmaf(static_cast<float>(c[mt][2] + dmult * c[mt][3]), wl, facc[p][mt][1]);
+          uint32_t r[4], o[4];
+          ldmatrix_x4(tile_base + aoff[u][mt], r);
+          if (BITS == 4) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              o[i] = r[i] & 0xF0F0F0F0u;                  // odd rows:  16 * code
+              r[i] = (r[i] << 4) & 0xF0F0F0F0u;           // even rows: 16 * code
+            }
+          }
+#pragma unroll
+          for (int p = 0; p < NP; ++p) {
+            int c[4];
+            mma_s8u8_first(c, r, bf[p][0], bf[p][1]);
+            if (BITS == 4) mma_s8u8(c, o, bf[p][2], bf[p][3]);
+            // digit sums -> float: |sum| < 2^31 (at most 64 rows x 255 x 127 per digit, times 257)
+            facc[p][mt][0] = fmaf(static_cast<float>(c[0] + dmult * c[1]), wl[p], facc[p][mt][0]);
+            facc[p][mt][1] = fmaf(static_cast<float>(c[2] + dmult * c[3]), wl[p], facc[p][mt][1]);
+          }
         }
       }
       __syncwarp();
@@ -370,7 +372,7 @@ int launch_mt(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg, const 
   }
 }
 
-constexpr int FIXED_SMEM = TWA_SMEM_HEADER + MMA_WARPS * PAIR_SCRATCH + 1024;
+int fixed_smem(int bits) { return TWA_SMEM_HEADER + MMA_WARPS * pair_bytes(bits) + 1024; }
 
 unsigned stage_bytes_of(const twa_basis* P, int gsz, int kt, int nb) {
   const unsigned tx = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt + twa_tile_rows(P->bits) * kt * gsz * nb;
@@ -380,7 +382,7 @@ unsigned stage_bytes_of(const twa_basis* P, int gsz, int kt, int nb) {
 // (segments per tile column, gradients per pass) for this basis, gradient type and device
 void pass_shape(const twa_ctx* ctx, const twa_basis* P, int gsz, int* kt, int* nb) {
   const int kt8 = P->n <= 64 ? 2 : 1;
-  const bool fits = (ctx->smem_optin - FIXED_SMEM) / static_cast<int>(stage_bytes_of(P, gsz, kt8, 8)) >= 3;
+  const bool fits = (ctx->smem_optin - fixed_smem(P->bits)) / static_cast<int>(stage_bytes_of(P, gsz, kt8, 8)) >= 3;
   const bool partials_fit = static_cast<size_t>(ctx->sm_count) * 8 * P->n <= static_cast<size_t>(TWA_MAX_GRID) * TWA_MAX_N;
   if (fits && partials_fit) {
     *kt = kt8;
@@ -437,7 +439,7 @@ extern "C" int twa_project_batch(twa_ctx* ctx, const twa_basis* P, const void* G
   a.g_off = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt;
   a.tx_bytes = a.g_off + static_cast<unsigned>(rows * gsz * nb);
   a.stage_bytes = (a.tx_bytes + 1023) / 1024 * 1024;
-  int stages = (ctx->smem_optin - FIXED_SMEM) / static_cast<int>(a.stage_bytes);
+  int stages = (ctx->smem_optin - fixed_smem(P->bits)) / static_cast<int>(a.stage_bytes);
   if (stages > TWA_MAX_STAGES) stages = TWA_MAX_STAGES;
   if (stages < 2) return TWA_ERR_UNSUPPORTED;
   // the ring is reused for the block's [16][NB][128] float sums after the tile loop
@@ -452,7 +454,7 @@ extern "C" int twa_project_batch(twa_ctx* ctx, const twa_basis* P, const void* G
   a.wait_limit_ns = ctx->wait_limit_ns;
   int grid = ctx->sm_count < a.tiles ? ctx->sm_count : a.tiles;
   while (static_cast<size_t>(grid) * nb * P->n > static_cast<size_t>(TWA_MAX_GRID) * TWA_MAX_N) --grid;
-  const int smem = static_cast<int>(a.scratch_off) + MMA_WARPS * PAIR_SCRATCH + 1024;
+  const int smem = static_cast<int>(a.scratch_off) + MMA_WARPS * pair_bytes(P->bits) + 1024;
   for (int b0 = 0; b0 < batch; b0 += nb) {
     a.b0 = b0;
     if (P->bits == 8)
