@@ -31,7 +31,9 @@
  *    synchronises the stream.  After a device-side error the outputs of that
  *    call are unspecified.
  *  - One context per stream; calls on one context must not overlap in time
- *    from several host threads.
+ *    from several host threads.  Different contexts may be driven from different
+ *    threads: the only state they share is a per-process cache of kernel attributes
+ *    (shared-memory limits already raised), kept under a lock.
  *  - Results are run-to-run bit-identical for fixed arguments on one device
  *    model: every reduction is combined in a fixed order, no floating-point
  *    atomics are used.

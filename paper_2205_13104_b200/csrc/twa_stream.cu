@@ -6,6 +6,7 @@
 // shared-memory stages guarded by full/empty mbarriers; the consumer warps dequantise from
 // shared memory and accumulate in float32 registers.  P~ is read exactly once per kernel.
 // Every wait is bounded; a wait that runs out raises the status word and the block leaves.
+#include <mutex>
 #include <stdio.h>
 
 #include "twa_common.cuh"
@@ -549,7 +550,12 @@ int launch_lift_t(twa_ctx* ctx, const CUtensorMap& mp, const LiftArgs& a, int gr
 
 }  // namespace
 
+// The limit is an attribute of the kernel on a device, shared by every context of the process: the
+// value reached so far is cached per kernel and device (`current`), and the cache is read and
+// raised under one lock so that contexts driven from several host threads do not race on it.
 int twa_ensure_smem(twa_ctx* ctx, const void* kernel, int* current, int wanted) {
+  static std::mutex lock;
+  std::lock_guard<std::mutex> guard(lock);
   if (wanted > *current) {
     TWA_CUDA_OK(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, wanted));
     *current = wanted;
