@@ -170,15 +170,15 @@ def unpack_codes(packed, D, bits):
     assert bits == 4
     codes = np.zeros((D, n), dtype=np.int8, order="F")
     for j in range(n):
-        b = packed[j].astype(np.int16)
-        lo = b & 0xF
-        hi = (b >> 4) & 0xF
-        lo = np.where(lo >= 8, lo - 16, lo)
-        hi = np.where(hi >= 8, hi - 16, hi)
-        inter = np.empty(2 * b.size, dtype=np.int16)
+        b = packed[j]
+        lo = (b & 0xF).astype(np.int8)
+        hi = (b >> 4).astype(np.int8)
+        lo = (lo ^ 8) - 8                    # two's-complement nibble -> its value in [-8, 7]
+        hi = (hi ^ 8) - 8
+        inter = np.empty(2 * b.size, dtype=np.int8)
         inter[0::2] = lo
         inter[1::2] = hi
-        codes[:, j] = inter[:D].astype(np.int8)
+        codes[:, j] = inter[:D]
     return codes
 
 
