@@ -598,9 +598,11 @@ def run_ours(args):
     cpu = None
     if with_configs:
         if 4 in bases:
+            s4 = ClockSampler(env.local).start() if rank == 0 else None
             m4 = measure_steps(env, ctx, twa, wl, bases[4], wbar, ws, pool, args.steps, args.warmup,
-                               args.configs_min_ms, None)
-            configs.append(config_entry(wl, 4, m4, peak, build_ms_all, quant_ms.get(4), None))
+                               args.configs_min_ms, s4)
+            c4 = s4.stop().summary(m4["walls"][0][0], m4["walls"][-1][1]) if s4 is not None else None
+            configs.append(config_entry(wl, 4, m4, peak, build_ms_all, quant_ms.get(4), c4))
     # CPU baseline: the oracle on the first rows of THIS basis (rank 0, N = 1 only)
     if rank == 0 and world == 1 and not args.no_cpu_baseline and bits != 32:
         rows = min(D, args.reference_rows)
@@ -702,25 +704,54 @@ def other_configs(env, ctx, twa, inputs, ws, args, peak):
             out.append(config_entry(wl, bits, m, peak, build_ms, quant_ms.get(bits), clocks))
         del bases, wbar, pool
         torch.cuda.empty_cache()
+    # the other modes of the library, each through its own benchmark routine, condensed
+    for name, bits in (("vitb16", 8), ("vitb16", 4), ("decoder1p3b", 4)):
+        line = layered_line(env, args, name, bits, args.configs_min_ms)
+        if line is not None:
+            r = line["roofline"]
+            out.append({"mode": "layer-wise construction, per-layer affine codes (the paper's default; B = 4 its default width)",
+                        "workload": line["config"]["workload"], "bits": bits, "ms_per_step": line["ms_per_step"],
+                        "ms_per_step_median": line["ms_per_step_median"], "repeats": line["repeats"],
+                        "GBps": line["value"], "frac_of_measured_copy_peak": line["frac_of_hbm_peak"],
+                        "frac_of_8TBps": line["frac_of_8TBps"], "bytes_per_step": line["bytes_per_step"],
+                        "project_ms": r["project_ms"], "lift_ms": r["lift_ms"],
+                        "sm_mhz": line["clocks"]["sm_mhz"] if line["clocks"] else None,
+                        "clock_reasons": line["clocks"]["reasons"] if line["clocks"] else None,
+                        "basis_build_ms": line["basis_build_ms"], "quantize_ms": line["quantize_ms"]})
+    if env.world == 1:
+        line = project_batch_line(env, args, "vitb16", 8, 8, args.configs_min_ms)
+        r = line["roofline"]
+        out.append({"mode": "8 gradients per projection (twa_project_batch)", "workload": line["config"]["workload"],
+                    "bits": 8, "ms_per_call": line["ms_per_step"], "gradients_per_s": line["value"],
+                    "GBps": r["achieved"], "frac_of_measured_copy_peak": r["frac"], "frac_of_8TBps": r["achieved"] / 8000.0,
+                    "single_calls_ms": line["single_calls_ms"], "speedup_over_single_calls": line["speedup_over_single_calls"],
+                    "sm_mhz": line["clocks"]["sm_mhz"], "clock_reasons": line["clocks"]["reasons"]})
     return out
 
 
 def run_layered(args):
+    env = Env()
+    line = layered_line(env, args, args.workload, args.bits, args.min_timed_ms)
+    if env.rank == 0:
+        print(json.dumps(line))
+    env.close()
+
+
+def layered_line(env, args, workload, bits, min_timed_ms):
     """The paper's default construction: per-layer centred and normalised basis, per-layer affine
-    B-bit codes, layer-wise step (one coefficient vector per layer)."""
+    B-bit codes, layer-wise step (one coefficient vector per layer).  Returns the JSON line (rank 0)."""
     import torch
     from paper_2205_13104_b200 import inputs, twa
 
-    env = Env()
     dev, world, rank = env.dev, env.world, env.rank
     twa.load()
-    wl = inputs.WORKLOADS[args.workload]
-    if args.bits == 32:
+    wl = inputs.WORKLOADS[workload]
+    if bits == 32:
         raise SystemExit("the layer-wise step runs on quantised codes")
-    layers = inputs.layer_offsets(args.workload, args.rows or None)
+    layers = inputs.layer_offsets(workload, args.rows or None)
     if args.rows:
         wl = dataclasses.replace(wl, name=f"{wl.name}[rows={args.rows}]", D=args.rows)
-    D, n, bits, L = wl.D, wl.n, args.bits, len(layers) - 1
+    D, n, L = wl.D, wl.n, len(layers) - 1
     if bits == 16 and n > 64:
         raise SystemExit("16-bit codes are stored as two 8-bit planes: at most 64 candidates")
     slot = {16: 16, 8: 8, 4: 4, 3: 4, 2: 2, 1: 1}[bits]   # bits of device memory per code
@@ -775,21 +806,22 @@ def run_layered(args):
     sampler = ClockSampler(env.local).start() if rank == 0 else None
     regions, walls = timed_regions(
         env, lambda t: twa.twa_layered_step(ctx, lb, pool[t % len(pool)], LR, LAM, beta, wbar, w, sws),
-        args.steps, args.warmup, args.min_timed_ms)
+        args.steps, args.warmup, min_timed_ms)
     if sampler is not None:
         sampler.stop()
     series = [r / args.steps for r in regions]
     # the two streaming launches apart (each call also runs its small per-layer kernel)
     part_steps = max(1, args.steps // 2)
     pr, _ = timed_regions(env, lambda t: twa.twa_layered_project(ctx, lb, pool[t % len(pool)], c, sws),
-                          part_steps, args.warmup, args.min_timed_ms / 4)
+                          part_steps, args.warmup, min_timed_ms / 4)
     lr_, _ = timed_regions(env, lambda t: twa.twa_layered_lift(ctx, lb, beta, wbar, w, sws),
-                           part_steps, args.warmup, args.min_timed_ms / 4)
+                           part_steps, args.warmup, min_timed_ms / 4)
     proj_ms, lift_ms = sum(pr) / len(pr) / part_steps, sum(lr_) / len(lr_) / part_steps
     code, detail = twa.twa_get_status(ctx)
     if code != 0:
         raise RuntimeError(f"layer-wise step failed: {twa.twa_strerror(code)} layer {detail}")
     build_ms, quant_ms = max_over_ranks([build_ms, quant_ms], dev)
+    line = None
     if rank == 0:
         peak, peak_kind = load_peaks()
         sb = step_bytes(D, n, slot, g_bytes)
@@ -827,24 +859,32 @@ def run_layered(args):
             "gpu_launches": 4 * args.steps * len(series),
             "clocks": clocks,
         }
-        print(json.dumps(line))
     twa.twa_destroy(ctx)
-    env.close()
+    del lb, sws, pool, w, wbar
+    torch.cuda.empty_cache()
+    return line if rank == 0 else None
 
 
 def run_project_batch(args):
-    """Projection of --project-batch gradients per call (P~ read once per group) beside the same
-    number of single-gradient calls, on the workload's column shape; D may be cut with --rows."""
+    env = Env()
+    line = project_batch_line(env, args, args.workload, args.bits, args.project_batch, args.min_timed_ms)
+    if env.rank == 0:
+        print(json.dumps(line))
+    env.close()
+
+
+def project_batch_line(env, args, workload, bits, B, min_timed_ms):
+    """Projection of B gradients per call (P~ read once per group) beside the same number of
+    single-gradient calls, on the workload's column shape; D may be cut with --rows."""
     import torch
     from paper_2205_13104_b200 import inputs, twa
 
-    env = Env()
     dev = env.dev
     twa.load()
-    wl = inputs.WORKLOADS[args.workload]
+    wl = inputs.WORKLOADS[workload]
     if args.rows:
         wl = dataclasses.replace(wl, name=f"{wl.name}[rows={args.rows}]", D=args.rows)
-    D, n, bits, B = wl.D, wl.n, args.bits, args.project_batch
+    D, n = wl.D, wl.n
     gdt = torch.bfloat16 if wl.g_dtype == "bf16" else torch.float32
     g_bytes = 2 if wl.g_dtype == "bf16" else 4
     ctx = twa.twa_create(env.local)
@@ -869,9 +909,9 @@ def run_project_batch(args):
 
     sampler = ClockSampler(env.local).start()
     br, walls = timed_regions(env, lambda _: twa.twa_project_batch(ctx, Pq, G, C, ws), args.steps, args.warmup,
-                              args.min_timed_ms)
+                              min_timed_ms)
     sampler.stop()
-    sr, _ = timed_regions(env, singles, max(1, args.steps // 4), args.warmup, args.min_timed_ms / 4)
+    sr, _ = timed_regions(env, singles, max(1, args.steps // 4), args.warmup, min_timed_ms / 4)
     batch_ms = sum(br) / len(br) / args.steps
     single_ms = sum(sr) / len(sr) / max(1, args.steps // 4)
     code, detail = twa.twa_get_status(ctx)
@@ -881,7 +921,7 @@ def run_project_batch(args):
     p_bytes = n * ((D * bits + 7) // 8)
     moved = -(-B // group) * p_bytes + B * D * g_bytes
     peak, peak_kind = load_peaks()
-    print(json.dumps({
+    line = {
         "metric": f"twa_project_batch_gradients_per_s_int{bits}", "value": B / (batch_ms * 1e-3), "unit": "gradients/s",
         "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": batch_ms, "repeats": len(br),
         "higher_is_better": True,
@@ -894,9 +934,11 @@ def run_project_batch(args):
                      "peak_kind": f"of {peak_kind} (copy bandwidth)", "traffic": None,
                      "bytes_per_launch": moved // -(-B // group)},
         "cpu_baseline": None, "gpu_launches": -(-B // group) * args.steps * len(br),
-        "clocks": sampler.summary(walls[0][0], walls[-1][1])}))
+        "clocks": sampler.summary(walls[0][0], walls[-1][1])}
     twa.twa_destroy(ctx)
-    env.close()
+    del Pq, G, C
+    torch.cuda.empty_cache()
+    return line
 
 
 def main():
