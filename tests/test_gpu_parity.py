@@ -715,3 +715,63 @@ def test_step_keeps_the_coefficients_when_the_gradient_is_not_finite(env):
         twa.twa_step(ctx, B, g, 0.1, 0.0, alpha, wbar, w, ws)
         status_ok(ctx)
         assert torch.equal(alpha, ref)
+
+
+# ------------------------------------------------------------------ the digit cut of the gradient at its limits
+def _digit_cut_bound(co, so, g64, rows_per_block, three_bytes):
+    """Bound of the projection's error from cutting g into byte digits: every value of a warp's block
+    of rows carries an absolute error of at most 2^-23 (three bytes) or 2^-31 (four) of the power of two
+    above the block's largest magnitude, so |delta c_j| <= sum over blocks of that times sum |p~[r, j]|."""
+    D, n = co.shape
+    bound = np.zeros(n)
+    eps = 2.0 ** -23 if three_bytes else 2.0 ** -31
+    absP = np.abs(co.astype(np.float64)) * np.abs(so.astype(np.float64))[None, :]
+    for r0 in range(0, D, rows_per_block):
+        m = np.max(np.abs(g64[r0:r0 + rows_per_block]))
+        if m > 0:
+            bound += eps * 2.0 ** np.ceil(np.log2(m) + 1e-12) * absP[r0:r0 + rows_per_block].sum(axis=0)
+    return bound
+
+
+@pytest.mark.parametrize("kind", ["heavy_tail", "one_outlier_per_block", "tiny", "huge", "ties"])
+@pytest.mark.parametrize("gdt", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("bits", [8, 4])
+def test_projection_digit_cut_on_hard_gradients(env, bits, gdt, kind):
+    """Gradients that stress the block-fixed-point cut: heavy tails (Student t, 1.5 degrees of freedom),
+    one value 2^20 times the rest in every block of rows, magnitudes near the ends of the float range, and
+    values that sit exactly on rounding ties of the cut.  The result stays within the stated relative bound
+    where the coefficients are well conditioned, and always within the bound derived from the cut plus the
+    float32 accumulation term."""
+    ctx, ws = env
+    D, n = 70001, 33
+    P = random_basis(D, n, 303)
+    B = twa.twa_quantize_basis(ctx, twa.basis_from_tensor(P, D), bits, ws)
+    codes, s = twa.twa_basis_export(ctx, B)
+    co, so = orc.unpack_codes(codes.cpu().numpy(), D, bits), s.cpu().numpy()
+    rng = np.random.default_rng(17)
+    if kind == "heavy_tail":
+        g = rng.standard_t(1.5, size=D) * 1e-3
+    elif kind == "one_outlier_per_block":
+        g = rng.standard_normal(D) * 1e-3
+        g[::64] *= 2.0 ** 20
+    elif kind == "tiny":
+        g = rng.standard_normal(D) * 1e-30
+    elif kind == "huge":
+        g = rng.standard_normal(D) * 1e30
+    else:
+        # multiples of 2^-12 with a block maximum of 1023.5: the cut scales them by 2^12 (bfloat16: exact
+        # integers) -- every value is an exact integer or half-integer of the digit grid
+        g = rng.integers(-2048, 2049, size=D) * 2.0 ** -2
+        g[::128] = 1023.5
+    gt = torch.from_numpy(g.astype(np.float32)).to(DEV).to(gdt)
+    g64 = gt.float().cpu().numpy().astype(np.float64)
+    c = torch.empty(n, device=DEV)
+    twa.twa_project(ctx, B, gt, c, ws)
+    status_ok(ctx)
+    c_ref = orc.project(co, so, g64)
+    err = np.abs(c.cpu().numpy().astype(np.float64) - c_ref)
+    # a warp cuts 32 * KT bytes of a column with one scale: at n = 33 (KT = 2) 64 rows at 8 bits, 128 at 4
+    cut = _digit_cut_bound(co, so, g64, 64 * 8 // bits, gdt == torch.bfloat16)
+    accumulate = 4e-6 * (np.abs(co.astype(np.float64)) * np.abs(so.astype(np.float64))[None, :]).T @ np.abs(g64)
+    assert np.all(err <= cut + accumulate + 1e-45)
+    assert rel(c.cpu().numpy(), c_ref) <= TOL
