@@ -184,7 +184,7 @@ int twa_set_tuning(twa_ctx* ctx, int key, int value) {
     case TWA_TUNE_LIFT_WARPS: ctx->tune_lift_warps = value; return TWA_OK;
     case TWA_TUNE_STAGES: ctx->tune_stages = value; return TWA_OK;
     case TWA_TUNE_TILE_SEGMENTS:
-      if (value > 2) return TWA_ERR_INVALID_ARG;
+      if (value == 3 || value > 4) return TWA_ERR_INVALID_ARG;
       ctx->tune_tile_segments = value;
       return TWA_OK;
     case TWA_TUNE_BUILD_PANEL:

@@ -267,7 +267,7 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
 
   if (warp == MMA_WARPS) {
     if (lane == 0)
-      producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, KT, 0, 0,
+      producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, TWA_TILE_COL_WORDS * KT, 0, 0,
                         0, 0, a.tx_bytes, false, a.status, a.wait_limit_ns);
     return;
   }
@@ -596,7 +596,7 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
   const int t_count = (a.tiles - t_first) < a.tpc ? (a.tiles - t_first) : a.tpc;
   if (warp == MMA_WARPS) {
     if (lane == 0)
-      producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, KT, 0, 0,
+      producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, TWA_TILE_COL_WORDS * KT, 0, 0,
                         0, 0, a.tx_bytes, true, a.status, a.wait_limit_ns);
     return;
   }

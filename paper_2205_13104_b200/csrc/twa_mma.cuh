@@ -189,12 +189,13 @@ __device__ __forceinline__ float byte_digit_weight(int tig, float w0) {
 }
 
 // Producer loop: tile k of this block's sequence is t_first + k * t_step (k < t_count); with
-// `reverse` the sequence is walked from its end.  g_boxes 1-D boxes of 256 gradient elements
-// follow the tile of P~ in a stage (project only).
+// `reverse` the sequence is walked from its end; x_per_tile = elements of the codes' tensor map a tile
+// advances along a column.  g_boxes 1-D boxes of 256 gradient elements follow the tile of P~ in a
+// stage (project only).
 __device__ __forceinline__ void producer_loop_mma(twa_smem_header* hdr, unsigned char* ring,
                                                   const CUtensorMap* map_p, const CUtensorMap* map_g,
                                                   int t_first, int t_step, int t_count, int stages,
-                                                  unsigned stage_bytes, int kt, int g_boxes,
+                                                  unsigned stage_bytes, int x_per_tile, int g_boxes,
                                                   int g_elem_bytes, int tile_rows, unsigned g_off,
                                                   unsigned tx_bytes, bool reverse, int* status,
                                                   unsigned long long limit) {
@@ -215,7 +216,7 @@ __device__ __forceinline__ void producer_loop_mma(twa_smem_header* hdr, unsigned
     const uint32_t fb = twa_smem_u32(&hdr->full[s]);
     const uint32_t dst = twa_smem_u32(ring + static_cast<size_t>(s) * stage_bytes);
     twa_mbar_expect_tx(fb, tx_bytes);
-    twa_tma_load_2d(dst, map_p, tile * TWA_TILE_COL_WORDS * kt, 0, fb);
+    twa_tma_load_2d(dst, map_p, tile * x_per_tile, 0, fb);
     for (int b = 0; b < g_boxes; ++b)
       twa_tma_load_1d(dst + g_off + b * 256 * g_elem_bytes, map_g, tile * tile_rows + b * 256, fb);
     ++issued;

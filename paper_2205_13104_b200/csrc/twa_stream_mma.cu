@@ -97,7 +97,7 @@ twa_project_mma_kernel(const __grid_constant__ CUtensorMap map_p,
       producer_loop_mma(hdr, ring, &map_p, &map_g, blockIdx.x, gridDim.x,
                         (a.tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
                             static_cast<int>(gridDim.x),
-                        a.stages, a.stage_bytes, KT, SROWS * KT / 256, GSZ, SROWS * KT, a.g_off,
+                        a.stages, a.stage_bytes, TWA_TILE_COL_BYTES / 8 * KT, SROWS * KT / 256, GSZ, SROWS * KT, a.g_off,
                         a.tx_bytes, false, a.status, a.wait_limit_ns);
   } else {
     unsigned char* digw = smem + a.scratch_off + warp * BYTE_DIGIT_SCRATCH;   // this warp's digit matrices
@@ -326,7 +326,7 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
       producer_loop_mma(hdr, ring, &map_p, &map_b, blockIdx.x, gridDim.x,
                         (a.tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
                             static_cast<int>(gridDim.x),
-                        a.stages, a.stage_bytes, KT, BTMA ? ROWS * KT / 256 : 0, 4, ROWS * KT, a.base_off,
+                        a.stages, a.stage_bytes, TWA_TILE_COL_BYTES / 8 * KT, BTMA ? ROWS * KT / 256 : 0, 4, ROWS * KT, a.base_off,
                         a.tx_bytes, a.reverse != 0, a.status, a.wait_limit_ns);
     return;
   }
@@ -562,21 +562,29 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
 // =================================================================================================
 // host side
 // =================================================================================================
-// segments per tile column: two for narrow bases, so that a tile stays worth a handshake
-int choose_kt(const twa_ctx* ctx, int n) {
-  if (ctx->tune_tile_segments == 1 || ctx->tune_tile_segments == 2) return ctx->tune_tile_segments;
+// Segments per tile column: more for narrow bases, so that a tile stays worth a handshake and the per-tile
+// work (digit scale, digit sums to float, barrier traffic) is spread over more bytes.  Four segments for
+// n <= 32 where three stages of that size still fit: the lift at both widths (1.3 B-sized lift 7.99 -> 7.67 ms
+// at 8 bits, 4.97 -> 4.66 ms at 4 bits) and the 8-bit projection; a 4-bit projection tile of four segments
+// carries 4096 rows of g as well and only two stages fit (3.55 -> 3.79 ms), so it keeps two.
+int choose_kt(const twa_ctx* ctx, int n, int bits, bool lift) {
+  const int t = ctx->tune_tile_segments;
+  if (t == 1 || t == 2 || (t == 4 && n <= 32)) return t;
+  if (n <= 32 && (lift || bits == 8)) return 4;
   return n <= 64 ? 2 : 1;
 }
 
+// The codes as a 2-D tensor of 8-byte elements {column bytes / 8, n}: a box dimension is limited to 256
+// elements, and a tile of four 512-byte segments is 256 of these.
 int encode_tile_map(twa_ctx* ctx, const twa_basis* P, int kt, CUtensorMap* map) {
   long long row_bytes = (P->D * P->bits + 7) / 8;
   // quantised columns are stored in whole, internally permuted 512-byte segments
-  if (P->bits != 32) row_bytes = (row_bytes + 511) / 512 * 512;
-  cuuint64_t dims[2] = {static_cast<cuuint64_t>((row_bytes + 3) / 4), static_cast<cuuint64_t>(P->n)};
+  row_bytes = (row_bytes + 511) / 512 * 512;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(row_bytes / 8), static_cast<cuuint64_t>(P->n)};
   cuuint64_t strides[1] = {static_cast<cuuint64_t>(P->col_stride)};
-  cuuint32_t box[2] = {static_cast<cuuint32_t>(TWA_TILE_COL_WORDS * kt), static_cast<cuuint32_t>(P->n)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(TWA_TILE_COL_BYTES / 8 * kt), static_cast<cuuint32_t>(P->n)};
   cuuint32_t es[2] = {1, 1};
-  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, P->data, dims, strides, box, es,
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, P->data, dims, strides, box, es,
                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -609,9 +617,12 @@ int round_up_i(int x, int m) { return (x + m - 1) / m * m; }
 template <int BITS, bool GBF16, int MT>
 int launch_project_mma_t(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg,
                          const ProjectMmaArgs& a, int grid, int smem) {
-  auto kern = a.kt == 2 ? twa_project_mma_kernel<BITS, GBF16, MT, 2> : twa_project_mma_kernel<BITS, GBF16, MT, 1>;
-  static int smem_limit[2][64] = {{0}};   // per tile height and device
-  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[a.kt - 1][ctx->device & 63], smem);
+  // four segments per tile exist for n <= 32 only (MT <= 2)
+  auto kern = (a.kt == 4 && MT <= 2) ? twa_project_mma_kernel<BITS, GBF16, MT, (MT <= 2 ? 4 : 1)>
+              : a.kt == 2            ? twa_project_mma_kernel<BITS, GBF16, MT, 2>
+                                     : twa_project_mma_kernel<BITS, GBF16, MT, 1>;
+  static int smem_limit[3][64] = {{0}};   // per tile height and device
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[a.kt >> 1][ctx->device & 63], smem);
   if (rc) return rc;
   kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, mg, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
@@ -628,9 +639,11 @@ struct LiftMaps {
 
 template <int BITS, int KS, int VEC>
 int launch_lift_mma_t(twa_ctx* ctx, const LiftMaps& m, const LiftMmaArgs& a, int grid, int smem) {
-  auto kern = a.kt == 2 ? twa_lift_mma_kernel<BITS, KS, 2, VEC> : twa_lift_mma_kernel<BITS, KS, 1, VEC>;
-  static int smem_limit[2][64] = {{0}};   // per tile height and device
-  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[a.kt - 1][ctx->device & 63], smem);
+  auto kern = (a.kt == 4 && KS == 1) ? twa_lift_mma_kernel<BITS, KS, (KS == 1 ? 4 : 1), VEC>
+              : a.kt == 2            ? twa_lift_mma_kernel<BITS, KS, 2, VEC>
+                                     : twa_lift_mma_kernel<BITS, KS, 1, VEC>;
+  static int smem_limit[3][64] = {{0}};   // per tile height and device
+  int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[a.kt >> 1][ctx->device & 63], smem);
   if (rc) return rc;
   kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(m.p, m.b, m.o, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
@@ -693,7 +706,7 @@ int encode_vector_map(twa_ctx* ctx, const float* v, long long D, int box, CUtens
 int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
                            const twa_project_epilogue& epi, void* ws) {
   const bool bf16 = g_dtype == TWA_BF16;
-  const int kt = choose_kt(ctx, P->n);
+  const int kt = choose_kt(ctx, P->n, P->bits, false);
   const int rows = twa_tile_rows(P->bits) * kt;
   const int gsz = bf16 ? 2 : 4;
   CUtensorMap mp, mg;
@@ -742,7 +755,7 @@ int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_
 
 int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
                         const float* base, float* out, bool reverse_tiles) {
-  const int kt = choose_kt(ctx, P->n);
+  const int kt = choose_kt(ctx, P->n, P->bits, true);
   const int rows = twa_tile_rows(P->bits) * kt;
   CUtensorMap mp;
   int rc = encode_tile_map(ctx, P, kt, &mp);

@@ -485,7 +485,7 @@ def test_chunked_build_reports_rank_deficiency(env):
     twa.twa_clear_status(ctx)
 
 
-@pytest.mark.parametrize("segments", [1, 2])
+@pytest.mark.parametrize("segments", [1, 2, 4])
 @pytest.mark.parametrize("bits", [8, 4])
 @pytest.mark.parametrize("D,n", [(4099, 33), (70001, 100), (131072, 8)])
 def test_tile_segments_knob(env, D, n, bits, segments):
