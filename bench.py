@@ -546,10 +546,11 @@ def run_ours(args):
     ctx = twa.twa_create(env.local)
     twa.twa_set_tuning(ctx, twa.TWA_TUNE_DEQUANT_PATH, args.dequant_path)
     twa.twa_set_tuning(ctx, twa.TWA_TUNE_LIFT_VECTORS, args.lift_vectors)
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_TILE_SEGMENTS, args.tile_segments)
     ws = twa.new_workspace(dev)
     peak, peak_kind = load_peaks()
     with_configs = (not args.no_configs and args.workload == "vitb16" and bits == 8 and not args.rows
-                    and not args.random_basis and args.dequant_path == 0)
+                    and not args.random_basis and args.dequant_path == 0 and args.tile_segments == 0)
 
     # ---- basis build and quantisation, timed once each -------------------------------
     extra_bits = [4] if with_configs else []
@@ -965,6 +966,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--lift-vectors", type=int, default=0, choices=[0, 1, 2, 3],
                     help="TWA_TUNE_LIFT_VECTORS: how base and output travel in the 8/4-bit lift (0 = built-in choice)")
+    ap.add_argument("--tile-segments", type=int, default=0, choices=[0, 1, 2, 4],
+                    help="TWA_TUNE_TILE_SEGMENTS: 512-byte segments of a column per tile (0 = built-in choice)")
     ap.add_argument("--dequant-path", type=int, default=0, choices=[0, 1],
                     help="0: integer dot products on the tensor pipe (default); 1: float32 FMA path")
     ap.add_argument("--rows", type=int, default=0, help="override D (smaller cases for profiler captures)")

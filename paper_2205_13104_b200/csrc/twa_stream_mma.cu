@@ -562,16 +562,25 @@ twa_lift_mma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
 // =================================================================================================
 // host side
 // =================================================================================================
-// Segments per tile column: more for narrow bases, so that a tile stays worth a handshake and the per-tile
-// work (digit scale, digit sums to float, barrier traffic) is spread over more bytes.  Four segments for
-// n <= 32 where three stages of that size still fit: the lift at both widths (1.3 B-sized lift 7.99 -> 7.67 ms
-// at 8 bits, 4.97 -> 4.66 ms at 4 bits) and the 8-bit projection; a 4-bit projection tile of four segments
-// carries 4096 rows of g as well and only two stages fit (3.55 -> 3.79 ms), so it keeps two.
-int choose_kt(const twa_ctx* ctx, int n, int bits, bool lift) {
+// Segments per tile column.  Taller tiles spread the per-tile work (digit scale, digit sums to float,
+// barrier traffic) over more bytes, but fewer of them fit in the ring.  The rule below is the one the
+// measurements on B200 agree with (1.3 B-sized n = 32, ResNet-50-sized n = 50, ViT-B/16-sized n = 100, both
+// widths): the tallest tile of 4 (n <= 32 only), 2 or 1 segments of which at least `want` stages fit, with
+// want = 2 for the 8-bit projection and the 4-bit lift, 3 for the 4-bit projection and the 8-bit lift.
+//   n = 32: lift 7.99 -> 7.67 ms (8 bits, 4 segments) and 4.97 -> 4.66 ms (4 bits, 4 segments, two stages);
+//           4-bit projection 3.55 ms with 2 segments against 3.79 ms with 4.
+//   n = 100: 8-bit projection 1.29 -> 1.24 ms with 2 segments (two stages), 8-bit lift 1.38 ms with 1 against
+//           1.39 ms with 2; 4-bit lift 0.754 -> 0.732 ms with 2, 4-bit projection 0.668 ms with 1 against 0.682.
+// row_bytes = bytes per tile row that ride the ring beside the codes (g, or the base vector).
+int choose_kt(const twa_ctx* ctx, int n, int bits, bool lift, int row_bytes, int fixed_smem) {
   const int t = ctx->tune_tile_segments;
   if (t == 1 || t == 2 || (t == 4 && n <= 32)) return t;
-  if (n <= 32 && (lift || bits == 8)) return 4;
-  return n <= 64 ? 2 : 1;
+  const int want = (lift ? bits == 8 : bits == 4) ? 3 : 2;
+  for (int kt = n <= 32 ? 4 : 2; kt > 1; kt >>= 1) {
+    const int stage = (n * TWA_TILE_COL_BYTES * kt + twa_tile_rows(bits) * kt * row_bytes + 1023) / 1024 * 1024;
+    if ((ctx->smem_optin - fixed_smem) / stage >= want) return kt;
+  }
+  return 1;
 }
 
 // The codes as a 2-D tensor of 8-byte elements {column bytes / 8, n}: a box dimension is limited to 256
@@ -706,9 +715,10 @@ int encode_vector_map(twa_ctx* ctx, const float* v, long long D, int box, CUtens
 int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype,
                            const twa_project_epilogue& epi, void* ws) {
   const bool bf16 = g_dtype == TWA_BF16;
-  const int kt = choose_kt(ctx, P->n, P->bits, false);
-  const int rows = twa_tile_rows(P->bits) * kt;
   const int gsz = bf16 ? 2 : 4;
+  const int fixed = TWA_SMEM_HEADER + MMA_WARPS * BYTE_DIGIT_SCRATCH + 1024;   // 1024: alignment slack
+  const int kt = choose_kt(ctx, P->n, P->bits, false, gsz, fixed);
+  const int rows = twa_tile_rows(P->bits) * kt;
   CUtensorMap mp, mg;
   int rc = encode_tile_map(ctx, P, kt, &mp);
   if (rc) return rc;
@@ -723,7 +733,6 @@ int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_
   a.g_off = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt;
   a.tx_bytes = a.g_off + static_cast<unsigned>(rows * gsz);
   a.stage_bytes = static_cast<unsigned>(round_up_i(static_cast<int>(a.tx_bytes), 1024));
-  const int fixed = TWA_SMEM_HEADER + MMA_WARPS * BYTE_DIGIT_SCRATCH + 1024;   // 1024: alignment slack
   int stages = (ctx->smem_optin - fixed) / static_cast<int>(a.stage_bytes);
   if (stages > TWA_MAX_STAGES) stages = TWA_MAX_STAGES;
   if (ctx->tune_stages >= 2 && ctx->tune_stages < stages) stages = ctx->tune_stages;
@@ -755,16 +764,6 @@ int twa_launch_project_mma(twa_ctx* ctx, const twa_basis* P, const void* g, twa_
 
 int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, float alpha_mult,
                         const float* base, float* out, bool reverse_tiles) {
-  const int kt = choose_kt(ctx, P->n, P->bits, true);
-  const int rows = twa_tile_rows(P->bits) * kt;
-  CUtensorMap mp;
-  int rc = encode_tile_map(ctx, P, kt, &mp);
-  if (rc) return rc;
-  LiftMmaArgs a;
-  a.D = P->D;
-  a.n = P->n;
-  a.tiles = static_cast<int>((P->D + rows - 1) / rows);
-  a.kt = kt;
   // How base and output travel (see the kernel): through the ring and bulk stores when tensor maps
   // can describe them (16-byte aligned starts) and the two vectors are a large share of the bytes
   // moved, 64 / (n * bits + 64).  Measured on B200: a third (n = 16 at 8 bits, n = 32 at 4 bits): base
@@ -775,6 +774,18 @@ int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, fl
   const int nb = P->n * P->bits;
   int vec = ctx->tune_lift_base_path == 0 ? (nb <= 192 ? 1 : (nb <= 320 ? 2 : 0)) : ctx->tune_lift_base_path - 1;
   if (base == nullptr || ((reinterpret_cast<uintptr_t>(base) | reinterpret_cast<uintptr_t>(out)) & 15u) != 0) vec = 0;
+  if (vec == 2 && P->D < 4) vec = 1;                      // nothing for a bulk store to write
+  const int fixed = TWA_SMEM_HEADER + 4 * TWA_MAX_N + 1024;               // 1024: alignment slack
+  const int kt = choose_kt(ctx, P->n, P->bits, true, vec >= 1 ? 4 : 0, fixed);
+  const int rows = twa_tile_rows(P->bits) * kt;
+  CUtensorMap mp;
+  int rc = encode_tile_map(ctx, P, kt, &mp);
+  if (rc) return rc;
+  LiftMmaArgs a;
+  a.D = P->D;
+  a.n = P->n;
+  a.tiles = static_cast<int>((P->D + rows - 1) / rows);
+  a.kt = kt;
   const bool btma = vec >= 1;
   LiftMaps maps;
   maps.p = mp;
@@ -785,9 +796,6 @@ int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, fl
     if (rc) return rc;
   }
   if (vec == 2) {
-    if (P->D < 4) vec = 1;                                // nothing for a bulk store to write
-  }
-  if (vec == 2) {
     // rows [D & ~3, D) are stored by the lanes: a bulk store clips in units of 16 bytes
     rc = encode_vector_map(ctx, out, P->D & ~3ll, kt * 32 * (8 / P->bits), &maps.o);
     if (rc) return rc;
@@ -795,7 +803,6 @@ int twa_launch_lift_mma(twa_ctx* ctx, const twa_basis* P, const float* alpha, fl
   a.base_off = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt;
   a.tx_bytes = a.base_off + (btma ? static_cast<unsigned>(rows) * 4u : 0u);
   a.stage_bytes = static_cast<unsigned>(round_up_i(static_cast<int>(a.tx_bytes), 1024));
-  const int fixed = TWA_SMEM_HEADER + 4 * TWA_MAX_N + 1024;               // 1024: alignment slack
   int stages = (ctx->smem_optin - fixed) / static_cast<int>(a.stage_bytes);
   if (stages > TWA_MAX_STAGES) stages = TWA_MAX_STAGES;
   if (ctx->tune_stages >= 2 && ctx->tune_stages < stages) stages = ctx->tune_stages;
