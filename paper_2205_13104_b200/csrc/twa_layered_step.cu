@@ -267,7 +267,7 @@ layered_project_kernel(const __grid_constant__ CUtensorMap map_p, const LProject
 
   if (warp == MMA_WARPS) {
     if (lane == 0)
-      producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, TWA_TILE_COL_WORDS * KT, 0, 0,
+      producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, TWA_TILE_COL_BYTES / 8 * KT, 0, 0,
                         0, 0, a.tx_bytes, false, a.status, a.wait_limit_ns);
     return;
   }
@@ -596,7 +596,7 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
   const int t_count = (a.tiles - t_first) < a.tpc ? (a.tiles - t_first) : a.tpc;
   if (warp == MMA_WARPS) {
     if (lane == 0)
-      producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, TWA_TILE_COL_WORDS * KT, 0, 0,
+      producer_loop_mma(hdr, ring, &map_p, nullptr, t_first, 1, t_count, a.stages, a.stage_bytes, TWA_TILE_COL_BYTES / 8 * KT, 0, 0,
                         0, 0, a.tx_bytes, true, a.status, a.wait_limit_ns);
     return;
   }
@@ -790,14 +790,16 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
+// The codes as a 2-D tensor of 8-byte elements {column bytes / 8, n} (a box dimension is limited to 256
+// elements; a tile of four 512-byte segments is 256 of these).
 int encode_codes_map(twa_ctx* ctx, const twa_basis* P, int kt, CUtensorMap* map) {
   long long row_bytes = (P->D * P->bits + 7) / 8;
   row_bytes = (row_bytes + 511) / 512 * 512;
-  cuuint64_t dims[2] = {static_cast<cuuint64_t>(row_bytes / 4), static_cast<cuuint64_t>(P->n)};
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(row_bytes / 8), static_cast<cuuint64_t>(P->n)};
   cuuint64_t strides[1] = {static_cast<cuuint64_t>(P->col_stride)};
-  cuuint32_t box[2] = {static_cast<cuuint32_t>(TWA_TILE_COL_WORDS * kt), static_cast<cuuint32_t>(P->n)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(TWA_TILE_COL_BYTES / 8 * kt), static_cast<cuuint32_t>(P->n)};
   cuuint32_t es[2] = {1, 1};
-  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, P->data, dims, strides, box, es,
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, P->data, dims, strides, box, es,
                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -850,6 +852,7 @@ int launch_lproject(twa_ctx* ctx, const CUtensorMap& mp, const LProjectArgs& a, 
 
 template <int BITS, int KS>
 int launch_llift_t(twa_ctx* ctx, const CUtensorMap& mp, const LLiftArgs& a, int kt, int grid, int smem) {
+  // slots below 4 bits are tiled with one segment only
   auto kern = (BITS >= 4 && kt == 2) ? layered_lift_kernel<BITS, KS, (BITS >= 4 ? 2 : 1)> : layered_lift_kernel<BITS, KS, 1>;
   static int smem_limit[2][64] = {{0}};
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[kt - 1][ctx->device & 63], smem);
@@ -927,7 +930,11 @@ int do_project(twa_ctx* ctx, const twa_layered_basis* lb, const void* g, twa_dty
 int do_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* beta, const float* base, float* out,
             bool digits_ready, char* sws) {
   const StepLayout w = step_layout(lb);
-  const int n = lb->codes.n, kt = lb->kt;
+  const int n = lb->codes.n;
+  // (One or two segments per tile, as fixed when the basis was quantised: a warp's share of a tile, 32 * KT bytes
+  // of every column, must lie inside one 64-byte granule, i.e. inside one layer.)
+  const int kt = lb->kt;
+  const int tiles = lb->tiles, tpc = lb->tiles_per_cta;
   unsigned char* dig = reinterpret_cast<unsigned char*>(sws + w.dig);
   int* ebits = reinterpret_cast<int*>(sws + w.ebits);
   float* konst = reinterpret_cast<float*>(sws + w.konst);
@@ -942,8 +949,8 @@ int do_lift(twa_ctx* ctx, const twa_layered_basis* lb, const float* beta, const 
   if (rc) return rc;
   LLiftArgs a;
   a.n = n;
-  a.tiles = lb->tiles;
-  a.tpc = lb->tiles_per_cta;
+  a.tiles = tiles;
+  a.tpc = tpc;
   a.D = lb->D;
   a.tx_bytes = static_cast<unsigned>(n) * TWA_TILE_COL_BYTES * kt;
   a.aux_off = a.tx_bytes;
