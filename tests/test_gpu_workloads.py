@@ -56,7 +56,7 @@ _PINNED = {}
 
 def to_host(t):
     """A device tensor's bytes as a numpy array, through one reused pinned staging buffer (pageable
-    copies of the 10 GB column blocks of the largest workload run at 2 GB/s on the test hosts)."""
+    copies of the 10 GB column blocks of the largest workload run at about 2 GB/s)."""
     flat = t.contiguous().view(torch.uint8).reshape(-1)
     buf = _PINNED.get("buf")
     if buf is None or buf.numel() < flat.numel():
@@ -189,7 +189,7 @@ def run_sequence(ctx, ws, wl, bases, wbar, T, sample_cols, step1_blocks=None):
     g_pin = torch.empty(D, dtype=torch.float32).pin_memory()
     g_host = g_pin.numpy()
     # The weighted sum of the gradients, an INPUT of the oracle's closing projection, is accumulated in
-    # float64 by torch on the device (the host of the GPU machine adds 1.3 G float64 numbers in seconds, fifty
+    # float64 by torch on the device (a host adds 1.3 G float64 numbers in seconds, and would do so fifty
     # times over); the same sum is accumulated on the host for sampled row ranges and must agree bit for bit.
     need_host_g = any(len(st["cols"]) for st in state)
     G_dev = torch.zeros(D, dtype=torch.float64, device=DEV)
