@@ -385,12 +385,16 @@ def gradient_pool(wl, D, dev, count):
 
 
 def build_resident(ctx, wl, dev, ws, bits_list, twa, inputs, random_basis=False):
-    """Candidates -> float32 basis (timed) -> one quantised basis per width (each timed).
-    Returns ({bits: basis}, wbar, build_ms, {bits: quantise ms})."""
+    """Candidates -> float32 basis (timed) -> one quantised basis per width (each timed, output buffers
+    allocated beforehand), then once more from fresh candidates through the one-call form
+    twa_build_quantized (timed; same buffers, same bytes).
+    Returns ({bits: basis}, wbar, build_ms, {bits: quantise ms}, fused build+quantise ms or None)."""
     import torch
     D, n = wl.D, wl.n
     wbar = torch.empty(D, dtype=torch.float32, device=dev)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    low = [b for b in bits_list if b != 32]
+    outs = {b: twa.new_quantised_basis(D, n, b, dev) for b in low}
     if random_basis:
         # profiling aid: skip the Gram-Schmidt launches; the step kernels do the same work on any values
         W = torch.randn((n, inputs.padded_ld(D, 128)), device=dev) / (D ** 0.5)
@@ -412,14 +416,28 @@ def build_resident(ctx, wl, dev, ws, bits_list, twa, inputs, random_basis=False)
             continue
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        bases[bits] = twa.twa_quantize_basis(ctx, P32, bits, ws)
+        bases[bits] = twa.twa_quantize_basis(ctx, P32, bits, ws, out=outs[bits])
         b.record()
         torch.cuda.synchronize()
         quant_ms[bits] = a.elapsed_time(b)
+    fused_ms = None
+    if low and not random_basis:
+        keep32 = 32 in bits_list
+        if not keep32:
+            del P32, W
+            torch.cuda.empty_cache()
+        W2 = wl.candidates(dev, ld=inputs.padded_ld(D, 128))
+        torch.cuda.synchronize()
+        ev[0].record()
+        P32b, _ = twa.twa_build_quantized(ctx, W2, D, wbar, low, ws, out=[outs[b] for b in low])
+        ev[1].record()
+        torch.cuda.synchronize()
+        fused_ms = ev[0].elapsed_time(ev[1])
+        del W2, P32b
     code, detail = twa.twa_get_status(ctx)
     if code != 0:
         raise RuntimeError(f"basis build failed: {twa.twa_strerror(code)} column {detail}")
-    return bases, wbar, build_ms, quant_ms
+    return bases, wbar, build_ms, quant_ms, fused_ms
 
 
 def build_chunked(ctx, wl, dev, bits_list, twa, inputs):
@@ -505,7 +523,17 @@ def clock_fields(sampler, walls, series):
     return clocks, per
 
 
-def config_entry(wl, bits, m, peak, build_ms, quant_ms, clocks, note=None):
+def fused_record(fused_ms, widths):
+    """What twa_build_quantized took: mean, basis and every low-bit width in one call."""
+    low = [b for b in widths if b != 32]
+    if fused_ms is None or not low:
+        return None
+    return {"ms": fused_ms, "widths": low,
+            "call": "twa_build_quantized: the column maxima are taken while the build writes its last pass, "
+                    "so each width costs one encoding pass"}
+
+
+def config_entry(wl, bits, m, peak, build_ms, quant_ms, clocks, fused_ms=None, widths=(), note=None):
     """One element of the line's "configs" array."""
     D, n = wl.D, wl.n
     g_bytes = 2 if wl.g_dtype == "bf16" else 4
@@ -523,6 +551,7 @@ def config_entry(wl, bits, m, peak, build_ms, quant_ms, clocks, note=None):
          "sm_mhz": None if clocks is None else clocks["sm_mhz"],
          "clock_reasons": None if clocks is None else clocks["reasons"],
          "basis_build_ms": build_ms, "quantize_ms": quant_ms,
+         "build_and_quantize_one_call": fused_record(fused_ms, widths),
          "l2": ("P~ (%.0f MB) fits the 126 MB L2 wholly or in good part: not an HBM fraction" % (p_bytes / 1e6))
                if p_bytes < 2.5 * L2_BYTES else "inputs larger than L2"}
     if note:
@@ -558,10 +587,10 @@ def run_ours(args):
         if bits == 32:
             raise SystemExit("the chunked workload has no resident float32 basis; use --bits 8 or 4")
         bases, wbar, build_ms = build_chunked(ctx, wl, dev, [bits] + extra_bits, twa, inputs)
-        quant_ms = {b: None for b in bases}
+        quant_ms, fused_ms = {b: None for b in bases}, None
     else:
-        bases, wbar, build_ms, quant_ms = build_resident(ctx, wl, dev, ws, [bits] + extra_bits, twa, inputs,
-                                                         args.random_basis)
+        bases, wbar, build_ms, quant_ms, fused_ms = build_resident(ctx, wl, dev, ws, [bits] + extra_bits, twa, inputs,
+                                                                   args.random_basis)
     Pq = bases[bits]
     if bits != 32:
         bases.pop(32, None)
@@ -603,7 +632,7 @@ def run_ours(args):
             m4 = measure_steps(env, ctx, twa, wl, bases[4], wbar, ws, pool, args.steps, args.warmup,
                                args.configs_min_ms, s4)
             c4 = s4.stop().summary(m4["walls"][0][0], m4["walls"][-1][1]) if s4 is not None else None
-            configs.append(config_entry(wl, 4, m4, peak, build_ms_all, quant_ms.get(4), c4))
+            configs.append(config_entry(wl, 4, m4, peak, build_ms_all, quant_ms.get(4), c4, fused_ms, [bits] + extra_bits))
     # CPU baseline: the oracle on the first rows of THIS basis (rank 0, N = 1 only)
     if rank == 0 and world == 1 and not args.no_cpu_baseline and bits != 32:
         rows = min(D, args.reference_rows)
@@ -654,6 +683,7 @@ def run_ours(args):
             "frac_of_8TBps": value / world / 8000.0,
             "basis_build_ms": None if args.random_basis else build_ms_all,
             "quantize_ms": None if wl.chunked_build else quant_ms_all,
+            "build_and_quantize_one_call": fused_record(fused_ms, [bits] + extra_bits),
             "basis_build": ("row-chunked Gram-form build incl. quantisation, 4 passes, chunk generation not counted"
                             if wl.chunked_build else
                             "resident block Gram-Schmidt with re-orthogonalisation: panels of 8 columns, "
@@ -690,9 +720,9 @@ def other_configs(env, ctx, twa, inputs, ws, args, peak):
         wl = inputs.WORKLOADS[name]
         if wl.chunked_build:
             bases, wbar, build_ms = build_chunked(ctx, wl, dev, widths, twa, inputs)
-            quant_ms = {b: None for b in widths}
+            quant_ms, fused_ms = {b: None for b in widths}, None
         else:
-            bases, wbar, build_ms, quant_ms = build_resident(ctx, wl, dev, ws, widths, twa, inputs)
+            bases, wbar, build_ms, quant_ms, fused_ms = build_resident(ctx, wl, dev, ws, widths, twa, inputs)
         pool = gradient_pool(wl, wl.D, dev, args.g_pool)
         for bits in widths:
             sampler = ClockSampler(env.local).start() if env.rank == 0 else None
@@ -702,7 +732,7 @@ def other_configs(env, ctx, twa, inputs, ws, args, peak):
             if sampler is not None:
                 sampler.stop()
                 clocks = sampler.summary(m["walls"][0][0], m["walls"][-1][1])
-            out.append(config_entry(wl, bits, m, peak, build_ms, quant_ms.get(bits), clocks))
+            out.append(config_entry(wl, bits, m, peak, build_ms, quant_ms.get(bits), clocks, fused_ms, widths))
         del bases, wbar, pool
         torch.cuda.empty_cache()
     # the other modes of the library, each through its own benchmark routine, condensed

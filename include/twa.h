@@ -163,9 +163,9 @@ size_t twa_workspace_bytes(int64_t D, int n, int bits);
  *           e_j, the j-th vector of the Gram-Schmidt orthonormalisation of the candidates in
  *           the given order (the factor Q of A = QR with positive diagonal).  Schedule: block
  *           classical Gram-Schmidt with one re-orthogonalisation -- panels of 8 columns are
- *           first made orthogonal to all earlier vectors (twice), then orthonormalised among
+ *           first made orthogonal to all earlier vectors, then orthonormalised among
  *           themselves from the panel's float64 Gram matrix (its Cholesky factor holds the
- *           Gram-Schmidt coefficients), twice.  TWA_TUNE_BUILD_PANEL = 1 selects the literal
+ *           Gram-Schmidt coefficients), and both steps are done a second time.  TWA_TUNE_BUILD_PANEL = 1 selects the literal
  *           column-after-column schedule (two projection passes per column); both give the
  *           same factor up to rounding.
  *  wbar_out out: D floats, the mean of the candidates (written before W is overwritten).
@@ -174,6 +174,19 @@ size_t twa_workspace_bytes(int64_t D, int n, int bits);
  * is below 1e-5 of its length; that column is set to zero). */
 int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float* wbar_out,
                     twa_basis* P32_out, void* ws, size_t ws_bytes);
+
+/* twa_build_basis followed by twa_quantize_basis for each of `widths` storage widths (Sections
+ * 4.1 and 4.6 in one call), with one pass over the float32 basis less: the largest magnitude
+ * of every column is taken while the build writes the column for the last time, so each width
+ * costs one encoding pass only.  Basis, scales and codes are those of the separate calls, bit
+ * for bit.
+ *  bits  host array of `widths` entries (1 <= widths <= 8), each 8 or 4.
+ *  Pq    host array of `widths` descriptors; the caller sets data (twa_basis_bytes(D, n,
+ *        bits[k]) bytes) and scales (n floats) of each, the call fills the rest.
+ * Other arguments and device-side errors as for twa_build_basis and twa_quantize_basis. */
+int twa_build_quantized(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float* wbar_out,
+                        twa_basis* P32_out, const int* bits, int widths, twa_basis* Pq, void* ws,
+                        size_t ws_bytes);
 
 /* The same basis for candidate sets too large to be resident (e.g. 1.3 G rows x 32 columns =
  * 168 GB of float32): the caller feeds row chunks of the candidates, once per pass, and never

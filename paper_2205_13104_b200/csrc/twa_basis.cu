@@ -19,6 +19,7 @@ __global__ void __launch_bounds__(BLOCK) mean_kernel(const float* __restrict__ W
   for (long long v = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; v < nvec;
        v += static_cast<long long>(gridDim.x) * BLOCK) {
     double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+#pragma unroll 8
     for (int i = 0; i < n; ++i) {
       const float4 x = __ldcs(reinterpret_cast<const float4*>(W + i * ldw) + v);
       s0 += x.x; s1 += x.y; s2 += x.z; s3 += x.w;
@@ -265,43 +266,108 @@ __global__ void scales_kernel(const unsigned* __restrict__ absmax, int n, float 
   }
 }
 
-// One thread produces 16 bytes of a column (16 rows at 8 bits, 32 rows at 4 bits), including
-// the padding up to the column stride, which is filled with the code 0.
+// The quantiser's code of p without a division per element.  With r = RN(1 / s) the product q0 = p r
+// lies within 2^-16 of the IEEE quotient p / s wherever the clamp to +-qmax (<= 127) does not decide
+// the code anyway, so both round to the same integer unless q0 is that close to a half-integer; then,
+// and only then, *hard is set and the caller takes the IEEE division.  The distance of q0 to the
+// integer it rounds to is exact in float32.  Valid while r is finite (the caller checks s).
+__device__ __forceinline__ int encode_by_reciprocal(float p, float r, float qmax, bool* hard) {
+  const float q0 = fminf(fmaxf(p * r, -qmax), qmax);
+  const float y = q0 + 12582912.0f;                    // 1.5 * 2^23: rounds to an integer, half to even
+  const float t = q0 - (y - 12582912.0f);
+  *hard = fabsf(t) >= 0.5f - 0x1p-15f;
+  return __float_as_int(y) - 0x4B400000;
+}
+
+// Rows r .. r + 3 of a column; rows from D on read as zero.
+__device__ __forceinline__ float4 load_four(const float* __restrict__ col, long long r, long long D) {
+  if (r + 3 < D) return __ldcs(reinterpret_cast<const float4*>(col + r));
+  float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (r < D) x.x = col[r];
+  if (r + 1 < D) x.y = col[r + 1];
+  if (r + 2 < D) x.z = col[r + 2];
+  return x;
+}
+
+// Four codes as the low bytes (BITS == 8) or nibbles (BITS == 4) of a word, x.x first.  `recip`:
+// RN(1 / s), or 0 when every element takes the division (s zero, or so small that its reciprocal is
+// not finite).
+template <int BITS>
+__device__ __forceinline__ uint32_t encode_four(float4 x, float s, float recip) {
+  constexpr float QMAX = BITS == 8 ? 127.0f : 7.0f;
+  constexpr uint32_t MASK = BITS == 8 ? 0xFFu : 0xFu;    // two's-complement byte or nibble
+  int c0, c1, c2, c3;
+  bool h0, h1, h2, h3;
+  c0 = encode_by_reciprocal(x.x, recip, QMAX, &h0);
+  c1 = encode_by_reciprocal(x.y, recip, QMAX, &h1);
+  c2 = encode_by_reciprocal(x.z, recip, QMAX, &h2);
+  c3 = encode_by_reciprocal(x.w, recip, QMAX, &h3);
+  if (recip == 0.0f || h0 || h1 || h2 || h3) {
+    c0 = twa_encode_one(x.x, s, QMAX);
+    c1 = twa_encode_one(x.y, s, QMAX);
+    c2 = twa_encode_one(x.z, s, QMAX);
+    c3 = twa_encode_one(x.w, s, QMAX);
+  }
+  return (static_cast<uint32_t>(c0) & MASK) | ((static_cast<uint32_t>(c1) & MASK) << BITS) |
+         ((static_cast<uint32_t>(c2) & MASK) << (2 * BITS)) | ((static_cast<uint32_t>(c3) & MASK) << (3 * BITS));
+}
+
+// A warp produces one aligned 128-byte line of a column's codes per step -- 128 rows at 8 bits, 256
+// at 4 -- including the padding up to the column stride, which is filled with the code 0.  A lane
+// reads four consecutive rows (the warp 512 contiguous bytes per load) and stores one 32-bit word;
+// the permutation of the 16-byte chunks stays inside the line, so every store covers the whole line.
+// At 4 bits a lane encodes four rows of each half of the line and neighbouring lanes swap one half:
+// even lanes complete words of the first half, odd lanes of the second.
 template <int BITS>
 __global__ void __launch_bounds__(BLOCK) encode_kernel(const float* __restrict__ P, long long D,
                                                        long long ld, const float* __restrict__ scales,
                                                        unsigned char* __restrict__ out,
                                                        long long out_stride) {
-  constexpr int RPT = 128 / BITS;                     // rows per thread-iteration
-  constexpr float QMAX = BITS == 8 ? 127.0f : 7.0f;
-  constexpr uint32_t MASK = BITS == 8 ? 0xFFu : 0xFu;    // two's-complement byte or nibble
+  constexpr int LINE_ROWS = 1024 / BITS;
+  constexpr int UNROLL = 4;                           // lines a warp has in flight
   const int j = blockIdx.y;
   const float* col = P + j * ld;
   const float s = scales[j];
-  uint4* dst = reinterpret_cast<uint4*>(out + j * out_stride);
-  const long long chunks = out_stride / 16;
-  for (long long q = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; q < chunks;
-       q += static_cast<long long>(gridDim.x) * BLOCK) {
-    const long long r0 = q * RPT;
-    float p[RPT];
-    if (r0 + RPT <= D) {
+  // the reciprocal path needs 1 / s finite and q0's error bound, which assumes a normal s
+  const float recip = s >= 0x1p-100f ? __frcp_rn(s) : 0.0f;
+  unsigned char* dst = out + j * out_stride;
+  const long long lines = out_stride / 128;
+  const int lane = threadIdx.x & 31;
+  const long long warp0 = (blockIdx.x * static_cast<long long>(BLOCK / 32) + (threadIdx.x >> 5)) * UNROLL;
+  const long long step = static_cast<long long>(gridDim.x) * (BLOCK / 32) * UNROLL;
+  // where this lane's word goes inside a line
+  int byte;
+  if (BITS == 8) byte = 4 * lane;
+  else byte = (lane & 1) ? 64 + 2 * (lane - 1) : 2 * lane;
+  for (long long l0 = warp0; l0 < lines; l0 += step) {
+    // every load of the step first, then the arithmetic
+    float4 xa[UNROLL], xb[BITS == 4 ? UNROLL : 1];
 #pragma unroll
-      for (int k = 0; k < RPT / 4; ++k) {
-        const float4 x = __ldcs(reinterpret_cast<const float4*>(col + r0) + k);
-        p[4 * k] = x.x; p[4 * k + 1] = x.y; p[4 * k + 2] = x.z; p[4 * k + 3] = x.w;
+    for (int u = 0; u < UNROLL; ++u) {
+      const long long r0 = (l0 + u) * LINE_ROWS;
+      xa[u] = load_four(col, r0 + 4 * lane, D);
+      if (BITS == 4) xb[u] = load_four(col, r0 + 128 + 4 * lane, D);
+    }
+    uint32_t w[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      if (BITS == 8) {
+        w[u] = encode_four<8>(xa[u], s, recip);
+      } else {
+        const uint32_t ha = encode_four<4>(xa[u], s, recip);
+        const uint32_t hb = encode_four<4>(xb[BITS == 4 ? u : 0], s, recip);
+        const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, (lane & 1) ? ha : hb, 1);
+        w[u] = (lane & 1) ? (got | (hb << 16)) : (ha | (got << 16));
       }
-    } else {
-#pragma unroll
-      for (int k = 0; k < RPT; ++k) p[k] = (r0 + k < D) ? col[r0 + k] : 0.0f;
     }
-    uint32_t w[4] = {0, 0, 0, 0};
 #pragma unroll
-    for (int k = 0; k < RPT; ++k) {
-      const uint32_t u = static_cast<uint32_t>(twa_encode_one(p[k], s, QMAX)) & MASK;
-      if (BITS == 8) w[k >> 2] |= u << (8 * (k & 3));
-      else w[k >> 3] |= u << (4 * (k & 7));
+    for (int u = 0; u < UNROLL; ++u) {
+      if (l0 + u < lines) {
+        const long long q = (l0 + u) * 8 + (byte >> 4);                      // logical 16-byte chunk
+        const long long slot = (q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j);
+        *reinterpret_cast<uint32_t*>(dst + slot * 16 + (byte & 15)) = w[u];
+      }
     }
-    dst[(q & ~31LL) | twa_chunk_slot(static_cast<int>(q & 31), j)] = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
 
@@ -338,6 +404,15 @@ __global__ void __launch_bounds__(BLOCK) import_kernel(const unsigned char* __re
     dst[internal_pos(b, j)] = (b < row_bytes) ? static_cast<unsigned char>(src[b] ^ mask) : mask;
 }
 
+// Blocks of `kernel` (BLOCK threads, no dynamic shared memory) that fit on the device at once: a grid of
+// that many blocks, or a divisor of it, runs as one wave with no tail.
+template <typename K>
+int resident_blocks(const twa_ctx* ctx, K kernel) {
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, BLOCK, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+  return per_sm * ctx->sm_count;
+}
+
 int grid_for(const twa_ctx* ctx, long long items, int per_block, int blocks_per_sm) {
   long long g = (items + per_block - 1) / per_block;
   const long long cap = static_cast<long long>(ctx->sm_count) * blocks_per_sm;
@@ -345,6 +420,37 @@ int grid_for(const twa_ctx* ctx, long long items, int per_block, int blocks_per_
   if (g > TWA_MAX_GRID) g = TWA_MAX_GRID;
   if (g < 1) g = 1;
   return static_cast<int>(g);
+}
+
+// Codes of every column of P32 into Pq->data with the scales already in Pq->scales.
+int launch_encode(twa_ctx* ctx, const twa_basis* P32, int bits, const twa_basis* Pq) {
+  const long long stride = twa_basis_col_stride(P32->D, bits);
+  const long long steps = (stride / 128 + 3) / 4;                    // warp steps per column (4 lines each)
+  const long long want = (steps + BLOCK / 32 - 1) / (BLOCK / 32);    // blocks that have work, per column
+  const int fit = bits == 8 ? resident_blocks(ctx, encode_kernel<8>) : resident_blocks(ctx, encode_kernel<4>);
+  long long per_col = fit / P32->n;
+  if (per_col > want) per_col = want;
+  if (per_col < 1) per_col = 1;
+  const dim3 grid(static_cast<unsigned>(per_col), P32->n);
+  const float* P = static_cast<const float*>(P32->data);
+  unsigned char* out = static_cast<unsigned char*>(Pq->data);
+  if (bits == 8)
+    encode_kernel<8><<<grid, BLOCK, 0, ctx->stream>>>(P, P32->D, P32->col_stride / 4, Pq->scales, out, stride);
+  else
+    encode_kernel<4><<<grid, BLOCK, 0, ctx->stream>>>(P, P32->D, P32->col_stride / 4, Pq->scales, out, stride);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+int launch_absmax(twa_ctx* ctx, const float* P, long long D, long long ld, int n, unsigned* absmax) {
+  int total = grid_for(ctx, D, BLOCK * 16, 8);
+  const int fit = resident_blocks(ctx, absmax_kernel);
+  if (total > fit) total = fit;
+  int per_col = total / n;
+  if (per_col < 1) per_col = 1;
+  absmax_kernel<<<dim3(per_col, n), BLOCK, 0, ctx->stream>>>(P, D, ld, absmax);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
 }
 
 int launch_sumsq(twa_ctx* ctx, const float* v, long long D, void* ws, double* result) {
@@ -385,14 +491,22 @@ int twa_mean(twa_ctx* ctx, const float* W, int64_t D, int n, int64_t ldw, float*
   if ((reinterpret_cast<uintptr_t>(W) & 15) || (ldw & 3) || (reinterpret_cast<uintptr_t>(wbar_out) & 15))
     return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-  const int grid = grid_for(ctx, D, BLOCK * 4, 8);
+  int grid = grid_for(ctx, D, BLOCK * 4, 8);
+  const int fit = resident_blocks(ctx, mean_kernel);
+  if (grid > fit) grid = fit;
   mean_kernel<<<grid, BLOCK, 0, ctx->stream>>>(W, D, n, ldw, wbar_out);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
 }
 
-int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float* wbar_out,
-                    twa_basis* P32_out, void* ws, size_t ws_bytes) {
+}  // extern "C"
+
+namespace {
+
+// twa_build_basis; with `absmax` (device, n words, zero on entry) the largest magnitude of every
+// finished column is folded into it while the column is written for the last time.
+int build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float* wbar_out, twa_basis* P32_out, void* ws,
+                size_t ws_bytes, unsigned* absmax) {
   if (!ctx || !W || !wbar_out || !P32_out) return TWA_ERR_INVALID_ARG;
   if (D < 1 || D >= (1LL << 31) || n < 1 || ldw < D) return TWA_ERR_INVALID_ARG;
   if (n > TWA_MAX_N) return TWA_ERR_UNSUPPORTED;
@@ -448,25 +562,38 @@ int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float
     // cancellation amplifies; the second round, applied to unit vectors, removes that.
     for (int j0 = 0; j0 < n; j0 += width) {
       const int pb = n - j0 < width ? n - j0 : width;
+      float* panel = W + j0 * ldw;
+      if (ctx->tune_build_panel == 0) {
+        // Gram form inside the panel: all coefficients of the panel's own Gram-Schmidt from its Gram
+        // matrix, the new columns in one pass.  The squared norms of the columns as given come out of
+        // the first projection, the Gram matrix out of the update (the first panel, which has neither,
+        // takes its Gram matrix in a pass of its own and its norms from the diagonal); in the second
+        // round the rank test compares against the columns' norms as this round found them (1, or 0
+        // for a column already found dependent).
+        for (int round = 0; round < 2; ++round) {
+          if (j0 > 0) {
+            rc = twa_launch_panel_project(ctx, W, D, ldw, j0, pb, ws, round == 0 ? given : nullptr);
+            if (rc) return rc;
+            rc = twa_launch_panel_lift(ctx, W, D, ldw, j0, pb, ws, given, round == 1);
+          } else {
+            rc = twa_launch_panel_gram(ctx, W, D, ldw, j0, pb, ws, given, true);
+          }
+          if (rc) return rc;
+          rc = twa_launch_panel_apply(ctx, W, D, ldw, j0, pb, ws, round == 1 && absmax ? absmax + j0 : nullptr);
+          if (rc) return rc;
+        }
+        continue;
+      }
       for (int q = 0; q < pb; ++q) {
-        rc = launch_sumsq(ctx, W + (j0 + q) * ldw, D, ws, given + q);   // |a_j|^2 as given
+        rc = launch_sumsq(ctx, panel + q * ldw, D, ws, given + q);        // |a_j|^2 as given
         if (rc) return rc;
       }
       for (int round = 0; round < 2; ++round) {
         if (j0 > 0) {
-          rc = twa_launch_panel_project(ctx, W, D, ldw, j0, pb, ws);
+          rc = twa_launch_panel_project(ctx, W, D, ldw, j0, pb, ws, nullptr);
           if (rc) return rc;
-          rc = twa_launch_panel_lift(ctx, W, D, ldw, j0, pb, ws);
+          rc = twa_launch_panel_lift(ctx, W, D, ldw, j0, pb, ws, nullptr, false);
           if (rc) return rc;
-        }
-        if (ctx->tune_build_panel == 0) {
-          // Gram form inside the panel: all coefficients of the panel's own Gram-Schmidt from its
-          // Gram matrix in one pass, the new columns in a second; in the second round the rank test
-          // compares against the columns' norms as this round found them (1, or 0 for a column
-          // already found dependent).
-          rc = twa_launch_panel_gram(ctx, W, D, ldw, j0, pb, ws, given, round == 1);
-          if (rc) return rc;
-          continue;
         }
         for (int q = 0; q < pb; ++q) {
           const int k = j0 + q;
@@ -495,12 +622,62 @@ int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float
       }
     }
   }
+  // the schedules that finish a column with normalise_kernel take the maxima in a pass of their own
+  if (absmax && ctx->tune_build_panel != 0) {
+    rc = launch_absmax(ctx, W, D, ldw, n, absmax);
+    if (rc) return rc;
+  }
   P32_out->data = W;
   P32_out->scales = nullptr;
   P32_out->D = D;
   P32_out->col_stride = 4 * ldw;
   P32_out->n = n;
   P32_out->bits = 32;
+  return TWA_OK;
+}
+
+int check_quantised_target(const twa_basis* Pq, int bits, const void* ws) {
+  if (bits != 8 && bits != 4) return TWA_ERR_UNSUPPORTED;
+  if (!Pq || !Pq->data || !Pq->scales) return TWA_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(Pq->data) & 15) || (reinterpret_cast<uintptr_t>(ws) & 15)) return TWA_ERR_MISALIGNED;
+  return TWA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int twa_build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float* wbar_out,
+                    twa_basis* P32_out, void* ws, size_t ws_bytes) {
+  return build_basis(ctx, W, D, n, ldw, wbar_out, P32_out, ws, ws_bytes, nullptr);
+}
+
+int twa_build_quantized(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float* wbar_out,
+                        twa_basis* P32_out, const int* bits, int widths, twa_basis* Pq, void* ws,
+                        size_t ws_bytes) {
+  if (!ctx || !bits || !Pq || widths < 1 || widths > 8) return TWA_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < TWA_WS_BYTES) return TWA_ERR_WORKSPACE;
+  if (n < 1) return TWA_ERR_INVALID_ARG;
+  if (n > TWA_MAX_N) return TWA_ERR_UNSUPPORTED;
+  for (int k = 0; k < widths; ++k) {
+    const int rc = check_quantised_target(&Pq[k], bits[k], ws);
+    if (rc) return rc;
+  }
+  TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  unsigned* absmax = reinterpret_cast<unsigned*>(static_cast<char*>(ws) + TWA_WS_ABSMAX);
+  TWA_CUDA_OK(ctx, cudaMemsetAsync(absmax, 0, sizeof(unsigned) * n, ctx->stream));
+  int rc = build_basis(ctx, W, D, n, ldw, wbar_out, P32_out, ws, ws_bytes, absmax);
+  if (rc) return rc;
+  for (int k = 0; k < widths; ++k) {
+    rc = twa_launch_scales(ctx, absmax, n, bits[k], Pq[k].scales);
+    if (rc) return rc;
+    rc = launch_encode(ctx, P32_out, bits[k], &Pq[k]);
+    if (rc) return rc;
+    Pq[k].D = D;
+    Pq[k].col_stride = twa_basis_col_stride(D, bits[k]);
+    Pq[k].n = n;
+    Pq[k].bits = bits[k];
+  }
   return TWA_OK;
 }
 
@@ -522,22 +699,13 @@ int twa_quantize_basis(twa_ctx* ctx, const twa_basis* P32, int bits, twa_basis* 
   const float* P = static_cast<const float*>(P32->data);
   unsigned* absmax = reinterpret_cast<unsigned*>(static_cast<char*>(ws) + TWA_WS_ABSMAX);
   TWA_CUDA_OK(ctx, cudaMemsetAsync(absmax, 0, sizeof(unsigned) * n, ctx->stream));
-  int per_col = grid_for(ctx, D, BLOCK * 16, 8) / n;
-  if (per_col < 1) per_col = 1;
-  absmax_kernel<<<dim3(per_col, n), BLOCK, 0, ctx->stream>>>(P, D, ld, absmax);
-  TWA_CUDA_OK(ctx, cudaGetLastError());
+  rc = launch_absmax(ctx, P, D, ld, n, absmax);
+  if (rc) return rc;
   rc = twa_launch_scales(ctx, absmax, n, bits, Pq->scales);
   if (rc) return rc;
+  rc = launch_encode(ctx, P32, bits, Pq);
+  if (rc) return rc;
   const long long stride = twa_basis_col_stride(D, bits);
-  int eper = grid_for(ctx, stride / 16, BLOCK, 8) / n;
-  if (eper < 1) eper = 1;
-  if (bits == 8)
-    encode_kernel<8><<<dim3(eper, n), BLOCK, 0, ctx->stream>>>(
-        P, D, ld, Pq->scales, static_cast<unsigned char*>(Pq->data), stride);
-  else
-    encode_kernel<4><<<dim3(eper, n), BLOCK, 0, ctx->stream>>>(
-        P, D, ld, Pq->scales, static_cast<unsigned char*>(Pq->data), stride);
-  TWA_CUDA_OK(ctx, cudaGetLastError());
   Pq->D = D;
   Pq->col_stride = stride;
   Pq->n = n;

@@ -70,7 +70,10 @@ constexpr size_t TWA_WS_ABSMAX = TWA_WS_DPART + sizeof(double) * TWA_MAX_GRID;
 constexpr int TWA_HOST_CHUNKS = 16;                      // row chunks of twa_step_host at most
 constexpr size_t TWA_WS_CHUNK_COEF = TWA_WS_ABSMAX + sizeof(unsigned) * TWA_MAX_N;
                                                          // float [TWA_HOST_CHUNKS][TWA_MAX_N]  per-chunk projections
-constexpr size_t TWA_WS_BYTES = TWA_WS_CHUNK_COEF + sizeof(float) * TWA_HOST_CHUNKS * TWA_MAX_N;
+constexpr int TWA_PANEL_SUMSQ_BLOCKS = 256;              // blocks of the panel projection at most
+constexpr size_t TWA_WS_PANEL_SUMSQ = TWA_WS_CHUNK_COEF + sizeof(float) * TWA_HOST_CHUNKS * TWA_MAX_N;
+                                                         // double [TWA_PANEL_SUMSQ_BLOCKS][8]  squared norms of a panel's columns
+constexpr size_t TWA_WS_BYTES = TWA_WS_PANEL_SUMSQ + sizeof(double) * TWA_PANEL_SUMSQ_BLOCKS * 8;
 
 // ------------------------------------------------------------------------------------------
 // Streaming-kernel geometry
@@ -259,11 +262,15 @@ constexpr float TWA_MAGIC_I8 = 8388608.0f + 128.0f;
 constexpr float TWA_MAGIC_I4 = 8388608.0f + 8.0f;
 
 // One element of the quantiser: IEEE float32 quotient, round half to even, clamp to +-qmax.
+// qmax is an integer, so clamping first gives the same code; adding 1.5 * 2^23 then rounds the clamped
+// quotient to an integer, half to even, in the float adder and leaves the code in the low bits of the
+// sum's pattern (the rounding and conversion instructions run at a quarter of the adder's rate, and
+// three of them per element held the encoding pass at half the memory rate).  A NaN quotient clamps to
+// -qmax either way.
 __device__ __forceinline__ int twa_encode_one(float p, float s, float qmax) {
   if (s == 0.0f) return 0;
-  float q = rintf(__fdiv_rn(p, s));
-  q = fminf(fmaxf(q, -qmax), qmax);
-  return static_cast<int>(q);
+  const float q = fminf(fmaxf(__fdiv_rn(p, s), -qmax), qmax);
+  return __float_as_int(q + 12582912.0f) - 0x4B400000;
 }
 
 __device__ __forceinline__ float twa_bf16_lo(uint32_t pair) { return __uint_as_float(pair << 16); }
@@ -317,12 +324,20 @@ int twa_launch_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, float 
 int twa_check_basis(const twa_basis* P);
 // Panel steps of the blocked basis build on the float32 matrix W (columns of stride ldw):
 // C = Q^T A_p into the workspace, then A_p <- A_p - Q C; Q = columns 0..nq-1, A_p = the next pb <= 8.
-int twa_launch_panel_project(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws);
-int twa_launch_panel_lift(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws);
-// Gram-Schmidt among the panel's own columns in Gram form: the coefficients from the panel's Gram
-// matrix (one pass), then A_p <- A_p T (one pass); rank and finiteness tests against `given`.
+// sumsq_out (device, 8 doubles) or null: the squared norms of the panel's columns as the projection read them.
+int twa_launch_panel_project(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws,
+                             double* sumsq_out);
+// given (device, 8 doubles) or null: with it the update also takes the Gram matrix of the panel as stored
+// and leaves the factor of the panel's own Gram-Schmidt for twa_launch_panel_apply (rank and finiteness
+// tests against `given`, or against the Gram matrix's diagonal, which then replaces `given`).
+int twa_launch_panel_lift(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws, double* given,
+                          bool given_from_diagonal);
+// The same factor from a pass over the panel (for a panel the update did not just store).
 int twa_launch_panel_gram(twa_ctx* ctx, float* W, long long D, long long ldw, int j0, int pb, void* ws, double* given,
                           bool given_from_diagonal);
+// A_p <- A_p T; absmax (device, one word per panel column) or null: largest magnitudes stored, as bit patterns.
+int twa_launch_panel_apply(twa_ctx* ctx, float* W, long long D, long long ldw, int j0, int pb, void* ws,
+                           unsigned* absmax);
 // Validates the optimiser constants and fills the kernel-side Adam arguments (bias corrections for opt->step).
 int twa_adam_device_args(const twa_adam* opt, float* m, float* v, twa_adam_args* out);
 // scales[j] = absmax_j / qmax from the bit patterns of the column maxima; flags NaN/Inf

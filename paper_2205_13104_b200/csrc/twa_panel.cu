@@ -10,8 +10,11 @@
 //    lanes -> block -> last block to finish, float64 over blocks in block order.
 //  * update: a lane owns two rows of a block of 1024 rows and walks all nq columns as they stream past
 //    in chunks of 8, so there is no reduction at all.
-//  * inside the panel: the Gram-Schmidt coefficients from the panel's Gram matrix (one pass), the new
-//    columns as A_p T (a second pass).
+//  * inside the panel: the Gram-Schmidt coefficients from the panel's Gram matrix, the new columns as
+//    A_p T (one pass).  The Gram matrix is taken by the update kernel from the values it stores (float64
+//    products on the tensor pipe), the squared norms of the panel's columns as given by the projection
+//    kernel from the tiles it streams anyway; only the first panel, which has nothing before it, takes
+//    its Gram matrix in a pass of its own.
 #include <stdio.h>
 
 #include "twa_common.cuh"
@@ -37,6 +40,8 @@ struct PanelArgs {
   float* panel;                // first column of the panel
   float* partials;             // [grid][nq * PANEL]
   float* C;                    // [nq][PANEL]
+  double* sumsq_part;          // [grid][PANEL] squared norms of the panel's columns, or null
+  double* sumsq;               // [PANEL]
   unsigned* ticket;
   int* status;
   unsigned long long wait_limit_ns;
@@ -103,12 +108,22 @@ panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a)
     volatile int* abort_flag = &hdr->abort_flag;
     int s = 0;
     unsigned phase = 0;
+    // warp q < pb also sums the squares of panel column q (float64), rows beyond D being zero in the tile
+    const bool norm_warp = a.sumsq_part != nullptr && warp < a.pb;
+    double ss = 0.0;
     for (int tile = blockIdx.x; tile < a.tiles; tile += gridDim.x) {
       if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
         twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
         break;
       }
       const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
+      if (norm_warp) {
+        const float4 v = *reinterpret_cast<const float4*>(st + goff + warp * PCOL_BYTES);
+        ss = fma(static_cast<double>(v.x), static_cast<double>(v.x), ss);
+        ss = fma(static_cast<double>(v.y), static_cast<double>(v.y), ss);
+        ss = fma(static_cast<double>(v.z), static_cast<double>(v.z), ss);
+        ss = fma(static_cast<double>(v.w), static_cast<double>(v.w), ss);
+      }
       constexpr int GQ = 4;                               // panel columns in registers at a time
 #pragma unroll
       for (int part = 0; part < PANEL / GQ; ++part) {
@@ -144,6 +159,11 @@ panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a)
         if (lane == 0 && warp + k * PJWARPS < a.nq) cpart[(warp + k * PJWARPS) * PANEL + q] = v;
       }
     }
+    if (norm_warp) {
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, off);
+      if (lane == 0) a.sumsq_part[static_cast<size_t>(blockIdx.x) * PANEL + warp] = ss;
+    }
   }
   __syncthreads();
   const int tid = threadIdx.x, outs = a.nq * PANEL;
@@ -163,8 +183,64 @@ panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a)
       if (!isfinite(sum)) twa_set_status(a.status, TWA_ERR_NONFINITE, a.detail + (i % PANEL));
       a.C[i] = static_cast<float>(sum);
     }
+    if (a.sumsq_part && tid < a.pb) {
+      double sum = 0.0;
+      for (unsigned b = 0; b < gridDim.x; ++b) sum += __ldcg(&a.sumsq_part[static_cast<size_t>(b) * PANEL + tid]);
+      a.sumsq[tid] = sum;
+    }
     if (tid == 0) *a.ticket = 0u;
   }
+}
+
+constexpr int NPAIR = PANEL * (PANEL + 1) / 2;                     // 36
+__host__ __device__ constexpr int pair_index(int i, int j) { return j * (j + 1) / 2 + i; }   // i <= j
+
+// One thread: from the panel's Gram matrix G (upper triangle, G[pair_index(i, j)] = <a_i, a_j>) the
+// Gram-Schmidt coefficients R (the Cholesky factor of G) with the rank and finiteness tests of the
+// column-by-column schedule, and T = R^-1 ([column j][row i] at T[j * 8 + i]; a column found dependent
+// or non-finite becomes zero and is reported).  `given`: the squared norms the rank test compares
+// against; with given_from_diagonal they are G's diagonal, which is then also written there.
+__device__ __noinline__ void panel_factor(const double* G, int pb, double* given, int given_from_diagonal, double* T, int* status,
+                             int col0) {
+  double r[NPAIR], tm[PANEL][PANEL];
+  bool dead[PANEL];
+  for (int j = 0; j < PANEL; ++j)
+    for (int i = 0; i < PANEL; ++i) tm[i][j] = 0.0;
+  for (int j = 0; j < pb; ++j) {
+    double d = G[pair_index(j, j)];
+    const double na = given_from_diagonal ? d : given[j];
+    for (int k = 0; k < j; ++k) {
+      double c = 0.0;
+      if (!dead[k]) {
+        c = G[pair_index(k, j)];
+        for (int i = 0; i < k; ++i) c -= r[pair_index(i, k)] * r[pair_index(i, j)];
+        c /= r[pair_index(k, k)];
+      }
+      r[pair_index(k, j)] = c;
+      d -= c * c;
+    }
+    const double rjj = d > 0.0 ? sqrt(d) : 0.0;
+    dead[j] = false;
+    if (!isfinite(na) || !isfinite(d)) {
+      twa_set_status(status, TWA_ERR_NONFINITE, col0 + j);
+      dead[j] = true;
+    } else if (!(rjj > 1e-5 * sqrt(na))) {
+      twa_set_status(status, TWA_ERR_RANK_DEFICIENT, col0 + j);
+      dead[j] = true;
+    }
+    r[pair_index(j, j)] = dead[j] ? 1.0 : rjj;
+    if (!dead[j]) {
+      // T[:, j] = (e_j - sum_{k<j} r_kj T[:, k]) / r_jj
+      for (int i = 0; i <= j; ++i) {
+        double v = i == j ? 1.0 : 0.0;
+        for (int k = i; k < j; ++k) v -= r[pair_index(k, j)] * tm[i][k];
+        tm[i][j] = v / rjj;
+      }
+    }
+    if (given_from_diagonal) given[j] = na;
+  }
+  for (int j = 0; j < PANEL; ++j)
+    for (int i = 0; i < PANEL; ++i) T[j * PANEL + i] = tm[i][j];
 }
 
 // Update kernel.  A block walks blocks of 1024 rows; a lane owns two neighbouring rows of the block
@@ -174,6 +250,12 @@ panel_project_kernel(const __grid_constant__ CUtensorMap map, const PanelArgs a)
 // warp consumes every stage, in order: the plain ring protocol, no reduction anywhere.  Two rows
 // per lane halve the shared-memory reads of the coefficients per product (with one row the kernel
 // ran at 69 % issue utilisation, a third of it those reads).
+//
+// With a.gpart set the kernel also leaves the Gram matrix of the panel as it stores it, and the factor
+// T of panel_factor: a warp writes its 64 rows x 8 columns of new values back into the stage, reads
+// them as operands of 16 float64 tensor-pipe products (4 rows each; the 8 x 8 matrix in two registers
+// per lane), the warps' matrices are added in warp order, the blocks' in block order by the block that
+// finishes last, which factorises.  That is the panel's Gram pass without reading the panel again.
 constexpr int LROWS_LANE = 2;
 constexpr int LROWS_BLOCK = PWARPS * 32 * LROWS_LANE;        // 1024 rows per row block
 constexpr int LCHUNK = PANEL;                                // columns per stage
@@ -187,7 +269,21 @@ struct PanelLiftArgs {
   const float* C;
   int* status;
   unsigned long long wait_limit_ns;
+  // Gram matrix of the stored panel and its factor (gpart == null: not wanted)
+  double* gpart;               // [grid][64]
+  double* given;
+  int given_from_diagonal, col0;
+  double* T;
+  unsigned* ticket;
 };
+
+// d += a (8 x 4, row-major) * b (4 x 8, column-major) in float64 on the tensor pipe: lane l holds
+// a[l >> 2][l & 3], b[l & 3][l >> 2] and d[l >> 2][2 * (l & 3) + {0, 1}].
+__device__ __forceinline__ void panel_dmma(double (&d)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+               : "+d"(d[0]), "+d"(d[1])
+               : "d"(a), "d"(b));
+}
 
 __global__ void __launch_bounds__(PTHREADS, 1)
 panel_lift_kernel(const __grid_constant__ CUtensorMap map, const PanelLiftArgs a) {
@@ -238,6 +334,10 @@ panel_lift_kernel(const __grid_constant__ CUtensorMap map, const PanelLiftArgs a
   // element (column c of the chunk, row r of the block) sits at ((r >> 8) * 8 + c) * 256 + (r & 255)
   const int r = (warp * 32 + lane) * LROWS_LANE;
   const int base = (r >> 8) * LCHUNK * 256 + (r & 255);
+  // Gram operands: lane (column c = lane >> 2, k = lane & 3) takes rows 16 t + 4 k .. + 3 of the warp's 64
+  const int gram_base = ((warp * 64) >> 8) * LCHUNK * 256 + ((warp * 64) & 255) + (lane >> 2) * 256 + (lane & 3) * 4;
+  const bool want_gram = a.gpart != nullptr;
+  double gacc[2] = {0.0, 0.0};
   int it = 0;
   bool alive = true;
   for (int rb = blockIdx.x; rb < a.row_blocks && alive; rb += gridDim.x) {
@@ -273,23 +373,81 @@ panel_lift_kernel(const __grid_constant__ CUtensorMap map, const PanelLiftArgs a
       } else {
         float2 old[PANEL];
 #pragma unroll
-        for (int q = 0; q < PANEL; ++q) old[q] = *reinterpret_cast<const float2*>(st + q * 256);
-        __syncwarp();
-        if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
+        for (int q = 0; q < PANEL; ++q) {
+          old[q] = *reinterpret_cast<const float2*>(st + q * 256);
+          old[q].x -= acc0[q];
+          old[q].y -= acc1[q];
+        }
+        if (want_gram) {
+          // the new values (zero in rows beyond D and in columns beyond pb, where everything read was
+          // zero) go back to the lane's own places; the warp's 64 x 8 patch is its alone
+          float* stw = const_cast<float*>(st);
+#pragma unroll
+          for (int q = 0; q < PANEL; ++q) *reinterpret_cast<float2*>(stw + q * 256) = old[q];
+        }
         const long long row = static_cast<long long>(rb) * LROWS_BLOCK + r;
         if (row + 1 < a.D) {
 #pragma unroll
           for (int q = 0; q < PANEL; ++q)
-            if (q < a.pb)
-              *reinterpret_cast<float2*>(a.panel + q * a.ldw + row) = make_float2(old[q].x - acc0[q], old[q].y - acc1[q]);
+            if (q < a.pb) *reinterpret_cast<float2*>(a.panel + q * a.ldw + row) = old[q];
         } else if (row < a.D) {
 #pragma unroll
           for (int q = 0; q < PANEL; ++q)
-            if (q < a.pb) a.panel[q * a.ldw + row] = old[q].x - acc0[q];
+            if (q < a.pb) a.panel[q * a.ldw + row] = old[q].x;
         }
+        if (want_gram) {
+          __syncwarp();
+          const float* gp = reinterpret_cast<const float*>(ring + static_cast<size_t>(s) * LSTAGE_BYTES) + gram_base;
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            const float4 gv = *reinterpret_cast<const float4*>(gp + 16 * t);
+            const double x0 = gv.x, x1 = gv.y, x2 = gv.z, x3 = gv.w;
+            panel_dmma(gacc, x0, x0);
+            panel_dmma(gacc, x1, x1);
+            panel_dmma(gacc, x2, x2);
+            panel_dmma(gacc, x3, x3);
+          }
+          twa_fence_proxy_async();       // the writes above before the copy that refills the stage
+        }
+        __syncwarp();
+        if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
       }
     }
   }
+  if (!want_gram) return;
+  // The 16 consumer warps only from here on (the producer warp has left): barrier 1, 512 threads.
+  // Every stage this block was sent has been consumed, so the ring is free to hold the warps' matrices.
+  constexpr int CONSUMERS = PWARPS * 32;
+  double* wsum = reinterpret_cast<double*>(ring);                       // [PWARPS][64]
+  __shared__ double Gs[NPAIR];
+  __shared__ int last;
+  twa_named_barrier(1, CONSUMERS);                                      // the slowest warp has read its last stage
+  wsum[warp * 64 + (lane >> 2) * 8 + 2 * (lane & 3)] = gacc[0];
+  wsum[warp * 64 + (lane >> 2) * 8 + 2 * (lane & 3) + 1] = gacc[1];
+  twa_named_barrier(1, CONSUMERS);
+  if (threadIdx.x < 64) {
+    double t = 0.0;
+    for (int w = 0; w < PWARPS; ++w) t += wsum[w * 64 + threadIdx.x];
+    a.gpart[static_cast<size_t>(blockIdx.x) * 64 + threadIdx.x] = t;
+  }
+  __threadfence();
+  twa_named_barrier(1, CONSUMERS);
+  if (threadIdx.x == 0) last = (atomicAdd(a.ticket, 1u) == gridDim.x - 1);
+  twa_named_barrier(1, CONSUMERS);
+  if (!last) return;
+  __threadfence();
+  if (threadIdx.x < 64) {
+    const int i = threadIdx.x >> 3, j = threadIdx.x & 7;
+    if (i <= j) {
+      double t = 0.0;
+      for (unsigned b = 0; b < gridDim.x; ++b) t += __ldcg(&a.gpart[static_cast<size_t>(b) * 64 + threadIdx.x]);
+      Gs[pair_index(i, j)] = t;
+    }
+  }
+  twa_named_barrier(1, CONSUMERS);
+  if (threadIdx.x != 0) return;
+  *a.ticket = 0u;
+  panel_factor(Gs, a.pb, a.given, a.given_from_diagonal, a.T, a.status, a.col0);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -303,8 +461,6 @@ panel_lift_kernel(const __grid_constant__ CUtensorMap map, const PanelLiftArgs a
 // reported) and leaves T; a second pass writes A_p T.  Twelve column passes per panel and round
 // instead of the 52 of the column sweeps.
 constexpr int GRAM_BLOCK = 256;
-constexpr int NPAIR = PANEL * (PANEL + 1) / 2;                     // 36
-__host__ __device__ constexpr int pair_index(int i, int j) { return j * (j + 1) / 2 + i; }   // i <= j
 
 __global__ void __launch_bounds__(GRAM_BLOCK, 2) panel_gram_kernel(const float* __restrict__ A0, long long ld, int pb,
                                                                long long D, double* __restrict__ gpart,
@@ -374,63 +530,33 @@ __global__ void __launch_bounds__(GRAM_BLOCK, 2) panel_gram_kernel(const float* 
   __syncthreads();
   if (threadIdx.x != 0) return;
   *ticket = 0u;
-  // R (upper triangular, r[pair_index(k, j)] = r_kj) and T = R^-1, column by column
-  double r[NPAIR], tm[PANEL][PANEL];
-  bool dead[PANEL];
-  for (int j = 0; j < PANEL; ++j)
-    for (int i = 0; i < PANEL; ++i) tm[i][j] = 0.0;
-  for (int j = 0; j < pb; ++j) {
-    double d = G[pair_index(j, j)];
-    const double na = given_from_diagonal ? d : given[j];
-    for (int k = 0; k < j; ++k) {
-      double c = 0.0;
-      if (!dead[k]) {
-        c = G[pair_index(k, j)];
-        for (int i = 0; i < k; ++i) c -= r[pair_index(i, k)] * r[pair_index(i, j)];
-        c /= r[pair_index(k, k)];
-      }
-      r[pair_index(k, j)] = c;
-      d -= c * c;
-    }
-    const double rjj = d > 0.0 ? sqrt(d) : 0.0;
-    dead[j] = false;
-    if (!isfinite(na) || !isfinite(d)) {
-      twa_set_status(status, TWA_ERR_NONFINITE, col0 + j);
-      dead[j] = true;
-    } else if (!(rjj > 1e-5 * sqrt(na))) {
-      twa_set_status(status, TWA_ERR_RANK_DEFICIENT, col0 + j);
-      dead[j] = true;
-    }
-    r[pair_index(j, j)] = dead[j] ? 1.0 : rjj;
-    if (!dead[j]) {
-      // T[:, j] = (e_j - sum_{k<j} r_kj T[:, k]) / r_jj
-      for (int i = 0; i <= j; ++i) {
-        double v = i == j ? 1.0 : 0.0;
-        for (int k = i; k < j; ++k) v -= r[pair_index(k, j)] * tm[i][k];
-        tm[i][j] = v / rjj;
-      }
-    }
-    if (given_from_diagonal) given[j] = na;
-  }
-  for (int j = 0; j < PANEL; ++j)
-    for (int i = 0; i < PANEL; ++i) T[j * PANEL + i] = tm[i][j];
+  panel_factor(G, pb, given, given_from_diagonal, T, status, col0);
 }
 
-// A_p <- A_p T (T upper triangular, [column j][row i] at T[j * 8 + i]); float64 sums, one rounding per stored value.
-__global__ void __launch_bounds__(GRAM_BLOCK) panel_apply_kernel(float* __restrict__ A0, long long ld, int pb, long long D,
-                                                                const double* __restrict__ T) {
+// A_p <- A_p T (T upper triangular, [column j][row i] at T[j * 8 + i]); float64 sums, one rounding per stored
+// value.  Column j needs columns 0 .. j only, so the columns are replaced from the last to the first in
+// the registers that hold them.  With `absmax` the largest magnitude stored in each column is folded
+// into absmax[j] (bit patterns of |x|: NaN and Inf compare above every finite value).
+__global__ void __launch_bounds__(GRAM_BLOCK, 2) panel_apply_kernel(float* __restrict__ A0, long long ld, int pb, long long D,
+                                                                   const double* __restrict__ T,
+                                                                   unsigned* __restrict__ absmax) {
   __shared__ double Ts[PANEL * PANEL];
+  __shared__ unsigned mx[PANEL];
   if (threadIdx.x < PANEL * PANEL) Ts[threadIdx.x] = T[threadIdx.x];
+  if (threadIdx.x < PANEL) mx[threadIdx.x] = 0u;
   __syncthreads();
+  unsigned m[PANEL];
+#pragma unroll
+  for (int j = 0; j < PANEL; ++j) m[j] = 0u;
   const long long nvec = D >> 2;
   for (long long t = blockIdx.x * static_cast<long long>(GRAM_BLOCK) + threadIdx.x; t < nvec;
        t += static_cast<long long>(gridDim.x) * GRAM_BLOCK) {
-    float4 x[PANEL], y[PANEL];
+    float4 x[PANEL];
 #pragma unroll
     for (int j = 0; j < PANEL; ++j)
       x[j] = j < pb ? __ldcs(reinterpret_cast<const float4*>(A0 + j * ld) + t) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int j = 0; j < PANEL; ++j) {
+    for (int j = PANEL - 1; j >= 0; --j) {
       double a = 0.0, b = 0.0, c = 0.0, d = 0.0;
 #pragma unroll
       for (int i = 0; i <= j; ++i) {
@@ -440,22 +566,41 @@ __global__ void __launch_bounds__(GRAM_BLOCK) panel_apply_kernel(float* __restri
         c = fma(static_cast<double>(x[i].z), w, c);
         d = fma(static_cast<double>(x[i].w), w, d);
       }
-      y[j] = make_float4(static_cast<float>(a), static_cast<float>(b), static_cast<float>(c), static_cast<float>(d));
+      x[j] = make_float4(static_cast<float>(a), static_cast<float>(b), static_cast<float>(c), static_cast<float>(d));
+      if (j < pb) {
+        __stcs(reinterpret_cast<float4*>(A0 + j * ld) + t, x[j]);
+        m[j] = max(max(m[j], __float_as_uint(x[j].x) & 0x7FFFFFFFu), max(__float_as_uint(x[j].y) & 0x7FFFFFFFu,
+                   max(__float_as_uint(x[j].z) & 0x7FFFFFFFu, __float_as_uint(x[j].w) & 0x7FFFFFFFu)));
+      }
     }
-#pragma unroll
-    for (int j = 0; j < PANEL; ++j)
-      if (j < pb) reinterpret_cast<float4*>(A0 + j * ld)[t] = y[j];
   }
   if (blockIdx.x == 0 && threadIdx.x < (D & 3)) {
     const long long r = (nvec << 2) + threadIdx.x;
     double x[PANEL];
+#pragma unroll
     for (int j = 0; j < PANEL; ++j) x[j] = j < pb ? static_cast<double>(A0[j * ld + r]) : 0.0;
-    for (int j = 0; j < pb; ++j) {
+#pragma unroll
+    for (int j = 0; j < PANEL; ++j) {
       double a = 0.0;
+#pragma unroll
       for (int i = 0; i <= j; ++i) a = fma(x[i], Ts[j * PANEL + i], a);
-      A0[j * ld + r] = static_cast<float>(a);
+      const float y = static_cast<float>(a);
+      if (j < pb) {
+        A0[j * ld + r] = y;
+        m[j] = max(m[j], __float_as_uint(y) & 0x7FFFFFFFu);
+      }
     }
   }
+  if (!absmax) return;
+#pragma unroll
+  for (int j = 0; j < PANEL; ++j) {
+    unsigned v = m[j];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, off));
+    if ((threadIdx.x & 31) == 0 && j < pb) atomicMax(&mx[j], v);
+  }
+  __syncthreads();
+  if (threadIdx.x < pb) atomicMax(&absmax[threadIdx.x], mx[threadIdx.x]);
 }
 
 int encode_panel_map(twa_ctx* ctx, const float* W, long long D, long long ldw, int cols, CUtensorMap* map) {
@@ -496,10 +641,13 @@ int fill_args(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb
   const size_t region_floats = static_cast<size_t>(TWA_MAX_GRID) * TWA_MAX_N;
   a->partials = region;
   a->C = region + region_floats - 1040;
+  a->sumsq_part = nullptr;
+  a->sumsq = nullptr;
   a->ticket = ctx->d_ticket;
   a->status = ctx->d_status;
   a->wait_limit_ns = ctx->wait_limit_ns;
   int g = ctx->sm_count < a->tiles ? ctx->sm_count : a->tiles;
+  if (g > TWA_PANEL_SUMSQ_BLOCKS) g = TWA_PANEL_SUMSQ_BLOCKS;
   const size_t per_block = static_cast<size_t>(nq) * PANEL;
   if (static_cast<size_t>(g) * per_block > region_floats - 1040) g = static_cast<int>((region_floats - 1040) / per_block);
   *grid = g;
@@ -519,11 +667,16 @@ int launch_panel_project(twa_ctx* ctx, const CUtensorMap& map, const PanelArgs& 
 
 }  // namespace
 
-int twa_launch_panel_project(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws) {
+int twa_launch_panel_project(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws,
+                             double* sumsq_out) {
   PanelArgs a;
   int grid, smem;
   int rc = fill_args(ctx, W, D, ldw, nq, pb, ws, &a, &grid, &smem);
   if (rc) return rc;
+  if (sumsq_out) {
+    a.sumsq_part = reinterpret_cast<double*>(static_cast<char*>(ws) + TWA_WS_PANEL_SUMSQ);
+    a.sumsq = sumsq_out;
+  }
   CUtensorMap map;
   rc = encode_panel_map(ctx, W, D, ldw, nq + pb, &map);
   if (rc) return rc;
@@ -540,7 +693,8 @@ int twa_launch_panel_project(twa_ctx* ctx, float* W, long long D, long long ldw,
   }
 }
 
-int twa_launch_panel_lift(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws) {
+int twa_launch_panel_lift(twa_ctx* ctx, float* W, long long D, long long ldw, int nq, int pb, void* ws, double* given,
+                          bool given_from_diagonal) {
   if (nq < LCHUNK || (nq % LCHUNK) != 0 || pb < 1 || pb > PANEL || nq + pb > TWA_MAX_N) return TWA_ERR_INVALID_ARG;
   PanelLiftArgs a;
   a.D = D;
@@ -558,6 +712,14 @@ int twa_launch_panel_lift(twa_ctx* ctx, float* W, long long D, long long ldw, in
   a.C = region + static_cast<size_t>(TWA_MAX_GRID) * TWA_MAX_N - 1040;      // where the projection left it
   a.status = ctx->d_status;
   a.wait_limit_ns = ctx->wait_limit_ns;
+  // with `given`: the Gram matrix of the stored panel, per block at the start of the float region (the
+  // coefficients this kernel reads sit at its end), and its factor where twa_launch_panel_apply reads it
+  a.gpart = given ? reinterpret_cast<double*>(static_cast<char*>(ws) + TWA_WS_PARTIALS) : nullptr;
+  a.given = given;
+  a.given_from_diagonal = given_from_diagonal ? 1 : 0;
+  a.col0 = nq;
+  a.T = reinterpret_cast<double*>(static_cast<char*>(ws) + TWA_WS_COEF);
+  a.ticket = ctx->d_ticket;
   // boxes of 256 rows x 8 columns over the matrix's first nq + pb columns (columns past them read as zero)
   CUtensorMap map;
   cuuint64_t dims[2] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(nq + pb)};
@@ -582,9 +744,33 @@ int twa_launch_panel_lift(twa_ctx* ctx, float* W, long long D, long long ldw, in
   return TWA_OK;
 }
 
-// Orthonormalises the panel's pb <= 8 columns among themselves in Gram form (see panel_gram_kernel).
-// `given`: device array of 8 doubles, the squared norms the rank test compares against; with
-// given_from_diagonal they are taken from (and written as) the diagonal of this pass's Gram matrix.
+namespace {
+int apply_grid(const twa_ctx* ctx, long long D) {
+  long long g = (D / 4 + GRAM_BLOCK - 1) / GRAM_BLOCK;
+  const long long cap = static_cast<long long>(ctx->sm_count) * 4;
+  if (g > cap) g = cap;
+  if (g > TWA_MAX_GRID) g = TWA_MAX_GRID;
+  if (g < 1) g = 1;
+  return static_cast<int>(g);
+}
+}  // namespace
+
+// A_p <- A_p T with the factor twa_launch_panel_lift or the Gram pass left in the workspace; with `absmax`
+// (device, one word per column of the panel) the largest magnitudes stored are folded into it.
+int twa_launch_panel_apply(twa_ctx* ctx, float* W, long long D, long long ldw, int j0, int pb, void* ws,
+                           unsigned* absmax) {
+  if (pb < 1 || pb > PANEL) return TWA_ERR_INVALID_ARG;
+  const double* T = reinterpret_cast<const double*>(static_cast<const char*>(ws) + TWA_WS_COEF);
+  panel_apply_kernel<<<apply_grid(ctx, D), GRAM_BLOCK, 0, ctx->stream>>>(W + static_cast<long long>(j0) * ldw, ldw, pb, D, T,
+                                                                        absmax);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+// The Gram pass of a panel that was not just stored by twa_launch_panel_lift (see panel_gram_kernel):
+// leaves the factor for twa_launch_panel_apply.  `given`: device array of 8 doubles, the squared norms the
+// rank test compares against; with given_from_diagonal they are taken from (and written as) the diagonal
+// of this pass's Gram matrix.
 int twa_launch_panel_gram(twa_ctx* ctx, float* W, long long D, long long ldw, int j0, int pb, void* ws, double* given,
                           bool given_from_diagonal) {
   if (pb < 1 || pb > PANEL) return TWA_ERR_INVALID_ARG;
@@ -592,17 +778,10 @@ int twa_launch_panel_gram(twa_ctx* ctx, float* W, long long D, long long ldw, in
   double* gpart = reinterpret_cast<double*>(w + TWA_WS_PARTIALS);           // [grid][36], start of the float region
   double* T = reinterpret_cast<double*>(w + TWA_WS_COEF);                    // 64 doubles
   static_assert(sizeof(float) * TWA_MAX_N >= sizeof(double) * PANEL * PANEL, "coefficient area too small for T");
-  long long g = (D / 4 + GRAM_BLOCK - 1) / GRAM_BLOCK;
-  const long long cap = static_cast<long long>(ctx->sm_count) * 4;
-  if (g > cap) g = cap;
-  if (g > TWA_MAX_GRID) g = TWA_MAX_GRID;
-  if (g < 1) g = 1;
-  const int grid = static_cast<int>(g);
   float* A0 = W + static_cast<long long>(j0) * ldw;
-  panel_gram_kernel<<<grid, GRAM_BLOCK, 0, ctx->stream>>>(A0, ldw, pb, D, gpart, given, given_from_diagonal ? 1 : 0, T,
-                                                          ctx->d_ticket, ctx->d_status, j0);
-  TWA_CUDA_OK(ctx, cudaGetLastError());
-  panel_apply_kernel<<<grid, GRAM_BLOCK, 0, ctx->stream>>>(A0, ldw, pb, D, T);
+  panel_gram_kernel<<<apply_grid(ctx, D), GRAM_BLOCK, 0, ctx->stream>>>(A0, ldw, pb, D, gpart, given,
+                                                                       given_from_diagonal ? 1 : 0, T, ctx->d_ticket,
+                                                                       ctx->d_status, j0);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
 }

@@ -44,7 +44,7 @@ EXPORTS = [
     "twa_create", "twa_destroy", "twa_get_status", "twa_clear_status", "twa_strerror",
     "twa_last_error", "twa_set_tuning", "twa_selftest_wait", "twa_profile_enable", "twa_profile_read",
     "twa_basis_col_stride", "twa_basis_bytes",
-    "twa_workspace_bytes", "twa_build_basis", "twa_build_workspace_bytes", "twa_build_begin",
+    "twa_workspace_bytes", "twa_build_basis", "twa_build_quantized", "twa_build_workspace_bytes", "twa_build_begin",
     "twa_build_feed", "twa_build_end_pass", "twa_mean", "twa_quantize_basis",
     "twa_basis_export", "twa_basis_import", "twa_project", "twa_lift", "twa_step",
     "twa_step_host", "twa_step_adam", "twa_cosine_lr", "twa_weighted_average", "twa_layered_step_adam", "twa_project_batch", "twa_project_batch_group", "twa_layered_workspace_bytes", "twa_layered_rows", "twa_layered_basis_bytes",
@@ -168,6 +168,7 @@ def load():
         "twa_basis_bytes": (szt, [i64, i32, i32]),
         "twa_workspace_bytes": (szt, [i64, i32, i32]),
         "twa_build_basis": (i32, [vp, vp, i64, i32, i64, vp, bp, vp, szt]),
+        "twa_build_quantized": (i32, [vp, vp, i64, i32, i64, vp, bp, ctypes.POINTER(i32), i32, bp, vp, szt]),
         "twa_build_workspace_bytes": (szt, [i32]),
         "twa_build_begin": (i32, [vp, i64, i32, vp, vp, szt]),
         "twa_build_feed": (i32, [vp, i32, vp, i64, i64, i64, bp, vp, i64]),
@@ -347,6 +348,27 @@ def twa_build_basis(ctx, W, D, wbar_out, ws):
     return Basis(desc, W, None)
 
 
+def twa_build_quantized(ctx, W, D, wbar_out, bits_list, ws, out=None):
+    """twa_build_basis and one quantised basis per entry of bits_list in one call; returns
+    (P32, [Pq, ...]).  out: a list of Basis from new_quantised_basis to fill (None: allocated here)."""
+    assert W.dtype == torch.float32 and W.is_contiguous()
+    n, ldw = W.shape
+    k = len(bits_list)
+    if out is None:
+        out = [new_quantised_basis(int(D), int(n), int(b), W.device) for b in bits_list]
+    desc32 = twa_basis()
+    descs = (twa_basis * k)()
+    bits = (ctypes.c_int * k)(*[int(b) for b in bits_list])
+    for i in range(k):
+        descs[i].data, descs[i].scales = out[i].desc.data, out[i].desc.scales
+    rc = load().twa_build_quantized(ctx, _ptr(W), int(D), int(n), int(ldw), _ptr(wbar_out),
+                                    ctypes.byref(desc32), bits, k, descs, _ptr(ws), ws.numel())
+    _check(rc, "twa_build_quantized", ctx)
+    for i in range(k):
+        ctypes.memmove(ctypes.byref(out[i].desc), ctypes.byref(descs[i]), ctypes.sizeof(twa_basis))
+    return Basis(desc32, W, None), out
+
+
 def twa_build_workspace_bytes(n):
     return int(load().twa_build_workspace_bytes(int(n)))
 
@@ -411,12 +433,14 @@ def _new_quantised(D, n, bits, device):
     return desc, data, scales
 
 
-def twa_quantize_basis(ctx, P32, bits, ws):
-    desc, data, scales = _new_quantised(P32.D, P32.n, bits, P32.data.device)
-    rc = load().twa_quantize_basis(ctx, ctypes.byref(P32.desc), int(bits), ctypes.byref(desc),
+def twa_quantize_basis(ctx, P32, bits, ws, out=None):
+    """out: a Basis from new_quantised_basis to fill (None: buffers are allocated here)."""
+    if out is None:
+        out = new_quantised_basis(P32.D, P32.n, bits, P32.data.device)
+    rc = load().twa_quantize_basis(ctx, ctypes.byref(P32.desc), int(bits), ctypes.byref(out.desc),
                                    _ptr(ws), ws.numel())
     _check(rc, "twa_quantize_basis", ctx)
-    return Basis(desc, data, scales)
+    return out
 
 
 def twa_basis_export(ctx, Pq):

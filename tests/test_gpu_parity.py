@@ -110,6 +110,45 @@ def test_quantize_ties_round_to_even(env):
 
 
 @pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("absmax", [1.0, 0.0123, 3.3e-3, 96.7, 2.9e-37, 1.1e-44, 2.5e38])
+def test_quantize_near_half_integers_matches_the_ieee_quotient(env, bits, absmax):
+    """Elements whose quotient p / s sits on, or within a few ulps of, a half-integer: the code then
+    hangs on the last bit of the IEEE float32 quotient (what the oracle rounds), for scales that are
+    not powers of two, for a scale so small that it is subnormal, and for a huge one."""
+    ctx, ws = env
+    qmax = 127 if bits == 8 else 7
+    am = np.float32(absmax)
+    sc = np.float32(am) / np.float32(qmax)
+    ks = np.arange(-qmax, qmax, dtype=np.float64) + 0.5
+    with np.errstate(over="ignore", under="ignore"):
+        base = (ks * np.float64(sc)).astype(np.float32)
+        vals = [base]
+        for _ in range(6):
+            vals.append(np.nextafter(vals[-1], np.float32(np.inf)))
+        lo = base
+        for _ in range(6):
+            lo = np.nextafter(lo, np.float32(-np.inf))
+            vals.append(lo)
+    col = np.concatenate(vals + [np.array([am, -am, 0.0], dtype=np.float32)])
+    col = col[np.abs(col) <= am]
+    D = col.size
+    P = torch.zeros((2, inputs.padded_ld(D, 4)), dtype=torch.float32, device=DEV)
+    P[0, :D] = torch.from_numpy(col).to(DEV)
+    P[1, :D] = torch.from_numpy(col[::-1].copy()).to(DEV)
+    Pq = twa.twa_quantize_basis(ctx, twa.basis_from_tensor(P, D), bits, ws)
+    status_ok(ctx)
+    codes_g, s_g = twa.twa_basis_export(ctx, Pq)
+    codes_o, s_o = orc.quantize(np.asfortranarray(host_cols(P, D)), bits)
+    assert s_o[0] == sc
+    np.testing.assert_array_equal(s_g.cpu().numpy(), s_o)
+    np.testing.assert_array_equal(codes_g.cpu().numpy(), orc.pack_codes(codes_o, bits))
+    # the case is what it claims: many of these quotients round differently from their neighbours one ulp away
+    if sc > 1e-40:
+        c = codes_o[: base.size * 13, 0].reshape(13, base.size)
+        assert np.count_nonzero(c.max(axis=0) != c.min(axis=0)) >= base.size // 2
+
+
+@pytest.mark.parametrize("bits", [8, 4])
 def test_export_import_roundtrip(env, bits):
     ctx, ws = env
     D, n = 7001, 5
@@ -599,6 +638,40 @@ def test_panel_build_agrees_with_column_build_and_oracle(env, D, n, step):
     # the schedules reach the same vectors to the accuracy each reaches the oracle
     for mode in (0, 2):
         assert np.max(np.linalg.norm(out[mode] - out[1], axis=0)) <= 20 * kappa * np.finfo(np.float32).eps, mode
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("D,n", [(1, 1), (5003, 3), (70001, 33), (300007, 20), (40001, 128)])
+def test_build_quantized_equals_build_then_quantize_bit_for_bit(env, D, n, mode):
+    """One call for mean, basis and both storage widths: the column maxima it takes while the build
+    writes its last pass are those a pass over the finished basis finds, so basis, scales and codes
+    are those of twa_build_basis followed by twa_quantize_basis -- and the codes are the oracle's
+    quantiser applied to that basis."""
+    ctx, ws = env
+    ld = inputs.padded_ld(D, 4)
+    wbar_a, wbar_b = torch.empty(D, device=DEV), torch.empty(D, device=DEV)
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_BUILD_PANEL, mode)
+    try:
+        Wa = inputs.trajectory_candidates(D, n, 0.005, 0.001, 77, DEV, ld=ld)
+        P32a = twa.twa_build_basis(ctx, Wa, D, wbar_a, ws)
+        qa = [twa.twa_quantize_basis(ctx, P32a, bits, ws) for bits in (8, 4)]
+        Wb = inputs.trajectory_candidates(D, n, 0.005, 0.001, 77, DEV, ld=ld)
+        P32b, qb = twa.twa_build_quantized(ctx, Wb, D, wbar_b, [8, 4], ws)
+    finally:
+        twa.twa_set_tuning(ctx, twa.TWA_TUNE_BUILD_PANEL, 0)
+    status_ok(ctx)
+    assert torch.equal(Wa, Wb) and torch.equal(wbar_a, wbar_b)
+    assert (P32b.D, P32b.n, P32b.bits, P32b.col_stride) == (D, n, 32, 4 * ld)
+    P_h = host_cols(Wb, D)
+    for bits, A, B in zip((8, 4), qa, qb):
+        assert (B.D, B.n, B.bits, B.col_stride) == (D, n, bits, twa.twa_basis_col_stride(D, bits))
+        ca, sa = twa.twa_basis_export(ctx, A)
+        cb, sb = twa.twa_basis_export(ctx, B)
+        assert torch.equal(sa, sb) and torch.equal(ca, cb)
+        assert torch.equal(A.data, B.data)                    # padding included
+        codes_o, scales_o = orc.quantize(np.asfortranarray(P_h), bits)
+        np.testing.assert_array_equal(sb.cpu().numpy(), scales_o)
+        np.testing.assert_array_equal(cb.cpu().numpy(), orc.pack_codes(codes_o, bits))
 
 
 @pytest.fixture(params=[0, 2], ids=["gram-in-panel", "sweeps-in-panel"])
