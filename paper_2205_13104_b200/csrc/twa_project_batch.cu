@@ -40,10 +40,22 @@ __device__ __forceinline__ void pair_digit_store(unsigned char* digw, int set, i
   d[2 * BYTE_DIGIT_STRIDE] = static_cast<unsigned char>(b >> 16);
 }
 
+// B fragments of a pair: result columns 0-3 = u0, u1, u2, ones of the pair's first gradient, 4-7 of its
+// second; with 4-bit codes registers 2, 3 hold the odd rows' digits.
+template <int BITS>
+__device__ __forceinline__ void load_pair_fragments(uint32_t dig_addr, uint32_t (&bf)[4]) {
+  if (BITS == 8) {
+    ldmatrix_x2(dig_addr, bf[0], bf[1]);
+  } else {
+    ldmatrix_x4(dig_addr, bf);
+  }
+}
+
 struct BatchArgs {
   long long D;
   int n, stages, tiles, b0, batch;
   unsigned stage_bytes, g_off, tx_bytes, scratch_off;
+  unsigned pair_stride;         // bytes between the digit matrices of a warp's pairs; 0: one set, reused pair after pair
   const float* scales;
   float* partials;              // [grid][NB][n]
   unsigned* ticket;
@@ -52,43 +64,29 @@ struct BatchArgs {
   unsigned long long wait_limit_ns;
 };
 
+// The block has no warp of its own for the copies (16 warps, four per scheduler, may use 128
+// registers a thread; a 17th would cap every thread at 96, and this kernel's 2 x NP x MT float sums
+// then leave too few to overlap the conversions).  Lane 0 of the last warp fills the ring: all stages
+// before the loop, and stage s again right after its own warp has released it, once the other 15
+// have too.  The warps run in step with the ring anyway, so that wait is short, and the other stages
+// of the ring are in flight or have landed meanwhile.
 template <int KT, int NB>
-__device__ __forceinline__ void producer_loop_batch(twa_smem_header* hdr, unsigned char* ring,
-                                                    const CUtensorMap* map_p, const CUtensorMap* map_g,
-                                                    const BatchArgs& a, int tile_rows, int g_elem_bytes) {
-  twa_prefetch_tensormap(map_p);
-  twa_prefetch_tensormap(map_g);
-  volatile int* abort_flag = &hdr->abort_flag;
-  int s = 0, issued = 0;
-  unsigned phase = 0;
-  bool ok = true;
-  for (int tile = blockIdx.x; tile < a.tiles; tile += gridDim.x) {
-    if (issued >= a.stages) {
-      if (!twa_mbar_wait(twa_smem_u32(&hdr->empty[s]), phase, abort_flag, a.wait_limit_ns)) {
-        ok = false;
-        break;
-      }
-    }
-    const uint32_t fb = twa_smem_u32(&hdr->full[s]);
-    const uint32_t dst = twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes);
-    twa_mbar_expect_tx(fb, a.tx_bytes);
-    twa_tma_load_2d(dst, map_p, tile * TWA_TILE_COL_WORDS * KT, 0, fb);
-    for (int q = 0; q < tile_rows / 256; ++q)
-      twa_tma_load_2d(dst + a.g_off + q * NB * 256 * g_elem_bytes, map_g, tile * tile_rows + q * 256, a.b0, fb);
-    ++issued;
-    if (++s == a.stages) {
-      s = 0;
-      if (issued > a.stages) phase ^= 1u;
-    }
-  }
-  // every copy issued has landed before this lane leaves, whatever the consumers did meanwhile
-  if (!twa_drain_ring(hdr, issued, a.stages, a.wait_limit_ns)) ok = false;
-  if (!ok) twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+__device__ __forceinline__ void issue_tile(twa_smem_header* hdr, unsigned char* ring, const CUtensorMap* map_p,
+                                           const CUtensorMap* map_g, const BatchArgs& a, int tile, int s, int tile_rows,
+                                           int g_elem_bytes) {
+  const uint32_t fb = twa_smem_u32(&hdr->full[s]);
+  const uint32_t dst = twa_smem_u32(ring + static_cast<size_t>(s) * a.stage_bytes);
+  twa_mbar_expect_tx(fb, a.tx_bytes);
+  twa_tma_load_2d(dst, map_p, tile * TWA_TILE_COL_WORDS * KT, 0, fb);
+  for (int q = 0; q < tile_rows / 256; ++q)
+    twa_tma_load_2d(dst + a.g_off + q * NB * 256 * g_elem_bytes, map_g, tile * tile_rows + q * 256, a.b0, fb);
 }
 
 // NP pairs of gradients per launch (NB = 2 NP); MT, KT as in the single-gradient kernel.
+constexpr int BATCH_THREADS = MMA_WARPS * 32;
+
 template <int BITS, bool GBF16, int MT, int KT, int NP>
-__global__ void __launch_bounds__(MMA_THREADS, 1)
+__global__ void __launch_bounds__(BATCH_THREADS, 1)
 twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_g,
                          const BatchArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -110,15 +108,26 @@ twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) facc[p][mt][0] = facc[p][mt][1] = 0.0f;
 
-  if (warp == MMA_WARPS) {
-    if (lane == 0) producer_loop_batch<KT, NB>(hdr, ring, &map_p, &map_g, a, SROWS * KT, GSZ);
-  } else {
+  const bool filler = threadIdx.x == (MMA_WARPS - 1) * 32;
+  const int my_tiles = blockIdx.x < a.tiles ? (a.tiles - 1 - static_cast<int>(blockIdx.x)) / static_cast<int>(gridDim.x) + 1 : 0;
+  int issued = 0;
+  if (filler) {
+    twa_prefetch_tensormap(&map_p);
+    twa_prefetch_tensormap(&map_g);
+    for (; issued < my_tiles && issued < a.stages; ++issued)
+      issue_tile<KT, NB>(hdr, ring, &map_p, &map_g, a, blockIdx.x + issued * gridDim.x, issued, SROWS * KT, GSZ);
+  }
+  {
     constexpr int PAIR_BYTES = pair_bytes(BITS);         // digit matrices of one pair of gradients
-    unsigned char* digw = smem + a.scratch_off + warp * PAIR_BYTES;   // reused pair after pair
-    pair_digit_init<BITS>(digw, lane);
+    // a set of digit matrices per pair where shared memory allows, else one set reused pair after pair
+    const int sets = a.pair_stride ? NP : 1;
+    unsigned char* digw = smem + a.scratch_off + warp * sets * PAIR_BYTES;
+    for (int p = 0; p < sets; ++p) pair_digit_init<BITS>(digw + p * PAIR_BYTES, lane);
     __syncwarp();
     const uint32_t dig_addr = byte_digit_ldmatrix_addr(digw, lane);
     const int dmult = (tig & 1) ? -64 : 256;
+    // weight of this lane's digit sums over the weight of u0; 4-bit codes enter the MMA times 16
+    const float wfac = ((tig & 1) ? 65536.0f : 1.0f) * (BITS == 4 ? 0.0625f : 1.0f);
     const int lm = lane >> 3, lr = lane & 7;
     const int jmax = a.n - 1;
     constexpr int col_bytes = TWA_TILE_COL_BYTES * KT;
@@ -143,7 +152,7 @@ twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
     volatile int* abort_flag = &hdr->abort_flag;
     int s = 0;
     unsigned phase = 0;
-    unsigned bad = 0u;                                   // bit b: gradient b of the group is not finite
+    unsigned bad = 0u;                                   // lane b < NB: gradient b of the group is not finite
     for (int t = blockIdx.x; t < a.tiles; t += gridDim.x) {
       if (!twa_mbar_wait(twa_smem_u32(&hdr->full[s]), phase, abort_flag, a.wait_limit_ns)) {
         twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
@@ -154,57 +163,58 @@ twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
 #pragma unroll
       for (int u = 0; u < KT; ++u) {
         // ---- digits of the warp's rows of every gradient of the group, one matrix per pair ------
+        // The lane's row (4-bit codes: two rows) of every gradient and each gradient's largest magnitude;
+        // lane b < NB then derives gradient b's digit scale once for the warp and the others fetch it.
+        float g0[NB], g1[NB];
+        unsigned mine = 0u;
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+          const int e = goff[u] + b * 256;
+          g1[b] = 0.0f;
+          if (GBF16) {
+            const unsigned short* gs = reinterpret_cast<const unsigned short*>(st + a.g_off);
+            g0[b] = __uint_as_float(static_cast<uint32_t>(gs[e]) << 16);
+            if (BITS == 4) g1[b] = __uint_as_float(static_cast<uint32_t>(gs[e + 1]) << 16);
+          } else {
+            const float* gs = reinterpret_cast<const float*>(st + a.g_off);
+            g0[b] = gs[e];
+            if (BITS == 4) g1[b] = gs[e + 1];
+          }
+          unsigned mb = __float_as_uint(g0[b]) & 0x7FFFFFFFu;
+          if (BITS == 4) mb = max(mb, __float_as_uint(g1[b]) & 0x7FFFFFFFu);
+          mb = __reduce_max_sync(0xFFFFFFFFu, mb);
+          if (b == 0 || lane == b) mine = mb;
+        }
+        const ByteDigitScale ds = byte_digit_scale(mine);
+        if (ds.bad && lane < NB) bad = 1u;
+        // a dead or non-finite gradient is cut with scale 0: its digits are those of zero
+        const float up_mine = ds.live ? ds.up : 0.0f;
+        const float w_mine = ds.live ? ds.w0 : 0.0f;
         float wl[NP];                                    // this lane's weight for pair p (0: nothing to add)
         uint32_t bf[NP][4];                              // B fragments of every pair
 #pragma unroll
         for (int p = 0; p < NP; ++p) {
-          float g0[2], g1[2];
-          unsigned mb[2];
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int e = goff[u] + (2 * p + h) * 256;
-            g1[h] = 0.0f;
-            if (GBF16) {
-              const unsigned short* gs = reinterpret_cast<const unsigned short*>(st + a.g_off);
-              g0[h] = __uint_as_float(static_cast<uint32_t>(gs[e]) << 16);
-              if (BITS == 4) g1[h] = __uint_as_float(static_cast<uint32_t>(gs[e + 1]) << 16);
-            } else {
-              const float* gs = reinterpret_cast<const float*>(st + a.g_off);
-              g0[h] = gs[e];
-              if (BITS == 4) g1[h] = gs[e + 1];
-            }
-            mb[h] = max(__float_as_uint(g0[h]) & 0x7FFFFFFFu, __float_as_uint(g1[h]) & 0x7FFFFFFFu);
-          }
-          // one digit scale per gradient for the warp's rows of this 32-byte block
-          mb[0] = __reduce_max_sync(0xFFFFFFFFu, mb[0]);
-          mb[1] = __reduce_max_sync(0xFFFFFFFFu, mb[1]);
-          const ByteDigitScale ds0 = byte_digit_scale(mb[0]), ds1 = byte_digit_scale(mb[1]);
-          if (ds0.bad) bad |= 1u << (2 * p);
-          if (ds1.bad) bad |= 1u << (2 * p + 1);
-          // a dead or non-finite gradient is cut with scale 0: its digits are those of zero
-          const float up0 = ds0.live ? ds0.up : 0.0f, up1 = ds1.live ? ds1.up : 0.0f;
+          const float up0 = __shfl_sync(0xFFFFFFFFu, up_mine, 2 * p), up1 = __shfl_sync(0xFFFFFFFFu, up_mine, 2 * p + 1);
           // lanes tig 0,1 finish the first gradient's digits (columns u0 u1 | u2 ones), tig 2,3 the second's
-          const bool livem = (tig < 2) ? ds0.live : ds1.live;
-          float w = !livem ? 0.0f : ((tig < 2) ? ds0.w0 : ds1.w0);
-          if (tig & 1) w *= 65536.0f;
-          if (BITS == 4) w *= 0.0625f;                   // 4-bit codes enter the MMA times 16
-          wl[p] = w;
-          pair_digit_store(digw, 0, 0, lane, g0[0], up0);
-          pair_digit_store(digw, 0, 1, lane, g0[1], up1);
+          wl[p] = __shfl_sync(0xFFFFFFFFu, w_mine, 2 * p + (tig >> 1)) * wfac;
+          unsigned char* dp = digw + p * a.pair_stride;
+          pair_digit_store(dp, 0, 0, lane, g0[2 * p], up0);
+          pair_digit_store(dp, 0, 1, lane, g0[2 * p + 1], up1);
           if (BITS == 4) {
-            pair_digit_store(digw, 1, 0, lane, g1[0], up0);
-            pair_digit_store(digw, 1, 1, lane, g1[1], up1);
+            pair_digit_store(dp, 1, 0, lane, g1[2 * p], up0);
+            pair_digit_store(dp, 1, 1, lane, g1[2 * p + 1], up1);
           }
+          if (a.pair_stride == 0) {
+            __syncwarp();
+            load_pair_fragments<BITS>(dig_addr, bf[p]);
+            __syncwarp();                                // the digit matrices are rewritten by the next pair
+          }
+        }
+        if (a.pair_stride != 0) {
           __syncwarp();
-          // B fragments: result columns 0-3 = u0, u1, u2, ones of the pair's first gradient, 4-7 of its second
-          if (BITS == 8) {
-            ldmatrix_x2(dig_addr, bf[p][0], bf[p][1]);
-          } else {
-            uint32_t bb[4];
-            ldmatrix_x4(dig_addr, bb);
-            bf[p][0] = bb[0]; bf[p][1] = bb[1]; bf[p][2] = bb[2]; bf[p][3] = bb[3];   // second pair: the odd rows
-          }
-          __syncwarp();                                  // the digit matrices are rewritten by the next pair
+#pragma unroll
+          for (int p = 0; p < NP; ++p) load_pair_fragments<BITS>(dig_addr + p * a.pair_stride, bf[p]);
+          __syncwarp();                                  // rewritten for the next block of rows
         }
         // ---- every 16-column group of the tile is loaded (and unpacked) once for all pairs -------
 #pragma unroll
@@ -231,18 +241,29 @@ twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       }
       __syncwarp();
       if (lane == 0) twa_mbar_arrive(twa_smem_u32(&hdr->empty[s]));
+      if (filler && issued < my_tiles) {
+        // the stage just released takes this block's tile number `issued` once every warp is done with it
+        if (twa_mbar_wait(twa_smem_u32(&hdr->empty[s]), phase, abort_flag, a.wait_limit_ns)) {
+          issue_tile<KT, NB>(hdr, ring, &map_p, &map_g, a, blockIdx.x + issued * gridDim.x, s, SROWS * KT, GSZ);
+          ++issued;
+        } else {
+          twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
+        }
+      }
       if (++s == a.stages) {
         s = 0;
         phase ^= 1u;
       }
     }
-    if (bad) atomicOr(&hdr->bad_flag, static_cast<int>(bad));
+    if (bad) atomicOr(&hdr->bad_flag, 1 << lane);
+    // every copy issued has landed before its issuer goes on, whatever the consumers did meanwhile
+    if (filler && !twa_drain_ring(hdr, issued, a.stages, a.wait_limit_ns)) twa_set_status(a.status, TWA_ERR_TIMEOUT, -1);
   }
   __syncthreads();                                       // every stage consumed; the ring is free
 
   // ---- sums of the block: lanes -> warps -> block, in a fixed order --------------------------
   float* part = reinterpret_cast<float*>(ring);         // [MMA_WARPS][NB][TWA_MAX_N]
-  if (warp < MMA_WARPS) {
+  {
 #pragma unroll
     for (int p = 0; p < NP; ++p)
 #pragma unroll
@@ -332,7 +353,7 @@ int launch_one(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg, const
   static int smem_limit[64] = {0};
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[ctx->device & 63], smem);
   if (rc) return rc;
-  kern<<<grid, MMA_THREADS, smem, ctx->stream>>>(mp, mg, a);
+  kern<<<grid, BATCH_THREADS, smem, ctx->stream>>>(mp, mg, a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   return TWA_OK;
 }
@@ -372,7 +393,7 @@ int launch_mt(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg, const 
   }
 }
 
-int fixed_smem(int bits) { return TWA_SMEM_HEADER + MMA_WARPS * pair_bytes(bits) + 1024; }
+int fixed_smem(int bits, int sets = 1) { return TWA_SMEM_HEADER + MMA_WARPS * sets * pair_bytes(bits) + 1024; }
 
 unsigned stage_bytes_of(const twa_basis* P, int gsz, int kt, int nb) {
   const unsigned tx = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt + twa_tile_rows(P->bits) * kt * gsz * nb;
@@ -440,6 +461,16 @@ extern "C" int twa_project_batch(twa_ctx* ctx, const twa_basis* P, const void* G
   a.tx_bytes = a.g_off + static_cast<unsigned>(rows * gsz * nb);
   a.stage_bytes = (a.tx_bytes + 1023) / 1024 * 1024;
   int stages = (ctx->smem_optin - fixed_smem(P->bits)) / static_cast<int>(a.stage_bytes);
+  // a set of digit matrices per pair if that costs no stage (or leaves three)
+  int sets = 1;
+  {
+    const int with_sets = (ctx->smem_optin - fixed_smem(P->bits, nb / 2)) / static_cast<int>(a.stage_bytes);
+    if (with_sets == stages || with_sets >= 3) {
+      sets = nb / 2;
+      stages = with_sets;
+    }
+  }
+  a.pair_stride = sets > 1 ? static_cast<unsigned>(pair_bytes(P->bits)) : 0u;
   if (stages > TWA_MAX_STAGES) stages = TWA_MAX_STAGES;
   if (stages < 2) return TWA_ERR_UNSUPPORTED;
   // the ring is reused for the block's [16][NB][128] float sums after the tile loop
@@ -454,7 +485,7 @@ extern "C" int twa_project_batch(twa_ctx* ctx, const twa_basis* P, const void* G
   a.wait_limit_ns = ctx->wait_limit_ns;
   int grid = ctx->sm_count < a.tiles ? ctx->sm_count : a.tiles;
   while (static_cast<size_t>(grid) * nb * P->n > static_cast<size_t>(TWA_MAX_GRID) * TWA_MAX_N) --grid;
-  const int smem = static_cast<int>(a.scratch_off) + MMA_WARPS * pair_bytes(P->bits) + 1024;
+  const int smem = static_cast<int>(a.scratch_off) + MMA_WARPS * sets * pair_bytes(P->bits) + 1024;
   for (int b0 = 0; b0 < batch; b0 += nb) {
     a.b0 = b0;
     if (P->bits == 8)
