@@ -648,10 +648,12 @@ layered_lift_kernel(const __grid_constant__ CUtensorMap map_p, const LLiftArgs a
     const int4 e = entries[gran_in_tile];
     const unsigned seg_off = (a.base && tile_is_packed<BITS, KT, 4>(entries, a.base)) ? seg_off_packed : seg_off_loose;
     const float* gs = reinterpret_cast<const float*>(st + seg_off);        // the granule's rows of base, staged
+    // only lanes tig 0, 1 finish rows: the other two would read the same banks a chunk further on
+    // (four-way conflicts on every such load)
     float bv[KT][LROWS];
 #pragma unroll
     for (int u = 0; u < KT; ++u) {
-      if (!a.base) {
+      if (!a.base || tig >= 2) {
 #pragma unroll
         for (int i = 0; i < LROWS; ++i) bv[u][i] = 0.0f;
       } else if (LROWS == 2) {
