@@ -116,7 +116,8 @@ const char* twa_last_error(const twa_ctx* ctx);
  *      float path and on 32-bit bases only.
  *  TWA_TUNE_TILE_SEGMENTS: tensor-pipe path, 512-byte segments of a column per tile: 1, 2 or 4
  *      (4 is honoured for n <= 32 only).  Default: per kernel and width, the tallest tile of which
- *      enough stages fit in shared memory.
+ *      enough stages fit in shared memory.  Also the projection on a 32-bit basis (default 4 for
+ *      n <= 32, 2 for n <= 64, else 1; 4 needs an even D and becomes 2 otherwise).
  *  TWA_TUNE_BUILD_PANEL: twa_build_basis: 0 = panels of 8 columns, the Gram-Schmidt coefficients
  *      inside a panel taken from the panel's Gram matrix (default); 1 = column by column;
  *      2 = panels of 8 columns with column-by-column sweeps inside a panel.

@@ -47,7 +47,7 @@ using SmemHeader = twa_smem_header;
 
 // Producer loop shared by both kernels.  G_BOXES 1-D boxes of the gradient follow the tile
 // of P~ in the same stage (project only).
-template <int ROWS, int G_BOXES, int G_BOX_ELEMS, int G_ELEM_BYTES>
+template <int ROWS, int G_BOXES, int G_BOX_ELEMS, int G_ELEM_BYTES, int KT = 1>
 __device__ __forceinline__ void producer_loop(SmemHeader* hdr, unsigned char* ring,
                                               const CUtensorMap* map_p, const CUtensorMap* map_g,
                                               int tiles, int stages, unsigned stage_bytes,
@@ -71,7 +71,7 @@ __device__ __forceinline__ void producer_loop(SmemHeader* hdr, unsigned char* ri
     const uint32_t fb = twa_smem_u32(&hdr->full[s]);
     const uint32_t dst = twa_smem_u32(ring + static_cast<size_t>(s) * stage_bytes);
     twa_mbar_expect_tx(fb, tx_bytes);
-    twa_tma_load_2d(dst, map_p, tile * TWA_TILE_COL_WORDS, 0, fb);
+    twa_tma_load_2d(dst, map_p, tile * (KT == 4 ? TWA_TILE_COL_BYTES / 8 * KT : TWA_TILE_COL_WORDS * KT), 0, fb);
 #pragma unroll
     for (int b = 0; b < G_BOXES; ++b)
       twa_tma_load_1d(dst + g_off + b * G_BOX_ELEMS * G_ELEM_BYTES, map_g,
@@ -133,13 +133,16 @@ __device__ __forceinline__ float lane_dot(const unsigned char* col16, const floa
   return t;
 }
 
-template <int BITS, bool GBF16>
+// KT: 512-byte segments of every column per tile (a float32 basis with few columns: tiles of 128 rows
+// are a few KB, and the per-tile hand-over then bounds the kernel, not the memory).
+template <int BITS, bool GBF16, int KT = 1>
 __global__ void __launch_bounds__(TWA_MAX_THREADS, 1)
 twa_project_kernel(const __grid_constant__ CUtensorMap map_p,
                    const __grid_constant__ CUtensorMap map_g, const ProjectArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
-  constexpr int ROWS = twa_tile_rows(BITS);
-  constexpr int LROWS = ROWS / 32;                     // gradient values one lane needs
+  constexpr int SROWS = twa_tile_rows(BITS);           // rows behind one segment
+  constexpr int ROWS = SROWS * KT;
+  constexpr int LROWS = SROWS / 32;                    // gradient values one lane needs per segment
   constexpr int GSZ = GBF16 ? 2 : 4;
   constexpr int GBOX = ROWS < 256 ? ROWS : 256;
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
@@ -161,9 +164,9 @@ twa_project_kernel(const __grid_constant__ CUtensorMap map_p,
 
   if (warp == W) {
     if (lane == 0)
-      producer_loop<ROWS, ROWS / GBOX, GBOX, GSZ>(hdr, ring, &map_p, &map_g, a.tiles, a.stages,
-                                                  a.stage_bytes, a.g_off, a.tx_bytes, false,
-                                                  a.status, a.wait_limit_ns);
+      producer_loop<ROWS, ROWS / GBOX, GBOX, GSZ, KT>(hdr, ring, &map_p, &map_g, a.tiles, a.stages,
+                                                      a.stage_bytes, a.g_off, a.tx_bytes, false,
+                                                      a.status, a.wait_limit_ns);
   } else {
     // warp owns columns warp, warp + W, ...
     const int cpw = warp < a.n ? (a.n - warp + W - 1) / W : 0;
@@ -179,36 +182,41 @@ twa_project_kernel(const __grid_constant__ CUtensorMap map_p,
         break;
       }
       const unsigned char* st = ring + static_cast<size_t>(s) * a.stage_bytes;
-      float g[LROWS];
-      if (GBF16) {
-        const uint4* gp = reinterpret_cast<const uint4*>(st + a.g_off + lane * (LROWS * 2));
 #pragma unroll
-        for (int q = 0; q < LROWS / 8; ++q) {
-          const uint4 v = gp[q];
-          g[8 * q + 0] = twa_bf16_lo(v.x); g[8 * q + 1] = twa_bf16_hi(v.x);
-          g[8 * q + 2] = twa_bf16_lo(v.y); g[8 * q + 3] = twa_bf16_hi(v.y);
-          g[8 * q + 4] = twa_bf16_lo(v.z); g[8 * q + 5] = twa_bf16_hi(v.z);
-          g[8 * q + 6] = twa_bf16_lo(v.w); g[8 * q + 7] = twa_bf16_hi(v.w);
-        }
-        if (LROWS == 4) {                                // float32 basis: 4 rows = 8 bytes
-          const uint2 v = *reinterpret_cast<const uint2*>(st + a.g_off + lane * 8);
-          g[0] = twa_bf16_lo(v.x); g[1] = twa_bf16_hi(v.x);
-          g[2] = twa_bf16_lo(v.y); g[3] = twa_bf16_hi(v.y);
-        }
-      } else {
-        const float4* gp = reinterpret_cast<const float4*>(st + a.g_off + lane * (LROWS * 4));
+      for (int u = 0; u < KT; ++u) {
+        // the lane's LROWS rows of segment u: rows u * SROWS + lane * LROWS ...
+        const unsigned char* gseg = st + a.g_off + (u * SROWS + lane * LROWS) * GSZ;
+        float g[LROWS];
+        if (GBF16) {
+          const uint4* gp = reinterpret_cast<const uint4*>(gseg);
 #pragma unroll
-        for (int q = 0; q < LROWS / 4; ++q) {
-          const float4 v = gp[q];
-          g[4 * q + 0] = v.x; g[4 * q + 1] = v.y; g[4 * q + 2] = v.z; g[4 * q + 3] = v.w;
-        }
-      }
+          for (int q = 0; q < LROWS / 8; ++q) {
+            const uint4 v = gp[q];
+            g[8 * q + 0] = twa_bf16_lo(v.x); g[8 * q + 1] = twa_bf16_hi(v.x);
+            g[8 * q + 2] = twa_bf16_lo(v.y); g[8 * q + 3] = twa_bf16_hi(v.y);
+            g[8 * q + 4] = twa_bf16_lo(v.z); g[8 * q + 5] = twa_bf16_hi(v.z);
+            g[8 * q + 6] = twa_bf16_lo(v.w); g[8 * q + 7] = twa_bf16_hi(v.w);
+          }
+          if (LROWS == 4) {                                // float32 basis: 4 rows = 8 bytes
+            const uint2 v = *reinterpret_cast<const uint2*>(gseg);
+            g[0] = twa_bf16_lo(v.x); g[1] = twa_bf16_hi(v.x);
+            g[2] = twa_bf16_lo(v.y); g[3] = twa_bf16_hi(v.y);
+          }
+        } else {
+          const float4* gp = reinterpret_cast<const float4*>(gseg);
 #pragma unroll
-      for (int k = 0; k < TWA_PROJECT_CPW; ++k) {
-        if (k < cpw) {
-          const int j = warp + k * W;
-          const int slot = BITS == 32 ? lane : twa_chunk_slot(lane, j);
-          acc[k] += lane_dot<BITS>(st + j * TWA_TILE_COL_BYTES + slot * 16, g);
+          for (int q = 0; q < LROWS / 4; ++q) {
+            const float4 v = gp[q];
+            g[4 * q + 0] = v.x; g[4 * q + 1] = v.y; g[4 * q + 2] = v.z; g[4 * q + 3] = v.w;
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < TWA_PROJECT_CPW; ++k) {
+          if (k < cpw) {
+            const int j = warp + k * W;
+            const int slot = BITS == 32 ? lane : twa_chunk_slot(lane, j);
+            acc[k] += lane_dot<BITS>(st + (j * KT + u) * TWA_TILE_COL_BYTES + slot * 16, g);
+          }
         }
       }
       __syncwarp();
@@ -458,15 +466,21 @@ twa_lift32_kernel(const float* __restrict__ P, long long ld, int n, const float*
 // ---- host side ----------------------------------------------------------------------------
 int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
-int encode_basis_map(twa_ctx* ctx, const twa_basis* P, CUtensorMap* map) {
+int encode_basis_map(twa_ctx* ctx, const twa_basis* P, CUtensorMap* map, int kt = 1) {
   long long row_bytes = (P->D * P->bits + 7) / 8;
   // quantised columns are stored in whole, internally permuted 512-byte segments
   if (P->bits != 32) row_bytes = (row_bytes + 511) / 512 * 512;
   cuuint64_t dims[2] = {static_cast<cuuint64_t>((row_bytes + 3) / 4), static_cast<cuuint64_t>(P->n)};
   cuuint64_t strides[1] = {static_cast<cuuint64_t>(P->col_stride)};
-  cuuint32_t box[2] = {TWA_TILE_COL_WORDS, static_cast<cuuint32_t>(P->n)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(TWA_TILE_COL_WORDS * kt), static_cast<cuuint32_t>(P->n)};
+  if (kt == 4) {
+    // a box dimension is limited to 256 elements: four segments are 256 elements of 8 bytes (the caller
+    // has checked that a column's bytes are a multiple of 8, so no element reaches past row D - 1)
+    dims[0] = static_cast<cuuint64_t>(row_bytes / 8);
+    box[0] = TWA_TILE_COL_BYTES / 8 * 4;
+  }
   cuuint32_t es[2] = {1, 1};
-  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, P->data, dims, strides, box,
+  CUresult r = ctx->encode_tiled(map, kt == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT64 : CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, P->data, dims, strides, box,
                                  es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -543,10 +557,10 @@ int choose_stages(const twa_ctx* ctx, int fixed_bytes, int stage_bytes) {
   return s;
 }
 
-template <int BITS, bool GBF16>
+template <int BITS, bool GBF16, int KT = 1>
 int launch_project_t(twa_ctx* ctx, const CUtensorMap& mp, const CUtensorMap& mg, const ProjectArgs& a,
                      int grid, int smem) {
-  auto kern = twa_project_kernel<BITS, GBF16>;
+  auto kern = twa_project_kernel<BITS, GBF16, KT>;
   static int smem_limit[64] = {0};   // per device
   int rc = twa_ensure_smem(ctx, reinterpret_cast<const void*>(kern), &smem_limit[ctx->device & 63], smem);
   if (rc) return rc;
@@ -598,10 +612,20 @@ int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtyp
   if (P->bits != 32 && ctx->tune_dequant_path == 0)
     return twa_launch_project_mma(ctx, P, g, g_dtype, epi, ws);
   const bool bf16 = g_dtype == TWA_BF16;
-  const int rows = twa_tile_rows(P->bits);
+  // a float32 basis of few columns takes tiles of two or four segments (256 or 512 rows): see
+  // twa_project_kernel; four need the tensor map of 8-byte elements, i.e. an even number of rows
+  int kt = 1;
+  if (P->bits == 32) {
+    kt = P->n <= 32 ? 4 : (P->n <= 64 ? 2 : 1);
+    if (ctx->tune_tile_segments == 1 || ctx->tune_tile_segments == 2 || ctx->tune_tile_segments == 4)
+      kt = ctx->tune_tile_segments;
+    if (kt == 4 && (P->D & 1)) kt = 2;
+    while (kt > 1 && (ctx->smem_optin - TWA_SMEM_HEADER) / (P->n * TWA_TILE_COL_BYTES * kt + twa_tile_rows(32) * kt * 4 + 128) < 3) kt >>= 1;
+  }
+  const int rows = twa_tile_rows(P->bits) * kt;
   const int gsz = bf16 ? 2 : 4;
   CUtensorMap mp, mg;
-  int rc = encode_basis_map(ctx, P, &mp);
+  int rc = encode_basis_map(ctx, P, &mp, kt);
   if (rc) return rc;
   rc = encode_vector_map(ctx, g, P->D, bf16, rows < 256 ? rows : 256, &mg);
   if (rc) return rc;
@@ -611,7 +635,7 @@ int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtyp
   a.n = P->n;
   a.warps = choose_project_warps(P->n, ctx->tune_project_warps);
   a.tiles = static_cast<int>((P->D + rows - 1) / rows);
-  a.g_off = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES;
+  a.g_off = static_cast<unsigned>(P->n) * TWA_TILE_COL_BYTES * kt;
   a.tx_bytes = a.g_off + static_cast<unsigned>(rows * gsz);
   a.stage_bytes = static_cast<unsigned>(round_up(static_cast<int>(a.tx_bytes), 128));
   a.stages = choose_stages(ctx, TWA_SMEM_HEADER, static_cast<int>(a.stage_bytes));
@@ -633,6 +657,12 @@ int twa_launch_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtyp
 
   switch (P->bits) {
     case 32:
+      if (kt == 4)
+        return bf16 ? launch_project_t<32, true, 4>(ctx, mp, mg, a, grid, smem)
+                    : launch_project_t<32, false, 4>(ctx, mp, mg, a, grid, smem);
+      if (kt == 2)
+        return bf16 ? launch_project_t<32, true, 2>(ctx, mp, mg, a, grid, smem)
+                    : launch_project_t<32, false, 2>(ctx, mp, mg, a, grid, smem);
       return bf16 ? launch_project_t<32, true>(ctx, mp, mg, a, grid, smem)
                   : launch_project_t<32, false>(ctx, mp, mg, a, grid, smem);
     case 8:

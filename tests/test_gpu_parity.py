@@ -556,6 +556,29 @@ def test_tile_segments_knob(env, D, n, bits, segments):
         twa.twa_set_tuning(ctx, twa.TWA_TUNE_TILE_SEGMENTS, 0)
 
 
+@pytest.mark.parametrize("segments", [0, 1, 2, 4])
+@pytest.mark.parametrize("gdt", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("D,n", [(2, 1), (4099, 33), (70002, 20), (70001, 20), (131072, 8), (40000, 64), (9000, 128)])
+def test_float32_projection_tile_heights(env, D, n, gdt, segments):
+    """The float32 projection in tiles of one, two and four 512-byte segments (four: even D only,
+    else the library falls back to two), with poison in the padding behind row D - 1 of every column."""
+    ctx, ws = env
+    P = random_basis(D, n, 4100 + D + n)
+    P[:, D:] = float("nan")
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(D * 3 + n)
+    g = (torch.randn(D, generator=gen, device=DEV) * 1e-3).to(gdt)
+    c = torch.full((n + 1,), 7.0, device=DEV)
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_TILE_SEGMENTS, segments)
+    try:
+        twa.twa_project(ctx, twa.basis_from_tensor(P, D), g, c, ws)
+    finally:
+        twa.twa_set_tuning(ctx, twa.TWA_TUNE_TILE_SEGMENTS, 0)
+    status_ok(ctx)
+    assert rel(c[:n].cpu().numpy(), orc.project_f32(host_cols(P, D), g.float().cpu().numpy())) <= TOL
+    assert c[n].item() == 7.0
+
+
 @pytest.mark.parametrize("bits", [8, 4])
 @pytest.mark.parametrize("D,n", [(1, 1), (4099, 33), (70001, 100), (131075, 8), (600001, 32)])
 def test_lift_vectors_knob(env, D, n, bits):
