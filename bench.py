@@ -815,10 +815,12 @@ def layered_line(env, args, workload, bits, min_timed_ms):
         W = wl.candidates(dev, ld=inputs.padded_ld(D, 128))
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
         torch.cuda.synchronize()
+        mem = torch.empty(twa.twa_layered_basis_bytes(layers, n, bits), dtype=torch.uint8, device=dev)
+        torch.cuda.synchronize()
         ev[0].record()
         P32 = twa.twa_build_centered(ctx, W, D, layers, wbar, lws)
         ev[1].record()
-        lb = twa.twa_quantize_affine(ctx, P32, layers, bits, lws)
+        lb = twa.twa_quantize_affine(ctx, P32, layers, bits, lws, mem=mem)
         ev[2].record()
         torch.cuda.synchronize()
         build_ms, quant_ms = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])

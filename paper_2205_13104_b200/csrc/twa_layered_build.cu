@@ -83,6 +83,21 @@ __device__ __forceinline__ double block_sum_d(double v, double* sh) {
   return t;
 }
 
+// Rows r .. r + 3 of p (r a multiple of 4); rows outside [lo, hi) read as zero.  One 16-byte load when p
+// is 16-byte aligned and all four rows exist: a thread's loads then cover whole 32-byte sectors between
+// them (with one float per load a warp touched 32 lines per instruction and the 4-bit pass ran at a
+// third of the 8-bit one).
+__device__ __forceinline__ float4 load_rows4(const float* __restrict__ p, long long r, long long lo, long long hi,
+                                             bool aligned) {
+  if (aligned && r >= lo && r + 3 < hi) return *reinterpret_cast<const float4*>(p + r);
+  float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (r >= lo && r < hi) x.x = p[r];
+  if (r + 1 >= lo && r + 1 < hi) x.y = p[r + 1];
+  if (r + 2 >= lo && r + 2 < hi) x.z = p[r + 2];
+  if (r + 3 >= lo && r + 3 < hi) x.w = p[r + 3];
+  return x;
+}
+
 // partial[item][i] = sum over the item's rows of (w - w_bar)^2
 __global__ void __launch_bounds__(BLOCK) centred_sumsq_kernel(const float* __restrict__ W, long long ldw,
                                                               const float* __restrict__ wbar,
@@ -91,10 +106,17 @@ __global__ void __launch_bounds__(BLOCK) centred_sumsq_kernel(const float* __res
   __shared__ double sh[BLOCK / 32];
   const Item it = items[blockIdx.x];
   const float* col = W + blockIdx.y * ldw;
+  const bool aligned = ((reinterpret_cast<uintptr_t>(col) | reinterpret_cast<uintptr_t>(wbar)) & 15) == 0;
   double s = 0;
-  for (long long r = it.r0 + threadIdx.x; r < it.r1; r += BLOCK) {
-    const double v = static_cast<double>(col[r]) - static_cast<double>(wbar[r]);
-    s += v * v;
+  for (long long g = (it.r0 & ~3LL) + 4 * threadIdx.x; g < it.r1; g += 4 * BLOCK) {
+    // four rows a thread; rows outside the item read as zero on both sides and add nothing
+    const float4 x = load_rows4(col, g, it.r0, it.r1, aligned), m = load_rows4(wbar, g, it.r0, it.r1, aligned);
+    const double v0 = static_cast<double>(x.x) - static_cast<double>(m.x), v1 = static_cast<double>(x.y) - static_cast<double>(m.y);
+    const double v2 = static_cast<double>(x.z) - static_cast<double>(m.z), v3 = static_cast<double>(x.w) - static_cast<double>(m.w);
+    s += v0 * v0;
+    s += v1 * v1;
+    s += v2 * v2;
+    s += v3 * v3;
   }
   const double t = block_sum_d(s, sh);
   if (threadIdx.x == 0) partial[static_cast<size_t>(blockIdx.x) * n + blockIdx.y] = t;
@@ -119,8 +141,23 @@ __global__ void __launch_bounds__(BLOCK) centre_scale_kernel(float* __restrict__
   const Item it = items[blockIdx.x];
   float* col = W + blockIdx.y * ldw;
   const double f = inv[static_cast<size_t>(it.layer) * n + blockIdx.y];
-  for (long long r = it.r0 + threadIdx.x; r < it.r1; r += BLOCK)
-    col[r] = static_cast<float>((static_cast<double>(col[r]) - static_cast<double>(wbar[r])) * f);
+  const bool aligned = ((reinterpret_cast<uintptr_t>(col) | reinterpret_cast<uintptr_t>(wbar)) & 15) == 0;
+  for (long long g = (it.r0 & ~3LL) + 4 * threadIdx.x; g < it.r1; g += 4 * BLOCK) {
+    const float4 x = load_rows4(col, g, it.r0, it.r1, aligned), m = load_rows4(wbar, g, it.r0, it.r1, aligned);
+    float4 y;
+    y.x = static_cast<float>((static_cast<double>(x.x) - static_cast<double>(m.x)) * f);
+    y.y = static_cast<float>((static_cast<double>(x.y) - static_cast<double>(m.y)) * f);
+    y.z = static_cast<float>((static_cast<double>(x.z) - static_cast<double>(m.z)) * f);
+    y.w = static_cast<float>((static_cast<double>(x.w) - static_cast<double>(m.w)) * f);
+    if (aligned && g >= it.r0 && g + 3 < it.r1) {
+      *reinterpret_cast<float4*>(col + g) = y;
+    } else {
+      if (g >= it.r0 && g < it.r1) col[g] = y.x;
+      if (g + 1 >= it.r0 && g + 1 < it.r1) col[g + 1] = y.y;
+      if (g + 2 >= it.r0 && g + 2 < it.r1) col[g + 2] = y.z;
+      if (g + 3 >= it.r0 && g + 3 < it.r1) col[g + 3] = y.w;
+    }
+  }
 }
 
 // partial min / max of one item over one column
@@ -132,11 +169,18 @@ __global__ void __launch_bounds__(BLOCK) minmax_kernel(const float* __restrict__
   const float* col = P + blockIdx.y * ld;
   float lo = INFINITY, hi = -INFINITY;
   bool bad = false;                              // fmin / fmax drop NaN: track non-finite input apart
-  for (long long r = it.r0 + threadIdx.x; r < it.r1; r += BLOCK) {
-    const float v = col[r];
-    lo = fminf(lo, v);
-    hi = fmaxf(hi, v);
-    bad |= !isfinite(v);
+  const bool aligned = (reinterpret_cast<uintptr_t>(col) & 15) == 0;
+  for (long long g = (it.r0 & ~3LL) + 4 * threadIdx.x; g < it.r1; g += 4 * BLOCK) {
+    const float4 x = load_rows4(col, g, it.r0, it.r1, aligned);
+    const float v[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (g + i >= it.r0 && g + i < it.r1) {
+        lo = fminf(lo, v[i]);
+        hi = fmaxf(hi, v[i]);
+        bad |= !isfinite(v[i]);
+      }
+    }
   }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
@@ -160,21 +204,41 @@ __global__ void __launch_bounds__(BLOCK) minmax_kernel(const float* __restrict__
   }
 }
 
-// a[l] = (max - min) / (2^B - 1), b[l] = min over the layer's items and all columns
-__global__ void factors_kernel(const float* __restrict__ pmin, const float* __restrict__ pmax,
-                               const int* __restrict__ first_item, int L, int n, float levels,
-                               float* __restrict__ a, float* __restrict__ b, int* status) {
-  const int l = blockIdx.x * blockDim.x + threadIdx.x;
-  if (l >= L) return;
+// a[l] = (max - min) / (2^B - 1), b[l] = min over the layer's items and all columns.  One block of 128
+// threads per layer (min and max do not depend on the order).
+__global__ void __launch_bounds__(128) factors_kernel(const float* __restrict__ pmin, const float* __restrict__ pmax,
+                                                      const int* __restrict__ first_item, int L, int n, float levels,
+                                                      float* __restrict__ a, float* __restrict__ b, int* status) {
+  __shared__ float slo[4], shi[4];
+  __shared__ int sbad[4];
+  const int l = blockIdx.x;
+  const size_t i0 = static_cast<size_t>(first_item[l]) * n, i1 = static_cast<size_t>(first_item[l + 1]) * n;
   float lo = INFINITY, hi = -INFINITY;
   bool bad = false;
-  for (int k = first_item[l]; k < first_item[l + 1]; ++k)
-    for (int i = 0; i < n; ++i) {
-      const float x = pmin[static_cast<size_t>(k) * n + i], y = pmax[static_cast<size_t>(k) * n + i];
-      bad |= isnan(x) || isnan(y);
-      lo = fminf(lo, x);
-      hi = fmaxf(hi, y);
-    }
+  for (size_t i = i0 + threadIdx.x; i < i1; i += 128) {
+    const float x = pmin[i], y = pmax[i];
+    bad |= isnan(x) || isnan(y);
+    lo = fminf(lo, x);
+    hi = fmaxf(hi, y);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, off));
+    hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, off));
+  }
+  bad = __any_sync(0xFFFFFFFFu, bad);
+  if ((threadIdx.x & 31) == 0) {
+    slo[threadIdx.x >> 5] = lo;
+    shi[threadIdx.x >> 5] = hi;
+    sbad[threadIdx.x >> 5] = bad ? 1 : 0;
+  }
+  __syncthreads();
+  if (threadIdx.x != 0) return;
+  for (int w = 1; w < 4; ++w) {
+    lo = fminf(lo, slo[w]);
+    hi = fmaxf(hi, shi[w]);
+    bad |= sbad[w] != 0;
+  }
   if (bad) {
     twa_set_status(status, TWA_ERR_NONFINITE, l);
     a[l] = 0.0f;
@@ -183,6 +247,32 @@ __global__ void factors_kernel(const float* __restrict__ pmin, const float* __re
   }
   a[l] = __fdiv_rn(__fsub_rn(hi, lo), levels);
   b[l] = lo;
+}
+
+// The quantiser's code of an element: round((e - b) / a) on IEEE float32 operations, half to even,
+// clamped to [0, top] (clamping first gives the same code: the bounds are integers; a NaN becomes 0
+// either way).  The rounding is an addition of 2^23, whose low mantissa bits are then the code.
+__device__ __forceinline__ uint32_t affine_code(float e, float bl, float al, float top) {
+  const float q = fminf(fmaxf(__fdiv_rn(__fsub_rn(e, bl), al), 0.0f), top);
+  return __float_as_uint(q + 8388608.0f) - 0x4B000000u;
+}
+
+// The same code without the division: with r = RN(1 / a) the product (e - b) r lies within
+// (top + 1) 2^-23 of the IEEE quotient wherever the clamp does not decide, so both round to the same
+// integer unless the product is within `near` = (top + 1) 2^-21 of a half-integer; then *hard is set and
+// the caller repeats the group with affine_code.  The distance to the integer is exact in float32.
+__device__ __forceinline__ uint32_t affine_code_by_reciprocal(float e, float bl, float r, float top, float near,
+                                                             bool* hard) {
+  const float q0 = fminf(fmaxf(__fsub_rn(e, bl) * r, 0.0f), top);
+  const float y = q0 + 8388608.0f;
+  *hard |= fabsf(q0 - (y - 8388608.0f)) >= 0.5f - near;
+  return __float_as_uint(y) - 0x4B000000u;
+}
+
+// r = RN(1 / a) when the reciprocal path is valid for this layer and width, else 0: a normal scale, and a
+// `near` band narrow enough to be met rarely (16-bit codes would meet it in every group).
+__device__ __forceinline__ float affine_reciprocal(float al, float top) {
+  return (al >= 0x1p-100f && top <= 255.0f) ? __frcp_rn(al) : 0.0f;
 }
 
 // Puts code u (k-th of a 16-byte chunk, slots of W bits) into the chunk's words.
@@ -211,23 +301,36 @@ __global__ void __launch_bounds__(BLOCK) affine_encode_kernel(const float* __res
   const float* col = P + j * ld + flat[l];
   uint4* dst = reinterpret_cast<uint4*>(out + j * out_stride);
   uint4* dst_lo = reinterpret_cast<uint4*>(out + (static_cast<long long>(n) + j) * out_stride);
+  const float recip = PLANES == 2 ? 0.0f : affine_reciprocal(al, top);
+  const float near = (top + 1.0f) * 0x1p-21f;
+  const bool aligned = (reinterpret_cast<uintptr_t>(col) & 15) == 0;
   for (long long c = blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; c < chunks;
        c += static_cast<long long>(gridDim.x) * BLOCK) {
     uint32_t w[4] = {0, 0, 0, 0}, wl[4] = {0, 0, 0, 0};
+    bool hard = recip == 0.0f;
+    if (!hard) {
 #pragma unroll
-    for (int k = 0; k < RPC; ++k) {
-      const long long r = c * RPC + k;
-      uint32_t u = 0;
-      if (r < len && al != 0.0f) {
-        float q = rintf(__fdiv_rn(__fsub_rn(col[r], bl), al));
-        q = fminf(fmaxf(q, 0.0f), top);
-        u = static_cast<uint32_t>(q);
+      for (int k = 0; k < RPC; k += 4) {
+        const long long r = c * RPC + k;
+        const float4 x = load_rows4(col, r, 0, len, aligned);
+        if (r < len) put_code<W>(w, k, affine_code_by_reciprocal(x.x, bl, recip, top, near, &hard));
+        if (r + 1 < len) put_code<W>(w, k + 1, affine_code_by_reciprocal(x.y, bl, recip, top, near, &hard));
+        if (r + 2 < len) put_code<W>(w, k + 2, affine_code_by_reciprocal(x.z, bl, recip, top, near, &hard));
+        if (r + 3 < len) put_code<W>(w, k + 3, affine_code_by_reciprocal(x.w, bl, recip, top, near, &hard));
       }
-      if (PLANES == 2) {
-        put_code<W>(w, k, u >> 8);
-        put_code<W>(wl, k, u & 0xFFu);
-      } else {
-        put_code<W>(w, k, u);
+    }
+    if (hard) {
+      w[0] = w[1] = w[2] = w[3] = 0u;
+#pragma unroll
+      for (int k = 0; k < RPC; ++k) {
+        const long long r = c * RPC + k;
+        const uint32_t u = (r < len && al != 0.0f) ? affine_code(col[r], bl, al, top) : 0u;
+        if (PLANES == 2) {
+          put_code<W>(w, k, u >> 8);
+          put_code<W>(wl, k, u & 0xFFu);
+        } else {
+          put_code<W>(w, k, u);
+        }
       }
     }
     const long long q = internal[l] / RPC + c;
@@ -249,10 +352,16 @@ __global__ void __launch_bounds__(BLOCK) chunk_centred_sumsq_kernel(const float*
   const Item it = items[blockIdx.x];
   const long long r0 = it.r0 > row0 ? it.r0 : row0, r1 = it.r1 < row1 ? it.r1 : row1;
   const float* col = chunk + blockIdx.y * ld - row0;
+  const bool aligned = ((reinterpret_cast<uintptr_t>(col) | reinterpret_cast<uintptr_t>(wbar)) & 15) == 0;
   double s = 0;
-  for (long long r = r0 + threadIdx.x; r < r1; r += BLOCK) {
-    const double v = static_cast<double>(col[r]) - static_cast<double>(wbar[r]);
-    s += v * v;
+  for (long long g = (r0 & ~3LL) + 4 * threadIdx.x; g < r1; g += 4 * BLOCK) {
+    const float4 x = load_rows4(col, g, r0, r1, aligned), m = load_rows4(wbar, g, r0, r1, aligned);
+    const double v0 = static_cast<double>(x.x) - static_cast<double>(m.x), v1 = static_cast<double>(x.y) - static_cast<double>(m.y);
+    const double v2 = static_cast<double>(x.z) - static_cast<double>(m.z), v3 = static_cast<double>(x.w) - static_cast<double>(m.w);
+    s += v0 * v0;
+    s += v1 * v1;
+    s += v2 * v2;
+    s += v3 * v3;
   }
   const double t = block_sum_d(s, sh);
   if (threadIdx.x == 0) partial[static_cast<size_t>(blockIdx.x) * n + blockIdx.y] += t;
@@ -274,12 +383,22 @@ __global__ void __launch_bounds__(BLOCK) chunk_minmax_kernel(const float* __rest
   const double f = inv[static_cast<size_t>(it.layer) * n + blockIdx.y];
   float lo = INFINITY, hi = -INFINITY;
   bool bad = false;
-  for (long long r = r0 + threadIdx.x; r < r1; r += BLOCK) {
-    const float v = static_cast<float>((static_cast<double>(col[r]) - static_cast<double>(wbar[r])) * f);
-    if (q32) q32[blockIdx.y * ldq + (r - row0)] = v;
-    lo = fminf(lo, v);
-    hi = fmaxf(hi, v);
-    bad |= !isfinite(v);
+  const bool aligned = ((reinterpret_cast<uintptr_t>(col) | reinterpret_cast<uintptr_t>(wbar)) & 15) == 0;
+  for (long long g = (r0 & ~3LL) + 4 * threadIdx.x; g < r1; g += 4 * BLOCK) {
+    const float4 x = load_rows4(col, g, r0, r1, aligned), m = load_rows4(wbar, g, r0, r1, aligned);
+    const float v[4] = {static_cast<float>((static_cast<double>(x.x) - static_cast<double>(m.x)) * f),
+                        static_cast<float>((static_cast<double>(x.y) - static_cast<double>(m.y)) * f),
+                        static_cast<float>((static_cast<double>(x.z) - static_cast<double>(m.z)) * f),
+                        static_cast<float>((static_cast<double>(x.w) - static_cast<double>(m.w)) * f)};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (g + i >= r0 && g + i < r1) {
+        if (q32) q32[blockIdx.y * ldq + (g + i - row0)] = v[i];
+        lo = fminf(lo, v[i]);
+        hi = fmaxf(hi, v[i]);
+        bad |= !isfinite(v[i]);
+      }
+    }
   }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
@@ -337,24 +456,44 @@ __global__ void __launch_bounds__(BLOCK) chunk_affine_encode_kernel(const float*
   const float* wb = wbar + lay0;
   uint4* dst = reinterpret_cast<uint4*>(out + j * out_stride);
   uint4* dst_lo = reinterpret_cast<uint4*>(out + (static_cast<long long>(n) + j) * out_stride);
+  const float recip = PLANES == 2 ? 0.0f : affine_reciprocal(al, top);
+  const float near = (top + 1.0f) * 0x1p-21f;
+  const bool aligned = ((reinterpret_cast<uintptr_t>(col) | reinterpret_cast<uintptr_t>(wb)) & 15) == 0;
   for (long long c = c0 + blockIdx.x * static_cast<long long>(BLOCK) + threadIdx.x; c < c1;
        c += static_cast<long long>(gridDim.x) * BLOCK) {
     uint32_t w[4] = {0, 0, 0, 0}, wl[4] = {0, 0, 0, 0};
+    bool hard = recip == 0.0f;
+    if (!hard) {
 #pragma unroll
-    for (int k = 0; k < RPC; ++k) {
-      const long long r = c * RPC + k;
-      uint32_t u = 0;
-      if (r >= f0 && r < f1 && al != 0.0f) {
-        const float e = static_cast<float>((static_cast<double>(col[r]) - static_cast<double>(wb[r])) * f);
-        float q = rintf(__fdiv_rn(__fsub_rn(e, bl), al));
-        q = fminf(fmaxf(q, 0.0f), top);
-        u = static_cast<uint32_t>(q);
+      for (int k = 0; k < RPC; k += 4) {
+        const long long r = c * RPC + k;
+        const float4 x = load_rows4(col, r, f0, f1, aligned), m = load_rows4(wb, r, f0, f1, aligned);
+        const float e0 = static_cast<float>((static_cast<double>(x.x) - static_cast<double>(m.x)) * f);
+        const float e1 = static_cast<float>((static_cast<double>(x.y) - static_cast<double>(m.y)) * f);
+        const float e2 = static_cast<float>((static_cast<double>(x.z) - static_cast<double>(m.z)) * f);
+        const float e3 = static_cast<float>((static_cast<double>(x.w) - static_cast<double>(m.w)) * f);
+        if (r >= f0 && r < f1) put_code<W>(w, k, affine_code_by_reciprocal(e0, bl, recip, top, near, &hard));
+        if (r + 1 >= f0 && r + 1 < f1) put_code<W>(w, k + 1, affine_code_by_reciprocal(e1, bl, recip, top, near, &hard));
+        if (r + 2 >= f0 && r + 2 < f1) put_code<W>(w, k + 2, affine_code_by_reciprocal(e2, bl, recip, top, near, &hard));
+        if (r + 3 >= f0 && r + 3 < f1) put_code<W>(w, k + 3, affine_code_by_reciprocal(e3, bl, recip, top, near, &hard));
       }
-      if (PLANES == 2) {
-        put_code<W>(w, k, u >> 8);
-        put_code<W>(wl, k, u & 0xFFu);
-      } else {
-        put_code<W>(w, k, u);
+    }
+    if (hard) {
+      w[0] = w[1] = w[2] = w[3] = 0u;
+#pragma unroll
+      for (int k = 0; k < RPC; ++k) {
+        const long long r = c * RPC + k;
+        uint32_t u = 0;
+        if (r >= f0 && r < f1 && al != 0.0f) {
+          const float e = static_cast<float>((static_cast<double>(col[r]) - static_cast<double>(wb[r])) * f);
+          u = affine_code(e, bl, al, top);
+        }
+        if (PLANES == 2) {
+          put_code<W>(w, k, u >> 8);
+          put_code<W>(wl, k, u & 0xFFu);
+        } else {
+          put_code<W>(w, k, u);
+        }
       }
     }
     const long long q = internal[l] / RPC + c;
@@ -461,6 +600,35 @@ size_t count_items(const int64_t* offsets, int L) {
 
 // Carves the caller's buffer of a layered basis (codes | a | b | granule table | flat offsets |
 // internal offsets | block tables), builds and uploads the tables, and fills the descriptor.
+// Entry k of the granule table: (layer, valid rows, first flat row, 0) of the 64-byte granule whose first
+// internal row is k * gr; layer -1 behind the last layer.  A layer's internal rows are its flat rows
+// rounded up to whole granules, so a granule lies in the last layer whose internal offset is not above
+// its first row (empty layers share their offset with the layer after them and are passed over).
+__global__ void __launch_bounds__(BLOCK) granule_table_kernel(const long long* __restrict__ flat,
+                                                              const long long* __restrict__ internal, int L,
+                                                              long long gr, size_t entries, int4* __restrict__ tab) {
+  for (size_t k = blockIdx.x * static_cast<size_t>(BLOCK) + threadIdx.x; k < entries;
+       k += static_cast<size_t>(gridDim.x) * BLOCK) {
+    const long long row = static_cast<long long>(k) * gr;
+    int4 e = make_int4(-1, 0, 0, 0);
+    if (row < internal[L]) {
+      int lo = 0, hi = L - 1;
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (internal[mid] <= row) lo = mid;
+        else hi = mid - 1;
+      }
+      const long long len = flat[lo + 1] - flat[lo], k0 = row - internal[lo];
+      if (k0 < len) {
+        e.x = lo;
+        e.y = static_cast<int>(len - k0 < gr ? len - k0 : gr);
+        e.z = static_cast<int>(flat[lo] + k0);
+      }
+    }
+    tab[k] = e;
+  }
+}
+
 int prepare_layered_storage(twa_ctx* ctx, const Partition& p, long long D, int L, int n_cand, int code_bits,
                             void* mem, twa_layered_basis* out) {
   // carve the caller's buffer: codes | a | b | granule table | flat offsets | internal offsets
@@ -506,23 +674,10 @@ int prepare_layered_storage(twa_ctx* ctx, const Partition& p, long long D, int L
       cta_base[k + 1] = cta_base[k] + (last - l + 1);
     }
   }
-  // granule table: layer, valid rows, first flat row of every 64-byte granule of a column
+  // granule table: layer, valid rows, first flat row of every 64-byte granule of a column, written on
+  // the device from the two offset arrays (the table has a million entries at ViT-B/16 size: built on the
+  // host and copied from pageable memory it cost more than the quantiser's kernels)
   {
-    const long long gr = granule_rows(bits);
-    // (with slack, so that the last tile of a two-segment tiling finds entries for all its granules)
-    std::vector<int> tab(4 * (n_gran + TABLE_SLACK), 0);
-    for (size_t k = 0; k < n_gran + TABLE_SLACK; ++k) tab[4 * k] = -1;   // granules behind the last layer
-    for (int l = 0; l < L; ++l) {
-      const long long len = p.flat[l + 1] - p.flat[l];
-      for (long long k0 = 0; k0 < len; k0 += gr) {
-        const size_t gidx = static_cast<size_t>((p.internal[l] + k0) / gr);
-        tab[4 * gidx] = l;
-        tab[4 * gidx + 1] = static_cast<int>(len - k0 < gr ? len - k0 : gr);
-        tab[4 * gidx + 2] = static_cast<int>(p.flat[l] + k0);
-      }
-    }
-    TWA_CUDA_OK(ctx, cudaMemcpyAsync(gran, tab.data(), sizeof(int) * tab.size(), cudaMemcpyHostToDevice,
-                                     ctx->stream));
     TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_flat, p.flat.data(), sizeof(long long) * (L + 1),
                                      cudaMemcpyHostToDevice, ctx->stream));
     TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_int, p.internal.data(), sizeof(long long) * (L + 1),
@@ -531,7 +686,14 @@ int prepare_layered_storage(twa_ctx* ctx, const Partition& p, long long D, int L
                                      ctx->stream));
     TWA_CUDA_OK(ctx, cudaMemcpyAsync(d_cta_base, cta_base.data(), sizeof(int) * (ctas + 1),
                                      cudaMemcpyHostToDevice, ctx->stream));
-    TWA_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));
+    // (with slack, so that the last tile of a two-segment tiling finds entries for all its granules)
+    const size_t entries = n_gran + TABLE_SLACK;
+    int tgrid = static_cast<int>((entries + BLOCK - 1) / BLOCK);
+    if (tgrid > ctx->sm_count * 8) tgrid = ctx->sm_count * 8;
+    granule_table_kernel<<<tgrid, BLOCK, 0, ctx->stream>>>(d_flat, d_int, L, granule_rows(bits), entries,
+                                                          reinterpret_cast<int4*>(gran));
+    TWA_CUDA_OK(ctx, cudaGetLastError());
+    TWA_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));       // the host arrays above end with this scope
   }
 
   unsigned char* codes = reinterpret_cast<unsigned char*>(m);
@@ -653,7 +815,7 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
   minmax_kernel<<<grid, BLOCK, 0, ctx->stream>>>(P, ld, items, n, pmin, pmax);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   const float top = top_code(bits);
-  factors_kernel<<<(L + 127) / 128, 128, 0, ctx->stream>>>(pmin, pmax, first_item, L, n, top, a, b, ctx->d_status);
+  factors_kernel<<<L, 128, 0, ctx->stream>>>(pmin, pmax, first_item, L, n, top, a, b, ctx->d_status);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   long long max_len = 0;
   for (int l = 0; l < L; ++l) max_len = std::max(max_len, p.internal[l + 1] - p.internal[l]);
@@ -848,7 +1010,7 @@ int twa_layered_build_end_pass(twa_ctx* ctx, const twa_layered_basis* lb, const 
                                                                  first_item, L, n, reinterpret_cast<double*>(ws + w.inv),
                                                                  ctx->d_status);
   } else if (pass == 1) {
-    factors_kernel<<<(L + 127) / 128, 128, 0, ctx->stream>>>(reinterpret_cast<const float*>(ws + w.pmin),
+    factors_kernel<<<L, 128, 0, ctx->stream>>>(reinterpret_cast<const float*>(ws + w.pmin),
                                                              reinterpret_cast<const float*>(ws + w.pmax), first_item, L, n,
                                                              top_code(lb->code_bits), lb->a, lb->b, ctx->d_status);
   }

@@ -584,10 +584,13 @@ def twa_build_centered(ctx, W, D, layers, wbar_out, lws):
     return Basis(desc, W, None)
 
 
-def twa_quantize_affine(ctx, P32, layers, bits, lws):
+def twa_quantize_affine(ctx, P32, layers, bits, lws, mem=None):
+    """mem: a uint8 CUDA tensor of twa_layered_basis_bytes(layers, n, bits) bytes to hold the basis
+    (None: allocated here)."""
     arr, L = _offsets(layers)
-    mem = torch.empty(twa_layered_basis_bytes(layers, P32.n, bits), dtype=torch.uint8,
-                      device=P32.data.device)
+    if mem is None:
+        mem = torch.empty(twa_layered_basis_bytes(layers, P32.n, bits), dtype=torch.uint8,
+                          device=P32.data.device)
     desc = twa_layered_basis()
     rc = load().twa_quantize_affine(ctx, ctypes.byref(P32.desc), arr, L, int(bits), _ptr(mem),
                                     mem.numel(), ctypes.byref(desc), _ptr(lws), lws.numel())

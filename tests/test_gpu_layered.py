@@ -103,6 +103,48 @@ def test_quantize_affine_bit_exact(env, D, n, layers, bits):
 
 
 @pytest.mark.parametrize("bits", ALL_BITS)
+@pytest.mark.parametrize("lo,span", [(-0.37, 1.0), (0.0123, 3.3e-3), (-96.7, 200.1), (0.0, 2.9e-37), (-5.0, 2.5e38)])
+def test_quantize_affine_near_half_integers_matches_the_ieee_quotient(env, bits, lo, span):
+    """Elements whose quotient (e - b) / a sits on, or within a few ulps of, a half-integer, where the
+    code hangs on the last bit of the IEEE float32 operations the oracle performs; two layers with
+    different factors, one of them with a tiny or huge scale."""
+    ctx, _ = env
+    top = 2 ** bits - 1
+    cols = []
+    for lo_l, span_l in ((lo, span), (0.25, 0.731)):
+        lo32 = np.float32(lo_l)
+        hi32 = np.float32(np.float64(lo32) + span_l)
+        a32 = np.float32(hi32 - lo32) / np.float32(top)
+        ks = np.arange(0, min(top, 300), dtype=np.float64) + 0.5
+        with np.errstate(over="ignore", under="ignore"):
+            base = (np.float64(lo32) + ks * np.float64(a32)).astype(np.float32)
+            vals = [base]
+            for _ in range(5):
+                vals.append(np.nextafter(vals[-1], np.float32(np.inf)))
+            dn = base
+            for _ in range(5):
+                dn = np.nextafter(dn, np.float32(-np.inf))
+                vals.append(dn)
+        col = np.concatenate(vals + [np.array([lo32, hi32], dtype=np.float32)])
+        cols.append(np.clip(col, lo32, hi32))
+    layers = [0, cols[0].size, cols[0].size + cols[1].size]
+    D = layers[-1]
+    n = 2
+    P = torch.zeros((n, inputs.padded_ld(D, 4)), dtype=torch.float32, device=DEV)
+    flat = np.concatenate(cols)
+    P[0, :D] = torch.from_numpy(flat).to(DEV)
+    P[1, :D] = torch.from_numpy(np.concatenate([c[::-1] for c in cols])).to(DEV)
+    lws = twa.new_layered_workspace(layers, n, DEV)
+    lb = twa.twa_quantize_affine(ctx, twa.basis_from_tensor(P, D), layers, bits, lws)
+    status_ok(ctx)
+    codes_g, a_g, b_g = twa.twa_layered_export(ctx, lb)
+    codes_o, a_o, b_o = orc.affine_quantize(np.asfortranarray(P[:, :D].cpu().numpy().T), layers, bits)
+    np.testing.assert_array_equal(a_g.cpu().numpy(), a_o)
+    np.testing.assert_array_equal(b_g.cpu().numpy(), b_o)
+    np.testing.assert_array_equal(unpack_unsigned(codes_g.cpu().numpy(), D, bits), codes_o)
+
+
+@pytest.mark.parametrize("bits", ALL_BITS)
 @pytest.mark.parametrize("D,n,layers,chunk_rows", [
     (1777, 6, [0, 7, 300, 301, 1000, 1777], 500),              # chunk edges inside layers and inside 16-byte code groups
     (70001, 33, [0, 64, 1000, 1001, 30000, 30017, 65536, 70001], 8192),
