@@ -442,6 +442,15 @@ def test_host_side_argument_errors(env):
     wide = torch.zeros((twa.TWA_MAX_N + 1, 16), device=DEV)
     assert code_of(lambda: twa.twa_build_basis(ctx, wide, 16, torch.zeros(16, device=DEV), ws)) == \
         twa.TWA_ERR_UNSUPPORTED
+    # the one-call build: a width it does not have, too many columns, a workspace too small -- all before any launch
+    W = random_basis(D, n, 2)
+    before = W.clone()
+    wbar = torch.zeros(D, device=DEV)
+    assert code_of(lambda: twa.twa_build_quantized(ctx, W, D, wbar, [8, 5], ws)) == twa.TWA_ERR_UNSUPPORTED
+    assert code_of(lambda: twa.twa_build_quantized(ctx, W, D, wbar, [8], ws[:16])) == twa.TWA_ERR_WORKSPACE
+    assert code_of(lambda: twa.twa_build_quantized(ctx, wide, 16, torch.zeros(16, device=DEV), [8], ws)) == \
+        twa.TWA_ERR_UNSUPPORTED
+    assert torch.equal(W, before)
     status_ok(ctx)
 
 
