@@ -510,6 +510,51 @@ def measure_steps(env, ctx, twa, wl, basis, wbar, ws, pool, steps, warmup, min_t
     return out
 
 
+def graph_replay_ms(env, twa, wl, basis, wbar, pool, steps, min_total_ms):
+    """The same K steps captured once into a CUDA graph (a context of its own on a side stream: the
+    default stream cannot be captured) and replayed: ms per step, max over ranks.  For the small
+    workloads, where a step is two launches of tens of microseconds."""
+    import torch
+    D, n = wl.D, wl.n
+    stream = torch.cuda.Stream(device=env.dev)
+    stream.wait_stream(torch.cuda.current_stream(env.dev))
+    with torch.cuda.stream(stream):
+        ctx = twa.twa_create(env.local, stream=stream)
+        ws = twa.new_workspace(env.dev)
+        alpha = torch.zeros(n, dtype=torch.float32, device=env.dev)
+        w = torch.empty(D, dtype=torch.float32, device=env.dev)
+        twa.twa_step(ctx, basis, pool[0], LR, LAM, alpha, wbar, w, ws)          # raises the kernels' limits
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for t in range(steps):
+                twa.twa_step(ctx, basis, pool[t % len(pool)], LR, LAM, alpha, wbar, w, ws)
+        for _ in range(3):
+            graph.replay()
+        stream.synchronize()
+        regions, repeats, k = [], 1, 0
+        while k < repeats:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            env.barrier()
+            e0.record(stream)
+            graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+            env.barrier()
+            ms = max_over_ranks([e0.elapsed_time(e1)], env.dev)[0]
+            regions.append(ms)
+            if k == 0:
+                repeats = max(1, min(400, int(math.ceil(min_total_ms / max(ms, 1e-3)))))
+            k += 1
+        code, _ = twa.twa_get_status(ctx)
+        del graph
+        twa.twa_destroy(ctx)
+    torch.cuda.current_stream(env.dev).wait_stream(stream)
+    if code != 0:
+        raise RuntimeError(f"replayed step failed: {twa.twa_strerror(code)}")
+    return sum(regions) / len(regions) / steps
+
+
 def clock_fields(sampler, walls, series):
     """The clocks over all repeats, and per repeat the sampled SM clock with ms x MHz (how the
     time follows the clock, without touching any clock)."""
@@ -732,7 +777,11 @@ def other_configs(env, ctx, twa, inputs, ws, args, peak):
             if sampler is not None:
                 sampler.stop()
                 clocks = sampler.summary(m["walls"][0][0], m["walls"][-1][1])
-            out.append(config_entry(wl, bits, m, peak, build_ms, quant_ms.get(bits), clocks, fused_ms, widths))
+            entry = config_entry(wl, bits, m, peak, build_ms, quant_ms.get(bits), clocks, fused_ms, widths)
+            if wl.n * ((wl.D * bits + 7) // 8) < 2.5 * L2_BYTES or name == "resnet18":
+                entry["cuda_graph_replay_ms_per_step"] = graph_replay_ms(env, twa, wl, bases[bits], wbar, pool,
+                                                                         args.steps, args.configs_min_ms / 2)
+            out.append(entry)
         del bases, wbar, pool
         torch.cuda.empty_cache()
     # the other modes of the library, each through its own benchmark routine, condensed

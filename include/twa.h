@@ -30,6 +30,11 @@
  *    context's status word and read with twa_get_status(), which
  *    synchronises the stream.  After a device-side error the outputs of that
  *    call are unspecified.
+ *  - twa_project, twa_lift, twa_step, twa_step_adam, twa_project_batch and the twa_layered_*
+ *    stepping calls only enqueue kernels on the context's stream: they may be captured into a
+ *    CUDA graph (after one call of the same shape outside the capture, which raises the kernels'
+ *    shared-memory limits) and replayed; pointers, sizes and scalar arguments are those of the
+ *    captured call.
  *  - One context per stream; calls on one context must not overlap in time
  *    from several host threads.  Different contexts may be driven from different
  *    threads: the only state they share is a per-process cache of kernel attributes

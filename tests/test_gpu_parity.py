@@ -268,6 +268,62 @@ def test_step_sequence_and_determinism(env, dequant_path, bits):
         assert torch.equal(a1, a2) and torch.equal(w1, w2) and torch.equal(c1, c2)
 
 
+@pytest.mark.parametrize("bits,gdt", [(8, torch.bfloat16), (4, torch.float32), (32, torch.float32)])
+def test_step_replayed_from_a_cuda_graph(bits, gdt):
+    """A training loop may capture twa_step once and replay it: the call only enqueues kernels (tensor
+    maps and arguments are fixed at capture), so a replay with new bytes in the same gradient buffer
+    is the next step.  Ten replayed steps against ten direct calls (bit for bit) and against the oracle."""
+    torch.cuda.set_device(0)
+    stream = torch.cuda.Stream()
+    D, n, steps = 150001, 24, 10
+    with torch.cuda.stream(stream):
+        ctx = twa.twa_create(0, stream=stream)
+        ws = twa.new_workspace(DEV)
+        P = random_basis(D, n, 808)
+        B = twa.basis_from_tensor(P, D)
+        if bits != 32:
+            B = twa.twa_quantize_basis(ctx, B, bits, ws)
+            codes, s = twa.twa_basis_export(ctx, B)
+            co, so = orc.unpack_codes(codes.cpu().numpy(), D, bits), s.cpu().numpy()
+        gen = torch.Generator(device=DEV)
+        gen.manual_seed(99)
+        gs = [(torch.randn(D, generator=gen, device=DEV) * 1e-3).to(gdt) for _ in range(steps)]
+        wbar = torch.randn(D, generator=gen, device=DEV)
+        # direct calls
+        alpha_d = torch.zeros(n, device=DEV)
+        w_d = torch.empty(D, device=DEV)
+        for g in gs:
+            twa.twa_step(ctx, B, g, 0.1, 0.01, alpha_d, wbar, w_d, ws)
+        # one captured call, replayed on fresh bytes in the same buffers
+        g_buf = torch.zeros(D, device=DEV, dtype=gdt)
+        alpha_g = torch.zeros(n, device=DEV)
+        w_g = torch.empty(D, device=DEV)
+        twa.twa_step(ctx, B, g_buf, 0.1, 0.01, alpha_g, wbar, w_g, ws)      # warm-up outside the capture
+        alpha_g.zero_()
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            twa.twa_step(ctx, B, g_buf, 0.1, 0.01, alpha_g, wbar, w_g, ws)
+        alpha_g.zero_()
+        for g in gs:
+            g_buf.copy_(g)
+            graph.replay()
+        stream.synchronize()
+        status_ok(ctx)
+        assert torch.equal(alpha_g, alpha_d) and torch.equal(w_g, w_d)
+        a_o = np.zeros(n)
+        for g in gs:
+            g_h = g.float().cpu().numpy()
+            if bits != 32:
+                a_o, w_o, _ = orc.step(co, so, g_h, a_o, wbar.cpu().numpy(), 0.1, 0.01)
+            else:
+                a_o, w_o, _ = orc.step_f32(host_cols(P, D), g_h, a_o, wbar.cpu().numpy(), 0.1, 0.01)
+        assert rel(alpha_g.cpu().numpy(), a_o) <= TOL
+        assert rel(w_g.cpu().numpy(), w_o) <= TOL
+        del graph
+        twa.twa_destroy(ctx)
+
+
 def test_step_host_matches_device_step(env):
     ctx, ws = env
     D, n = 30011, 10
