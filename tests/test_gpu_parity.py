@@ -415,6 +415,33 @@ def test_build_basis(env, D, n):
     assert torch.all(W[:, D:] == 0)
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("scale", [1e15, 1e-15])
+def test_build_basis_on_very_large_and_very_small_candidates(env, scale, mode):
+    """Q does not depend on the scale of the candidates: with columns of norm 1e15 and 1e-15 the build
+    still returns the oracle's vectors (norms, Gram matrix and coefficients must not overflow or
+    flush on the way)."""
+    ctx, ws = env
+    D, n = 60001, 19
+    W = inputs.trajectory_candidates(D, n, 0.005, 0.001, 5, DEV, ld=inputs.padded_ld(D, 4))
+    W *= scale
+    A = host_cols(W, D).copy()
+    wbar = torch.empty(D, device=DEV)
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_BUILD_PANEL, mode)
+    try:
+        twa.twa_build_basis(ctx, W, D, wbar, ws)
+    finally:
+        twa.twa_set_tuning(ctx, twa.TWA_TUNE_BUILD_PANEL, 0)
+    status_ok(ctx)
+    Pg = host_cols(W, D).astype(np.float64)
+    assert np.max(np.abs(Pg.T @ Pg - np.eye(n))) <= 1e-5
+    Q, _, bad = orc.cgs2(A)
+    assert bad is None
+    kappa = np.linalg.cond(A.astype(np.float64))
+    assert np.max(np.linalg.norm(Pg - Q, axis=0)) <= 10 * kappa * np.finfo(np.float32).eps
+    np.testing.assert_array_equal(wbar.cpu().numpy(), orc.mean(A).astype(np.float32))
+
+
 def test_basis_invariants_recover_candidates_and_reject_orthogonal(env):
     ctx, ws = env
     D, n = 60013, 10
