@@ -755,6 +755,34 @@ def test_panel_build_agrees_with_column_build_and_oracle(env, D, n, step):
         assert np.max(np.linalg.norm(out[mode] - out[1], axis=0)) <= 20 * kappa * np.finfo(np.float32).eps, mode
 
 
+def test_build_quantized_with_a_dependent_candidate(env):
+    """A candidate that repeats an earlier one: both forms of the call report it, zero its column and
+    give it the scale 0 and the codes 0."""
+    ctx, ws = env
+    D, n = 30011, 21
+    ld = inputs.padded_ld(D, 4)
+    outs = []
+    for one_call in (False, True):
+        W = inputs.trajectory_candidates(D, n, 0.005, 0.001, 78, DEV, ld=ld)
+        W[13] = W[4]
+        wbar = torch.empty(D, device=DEV)
+        if one_call:
+            P32, (q8, q4) = twa.twa_build_quantized(ctx, W, D, wbar, [8, 4], ws)
+        else:
+            P32 = twa.twa_build_basis(ctx, W, D, wbar, ws)
+            q8, q4 = twa.twa_quantize_basis(ctx, P32, 8, ws), twa.twa_quantize_basis(ctx, P32, 4, ws)
+        code, detail = twa.twa_get_status(ctx)
+        assert (code, detail) == (twa.TWA_ERR_RANK_DEFICIENT, 13)
+        twa.twa_clear_status(ctx)
+        assert torch.all(W[13] == 0)
+        for q in (q8, q4):
+            codes, scales = twa.twa_basis_export(ctx, q)
+            assert scales[13].item() == 0.0 and torch.all(codes[13] == 0)
+        outs.append((W, q8.data, q8.scales, q4.data, q4.scales))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
 @pytest.mark.parametrize("mode", [0, 1, 2])
 @pytest.mark.parametrize("D,n", [(1, 1), (5003, 3), (70001, 33), (300007, 20), (40001, 128)])
 def test_build_quantized_equals_build_then_quantize_bit_for_bit(env, D, n, mode):
