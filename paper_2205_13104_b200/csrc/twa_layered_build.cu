@@ -103,9 +103,13 @@ __global__ void __launch_bounds__(BLOCK) centred_sumsq_kernel(const float* __res
                                                               const float* __restrict__ wbar,
                                                               const Item* __restrict__ items, int n,
                                                               double* __restrict__ partial) {
+  // blocks of one item and neighbouring columns run together, so the item's rows of the shared vectors
+  // (w_bar) are fetched from memory once and found in the cache by the other columns
+  const unsigned item_k = blockIdx.x / n;
+  const int col_j = blockIdx.x % n;
   __shared__ double sh[BLOCK / 32];
-  const Item it = items[blockIdx.x];
-  const float* col = W + blockIdx.y * ldw;
+  const Item it = items[item_k];
+  const float* col = W + col_j * ldw;
   const bool aligned = ((reinterpret_cast<uintptr_t>(col) | reinterpret_cast<uintptr_t>(wbar)) & 15) == 0;
   double s = 0;
   for (long long g = (it.r0 & ~3LL) + 4 * threadIdx.x; g < it.r1; g += 4 * BLOCK) {
@@ -119,7 +123,7 @@ __global__ void __launch_bounds__(BLOCK) centred_sumsq_kernel(const float* __res
     s += v3 * v3;
   }
   const double t = block_sum_d(s, sh);
-  if (threadIdx.x == 0) partial[static_cast<size_t>(blockIdx.x) * n + blockIdx.y] = t;
+  if (threadIdx.x == 0) partial[static_cast<size_t>(item_k) * n + col_j] = t;
 }
 
 // inv[l][i] = 1 / sqrt(sum of the layer's partials in item order), 0 for a zero vector
@@ -138,9 +142,13 @@ __global__ void __launch_bounds__(BLOCK) centre_scale_kernel(float* __restrict__
                                                              const float* __restrict__ wbar,
                                                              const Item* __restrict__ items, int n,
                                                              const double* __restrict__ inv) {
-  const Item it = items[blockIdx.x];
-  float* col = W + blockIdx.y * ldw;
-  const double f = inv[static_cast<size_t>(it.layer) * n + blockIdx.y];
+  // blocks of one item and neighbouring columns run together, so the item's rows of the shared vectors
+  // (w_bar) are fetched from memory once and found in the cache by the other columns
+  const unsigned item_k = blockIdx.x / n;
+  const int col_j = blockIdx.x % n;
+  const Item it = items[item_k];
+  float* col = W + col_j * ldw;
+  const double f = inv[static_cast<size_t>(it.layer) * n + col_j];
   const bool aligned = ((reinterpret_cast<uintptr_t>(col) | reinterpret_cast<uintptr_t>(wbar)) & 15) == 0;
   for (long long g = (it.r0 & ~3LL) + 4 * threadIdx.x; g < it.r1; g += 4 * BLOCK) {
     const float4 x = load_rows4(col, g, it.r0, it.r1, aligned), m = load_rows4(wbar, g, it.r0, it.r1, aligned);
@@ -164,9 +172,13 @@ __global__ void __launch_bounds__(BLOCK) centre_scale_kernel(float* __restrict__
 __global__ void __launch_bounds__(BLOCK) minmax_kernel(const float* __restrict__ P, long long ld,
                                                        const Item* __restrict__ items, int n,
                                                        float* __restrict__ pmin, float* __restrict__ pmax) {
+  // (column, item), the item running fastest: neighbouring blocks read neighbouring rows of one column
+  const unsigned items_n = gridDim.x / n;
+  const unsigned item_k = blockIdx.x % items_n;
+  const int col_j = blockIdx.x / items_n;
   __shared__ float smin[BLOCK / 32], smax[BLOCK / 32];
-  const Item it = items[blockIdx.x];
-  const float* col = P + blockIdx.y * ld;
+  const Item it = items[item_k];
+  const float* col = P + col_j * ld;
   float lo = INFINITY, hi = -INFINITY;
   bool bad = false;                              // fmin / fmax drop NaN: track non-finite input apart
   const bool aligned = (reinterpret_cast<uintptr_t>(col) & 15) == 0;
@@ -199,8 +211,8 @@ __global__ void __launch_bounds__(BLOCK) minmax_kernel(const float* __restrict__
       lo = fminf(lo, smin[w]);
       hi = fmaxf(hi, smax[w]);
     }
-    pmin[static_cast<size_t>(blockIdx.x) * n + blockIdx.y] = bad ? NAN : lo;
-    pmax[static_cast<size_t>(blockIdx.x) * n + blockIdx.y] = hi;
+    pmin[static_cast<size_t>(item_k) * n + col_j] = bad ? NAN : lo;
+    pmax[static_cast<size_t>(item_k) * n + col_j] = hi;
   }
 }
 
@@ -348,10 +360,14 @@ __global__ void __launch_bounds__(BLOCK) chunk_centred_sumsq_kernel(const float*
                                                                     const float* __restrict__ wbar,
                                                                     const Item* __restrict__ items, int n,
                                                                     double* __restrict__ partial) {
+  // blocks of one item and neighbouring columns run together, so the item's rows of the shared vectors
+  // (w_bar) are fetched from memory once and found in the cache by the other columns
+  const unsigned item_k = blockIdx.x / n;
+  const int col_j = blockIdx.x % n;
   __shared__ double sh[BLOCK / 32];
-  const Item it = items[blockIdx.x];
+  const Item it = items[item_k];
   const long long r0 = it.r0 > row0 ? it.r0 : row0, r1 = it.r1 < row1 ? it.r1 : row1;
-  const float* col = chunk + blockIdx.y * ld - row0;
+  const float* col = chunk + col_j * ld - row0;
   const bool aligned = ((reinterpret_cast<uintptr_t>(col) | reinterpret_cast<uintptr_t>(wbar)) & 15) == 0;
   double s = 0;
   for (long long g = (r0 & ~3LL) + 4 * threadIdx.x; g < r1; g += 4 * BLOCK) {
@@ -364,7 +380,7 @@ __global__ void __launch_bounds__(BLOCK) chunk_centred_sumsq_kernel(const float*
     s += v3 * v3;
   }
   const double t = block_sum_d(s, sh);
-  if (threadIdx.x == 0) partial[static_cast<size_t>(blockIdx.x) * n + blockIdx.y] += t;
+  if (threadIdx.x == 0) partial[static_cast<size_t>(item_k) * n + col_j] += t;
 }
 
 // e = (w - w_bar) / ||.|| for the chunk's rows (the expression of centre_scale_kernel), its min / max
@@ -376,11 +392,15 @@ __global__ void __launch_bounds__(BLOCK) chunk_minmax_kernel(const float* __rest
                                                              const double* __restrict__ inv, float* __restrict__ pmin,
                                                              float* __restrict__ pmax, float* __restrict__ q32,
                                                              long long ldq) {
+  // blocks of one item and neighbouring columns run together, so the item's rows of the shared vectors
+  // (w_bar) are fetched from memory once and found in the cache by the other columns
+  const unsigned item_k = blockIdx.x / n;
+  const int col_j = blockIdx.x % n;
   __shared__ float smin[BLOCK / 32], smax[BLOCK / 32];
-  const Item it = items[blockIdx.x];
+  const Item it = items[item_k];
   const long long r0 = it.r0 > row0 ? it.r0 : row0, r1 = it.r1 < row1 ? it.r1 : row1;
-  const float* col = chunk + blockIdx.y * ld - row0;
-  const double f = inv[static_cast<size_t>(it.layer) * n + blockIdx.y];
+  const float* col = chunk + col_j * ld - row0;
+  const double f = inv[static_cast<size_t>(it.layer) * n + col_j];
   float lo = INFINITY, hi = -INFINITY;
   bool bad = false;
   const bool aligned = ((reinterpret_cast<uintptr_t>(col) | reinterpret_cast<uintptr_t>(wbar)) & 15) == 0;
@@ -393,7 +413,7 @@ __global__ void __launch_bounds__(BLOCK) chunk_minmax_kernel(const float* __rest
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       if (g + i >= r0 && g + i < r1) {
-        if (q32) q32[blockIdx.y * ldq + (g + i - row0)] = v[i];
+        if (q32) q32[col_j * ldq + (g + i - row0)] = v[i];
         lo = fminf(lo, v[i]);
         hi = fmaxf(hi, v[i]);
         bad |= !isfinite(v[i]);
@@ -417,7 +437,7 @@ __global__ void __launch_bounds__(BLOCK) chunk_minmax_kernel(const float* __rest
       lo = fminf(lo, smin[w]);
       hi = fmaxf(hi, smax[w]);
     }
-    const size_t at = static_cast<size_t>(blockIdx.x) * n + blockIdx.y;
+    const size_t at = static_cast<size_t>(item_k) * n + col_j;
     const float old_lo = pmin[at], old_hi = pmax[at];
     bad |= isnan(old_lo);
     pmin[at] = bad ? NAN : fminf(lo, old_lo);
@@ -765,7 +785,7 @@ int twa_build_centered(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, co
   const int* first_item = reinterpret_cast<const int*>(ws + w.first_item);
   double* partial = reinterpret_cast<double*>(ws + w.partial);
   double* inv = reinterpret_cast<double*>(ws + w.inv);
-  const dim3 grid(static_cast<unsigned>(p.items.size()), static_cast<unsigned>(n));
+  const unsigned grid = static_cast<unsigned>(p.items.size() * n);      // (item, column), the column running fastest
   centred_sumsq_kernel<<<grid, BLOCK, 0, ctx->stream>>>(W, ldw, wbar_out, items, n, partial);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   inv_norm_kernel<<<(L * n + 255) / 256, 256, 0, ctx->stream>>>(partial, first_item, L, n, inv, ctx->d_status);
@@ -811,7 +831,7 @@ int twa_quantize_affine(twa_ctx* ctx, const twa_basis* P32, const int64_t* offse
   float* pmax = reinterpret_cast<float*>(ws + w.pmax);
   const float* P = static_cast<const float*>(P32->data);
   const long long ld = P32->col_stride / 4;
-  const dim3 grid(static_cast<unsigned>(p.items.size()), static_cast<unsigned>(n));
+  const unsigned grid = static_cast<unsigned>(p.items.size() * n);      // (item, column), the column running fastest
   minmax_kernel<<<grid, BLOCK, 0, ctx->stream>>>(P, ld, items, n, pmin, pmax);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   const float top = top_code(bits);
@@ -961,7 +981,7 @@ int twa_layered_build_feed(twa_ctx* ctx, const twa_layered_basis* lb, const int6
   char* ws = static_cast<char*>(lws);
   const Item* items = reinterpret_cast<const Item*>(ws + w.items) + k0;
   const size_t cell0 = static_cast<size_t>(k0) * n;
-  const dim3 grid(static_cast<unsigned>(k1 - k0), static_cast<unsigned>(n));
+  const unsigned grid = static_cast<unsigned>((k1 - k0) * n);            // (item, column), the column running fastest
   const double* inv = reinterpret_cast<const double*>(ws + w.inv);
   if (pass == 0) {
     rc = twa_mean(ctx, chunk, rows, n, ld, wbar + row0);
