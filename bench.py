@@ -555,6 +555,49 @@ def graph_replay_ms(env, twa, wl, basis, wbar, pool, steps, min_total_ms):
     return sum(regions) / len(regions) / steps
 
 
+def optimiser_entries(env, ctx, twa, inputs, wl, basis, wbar, ws, pool, steps, min_total_ms, peak):
+    """Two more calls of the library on this workload, as "configs" entries: the fused step with Adam
+    and a cosine schedule on the coefficients, and a fixed-weight average of the candidates."""
+    import torch
+    D, n, bits = wl.D, wl.n, basis.bits
+    g_bytes = 2 if wl.g_dtype == "bf16" else 4
+    alpha = torch.zeros(n, dtype=torch.float32, device=env.dev)
+    m1 = torch.zeros(n, dtype=torch.float32, device=env.dev)
+    m2 = torch.zeros(n, dtype=torch.float32, device=env.dev)
+    w = torch.empty(D, dtype=torch.float32, device=env.dev)
+
+    def adam_step(t):
+        lr = twa.twa_cosine_lr(0.01, t % 1000, 1000)
+        twa.twa_step_adam(ctx, basis, pool[t % len(pool)], lr, t + 1, alpha, m1, m2, wbar, w, ws, weight_decay=0.01)
+
+    regions, _ = timed_regions(env, adam_step, steps, 3, min_total_ms)
+    ms = sum(regions) / len(regions) / steps
+    sb = step_bytes(D, n, bits, g_bytes)
+    out = [{"mode": "fused step with Adam (decoupled decay) and a cosine schedule on the coefficients (twa_step_adam)",
+            "workload": workload_label(wl, D, bits), "bits": bits, "ms_per_step": ms, "repeats": len(regions),
+            "GBps": sb / (ms * 1e-3) / 1e9, "frac_of_measured_copy_peak": sb / (ms * 1e-3) / 1e9 / peak,
+            "frac_of_8TBps": sb / (ms * 1e-3) / 1e9 / 8000.0, "bytes_per_step": sb}]
+    W = wl.candidates(env.dev, ld=inputs.padded_ld(D, 128))
+    weights = torch.full((n,), 1.0 / n, dtype=torch.float32, device=env.dev)
+
+    def average(t):
+        twa.twa_weighted_average(ctx, W, D, weights, w, ws)
+
+    regions, _ = timed_regions(env, average, steps, 3, min_total_ms)
+    ms = sum(regions) / len(regions) / steps
+    ab = 4 * D * (n + 1)
+    out.append({"mode": "fixed-weight average of the n candidates (twa_weighted_average: SWA, LAWA, EMA by the weights)",
+                "workload": f"{wl.name}: D={D} n={n} float32 candidates", "bits": 32, "ms_per_call": ms,
+                "repeats": len(regions), "GBps": ab / (ms * 1e-3) / 1e9,
+                "frac_of_measured_copy_peak": ab / (ms * 1e-3) / 1e9 / peak, "frac_of_8TBps": ab / (ms * 1e-3) / 1e9 / 8000.0,
+                "bytes_per_call": ab})
+    code, _ = twa.twa_get_status(ctx)
+    if code != 0:
+        raise RuntimeError(f"optimiser entries failed: {twa.twa_strerror(code)}")
+    del W, w
+    return out
+
+
 def clock_fields(sampler, walls, series):
     """The clocks over all repeats, and per repeat the sampled SM clock with ms x MHz (how the
     time follows the clock, without touching any clock)."""
@@ -782,6 +825,9 @@ def other_configs(env, ctx, twa, inputs, ws, args, peak):
                 entry["cuda_graph_replay_ms_per_step"] = graph_replay_ms(env, twa, wl, bases[bits], wbar, pool,
                                                                          args.steps, args.configs_min_ms / 2)
             out.append(entry)
+        if name == "resnet50":
+            out.extend(optimiser_entries(env, ctx, twa, inputs, wl, bases[8], wbar, ws, pool, args.steps,
+                                         args.configs_min_ms / 2, peak))
         del bases, wbar, pool
         torch.cuda.empty_cache()
     # the other modes of the library, each through its own benchmark routine, condensed
