@@ -83,6 +83,37 @@ def test_project_batch(env, D, n, batch, bits, gdt):
     assert torch.equal(C2, C[:batch])
 
 
+@pytest.mark.parametrize("bits", [8, 4])
+def test_project_batch_replayed_from_a_cuda_graph(bits):
+    """twa_project_batch (two passes of eight gradients here) captured once and replayed on new bytes
+    in the same gradient buffer: the coefficients of a direct call, bit for bit."""
+    torch.cuda.set_device(0)
+    stream = torch.cuda.Stream()
+    D, n, batch = 70001, 33, 11
+    with torch.cuda.stream(stream):
+        ctx = twa.twa_create(0, stream=stream)
+        ws = twa.new_workspace(DEV)
+        B, _ = _basis(ctx, ws, D, n, bits, 5)
+        G_buf = torch.zeros_like(_gradients(D, batch, torch.bfloat16, 1))
+        C_g = torch.empty((batch, n), device=DEV)
+        twa.twa_project_batch(ctx, B, G_buf, C_g, ws)                  # warm-up outside the capture
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            twa.twa_project_batch(ctx, B, G_buf, C_g, ws)
+        for seed in (2, 3):
+            G = _gradients(D, batch, torch.bfloat16, seed)
+            C_d = torch.empty((batch, n), device=DEV)
+            twa.twa_project_batch(ctx, B, G, C_d, ws)
+            G_buf.copy_(G)
+            graph.replay()
+            stream.synchronize()
+            assert torch.equal(C_g, C_d)
+        status_ok(ctx)
+        del graph
+        twa.twa_destroy(ctx)
+
+
 def test_project_batch_float32_basis_and_group(env):
     ctx, ws = env
     D, n, batch = 10007, 6, 3

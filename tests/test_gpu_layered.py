@@ -358,6 +358,40 @@ def test_layered_step_matches_oracle_over_iterations(env, D, n, layers, bits):
         beta_o = beta.cpu().numpy().astype(np.float64)
 
 
+@pytest.mark.parametrize("bits", [8, 4])
+def test_layered_step_replayed_from_a_cuda_graph(bits):
+    """twa_layered_step (three launches) captured once and replayed on new gradient bytes: the same
+    coefficients and weights as direct calls, bit for bit."""
+    torch.cuda.set_device(0)
+    stream = torch.cuda.Stream()
+    D, n, layers = 90001, 12, [0, 100, 101, 30000, 65536, 90001]
+    L = len(layers) - 1
+    with torch.cuda.stream(stream):
+        ctx = twa.twa_create(0, stream=stream)
+        lb, wbar, _, _, _ = _layered_basis(ctx, D, n, layers, bits, 77)
+        sws = twa.new_layered_step_workspace(lb)
+        gs = [inputs.gradient(D, 1e-2, 3, it, torch.bfloat16, DEV) for it in range(6)]
+        beta_d, w_d = torch.zeros((L, n), device=DEV), torch.empty(D, device=DEV)
+        for g in gs:
+            twa.twa_layered_step(ctx, lb, g, 0.5, 1e-2, beta_d, wbar, w_d, sws)
+        g_buf = torch.zeros(D, device=DEV, dtype=torch.bfloat16)
+        beta_g, w_g = torch.zeros((L, n), device=DEV), torch.empty(D, device=DEV)
+        twa.twa_layered_step(ctx, lb, g_buf, 0.5, 1e-2, beta_g, wbar, w_g, sws)     # warm-up outside the capture
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            twa.twa_layered_step(ctx, lb, g_buf, 0.5, 1e-2, beta_g, wbar, w_g, sws)
+        beta_g.zero_()
+        for g in gs:
+            g_buf.copy_(g)
+            graph.replay()
+        stream.synchronize()
+        status_ok(ctx)
+        assert torch.equal(beta_g, beta_d) and torch.equal(w_g, w_d)
+        del graph
+        twa.twa_destroy(ctx)
+
+
 def test_layered_step_reports_nonfinite_and_bad_arguments(env):
     ctx, _ = env
     D, n, layers = 40000, 5, [0, 100, 20000, 40000]
