@@ -34,7 +34,8 @@
  *    stepping calls only enqueue kernels on the context's stream: they may be captured into a
  *    CUDA graph (after one call of the same shape outside the capture, which raises the kernels'
  *    shared-memory limits) and replayed; pointers, sizes and scalar arguments are those of the
- *    captured call.
+ *    captured call (the learning rate, and for the Adam steps the step count behind the bias
+ *    corrections, are such scalars: a schedule needs one capture per value).
  *  - One context per stream; calls on one context must not overlap in time
  *    from several host threads.  Different contexts may be driven from different
  *    threads: the only state they share is a per-process cache of kernel attributes
