@@ -92,6 +92,48 @@ __device__ __forceinline__ void gram_accumulate(const double* T, double (&acc)[(
   }
 }
 
+// The same for 32 columns (four 8 x 8 blocks a side) with the symmetry used: only the ten blocks on and
+// above the diagonal are formed, three or two per warp (`pairs`), ten tensor-pipe products per four rows
+// instead of sixteen; the factorisation reads the upper triangle only, and sym4_store writes zeros below.
+struct Sym4Pairs {
+  int ib[3], jb[3], count;
+};
+__device__ __forceinline__ Sym4Pairs sym4_pairs(int warp) {
+  switch (warp) {
+    case 0: return {{0, 0, 0}, {0, 1, 2}, 3};
+    case 1: return {{0, 1, 3}, {3, 3, 3}, 3};
+    case 2: return {{1, 1, 1}, {1, 2, 2}, 2};
+    default: return {{2, 2, 2}, {2, 3, 3}, 2};
+  }
+}
+__device__ __forceinline__ void gram_accumulate_sym4(const double* T, double (&acc)[1][4][2], int warp, int lane) {
+  const Sym4Pairs p = sym4_pairs(warp);
+  const int off = (lane >> 2) * DSTR + (lane & 3);
+  const int oa0 = p.ib[0] * 8 * DSTR + off, oa1 = p.ib[1] * 8 * DSTR + off, oa2 = p.ib[2] * 8 * DSTR + off;
+  const int ob0 = p.jb[0] * 8 * DSTR + off, ob1 = p.jb[1] * 8 * DSTR + off, ob2 = p.jb[2] * 8 * DSTR + off;
+  const bool three = p.count == 3;
+#pragma unroll 2
+  for (int k0 = 0; k0 < RT; k0 += 4) {
+    dmma_8x8x4(acc[0][0], T[oa0 + k0], T[ob0 + k0]);
+    dmma_8x8x4(acc[0][1], T[oa1 + k0], T[ob1 + k0]);
+    if (three) dmma_8x8x4(acc[0][2], T[oa2 + k0], T[ob2 + k0]);
+  }
+}
+// This warp's blocks of the block's Gram matrix (row-major [32][32]) and zeros in their mirror images.
+__device__ __forceinline__ void sym4_store(double* out, const double (&acc)[1][4][2], int warp, int lane) {
+  const Sym4Pairs p = sym4_pairs(warp);
+  for (int s = 0; s < p.count; ++s) {
+    double* at = out + (p.ib[s] * 8 + (lane >> 2)) * 32 + p.jb[s] * 8 + 2 * (lane & 3);
+    at[0] = acc[0][s][0];
+    at[1] = acc[0][s][1];
+    if (p.ib[s] != p.jb[s]) {
+      double* mirror = out + (p.jb[s] * 8 + (lane >> 2)) * 32 + p.ib[s] * 8 + 2 * (lane & 3);
+      mirror[0] = 0.0;
+      mirror[1] = 0.0;
+    }
+  }
+}
+
 // MODE 0: mean rows + Gram of A.  MODE 1: Gram of A*M.  MODE 2: absmax (and float32 copy) of A*M.
 // MODE 3: codes of A*M.
 template <int NP, int MODE>
@@ -154,7 +196,8 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
 #pragma unroll
       for (int j = 0; j < NP; ++j) T0[j * DSTR + tid] = static_cast<double>(row[j]);
       __syncthreads();
-      gram_accumulate<NP>(T0, acc, warp, lane);
+      if constexpr (NP == 32) gram_accumulate_sym4(T0, acc, warp, lane);
+      else gram_accumulate<NP>(T0, acc, warp, lane);
     } else {
       // the tile's rows of A*M, q[r][j] = sum_{i <= j} a[r][i] M[i][j], as float64 tensor-pipe products:
       // warp w takes the 8-row bands 4w .. 4w+3 of the tile; a band's fragment of A serves all column
@@ -186,7 +229,8 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
       }
       __syncthreads();
       if (MODE == 1) {
-        gram_accumulate<NP>(T, acc, warp, lane);
+        if constexpr (NP == 32) gram_accumulate_sym4(T, acc, warp, lane);
+        else gram_accumulate<NP>(T, acc, warp, lane);
       } else {
 #pragma unroll
         for (int j = 0; j < NP; ++j) {
@@ -226,7 +270,9 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
     __syncthreads();
   }
 
-  if (MODE <= 1) {
+  if (MODE <= 1 && NP == 32) {
+    if constexpr (NP == 32) sym4_store(a.partials + static_cast<size_t>(blockIdx.x) * NP * NP, acc, warp, lane);
+  } else if (MODE <= 1) {
     double* out = a.partials + static_cast<size_t>(blockIdx.x) * NP * NP;
 #pragma unroll
     for (int u = 0; u < IBW; ++u) {
