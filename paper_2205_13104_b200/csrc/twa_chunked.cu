@@ -22,7 +22,7 @@ namespace {
 constexpr int RT = 128;                 // rows per tile = threads per block
 constexpr int ASTR = RT + 1;            // padded strides: conflict-free column-strided reads
 constexpr int DSTR = RT + 4;            // stride of the float64 tile: the matrix-fragment loads below are conflict-free
-constexpr int MAX_BLOCKS = 512;
+constexpr int MAX_BLOCKS = 1024;
 constexpr int BUILD_MAX_N = 64;
 
 struct ChunkArgs {
@@ -361,7 +361,7 @@ __global__ void factor_kernel(const double* G, const double* prev, double* out, 
 }
 
 template <int NP, int MODE>
-int launch_chunk(twa_ctx* ctx, const ChunkArgs& a, int grid) {
+int launch_chunk(twa_ctx* ctx, const ChunkArgs& a, int grid, int* grid_used) {
   size_t smem = sizeof(float) * NP * ASTR + 8;
   if (MODE >= 1) smem += sizeof(double) * NP * NP;
   if (MODE <= 1) smem += sizeof(double) * NP * DSTR;      // the tile (mode 0) or A*M (mode 1) as float64
@@ -373,18 +373,25 @@ int launch_chunk(twa_ctx* ctx, const ChunkArgs& a, int grid) {
                              static_cast<int>(smem));
     if (rc) return rc;
   }
+  // as many blocks as are resident at once (three to five per SM, by shared memory): one wave, and the
+  // warps of the other blocks cover a block's load and barrier phases
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, RT, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
+  const int fit = per_sm * ctx->sm_count;
+  if (grid > fit) grid = fit;
   kern<<<grid, RT, smem, ctx->stream>>>(a);
   TWA_CUDA_OK(ctx, cudaGetLastError());
+  *grid_used = grid;
   return TWA_OK;
 }
 
 template <int MODE>
-int launch_chunk_np(twa_ctx* ctx, int np, const ChunkArgs& a, int grid) {
+int launch_chunk_np(twa_ctx* ctx, int np, const ChunkArgs& a, int grid, int* grid_used) {
   switch (np) {
-    case 16: return launch_chunk<16, MODE>(ctx, a, grid);
-    case 32: return launch_chunk<32, MODE>(ctx, a, grid);
-    case 48: return launch_chunk<48, MODE>(ctx, a, grid);
-    default: return launch_chunk<64, MODE>(ctx, a, grid);
+    case 16: return launch_chunk<16, MODE>(ctx, a, grid, grid_used);
+    case 32: return launch_chunk<32, MODE>(ctx, a, grid, grid_used);
+    case 48: return launch_chunk<48, MODE>(ctx, a, grid, grid_used);
+    default: return launch_chunk<64, MODE>(ctx, a, grid, grid_used);
   }
 }
 
@@ -456,16 +463,13 @@ int twa_build_feed(twa_ctx* ctx, int pass, const float* chunk, int64_t ldc, int6
     }
   }
   long long tiles = (a.rows_padded + RT - 1) / RT;
-  int grid = static_cast<int>(tiles < MAX_BLOCKS ? tiles : MAX_BLOCKS);
-  const int cap = ctx->sm_count * 3;
-  if (grid > cap) grid = cap;
-  if (grid > MAX_BLOCKS) grid = MAX_BLOCKS;
+  int grid = static_cast<int>(tiles < MAX_BLOCKS ? tiles : MAX_BLOCKS);     // cut to one resident wave at the launch
   int rc;
   switch (pass) {
-    case 0: rc = launch_chunk_np<0>(ctx, np, a, grid); break;
-    case 1: rc = launch_chunk_np<1>(ctx, np, a, grid); break;
-    case 2: rc = launch_chunk_np<2>(ctx, np, a, grid); break;
-    default: rc = launch_chunk_np<3>(ctx, np, a, grid); break;
+    case 0: rc = launch_chunk_np<0>(ctx, np, a, grid, &grid); break;
+    case 1: rc = launch_chunk_np<1>(ctx, np, a, grid, &grid); break;
+    case 2: rc = launch_chunk_np<2>(ctx, np, a, grid, &grid); break;
+    default: rc = launch_chunk_np<3>(ctx, np, a, grid, &grid); break;
   }
   if (rc) return rc;
   if (pass <= 1) {
