@@ -5,6 +5,7 @@
 #include <stdio.h>
 
 #include "twa_common.cuh"
+#include "twa_quant.cuh"
 
 namespace {
 
@@ -266,19 +267,6 @@ __global__ void scales_kernel(const unsigned* __restrict__ absmax, int n, float 
   }
 }
 
-// The quantiser's code of p without a division per element.  With r = RN(1 / s) the product q0 = p r
-// lies within 2^-16 of the IEEE quotient p / s wherever the clamp to +-qmax (<= 127) does not decide
-// the code anyway, so both round to the same integer unless q0 is that close to a half-integer; then,
-// and only then, *hard is set and the caller takes the IEEE division.  The distance of q0 to the
-// integer it rounds to is exact in float32.  Valid while r is finite (the caller checks s).
-__device__ __forceinline__ int encode_by_reciprocal(float p, float r, float qmax, bool* hard) {
-  const float q0 = fminf(fmaxf(p * r, -qmax), qmax);
-  const float y = q0 + 12582912.0f;                    // 1.5 * 2^23: rounds to an integer, half to even
-  const float t = q0 - (y - 12582912.0f);
-  *hard = fabsf(t) >= 0.5f - 0x1p-15f;
-  return __float_as_int(y) - 0x4B400000;
-}
-
 // Rows r .. r + 3 of a column; rows from D on read as zero.
 __device__ __forceinline__ float4 load_four(const float* __restrict__ col, long long r, long long D) {
   if (r + 3 < D) return __ldcs(reinterpret_cast<const float4*>(col + r));
@@ -328,8 +316,7 @@ __global__ void __launch_bounds__(BLOCK) encode_kernel(const float* __restrict__
   const int j = blockIdx.y;
   const float* col = P + j * ld;
   const float s = scales[j];
-  // the reciprocal path needs 1 / s finite and q0's error bound, which assumes a normal s
-  const float recip = s >= 0x1p-100f ? __frcp_rn(s) : 0.0f;
+  const float recip = encode_reciprocal(s);
   unsigned char* dst = out + j * out_stride;
   const long long lines = out_stride / 128;
   const int lane = threadIdx.x & 31;

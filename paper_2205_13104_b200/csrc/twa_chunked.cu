@@ -16,6 +16,7 @@
 #include <stdio.h>
 
 #include "twa_common.cuh"
+#include "twa_quant.cuh"
 
 namespace {
 
@@ -249,16 +250,40 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
           for (int task = tid; task < a.n * chunks_per_col; task += RT) {
             const int j = task / chunks_per_col, c = task - j * chunks_per_col;
             const float s = a.scales[j];
+            const float recip = encode_reciprocal(s);
             const float* src = Tq + j * ASTR + c * rows_per_chunk;
             uint32_t w[4] = {0, 0, 0, 0};
-            if (a.bits == 8) {
+            // by the reciprocal first; the whole group again by the IEEE division if an element came
+            // too close to a half-integer (or the scale has no usable reciprocal)
+            bool hard = recip == 0.0f;
+            if (!hard) {
+              if (a.bits == 8) {
 #pragma unroll
-              for (int k = 0; k < 16; ++k)
-                w[k >> 2] |= (static_cast<uint32_t>(twa_encode_one(src[k], s, qmax)) & 0xFFu) << (8 * (k & 3));
-            } else {
+                for (int k = 0; k < 16; ++k) {
+                  bool h;
+                  w[k >> 2] |= (static_cast<uint32_t>(encode_by_reciprocal(src[k], recip, qmax, &h)) & 0xFFu) << (8 * (k & 3));
+                  hard |= h;
+                }
+              } else {
 #pragma unroll
-              for (int k = 0; k < 32; ++k)
-                w[k >> 3] |= (static_cast<uint32_t>(twa_encode_one(src[k], s, qmax)) & 0xFu) << (4 * (k & 7));
+                for (int k = 0; k < 32; ++k) {
+                  bool h;
+                  w[k >> 3] |= (static_cast<uint32_t>(encode_by_reciprocal(src[k], recip, qmax, &h)) & 0xFu) << (4 * (k & 7));
+                  hard |= h;
+                }
+              }
+            }
+            if (hard) {
+              w[0] = w[1] = w[2] = w[3] = 0u;
+              if (a.bits == 8) {
+#pragma unroll
+                for (int k = 0; k < 16; ++k)
+                  w[k >> 2] |= (static_cast<uint32_t>(twa_encode_one(src[k], s, qmax)) & 0xFFu) << (8 * (k & 3));
+              } else {
+#pragma unroll
+                for (int k = 0; k < 32; ++k)
+                  w[k >> 3] |= (static_cast<uint32_t>(twa_encode_one(src[k], s, qmax)) & 0xFu) << (4 * (k & 7));
+              }
             }
             const long long qidx = (a.row0 + tile * RT) / rows_per_chunk + c;   // logical 16-byte chunk of the column
             const long long slot = (qidx & ~31LL) | twa_chunk_slot(static_cast<int>(qidx & 31), j);
