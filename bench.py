@@ -462,8 +462,10 @@ def build_chunked(ctx, wl, dev, bits_list, twa, inputs):
             if p < 3:
                 twa.twa_build_feed(ctx, p, buf, r0, rows)
             else:
-                for bits in bits_list:
-                    twa.twa_build_feed(ctx, p, buf, r0, rows, Pq=bases[bits])
+                # the chunk's rows of Q are formed once and encoded for every width (two at a time)
+                todo = [bases[bits] for bits in bits_list]
+                for i in range(0, len(todo), 2):
+                    twa.twa_build_feed_codes(ctx, buf, r0, rows, todo[i:i + 2])
             if r0 + rows == D:
                 if p == 2:
                     for bits in bits_list:

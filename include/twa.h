@@ -232,6 +232,13 @@ int twa_build_begin(twa_ctx* ctx, int64_t D, int n, float* wbar_out, void* bws, 
 int twa_build_feed(twa_ctx* ctx, int pass, const float* chunk, int64_t ldc, int64_t row0,
                    int64_t rows, const twa_basis* Pq, float* q32_out, int64_t ldq);
 int twa_build_end_pass(twa_ctx* ctx, int pass, int bits, twa_basis* Pq);
+/* Pass 3 for one or two widths at once: twa_build_feed(ctx, 3, ...) with a host array of `widths`
+ * (1 or 2) quantised bases, e.g. the 8-bit and the 4-bit one of the same build.  The chunk's rows
+ * of Q are formed once and encoded for every basis of the array; the codes are those of one
+ * twa_build_feed per basis, bit for bit.  A chunk fed through this call counts as fed for each
+ * of the bases. */
+int twa_build_feed_codes(twa_ctx* ctx, const float* chunk, int64_t ldc, int64_t row0, int64_t rows,
+                         const twa_basis* Pq, int widths, float* q32_out, int64_t ldq);
 
 /* Mean only: wbar_out[r] = (1/n) sum_i W[r, i]. */
 int twa_mean(twa_ctx* ctx, const float* W, int64_t D, int n, int64_t ldw, float* wbar_out);

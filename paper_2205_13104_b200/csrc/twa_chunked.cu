@@ -36,10 +36,14 @@ struct ChunkArgs {
   unsigned* absmax;         // mode 2
   float* q32;               // modes 2, 3, optional: q32[j * ldq + row inside the chunk]
   long long ldq;
-  unsigned char* codes;     // mode 3
-  long long code_stride;
-  const float* scales;
-  int bits;
+  // mode 3: the quantised bases that receive the codes of this chunk's rows (one or two widths)
+  struct CodeTarget {
+    unsigned char* codes;
+    long long stride, rows_padded;   // bytes between columns; rows of the chunk incl. the zero fill of the last segment
+    const float* scales;
+    int bits;
+  } target[2];
+  int targets;
 };
 
 // workspace layout for padded size NP
@@ -243,51 +247,56 @@ __global__ void __launch_bounds__(RT) chunk_kernel(const ChunkArgs a) {
           }
         }
         if (MODE == 3) {
-          // 16 output bytes per task: 16 rows (8-bit) or 32 rows (4-bit) of one column
-          const int rows_per_chunk = 128 / a.bits;
-          const int chunks_per_col = RT / rows_per_chunk;
-          const float qmax = a.bits == 8 ? 127.0f : 7.0f;
-          for (int task = tid; task < a.n * chunks_per_col; task += RT) {
-            const int j = task / chunks_per_col, c = task - j * chunks_per_col;
-            const float s = a.scales[j];
-            const float recip = encode_reciprocal(s);
-            const float* src = Tq + j * ASTR + c * rows_per_chunk;
-            uint32_t w[4] = {0, 0, 0, 0};
-            // by the reciprocal first; the whole group again by the IEEE division if an element came
-            // too close to a half-integer (or the scale has no usable reciprocal)
-            bool hard = recip == 0.0f;
-            if (!hard) {
-              if (a.bits == 8) {
+          // 16 output bytes per task: 16 rows (8-bit) or 32 rows (4-bit) of one column; the tile of Q just
+          // formed serves every target in turn
+          for (int tg = 0; tg < a.targets; ++tg) {
+            const ChunkArgs::CodeTarget& t = a.target[tg];
+            const int rows_per_chunk = 128 / t.bits;
+            const int chunks_per_col = RT / rows_per_chunk;
+            const float qmax = t.bits == 8 ? 127.0f : 7.0f;
+            for (int task = tid; task < a.n * chunks_per_col; task += RT) {
+              const int j = task / chunks_per_col, c = task - j * chunks_per_col;
+              if (tile * RT + c * rows_per_chunk >= t.rows_padded) continue;   // past this width's last segment
+              const float s = t.scales[j];
+              const float recip = encode_reciprocal(s);
+              const float* src = Tq + j * ASTR + c * rows_per_chunk;
+              uint32_t w[4] = {0, 0, 0, 0};
+              // by the reciprocal first; the whole group again by the IEEE division if an element came
+              // too close to a half-integer (or the scale has no usable reciprocal)
+              bool hard = recip == 0.0f;
+              if (!hard) {
+                if (t.bits == 8) {
 #pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                  bool h;
-                  w[k >> 2] |= (static_cast<uint32_t>(encode_by_reciprocal(src[k], recip, qmax, &h)) & 0xFFu) << (8 * (k & 3));
-                  hard |= h;
-                }
-              } else {
+                  for (int k = 0; k < 16; ++k) {
+                    bool h;
+                    w[k >> 2] |= (static_cast<uint32_t>(encode_by_reciprocal(src[k], recip, qmax, &h)) & 0xFFu) << (8 * (k & 3));
+                    hard |= h;
+                  }
+                } else {
 #pragma unroll
-                for (int k = 0; k < 32; ++k) {
-                  bool h;
-                  w[k >> 3] |= (static_cast<uint32_t>(encode_by_reciprocal(src[k], recip, qmax, &h)) & 0xFu) << (4 * (k & 7));
-                  hard |= h;
+                  for (int k = 0; k < 32; ++k) {
+                    bool h;
+                    w[k >> 3] |= (static_cast<uint32_t>(encode_by_reciprocal(src[k], recip, qmax, &h)) & 0xFu) << (4 * (k & 7));
+                    hard |= h;
+                  }
                 }
               }
-            }
-            if (hard) {
-              w[0] = w[1] = w[2] = w[3] = 0u;
-              if (a.bits == 8) {
+              if (hard) {
+                w[0] = w[1] = w[2] = w[3] = 0u;
+                if (t.bits == 8) {
 #pragma unroll
-                for (int k = 0; k < 16; ++k)
-                  w[k >> 2] |= (static_cast<uint32_t>(twa_encode_one(src[k], s, qmax)) & 0xFFu) << (8 * (k & 3));
-              } else {
+                  for (int k = 0; k < 16; ++k)
+                    w[k >> 2] |= (static_cast<uint32_t>(twa_encode_one(src[k], s, qmax)) & 0xFFu) << (8 * (k & 3));
+                } else {
 #pragma unroll
-                for (int k = 0; k < 32; ++k)
-                  w[k >> 3] |= (static_cast<uint32_t>(twa_encode_one(src[k], s, qmax)) & 0xFu) << (4 * (k & 7));
+                  for (int k = 0; k < 32; ++k)
+                    w[k >> 3] |= (static_cast<uint32_t>(twa_encode_one(src[k], s, qmax)) & 0xFu) << (4 * (k & 7));
+                }
               }
+              const long long qidx = (a.row0 + tile * RT) / rows_per_chunk + c;   // logical 16-byte chunk of the column
+              const long long slot = (qidx & ~31LL) | twa_chunk_slot(static_cast<int>(qidx & 31), j);
+              reinterpret_cast<uint4*>(t.codes + j * t.stride)[slot] = make_uint4(w[0], w[1], w[2], w[3]);
             }
-            const long long qidx = (a.row0 + tile * RT) / rows_per_chunk + c;   // logical 16-byte chunk of the column
-            const long long slot = (qidx & ~31LL) | twa_chunk_slot(static_cast<int>(qidx & 31), j);
-            reinterpret_cast<uint4*>(a.codes + j * a.code_stride)[slot] = make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
       }
@@ -444,8 +453,13 @@ int twa_build_begin(twa_ctx* ctx, int64_t D, int n, float* wbar_out, void* bws, 
   return TWA_OK;
 }
 
-int twa_build_feed(twa_ctx* ctx, int pass, const float* chunk, int64_t ldc, int64_t row0, int64_t rows,
-                   const twa_basis* Pq, float* q32_out, int64_t ldq) {
+}  // extern "C"
+
+namespace {
+
+// twa_build_feed; in pass 3 `Pq` is a host array of `widths` (1 or 2) quantised bases.
+int build_feed(twa_ctx* ctx, int pass, const float* chunk, int64_t ldc, int64_t row0, int64_t rows,
+               const twa_basis* Pq, int widths, float* q32_out, int64_t ldq) {
   if (!ctx || !ctx->build_ws || !chunk || pass < 0 || pass > 3) return TWA_ERR_INVALID_ARG;
   const long long D = ctx->build_D;
   const int n = ctx->build_n, np = padded_n(n);
@@ -470,22 +484,26 @@ int twa_build_feed(twa_ctx* ctx, int pass, const float* chunk, int64_t ldc, int6
   a.absmax = reinterpret_cast<unsigned*>(ws + l.absmax);
   a.q32 = (pass >= 2) ? q32_out : nullptr;
   a.ldq = ldq;
-  a.codes = nullptr;
-  a.code_stride = 0;
-  a.scales = nullptr;
-  a.bits = 8;
+  a.targets = 0;
   if (pass == 3) {
-    if (!Pq || !Pq->data || !Pq->scales || (Pq->bits != 8 && Pq->bits != 4) || Pq->D != D || Pq->n != n)
-      return TWA_ERR_INVALID_ARG;
-    a.codes = static_cast<unsigned char*>(Pq->data);
-    a.code_stride = Pq->col_stride;
-    a.scales = Pq->scales;
-    a.bits = Pq->bits;
-    if (row0 + rows == D) {
-      // the last chunk also fills the rest of the last 512-byte segment with the code 0
-      const long long seg_rows = 512LL * 8 / Pq->bits;
-      a.rows_padded = (D + seg_rows - 1) / seg_rows * seg_rows - row0;
+    if (!Pq || widths < 1 || widths > 2) return TWA_ERR_INVALID_ARG;
+    for (int k = 0; k < widths; ++k) {
+      const twa_basis& q = Pq[k];
+      if (!q.data || !q.scales || (q.bits != 8 && q.bits != 4) || q.D != D || q.n != n) return TWA_ERR_INVALID_ARG;
+      ChunkArgs::CodeTarget& t = a.target[k];
+      t.codes = static_cast<unsigned char*>(q.data);
+      t.stride = q.col_stride;
+      t.scales = q.scales;
+      t.bits = q.bits;
+      t.rows_padded = rows;
+      if (row0 + rows == D) {
+        // the last chunk also fills the rest of the width's last 512-byte segment with the code 0
+        const long long seg_rows = 512LL * 8 / q.bits;
+        t.rows_padded = (D + seg_rows - 1) / seg_rows * seg_rows - row0;
+      }
+      if (t.rows_padded > a.rows_padded) a.rows_padded = t.rows_padded;
     }
+    a.targets = widths;
   }
   long long tiles = (a.rows_padded + RT - 1) / RT;
   int grid = static_cast<int>(tiles < MAX_BLOCKS ? tiles : MAX_BLOCKS);     // cut to one resident wave at the launch
@@ -504,6 +522,20 @@ int twa_build_feed(twa_ctx* ctx, int pass, const float* chunk, int64_t ldc, int6
     TWA_CUDA_OK(ctx, cudaGetLastError());
   }
   return TWA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int twa_build_feed(twa_ctx* ctx, int pass, const float* chunk, int64_t ldc, int64_t row0, int64_t rows,
+                   const twa_basis* Pq, float* q32_out, int64_t ldq) {
+  return build_feed(ctx, pass, chunk, ldc, row0, rows, Pq, 1, q32_out, ldq);
+}
+
+int twa_build_feed_codes(twa_ctx* ctx, const float* chunk, int64_t ldc, int64_t row0, int64_t rows,
+                         const twa_basis* Pq, int widths, float* q32_out, int64_t ldq) {
+  return build_feed(ctx, 3, chunk, ldc, row0, rows, Pq, widths, q32_out, ldq);
 }
 
 int twa_build_end_pass(twa_ctx* ctx, int pass, int bits, twa_basis* Pq) {

@@ -45,7 +45,7 @@ EXPORTS = [
     "twa_last_error", "twa_set_tuning", "twa_selftest_wait", "twa_profile_enable", "twa_profile_read",
     "twa_basis_col_stride", "twa_basis_bytes",
     "twa_workspace_bytes", "twa_build_basis", "twa_build_quantized", "twa_build_workspace_bytes", "twa_build_begin",
-    "twa_build_feed", "twa_build_end_pass", "twa_mean", "twa_quantize_basis",
+    "twa_build_feed", "twa_build_feed_codes", "twa_build_end_pass", "twa_mean", "twa_quantize_basis",
     "twa_basis_export", "twa_basis_import", "twa_project", "twa_lift", "twa_step",
     "twa_step_host", "twa_step_adam", "twa_cosine_lr", "twa_weighted_average", "twa_layered_step_adam", "twa_project_batch", "twa_project_batch_group", "twa_layered_workspace_bytes", "twa_layered_rows", "twa_layered_basis_bytes",
     "twa_build_centered", "twa_quantize_affine", "twa_layered_export",
@@ -173,6 +173,7 @@ def load():
         "twa_build_begin": (i32, [vp, i64, i32, vp, vp, szt]),
         "twa_build_feed": (i32, [vp, i32, vp, i64, i64, i64, bp, vp, i64]),
         "twa_build_end_pass": (i32, [vp, i32, i32, bp]),
+        "twa_build_feed_codes": (i32, [vp, vp, i64, i64, i64, bp, i32, vp, i64]),
         "twa_mean": (i32, [vp, vp, i64, i32, i64, vp]),
         "twa_quantize_basis": (i32, [vp, bp, i32, bp, vp, szt]),
         "twa_basis_export": (i32, [vp, bp, vp, vp]),
@@ -387,6 +388,17 @@ def twa_build_feed(ctx, pass_index, chunk, row0, rows, Pq=None, q32_out=None):
                                int(rows), ctypes.byref(Pq.desc) if Pq is not None else None,
                                _ptr(q32_out), int(q32_out.stride(0)) if q32_out is not None else 0)
     _check(rc, "twa_build_feed", ctx)
+
+
+def twa_build_feed_codes(ctx, chunk, row0, rows, Pqs, q32_out=None):
+    """Pass 3 of the row-chunked build for one or two quantised bases at once (Pqs: list of Basis)."""
+    assert chunk.dtype == torch.float32 and chunk.stride(1) == 1
+    arr = (twa_basis * len(Pqs))()
+    for i, q in enumerate(Pqs):
+        ctypes.memmove(ctypes.byref(arr[i]), ctypes.byref(q.desc), ctypes.sizeof(twa_basis))
+    rc = load().twa_build_feed_codes(ctx, _ptr(chunk), int(chunk.stride(0)), int(row0), int(rows), arr, len(Pqs),
+                                     _ptr(q32_out), int(q32_out.stride(0)) if q32_out is not None else 0)
+    _check(rc, "twa_build_feed_codes", ctx)
 
 
 def twa_build_end_pass(ctx, pass_index, bits=0, Pq=None):

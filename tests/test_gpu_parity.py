@@ -605,6 +605,46 @@ def test_chunked_build_codes_are_the_quantiser_of_its_float32_rows(env, bits):
     status_ok(ctx)
 
 
+@pytest.mark.parametrize("D,n,chunk_rows", [(150001, 12, 32768), (100, 3, 1024), (600, 2, 1024), (70001, 33, 8192),
+                                            (5121, 64, 2048)])
+def test_chunked_build_two_widths_in_one_last_pass(env, D, n, chunk_rows):
+    """twa_build_feed_codes with the 8-bit and the 4-bit basis together: the bytes of one
+    twa_build_feed per basis, padding included -- also where the last segment of the 4-bit columns
+    ends later than that of the 8-bit ones -- and the oracle's quantiser on the float32 rows."""
+    ctx, ws = env
+    W = inputs.trajectory_candidates(D, n, 0.005, 0.001, 36, DEV, ld=inputs.padded_ld(D, 4))
+    bws = torch.empty(twa.twa_build_workspace_bytes(n), dtype=torch.uint8, device=DEV)
+    wbar = torch.empty(D, device=DEV)
+    q32 = torch.zeros((n, inputs.padded_ld(D, 4)), device=DEV)
+    sep = {bits: twa.new_quantised_basis(D, n, bits, DEV) for bits in (8, 4)}
+    both = {bits: twa.new_quantised_basis(D, n, bits, DEV) for bits in (8, 4)}
+    for q in list(sep.values()) + list(both.values()):
+        q.data.fill_(0xA5)                                    # whatever was there must be overwritten
+    starts = list(range(0, D, chunk_rows))
+    twa.twa_build_begin(ctx, D, n, wbar, bws)
+    for p in range(3):
+        for r0 in starts:
+            twa.twa_build_feed(ctx, p, W[:, r0:], r0, min(chunk_rows, D - r0), q32_out=q32[:, r0:] if p == 2 else None)
+        if p < 2:
+            twa.twa_build_end_pass(ctx, p, 0, None)
+    for bits in (8, 4):
+        twa.twa_build_end_pass(ctx, 2, bits, sep[bits])
+        twa.twa_build_end_pass(ctx, 2, bits, both[bits])
+    for r0 in starts:
+        rows = min(chunk_rows, D - r0)
+        for bits in (8, 4):
+            twa.twa_build_feed(ctx, 3, W[:, r0:], r0, rows, Pq=sep[bits])
+        twa.twa_build_feed_codes(ctx, W[:, r0:], r0, rows, [both[8], both[4]])
+    twa.twa_build_end_pass(ctx, 3, 0, None)
+    status_ok(ctx)
+    for bits in (8, 4):
+        assert torch.equal(sep[bits].data, both[bits].data) and torch.equal(sep[bits].scales, both[bits].scales)
+        codes_g, s_g = twa.twa_basis_export(ctx, both[bits])
+        codes_o, s_o = orc.quantize(np.asfortranarray(host_cols(q32, D)), bits)
+        np.testing.assert_array_equal(s_g.cpu().numpy(), s_o)
+        np.testing.assert_array_equal(codes_g.cpu().numpy(), orc.pack_codes(codes_o, bits))
+
+
 def test_chunked_build_reports_rank_deficiency(env):
     ctx, ws = env
     D, n = 20000, 5

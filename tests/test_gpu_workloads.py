@@ -413,7 +413,7 @@ def test_workload_resident_build_sampled(env, name, bits_list):
 # ------------------------------------------------------------------ 1.3 B-sized: chunked build, sampled
 def test_workload_decoder_chunked_build_sampled(env):
     """The 1.3 B-sized workload: one row-chunked build gives the int8 and the int4 basis (the scales
-    of both widths come from the absmax of pass 2, the codes of both from the chunks of pass 3);
+    of both widths come from the absmax of pass 2, the codes of both from one feed of pass 3 per chunk);
     then the workload's 50 steps on both, checked as run_sequence describes."""
     ctx, ws = env
     wl = inputs.WORKLOADS["decoder1p3b"]
@@ -435,8 +435,7 @@ def test_workload_decoder_chunked_build_sampled(env):
             if p < 3:
                 twa.twa_build_feed(ctx, p, buf, r0, rows)
             else:
-                twa.twa_build_feed(ctx, p, buf, r0, rows, Pq=bases[8], q32_out=qbuf if keep else None)
-                twa.twa_build_feed(ctx, p, buf, r0, rows, Pq=bases[4])
+                twa.twa_build_feed_codes(ctx, buf, r0, rows, [bases[8], bases[4]], q32_out=qbuf if keep else None)
             if keep:
                 sampled[r0] = (qbuf[:, :rows].cpu().numpy().T.copy(), buf[:, :rows].cpu().numpy().T.copy())
         if p == 2:
