@@ -22,7 +22,13 @@
  *    data + j * col_stride (bytes).  Vectors are contiguous.
  *  - Alignment: data pointers of matrices, g, base, w and workspaces must be
  *    16-byte aligned; col_stride must be a multiple of 16 bytes.
- *  - Limits: 1 <= n <= TWA_MAX_N, 1 <= D < 2^31.
+ *  - Limits: 1 <= n <= TWA_MAX_N, 1 <= D < 2^31.  The per-column stepping calls (twa_project,
+ *    twa_lift, twa_step, twa_step_adam, twa_step_host, twa_weighted_average), the row-chunked
+ *    build (twa_build_begin / feed / end_pass) and twa_basis_export / twa_basis_import take
+ *    D <= TWA_MAX_ROWS = 2^34: from 2^31 rows on they walk the basis in slabs of 2^30 rows, one
+ *    launch per slab and kernel, the projection being the float64 sum of the slabs' projections
+ *    in slab order (the stepping calls stay capturable).  A view of fewer than 2^31 rows of such
+ *    a basis (twa_basis with data moved to a row on a 512-byte segment) serves every other call.
  *  - Calls enqueue work on the context's stream and return without waiting
  *    for it.  Return value 0 = enqueued; a negative TWA_ERR_* = rejected on
  *    the host, nothing enqueued.  Errors found on the device (non-finite
@@ -55,6 +61,7 @@ extern "C" {
 #endif
 
 #define TWA_MAX_N 128
+#define TWA_MAX_ROWS (1LL << 34) /* the stepping calls, the row-chunked build, export and import */
 
 enum {
   TWA_OK = 0,

@@ -36,18 +36,84 @@ __global__ void wait_selftest_kernel(int* status, unsigned long long limit_ns) {
 }  // namespace
 
 namespace {
-// twa_step_host: the coefficients' gradient is the sum of the chunks' projections (float64, chunk
-// order), then the update of Algorithm 1.  One block of TWA_MAX_N threads.
-__global__ void chunk_combine_kernel(const float* __restrict__ chunk_c, int chunks, int n, float* alpha, float lr,
-                                     float lambda, int* status) {
+// twa_step_host and the row slabs of a basis of 2^31 rows or more: the coefficients' gradient is the
+// sum of the chunks' projections (float64, chunk order); written to c_out when that is non-null,
+// and followed by the update of Algorithm 1 (or the Adam step) when alpha is.  One block of
+// TWA_MAX_N threads.
+__global__ void chunk_combine_kernel(const float* __restrict__ chunk_c, int chunks, int n, float* c_out, float* alpha,
+                                     float lr, float lambda, twa_adam_args adam, int* status) {
   const int j = threadIdx.x;
   double c = 0.0;
   if (j < n)
     for (int k = 0; k < chunks; ++k) c += static_cast<double>(chunk_c[static_cast<size_t>(k) * TWA_MAX_N + j]);
   if (j < n && !isfinite(c)) twa_set_status(status, TWA_ERR_NONFINITE, j);
+  if (j < n && c_out) c_out[j] = static_cast<float>(c);
   // alpha stays as it was when the projection is unusable (see twa_step)
   const int unusable = __syncthreads_or(!isfinite(c)) | (__ldcg(status) == TWA_ERR_TIMEOUT);
-  if (j < n && !unusable) alpha[j] = twa_coefficient_update(alpha[j], c, lr, lambda, twa_adam_args{}, j);
+  if (j < n && alpha && !unusable) alpha[j] = twa_coefficient_update(alpha[j], c, lr, lambda, adam, j);
+}
+
+// A basis of 2^31 rows or more is walked in slabs of 2^30 rows: the kernels index rows with 32-bit
+// integers, the projection is a sum over row ranges and the lift is independent per row.
+constexpr long long TWA_SLAB_ROWS = 1LL << 30;
+static_assert(TWA_MAX_ROWS == TWA_SLAB_ROWS * TWA_HOST_CHUNKS, "one slot of per-slab coefficients in ws per slab");
+
+int slab_count(long long D) {
+  return D < (1LL << 31) ? 1 : static_cast<int>((D + TWA_SLAB_ROWS - 1) / TWA_SLAB_ROWS);
+}
+
+// Rows [k * TWA_SLAB_ROWS, ...) of P as a basis of its own; 2^30 rows are whole 512-byte segments
+// at every storage width.
+twa_basis slab_view(const twa_basis* P, int k, long long* r0) {
+  *r0 = static_cast<long long>(k) * TWA_SLAB_ROWS;
+  twa_basis v = *P;
+  v.data = static_cast<char*>(P->data) + (*r0 * P->bits) / 8;
+  v.D = (*r0 + TWA_SLAB_ROWS < P->D) ? TWA_SLAB_ROWS : P->D - *r0;
+  return v;
+}
+
+// twa_check_basis with the row limit of the slab-walking calls instead of the kernels' own.
+int check_basis_slabbed(const twa_basis* P) {
+  if (!P) return TWA_ERR_INVALID_ARG;
+  if (P->D < (1LL << 31)) return twa_check_basis(P);
+  if (P->D > TWA_MAX_ROWS) return TWA_ERR_INVALID_ARG;
+  twa_basis head = *P;
+  head.D = TWA_SLAB_ROWS;
+  int rc = twa_check_basis(&head);
+  if (rc) return rc;
+  return P->col_stride < (P->D * P->bits + 7) / 8 ? TWA_ERR_INVALID_ARG : TWA_OK;
+}
+
+// Projection of every slab into its slot of ws, then the combine (and the optimiser step, if any).
+int project_slabs(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype, const twa_project_epilogue& epi,
+                  void* ws) {
+  const int slabs = slab_count(P->D);
+  const size_t gsz = g_dtype == TWA_BF16 ? 2 : 4;
+  float* slab_c = reinterpret_cast<float*>(static_cast<char*>(ws) + TWA_WS_CHUNK_COEF);
+  for (int k = 0; k < slabs; ++k) {
+    long long r0;
+    const twa_basis v = slab_view(P, k, &r0);
+    twa_project_epilogue part = {slab_c + static_cast<size_t>(k) * TWA_MAX_N, nullptr, 0.0f, 0.0f, -1};
+    int rc = twa_launch_project(ctx, &v, static_cast<const char*>(g) + r0 * gsz, g_dtype, part, ws);
+    if (rc) return rc;
+  }
+  chunk_combine_kernel<<<1, TWA_MAX_N, 0, ctx->stream>>>(slab_c, slabs, P->n, epi.c_out, epi.alpha, epi.lr, epi.lambda,
+                                                         epi.adam, ctx->d_status);
+  TWA_CUDA_OK(ctx, cudaGetLastError());
+  return TWA_OK;
+}
+
+// Lift of every slab, last slab first when the projection has just run (its rows are the likeliest in L2).
+int lift_slabs(twa_ctx* ctx, const twa_basis* P, const float* alpha, const float* base, float* out, bool reverse) {
+  const int slabs = slab_count(P->D);
+  for (int i = 0; i < slabs; ++i) {
+    const int k = reverse ? slabs - 1 - i : i;
+    long long r0;
+    const twa_basis v = slab_view(P, k, &r0);
+    int rc = twa_launch_lift(ctx, &v, alpha, 1.0f, base ? base + r0 : nullptr, out + r0, reverse);
+    if (rc) return rc;
+  }
+  return TWA_OK;
 }
 }  // namespace
 
@@ -210,25 +276,27 @@ int twa_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dty
                 void* ws, size_t ws_bytes) {
   if (!ctx || !g || !c_out) return TWA_ERR_INVALID_ARG;
   if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
-  int rc = twa_check_basis(P);
+  int rc = check_basis_slabbed(P);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes);
   if (rc) return rc;
   if (misaligned16(g)) return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
   twa_project_epilogue epi = {c_out, nullptr, 0.0f, 0.0f, -1};
+  if (slab_count(P->D) > 1) return project_slabs(ctx, P, g, g_dtype, epi, ws);
   return twa_launch_project(ctx, P, g, g_dtype, epi, ws);
 }
 
 int twa_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, const float* base, float* w_out,
              void* ws, size_t ws_bytes) {
   if (!ctx || !alpha || !w_out) return TWA_ERR_INVALID_ARG;
-  int rc = twa_check_basis(P);
+  int rc = check_basis_slabbed(P);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes);
   if (rc) return rc;
   if (misaligned16(w_out) || (base && misaligned16(base))) return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+  if (slab_count(P->D) > 1) return lift_slabs(ctx, P, alpha, base, w_out, false);
   return twa_launch_lift(ctx, P, alpha, 1.0f, base, w_out, false);
 }
 
@@ -237,22 +305,23 @@ static int step_impl(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype 
                      size_t ws_bytes) {
   if (!ctx || !g || !alpha || !wbar || !w) return TWA_ERR_INVALID_ARG;
   if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
-  int rc = twa_check_basis(P);
+  int rc = check_basis_slabbed(P);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes);
   if (rc) return rc;
   if (misaligned16(g) || misaligned16(w) || misaligned16(wbar)) return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
   twa_project_epilogue epi = {c_out, alpha, lr, lambda, -1, adam};
+  const bool slabbed = slab_count(P->D) > 1;
   cudaEvent_t* ev = nullptr;
   if (ctx->prof_events && ctx->prof_count < ctx->prof_cap) ev = ctx->prof_events + 3 * ctx->prof_count;
   if (ev) TWA_CUDA_OK(ctx, cudaEventRecord(ev[0], ctx->stream));
-  rc = twa_launch_project(ctx, P, g, g_dtype, epi, ws);
+  rc = slabbed ? project_slabs(ctx, P, g, g_dtype, epi, ws) : twa_launch_project(ctx, P, g, g_dtype, epi, ws);
   if (rc) return rc;
   if (ev) TWA_CUDA_OK(ctx, cudaEventRecord(ev[1], ctx->stream));
   // The lift walks the tiles backwards: the part of P~ the projection read last is the part
   // most likely still in L2.
-  rc = twa_launch_lift(ctx, P, alpha, 1.0f, wbar, w, true);
+  rc = slabbed ? lift_slabs(ctx, P, alpha, wbar, w, true) : twa_launch_lift(ctx, P, alpha, 1.0f, wbar, w, true);
   if (rc) return rc;
   if (ev) {
     TWA_CUDA_OK(ctx, cudaEventRecord(ev[2], ctx->stream));
@@ -350,7 +419,7 @@ int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host, twa_dtyp
     return TWA_OK;
   }
   if (!alpha || !wbar || !w) return TWA_ERR_INVALID_ARG;
-  int rc = twa_check_basis(P);
+  int rc = check_basis_slabbed(P);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes);
   if (rc) return rc;
@@ -397,7 +466,8 @@ int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host, twa_dtyp
     rc = twa_launch_project(ctx, &v, gs + r0 * gsz, g_dtype, epi, ws);
     if (rc) return rc;
   }
-  chunk_combine_kernel<<<1, TWA_MAX_N, 0, ctx->stream>>>(chunk_c, chunks, P->n, alpha, lr, lambda, ctx->d_status);
+  chunk_combine_kernel<<<1, TWA_MAX_N, 0, ctx->stream>>>(chunk_c, chunks, P->n, nullptr, alpha, lr, lambda,
+                                                         twa_adam_args{}, ctx->d_status);
   TWA_CUDA_OK(ctx, cudaGetLastError());
   // lift chunk by chunk; every chunk of w leaves for the host while the next one is computed
   for (int k = 0; k < chunks; ++k) {

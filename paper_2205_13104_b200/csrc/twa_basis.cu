@@ -701,9 +701,13 @@ int twa_quantize_basis(twa_ctx* ctx, const twa_basis* P32, int bits, twa_basis* 
 }
 
 int twa_basis_export(twa_ctx* ctx, const twa_basis* Pq, void* codes_out, float* scales_out) {
-  if (!ctx || !codes_out || !scales_out) return TWA_ERR_INVALID_ARG;
-  int rc = twa_check_basis(Pq);
+  if (!ctx || !codes_out || !scales_out || !Pq) return TWA_ERR_INVALID_ARG;
+  // the conversion kernels index bytes with 64-bit integers: up to TWA_MAX_ROWS rows
+  twa_basis head = *Pq;
+  if (Pq->D >= (1LL << 31)) head.D = (1LL << 31) - 1;
+  int rc = twa_check_basis(&head);
   if (rc) return rc;
+  if (Pq->D > TWA_MAX_ROWS || Pq->col_stride < (Pq->D * Pq->bits + 7) / 8) return TWA_ERR_INVALID_ARG;
   if (Pq->bits == 32) return TWA_ERR_UNSUPPORTED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
   const long long row_bytes = (Pq->D * Pq->bits + 7) / 8;
@@ -722,7 +726,7 @@ int twa_basis_import(twa_ctx* ctx, const void* codes, const float* scales, int64
                      twa_basis* Pq) {
   if (!ctx || !codes || !scales || !Pq || !Pq->data || !Pq->scales) return TWA_ERR_INVALID_ARG;
   if (bits != 8 && bits != 4) return TWA_ERR_UNSUPPORTED;
-  if (D < 1 || D >= (1LL << 31) || n < 1) return TWA_ERR_INVALID_ARG;
+  if (D < 1 || D > TWA_MAX_ROWS || n < 1) return TWA_ERR_INVALID_ARG;
   if (n > TWA_MAX_N) return TWA_ERR_UNSUPPORTED;
   if (reinterpret_cast<uintptr_t>(Pq->data) & 15) return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));

@@ -439,7 +439,7 @@ size_t twa_build_workspace_bytes(int n) {
 }
 
 int twa_build_begin(twa_ctx* ctx, int64_t D, int n, float* wbar_out, void* bws, size_t bws_bytes) {
-  if (!ctx || !wbar_out || D < 1 || D >= (1LL << 31) || n < 1) return TWA_ERR_INVALID_ARG;
+  if (!ctx || !wbar_out || D < 1 || D > TWA_MAX_ROWS || n < 1) return TWA_ERR_INVALID_ARG;
   if (n > BUILD_MAX_N) return TWA_ERR_UNSUPPORTED;
   const BuildLayout l = layout_for(padded_n(n));
   if (!bws || bws_bytes < l.total) return TWA_ERR_WORKSPACE;

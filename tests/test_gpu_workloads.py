@@ -133,7 +133,8 @@ def check_lift_rows(ctx, Pq, bits, w, alpha64, wbar, row_ranges, offset=None):
 
 def sampled_row_ranges(D, bits, n):
     """Row ranges of the lift to compare: the first tiles, the tiles where the second and a middle
-    sweep of the persistent grid begin, a range across row 2^30 (where it exists), the middle, the
+    sweep of the persistent grid begin, a range across every multiple of 2^30 rows (the slab boundaries of
+    a basis of 2^31 rows or more), the middle, the
     last whole tile and the ragged end.  All start on a 512-byte segment of the codes."""
     seg = 512 * 8 // bits
     tile = seg * (2 if n <= 64 else 1)
@@ -142,8 +143,9 @@ def sampled_row_ranges(D, bits, n):
     for t in (148, 148 * 37 + 5):
         if (t + 2) * tile < D:
             out.append((t * tile - seg, 2 * tile))
-    if D > (1 << 30) + 2 * tile:
-        out.append(((1 << 30) - tile, 2 * tile))
+    for k in range(1, (D >> 30) + 1):                   # 2^30 and, from 2^31 rows on, every slab boundary
+        if D > (k << 30) + 2 * tile:
+            out.append(((k << 30) - tile, 2 * tile))
     return sorted(set(out))
 
 
@@ -478,6 +480,79 @@ def test_workload_decoder_chunked_build_sampled(env):
     del codes, col
     torch.cuda.empty_cache()
     run_sequence(ctx, ws, wl, [bases[8], bases[4]], wbar, wl.steps, [], step1_blocks=[0, 24])
+
+
+def test_basis_of_more_than_2_31_rows(env):
+    """A basis of 2^31 + 3 * 2^22 + 70,001 rows (three slabs of the stepping calls; odd, so the 4-bit
+    column ends on a half byte) and four columns: row-chunked build of the int8 and the int4 basis,
+    mean, codes and scales of sampled chunks (the first, the one that ends at row 2^31, the last)
+    against the oracle, then two fused steps on both widths checked as run_sequence describes: all
+    coefficients after step 1 and step 2, rows of w at the start, across 2^30, across 2^31, in the
+    last slab and at the ragged end."""
+    ctx, ws = env
+    D, n = (1 << 31) + 3 * (1 << 22) + 70_001, 4
+    wl = inputs.Workload("rows_2g", D, n, 0.002, 0.0005, 1e-4, "bf16", (8, 4), 2, seed=11, chunked_build=True)
+    CH = inputs.CHUNK_ROWS
+    starts = list(range(0, D, CH))
+    sampled = {starts[0]: None, (1 << 31) - CH: None, starts[-1]: None}
+    bws = torch.empty(twa.twa_build_workspace_bytes(n), dtype=torch.uint8, device=DEV)
+    wbar = torch.empty(D, device=DEV)
+    bases = {bits: twa.new_quantised_basis(D, n, bits, DEV) for bits in (8, 4)}
+    buf = torch.empty((n, CH), device=DEV)
+    qbuf = torch.empty((n, CH), device=DEV)
+    twa.twa_build_begin(ctx, D, n, wbar, bws)
+    for p in range(4):
+        for r0 in starts:
+            rows = min(CH, D - r0)
+            inputs.trajectory_rows(D, n, wl.step, wl.drift, wl.seed, DEV, row0=r0, rows=rows, out=buf[:, :rows])
+            keep = p == 3 and r0 in sampled
+            if p < 3:
+                twa.twa_build_feed(ctx, p, buf, r0, rows)
+            else:
+                twa.twa_build_feed_codes(ctx, buf, r0, rows, [bases[8], bases[4]], q32_out=qbuf if keep else None)
+            if keep:
+                sampled[r0] = (qbuf[:, :rows].cpu().numpy().T.copy(), buf[:, :rows].cpu().numpy().T.copy())
+        if p == 2:
+            twa.twa_build_end_pass(ctx, p, 8, bases[8])
+            twa.twa_build_end_pass(ctx, p, 4, bases[4])
+        else:
+            twa.twa_build_end_pass(ctx, p, 0, None)
+    status_ok(ctx)
+    del buf, qbuf, bws
+    torch.cuda.empty_cache()
+    M0 = None
+    for r0, (q32, a_rows) in sampled.items():
+        rows = q32.shape[0]
+        np.testing.assert_array_equal(wbar[r0:r0 + rows].cpu().numpy(), orc.mean(a_rows).astype(np.float32))
+        for bits, Pq in bases.items():
+            scales = Pq.scales.cpu().numpy()
+            codes, _ = twa.twa_basis_export(ctx, twa.basis_view(Pq, row0=r0, rows=rows))
+            co = orc.encode(np.asfortranarray(q32), scales, bits)
+            np.testing.assert_array_equal(codes.cpu().numpy(), orc.pack_codes(co, bits))
+            assert np.all(np.abs(q32).max(axis=0) <= scales * orc.QMAX[bits] * (1 + 1e-6))
+            del codes, co
+        # rows of Q are rows of A times one upper-triangular matrix with a positive diagonal: the same for every chunk
+        if M0 is None:
+            M0, *_ = np.linalg.lstsq(a_rows[:65536].astype(np.float64), q32[:65536].astype(np.float64), rcond=None)
+            assert np.max(np.abs(np.tril(M0, -1))) <= 1e-3 * np.max(np.abs(M0))
+            assert np.all(np.diag(M0) > 0)
+        else:
+            resid = a_rows[:65536].astype(np.float64) @ M0 - q32[:65536]
+            assert np.linalg.norm(resid) <= 1e-5 * np.linalg.norm(q32[:65536])
+    sampled.clear()
+    # unit columns: the dequantised int8 column has norm 1 up to the quantisation error (whole-basis export)
+    codes, s = twa.twa_basis_export(ctx, bases[8])
+    col = codes[n - 1].cpu().numpy().view(np.int8)[:D]
+    sq = sum(float(np.dot(col[a:a + (1 << 26)].astype(np.float64), col[a:a + (1 << 26)].astype(np.float64)))
+             for a in range(0, D, 1 << 26))
+    assert abs(np.sqrt(sq) * float(s[n - 1]) - 1.0) <= 2e-3
+    del codes, col
+    torch.cuda.empty_cache()
+    run_sequence(ctx, ws, wl, [bases[8], bases[4]], wbar, wl.steps, [])
+    # the calls whose kernels index rows with 32-bit integers refuse the whole basis and take a view of it
+    c = torch.empty(n, device=DEV)
+    with pytest.raises(twa.TwaError):
+        twa.twa_project_noalloc(0, None, bases[8], torch.zeros(D, dtype=torch.bfloat16, device=DEV), c)
 
 
 # ------------------------------------------------------------------ the layer-wise construction, full size
