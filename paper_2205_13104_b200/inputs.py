@@ -34,6 +34,7 @@ CHUNK_ROWS = 1 << 22
 
 _STREAM_TRAJECTORY = 1
 _STREAM_SHARED_W0 = 2
+_STREAM_INTEGERS = 9
 _STREAM_GRADIENT = 3
 
 
@@ -125,6 +126,18 @@ def multi_trajectory_candidates(D, groups, per_group, step, drift, seed, device,
                 prev = cur
             del xi
     return W
+
+
+def small_integers(out, low, high, seed):
+    """Fills the rows of `out` (k, D) with integers drawn uniformly from [low, high]: sums of products of
+    such values are exact in float32 whatever the order of the additions, so a result on them is
+    one number, not a number within a bound."""
+    k, D = out.shape
+    for ci, r, nr in _chunks(D):
+        gen = _generator(out.device, seed, _STREAM_INTEGERS, ci)
+        z = torch.randint(low, high + 1, (k, nr), generator=gen, device=out.device)
+        out[:, r: r + nr] = z.to(out.dtype)
+    return out
 
 
 def gradient(D, std, seed, step_index, dtype, device, out=None):

@@ -243,6 +243,7 @@ def run_sequence(ctx, ws, wl, bases, wbar, T, sample_cols, step1_blocks=None):
         assert seen.sum() >= min(n, 8)
         assert_coefficients(st["c0"][seen], c0_ref[seen], norm_low[seen], g0_norm)
         a0_ref = orc.sgd_update(np.zeros(n), c0_ref, LR, 0.0)
+        st["c0_ref"] = c0_ref
         assert_coefficients(st["a0"][seen], a0_ref[seen], LR * norm_low[seen], g0_norm)
         # the lift of step 1 is compared with the oracle's lift of the library's own alpha where the oracle
         # did not project every column (alpha itself is checked on the sampled columns above)
@@ -548,11 +549,83 @@ def test_basis_of_more_than_2_31_rows(env):
     assert abs(np.sqrt(sq) * float(s[n - 1]) - 1.0) <= 2e-3
     del codes, col
     torch.cuda.empty_cache()
-    run_sequence(ctx, ws, wl, [bases[8], bases[4]], wbar, wl.steps, [])
+    state = run_sequence(ctx, ws, wl, [bases[8], bases[4]], wbar, wl.steps, [])
+    # the Adam step over the slabs: first step from zero moments on the first gradient, against the oracle's
+    # Adam update of the oracle's own coefficients' gradient
+    g = wl.gradient(0, DEV)
+    for st in state:
+        alpha, m, v = (torch.zeros(n, device=DEV) for _ in range(3))
+        w = st["w"]
+        twa.twa_step_adam(ctx, st["basis"], g, 1e-2, 1, alpha, m, v, wbar, w, ws, weight_decay=0.01)
+        a_ref, m_ref, v_ref = orc.adam_update(np.zeros(n), np.zeros(n), np.zeros(n), st["c0_ref"], 1e-2, 1,
+                                              weight_decay=0.01)
+        assert rel(m.cpu().numpy(), m_ref) <= TOL and rel(v.cpu().numpy(), v_ref) <= 2 * TOL
+        assert rel(alpha.cpu().numpy(), a_ref) <= TOL
+        check_lift_rows(ctx, st["basis"], st["basis"].bits, w, a_ref, wbar, st["ranges"][-3:])
+    # the step from host memory (sixteen row chunks, not the three slabs): same alpha to rounding, same rows of w
+    st = state[0]
+    g_host = torch.empty(D, dtype=torch.bfloat16).pin_memory()
+    g_host.copy_(g)
+    w_host = torch.empty(D, dtype=torch.float32).pin_memory()
+    g_stage = torch.empty(D, dtype=torch.bfloat16, device=DEV)
+    alpha = torch.zeros(n, device=DEV)
+    twa.twa_step_host(ctx, st["basis"], g_host, LR, 0.0, alpha, wbar, st["w"], w_host, g_stage, ws)
+    status_ok(ctx)
+    a0_ref = orc.sgd_update(np.zeros(n), st["c0_ref"], LR, 0.0)
+    assert rel(alpha.cpu().numpy(), a0_ref) <= TOL
+    check_lift_rows(ctx, st["basis"], 8, st["w"], a0_ref, wbar, st["ranges"])
+    for r0, rows in st["ranges"]:
+        np.testing.assert_array_equal(w_host[r0:r0 + rows].numpy(), st["w"][r0:r0 + rows].cpu().numpy())
+    del g_host, w_host, g_stage
     # the calls whose kernels index rows with 32-bit integers refuse the whole basis and take a view of it
     c = torch.empty(n, device=DEV)
     with pytest.raises(twa.TwaError):
         twa.twa_project_noalloc(0, None, bases[8], torch.zeros(D, dtype=torch.bfloat16, device=DEV), c)
+
+
+def test_float32_candidates_of_more_than_2_31_rows(env):
+    """Two float32 candidates of 2^31 + 70,001 rows: the fixed-weight average (the float32 lift over the
+    slabs) on rows at the start, across 2^30 and 2^31 and at the end against the oracle, and the float32
+    projection on all rows against the oracle's, streamed through the host, on integer-valued inputs
+    that make the result exact."""
+    ctx, ws = env
+    D, n = (1 << 31) + 70_001, 2
+    wl = inputs.Workload("rows_2g_f32", D, n, 0.002, 0.0005, 1e-3, "f32", (32,), 1, seed=12)
+    W = torch.zeros((n, D + 3), device=DEV)                 # columns start on 16 bytes
+    CH = inputs.CHUNK_ROWS
+    for r0 in range(0, D, CH):
+        rows = min(CH, D - r0)
+        inputs.trajectory_rows(D, n, wl.step, wl.drift, wl.seed, DEV, row0=r0, rows=rows, out=W[:, r0:r0 + rows])
+    weights = torch.tensor([0.25, 0.75], device=DEV)
+    w = torch.empty(D, device=DEV)
+    twa.twa_weighted_average(ctx, W, D, weights, w, ws)
+    status_ok(ctx)
+    span = 1 << 16
+    for r0 in (0, (1 << 30) - span // 2, (1 << 31) - span // 2, D - span):
+        rows_h = W[:, r0:r0 + span].cpu().numpy().T
+        ref = orc.weighted_average(rows_h, [0.25, 0.75])
+        got = w[r0:r0 + span].cpu().numpy()
+        assert rel(got, ref) <= TOL
+        assert np.max(np.abs(got - ref.astype(np.float32))) <= 4 * np.spacing(np.float32(np.abs(ref).max()))
+    # the float32 projection on small integers (candidates in [-2, 2], gradient in [-1, 1]): every partial
+    # sum is an integer below 2^24, so the float32 sums are exact in any order and the oracle's float64
+    # result must be met to the last bit, float32 and bfloat16 gradient alike
+    inputs.small_integers(W[:, :D], -2, 2, wl.seed)
+    g = inputs.small_integers(torch.empty((1, D), device=DEV), -1, 1, wl.seed + 1)[0]
+    c = torch.empty(n, device=DEV)
+    twa.twa_project(ctx, twa.basis_from_tensor(W, D), g, c, ws)
+    status_ok(ctx)
+    c16 = torch.empty(n, device=DEV)
+    twa.twa_project(ctx, twa.basis_from_tensor(W, D), g.to(torch.bfloat16), c16, ws)
+    status_ok(ctx)
+    g_h = to_host(g.view(torch.uint8)).view(np.float32).copy()
+    c_ref = np.zeros(n)
+    for j in range(n):
+        col = to_host(W[j, :D].view(torch.uint8)).view(np.float32).reshape(-1, 1)
+        c_ref[j] = project_f32_columns(col, [g_h])[0, 0]
+    assert np.all(c_ref == np.rint(c_ref)) and np.all(np.abs(c_ref) < 2 ** 24) and np.any(c_ref != 0)
+    np.testing.assert_array_equal(c.cpu().numpy().astype(np.float64), c_ref)
+    np.testing.assert_array_equal(c16.cpu().numpy().astype(np.float64), c_ref)
 
 
 # ------------------------------------------------------------------ the layer-wise construction, full size
