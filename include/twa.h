@@ -366,7 +366,11 @@ int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host /* host *
  * width, i.e. B bits except for B = 3 (4 bits).  The columns use the same column-major
  * chunk-permuted bytes as twa_basis, except that every layer starts on a 64-byte granule of the
  * column; `granules` maps each granule back to {layer, valid rows, first flat row, 0}.  All
- * pointers are device pointers into the one buffer `mem` the caller passed to twa_quantize_affine. */
+ * pointers are device pointers into the one buffer `mem` the caller passed to twa_quantize_affine.
+ * A layered basis holds fewer than 2^31 padded rows.  The layers' coefficients do not interact
+ * (Section 4.5: one projection, one update and one lift per layer), so a model of more rows is
+ * several layered bases over consecutive groups of layers, each stepped with its own rows of g,
+ * wbar and w. */
 typedef struct {
   twa_basis codes;            /* D = padded rows, bits = slot width 8, 4, 2 or 1, scales == NULL */
   float* a;                   /* L scaling factors                                              */
