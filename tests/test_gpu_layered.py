@@ -359,6 +359,63 @@ def test_layered_step_matches_oracle_over_iterations(env, D, n, layers, bits):
 
 
 @pytest.mark.parametrize("bits", [8, 4])
+def test_groups_of_layers_as_separate_bases_step_like_the_whole(env, bits):
+    """Layers do not interact (Section 4.5), so a model may be held as several layered bases over
+    consecutive groups of layers -- the way a model of more than 2^31 rows is held: the same factors and
+    codes as the one basis over all layers, and after three steps the same coefficients and weights
+    (to rounding: the layers sit differently in the kernels' tiles), both within the bound of the oracle
+    on the whole model."""
+    ctx, _ = env
+    D, n, layers = 90001, 12, [0, 100, 101, 30000, 65536, 90001]
+    cut_layer, cut = 3, 30000
+    L = len(layers) - 1
+    W = inputs.trajectory_candidates(D, n, 0.005, 0.001, 61, DEV, ld=inputs.padded_ld(D, 4))
+    parts = []
+    for r0, r1, ls in ((0, cut, layers[:cut_layer + 1]), (cut, D, [o - cut for o in layers[cut_layer:]])):
+        Wp = torch.zeros((n, inputs.padded_ld(r1 - r0, 4)), device=DEV)
+        Wp[:, :r1 - r0] = W[:, r0:r1]
+        wbar_p = torch.empty(r1 - r0, device=DEV)
+        lws = twa.new_layered_workspace(ls, n, DEV)
+        lb_p = twa.twa_quantize_affine(ctx, twa.twa_build_centered(ctx, Wp, r1 - r0, ls, wbar_p, lws), ls, bits, lws)
+        parts.append((r0, r1, ls, lb_p, wbar_p, twa.new_layered_step_workspace(lb_p), Wp))
+    wbar = torch.empty(D, device=DEV)
+    lws = twa.new_layered_workspace(layers, n, DEV)
+    lb = twa.twa_quantize_affine(ctx, twa.twa_build_centered(ctx, W, D, layers, wbar, lws), layers, bits, lws)
+    codes_g, a_g, b_g = twa.twa_layered_export(ctx, lb)
+    status_ok(ctx)
+    l0 = 0
+    for r0, r1, ls, lb_p, wbar_p, _, _ in parts:
+        cp, ap, bp = twa.twa_layered_export(ctx, lb_p)
+        Lp = len(ls) - 1
+        assert torch.equal(ap, a_g[l0:l0 + Lp]) and torch.equal(bp, b_g[l0:l0 + Lp])
+        np.testing.assert_array_equal(unpack_unsigned(cp.cpu().numpy(), r1 - r0, bits),
+                                      unpack_unsigned(codes_g.cpu().numpy(), D, bits)[r0:r1])
+        assert torch.equal(wbar_p, wbar[r0:r1])
+        l0 += Lp
+    codes = unpack_unsigned(codes_g.cpu().numpy(), D, bits)
+    a, b = a_g.cpu().numpy(), b_g.cpu().numpy()
+    sws = twa.new_layered_step_workspace(lb)
+    beta, w = torch.zeros((L, n), device=DEV), torch.empty(D, device=DEV)
+    beta_p, w_p = torch.zeros((L, n), device=DEV), torch.empty(D, device=DEV)
+    beta_o, wbar_o = np.zeros((L, n)), wbar.cpu().numpy()
+    lr, lam = 0.5, 1e-2
+    for it in range(3):
+        g = inputs.gradient(D, 1e-2, 10, it, torch.bfloat16, DEV)
+        twa.twa_layered_step(ctx, lb, g, lr, lam, beta, wbar, w, sws)
+        l0 = 0
+        for r0, r1, ls, lb_p, wbar_p, sws_p, _ in parts:
+            Lp = len(ls) - 1
+            twa.twa_layered_step(ctx, lb_p, g[r0:r1], lr, lam, beta_p[l0:l0 + Lp], wbar_p, w_p[r0:r1], sws_p)
+            l0 += Lp
+        status_ok(ctx)
+        beta_o, w_o, _ = orc.step_layerwise(codes, layers, a, b, g.float().cpu().numpy(), beta_o, wbar_o, lr, lam)
+        assert rel(beta_p.cpu().numpy(), beta.cpu().numpy()) <= 1e-6
+        assert rel(beta_p.cpu().numpy(), beta_o) <= TOL and rel(beta.cpu().numpy(), beta_o) <= TOL
+        assert rel(w_p.cpu().numpy(), w_o) <= 2e-5
+        assert torch.max(torch.abs(w_p - w)).item() <= 4 * np.spacing(np.float32(np.abs(w_o).max()))
+
+
+@pytest.mark.parametrize("bits", [8, 4])
 def test_layered_step_replayed_from_a_cuda_graph(bits):
     """twa_layered_step (three launches) captured once and replayed on new gradient bytes: the same
     coefficients and weights as direct calls, bit for bit."""
