@@ -22,12 +22,13 @@
  *    data + j * col_stride (bytes).  Vectors are contiguous.
  *  - Alignment: data pointers of matrices, g, base, w and workspaces must be
  *    16-byte aligned; col_stride must be a multiple of 16 bytes.
- *  - Limits: 1 <= n <= TWA_MAX_N, 1 <= D < 2^31.  The per-column stepping calls (twa_project,
+ *  - Limits: 1 <= n <= TWA_MAX_N, 1 <= D <= TWA_MAX_LAUNCH_ROWS = 2^31 - 2^20 (the kernels count rows in
+ *    32-bit integers and round them up to whole tiles).  The per-column stepping calls (twa_project,
  *    twa_lift, twa_step, twa_step_adam, twa_step_host, twa_weighted_average), the row-chunked
  *    build (twa_build_begin / feed / end_pass) and twa_basis_export / twa_basis_import take
- *    D <= TWA_MAX_ROWS = 2^34: from 2^31 rows on they walk the basis in slabs of 2^30 rows, one
+ *    D <= TWA_MAX_ROWS = 2^34: above TWA_MAX_LAUNCH_ROWS they walk the basis in slabs of 2^30 rows, one
  *    launch per slab and kernel, the projection being the float64 sum of the slabs' projections
- *    in slab order (the stepping calls stay capturable).  A view of fewer than 2^31 rows of such
+ *    in slab order (the stepping calls stay capturable).  A view of at most TWA_MAX_LAUNCH_ROWS rows of such
  *    a basis (twa_basis with data moved to a row on a 512-byte segment) serves every other call.
  *  - Calls enqueue work on the context's stream and return without waiting
  *    for it.  Return value 0 = enqueued; a negative TWA_ERR_* = rejected on
@@ -62,6 +63,7 @@ extern "C" {
 
 #define TWA_MAX_N 128
 #define TWA_MAX_ROWS (1LL << 34) /* the stepping calls, the row-chunked build, export and import */
+#define TWA_MAX_LAUNCH_ROWS ((1LL << 31) - (1LL << 20)) /* every other call; one launch of the stepping calls */
 
 enum {
   TWA_OK = 0,
@@ -367,7 +369,7 @@ int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host /* host *
  * chunk-permuted bytes as twa_basis, except that every layer starts on a 64-byte granule of the
  * column; `granules` maps each granule back to {layer, valid rows, first flat row, 0}.  All
  * pointers are device pointers into the one buffer `mem` the caller passed to twa_quantize_affine.
- * A layered basis holds fewer than 2^31 padded rows.  The layers' coefficients do not interact
+ * A layered basis holds at most TWA_MAX_LAUNCH_ROWS padded rows.  The layers' coefficients do not interact
  * (Section 4.5: one projection, one update and one lift per layer), so a model of more rows is
  * several layered bases over consecutive groups of layers, each stepped with its own rows of g,
  * wbar and w. */

@@ -58,8 +58,10 @@ __global__ void chunk_combine_kernel(const float* __restrict__ chunk_c, int chun
 constexpr long long TWA_SLAB_ROWS = 1LL << 30;
 static_assert(TWA_MAX_ROWS == TWA_SLAB_ROWS * TWA_HOST_CHUNKS, "one slot of per-slab coefficients in ws per slab");
 
+// One launch up to TWA_MAX_LAUNCH_ROWS: the kernels round row numbers up to whole tiles (at most 4096 rows)
+// in 32-bit integers, and the margin below 2^31 keeps those sums from wrapping.
 int slab_count(long long D) {
-  return D < (1LL << 31) ? 1 : static_cast<int>((D + TWA_SLAB_ROWS - 1) / TWA_SLAB_ROWS);
+  return D <= TWA_MAX_LAUNCH_ROWS ? 1 : static_cast<int>((D + TWA_SLAB_ROWS - 1) / TWA_SLAB_ROWS);
 }
 
 // Rows [k * TWA_SLAB_ROWS, ...) of P as a basis of its own; 2^30 rows are whole 512-byte segments
@@ -75,7 +77,7 @@ twa_basis slab_view(const twa_basis* P, int k, long long* r0) {
 // twa_check_basis with the row limit of the slab-walking calls instead of the kernels' own.
 int check_basis_slabbed(const twa_basis* P) {
   if (!P) return TWA_ERR_INVALID_ARG;
-  if (P->D < (1LL << 31)) return twa_check_basis(P);
+  if (P->D <= TWA_MAX_LAUNCH_ROWS) return twa_check_basis(P);
   if (P->D > TWA_MAX_ROWS) return TWA_ERR_INVALID_ARG;
   twa_basis head = *P;
   head.D = TWA_SLAB_ROWS;

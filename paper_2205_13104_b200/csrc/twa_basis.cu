@@ -495,7 +495,7 @@ namespace {
 int build_basis(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, float* wbar_out, twa_basis* P32_out, void* ws,
                 size_t ws_bytes, unsigned* absmax) {
   if (!ctx || !W || !wbar_out || !P32_out) return TWA_ERR_INVALID_ARG;
-  if (D < 1 || D >= (1LL << 31) || n < 1 || ldw < D) return TWA_ERR_INVALID_ARG;
+  if (D < 1 || D > TWA_MAX_LAUNCH_ROWS || n < 1 || ldw < D) return TWA_ERR_INVALID_ARG;
   if (n > TWA_MAX_N) return TWA_ERR_UNSUPPORTED;
   if (!ws || ws_bytes < TWA_WS_BYTES) return TWA_ERR_WORKSPACE;
   if ((reinterpret_cast<uintptr_t>(W) & 15) || (ldw & 3) || (reinterpret_cast<uintptr_t>(ws) & 15) ||
@@ -704,7 +704,7 @@ int twa_basis_export(twa_ctx* ctx, const twa_basis* Pq, void* codes_out, float* 
   if (!ctx || !codes_out || !scales_out || !Pq) return TWA_ERR_INVALID_ARG;
   // the conversion kernels index bytes with 64-bit integers: up to TWA_MAX_ROWS rows
   twa_basis head = *Pq;
-  if (Pq->D >= (1LL << 31)) head.D = (1LL << 31) - 1;
+  if (Pq->D > TWA_MAX_LAUNCH_ROWS) head.D = TWA_MAX_LAUNCH_ROWS;
   int rc = twa_check_basis(&head);
   if (rc) return rc;
   if (Pq->D > TWA_MAX_ROWS || Pq->col_stride < (Pq->D * Pq->bits + 7) / 8) return TWA_ERR_INVALID_ARG;

@@ -68,7 +68,7 @@ int make_partition(const int64_t* offsets, int L, long long D, int bits, Partiti
   p->internal[L] = io;
   p->first_item[L] = static_cast<int>(p->items.size());
   p->D_int = io;
-  return io < (1LL << 31) ? TWA_OK : TWA_ERR_UNSUPPORTED;
+  return io <= TWA_MAX_LAUNCH_ROWS ? TWA_OK : TWA_ERR_UNSUPPORTED;
 }
 
 // ---- kernels ------------------------------------------------------------------------------
@@ -767,7 +767,7 @@ size_t twa_layered_basis_bytes(const int64_t* offsets_host, int L, int n, int bi
 int twa_build_centered(twa_ctx* ctx, float* W, int64_t D, int n, int64_t ldw, const int64_t* offsets_host,
                        int L, float* wbar_out, twa_basis* P32_out, void* lws, size_t lws_bytes) {
   if (!ctx || !W || !wbar_out || !P32_out || !offsets_host) return TWA_ERR_INVALID_ARG;
-  if (D < 1 || D >= (1LL << 31) || n < 1 || ldw < D) return TWA_ERR_INVALID_ARG;
+  if (D < 1 || D > TWA_MAX_LAUNCH_ROWS || n < 1 || ldw < D) return TWA_ERR_INVALID_ARG;
   if (n > TWA_MAX_N) return TWA_ERR_UNSUPPORTED;
   Partition p;
   int rc = make_partition(offsets_host, L, D, 8, &p);
@@ -934,7 +934,7 @@ int twa_layered_build_begin(twa_ctx* ctx, int64_t D, int n, const int64_t* offse
                             size_t mem_bytes, twa_layered_basis* out, void* lws, size_t lws_bytes) {
   if (!ctx || !out || !offsets_host || !mem) return TWA_ERR_INVALID_ARG;
   if (slot_bits(bits) == 0) return TWA_ERR_UNSUPPORTED;
-  if (D < 1 || D >= (1LL << 31) || n < 1) return TWA_ERR_INVALID_ARG;
+  if (D < 1 || D > TWA_MAX_LAUNCH_ROWS || n < 1) return TWA_ERR_INVALID_ARG;
   if (n * plane_count(bits) > TWA_MAX_N || L > 65535) return TWA_ERR_UNSUPPORTED;
   Partition p;
   int rc = make_partition(offsets_host, L, D, slot_bits(bits), &p);

@@ -598,7 +598,7 @@ int twa_ensure_smem(twa_ctx* ctx, const void* kernel, int* current, int wanted) 
 int twa_check_basis(const twa_basis* P) {
   if (!P || !P->data) return TWA_ERR_INVALID_ARG;
   if (P->bits != 32 && P->bits != 8 && P->bits != 4) return TWA_ERR_UNSUPPORTED;
-  if (P->n < 1 || P->D < 1 || P->D >= (1LL << 31)) return TWA_ERR_INVALID_ARG;
+  if (P->n < 1 || P->D < 1 || P->D > TWA_MAX_LAUNCH_ROWS) return TWA_ERR_INVALID_ARG;
   if (P->n > TWA_MAX_N) return TWA_ERR_UNSUPPORTED;
   if (P->bits != 32 && !P->scales) return TWA_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(P->data) & 15) || (P->col_stride & 15)) return TWA_ERR_MISALIGNED;

@@ -583,13 +583,15 @@ def test_basis_of_more_than_2_31_rows(env):
         twa.twa_project_noalloc(0, None, bases[8], torch.zeros(D, dtype=torch.bfloat16, device=DEV), c)
 
 
-def test_float32_candidates_of_more_than_2_31_rows(env):
-    """Two float32 candidates of 2^31 + 70,001 rows: the fixed-weight average (the float32 lift over the
+@pytest.mark.parametrize("D", [(1 << 31) - 5, (1 << 31) + 70_001])
+def test_float32_candidates_of_more_than_2_31_rows(env, D):
+    """Two float32 candidates of 2^31 - 5 rows (above the row count one launch takes, so two slabs whose
+    second is five rows short of 2^30) and of 2^31 + 70,001 rows: the fixed-weight average (the float32 lift over the
     slabs) on rows at the start, across 2^30 and 2^31 and at the end against the oracle, and the float32
     projection on all rows against the oracle's, streamed through the host, on integer-valued inputs
     that make the result exact."""
     ctx, ws = env
-    D, n = (1 << 31) + 70_001, 2
+    n = 2
     wl = inputs.Workload("rows_2g_f32", D, n, 0.002, 0.0005, 1e-3, "f32", (32,), 1, seed=12)
     W = torch.zeros((n, D + 3), device=DEV)                 # columns start on 16 bytes
     CH = inputs.CHUNK_ROWS
@@ -601,7 +603,7 @@ def test_float32_candidates_of_more_than_2_31_rows(env):
     twa.twa_weighted_average(ctx, W, D, weights, w, ws)
     status_ok(ctx)
     span = 1 << 16
-    for r0 in (0, (1 << 30) - span // 2, (1 << 31) - span // 2, D - span):
+    for r0 in sorted({0, (1 << 30) - span // 2, min((1 << 31) - span // 2, D - span), D - span}):
         rows_h = W[:, r0:r0 + span].cpu().numpy().T
         ref = orc.weighted_average(rows_h, [0.25, 0.75])
         got = w[r0:r0 + span].cpu().numpy()
