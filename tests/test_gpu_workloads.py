@@ -593,7 +593,7 @@ def test_float32_candidates_of_more_than_2_31_rows(env, D):
     ctx, ws = env
     n = 2
     wl = inputs.Workload("rows_2g_f32", D, n, 0.002, 0.0005, 1e-3, "f32", (32,), 1, seed=12)
-    W = torch.zeros((n, D + 3), device=DEV)                 # columns start on 16 bytes
+    W = torch.zeros((n, (D + 3) // 4 * 4), device=DEV)      # columns start on 16 bytes
     CH = inputs.CHUNK_ROWS
     for r0 in range(0, D, CH):
         rows = min(CH, D - r0)
