@@ -832,6 +832,25 @@ def other_configs(env, ctx, twa, inputs, ws, args, peak):
                                          args.configs_min_ms / 2, peak))
         del bases, wbar, pool
         torch.cuda.empty_cache()
+    # a basis of more than 2^31 rows: the 1.3 B-sized workload's recipe stretched to 2^31 + 3 * 2^22 + 70,001 rows
+    # (row-chunked build, int8); the step walks it in three slabs of 2^30 rows
+    if not args.no_large_rows:
+        import dataclasses
+        wl = dataclasses.replace(inputs.WORKLOADS["decoder1p3b"], name="decoder-recipe rows > 2^31",
+                                 D=(1 << 31) + 3 * (1 << 22) + 70_001)
+        bases, wbar, build_ms = build_chunked(ctx, wl, dev, [8], twa, inputs)
+        pool = gradient_pool(wl, wl.D, dev, 2)
+        sampler = ClockSampler(env.local).start() if env.rank == 0 else None
+        m = measure_steps(env, ctx, twa, wl, bases[8], wbar, ws, pool, args.steps, args.warmup,
+                          args.configs_min_ms, sampler)
+        clocks = None
+        if sampler is not None:
+            sampler.stop()
+            clocks = sampler.summary(m["walls"][0][0], m["walls"][-1][1])
+        out.append(config_entry(wl, 8, m, peak, build_ms, None, clocks,
+                                note="three slabs of 2^30 rows per kernel; the projection's slab sums are added in float64"))
+        del bases, wbar, pool
+        torch.cuda.empty_cache()
     # the other modes of the library, each through its own benchmark routine, condensed
     for name, bits in (("vitb16", 8), ("vitb16", 4), ("decoder1p3b", 4)):
         line = layered_line(env, args, name, bits, args.configs_min_ms)
@@ -1100,6 +1119,8 @@ def main():
     ap.add_argument("--dequant-path", type=int, default=0, choices=[0, 1],
                     help="0: integer dot products on the tensor pipe (default); 1: float32 FMA path")
     ap.add_argument("--rows", type=int, default=0, help="override D (smaller cases for profiler captures)")
+    ap.add_argument("--no-large-rows", action="store_true",
+                    help="leave the basis of more than 2^31 rows (about 95 GB on the device) out of the configs array")
     ap.add_argument("--random-basis", action="store_true",
                     help="profiling aid: quantise a random matrix instead of building the basis")
     ap.add_argument("--layered", action="store_true",
