@@ -140,10 +140,16 @@ const char* twa_last_error(const twa_ctx* ctx);
  *      1 = every lane loads and stores its own rows; 2 = `base` comes through the shared-memory
  *      ring beside the codes; 3 = as 2, and the results leave through bulk stores from shared
  *      memory; 0 = built-in choice by the share of the two vectors in the bytes moved
- *      (n * bits <= 192: 2, <= 320: 3, else 1). */
+ *      (n * bits <= 192: 2, <= 320: 3, else 1).
+ *  TWA_TUNE_SLAB_ROWS: rows per launch of the per-column stepping calls (twa_project, twa_lift,
+ *      twa_step, twa_step_adam, twa_weighted_average): a multiple of 65536, at most 2^30.  A basis
+ *      of more rows is walked in slabs of that many rows (at most 16 of them, else the call
+ *      returns TWA_ERR_INVALID_ARG), exactly as bases above TWA_MAX_LAUNCH_ROWS always are: shorter
+ *      kernels where the GPU is shared and a long launch holds others up.  0 = one launch up to
+ *      TWA_MAX_LAUNCH_ROWS, slabs of 2^30 rows above. */
 enum { TWA_TUNE_PROJECT_WARPS = 1, TWA_TUNE_LIFT_WARPS = 2, TWA_TUNE_STAGES = 3,
        TWA_TUNE_WAIT_LIMIT_MS = 4, TWA_TUNE_DEQUANT_PATH = 5, TWA_TUNE_TILE_SEGMENTS = 6,
-       TWA_TUNE_BUILD_PANEL = 7, TWA_TUNE_LIFT_VECTORS = 8 };
+       TWA_TUNE_BUILD_PANEL = 7, TWA_TUNE_LIFT_VECTORS = 8, TWA_TUNE_SLAB_ROWS = 9 };
 int twa_set_tuning(twa_ctx* ctx, int key, int value);
 
 /* Exercises the bounded wait every streaming kernel uses, without any fault: enqueues one block

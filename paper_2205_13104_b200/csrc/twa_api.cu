@@ -53,32 +53,41 @@ __global__ void chunk_combine_kernel(const float* __restrict__ chunk_c, int chun
   if (j < n && alpha && !unusable) alpha[j] = twa_coefficient_update(alpha[j], c, lr, lambda, adam, j);
 }
 
-// A basis of 2^31 rows or more is walked in slabs of 2^30 rows: the kernels index rows with 32-bit
-// integers, the projection is a sum over row ranges and the lift is independent per row.
+// A basis of more than TWA_MAX_LAUNCH_ROWS rows (or of more than TWA_TUNE_SLAB_ROWS, where that is set) is
+// walked in slabs: the kernels index rows with 32-bit integers, the projection is a sum over row
+// ranges and the lift is independent per row.  One launch takes up to TWA_MAX_LAUNCH_ROWS: the kernels
+// round row numbers up to whole tiles (at most 4096 rows) in 32-bit integers, and the margin below
+// 2^31 keeps those sums from wrapping.
 constexpr long long TWA_SLAB_ROWS = 1LL << 30;
 static_assert(TWA_MAX_ROWS == TWA_SLAB_ROWS * TWA_HOST_CHUNKS, "one slot of per-slab coefficients in ws per slab");
 
-// One launch up to TWA_MAX_LAUNCH_ROWS: the kernels round row numbers up to whole tiles (at most 4096 rows)
-// in 32-bit integers, and the margin below 2^31 keeps those sums from wrapping.
-int slab_count(long long D) {
-  return D <= TWA_MAX_LAUNCH_ROWS ? 1 : static_cast<int>((D + TWA_SLAB_ROWS - 1) / TWA_SLAB_ROWS);
+struct SlabPlan {
+  long long rows;    // rows per slab: whole 512-byte segments at every storage width
+  int count;         // 1: the whole basis in one launch
+};
+
+SlabPlan slab_plan(const twa_ctx* ctx, long long D) {
+  const long long one = ctx->tune_slab_rows ? ctx->tune_slab_rows : TWA_MAX_LAUNCH_ROWS;
+  if (D <= one) return {D, 1};
+  const long long rows = ctx->tune_slab_rows ? ctx->tune_slab_rows : TWA_SLAB_ROWS;
+  return {rows, static_cast<int>((D + rows - 1) / rows)};
 }
 
-// Rows [k * TWA_SLAB_ROWS, ...) of P as a basis of its own; 2^30 rows are whole 512-byte segments
-// at every storage width.
-twa_basis slab_view(const twa_basis* P, int k, long long* r0) {
-  *r0 = static_cast<long long>(k) * TWA_SLAB_ROWS;
+// Rows [k * plan.rows, ...) of P as a basis of its own.
+twa_basis slab_view(const twa_basis* P, const SlabPlan& plan, int k, long long* r0) {
+  *r0 = static_cast<long long>(k) * plan.rows;
   twa_basis v = *P;
   v.data = static_cast<char*>(P->data) + (*r0 * P->bits) / 8;
-  v.D = (*r0 + TWA_SLAB_ROWS < P->D) ? TWA_SLAB_ROWS : P->D - *r0;
+  v.D = (*r0 + plan.rows < P->D) ? plan.rows : P->D - *r0;
   return v;
 }
 
 // twa_check_basis with the row limit of the slab-walking calls instead of the kernels' own.
-int check_basis_slabbed(const twa_basis* P) {
+int check_basis_slabbed(const twa_ctx* ctx, const twa_basis* P) {
   if (!P) return TWA_ERR_INVALID_ARG;
-  if (P->D <= TWA_MAX_LAUNCH_ROWS) return twa_check_basis(P);
   if (P->D > TWA_MAX_ROWS) return TWA_ERR_INVALID_ARG;
+  if (slab_plan(ctx, P->D).count > TWA_HOST_CHUNKS) return TWA_ERR_INVALID_ARG;
+  if (P->D <= TWA_MAX_LAUNCH_ROWS) return twa_check_basis(P);
   twa_basis head = *P;
   head.D = TWA_SLAB_ROWS;
   int rc = twa_check_basis(&head);
@@ -89,12 +98,13 @@ int check_basis_slabbed(const twa_basis* P) {
 // Projection of every slab into its slot of ws, then the combine (and the optimiser step, if any).
 int project_slabs(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dtype, const twa_project_epilogue& epi,
                   void* ws) {
-  const int slabs = slab_count(P->D);
+  const SlabPlan plan = slab_plan(ctx, P->D);
+  const int slabs = plan.count;
   const size_t gsz = g_dtype == TWA_BF16 ? 2 : 4;
   float* slab_c = reinterpret_cast<float*>(static_cast<char*>(ws) + TWA_WS_CHUNK_COEF);
   for (int k = 0; k < slabs; ++k) {
     long long r0;
-    const twa_basis v = slab_view(P, k, &r0);
+    const twa_basis v = slab_view(P, plan, k, &r0);
     twa_project_epilogue part = {slab_c + static_cast<size_t>(k) * TWA_MAX_N, nullptr, 0.0f, 0.0f, -1};
     int rc = twa_launch_project(ctx, &v, static_cast<const char*>(g) + r0 * gsz, g_dtype, part, ws);
     if (rc) return rc;
@@ -107,11 +117,12 @@ int project_slabs(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_d
 
 // Lift of every slab, last slab first when the projection has just run (its rows are the likeliest in L2).
 int lift_slabs(twa_ctx* ctx, const twa_basis* P, const float* alpha, const float* base, float* out, bool reverse) {
-  const int slabs = slab_count(P->D);
+  const SlabPlan plan = slab_plan(ctx, P->D);
+  const int slabs = plan.count;
   for (int i = 0; i < slabs; ++i) {
     const int k = reverse ? slabs - 1 - i : i;
     long long r0;
-    const twa_basis v = slab_view(P, k, &r0);
+    const twa_basis v = slab_view(P, plan, k, &r0);
     int rc = twa_launch_lift(ctx, &v, alpha, 1.0f, base ? base + r0 : nullptr, out + r0, reverse);
     if (rc) return rc;
   }
@@ -267,6 +278,10 @@ int twa_set_tuning(twa_ctx* ctx, int key, int value) {
       if (value > 1) return TWA_ERR_INVALID_ARG;
       ctx->tune_dequant_path = value;
       return TWA_OK;
+    case TWA_TUNE_SLAB_ROWS:
+      if ((value & 65535) || static_cast<long long>(value) > TWA_SLAB_ROWS) return TWA_ERR_INVALID_ARG;
+      ctx->tune_slab_rows = value;
+      return TWA_OK;
     case TWA_TUNE_WAIT_LIMIT_MS:
       ctx->wait_limit_ns = (value ? static_cast<unsigned long long>(value) : 2000ull) * 1000000ull;
       return TWA_OK;
@@ -278,27 +293,27 @@ int twa_project(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype g_dty
                 void* ws, size_t ws_bytes) {
   if (!ctx || !g || !c_out) return TWA_ERR_INVALID_ARG;
   if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
-  int rc = check_basis_slabbed(P);
+  int rc = check_basis_slabbed(ctx, P);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes);
   if (rc) return rc;
   if (misaligned16(g)) return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
   twa_project_epilogue epi = {c_out, nullptr, 0.0f, 0.0f, -1};
-  if (slab_count(P->D) > 1) return project_slabs(ctx, P, g, g_dtype, epi, ws);
+  if (slab_plan(ctx, P->D).count > 1) return project_slabs(ctx, P, g, g_dtype, epi, ws);
   return twa_launch_project(ctx, P, g, g_dtype, epi, ws);
 }
 
 int twa_lift(twa_ctx* ctx, const twa_basis* P, const float* alpha, const float* base, float* w_out,
              void* ws, size_t ws_bytes) {
   if (!ctx || !alpha || !w_out) return TWA_ERR_INVALID_ARG;
-  int rc = check_basis_slabbed(P);
+  int rc = check_basis_slabbed(ctx, P);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes);
   if (rc) return rc;
   if (misaligned16(w_out) || (base && misaligned16(base))) return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-  if (slab_count(P->D) > 1) return lift_slabs(ctx, P, alpha, base, w_out, false);
+  if (slab_plan(ctx, P->D).count > 1) return lift_slabs(ctx, P, alpha, base, w_out, false);
   return twa_launch_lift(ctx, P, alpha, 1.0f, base, w_out, false);
 }
 
@@ -307,14 +322,14 @@ static int step_impl(twa_ctx* ctx, const twa_basis* P, const void* g, twa_dtype 
                      size_t ws_bytes) {
   if (!ctx || !g || !alpha || !wbar || !w) return TWA_ERR_INVALID_ARG;
   if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
-  int rc = check_basis_slabbed(P);
+  int rc = check_basis_slabbed(ctx, P);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes);
   if (rc) return rc;
   if (misaligned16(g) || misaligned16(w) || misaligned16(wbar)) return TWA_ERR_MISALIGNED;
   TWA_CUDA_OK(ctx, cudaSetDevice(ctx->device));
   twa_project_epilogue epi = {c_out, alpha, lr, lambda, -1, adam};
-  const bool slabbed = slab_count(P->D) > 1;
+  const bool slabbed = slab_plan(ctx, P->D).count > 1;
   cudaEvent_t* ev = nullptr;
   if (ctx->prof_events && ctx->prof_count < ctx->prof_cap) ev = ctx->prof_events + 3 * ctx->prof_count;
   if (ev) TWA_CUDA_OK(ctx, cudaEventRecord(ev[0], ctx->stream));
@@ -421,7 +436,7 @@ int twa_step_host(twa_ctx* ctx, const twa_basis* P, const void* g_host, twa_dtyp
     return TWA_OK;
   }
   if (!alpha || !wbar || !w) return TWA_ERR_INVALID_ARG;
-  int rc = check_basis_slabbed(P);
+  int rc = check_basis_slabbed(ctx, P);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes);
   if (rc) return rc;

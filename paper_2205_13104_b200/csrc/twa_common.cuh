@@ -31,6 +31,7 @@ struct twa_ctx {
   int tune_tile_segments;     // tensor-pipe path: 512-byte segments per tile column (0 = choose)
   int tune_build_panel;       // resident basis build: 0 = panels of 8 columns, Gram form inside; 1 = column by column; 2 = panels, column sweeps inside
   int tune_lift_base_path;    // tensor-pipe lift, base / output vectors: 0 = choose, 1 = lanes, 2 = base through the ring, 3 = both
+  int tune_slab_rows;         // stepping calls: rows per launch (0 = one launch up to TWA_MAX_LAUNCH_ROWS, slabs of 2^30 above)
   cudaEvent_t* prof_events;   // 3 per recorded step, or null
   int prof_cap, prof_count;   // steps
   // state of a row-chunked basis build (twa_build_begin .. twa_build_end_pass)

@@ -39,6 +39,7 @@ TWA_TUNE_DEQUANT_PATH = 5
 TWA_TUNE_TILE_SEGMENTS = 6
 TWA_TUNE_BUILD_PANEL = 7
 TWA_TUNE_LIFT_VECTORS = 8
+TWA_TUNE_SLAB_ROWS = 9
 
 EXPORTS = [
     "twa_create", "twa_destroy", "twa_get_status", "twa_clear_status", "twa_strerror",

@@ -165,3 +165,83 @@ def test_random_shapes_layer_wise(env, seed):
         w_o = orc.lift_layerwise(co, layers, ao, bo, beta.cpu().numpy(), wbar.cpu().numpy())
         assert rel(w.cpu().numpy(), w_o) <= TOL, tag
         status_ok(ctx, tag)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_shapes_walked_in_slabs(seed):
+    """TWA_TUNE_SLAB_ROWS makes the stepping calls walk a basis in slabs of 65536 k rows -- the walk every
+    basis above 2^31 - 2^20 rows gets -- so that random shapes meet it: D on, just past and far from a slab
+    boundary, 2 to 16 slabs, 8-bit, 4-bit and float32 bases.  The lift must equal the one-launch lift bit
+    for bit (rows do not interact); projection, SGD step and Adam step must meet the oracle within the
+    bounds of the one-launch calls and the one-launch result to rounding."""
+    torch.cuda.set_device(0)
+    ctx, ref = twa.twa_create(0), twa.twa_create(0)
+    ws, ws_ref = twa.new_workspace(DEV), twa.new_workspace(DEV)
+    rng = np.random.default_rng(4000 + seed)
+    for case in range(6):
+        n = int(rng.choice(N_CHOICES))
+        slab = 65536 * int(rng.integers(1, 4))
+        slabs = int(rng.integers(2, 17))
+        tail = int(rng.choice([0, 1, 2, 511, 512, 1023, 4097, slab - 1, int(rng.integers(1, slab))]))
+        D = slab * (slabs - 1) + (tail if tail else slab)
+        bits = int(rng.choice([8, 4, 32]))
+        tag = f"seed={seed} case={case} D={D} n={n} bits={bits} slab={slab}"
+        gen = torch.Generator(device=DEV).manual_seed(seed * 100 + case)
+        P = torch.zeros((n, inputs.padded_ld(D, 4)), device=DEV)
+        P[:, :D] = torch.randn((n, D), generator=gen, device=DEV) / np.sqrt(D)
+        B = twa.basis_from_tensor(P, D)
+        if bits != 32:
+            B = twa.twa_quantize_basis(ref, B, bits, ws_ref)
+            codes, s = twa.twa_basis_export(ref, B)
+            co, so = orc.unpack_codes(codes.cpu().numpy(), D, bits), s.cpu().numpy()
+        else:
+            P_h = P[:, :D].cpu().numpy().T
+        twa.twa_set_tuning(ctx, twa.TWA_TUNE_SLAB_ROWS, slab)
+        gdt = torch.bfloat16 if rng.random() < 0.5 else torch.float32
+        g = (torch.randn(D, generator=gen, device=DEV) * 1e-3).to(gdt)
+        g_h = g.float().cpu().numpy()
+        wbar = torch.randn(D, generator=gen, device=DEV)
+        # projection
+        c, c1 = torch.empty(n, device=DEV), torch.empty(n, device=DEV)
+        twa.twa_project(ctx, B, g, c, ws)
+        twa.twa_project(ref, B, g, c1, ws_ref)
+        c_o = orc.project(co, so, g_h) if bits != 32 else orc.project_f32(P_h, g_h)
+        g_norm = np.linalg.norm(g_h.astype(np.float64))
+        p_norm = (np.linalg.norm(co.astype(np.float64), axis=0) * np.abs(so) if bits != 32
+                  else np.linalg.norm(P_h.astype(np.float64), axis=0))
+        assert np.all(np.abs(c.cpu().numpy() - c_o) <= TOL * p_norm * g_norm + 1e-30), tag
+        assert np.all(np.abs(c.cpu().numpy() - c1.cpu().numpy()) <= 2e-6 * p_norm * g_norm + 1e-30), tag
+        # lift: bit for bit the one-launch lift, with and without the base point
+        alpha = torch.randn(n, generator=gen, device=DEV)
+        w, w1 = torch.empty(D, device=DEV), torch.empty(D, device=DEV)
+        for base in (wbar, None):
+            twa.twa_lift(ctx, B, alpha, base, w, ws)
+            twa.twa_lift(ref, B, alpha, base, w1, ws_ref)
+            assert torch.equal(w, w1), tag
+        # SGD step and Adam step from zero state
+        a, a1 = torch.zeros(n, device=DEV), torch.zeros(n, device=DEV)
+        twa.twa_step(ctx, B, g, 0.1, 0.01, a, wbar, w, ws, c_out=c)
+        a_o = orc.sgd_update(np.zeros(n), c_o, 0.1, 0.01)
+        assert np.all(np.abs(a.cpu().numpy() - a_o) <= 0.1 * TOL * p_norm * g_norm + 1e-30), tag
+        twa.twa_lift(ref, B, a, wbar, w1, ws_ref)
+        assert torch.equal(w, w1), tag
+        m, v = torch.zeros(n, device=DEV), torch.zeros(n, device=DEV)
+        twa.twa_step_adam(ctx, B, g, 1e-2, 1, a1, m, v, wbar, w, ws, weight_decay=0.01)
+        _, m_o, v_o = orc.adam_update(np.zeros(n), np.zeros(n), np.zeros(n), c_o, 1e-2, 1, weight_decay=0.01)
+        assert np.all(np.abs(m.cpu().numpy() - m_o) <= 0.1 * TOL * p_norm * g_norm + 1e-30), tag
+        assert rel(v.cpu().numpy(), v_o) <= 1e-3, tag
+        twa.twa_lift(ref, B, a1, wbar, w1, ws_ref)
+        assert torch.equal(w, w1), tag
+        status_ok(ctx, tag)
+        status_ok(ref, tag)
+    # more than sixteen slabs do not fit the workspace's slots: refused on the host
+    twa.twa_set_tuning(ctx, twa.TWA_TUNE_SLAB_ROWS, 65536)
+    Pbig = torch.zeros((1, 65536 * 16 + 4), device=DEV)
+    with pytest.raises(twa.TwaError):
+        twa.twa_project(ctx, twa.basis_from_tensor(Pbig, 65536 * 16 + 1), torch.zeros(65536 * 16 + 4, device=DEV),
+                        torch.empty(1, device=DEV), ws)
+    with pytest.raises(twa.TwaError):
+        twa.twa_set_tuning(ctx, twa.TWA_TUNE_SLAB_ROWS, 65536 + 512)
+    torch.cuda.synchronize()
+    twa.twa_destroy(ctx)
+    twa.twa_destroy(ref)
