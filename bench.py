@@ -834,10 +834,20 @@ def other_configs(env, ctx, twa, inputs, ws, args, peak):
         torch.cuda.empty_cache()
     # a basis of more than 2^31 rows: the 1.3 B-sized workload's recipe stretched to 2^31 + 3 * 2^22 + 70,001 rows
     # (row-chunked build, int8); the step walks it in three slabs of 2^30 rows
-    if not args.no_large_rows:
+    large_rows = not args.no_large_rows
+    if large_rows:
         import dataclasses
         wl = dataclasses.replace(inputs.WORKLOADS["decoder1p3b"], name="decoder-recipe rows > 2^31",
                                  D=(1 << 31) + 3 * (1 << 22) + 70_001)
+        torch.cuda.empty_cache()
+        free_bytes, _ = torch.cuda.mem_get_info(dev)
+        free_bytes = -max_over_ranks([-float(free_bytes)], dev)[0]       # every rank takes the same decision
+        need = wl.n * wl.D + 2 * 2 * wl.D + 3 * 4 * wl.D + (2 << 30)      # codes, two gradients, w-bar, w, slack
+        if free_bytes < need:
+            out.append({"workload": workload_label(wl, wl.D, 8), "bits": 8,
+                        "skipped": "%.0f GB free on the device, %.0f GB needed" % (free_bytes / 1e9, need / 1e9)})
+            large_rows = False
+    if large_rows:
         bases, wbar, build_ms = build_chunked(ctx, wl, dev, [8], twa, inputs)
         pool = gradient_pool(wl, wl.D, dev, 2)
         sampler = ClockSampler(env.local).start() if env.rank == 0 else None
