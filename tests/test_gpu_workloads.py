@@ -68,6 +68,17 @@ def to_host(t):
     return buf[:flat.numel()].numpy().view(np.uint8).reshape(t.shape)
 
 
+def need_memory(device_gb, host_gb):
+    """Skips a test on a box that cannot hold it: free device memory and available host memory in GB."""
+    import psutil
+    free, _ = torch.cuda.mem_get_info(0)
+    if free < device_gb * 1e9:
+        pytest.skip(f"{free / 1e9:.0f} GB free on the device, {device_gb} GB needed")
+    avail = psutil.virtual_memory().available
+    if avail < host_gb * 1e9:
+        pytest.skip(f"{avail / 1e9:.0f} GB of host memory available, {host_gb} GB needed")
+
+
 def oracle_project_all(ctx, basis, gs, block=8, first_only_blocks=None):
     """The oracle's projection of ALL n columns at full size, for every gradient of the list gs in
     one pass: the canonical codes leave the device eight columns at a time and go through
@@ -491,6 +502,7 @@ def test_basis_of_more_than_2_31_rows(env):
     coefficients after step 1 and step 2, rows of w at the start, across 2^30, across 2^31, in the
     last slab and at the ragged end."""
     ctx, ws = env
+    need_memory(100, 80)
     D, n = (1 << 31) + 3 * (1 << 22) + 70_001, 4
     wl = inputs.Workload("rows_2g", D, n, 0.002, 0.0005, 1e-4, "bf16", (8, 4), 2, seed=11, chunked_build=True)
     CH = inputs.CHUNK_ROWS
@@ -591,6 +603,7 @@ def test_float32_candidates_of_more_than_2_31_rows(env, D):
     projection on all rows against the oracle's, streamed through the host, on integer-valued inputs
     that make the result exact."""
     ctx, ws = env
+    need_memory(60, 40)
     n = 2
     wl = inputs.Workload("rows_2g_f32", D, n, 0.002, 0.0005, 1e-3, "f32", (32,), 1, seed=12)
     W = torch.zeros((n, (D + 3) // 4 * 4), device=DEV)      # columns start on 16 bytes
