@@ -24,11 +24,11 @@
  *    16-byte aligned; col_stride must be a multiple of 16 bytes.
  *  - Limits: 1 <= n <= TWA_MAX_N, 1 <= D <= TWA_MAX_LAUNCH_ROWS = 2^31 - 2^20 (the kernels count rows in
  *    32-bit integers and round them up to whole tiles).  The per-column stepping calls (twa_project,
- *    twa_lift, twa_step, twa_step_adam, twa_step_host, twa_weighted_average), the row-chunked
+ *    twa_lift, twa_step, twa_step_adam, twa_step_host, twa_weighted_average, twa_project_batch), the row-chunked
  *    build (twa_build_begin / feed / end_pass) and twa_basis_export / twa_basis_import take
  *    D <= TWA_MAX_ROWS = 2^34: above TWA_MAX_LAUNCH_ROWS they walk the basis in slabs of 2^30 rows, one
  *    launch per slab and kernel, the projection being the float64 sum of the slabs' projections
- *    in slab order (the stepping calls stay capturable).  A view of at most TWA_MAX_LAUNCH_ROWS rows of such
+ *    in slab order (twa_project_batch: every slab after the first adds to C_out; the stepping calls stay capturable).  A view of at most TWA_MAX_LAUNCH_ROWS rows of such
  *    a basis (twa_basis with data moved to a row on a 512-byte segment) serves every other call.
  *  - Calls enqueue work on the context's stream and return without waiting
  *    for it.  Return value 0 = enqueued; a negative TWA_ERR_* = rejected on
@@ -142,7 +142,7 @@ const char* twa_last_error(const twa_ctx* ctx);
  *      memory; 0 = built-in choice by the share of the two vectors in the bytes moved
  *      (n * bits <= 192: 2, <= 320: 3, else 1).
  *  TWA_TUNE_SLAB_ROWS: rows per launch of the per-column stepping calls (twa_project, twa_lift,
- *      twa_step, twa_step_adam, twa_weighted_average): a multiple of 65536, at most 2^30.  A basis
+ *      twa_step, twa_step_adam, twa_weighted_average, twa_project_batch): a multiple of 65536, at most 2^30.  A basis
  *      of more rows is walked in slabs of that many rows (at most 16 of them, else the call
  *      returns TWA_ERR_INVALID_ARG), exactly as bases above TWA_MAX_LAUNCH_ROWS always are: shorter
  *      kernels where the GPU is shared and a long launch holds others up.  0 = one launch up to

@@ -12,6 +12,7 @@
 #include <stdio.h>
 
 #include "twa_mma.cuh"
+#include "twa_slabs.cuh"
 
 namespace {
 
@@ -61,6 +62,7 @@ struct BatchArgs {
   unsigned* ticket;
   int* status;
   float* c_out;                 // [batch][n]
+  int accumulate;               // 1: the results are added to c_out (a later row slab of the basis)
   unsigned long long wait_limit_ns;
 };
 
@@ -304,9 +306,10 @@ twa_project_batch_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       double sum = 0.0;
       for (unsigned k = 0; k < gridDim.x; ++k)
         sum += static_cast<double>(__ldcg(&a.partials[static_cast<size_t>(k) * outs + idx]));
-      const double c = sum * static_cast<double>(a.scales[j]);
+      float* out = a.c_out + static_cast<size_t>(a.b0 + b) * a.n + j;
+      const double c = sum * static_cast<double>(a.scales[j]) + (a.accumulate ? static_cast<double>(*out) : 0.0);
       if (!isfinite(c)) twa_set_status(a.status, TWA_ERR_NONFINITE, a.b0 + b);
-      a.c_out[static_cast<size_t>(a.b0 + b) * a.n + j] = static_cast<float>(c);
+      *out = static_cast<float>(c);
     }
     if (tid == 0) *a.ticket = 0u;
   }
@@ -423,11 +426,16 @@ extern "C" int twa_project_batch_group(twa_ctx* ctx, const twa_basis* P, twa_dty
   return nb;
 }
 
+namespace {
+int project_batch_rows(twa_ctx* ctx, const twa_basis* P, const void* G, long long ldg, int batch, twa_dtype g_dtype,
+                       float* C_out, void* ws, int accumulate);
+}
+
 extern "C" int twa_project_batch(twa_ctx* ctx, const twa_basis* P, const void* G, int64_t ldg, int batch,
                                  twa_dtype g_dtype, float* C_out, void* ws, size_t ws_bytes) {
   if (!ctx || !P || !G || !C_out || batch < 1) return TWA_ERR_INVALID_ARG;
   if (g_dtype != TWA_F32 && g_dtype != TWA_BF16) return TWA_ERR_INVALID_ARG;
-  int rc = twa_check_basis(P);
+  int rc = check_basis_slabbed(ctx, P);
   if (rc) return rc;
   if (ldg < P->D) return TWA_ERR_INVALID_ARG;
   if (!ws || ws_bytes < TWA_WS_BYTES) return TWA_ERR_WORKSPACE;
@@ -444,6 +452,23 @@ extern "C" int twa_project_batch(twa_ctx* ctx, const twa_basis* P, const void* G
     }
     return TWA_OK;
   }
+  // a basis of more rows than one launch takes: slab after slab, every slab after the first adding to C_out
+  const SlabPlan plan = slab_plan(ctx, P->D);
+  for (int k = 0; k < plan.count; ++k) {
+    long long r0;
+    const twa_basis v = slab_view(P, plan, k, &r0);
+    rc = project_batch_rows(ctx, &v, static_cast<const char*>(G) + r0 * gsz, ldg, batch, g_dtype, C_out, ws, k > 0);
+    if (rc) return rc;
+  }
+  return TWA_OK;
+}
+
+namespace {
+int project_batch_rows(twa_ctx* ctx, const twa_basis* P, const void* G, long long ldg, int batch, twa_dtype g_dtype,
+                       float* C_out, void* ws, int accumulate) {
+  const bool bf16 = g_dtype == TWA_BF16;
+  const int gsz = bf16 ? 2 : 4;
+  int rc;
   int kt, nb;
   pass_shape(ctx, P, gsz, &kt, &nb);
   const int rows = twa_tile_rows(P->bits) * kt;
@@ -482,6 +507,7 @@ extern "C" int twa_project_batch(twa_ctx* ctx, const twa_basis* P, const void* G
   a.ticket = ctx->d_ticket;
   a.status = ctx->d_status;
   a.c_out = C_out;
+  a.accumulate = accumulate;
   a.wait_limit_ns = ctx->wait_limit_ns;
   int grid = ctx->sm_count < a.tiles ? ctx->sm_count : a.tiles;
   while (static_cast<size_t>(grid) * nb * P->n > static_cast<size_t>(TWA_MAX_GRID) * TWA_MAX_N) --grid;
@@ -496,3 +522,4 @@ extern "C" int twa_project_batch(twa_ctx* ctx, const twa_basis* P, const void* G
   }
   return TWA_OK;
 }
+}  // namespace

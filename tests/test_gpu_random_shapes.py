@@ -173,7 +173,7 @@ def test_random_shapes_walked_in_slabs(seed):
     basis above 2^31 - 2^20 rows gets -- so that random shapes meet it: D on, just past and far from a slab
     boundary, 2 to 16 slabs, 8-bit, 4-bit and float32 bases.  The lift must equal the one-launch lift bit
     for bit (rows do not interact); projection, SGD step and Adam step must meet the oracle within the
-    bounds of the one-launch calls and the one-launch result to rounding."""
+    bounds of the one-launch calls and the one-launch result to rounding; so must the batched projection."""
     torch.cuda.set_device(0)
     ctx, ref = twa.twa_create(0), twa.twa_create(0)
     ws, ws_ref = twa.new_workspace(DEV), twa.new_workspace(DEV)
@@ -211,6 +211,17 @@ def test_random_shapes_walked_in_slabs(seed):
                   else np.linalg.norm(P_h.astype(np.float64), axis=0))
         assert np.all(np.abs(c.cpu().numpy() - c_o) <= TOL * p_norm * g_norm + 1e-30), tag
         assert np.all(np.abs(c.cpu().numpy() - c1.cpu().numpy()) <= 2e-6 * p_norm * g_norm + 1e-30), tag
+        # several gradients per projection: every slab after the first adds to the results
+        batch = int(rng.integers(1, 11))
+        G = torch.zeros((batch, inputs.padded_ld(D, 8)), dtype=gdt, device=DEV)
+        G[:, :D] = (torch.randn((batch, D), generator=gen, device=DEV) * 1e-3).to(gdt)
+        C = torch.full((batch, n), 7.0, device=DEV)
+        twa.twa_project_batch(ctx, B, G, C, ws)
+        for b_ in range(batch):
+            gb = G[b_, :D].float().cpu().numpy()
+            cb = orc.project(co, so, gb) if bits != 32 else orc.project_f32(P_h, gb)
+            bound = TOL * p_norm * np.linalg.norm(gb.astype(np.float64)) + 1e-30
+            assert np.all(np.abs(C[b_].cpu().numpy() - cb) <= bound), (tag, b_)
         # lift: bit for bit the one-launch lift, with and without the base point
         alpha = torch.randn(n, generator=gen, device=DEV)
         w, w1 = torch.empty(D, device=DEV), torch.empty(D, device=DEV)
