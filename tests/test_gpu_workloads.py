@@ -420,8 +420,41 @@ def test_workload_resident_build_sampled(env, name, bits_list):
     torch.cuda.empty_cache()
     # the workload's 100 steps; the oracle steps two sampled columns
     run_sequence(ctx, ws, wl, bases, wbar, wl.steps, [17, n - 1])
+    if name == "vitb16":
+        check_batched_projection(ctx, ws, wl, bases)
     del bases
     torch.cuda.empty_cache()
+
+
+def check_batched_projection(ctx, ws, wl, bases):
+    """Eight gradients per projection at full size, in the shape the benchmark times: all n coefficients of
+    the group's first and last gradient against the oracle (streamed through the host), and every
+    gradient's coefficients against the single projection of the same bytes."""
+    D, n = wl.D, wl.n
+    batch = 8
+    gdt = torch.bfloat16 if wl.g_dtype == "bf16" else torch.float32
+    G = torch.zeros((batch, inputs.padded_ld(D, 8)), dtype=gdt, device=DEV)
+    for b in range(batch):
+        wl.gradient(1000 + b, DEV, out=G[b, :D])
+    g_first = G[0, :D].float().cpu().numpy()
+    g_last = G[batch - 1, :D].float().cpu().numpy()
+    norms = [float(np.sqrt(np.dot(x.astype(np.float64), x.astype(np.float64)))) for x in (g_first, g_last)]
+    for basis in bases:
+        assert twa.twa_project_batch_group(ctx, basis, gdt) == batch
+        C = torch.empty((batch, n), device=DEV)
+        twa.twa_project_batch(ctx, basis, G, C, ws)
+        status_ok(ctx)
+        C_h = C.cpu().numpy()
+        C_or, norm_low = oracle_project_all(ctx, basis, [g_first, g_last])
+        assert_coefficients(C_h[0], C_or[:, 0], norm_low, norms[0])
+        assert_coefficients(C_h[batch - 1], C_or[:, 1], norm_low, norms[1])
+        c = torch.empty(n, device=DEV)
+        for b in range(batch):
+            twa.twa_project(ctx, basis, G[b, :D], c, ws)
+            single = c.cpu().numpy().astype(np.float64)
+            assert rel(C_h[b], single) <= 2e-6
+            assert np.all(np.abs(C_h[b] - single) <= 2e-6 * np.max(np.abs(single)))
+        status_ok(ctx)
 
 
 # ------------------------------------------------------------------ 1.3 B-sized: chunked build, sampled
