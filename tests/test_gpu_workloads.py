@@ -70,7 +70,10 @@ def to_host(t):
 
 def need_memory(device_gb, host_gb):
     """Skips a test on a box that cannot hold it: free device memory and available host memory in GB."""
+    import gc
     import psutil
+    gc.collect()
+    torch.cuda.empty_cache()                 # what earlier tests freed is still held by the caching allocator
     free, _ = torch.cuda.mem_get_info(0)
     if free < device_gb * 1e9:
         pytest.skip(f"{free / 1e9:.0f} GB free on the device, {device_gb} GB needed")
