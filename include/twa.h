@@ -22,14 +22,17 @@
  *    data + j * col_stride (bytes).  Vectors are contiguous.
  *  - Alignment: data pointers of matrices, g, base, w and workspaces must be
  *    16-byte aligned; col_stride must be a multiple of 16 bytes.
- *  - Limits: 1 <= n <= TWA_MAX_N, 1 <= D <= TWA_MAX_LAUNCH_ROWS = 2^31 - 2^20 (the kernels count rows in
- *    32-bit integers and round them up to whole tiles).  The per-column stepping calls (twa_project,
- *    twa_lift, twa_step, twa_step_adam, twa_step_host, twa_weighted_average, twa_project_batch), the row-chunked
- *    build (twa_build_begin / feed / end_pass) and twa_basis_export / twa_basis_import take
- *    D <= TWA_MAX_ROWS = 2^34: above TWA_MAX_LAUNCH_ROWS they walk the basis in slabs of 2^30 rows, one
- *    launch per slab and kernel, the projection being the float64 sum of the slabs' projections
- *    in slab order (twa_project_batch: every slab after the first adds to C_out; the stepping calls stay capturable).  A view of at most TWA_MAX_LAUNCH_ROWS rows of such
- *    a basis (twa_basis with data moved to a row on a 512-byte segment) serves every other call.
+ *  - Limits: 1 <= n <= TWA_MAX_N, 1 <= D <= TWA_MAX_LAUNCH_ROWS = 2^31 - 2^20 (the kernels
+ *    count rows in 32-bit integers and round them up to whole tiles).  The per-column
+ *    stepping calls (twa_project, twa_project_batch, twa_lift, twa_step, twa_step_adam,
+ *    twa_step_host, twa_weighted_average), the row-chunked build (twa_build_begin / feed /
+ *    end_pass) and twa_basis_export / twa_basis_import take D <= TWA_MAX_ROWS = 2^34.  Above
+ *    TWA_MAX_LAUNCH_ROWS the stepping calls walk the basis in slabs of 2^30 rows, one launch
+ *    per slab and kernel: the projection is the float64 sum of the slabs' projections in slab
+ *    order (twa_project_batch: every slab after the first adds to C_out), the lift is
+ *    independent per row; the calls stay capturable.  Every other call takes a view of at most
+ *    TWA_MAX_LAUNCH_ROWS rows of such a basis (a twa_basis whose data points at a row on a
+ *    512-byte segment of the columns).
  *  - Calls enqueue work on the context's stream and return without waiting
  *    for it.  Return value 0 = enqueued; a negative TWA_ERR_* = rejected on
  *    the host, nothing enqueued.  Errors found on the device (non-finite
