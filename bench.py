@@ -875,11 +875,11 @@ def other_configs(env, ctx, twa, inputs, ws, args, peak):
                         "sm_mhz": line["clocks"]["sm_mhz"] if line["clocks"] else None,
                         "clock_reasons": line["clocks"]["reasons"] if line["clocks"] else None,
                         "basis_build_ms": line["basis_build_ms"], "quantize_ms": line["quantize_ms"]})
-    if env.world == 1:
-        line = project_batch_line(env, args, "vitb16", 8, 8, args.configs_min_ms)
+    for bits in ((8, 4) if env.world == 1 else ()):
+        line = project_batch_line(env, args, "vitb16", bits, 8, args.configs_min_ms)
         r = line["roofline"]
         out.append({"mode": "8 gradients per projection (twa_project_batch)", "workload": line["config"]["workload"],
-                    "bits": 8, "ms_per_call": line["ms_per_step"], "gradients_per_s": line["value"],
+                    "bits": bits, "ms_per_call": line["ms_per_step"], "gradients_per_s": line["value"],
                     "GBps": r["achieved"], "frac_of_measured_copy_peak": r["frac"], "frac_of_8TBps": r["achieved"] / 8000.0,
                     "single_calls_ms": line["single_calls_ms"], "speedup_over_single_calls": line["speedup_over_single_calls"],
                     "sm_mhz": line["clocks"]["sm_mhz"], "clock_reasons": line["clocks"]["reasons"]})
